@@ -1,0 +1,234 @@
+"""Seeded synthetic inputs for the decode hot path (weights, KV prefill, tokens).
+
+This module holds no arithmetic of the decode method itself: it only draws
+numbers.  It serves both the CUDA path and the CPU oracle, which otherwise
+share nothing.
+
+Generator.  Every tensor element is a pure function of (seed, tensor name,
+layer, flat element index), so any tensor -- or any single layer of it -- can be
+regenerated on demand on either device, and the values are bit-identical on CPU
+and CUDA because only 64-bit integer operations and one table lookup are used:
+
+    key   = mix(seed, name, layer)                     (Python integers)
+    u64   = fmix64((index + 1) * GOLDEN + key)         (wrapping int64 torch ops)
+    code  = top 16 bits of u64
+    value = mean + std * QUANTILE[code]                (fp32), rounded to bf16
+
+QUANTILE is the 65536-point table of standard-normal quantiles at the bin
+centres (k + 0.5) / 65536, i.e. a normal distribution discretised far below
+bf16 resolution and truncated at about +-4.3 sigma.
+
+Workload recipe (shapes follow the Llama-3.1 decode configurations of the
+paper's operation-intensity table):
+  matrices and embedding  ~ N(0, 0.02^2)  bf16
+  RMSNorm gains           ~ 1 + N(0, 0.02^2) bf16
+  KV-cache prefill        ~ N(0, 1) bf16 at positions [0, T), zero elsewhere
+  tokens                  uniform in [0, vocab)
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, asdict
+
+import torch
+
+_M64 = (1 << 64) - 1
+_GOLDEN = 0x9E3779B97F4A7C15
+_C1 = 0xFF51AFD7ED558CCD
+_C2 = 0xC4CEB9FE1A85EC53
+_CHUNK = 1 << 25  # elements generated per pass (bounds temporary memory)
+
+
+@dataclass(frozen=True)
+class ModelShape:
+    """Decoder-only transformer shape (names as in the decode step definition)."""
+    n_layers: int
+    hidden: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    ffn: int
+    vocab: int
+    rms_eps: float = 1e-5
+    rope_theta: float = 10000.0
+
+    @property
+    def q_dim(self) -> int:
+        return self.n_q_heads * self.head_dim
+
+    @property
+    def kv_dim(self) -> int:
+        return self.n_kv_heads * self.head_dim
+
+    def as_dict(self) -> dict:
+        return asdict(self)
+
+
+TINY = ModelShape(4, 256, 4, 2, 64, 512, 1024, 1e-5, 10000.0)
+LLAMA31_8B = ModelShape(32, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0)
+LLAMA31_70B = ModelShape(80, 8192, 64, 8, 128, 28672, 128256, 1e-5, 500000.0)
+
+# name -> (rows, cols) of each tensor as handed to the library (row-major [out, in]).
+MATRIX_NAMES = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
+LAYER_TENSORS = MATRIX_NAMES + ("norm1", "norm2")
+GLOBAL_TENSORS = ("embed", "norm_f", "lm_head")
+
+
+def tensor_shape(shape: ModelShape, name: str) -> tuple[int, ...]:
+    s = shape
+    return {
+        "wq": (s.q_dim, s.hidden),
+        "wk": (s.kv_dim, s.hidden),
+        "wv": (s.kv_dim, s.hidden),
+        "wo": (s.hidden, s.q_dim),
+        "wgate": (s.ffn, s.hidden),
+        "wup": (s.ffn, s.hidden),
+        "wdown": (s.hidden, s.ffn),
+        "norm1": (s.hidden,),
+        "norm2": (s.hidden,),
+        "norm_f": (s.hidden,),
+        "embed": (s.vocab, s.hidden),
+        "lm_head": (s.vocab, s.hidden),
+    }[name]
+
+
+def _s64(v: int) -> int:
+    """Reinterpret an unsigned 64-bit Python integer as signed (for torch int64)."""
+    v &= _M64
+    return v - (1 << 64) if v >= (1 << 63) else v
+
+
+def _fmix64_py(x: int) -> int:
+    x &= _M64
+    x ^= x >> 33
+    x = (x * _C1) & _M64
+    x ^= x >> 33
+    x = (x * _C2) & _M64
+    x ^= x >> 33
+    return x
+
+
+def tensor_key(seed: int, name: str, *ids: int) -> int:
+    """64-bit key of one tensor: a hash of the seed, its name and integer ids."""
+    k = _fmix64_py(seed + 0x243F6A8885A308D3)
+    for ch in name.encode():
+        k = _fmix64_py(k ^ (ch + 0x100))
+    for i in ids:
+        k = _fmix64_py(k ^ ((i + 1) * _GOLDEN))
+    return k
+
+
+def _fmix64(x: torch.Tensor) -> torch.Tensor:
+    """murmur3 finaliser on int64 tensors; shifts made logical by masking."""
+    x = x ^ ((x >> 33) & 0x7FFFFFFF)
+    x = x * _s64(_C1)
+    x = x ^ ((x >> 33) & 0x7FFFFFFF)
+    x = x * _s64(_C2)
+    x = x ^ ((x >> 33) & 0x7FFFFFFF)
+    return x
+
+
+def hash_u64(key: int, start: int, count: int, device) -> torch.Tensor:
+    """Hash of element indices [start, start+count) under `key` (int64 bit patterns)."""
+    idx = torch.arange(start + 1, start + 1 + count, dtype=torch.int64, device=device)
+    return _fmix64(idx * _s64(_GOLDEN) + _s64(key))
+
+
+_QUANTILE_CACHE: dict[str, torch.Tensor] = {}
+
+
+def normal_quantile_table(device="cpu") -> torch.Tensor:
+    """65536 standard-normal quantiles at bin centres, fp32 (computed once, in fp64, on CPU)."""
+    dev = str(torch.device(device))
+    if "cpu" not in _QUANTILE_CACHE:
+        k = torch.arange(65536, dtype=torch.float64)
+        u = (k + 0.5) / 65536.0
+        z = math.sqrt(2.0) * torch.special.erfinv(2.0 * u - 1.0)
+        _QUANTILE_CACHE["cpu"] = z.to(torch.float32)
+    if dev not in _QUANTILE_CACHE:
+        _QUANTILE_CACHE[dev] = _QUANTILE_CACHE["cpu"].to(device)
+    return _QUANTILE_CACHE[dev]
+
+
+def normal_bf16(key: int, numel: int, std: float, mean: float = 0.0, device="cpu",
+                out: torch.Tensor | None = None) -> torch.Tensor:
+    """`numel` draws of mean + std * N(0,1), rounded to bf16 (flat tensor)."""
+    table = normal_quantile_table(device)
+    if out is None:
+        out = torch.empty(numel, dtype=torch.bfloat16, device=device)
+    flat = out.view(-1)
+    assert flat.numel() == numel
+    for s in range(0, numel, _CHUNK):
+        n = min(_CHUNK, numel - s)
+        code = (hash_u64(key, s, n, device) >> 48) & 0xFFFF
+        v = table[code]
+        v = v * std
+        if mean != 0.0:
+            v = v + mean
+        flat[s:s + n] = v.to(torch.bfloat16)
+    return out
+
+
+def make_tensor(shape: ModelShape, name: str, layer: int = -1, seed: int = 0, device="cpu") -> torch.Tensor:
+    """One weight tensor (bf16, row-major [out, in]) of the synthetic model."""
+    dims = tensor_shape(shape, name)
+    numel = math.prod(dims)
+    key = tensor_key(seed, name, layer)
+    if name.startswith("norm"):
+        t = normal_bf16(key, numel, 0.02, 1.0, device)
+    else:
+        t = normal_bf16(key, numel, 0.02, 0.0, device)
+    return t.view(*dims)
+
+
+def make_layer(shape: ModelShape, layer: int, seed: int = 0, device="cpu") -> dict[str, torch.Tensor]:
+    return {n: make_tensor(shape, n, layer, seed, device) for n in LAYER_TENSORS}
+
+
+def make_globals(shape: ModelShape, seed: int = 0, device="cpu", with_embed_table: bool = True) -> dict[str, torch.Tensor]:
+    names = GLOBAL_TENSORS if with_embed_table else ("norm_f", "lm_head")
+    return {n: make_tensor(shape, n, -1, seed, device) for n in names}
+
+
+def embed_rows(shape: ModelShape, tokens, seed: int = 0, device="cpu") -> torch.Tensor:
+    """Rows `tokens` of the embedding table without materialising the table."""
+    key = tensor_key(seed, "embed", -1)
+    rows = []
+    for t in tokens:
+        buf = torch.empty(shape.hidden, dtype=torch.bfloat16, device=device)
+        table = normal_quantile_table(device)
+        code = (hash_u64(key, int(t) * shape.hidden, shape.hidden, device) >> 48) & 0xFFFF
+        buf[:] = (table[code] * 0.02).to(torch.bfloat16)
+        rows.append(buf)
+    return torch.stack(rows)
+
+
+def kv_cache_shape(shape: ModelShape, batch: int, max_ctx: int) -> tuple[int, ...]:
+    """Cache layout [L][2 (K,V)][B][n_kv_heads][max_ctx][head_dim], bf16."""
+    return (shape.n_layers, 2, batch, shape.n_kv_heads, max_ctx, shape.head_dim)
+
+
+def fill_kv_layer(shape: ModelShape, cache_layer: torch.Tensor, layer: int, context: int, seed: int = 0) -> None:
+    """Prefill one layer's slice [2][B][nkv][max_ctx][hd] with N(0,1) at positions [0, context)."""
+    two, batch, nkv, max_ctx, hd = cache_layer.shape
+    assert two == 2 and context <= max_ctx
+    dev = cache_layer.device
+    for kv in range(2):
+        for b in range(batch):
+            key = tensor_key(seed, "kv", layer, kv, b)
+            blk = normal_bf16(key, nkv * context * hd, 1.0, 0.0, dev).view(nkv, context, hd)
+            cache_layer[kv, b, :, :context, :] = blk
+
+
+def make_kv_cache(shape: ModelShape, batch: int, context: int, max_ctx: int, seed: int = 0, device="cpu") -> torch.Tensor:
+    cache = torch.zeros(kv_cache_shape(shape, batch, max_ctx), dtype=torch.bfloat16, device=device)
+    for l in range(shape.n_layers):
+        fill_kv_layer(shape, cache[l], l, context, seed)
+    return cache
+
+
+def make_tokens(shape: ModelShape, batch: int, seed: int = 0, stream: int = 0, device="cpu") -> torch.Tensor:
+    """`batch` token ids uniform in [0, vocab) (int32)."""
+    key = tensor_key(seed, "tokens", stream)
+    h = (hash_u64(key, 0, batch, device) >> 16) & 0x7FFFFFFF
+    return (h % shape.vocab).to(torch.int32)
