@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Decode-throughput benchmark of the kernel-looped decoder (one JSON line on stdout).
+
+A step is one pass of the whole hot path -- Embedding, L decoder layers, Classifier, greedy Sampling -- for one
+batch of sequences.  Default workload: Llama-3.1-8B shape, batch 1, context 4096 (the configuration the paper's
+operation-intensity table and headline figure are quoted on), synthetic seeded weights and KV cache.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 (under torchrun) runs N independent replicas: a decode stream is a strict chain, so the path does not shard
+and no data-path collective exists; torch.distributed is used for the barrier and the max-over-ranks only.
+`--impl reference` times the CPU oracle on the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import torch
+
+from paper_2410_23668_b200 import inputs as gen
+
+WORKLOADS = {
+    # name: (shape, batch, context, default steps)
+    "tiny_b1_ctx128": (gen.TINY, 1, 128, 16),
+    "llama31_8b_b1_ctx4096": (gen.LLAMA31_8B, 1, 4096, 128),
+    "llama31_8b_b1_ctx65536": (gen.LLAMA31_8B, 1, 65536, 64),
+    "llama31_70b_b1_ctx4096": (gen.LLAMA31_70B, 1, 4096, 32),
+}
+DEFAULT_WORKLOAD = "llama31_8b_b1_ctx4096"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def layer_weight_bytes(s) -> int:
+    return 2 * (s.hidden * s.head_dim * (2 * s.n_q_heads + 2 * s.n_kv_heads) + 3 * s.hidden * s.ffn + 2 * s.hidden)
+
+
+def kv_bytes(s, batch: int, position: int) -> int:
+    """KV rows 0..position-1 read plus row `position` written, every layer."""
+    return batch * s.n_layers * 2 * s.n_kv_heads * s.head_dim * 2 * (position + 1)
+
+
+def decoder_bytes(s, batch: int, position: int) -> int:
+    """Algorithmic HBM bytes of the decoder kernel(s) of one step: all layers' matrices and gains once + KV."""
+    return s.n_layers * layer_weight_bytes(s) + kv_bytes(s, batch, position)
+
+
+def step_bytes(s, batch: int, position: int) -> int:
+    """Algorithmic HBM bytes of one whole step: decoder + final gain + lm_head + B embedding rows."""
+    return decoder_bytes(s, batch, position) + 2 * s.hidden + 2 * s.vocab * s.hidden + batch * 2 * s.hidden
+
+
+def measured_peaks() -> dict:
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        d = json.loads(f.read_text())
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML (read-only) while the timed regions run."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if visible:
+                ids = [v for v in visible.split(",") if v.strip() != ""]
+                if index < len(ids) and ids[index].strip().isdigit():
+                    phys = int(ids[index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def start(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self) -> dict:
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def build_model(shape, batch, context, steps_total, seed=0):
+    from paper_2410_23668_b200 import binding
+    max_ctx = context + steps_total + 8
+    dec = binding.Decoder(shape, batch, max_ctx)
+    for l in range(shape.n_layers):
+        for name, t in gen.make_layer(shape, l, seed, "cuda").items():
+            dec.kl_load_weights(name, l, t)
+        torch.cuda.synchronize()
+    for name, t in gen.make_globals(shape, seed, "cuda").items():
+        dec.kl_load_weights(name, -1, t)
+    torch.cuda.synchronize()
+    cache = gen.make_kv_cache(shape, batch, context, max_ctx, seed, "cuda")
+    return dec, cache, max_ctx
+
+
+def run_device_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
+    """W + K greedy steps with tokens and positions resident on the device; returns ms for the K timed steps."""
+    tok = tok0.clone()
+    pos = torch.full((batch,), context, dtype=torch.int32, device="cuda")
+    logits = torch.empty(batch, dec.shape.vocab, dtype=torch.float32, device="cuda")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(warmup):
+        dec.kl_decode_step(tok, pos, cache, logits, batch, stream)
+        dec.kl_argmax_advance(logits, tok, pos, batch, stream)
+    torch.cuda.synchronize()
+    barrier()
+    e0.record(stream)
+    for _ in range(steps):
+        dec.kl_decode_step(tok, pos, cache, logits, batch, stream)
+        dec.kl_argmax_advance(logits, tok, pos, batch, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    st = dec.kl_last_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} after the timed loop")
+    return e0.elapsed_time(e1)
+
+
+def run_host_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
+    """End to end through the host-buffer entry point: every step copies tokens and positions host->device,
+    runs the step, copies the logits device->host, and the host picks the next token."""
+    V = dec.shape.vocab
+    tok_h = tok0.cpu().pin_memory()
+    pos_h = torch.full((batch,), context, dtype=torch.int32).pin_memory()
+    logits_h = torch.empty(batch, V, dtype=torch.float32).pin_memory()
+
+    def one():
+        dec.kl_decode_step_host(tok_h, pos_h, cache, logits_h, batch, stream)
+        tok_h.copy_(logits_h.argmax(dim=1).to(torch.int32))
+        pos_h.add_(1)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)
+
+
+_DIST = {"on": False}
+
+
+def barrier():
+    if _DIST["on"]:
+        torch.distributed.barrier()
+
+
+def max_over_ranks(v: float) -> float:
+    if not _DIST["on"]:
+        return v
+    t = torch.tensor([v], dtype=torch.float64, device="cuda")
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def oracle_sample(shape, batch, context, n_layers_sample, seed=0, device="cpu"):
+    """Times the oracle, as it stands, on `n_layers_sample` decoder layers + the classifier of one decode step
+    and scales the layer part to the full depth.  Returns (seconds per token, description, threads)."""
+    from oracle import kl_oracle as ko
+    import numpy as np
+    max_ctx = context + 8
+    layers = {}
+    for l in range(n_layers_sample):
+        layers[l] = {k: v.cpu() for k, v in gen.make_layer(shape, l, seed, device).items()}
+    glob = {k: v.cpu() for k, v in gen.make_globals(shape, seed, device, with_embed_table=False).items()}
+    glob["embed_row"] = lambda tok: gen.embed_rows(shape, [tok], seed)[0]
+    orc = ko.Oracle(shape, max_ctx, lambda l: layers[l], glob)
+    cache = np.zeros(gen.kv_cache_shape(shape, batch, max_ctx), dtype=np.uint16)
+    for l in range(n_layers_sample):
+        blk = torch.zeros(gen.kv_cache_shape(shape, batch, max_ctx)[1:], dtype=torch.bfloat16, device=device)
+        gen.fill_kv_layer(shape, blk, l, context, seed)
+        cache[l] = blk.cpu().view(torch.uint16).numpy()
+    toks = gen.make_tokens(shape, batch, seed).tolist()
+    t0 = time.perf_counter()
+    hidden, _, _ = orc.step(cache, toks, [context] * batch, layers=range(n_layers_sample), want_logits=False)
+    t_layers = time.perf_counter() - t0
+    import ctypes as C
+    logits = np.empty(shape.vocab, dtype=np.float64)
+    t0 = time.perf_counter()
+    for b in range(batch):
+        ko.lib().ko_classifier(C.byref(orc.desc), C.c_void_p(ko.as_u16(glob["norm_f"]).ctypes.data),
+                               C.c_void_p(ko.as_u16(glob["lm_head"]).ctypes.data),
+                               hidden[b].ctypes.data_as(C.POINTER(C.c_double)),
+                               logits.ctypes.data_as(C.POINTER(C.c_double)), None, 0)
+    t_cls = time.perf_counter() - t0
+    per_token = t_layers * shape.n_layers / n_layers_sample + t_cls
+    desc = (f"one decode step at position {context}: {n_layers_sample} of {shape.n_layers} decoder layers + classifier "
+            f"executed ({t_layers:.2f} s + {t_cls:.2f} s), layer time scaled to {shape.n_layers} layers")
+    return per_token / batch, desc, ko.num_threads()
+
+
+def run_reference(args, shape, batch, context):
+    """Reference arm = the CPU oracle on the host cores (bounded sample per step)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import kl_oracle as ko
+    ko.build()
+    total = args.steps + args.warmup
+    budget = 150.0 / max(total, 1)
+    # calibrate on one layer, then pick how many layers one step can afford
+    t1, _, threads = oracle_sample(shape, batch, context, 1)
+    t_layer = t1 / shape.n_layers  # rough: classifier included, fine for sizing
+    n_layers_sample = max(1, min(shape.n_layers, int(budget / max(t_layer, 1e-6))))
+    n_layers_sample = min(n_layers_sample, 4)
+    times = []
+    desc = ""
+    for i in range(total):
+        sec, desc, threads = oracle_sample(shape, batch, context, n_layers_sample)
+        if i >= args.warmup:
+            times.append(sec)
+    sec = statistics.mean(times)
+    value = 1.0 / sec
+    line = {
+        "impl": "reference", "metric": "decode tokens/s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * batch, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": batch, "context": context},
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, shape, batch, context):
+    from paper_2410_23668_b200 import binding, build
+    if build.needs_build():
+        build.build_library()
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
+        _DIST["on"] = True
+    K, W = args.steps, max(args.warmup, 3)
+    passes = 4  # looped, per-layer, profiled, end-to-end
+    dec, cache, max_ctx = build_model(shape, batch, context, passes * (K + W), seed=rank)
+    tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
+    stream = torch.cuda.current_stream()
+    cache0 = cache.clone() if cache.numel() * 2 < (8 << 30) else None
+
+    def fresh_cache():
+        if cache0 is not None:
+            cache.copy_(cache0)
+        return cache
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    # 1. headline: looped, device-resident
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    l0 = dec.kl_launch_count()
+    ms_looped = max_over_ranks(run_device_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    launches = (dec.kl_launch_count() - l0) * K // (K + W)
+    # 2. the synchronisation-boundary schedule: one launch per layer
+    dec.kl_set_mode(binding.KL_MODE_PER_LAYER)
+    ms_layer = max_over_ranks(run_device_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    # 3. roofline of the dominant kernel: events around the decoder launch inside the timed steps
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    dec.kl_profile_enable(K)
+    run_device_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream)
+    dec_ms, cls_ms = dec.kl_profile_read(K)
+    dec.kl_profile_enable(0)
+    clocks = sampler.stop()
+    # 4. end to end through the host-buffer entry point
+    ms_e2e = max_over_ranks(run_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+
+    tokens = K * batch * world
+    value = tokens / (ms_looped * 1e-3)
+    pos_avg = context + W + (K - 1) / 2.0
+    bytes_step = step_bytes(shape, batch, 0) + kv_bytes(shape, batch, 0) * pos_avg  # kv_bytes(.,.,0) = one row set
+    bytes_dec = decoder_bytes(shape, batch, 0) + kv_bytes(shape, batch, 0) * pos_avg
+    peaks = measured_peaks()
+    dec_avg_ms = statistics.mean(dec_ms)
+    achieved = bytes_dec / (dec_avg_ms * 1e-3) / 1e9
+    line = {
+        "metric": "decode tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_looped / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": batch, "context": context, "mode": "looped",
+                   "storage": "bf16 weights and KV, fp32 activations and accumulation",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (weights streamed once per step)", "max_ctx": max_ctx},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
+                "d2h_bytes_per_step": 4 * shape.vocab * batch},
+        "roofline": {"bound": "hbm", "kernel": "kl_decoder_kernel (looped, all layers)", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                     "peak_source": peaks["source"], "traffic": None, "bytes_per_launch": bytes_dec,
+                     "ms_per_launch": dec_avg_ms, "classifier_ms": statistics.mean(cls_ms)},
+        "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_looped / K * 1e-3) / 1e9,
+                       "frac_of_measured_copy": bytes_step / (ms_looped / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "frac_of_8tbs": bytes_step / (ms_looped / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+        "per_layer": {"value": tokens / (ms_layer * 1e-3), "ms_per_step": ms_layer / K,
+                      "launches_per_step": shape.n_layers + 3,
+                      "looped_speedup": ms_layer / ms_looped},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import kl_oracle as ko
+        ko.build()
+        n_s = 2 if shape.n_layers > 4 else shape.n_layers
+        sec, desc, threads = oracle_sample(shape, batch, context, n_s, device="cuda")
+        line["cpu_baseline"] = {"value": 1.0 / sec, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc}
+    dec.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    shape, batch, context, dsteps = WORKLOADS[args.workload]
+    if args.steps is None:
+        args.steps = dsteps
+    if args.impl == "reference":
+        run_reference(args, shape, batch, context)
+    else:
+        run_ours(args, shape, batch, context)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,149 @@
+/*
+ * kl -- kernel-looped transformer decode on one NVIDIA B200 (sm_100a).  C ABI.
+ *
+ * The library implements the decode step of a decoder-only transformer the way the paper
+ * "Kernel Looping" (arXiv 2410.23668) schedules it: Embedding, L x Decoder, Classifier, Sampling
+ * (Section 2, call-schedule figure).  In KL_MODE_LOOPED the L consecutive calls to the decoder-layer
+ * kernel are one call to a persistent kernel with an outer loop over layers (Section 3.2, rules
+ * (1)-(10)); in KL_MODE_PER_LAYER the same kernel body is launched once per layer, which is the
+ * synchronisation-boundary schedule the transformation removes (Section 2, schedule (ii)).
+ *
+ * Conventions
+ *   - All pointers named *_d are DEVICE pointers, *_h are HOST pointers.  Nothing here allocates or frees
+ *     device memory: the caller owns the weight arena, the scratch arena, the KV cache, token/position/logit
+ *     buffers and the CUDA stream (passed as a void* holding a cudaStream_t; NULL = default stream).
+ *   - Every function returns a kl_status (0 = KL_OK, negative = error); nothing throws, aborts or traps.
+ *   - Calls on one handle must not overlap on the GPU (use one stream per handle).
+ *   - Storage is bf16 for weights and KV cache; activations and all accumulation are fp32.
+ */
+#ifndef KL_H_
+#define KL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kl_handle kl_handle;
+typedef int32_t kl_status;
+
+enum {
+    KL_OK = 0,
+    KL_ERR_INVALID_ARG = -1,       /* null pointer, bad enum, size mismatch */
+    KL_ERR_UNSUPPORTED_SHAPE = -2, /* model or batch shape outside what the kernels cover */
+    KL_ERR_NOT_LOADED = -3,        /* kl_decode_step before every tensor was loaded */
+    KL_ERR_CUDA = -4,              /* a CUDA runtime call failed */
+    KL_ERR_SYNC_TIMEOUT = -5,      /* a bounded device-side wait ran out (reported by kl_last_status) */
+    KL_ERR_OUT_OF_RANGE = -6       /* token >= vocab or position >= max_ctx seen on the device */
+};
+
+enum { KL_MODE_LOOPED = 0, KL_MODE_PER_LAYER = 1 };
+
+/* Tensors accepted by kl_load_weights; all bf16, row-major [out_features, in_features] (gains: [hidden]). */
+enum {
+    KL_EMBED = 0,   /* [vocab, hidden]           layer = -1 */
+    KL_WQ = 1,      /* [n_q_heads*head_dim, hidden] */
+    KL_WK = 2,      /* [n_kv_heads*head_dim, hidden] */
+    KL_WV = 3,      /* [n_kv_heads*head_dim, hidden] */
+    KL_WO = 4,      /* [hidden, n_q_heads*head_dim] */
+    KL_WGATE = 5,   /* [ffn, hidden] */
+    KL_WUP = 6,     /* [ffn, hidden] */
+    KL_WDOWN = 7,   /* [hidden, ffn] */
+    KL_NORM1 = 8,   /* [hidden]  gain of the RMSNorm before attention */
+    KL_NORM2 = 9,   /* [hidden]  gain of the RMSNorm before the MLP */
+    KL_NORM_F = 10, /* [hidden]  final gain              layer = -1 */
+    KL_LM_HEAD = 11 /* [vocab, hidden]                  layer = -1 */
+};
+
+typedef struct {
+    uint32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    float rms_eps;    /* added to the mean of squares, inside the root */
+    float rope_theta; /* RoPE base; pair (i, i + head_dim/2) rotates by position * theta^(-2i/head_dim) */
+    uint32_t max_batch;
+    uint32_t max_ctx; /* capacity of the KV cache in positions */
+    uint32_t flags;   /* reserved, must be 0 */
+} kl_model_desc;
+
+/* Sizes of the two device arenas the caller must provide to kl_create (both 256-byte aligned).
+ * weight_bytes holds the library's own copy of every tensor, grouped per layer and laid out linearly in the
+ * order the persistent kernel streams it (Section 3.2: grouped parameters [N x S], "linear in memory").
+ * scratch_bytes holds activations, split-K attention partials, synchronisation counters, the status word and
+ * staging buffers for the host-buffer entry point. */
+kl_status kl_workspace_bytes(const kl_model_desc* desc, size_t* weight_bytes, size_t* scratch_bytes);
+
+/* Creates a handle over caller-owned arenas (device pointers, sizes as reported by kl_workspace_bytes).
+ * Uses the current CUDA device.  The scratch arena is cleared synchronously.  *out is set on success only. */
+kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scratch_arena_d, kl_handle** out);
+
+/* Copies one tensor into the weight arena (host or device source, any pageable/pinned/device memory), in the
+ * library's streaming layout.  `bytes` must equal the tensor's size.  layer = -1 for KL_EMBED, KL_NORM_F,
+ * KL_LM_HEAD.  The copy is ordered on `stream`; the source may be released once the stream has passed it. */
+kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, size_t bytes, void* stream);
+
+/* Bytes of a KV cache for `batch` sequences: layout [n_layers][2 (K,V)][batch][n_kv_heads][max_ctx][head_dim]
+ * bf16.  Cached keys are stored already rotated.  The cache is caller-owned and updated in place. */
+size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch);
+
+/* KL_MODE_LOOPED (default): one persistent kernel runs all layers.  KL_MODE_PER_LAYER: one launch per layer. */
+kl_status kl_set_mode(kl_handle* h, int mode);
+
+/* One decode step for `batch` sequences, asynchronous on `stream`.
+ *   tokens_d[b]    token to embed (int32, < vocab)
+ *   positions_d[b] number of valid cached positions of sequence b = index written by this step (< max_ctx);
+ *                  attention covers positions 0..positions_d[b] inclusive
+ *   kv_cache_d     cache in the layout above; row positions_d[b] of every layer is written
+ *   logits_d       [batch, vocab] fp32, written
+ * Merged-call argument rule of Section 3.2: weights (grouped, all layers) come from the handle, the hidden
+ * state enters once (from the embedding) and leaves once (kl_read_hidden / the classifier), the KV cache is the
+ * grouped in/out parameter.  Device-detected errors make the step a no-op and are reported by kl_last_status. */
+kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
+                         float* logits_d, uint32_t batch, void* stream);
+
+/* Same step with HOST token / position / logit buffers: copies tokens and positions to the device, runs the
+ * step, copies the logits back and synchronises `stream` before returning.  The KV cache stays on the device. */
+kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
+                              float* logits_h, uint32_t batch, void* stream);
+
+/* Sampling block (greedy): tokens_d[b] = argmax_v logits_d[b, v] (lowest index on ties); positions_d[b] += 1. */
+kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d,
+                            uint32_t batch, void* stream);
+
+/* Copies the hidden state after the last decoder layer (before the final RMSNorm) of the latest step:
+ * hidden_d [batch, hidden] fp32. */
+kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream);
+
+/* Synchronises nothing: call after the stream has been synchronised.  Reads and clears the device status word
+ * (KL_OK, KL_ERR_SYNC_TIMEOUT or KL_ERR_OUT_OF_RANGE). */
+kl_status kl_last_status(kl_handle* h);
+
+/* Number of kernels this handle has launched so far (for reporting). */
+uint64_t kl_launch_count(const kl_handle* h);
+
+/* Per-kernel timing for roofline reports.  kl_profile_enable creates `capacity` sets of CUDA events (no device
+ * memory); from then on every kl_decode_step records events around its decoder launches and its classifier launch
+ * on the caller's stream, into set (step index mod capacity).  capacity = 0 switches recording off and destroys
+ * the events.  kl_profile_read (after the stream has been synchronised) returns, for the latest min(steps,
+ * capacity) steps, the milliseconds between the first decoder launch and the end of the last one, and of the
+ * classifier kernel; *n is in: room in the arrays, out: entries written. */
+kl_status kl_profile_enable(kl_handle* h, uint32_t capacity);
+kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* classifier_ms);
+
+/* Limit, in nanoseconds, of every device-side wait (flag, counter or mbarrier).  Default 2e9. */
+kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
+
+/* Test hook for the bounded waits: when stage >= 0 the CTAs of the persistent kernel do not signal the end of
+ * that stage (0..4) of layer 0 on the NEXT kl_decode_step only, so the waits on it run out and the step reports
+ * KL_ERR_SYNC_TIMEOUT.  No fault, trap or endless loop is involved. */
+kl_status kl_debug_skip_signal_once(kl_handle* h, int stage);
+
+const char* kl_status_string(kl_status s);
+
+/* Releases host-side state only (the arenas belong to the caller). */
+void kl_destroy(kl_handle* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KL_H_ */

@@ -1,0 +1,679 @@
+// Kernels and C ABI of the kernel-looped decoder (see include/kl.h for the contract of every entry point).
+//
+// Kernel schedule per decode step (Section 2 of the paper, call-schedule figure):
+//   looped    : embed -> decoder(layers 0..L-1, ONE persistent launch) -> classifier      (+ sampling)
+//   per-layer : embed -> decoder(l), l = 0..L-1 (L launches of the same body) -> classifier (+ sampling)
+//
+// The decoder kernel is persistent: one CTA per SM, one producer warp that streams this CTA's share of every
+// weight matrix through a shared-memory ring with TMA bulk copies, and NCW consumer warps.  Weight addresses do
+// not depend on activations, so the producer runs ahead of the consumers across stage boundaries and, in looped
+// mode, across layer boundaries: while the CTAs wait on the acquire/release counter that replaces a kernel
+// boundary, HBM keeps streaming the next stage's (next layer's) tiles.
+#include "kl_device.cuh"
+
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/kl.h"
+
+namespace kl {
+
+// ------------------------------------------------------------------------------------------------ kernels
+
+__global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
+    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    int32_t tok = p.tokens[b];
+    const int32_t pos = p.positions[b];
+    if (tid == 0 && (tok < 0 || tok >= (int32_t)p.V || pos < 0 || pos >= (int32_t)p.max_ctx))
+        atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+    if (tok < 0 || tok >= (int32_t)p.V) tok = 0;
+    const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
+    for (uint32_t i = tid; i < p.H; i += blockDim.x) p.x[(size_t)b * p.H + i] = __bfloat162float(row[i]);
+    // RoPE table of this step: angle in double so that large positions keep their phase
+    for (uint32_t i = tid; i < p.hd / 2; i += blockDim.x) {
+        double sn, cs;
+        sincos((double)pos * p.inv_freq[i], &sn, &cs);
+        p.rope_cs[((size_t)b * (p.hd / 2) + i) * 2] = (float)cs;
+        p.rope_cs[((size_t)b * (p.hd / 2) + i) * 2 + 1] = (float)sn;
+    }
+    if (b == 0) {
+        const uint32_t nw = p.L * 8 + p.L * p.B * p.nkv;  // counters, then tickets (contiguous)
+        for (uint32_t i = tid; i < nw; i += blockDim.x) p.counters[i] = 0u;
+    }
+}
+
+// Layers [l0, l1) of the decoder.  l1 - l0 == L is the looped kernel; l1 - l0 == 1 the per-layer launch.
+__global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, p);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    if (tid == 0) {
+        for (uint32_t i = 0; i < p.nslots; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        *s.abort_flag = 0;
+        *s.bcast = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    __syncthreads();
+    if (*p.status != 0) return;  // an earlier kernel of this step flagged bad input: the step is a no-op
+
+    if (warp == NCW) {
+        // ---------------- producer: the weight stream of this CTA, in consumption order
+        if (lane == 0) {
+            const uint64_t pol = l2_policy_evict_first();
+            RingPos rp = {0u, 0u, 0ull};
+            bool ok = true;
+            for (uint32_t l = l0; l < l1 && ok; ++l) {
+                const size_t lo = (size_t)l * p.layer_stride;
+                ok = produce_matrix(p, s, p.plan[PL_QKV], p.wqkv + lo, cta, rp, pol) &&
+                     produce_matrix(p, s, p.plan[PL_O], p.wo + lo, cta, rp, pol) &&
+                     produce_matrix(p, s, p.plan[PL_GU], p.wgu + lo, cta, rp, pol) &&
+                     produce_matrix(p, s, p.plan[PL_D], p.wd + lo, cta, rp, pol);
+            }
+            if (!ok) drain_ring(p, s, rp);
+        }
+        return;
+    }
+
+    // ---------------- consumers
+    const uint32_t ctid = tid;
+    uint64_t nbase = 0;
+    for (uint32_t l = l0; l < l1; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        uint32_t* ctr = p.counters + (size_t)l * 8;
+        const int skip = (l == 0) ? p.skip_stage : -1;
+        // S1: RMSNorm + QKV projection.  The hidden state of the previous layer must be complete.
+        if (l > l0) stage_wait(p, s, p.counters + (size_t)(l - 1) * 8 + ST_D, p.P, ctid);
+        load_vec(p, s, p.x, p.H, true, p.g1 + lo, ctid);
+        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, nbase);
+        stage_signal(ctr + ST_QKV, ctid, skip == ST_QKV);
+        // S2: RoPE, KV append, split-K attention, merge
+        stage_wait(p, s, ctr + ST_QKV, p.P, ctid);
+        switch (p.G) {
+            case 1: attention_stage<1>(p, s, l, cta, ctid, warp, lane); break;
+            case 2: attention_stage<2>(p, s, l, cta, ctid, warp, lane); break;
+            case 4: attention_stage<4>(p, s, l, cta, ctid, warp, lane); break;
+            default: attention_stage<8>(p, s, l, cta, ctid, warp, lane); break;
+        }
+        stage_signal(ctr + ST_ATTN, ctid, skip == ST_ATTN);
+        // S3: output projection + residual
+        stage_wait(p, s, ctr + ST_ATTN, p.P, ctid);
+        load_vec(p, s, p.o, p.QD, false, nullptr, ctid);
+        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, nbase);
+        stage_signal(ctr + ST_O, ctid, skip == ST_O);
+        // S4: RMSNorm + gate/up projections + SwiGLU
+        stage_wait(p, s, ctr + ST_O, p.P, ctid);
+        load_vec(p, s, p.x, p.H, true, p.g2 + lo, ctid);
+        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, nbase);
+        stage_signal(ctr + ST_GU, ctid, skip == ST_GU);
+        // S5: down projection + residual
+        stage_wait(p, s, ctr + ST_GU, p.P, ctid);
+        load_vec(p, s, p.h, p.F, false, nullptr, ctid);
+        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, nbase);
+        stage_signal(ctr + ST_D, ctid, skip == ST_D);
+    }
+}
+
+// Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
+__global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid_constant__ Params p) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, p);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    if (tid == 0) {
+        for (uint32_t i = 0; i < p.nslots; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        *s.abort_flag = 0;
+        *s.bcast = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    __syncthreads();
+    if (*p.status != 0) return;
+    if (warp == NCW) {
+        if (lane == 0) {
+            const uint64_t pol = l2_policy_evict_first();
+            RingPos rp = {0u, 0u, 0ull};
+            if (!produce_matrix(p, s, p.plan[PL_LM], p.wlm, cta, rp, pol)) drain_ring(p, s, rp);
+        }
+        return;
+    }
+    uint64_t nbase = 0;
+    load_vec(p, s, p.x, p.H, true, p.gf, tid);
+    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, nbase);
+}
+
+// Sampling block (greedy): lowest index among the maxima; then advance the position.
+__global__ void __launch_bounds__(1024) kl_argmax_kernel(const float* logits, uint32_t V, int32_t* tokens, int32_t* positions) {
+    __shared__ float sv[32];
+    __shared__ uint32_t si[32];
+    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    const float* row = logits + (size_t)b * V;
+    float bv = -INFINITY;
+    uint32_t bi = 0xffffffffu;
+    for (uint32_t i = tid; i < V; i += blockDim.x) {
+        const float v = row[i];
+        if (v > bv || (v == bv && i < bi)) {
+            bv = v;
+            bi = i;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const uint32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) {
+            bv = ov;
+            bi = oi;
+        }
+    }
+    if ((tid & 31) == 0) {
+        sv[tid >> 5] = bv;
+        si[tid >> 5] = bi;
+    }
+    __syncthreads();
+    if (tid < 32) {
+        const uint32_t nw = (blockDim.x + 31) / 32;
+        bv = tid < nw ? sv[tid] : -INFINITY;
+        bi = tid < nw ? si[tid] : 0xffffffffu;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const uint32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) {
+                bv = ov;
+                bi = oi;
+            }
+        }
+        if (tid == 0) {
+            tokens[b] = (int32_t)(bi == 0xffffffffu ? 0u : bi);
+            positions[b] += 1;
+        }
+    }
+}
+
+}  // namespace kl
+
+// ------------------------------------------------------------------------------------------------ host side
+
+using namespace kl;
+
+struct kl_handle {
+    kl_model_desc desc;
+    Params prm;
+    int mode;
+    int device;
+    int num_sms;
+    size_t smem_bytes;
+    uint8_t* weights;  // arena
+    uint8_t* scratch;  // arena
+    size_t weight_bytes, scratch_bytes;
+    // scratch sub-allocations used by the host-buffer entry point
+    int32_t* stage_tokens;
+    int32_t* stage_positions;
+    float* stage_logits;
+    uint64_t launches;
+    uint64_t loaded_layer_mask_count;  // number of (tensor, layer) pairs loaded
+    uint8_t* loaded;                   // [12][L] flags (host)
+    int pending_skip_stage;
+    // optional event recording around the decoder and classifier launches
+    uint32_t prof_capacity;
+    uint64_t prof_steps;
+    cudaEvent_t* prof_events;  // [capacity][3]
+};
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
+inline uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
+
+struct Layout {
+    // weight arena, element offsets (bf16)
+    size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
+    size_t off_gf, off_lm, off_embed, weight_elems;
+    // scratch arena, byte offsets
+    size_t sx, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, scratch_bytes;
+    uint32_t cps;
+};
+
+bool shape_supported(const kl_model_desc& d, int num_sms) {
+    if (!d.n_layers || !d.hidden || !d.n_q_heads || !d.n_kv_heads || !d.head_dim || !d.ffn || !d.vocab) return false;
+    if (!d.max_batch || !d.max_ctx || d.flags != 0) return false;
+    if (d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128 && d.head_dim != 256) return false;
+    if (d.hidden % 8 || d.ffn % 8) return false;
+    if (d.n_q_heads % d.n_kv_heads) return false;
+    const uint32_t G = d.n_q_heads / d.n_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return false;
+    if ((uint64_t)d.max_batch * d.n_kv_heads > (uint64_t)num_sms) return false;
+    if (!(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f)) return false;
+    return true;
+}
+
+Layout make_layout(const kl_model_desc& d, int num_sms) {
+    Layout y;
+    const size_t H = d.hidden, QD = (size_t)d.n_q_heads * d.head_dim, KVD = (size_t)d.n_kv_heads * d.head_dim, F = d.ffn,
+                 V = d.vocab, B = d.max_batch;
+    size_t o = 0;
+    y.off_qkv = o; o += (QD + 2 * KVD) * H;
+    y.off_o = o;   o += H * QD;
+    y.off_gu = o;  o += 2 * F * H;
+    y.off_d = o;   o += H * F;
+    y.off_g1 = o;  o += H;
+    y.off_g2 = o;  o += H;
+    y.layer_stride = align_up(o * 2, ALIGN) / 2;
+    o = y.layer_stride * d.n_layers;
+    y.off_gf = o;    o += align_up(H * 2, ALIGN) / 2;
+    y.off_lm = o;    o += align_up(V * H * 2, ALIGN) / 2;
+    y.off_embed = o; o += align_up(V * H * 2, ALIGN) / 2;
+    y.weight_elems = o;
+
+    y.cps = (uint32_t)num_sms / (uint32_t)(B * d.n_kv_heads);
+    const uint32_t G = d.n_q_heads / d.n_kv_heads;
+    const size_t units = (size_t)num_sms;  // at most one attention unit per CTA
+    size_t s = 0;
+    y.sx = s;        s += align_up(B * H * 4);
+    y.sqkv = s;      s += align_up(B * (QD + 2 * KVD) * 4);
+    y.so = s;        s += align_up(B * QD * 4);
+    y.sh = s;        s += align_up(B * F * 4);
+    y.spart = s;     s += align_up(units * G * d.head_dim * 4);
+    y.spart_ml = s;  s += align_up(units * G * 2 * 4);
+    y.srope = s;     s += align_up(B * d.head_dim * 4);
+    y.sinvf = s;     s += align_up((size_t)(d.head_dim / 2) * 8);
+    y.scounters = s; s += align_up(((size_t)d.n_layers * 8 + (size_t)d.n_layers * B * d.n_kv_heads) * 4);
+    y.sstatus = s;   s += ALIGN;
+    y.stok = s;      s += align_up(B * 4);
+    y.spos = s;      s += align_up(B * 4);
+    y.slogits = s;   s += align_up(B * V * 4);
+    y.scratch_bytes = s;
+    return y;
+}
+
+GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P) {
+    GemvPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    pl.R = R;
+    pl.K = K;
+    const uint32_t rowbytes = K * 2;
+    const uint32_t minrows = pairs ? 2u : 1u;
+    if (rowbytes * minrows <= (uint32_t)SLOT_BYTES) {
+        uint32_t rpc = SLOT_BYTES / rowbytes;
+        uint32_t cap = R / (2 * P);  // keep at least ~2 chunks per CTA on small matrices
+        if (cap < minrows) cap = minrows;
+        if (rpc > cap) rpc = cap;
+        if (pairs) rpc &= ~1u;
+        pl.rpc = rpc;
+        pl.ksplit = 1;
+        pl.klen = K;
+        pl.rows_per_unit = rpc;
+        pl.nunits = ceil_div(R, rpc);
+        pl.chunks_per_unit = 1;
+    } else {
+        pl.rpc = 0;
+        uint32_t ksplit = ceil_div(rowbytes, SLOT_BYTES);
+        pl.klen = ceil_div(ceil_div(K, ksplit), 256) * 256;
+        pl.ksplit = ceil_div(K, pl.klen);
+        pl.rows_per_unit = minrows;
+        pl.nunits = R / minrows;
+        pl.chunks_per_unit = pl.rows_per_unit * pl.ksplit;
+    }
+    return pl;
+}
+
+bool plans_ok(const Params& p) {
+    for (int i = 0; i < PL_COUNT; ++i) {
+        const GemvPlan& pl = p.plan[i];
+        if (pl.rpc == 0 && (pl.chunks_per_unit > (uint32_t)MAX_PIECES || pl.klen * 2 > (uint32_t)SLOT_BYTES)) return false;
+        if (pl.rpc != 0 && pl.rpc * pl.K * 2 > (uint32_t)SLOT_BYTES) return false;
+    }
+    return true;
+}
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+}  // namespace
+
+extern "C" {
+
+const char* kl_status_string(kl_status s) {
+    switch (s) {
+        case KL_OK: return "KL_OK";
+        case KL_ERR_INVALID_ARG: return "KL_ERR_INVALID_ARG";
+        case KL_ERR_UNSUPPORTED_SHAPE: return "KL_ERR_UNSUPPORTED_SHAPE";
+        case KL_ERR_NOT_LOADED: return "KL_ERR_NOT_LOADED";
+        case KL_ERR_CUDA: return "KL_ERR_CUDA";
+        case KL_ERR_SYNC_TIMEOUT: return "KL_ERR_SYNC_TIMEOUT";
+        case KL_ERR_OUT_OF_RANGE: return "KL_ERR_OUT_OF_RANGE";
+        default: return "KL_ERR_UNKNOWN";
+    }
+}
+
+static int query_sms(int* dev_out) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    if (dev_out) *dev_out = dev;
+    return sms;
+}
+
+kl_status kl_workspace_bytes(const kl_model_desc* desc, size_t* weight_bytes, size_t* scratch_bytes) {
+    if (!desc || !weight_bytes || !scratch_bytes) return KL_ERR_INVALID_ARG;
+    int sms = query_sms(nullptr);
+    if (sms <= 0) sms = 148;  // sizes must be computable without a device; B200 has 148 SMs
+    if (!shape_supported(*desc, sms)) return KL_ERR_UNSUPPORTED_SHAPE;
+    const Layout y = make_layout(*desc, sms);
+    *weight_bytes = y.weight_elems * 2;
+    *scratch_bytes = y.scratch_bytes;
+    return KL_OK;
+}
+
+kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scratch_arena_d, kl_handle** out) {
+    if (!desc || !weight_arena_d || !scratch_arena_d || !out) return KL_ERR_INVALID_ARG;
+    if (((uintptr_t)weight_arena_d | (uintptr_t)scratch_arena_d) & (ALIGN - 1)) return KL_ERR_INVALID_ARG;
+    int dev = 0;
+    const int sms = query_sms(&dev);
+    if (sms <= 0) return KL_ERR_CUDA;
+    if (!shape_supported(*desc, sms)) return KL_ERR_UNSUPPORTED_SHAPE;
+    const kl_model_desc& d = *desc;
+    const Layout y = make_layout(d, sms);
+
+    kl_handle* h = new (std::nothrow) kl_handle();
+    if (!h) return KL_ERR_INVALID_ARG;
+    memset(h, 0, sizeof(*h));
+    h->desc = d;
+    h->mode = KL_MODE_LOOPED;
+    h->device = dev;
+    h->num_sms = sms;
+    h->weights = (uint8_t*)weight_arena_d;
+    h->scratch = (uint8_t*)scratch_arena_d;
+    h->weight_bytes = y.weight_elems * 2;
+    h->scratch_bytes = y.scratch_bytes;
+    h->pending_skip_stage = -1;
+    h->loaded = (uint8_t*)calloc(12 * (size_t)d.n_layers, 1);
+    if (!h->loaded) { delete h; return KL_ERR_INVALID_ARG; }
+
+    Params& p = h->prm;
+    p.L = d.n_layers; p.H = d.hidden; p.nq = d.n_q_heads; p.nkv = d.n_kv_heads; p.hd = d.head_dim; p.F = d.ffn;
+    p.V = d.vocab; p.G = d.n_q_heads / d.n_kv_heads; p.QD = d.n_q_heads * d.head_dim; p.KVD = d.n_kv_heads * d.head_dim;
+    p.max_ctx = d.max_ctx; p.B = 1;
+    p.P = (uint32_t)sms;
+    p.cps = y.cps;
+    p.eps = d.rms_eps;
+    p.skip_stage = -1;
+    p.wait_ns = 2000000000ull;
+    p.layer_stride = y.layer_stride;
+    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P);
+    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P);
+    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P);
+    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P);
+    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P);
+    if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+
+    // shared memory: input vector area (also the attention workspace), then as many ring slots as fit
+    uint32_t vecf = p.H > p.QD ? p.H : p.QD;
+    if (p.F > vecf) vecf = p.F;
+    vecf = ceil_div(vecf, 256) * 256;
+    const uint32_t attnf = p.G * p.hd + 2 * p.hd + NCW * p.G * (p.hd + 2);
+    if (attnf > vecf) vecf = ceil_div(attnf, 256) * 256;
+    p.vec_floats = vecf;
+    int max_optin = 0;
+    if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+        free(h->loaded); delete h; return KL_ERR_CUDA;
+    }
+    const long avail = (long)max_optin - (long)vecf * 4 - SMEM_MISC_BYTES;
+    long nslots = avail / SLOT_BYTES;
+    if (nslots > MAX_SLOTS) nslots = MAX_SLOTS;
+    if (nslots < 3) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    p.nslots = (uint32_t)nslots;
+    h->smem_bytes = (size_t)nslots * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
+    if (cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess) {
+        free(h->loaded); delete h; return KL_ERR_CUDA;
+    }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes) != cudaSuccess || occ < 1) {
+        free(h->loaded); delete h; return KL_ERR_CUDA;
+    }
+
+    const __nv_bfloat16* w = reinterpret_cast<const __nv_bfloat16*>(h->weights);
+    p.wqkv = w + y.off_qkv; p.wo = w + y.off_o; p.wgu = w + y.off_gu; p.wd = w + y.off_d;
+    p.g1 = w + y.off_g1; p.g2 = w + y.off_g2; p.gf = w + y.off_gf; p.wlm = w + y.off_lm; p.embed = w + y.off_embed;
+    uint8_t* sc = h->scratch;
+    p.x = (float*)(sc + y.sx); p.qkv = (float*)(sc + y.sqkv); p.o = (float*)(sc + y.so); p.h = (float*)(sc + y.sh);
+    p.part = (float*)(sc + y.spart); p.part_ml = (float*)(sc + y.spart_ml); p.rope_cs = (float*)(sc + y.srope);
+    p.inv_freq = (const double*)(sc + y.sinvf);
+    p.counters = (uint32_t*)(sc + y.scounters);
+    p.tickets = p.counters + (size_t)p.L * 8;
+    p.status = (int32_t*)(sc + y.sstatus);
+    h->stage_tokens = (int32_t*)(sc + y.stok);
+    h->stage_positions = (int32_t*)(sc + y.spos);
+    h->stage_logits = (float*)(sc + y.slogits);
+
+    if (cudaMemset(h->scratch, 0, h->scratch_bytes) != cudaSuccess) { free(h->loaded); delete h; return KL_ERR_CUDA; }
+    double invf[128];
+    for (uint32_t i = 0; i < d.head_dim / 2; ++i) invf[i] = pow((double)d.rope_theta, -2.0 * (double)i / (double)d.head_dim);
+    if (cudaMemcpy(sc + y.sinvf, invf, (d.head_dim / 2) * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess) {
+        free(h->loaded); delete h; return KL_ERR_CUDA;
+    }
+    *out = h;
+    return KL_OK;
+}
+
+kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, size_t bytes, void* stream) {
+    if (!h || !src) return KL_ERR_INVALID_ARG;
+    const Params& p = h->prm;
+    const Layout y = make_layout(h->desc, h->num_sms);
+    const bool global_t = (tensor == KL_EMBED || tensor == KL_NORM_F || tensor == KL_LM_HEAD);
+    if (tensor < 0 || tensor > KL_LM_HEAD) return KL_ERR_INVALID_ARG;
+    if (global_t ? (layer != -1) : (layer < 0 || layer >= (int)p.L)) return KL_ERR_INVALID_ARG;
+    __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(h->weights);
+    const size_t lo = global_t ? 0 : (size_t)layer * y.layer_stride;
+    size_t rows = 0, cols = 0, dst = 0, dpitch_elems = 0;
+    switch (tensor) {
+        case KL_EMBED: rows = p.V; cols = p.H; dst = y.off_embed; break;
+        case KL_LM_HEAD: rows = p.V; cols = p.H; dst = y.off_lm; break;
+        case KL_NORM_F: rows = 1; cols = p.H; dst = y.off_gf; break;
+        case KL_WQ: rows = p.QD; cols = p.H; dst = lo + y.off_qkv; break;
+        case KL_WK: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv + (size_t)p.QD * p.H; break;
+        case KL_WV: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv + (size_t)(p.QD + p.KVD) * p.H; break;
+        case KL_WO: rows = p.H; cols = p.QD; dst = lo + y.off_o; break;
+        case KL_WGATE: rows = p.F; cols = p.H; dst = lo + y.off_gu; dpitch_elems = 2 * (size_t)p.H; break;
+        case KL_WUP: rows = p.F; cols = p.H; dst = lo + y.off_gu + p.H; dpitch_elems = 2 * (size_t)p.H; break;
+        case KL_WDOWN: rows = p.H; cols = p.F; dst = lo + y.off_d; break;
+        case KL_NORM1: rows = 1; cols = p.H; dst = lo + y.off_g1; break;
+        case KL_NORM2: rows = 1; cols = p.H; dst = lo + y.off_g2; break;
+        default: return KL_ERR_INVALID_ARG;
+    }
+    if (bytes != rows * cols * 2) return KL_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (dpitch_elems) {
+        // gate and up rows are interleaved (row 2f = gate f, row 2f+1 = up f) so one chunk holds both halves of a pair
+        e = cudaMemcpy2DAsync(w + dst, dpitch_elems * 2, src, cols * 2, cols * 2, rows, cudaMemcpyDefault, as_stream(stream));
+    } else {
+        e = cudaMemcpyAsync(w + dst, src, bytes, cudaMemcpyDefault, as_stream(stream));
+    }
+    if (e != cudaSuccess) return KL_ERR_CUDA;
+    h->loaded[(size_t)tensor * p.L + (global_t ? 0 : layer)] = 1;
+    return KL_OK;
+}
+
+static bool all_loaded(const kl_handle* h) {
+    const uint32_t L = h->prm.L;
+    for (int t = 0; t <= KL_LM_HEAD; ++t) {
+        const bool global_t = (t == KL_EMBED || t == KL_NORM_F || t == KL_LM_HEAD);
+        for (uint32_t l = 0; l < (global_t ? 1u : L); ++l)
+            if (!h->loaded[(size_t)t * L + l]) return false;
+    }
+    return true;
+}
+
+size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch) {
+    if (!h) return 0;
+    const kl_model_desc& d = h->desc;
+    return (size_t)d.n_layers * 2 * batch * d.n_kv_heads * d.max_ctx * d.head_dim * 2;
+}
+
+kl_status kl_set_mode(kl_handle* h, int mode) {
+    if (!h || (mode != KL_MODE_LOOPED && mode != KL_MODE_PER_LAYER)) return KL_ERR_INVALID_ARG;
+    h->mode = mode;
+    return KL_OK;
+}
+
+static kl_status launch_persistent(kl_handle* h, const void* func, void** args, cudaStream_t st) {
+    // cooperative launch: the driver guarantees that all CTAs are co-resident (the counters depend on it)
+    const cudaError_t e = cudaLaunchCooperativeKernel(func, dim3(h->prm.P), dim3(NTHREADS), args, h->smem_bytes, st);
+    if (e != cudaSuccess) return KL_ERR_CUDA;
+    ++h->launches;
+    return KL_OK;
+}
+
+kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
+                         float* logits_d, uint32_t batch, void* stream) {
+    if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    if (batch != 1) return KL_ERR_UNSUPPORTED_SHAPE;  // batched tensor-core path not built yet
+    if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
+    cudaStream_t st = as_stream(stream);
+    Params p = h->prm;
+    p.B = batch;
+    p.cps = (uint32_t)h->num_sms / (batch * p.nkv);
+    p.tokens = tokens_d;
+    p.positions = positions_d;
+    p.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
+    p.logits = logits_d;
+    p.skip_stage = h->pending_skip_stage;
+    h->pending_skip_stage = -1;
+
+    kl_embed_kernel<<<batch, 256, 0, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+    ++h->launches;
+    kl_status rc;
+    cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
+    if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+    if (h->mode == KL_MODE_LOOPED) {
+        uint32_t l0 = 0, l1 = p.L;
+        void* args[] = {&p, &l0, &l1};
+        if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+    } else {
+        for (uint32_t l = 0; l < p.L; ++l) {
+            uint32_t l0 = l, l1 = l + 1;
+            void* args[] = {&p, &l0, &l1};
+            if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+        }
+    }
+    if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
+    void* cargs[] = {&p};
+    if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
+    if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
+    return KL_OK;
+}
+
+kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
+                              float* logits_h, uint32_t batch, void* stream) {
+    if (!h || !tokens_h || !positions_h || !kv_cache_d || !logits_h) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(h->stage_tokens, tokens_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+    if (cudaMemcpyAsync(h->stage_positions, positions_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+    const kl_status rc = kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
+    if (rc != KL_OK) return rc;
+    if (cudaMemcpyAsync(logits_h, h->stage_logits, (size_t)batch * h->prm.V * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KL_ERR_CUDA;
+    return KL_OK;
+}
+
+kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d, uint32_t batch,
+                            void* stream) {
+    if (!h || !logits_d || !tokens_d || !positions_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    kl_argmax_kernel<<<batch, 1024, 0, as_stream(stream)>>>(logits_d, h->prm.V, tokens_d, positions_d);
+    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+    ++h->launches;
+    return KL_OK;
+}
+
+kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream) {
+    if (!h || !hidden_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    if (cudaMemcpyAsync(hidden_d, h->prm.x, (size_t)batch * h->prm.H * 4, cudaMemcpyDeviceToDevice, as_stream(stream)) != cudaSuccess)
+        return KL_ERR_CUDA;
+    return KL_OK;
+}
+
+kl_status kl_last_status(kl_handle* h) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    int32_t v = 0;
+    if (cudaMemcpy(&v, h->prm.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return KL_ERR_CUDA;
+    if (v != 0) {
+        const int32_t zero = 0;
+        if (cudaMemcpy(h->prm.status, &zero, 4, cudaMemcpyHostToDevice) != cudaSuccess) return KL_ERR_CUDA;
+    }
+    return (kl_status)v;
+}
+
+uint64_t kl_launch_count(const kl_handle* h) { return h ? h->launches : 0; }
+
+kl_status kl_profile_enable(kl_handle* h, uint32_t capacity) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    if (h->prof_events) {
+        for (uint32_t i = 0; i < 3 * h->prof_capacity; ++i) cudaEventDestroy(h->prof_events[i]);
+        free(h->prof_events);
+        h->prof_events = nullptr;
+    }
+    h->prof_capacity = 0;
+    h->prof_steps = 0;
+    if (capacity == 0) return KL_OK;
+    h->prof_events = (cudaEvent_t*)calloc(3 * (size_t)capacity, sizeof(cudaEvent_t));
+    if (!h->prof_events) return KL_ERR_INVALID_ARG;
+    for (uint32_t i = 0; i < 3 * capacity; ++i) {
+        if (cudaEventCreate(&h->prof_events[i]) != cudaSuccess) {
+            for (uint32_t j = 0; j < i; ++j) cudaEventDestroy(h->prof_events[j]);
+            free(h->prof_events);
+            h->prof_events = nullptr;
+            return KL_ERR_CUDA;
+        }
+    }
+    h->prof_capacity = capacity;
+    return KL_OK;
+}
+
+kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* classifier_ms) {
+    if (!h || !n || !decoder_ms || !classifier_ms) return KL_ERR_INVALID_ARG;
+    const uint64_t have = h->prof_steps < h->prof_capacity ? h->prof_steps : h->prof_capacity;
+    const uint32_t cnt = (uint32_t)(have < *n ? have : *n);
+    for (uint32_t i = 0; i < cnt; ++i) {
+        cudaEvent_t* ev = h->prof_events + 3 * ((h->prof_steps - 1 - i) % h->prof_capacity);
+        if (cudaEventElapsedTime(&decoder_ms[i], ev[0], ev[1]) != cudaSuccess) return KL_ERR_CUDA;
+        if (cudaEventElapsedTime(&classifier_ms[i], ev[1], ev[2]) != cudaSuccess) return KL_ERR_CUDA;
+    }
+    *n = cnt;
+    return KL_OK;
+}
+
+kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns) {
+    if (!h || ns == 0) return KL_ERR_INVALID_ARG;
+    h->prm.wait_ns = ns;
+    return KL_OK;
+}
+
+kl_status kl_debug_skip_signal_once(kl_handle* h, int stage) {
+    if (!h || stage < -1 || stage > 4) return KL_ERR_INVALID_ARG;
+    h->pending_skip_stage = stage;
+    return KL_OK;
+}
+
+void kl_destroy(kl_handle* h) {
+    if (!h) return;
+    kl_profile_enable(h, 0);
+    free(h->loaded);
+    delete h;
+}
+
+}  // extern "C"
