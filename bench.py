@@ -34,6 +34,8 @@ WORKLOADS = {
     # name: (shape, batch, context, default steps)
     "tiny_b1_ctx128": (gen.TINY, 1, 128, 16),
     "llama31_8b_b1_ctx4096": (gen.LLAMA31_8B, 1, 4096, 128),
+    # four layers of the same shape: a few GB on the device, for multi-pass profiler captures
+    "llama31_8b_4layers_b1_ctx4096": (gen.ModelShape(4, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 1, 4096, 8),
     "llama31_8b_b1_ctx65536": (gen.LLAMA31_8B, 1, 65536, 64),
     "llama31_70b_b1_ctx4096": (gen.LLAMA31_70B, 1, 4096, 32),
 }

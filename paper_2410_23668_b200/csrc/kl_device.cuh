@@ -9,11 +9,11 @@
 
 namespace kl {
 
-constexpr int NCW = 8;                     // consumer warps per CTA
+constexpr int NCW = 10;                    // consumer warps per CTA; consumer warp w owns ring slot w
 constexpr int NCT = NCW * 32;              // consumer threads
 constexpr int NTHREADS = NCT + 32;         // + one producer warp (the last warp)
 constexpr int SLOT_BYTES = 16384;          // one ring slot = one TMA bulk copy
-constexpr int MAX_SLOTS = 13;
+constexpr int MAX_SLOTS = NCW;             // one owner warp per slot (see gemv_stage)
 constexpr int MAX_PIECES = 8;              // chunks per unit when a unit spans several chunks
 constexpr int UNIT_SLOTS = 32;             // in-flight multi-chunk units tracked per CTA
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
@@ -363,13 +363,18 @@ __device__ __forceinline__ float silu(float z) { return z / (1.0f + __expf(-z));
 //   EP_RESIDUAL out[row] = out[row] + y            (out is the hidden state, owned row-wise by this CTA)
 //   EP_SWIGLU   rows come in (gate, up) pairs: out[row/2] = silu(y_gate) * y_up
 // nbase counts the chunks this CTA has consumed so far (identical to the producer's issue order).
+// Chunk n lives in slot n % nslots and is consumed by warp n % nslots: every use of a slot is waited on by the
+// same warp, in order, so a parity wait can never be satisfied by a phase two uses old.  (With free chunk-to-warp
+// assignment a fast warp can test the barrier of use k while use k-1 is still in flight, and parity k&1 then
+// reads as complete.)
 __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, float* out,
                                            uint32_t cta, uint32_t warp, uint32_t lane, uint64_t& nbase) {
     const CtaRange r = cta_units(pl, cta, p.P);
     const uint32_t nch = (r.u1 - r.u0) * pl.chunks_per_unit;
-    for (uint32_t i = warp; i < nch; i += NCW) {
+    const uint32_t first = (warp + p.nslots - (uint32_t)(nbase % p.nslots)) % p.nslots;
+    for (uint32_t i = (warp < p.nslots ? first : nch); i < nch; i += p.nslots) {
         const uint64_t n = nbase + i;
-        const uint32_t slot = (uint32_t)(n % p.nslots);
+        const uint32_t slot = warp;
         const uint32_t phase = (uint32_t)((n / p.nslots) & 1u);
         mbar_wait(p, s, smem_u32(&s.full[slot]), phase);
         const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
