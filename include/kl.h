@@ -130,6 +130,26 @@ uint64_t kl_launch_count(const kl_handle* h);
 kl_status kl_profile_enable(kl_handle* h, uint32_t capacity);
 kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* classifier_ms);
 
+/* Stage timeline of the decoder kernel (the analogue of the paper's per-socket HBM-bandwidth trace, Section 4).
+ * trace_d: DEVICE buffer of n_ctas * n_layers * n_stamps + 8192 * 4 uint64 (zero it first), or NULL to switch
+ * tracing off; the three sizes
+ * are returned through the out pointers (each may be NULL).  While set, consumer thread 0 of every CTA stores the
+ * GPU global timer (ns) at fixed points of every layer: 0 previous layer complete, 1 input normalised, 2 QKV rows
+ * done and signalled, 3 all QKV seen, 4 attention unit done and signalled, 5 all attention seen, 6 o loaded,
+ * 7 O-projection done, 8 all O seen, 9 input normalised, 10 gate/up done, 11 all gate/up seen, 12 h loaded,
+ * 13 down-projection done, 14 attention prologue done, 15 attention ring chunks consumed.  The trailing
+ * 8192 x 4 block logs the first 8192 ring chunks of CTA 0: issue by the producer, consumer starts waiting, chunk
+ * landed, chunk consumed and released.  Stamps of the latest step overwrite earlier ones. */
+kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32_t* n_layers, uint32_t* n_stamps);
+
+/* Attention inner loop.  on = 1 (default when head_dim is 64 or 128): tensor-core loop (mma.sync on 128-byte
+ * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
+kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
+
+/* Tuning knob: how many 16 KB chunks beyond its shared-memory ring each CTA's producer asks L2 to prefetch
+ * (0..64, default 0 = off).  The look-ahead of all CTAs together must stay well inside L2. */
+kl_status kl_set_prefetch_chunks(kl_handle* h, uint32_t chunks);
+
 /* Limit, in nanoseconds, of every device-side wait (flag, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
 

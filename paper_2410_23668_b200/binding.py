@@ -28,7 +28,8 @@ TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup":
 EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_bytes", "kl_set_mode", "kl_decode_step",
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
-           "kl_profile_read")
+           "kl_profile_read", "kl_set_trace", "kl_set_prefetch_chunks",
+           "kl_set_tensor_core_attention")
 
 
 class ModelDesc(C.Structure):
@@ -81,6 +82,12 @@ def lib():
     l.kl_profile_enable.restype = i32
     l.kl_profile_read.argtypes = [vp, C.POINTER(u32), C.POINTER(C.c_float), C.POINTER(C.c_float)]
     l.kl_profile_read.restype = i32
+    l.kl_set_trace.argtypes = [vp, vp, C.POINTER(u32), C.POINTER(u32), C.POINTER(u32)]
+    l.kl_set_trace.restype = i32
+    l.kl_set_prefetch_chunks.argtypes = [vp, u32]
+    l.kl_set_prefetch_chunks.restype = i32
+    l.kl_set_tensor_core_attention.argtypes = [vp, C.c_int]
+    l.kl_set_tensor_core_attention.restype = i32
     l.kl_status_string.argtypes = [i32]
     l.kl_status_string.restype = C.c_char_p
     l.kl_destroy.argtypes = [vp]
@@ -195,6 +202,18 @@ class Decoder:
         dec, cls = (C.c_float * n)(), (C.c_float * n)()
         _check(lib().kl_profile_read(self.handle, C.byref(cnt), dec, cls), "kl_profile_read")
         return list(dec[:cnt.value]), list(cls[:cnt.value])
+
+    def kl_set_trace(self, trace_d=None) -> tuple[int, int, int]:
+        a, b, c = C.c_uint32(), C.c_uint32(), C.c_uint32()
+        _check(lib().kl_set_trace(self.handle, _ptr(trace_d), C.byref(a), C.byref(b), C.byref(c)), "kl_set_trace")
+        return a.value, b.value, c.value
+
+    def kl_set_tensor_core_attention(self, on: bool) -> None:
+        _check(lib().kl_set_tensor_core_attention(self.handle, 1 if on else 0), "kl_set_tensor_core_attention")
+
+    def kl_set_prefetch_chunks(self, chunks: int) -> None:
+        _check(lib().kl_set_prefetch_chunks(self.handle, chunks), "kl_set_prefetch_chunks",
+           "kl_set_tensor_core_attention")
 
     def kl_set_wait_limit_ns(self, ns: int) -> None:
         _check(lib().kl_set_wait_limit_ns(self.handle, ns), "kl_set_wait_limit_ns")

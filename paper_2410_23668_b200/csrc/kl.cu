@@ -48,14 +48,12 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
 
 // Layers [l0, l1) of the decoder.  l1 - l0 == L is the looped kernel; l1 - l0 == 1 the per-layer launch.
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1) {
-    extern __shared__ __align__(128) uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
+        for (uint32_t i = 0; i < p.nslots; ++i) mbar_init(smem_u32(&s.full[i]), 1);
+        make_decoder_plan(*s.plan, p, cta, l1);
         *s.abort_flag = 0;
         *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -65,73 +63,75 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     __syncthreads();
     if (*p.status != 0) return;  // an earlier kernel of this step flagged bad input: the step is a no-op
 
-    if (warp == NCW) {
-        // ---------------- producer: the weight stream of this CTA, in consumption order
-        if (lane == 0) {
-            const uint64_t pol = l2_policy_evict_first();
-            RingPos rp = {0u, 0u, 0ull};
-            bool ok = true;
-            for (uint32_t l = l0; l < l1 && ok; ++l) {
-                const size_t lo = (size_t)l * p.layer_stride;
-                ok = produce_matrix(p, s, p.plan[PL_QKV], p.wqkv + lo, cta, rp, pol) &&
-                     produce_matrix(p, s, p.plan[PL_O], p.wo + lo, cta, rp, pol) &&
-                     produce_matrix(p, s, p.plan[PL_GU], p.wgu + lo, cta, rp, pol) &&
-                     produce_matrix(p, s, p.plan[PL_D], p.wd + lo, cta, rp, pol);
-            }
-            if (!ok) drain_ring(p, s, rp);
-        }
-        return;
-    }
+    // every warp starts the copy of its first chunk, then follows the stages
+    const uint64_t pol = l2_policy_evict_first();
+    WarpRing wr = ring_begin(p, s, warp, l0);
+    ring_issue_next(p, s, wr, warp, lane, pol);
 
     // ---------------- consumers
     const uint32_t ctid = tid;
-    uint64_t nbase = 0;
+    RingCursor rc = {0u, 0u};
     for (uint32_t l = l0; l < l1; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         uint32_t* ctr = p.counters + (size_t)l * 8;
         const int skip = (l == 0) ? p.skip_stage : -1;
         // S1: RMSNorm + QKV projection.  The hidden state of the previous layer must be complete.
         if (l > l0) stage_wait(p, s, p.counters + (size_t)(l - 1) * 8 + ST_D, p.P, ctid);
+        trace_stamp(p, cta, l, 0, ctid);
         load_vec(p, s, p.x, p.H, true, p.g1 + lo, ctid);
-        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, nbase);
+        trace_stamp(p, cta, l, 1, ctid);
+        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, rc, wr, pol);
         stage_signal(ctr + ST_QKV, ctid, skip == ST_QKV);
+        trace_stamp(p, cta, l, 2, ctid);
         // S2: RoPE, KV append, split-K attention, merge
         stage_wait(p, s, ctr + ST_QKV, p.P, ctid);
-        switch (p.G) {
-            case 1: attention_stage<1>(p, s, l, cta, ctid, warp, lane); break;
-            case 2: attention_stage<2>(p, s, l, cta, ctid, warp, lane); break;
-            case 4: attention_stage<4>(p, s, l, cta, ctid, warp, lane); break;
-            default: attention_stage<8>(p, s, l, cta, ctid, warp, lane); break;
+        trace_stamp(p, cta, l, 3, ctid);
+        if (p.attn_tc) {
+            attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr, pol);
+        } else switch (p.G) {
+            case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
+            case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
+            case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
+            default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
         }
         stage_signal(ctr + ST_ATTN, ctid, skip == ST_ATTN);
+        trace_stamp(p, cta, l, 4, ctid);
         // S3: output projection + residual
         stage_wait(p, s, ctr + ST_ATTN, p.P, ctid);
+        trace_stamp(p, cta, l, 5, ctid);
         load_vec(p, s, p.o, p.QD, false, nullptr, ctid);
-        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, nbase);
+        trace_stamp(p, cta, l, 6, ctid);
+        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, pol);
         stage_signal(ctr + ST_O, ctid, skip == ST_O);
+        trace_stamp(p, cta, l, 7, ctid);
         // S4: RMSNorm + gate/up projections + SwiGLU
         stage_wait(p, s, ctr + ST_O, p.P, ctid);
+        trace_stamp(p, cta, l, 8, ctid);
         load_vec(p, s, p.x, p.H, true, p.g2 + lo, ctid);
-        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, nbase);
+        trace_stamp(p, cta, l, 9, ctid);
+        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, rc, wr, pol);
         stage_signal(ctr + ST_GU, ctid, skip == ST_GU);
+        trace_stamp(p, cta, l, 10, ctid);
         // S5: down projection + residual
         stage_wait(p, s, ctr + ST_GU, p.P, ctid);
+        trace_stamp(p, cta, l, 11, ctid);
         load_vec(p, s, p.h, p.F, false, nullptr, ctid);
-        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, nbase);
+        trace_stamp(p, cta, l, 12, ctid);
+        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, pol);
         stage_signal(ctr + ST_D, ctid, skip == ST_D);
+        trace_stamp(p, cta, l, 13, ctid);
     }
+    ring_finish(p, s, wr, warp);
 }
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
 __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid_constant__ Params p) {
-    extern __shared__ __align__(128) uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
+        for (uint32_t i = 0; i < p.nslots; ++i) mbar_init(smem_u32(&s.full[i]), 1);
+        make_classifier_plan(*s.plan, p, cta);
         *s.abort_flag = 0;
         *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -140,62 +140,64 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
     __syncthreads();
     if (*p.status != 0) return;
-    if (warp == NCW) {
-        if (lane == 0) {
-            const uint64_t pol = l2_policy_evict_first();
-            RingPos rp = {0u, 0u, 0ull};
-            if (!produce_matrix(p, s, p.plan[PL_LM], p.wlm, cta, rp, pol)) drain_ring(p, s, rp);
-        }
-        return;
-    }
-    uint64_t nbase = 0;
+    const uint64_t pol = l2_policy_evict_first();
+    WarpRing wr = ring_begin(p, s, warp, 0);
+    ring_issue_next(p, s, wr, warp, lane, pol);
+    RingCursor rc = {0u, 0u};
     load_vec(p, s, p.x, p.H, true, p.gf, tid);
-    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, nbase);
+    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, rc, wr, pol);
+    ring_finish(p, s, wr, warp);
 }
 
-// Sampling block (greedy): lowest index among the maxima; then advance the position.
-__global__ void __launch_bounds__(1024) kl_argmax_kernel(const float* logits, uint32_t V, int32_t* tokens, int32_t* positions) {
-    __shared__ float sv[32];
-    __shared__ uint32_t si[32];
-    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+// Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per
+// sequence scan slices of the row; the last one to finish (ticket) reduces the partial results.
+constexpr int ARGMAX_BLOCKS = 64;
+
+__device__ __forceinline__ void argmax_merge(float& bv, uint32_t& bi, float ov, uint32_t oi) {
+    if (ov > bv || (ov == bv && oi < bi)) {
+        bv = ov;
+        bi = oi;
+    }
+}
+
+__global__ void __launch_bounds__(256) kl_argmax_kernel(const float* logits, uint32_t V, int32_t* tokens, int32_t* positions,
+                                                        float* part_val, uint32_t* part_idx, uint32_t* tickets) {
+    __shared__ float sv[8];
+    __shared__ uint32_t si[8];
+    __shared__ uint32_t last;
+    const uint32_t b = blockIdx.y, blk = blockIdx.x, tid = threadIdx.x;
     const float* row = logits + (size_t)b * V;
+    const uint32_t per = (V + ARGMAX_BLOCKS - 1) / ARGMAX_BLOCKS;
+    const uint32_t i0 = blk * per, i1 = min(V, i0 + per);
     float bv = -INFINITY;
     uint32_t bi = 0xffffffffu;
-    for (uint32_t i = tid; i < V; i += blockDim.x) {
-        const float v = row[i];
-        if (v > bv || (v == bv && i < bi)) {
-            bv = v;
-            bi = i;
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const uint32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (ov > bv || (ov == bv && oi < bi)) {
-            bv = ov;
-            bi = oi;
-        }
-    }
+    for (uint32_t i = i0 + tid; i < i1; i += blockDim.x) argmax_merge(bv, bi, row[i], i);
+    for (int o = 16; o > 0; o >>= 1)
+        argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
     if ((tid & 31) == 0) {
         sv[tid >> 5] = bv;
         si[tid >> 5] = bi;
     }
     __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w) argmax_merge(bv, bi, sv[w], si[w]);
+        part_val[b * ARGMAX_BLOCKS + blk] = bv;
+        part_idx[b * ARGMAX_BLOCKS + blk] = bi;
+        last = (atom_add_acq_rel(tickets + b, 1u) == ARGMAX_BLOCKS - 1) ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!last) return;
     if (tid < 32) {
-        const uint32_t nw = (blockDim.x + 31) / 32;
-        bv = tid < nw ? sv[tid] : -INFINITY;
-        bi = tid < nw ? si[tid] : 0xffffffffu;
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const uint32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) {
-                bv = ov;
-                bi = oi;
-            }
-        }
+        bv = -INFINITY;
+        bi = 0xffffffffu;
+        for (uint32_t j = tid; j < ARGMAX_BLOCKS; j += 32)
+            argmax_merge(bv, bi, __ldcg(part_val + b * ARGMAX_BLOCKS + j), __ldcg(part_idx + b * ARGMAX_BLOCKS + j));
+        for (int o = 16; o > 0; o >>= 1)
+            argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
         if (tid == 0) {
             tokens[b] = (int32_t)(bi == 0xffffffffu ? 0u : bi);
             positions[b] += 1;
+            tickets[b] = 0u;  // ready for the next call (calls on one handle do not overlap)
         }
     }
 }
@@ -220,10 +222,15 @@ struct kl_handle {
     int32_t* stage_tokens;
     int32_t* stage_positions;
     float* stage_logits;
+    float* argmax_val;
+    uint32_t* argmax_idx;
+    uint32_t* argmax_tickets;
     uint64_t launches;
     uint64_t loaded_layer_mask_count;  // number of (tensor, layer) pairs loaded
     uint8_t* loaded;                   // [12][L] flags (host)
     int pending_skip_stage;
+    int use_tc_attention;
+    void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no link against libcuda)
     // optional event recording around the decoder and classifier launches
     uint32_t prof_capacity;
     uint64_t prof_steps;
@@ -241,7 +248,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sx, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, scratch_bytes;
+    size_t sx, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, scratch_bytes;
     uint32_t cps;
 };
 
@@ -293,6 +300,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.stok = s;      s += align_up(B * 4);
     y.spos = s;      s += align_up(B * 4);
     y.slogits = s;   s += align_up(B * V * 4);
+    y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
     y.scratch_bytes = s;
     return y;
 }
@@ -397,6 +405,16 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->weight_bytes = y.weight_elems * 2;
     h->scratch_bytes = y.scratch_bytes;
     h->pending_skip_stage = -1;
+    h->use_tc_attention = 1;
+    {
+        cudaDriverEntryPointQueryResult qres;
+        void* fn = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            h->encode_tiled = fn;
+        else
+            h->use_tc_attention = 0;
+    }
     h->loaded = (uint8_t*)calloc(12 * (size_t)d.n_layers, 1);
     if (!h->loaded) { delete h; return KL_ERR_INVALID_ARG; }
 
@@ -409,6 +427,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.eps = d.rms_eps;
     p.skip_stage = -1;
     p.wait_ns = 2000000000ull;
+    p.prefetch_chunks = 0;
     p.layer_stride = y.layer_stride;
     p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P);
     p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P);
@@ -421,7 +440,8 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     uint32_t vecf = p.H > p.QD ? p.H : p.QD;
     if (p.F > vecf) vecf = p.F;
     vecf = ceil_div(vecf, 256) * 256;
-    const uint32_t attnf = p.G * p.hd + 2 * p.hd + NCW * p.G * (p.hd + 2);
+    // attention workspace: rotated q, the new K/V row, per-warp partial results, the staging tile of the new row
+    const uint32_t attnf = p.G * p.hd + 2 * p.hd + NCW * p.G * (p.hd + 2) + 16 * p.hd;
     if (attnf > vecf) vecf = ceil_div(attnf, 256) * 256;
     p.vec_floats = vecf;
     int max_optin = 0;
@@ -456,6 +476,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->stage_tokens = (int32_t*)(sc + y.stok);
     h->stage_positions = (int32_t*)(sc + y.spos);
     h->stage_logits = (float*)(sc + y.slogits);
+    h->argmax_val = (float*)(sc + y.samax);
+    h->argmax_idx = (uint32_t*)(h->argmax_val + (size_t)d.max_batch * ARGMAX_BLOCKS);
+    h->argmax_tickets = h->argmax_idx + (size_t)d.max_batch * ARGMAX_BLOCKS;
 
     if (cudaMemset(h->scratch, 0, h->scratch_bytes) != cudaSuccess) { free(h->loaded); delete h; return KL_ERR_CUDA; }
     double invf[128];
@@ -505,6 +528,28 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
     return KL_OK;
 }
 
+// The KV cache as a 2-D bf16 tensor [n_layers*2*batch*n_kv_heads*max_ctx rows, head_dim columns]; boxes of
+// [positions per chunk] x [64 columns] with the 128-byte swizzle.  Encoded per call because the cache is the caller's.
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch) {
+    if (!h->encode_tiled) return KL_ERR_CUDA;
+    if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
+    const kl_model_desc& d = h->desc;
+    const cuuint64_t rows = (cuuint64_t)d.n_layers * 2 * batch * d.n_kv_heads * d.max_ctx;
+    if (rows > 0x7fffffffull) return KL_ERR_UNSUPPORTED_SHAPE;  // box coordinates are 32-bit signed
+    const cuuint64_t gdim[2] = {d.head_dim, rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)d.head_dim * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)(SLOT_BYTES / (4 * d.head_dim))};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ((encode_tiled_fn)h->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_cache_d, gdim, gstride, box,
+                                                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                         CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? KL_OK : KL_ERR_CUDA;
+}
+
 static bool all_loaded(const kl_handle* h) {
     const uint32_t L = h->prm.L;
     for (int t = 0; t <= KL_LM_HEAD; ++t) {
@@ -551,6 +596,12 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     p.logits = logits_d;
     p.skip_stage = h->pending_skip_stage;
     h->pending_skip_stage = -1;
+    p.attn_tc = 0;
+    if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
+        const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, batch);
+        if (trc != KL_OK) return trc;
+        p.attn_tc = 1;
+    }
 
     kl_embed_kernel<<<batch, 256, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
@@ -570,6 +621,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         }
     }
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
+    p.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
     void* cargs[] = {&p};
     if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
     if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
@@ -594,7 +646,8 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
 kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d, uint32_t batch,
                             void* stream) {
     if (!h || !logits_d || !tokens_d || !positions_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
-    kl_argmax_kernel<<<batch, 1024, 0, as_stream(stream)>>>(logits_d, h->prm.V, tokens_d, positions_d);
+    kl_argmax_kernel<<<dim3(ARGMAX_BLOCKS, batch), 256, 0, as_stream(stream)>>>(logits_d, h->prm.V, tokens_d, positions_d,
+                                                                                 h->argmax_val, h->argmax_idx, h->argmax_tickets);
     if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
     ++h->launches;
     return KL_OK;
@@ -660,6 +713,30 @@ kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* c
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns) {
     if (!h || ns == 0) return KL_ERR_INVALID_ARG;
     h->prm.wait_ns = ns;
+    return KL_OK;
+}
+
+kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32_t* n_layers, uint32_t* n_stamps) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    h->prm.trace = reinterpret_cast<unsigned long long*>(trace_d);
+    // the per-chunk log of CTA 0 follows the stage stamps in the same buffer
+    h->prm.chunk_trace = trace_d ? h->prm.trace + (size_t)h->prm.P * h->prm.L * TRACE_STAMPS : nullptr;
+    if (n_ctas) *n_ctas = h->prm.P;
+    if (n_layers) *n_layers = h->prm.L;
+    if (n_stamps) *n_stamps = TRACE_STAMPS;
+    return KL_OK;
+}
+
+kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    if (on && !h->encode_tiled) return KL_ERR_CUDA;
+    h->use_tc_attention = on ? 1 : 0;
+    return KL_OK;
+}
+
+kl_status kl_set_prefetch_chunks(kl_handle* h, uint32_t chunks) {
+    if (!h || chunks > 64) return KL_ERR_INVALID_ARG;
+    h->prm.prefetch_chunks = chunks;
     return KL_OK;
 }
 
