@@ -146,10 +146,6 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
-/* Tuning knob: how many 16 KB chunks beyond its shared-memory ring each CTA's producer asks L2 to prefetch
- * (0..64, default 0 = off).  The look-ahead of all CTAs together must stay well inside L2. */
-kl_status kl_set_prefetch_chunks(kl_handle* h, uint32_t chunks);
-
 /* Limit, in nanoseconds, of every device-side wait (flag, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
 

@@ -52,8 +52,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots; ++i) mbar_init(smem_u32(&s.full[i]), 1);
-        make_decoder_plan(*s.plan, p, cta, l1);
+        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
         *s.abort_flag = 0;
         *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -63,10 +65,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     __syncthreads();
     if (*p.status != 0) return;  // an earlier kernel of this step flagged bad input: the step is a no-op
 
-    // every warp starts the copy of its first chunk, then follows the stages
-    const uint64_t pol = l2_policy_evict_first();
-    WarpRing wr = ring_begin(p, s, warp, l0);
-    ring_issue_next(p, s, wr, warp, lane, pol);
+    if (warp == NCW) {
+        // producer warp: one thread streams the CTA's chunk sequence into the ring
+        if (lane == 0) produce_decoder(p, s, cta, l0, l1);
+        return;
+    }
+    const uint64_t pol = 0;
+    WarpRing wr = ring_begin();
 
     // ---------------- consumers
     const uint32_t ctid = tid;
@@ -80,28 +85,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
         trace_stamp(p, cta, l, 0, ctid);
         load_vec(p, s, p.x, p.H, true, p.g1 + lo, ctid);
         trace_stamp(p, cta, l, 1, ctid);
-        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, rc, wr, pol);
+        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, rc, wr, nullptr);
         stage_signal(ctr + ST_QKV, ctid, skip == ST_QKV);
         trace_stamp(p, cta, l, 2, ctid);
         // S2: RoPE, KV append, split-K attention, merge
         stage_wait(p, s, ctr + ST_QKV, p.P, ctid);
         trace_stamp(p, cta, l, 3, ctid);
+        uint32_t aw;
         if (p.attn_tc) {
-            attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr, pol);
+            aw = attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
         } else switch (p.G) {
-            case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
-            case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
-            case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
-            default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr, pol); break;
+            case 1: aw = attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            case 2: aw = attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            case 4: aw = attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            default: aw = attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
         }
-        stage_signal(ctr + ST_ATTN, ctid, skip == ST_ATTN);
+        stage_signal(ctr + ST_ATTN, ctid, skip == ST_ATTN, aw);
+        attention_flush_new_row(p, s, l, cta, ctid);
         trace_stamp(p, cta, l, 4, ctid);
         // S3: output projection + residual
         stage_wait(p, s, ctr + ST_ATTN, p.P, ctid);
         trace_stamp(p, cta, l, 5, ctid);
         load_vec(p, s, p.o, p.QD, false, nullptr, ctid);
         trace_stamp(p, cta, l, 6, ctid);
-        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, pol);
+        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, nullptr);
         stage_signal(ctr + ST_O, ctid, skip == ST_O);
         trace_stamp(p, cta, l, 7, ctid);
         // S4: RMSNorm + gate/up projections + SwiGLU
@@ -109,19 +116,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
         trace_stamp(p, cta, l, 8, ctid);
         load_vec(p, s, p.x, p.H, true, p.g2 + lo, ctid);
         trace_stamp(p, cta, l, 9, ctid);
-        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, rc, wr, pol);
+        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, rc, wr, nullptr);
         stage_signal(ctr + ST_GU, ctid, skip == ST_GU);
         trace_stamp(p, cta, l, 10, ctid);
         // S5: down projection + residual
         stage_wait(p, s, ctr + ST_GU, p.P, ctid);
         trace_stamp(p, cta, l, 11, ctid);
-        load_vec(p, s, p.h, p.F, false, nullptr, ctid);
         trace_stamp(p, cta, l, 12, ctid);
-        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, pol);
+        // h is read per warp and per column piece straight from L2 into registers (no shared-memory staging)
+        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, p.h);
         stage_signal(ctr + ST_D, ctid, skip == ST_D);
         trace_stamp(p, cta, l, 13, ctid);
     }
-    ring_finish(p, s, wr, warp);
 }
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
@@ -130,8 +136,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots; ++i) mbar_init(smem_u32(&s.full[i]), 1);
-        make_classifier_plan(*s.plan, p, cta);
+        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
         *s.abort_flag = 0;
         *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -140,13 +148,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
     __syncthreads();
     if (*p.status != 0) return;
-    const uint64_t pol = l2_policy_evict_first();
-    WarpRing wr = ring_begin(p, s, warp, 0);
-    ring_issue_next(p, s, wr, warp, lane, pol);
+    if (warp == NCW) {
+        if (lane == 0) produce_classifier(p, s, cta);
+        return;
+    }
+    const uint64_t pol = 0;
+    WarpRing wr = ring_begin();
     RingCursor rc = {0u, 0u};
     load_vec(p, s, p.x, p.H, true, p.gf, tid);
-    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, rc, wr, pol);
-    ring_finish(p, s, wr, warp);
+    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, rc, wr, nullptr);
 }
 
 // Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per
@@ -305,44 +315,93 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     return y;
 }
 
-GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P) {
+// `align`: units must not straddle multiples of `align` rows (sources that are concatenated row-wise, such as
+// Wq | Wk | Wv, start at multiples of it); 0 = no constraint.
+GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t align) {
     GemvPlan pl;
     memset(&pl, 0, sizeof(pl));
     pl.R = R;
     pl.K = K;
     const uint32_t rowbytes = K * 2;
     const uint32_t minrows = pairs ? 2u : 1u;
-    if (rowbytes * minrows <= (uint32_t)SLOT_BYTES) {
+    if (K <= MAX_KP && rowbytes * minrows <= (uint32_t)SLOT_BYTES) {
+        // whole rows: as many as fit a slot, but keep at least ~2 chunks per CTA on small matrices
         uint32_t rpc = SLOT_BYTES / rowbytes;
-        uint32_t cap = R / (2 * P);  // keep at least ~2 chunks per CTA on small matrices
+        uint32_t cap = R / (2 * P);
         if (cap < minrows) cap = minrows;
         if (rpc > cap) rpc = cap;
         if (pairs) rpc &= ~1u;
+        while (align && rpc > 1 && align % rpc) --rpc;
         pl.rpc = rpc;
-        pl.ksplit = 1;
-        pl.klen = K;
-        pl.rows_per_unit = rpc;
-        pl.nunits = ceil_div(R, rpc);
-        pl.chunks_per_unit = 1;
+        pl.kp = K;
+        pl.npieces = 1;
     } else {
-        pl.rpc = 0;
-        uint32_t ksplit = ceil_div(rowbytes, SLOT_BYTES);
-        pl.klen = ceil_div(ceil_div(K, ksplit), 256) * 256;
-        pl.ksplit = ceil_div(K, pl.klen);
-        pl.rows_per_unit = minrows;
-        pl.nunits = R / minrows;
-        pl.chunks_per_unit = pl.rows_per_unit * pl.ksplit;
+        // units cut into column pieces.  A piece count that divides the consumer count (or is a multiple of it)
+        // keeps every consumer on the same column piece for a whole stage, so its share of the input vector
+        // stays in registers.
+        const uint32_t kp_max = MAX_KP / 256u * 256u;
+        uint32_t np = ceil_div(K, kp_max);
+        const uint32_t cand[5] = {1, 2, 3, NCW, 2 * NCW};
+        for (int q = 0; q < 5; ++q)
+            if (cand[q] >= np) { np = cand[q]; break; }
+        pl.kp = ceil_div(ceil_div(K, np), 256) * 256;
+        pl.npieces = ceil_div(K, pl.kp);
+        uint32_t rpc = SLOT_BYTES / (pl.kp * 2);
+        if (rpc > (uint32_t)MAX_RPC_SPLIT) rpc = MAX_RPC_SPLIT;
+        if (pairs) rpc = 2;
+        while (align && rpc > 1 && align % rpc) --rpc;
+        if (rpc < 1) rpc = 1;
+        pl.rpc = rpc;
     }
+    pl.nunits = ceil_div(R, pl.rpc);
     return pl;
 }
 
 bool plans_ok(const Params& p) {
     for (int i = 0; i < PL_COUNT; ++i) {
         const GemvPlan& pl = p.plan[i];
-        if (pl.rpc == 0 && (pl.chunks_per_unit > (uint32_t)MAX_PIECES || pl.klen * 2 > (uint32_t)SLOT_BYTES)) return false;
-        if (pl.rpc != 0 && pl.rpc * pl.K * 2 > (uint32_t)SLOT_BYTES) return false;
+        if (pl.npieces > (uint32_t)MAX_PIECES || pl.kp > MAX_KP || pl.rpc < 1) return false;
+        if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
+        if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % 256)) return false;
+        if (i == PL_GU && (pl.rpc & 1u)) return false;
+        if (i == PL_GU && pl.npieces > 1 && pl.rpc != 2) return false;
     }
     return true;
+}
+
+// Writes `rows` source rows (row-major [rows, K]) into the library's copy of a matrix in chunk order (see GemvPlan):
+// source row s becomes row v0 + s * vstep of the matrix.  vstep = 1 with v0 a multiple of the unit size, or
+// vstep = 2 (gate / up rows interleaved) with units of two rows.
+cudaError_t store_rows(const GemvPlan& pl, __nv_bfloat16* mat, const __nv_bfloat16* src, size_t rows, uint32_t v0,
+                       uint32_t vstep, cudaStream_t st) {
+    const size_t K = pl.K;
+    cudaError_t e = cudaSuccess;
+    if (pl.npieces == 1) {
+        // plain row-major
+        if (vstep == 1) return cudaMemcpyAsync(mat + (size_t)v0 * K, src, rows * K * 2, cudaMemcpyDefault, st);
+        return cudaMemcpy2DAsync(mat + (size_t)v0 * K, vstep * K * 2, src, K * 2, K * 2, rows, cudaMemcpyDefault, st);
+    }
+    const size_t rpc = pl.rpc;
+    for (uint32_t j = 0; j < pl.npieces && e == cudaSuccess; ++j) {
+        const size_t c0 = (size_t)j * pl.kp;
+        const size_t len = (j == pl.npieces - 1) ? K - c0 : pl.kp;
+        if (vstep == 2) {
+            // units of two rows (gate f, up f): this tensor fills row v0 of every unit
+            e = cudaMemcpy2DAsync(mat + rpc * c0 + (size_t)v0 * len, rpc * K * 2, src + c0, K * 2, len * 2, rows,
+                                  cudaMemcpyDefault, st);
+            continue;
+        }
+        const size_t u_first = v0 / rpc;
+        const size_t full = rows / rpc;           // whole units covered by this tensor
+        for (size_t rr = 0; rr < rpc && e == cudaSuccess && full > 0; ++rr)
+            e = cudaMemcpy2DAsync(mat + u_first * rpc * K + rpc * c0 + rr * len, rpc * K * 2, src + rr * K + c0, rpc * K * 2,
+                                  len * 2, full, cudaMemcpyDefault, st);
+        const size_t rest = rows - full * rpc;    // rows of a last, short unit (end of the matrix)
+        for (size_t rr = 0; rr < rest && e == cudaSuccess; ++rr)
+            e = cudaMemcpyAsync(mat + (u_first + full) * rpc * K + rest * c0 + rr * len, src + (full * rpc + rr) * K + c0,
+                                len * 2, cudaMemcpyDefault, st);
+    }
+    return e;
 }
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
@@ -427,21 +486,19 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.eps = d.rms_eps;
     p.skip_stage = -1;
     p.wait_ns = 2000000000ull;
-    p.prefetch_chunks = 0;
     p.layer_stride = y.layer_stride;
-    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P);
-    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P);
-    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P);
-    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P);
-    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P);
+    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD);  // KVD divides QD: Wq | Wk | Wv stay aligned
+    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P, 0);
+    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P, 0);
+    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0);
+    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0);
     if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
 
     // shared memory: input vector area (also the attention workspace), then as many ring slots as fit
-    uint32_t vecf = p.H > p.QD ? p.H : p.QD;
-    if (p.F > vecf) vecf = p.F;
+    uint32_t vecf = p.H > p.QD ? p.H : p.QD;  // the down projection reads its input from L2, not from this area
     vecf = ceil_div(vecf, 256) * 256;
     // attention workspace: rotated q, the new K/V row, per-warp partial results, the staging tile of the new row
-    const uint32_t attnf = p.G * p.hd + 2 * p.hd + NCW * p.G * (p.hd + 2) + 16 * p.hd;
+    const uint32_t attnf = p.G * p.hd + 2 * p.hd + 128 + NCW * p.G * (p.hd + 2);
     if (attnf > vecf) vecf = ceil_div(attnf, 256) * 256;
     p.vec_floats = vecf;
     int max_optin = 0;
@@ -449,11 +506,12 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
         free(h->loaded); delete h; return KL_ERR_CUDA;
     }
     const long avail = (long)max_optin - (long)vecf * 4 - SMEM_MISC_BYTES;
-    long nslots = avail / SLOT_BYTES;
-    if (nslots > MAX_SLOTS) nslots = MAX_SLOTS;
-    if (nslots < 3) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
-    p.nslots = (uint32_t)nslots;
-    h->smem_bytes = (size_t)nslots * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
+    long nsw = avail / ((long)NCW * SLOT_BYTES);
+    if (nsw > MAX_NSW) nsw = MAX_NSW;
+    if (nsw < 1) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    p.nslots = NCW;
+    p.nsw = (uint32_t)nsw;
+    h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
     if (cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess ||
         cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess) {
         free(h->loaded); delete h; return KL_ERR_CUDA;
@@ -499,30 +557,29 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
     if (global_t ? (layer != -1) : (layer < 0 || layer >= (int)p.L)) return KL_ERR_INVALID_ARG;
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(h->weights);
     const size_t lo = global_t ? 0 : (size_t)layer * y.layer_stride;
-    size_t rows = 0, cols = 0, dst = 0, dpitch_elems = 0;
+    size_t rows = 0, cols = 0, dst = 0;
+    const GemvPlan* pl = nullptr;   // matrices streamed through the ring are stored in chunk order
+    uint32_t v0 = 0, vstep = 1;
     switch (tensor) {
         case KL_EMBED: rows = p.V; cols = p.H; dst = y.off_embed; break;
-        case KL_LM_HEAD: rows = p.V; cols = p.H; dst = y.off_lm; break;
+        case KL_LM_HEAD: rows = p.V; cols = p.H; dst = y.off_lm; pl = &p.plan[PL_LM]; break;
         case KL_NORM_F: rows = 1; cols = p.H; dst = y.off_gf; break;
-        case KL_WQ: rows = p.QD; cols = p.H; dst = lo + y.off_qkv; break;
-        case KL_WK: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv + (size_t)p.QD * p.H; break;
-        case KL_WV: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv + (size_t)(p.QD + p.KVD) * p.H; break;
-        case KL_WO: rows = p.H; cols = p.QD; dst = lo + y.off_o; break;
-        case KL_WGATE: rows = p.F; cols = p.H; dst = lo + y.off_gu; dpitch_elems = 2 * (size_t)p.H; break;
-        case KL_WUP: rows = p.F; cols = p.H; dst = lo + y.off_gu + p.H; dpitch_elems = 2 * (size_t)p.H; break;
-        case KL_WDOWN: rows = p.H; cols = p.F; dst = lo + y.off_d; break;
+        case KL_WQ: rows = p.QD; cols = p.H; dst = lo + y.off_qkv; pl = &p.plan[PL_QKV]; break;
+        case KL_WK: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv; pl = &p.plan[PL_QKV]; v0 = p.QD; break;
+        case KL_WV: rows = p.KVD; cols = p.H; dst = lo + y.off_qkv; pl = &p.plan[PL_QKV]; v0 = p.QD + p.KVD; break;
+        case KL_WO: rows = p.H; cols = p.QD; dst = lo + y.off_o; pl = &p.plan[PL_O]; break;
+        // gate and up rows are interleaved (row 2f = gate f, row 2f+1 = up f) so one chunk holds both halves of a pair
+        case KL_WGATE: rows = p.F; cols = p.H; dst = lo + y.off_gu; pl = &p.plan[PL_GU]; v0 = 0; vstep = 2; break;
+        case KL_WUP: rows = p.F; cols = p.H; dst = lo + y.off_gu; pl = &p.plan[PL_GU]; v0 = 1; vstep = 2; break;
+        case KL_WDOWN: rows = p.H; cols = p.F; dst = lo + y.off_d; pl = &p.plan[PL_D]; break;
         case KL_NORM1: rows = 1; cols = p.H; dst = lo + y.off_g1; break;
         case KL_NORM2: rows = 1; cols = p.H; dst = lo + y.off_g2; break;
         default: return KL_ERR_INVALID_ARG;
     }
     if (bytes != rows * cols * 2) return KL_ERR_INVALID_ARG;
     cudaError_t e;
-    if (dpitch_elems) {
-        // gate and up rows are interleaved (row 2f = gate f, row 2f+1 = up f) so one chunk holds both halves of a pair
-        e = cudaMemcpy2DAsync(w + dst, dpitch_elems * 2, src, cols * 2, cols * 2, rows, cudaMemcpyDefault, as_stream(stream));
-    } else {
-        e = cudaMemcpyAsync(w + dst, src, bytes, cudaMemcpyDefault, as_stream(stream));
-    }
+    if (pl) e = store_rows(*pl, w + dst, reinterpret_cast<const __nv_bfloat16*>(src), rows, v0, vstep, as_stream(stream));
+    else e = cudaMemcpyAsync(w + dst, src, bytes, cudaMemcpyDefault, as_stream(stream));
     if (e != cudaSuccess) return KL_ERR_CUDA;
     h->loaded[(size_t)tensor * p.L + (global_t ? 0 : layer)] = 1;
     return KL_OK;
@@ -731,12 +788,6 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
     if (on && !h->encode_tiled) return KL_ERR_CUDA;
     h->use_tc_attention = on ? 1 : 0;
-    return KL_OK;
-}
-
-kl_status kl_set_prefetch_chunks(kl_handle* h, uint32_t chunks) {
-    if (!h || chunks > 64) return KL_ERR_INVALID_ARG;
-    h->prm.prefetch_chunks = chunks;
     return KL_OK;
 }
 

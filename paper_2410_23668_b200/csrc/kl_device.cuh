@@ -10,17 +10,19 @@
 
 namespace kl {
 
-constexpr int NCW = 8;                     // warps per CTA (two per scheduler, 255 registers each); warp w owns ring
-                                           // slot w and keeps it filled itself
-constexpr int NCT = NCW * 32;              // threads that take part in the CTA-wide steps (all of them)
-constexpr int NTHREADS = NCT;
-constexpr int SLOT_BYTES = 16384;          // one ring slot = one TMA bulk copy
-constexpr int MAX_SLOTS = NCW;             // one owner warp per slot (see WarpRing)
-constexpr int MAX_PIECES = 8;              // chunks per unit when a unit spans several chunks
-constexpr int UNIT_SLOTS = 32;             // in-flight multi-chunk units tracked per CTA
+constexpr int NCW = 6;                     // consumer warps per CTA; consumer c takes chunks c, c + NCW, ... and so
+                                           // always meets the same nsw ring slots, in order
+constexpr int NCT = NCW * 32;              // consumer threads (they take part in the CTA-wide steps)
+constexpr int NTHREADS = NCT + 32;         // + the producer warp (the last warp; 7 warps leave 255 registers each)
+constexpr int SLOT_BYTES = 16384;          // one ring slot = one chunk (one or two TMA copies)
+constexpr int MAX_NSW = 4;                 // ring slots per consumer warp
+constexpr int MAX_SLOTS = NCW * MAX_NSW;
+constexpr int MAX_PIECES = 16;             // chunks per unit when a unit spans several chunks
+constexpr int UNIT_SLOTS = 16;             // in-flight multi-chunk units tracked per CTA
+constexpr int MAX_RPC_SPLIT = 4;           // rows per unit when units are split into column pieces
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
 constexpr int MAX_G = 8;                   // query heads per KV head
-constexpr int SMEM_MISC_BYTES = 4096;
+constexpr int SMEM_MISC_BYTES = 8192;  // barriers, chunk-sequence plan, reduction scratch, unit table (see carve_smem)
 
 enum StageId { ST_QKV = 0, ST_ATTN = 1, ST_O = 2, ST_GU = 3, ST_D = 4, ST_LM = 5 };
 enum EpilogueKind { EP_STORE = 0, EP_RESIDUAL = 1, EP_SWIGLU = 2 };
@@ -29,30 +31,32 @@ enum PlanId { PL_QKV = 0, PL_O = 1, PL_GU = 2, PL_D = 3, PL_LM = 4, PL_COUNT = 5
 constexpr int ERR_SYNC_TIMEOUT = -5;
 constexpr int ERR_OUT_OF_RANGE = -6;
 
-// How one matrix [R, K] (bf16, row-major, rows contiguous) is cut into ring chunks and units.
-//  rpc > 0 : a chunk holds rpc whole rows (the last chunk of the matrix may hold fewer); unit == chunk.
-//  rpc == 0: a chunk is one piece (klen elements, the last piece of a row may be shorter) of one row; a unit is
-//            rows_per_unit consecutive rows = rows_per_unit * ksplit consecutive chunks.
-// Units are dealt to CTAs in contiguous ranges, so each CTA's share of a matrix is one linear byte range.
+// How one matrix [R, K] (bf16) is cut into ring chunks.  Rows are grouped into units of `rpc` consecutive rows,
+// dealt to the CTAs in contiguous ranges.  A unit is streamed as `npieces` chunks; chunk j holds columns
+// [j*kp, min(K, (j+1)*kp)) of the unit's rows, row after row.  kp <= MAX_KP so that a lane keeps its share of the
+// matching slice of the input vector in registers for the whole stage, and rpc * kp * 2 <= SLOT_BYTES.
+// The library's copy of the matrix is stored in exactly this order -- unit, then piece, then row, then column --
+// so every chunk, and in fact the whole share of a CTA, is one linear run of bytes ("grouped tensors laid out
+// linearly in memory", Section 3.2).  With npieces == 1 this is plain row-major.
 struct GemvPlan {
     uint32_t R, K;
     uint32_t rpc;
-    uint32_t ksplit;
-    uint32_t klen;
-    uint32_t rows_per_unit;
+    uint32_t kp;
+    uint32_t npieces;
     uint32_t nunits;
-    uint32_t chunks_per_unit;
 };
+constexpr uint32_t MAX_KP = 4096;           // columns per chunk piece: 16 blocks of 256, 8 per lane and block
+constexpr int MAX_XB = MAX_KP / 256;
 
 struct Params {
     CUtensorMap kv_map;    // the whole KV cache as a 2-D tensor [rows, head_dim], 128-byte swizzle (64-byte aligned)
     uint32_t attn_tc;      // 1: tensor-core attention loop fed by kv_map boxes; 0: CUDA-core loop fed by linear copies
     uint32_t L, H, nq, nkv, hd, F, V, G, QD, KVD, max_ctx, B;
     uint32_t P;            // CTAs in the persistent grid
-    uint32_t nslots;       // ring slots
+    uint32_t nslots;       // ways of the ring = consumer warps (chunk n belongs to consumer n % nslots)
+    uint32_t nsw;          // slots per consumer (chunk n sits in slot (n % nslots) * nsw + (n / nslots) % nsw)
     uint32_t vec_floats;   // capacity of the shared input-vector area
     uint32_t cps;          // attention: CTA slots per (sequence, kv head)
-    uint32_t prefetch_chunks;  // L2 look-ahead of the producer beyond the ring, in chunks (0 = off)
     float eps;
     int32_t skip_stage;    // test hook: stage of layer 0 whose end is not signalled (-1 = none)
     uint64_t wait_ns;
@@ -154,8 +158,8 @@ __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 
 struct Smem {
     uint8_t* ring;          // nslots * SLOT_BYTES
     float* vec;             // input vector of the current GEMV stage (lane-permuted), or attention workspace
-    uint64_t* full;         // [MAX_SLOTS]
-    struct SeqPlan* plan;   // this CTA's chunk sequence (written once by thread 0)
+    uint64_t* full;         // [MAX_SLOTS] copy landed
+    uint64_t* empty;        // [MAX_SLOTS] consumer has finished reading
     float* red;             // [NCW]
     float* unit_part;       // [UNIT_SLOTS][MAX_PIECES]
     int* unit_cnt;          // [UNIT_SLOTS]
@@ -166,13 +170,13 @@ struct Smem {
 __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
     Smem s;
     s.ring = base;
-    s.vec = reinterpret_cast<float*>(base + (size_t)p.nslots * SLOT_BYTES);
+    s.vec = reinterpret_cast<float*>(base + (size_t)p.nslots * p.nsw * SLOT_BYTES);
     uint8_t* misc = reinterpret_cast<uint8_t*>(s.vec) + (size_t)p.vec_floats * 4;
-    s.full = reinterpret_cast<uint64_t*>(misc);
-    s.plan = reinterpret_cast<struct SeqPlan*>(misc + 128);
-    s.red = reinterpret_cast<float*>(misc + 1024);
-    s.unit_part = s.red + 32;
-    s.unit_cnt = reinterpret_cast<int*>(s.unit_part + UNIT_SLOTS * MAX_PIECES);
+    s.full = reinterpret_cast<uint64_t*>(misc);                    // [MAX_SLOTS] 192 B
+    s.empty = reinterpret_cast<uint64_t*>(misc + 256);             // [MAX_SLOTS]
+    s.red = reinterpret_cast<float*>(misc + 1536);                 // 128 B
+    s.unit_part = reinterpret_cast<float*>(misc + 2048);           // [UNIT_SLOTS][MAX_PIECES][MAX_RPC_SPLIT] 4 KB
+    s.unit_cnt = reinterpret_cast<int*>(misc + 6144);              // [UNIT_SLOTS]
     s.abort_flag = s.unit_cnt + UNIT_SLOTS;
     s.bcast = s.abort_flag + 1;
     return s;
@@ -217,34 +221,26 @@ __device__ __forceinline__ CtaRange cta_units(const GemvPlan& pl, uint32_t cta, 
 }
 
 struct ChunkGeom {
-    uint64_t elem_off;  // offset of the chunk inside the matrix, elements
-    uint32_t elems;     // elements in the chunk
-    uint32_t row;       // first row
-    uint32_t nrows;     // whole rows held (rpc > 0) or 1
-    uint32_t kofs;      // first column (piece chunks)
-    uint32_t piece;     // index of the chunk inside its unit
     uint32_t unit;      // unit index (matrix-wide)
+    uint32_t piece;     // column piece
+    uint32_t row;       // first row of the unit
+    uint32_t nrows;     // rows in the chunk
+    uint32_t kofs;      // first column
+    uint32_t klen;      // columns (row pitch inside the slot = klen * 2 bytes)
 };
 __device__ __forceinline__ ChunkGeom chunk_geom(const GemvPlan& pl, uint32_t u0, uint32_t i) {
     ChunkGeom g;
-    if (pl.rpc) {
+    if (pl.npieces == 1) {
         g.unit = u0 + i;
         g.piece = 0;
-        g.row = g.unit * pl.rpc;
-        g.nrows = min(pl.rpc, pl.R - g.row);
-        g.kofs = 0;
-        g.elem_off = (uint64_t)g.row * pl.K;
-        g.elems = g.nrows * pl.K;
     } else {
-        g.unit = u0 + i / pl.chunks_per_unit;
-        g.piece = i % pl.chunks_per_unit;
-        const uint32_t rr = g.piece / pl.ksplit, j = g.piece % pl.ksplit;
-        g.row = g.unit * pl.rows_per_unit + rr;
-        g.nrows = 1;
-        g.kofs = j * pl.klen;
-        g.elems = min(pl.klen, pl.K - g.kofs);
-        g.elem_off = (uint64_t)g.row * pl.K + g.kofs;
+        g.unit = u0 + i / pl.npieces;
+        g.piece = i % pl.npieces;
     }
+    g.row = g.unit * pl.rpc;
+    g.nrows = min(pl.rpc, pl.R - g.row);
+    g.kofs = g.piece * pl.kp;
+    g.klen = min(pl.kp, pl.K - g.kofs);
     return g;
 }
 
@@ -288,35 +284,6 @@ __device__ __forceinline__ const __nv_bfloat16* kv_head(const Params& p, uint32_
 
 // ------------------------------------------------------------------------------------------------ chunk streams
 
-// This CTA's share of one matrix: a run of contiguous chunks.
-struct StageStream {
-    uint64_t byte_off;    // offset of the first chunk inside the matrix
-    uint32_t nch;         // chunks
-    uint32_t bytes_a;     // size of a regular chunk
-    uint32_t bytes_b;     // size of every period-th chunk (the last piece of a row); == bytes_a for whole-row chunks
-    uint32_t period;
-    uint32_t bytes_last;  // size of the final chunk of the share (ragged tail of the matrix)
-};
-__device__ __forceinline__ StageStream make_stream(const GemvPlan& pl, uint32_t cta, uint32_t P) {
-    const CtaRange r = cta_units(pl, cta, P);
-    StageStream st;
-    if (pl.rpc) {
-        st.byte_off = (uint64_t)r.u0 * pl.rpc * pl.K * 2u;
-        st.nch = r.u1 - r.u0;
-        st.bytes_a = st.bytes_b = pl.rpc * pl.K * 2u;
-        st.period = 1;
-        st.bytes_last = (r.u1 == pl.nunits) ? (pl.R - (pl.nunits - 1) * pl.rpc) * pl.K * 2u : st.bytes_a;
-    } else {
-        st.byte_off = (uint64_t)r.u0 * pl.rows_per_unit * pl.K * 2u;
-        st.nch = (r.u1 - r.u0) * pl.chunks_per_unit;
-        st.bytes_a = pl.klen * 2u;
-        st.bytes_b = (pl.K - (pl.ksplit - 1) * pl.klen) * 2u;
-        st.period = pl.ksplit;
-        st.bytes_last = st.bytes_b;
-    }
-    return st;
-}
-
 __device__ __forceinline__ void tma_tensor_2d_g2s(uint32_t dst, const void* tmap, int32_t x, int32_t y, uint32_t bar,
                                                   uint64_t pol) {
     asm volatile(
@@ -343,255 +310,185 @@ __device__ __forceinline__ AttnWindow attn_window(uint32_t c0, uint32_t cend, ui
     return w;
 }
 
-// ------------------------------------------------------------------------------------------------ chunk sequence
+// ------------------------------------------------------------------------------------------------ the ring
 //
-// The whole launch as one sequence of 16 KB chunks per CTA, in consumption order: for every layer the CTA's QKV
-// rows, the K/V rows of its attention unit, its O rows, gate/up rows and down rows.  Every address is known when
-// the kernel starts (weights are grouped per layer and linear in memory; cached K/V rows were written by earlier
-// launches).  Chunk n lives in ring slot n % nslots, and warp (n % nslots) both consumes it and, the moment it has
-// read the slot for the last time, starts the TMA copy of chunk n + nslots into the same slot.  So each warp runs
-// its own pipeline through its own slot: there is no producer thread to serialise the issue, every parity wait is
-// made by the one warp that armed the barrier, and the copies for the next stage -- or, in the looped kernel, the
-// next layer -- are in flight while the warp sits in the counter wait that replaces a kernel boundary.
-struct SeqPlan {
-    StageStream st[4];         // QKV, O, GU, D  (for the classifier kernel: st[0] only)
-    const uint8_t* base[4];    // layer-0 base of each matrix
-    uint64_t layer_bytes;      // bytes between layers of a matrix
-    uint32_t cnt[5];           // chunks per stage: QKV, attention, O, GU, D
-    uint32_t per_layer;        // sum of cnt
-    // attention unit (one slot holds K rows in its first half, V rows of the same positions in its second half)
-    uint32_t attn_len, pb, row_bytes;
-    const uint8_t* k0;         // layer-0 K rows of the unit's first position
-    const uint8_t* v0;
-    uint64_t kv_layer_bytes;
-    // tensor-core attention: the same rows addressed as rows of the 2-D cache tensor
-    uint32_t tc, c0, cend;
-    uint32_t k_row0;           // tensor row of position 0 of the unit's (sequence, kv head), K half, layer 0
-    uint32_t v_row_delta;      // rows from a K row to the matching V row
-    uint32_t rows_per_layer;
-    uint32_t l1;
-};
+// The whole launch is one sequence of chunks per CTA, in consumption order: for every layer the CTA's QKV rows, the
+// K/V rows of its attention unit, its O rows, gate/up rows and down rows.  Every address is known when the kernel
+// starts (weights are grouped per layer and linear in memory; cached K/V rows were written by earlier launches),
+// so the producer thread runs ahead of the consumers across stage boundaries and, in the looped kernel, across
+// layer boundaries: while the consumers sit in the counter wait that replaces a kernel boundary, the copies of the
+// next stage's (next layer's) chunks are already in flight.
+//
+// Chunk n goes to consumer n % nslots, into that consumer's slot (n / nslots) % nsw.  Each slot therefore sees its
+// uses in order on both sides, and every parity wait is made by the one warp that will read the data (a fast warp
+// can never test a barrier two phases behind).
 
-__device__ __forceinline__ void make_decoder_plan(SeqPlan& q, const Params& p, uint32_t cta, uint32_t l1) {
-    q.st[0] = make_stream(p.plan[PL_QKV], cta, p.P);
-    q.st[1] = make_stream(p.plan[PL_O], cta, p.P);
-    q.st[2] = make_stream(p.plan[PL_GU], cta, p.P);
-    q.st[3] = make_stream(p.plan[PL_D], cta, p.P);
-    q.base[0] = reinterpret_cast<const uint8_t*>(p.wqkv);
-    q.base[1] = reinterpret_cast<const uint8_t*>(p.wo);
-    q.base[2] = reinterpret_cast<const uint8_t*>(p.wgu);
-    q.base[3] = reinterpret_cast<const uint8_t*>(p.wd);
-    q.layer_bytes = p.layer_stride * 2ull;
-    const AttnUnit u = attn_unit(p, cta);
-    q.attn_len = u.active ? u.cend - u.c0 : 0u;
-    q.pb = attn_positions_per_chunk(p);
-    q.row_bytes = p.hd * 2u;
-    q.k0 = q.v0 = nullptr;
-    if (u.active) {
-        q.k0 = reinterpret_cast<const uint8_t*>(kv_head(p, 0, 0, u.b, u.g)) + (size_t)u.c0 * q.row_bytes;
-        q.v0 = reinterpret_cast<const uint8_t*>(kv_head(p, 0, 1, u.b, u.g)) + (size_t)u.c0 * q.row_bytes;
-    }
-    q.kv_layer_bytes = 2ull * p.B * p.nkv * p.max_ctx * p.hd * 2ull;
-    q.tc = p.attn_tc;
-    q.c0 = u.active ? u.c0 : 0u;
-    q.cend = u.active ? u.cend : 0u;
-    q.k_row0 = u.active ? (u.b * p.nkv + u.g) * p.max_ctx : 0u;
-    q.v_row_delta = p.B * p.nkv * p.max_ctx;
-    q.rows_per_layer = 2u * q.v_row_delta;
-    q.cnt[0] = q.st[0].nch;
-    q.cnt[1] = u.nring;
-    q.cnt[2] = q.st[1].nch;
-    q.cnt[3] = q.st[2].nch;
-    q.cnt[4] = q.st[3].nch;
-    q.per_layer = q.cnt[0] + q.cnt[1] + q.cnt[2] + q.cnt[3] + q.cnt[4];
-    q.l1 = l1;
-}
-__device__ __forceinline__ void make_classifier_plan(SeqPlan& q, const Params& p, uint32_t cta) {
-    q.st[0] = make_stream(p.plan[PL_LM], cta, p.P);
-    q.st[1] = q.st[2] = q.st[3] = q.st[0];
-    q.base[0] = q.base[1] = q.base[2] = q.base[3] = reinterpret_cast<const uint8_t*>(p.wlm);
-    q.layer_bytes = 0;
-    q.attn_len = 0;
-    q.pb = 1;
-    q.row_bytes = 0;
-    q.k0 = q.v0 = nullptr;
-    q.kv_layer_bytes = 0;
-    q.tc = q.c0 = q.cend = q.k_row0 = q.v_row_delta = q.rows_per_layer = 0;
-    q.cnt[0] = q.st[0].nch;
-    q.cnt[1] = q.cnt[2] = q.cnt[3] = q.cnt[4] = 0;
-    q.per_layer = q.cnt[0];
-    q.l1 = 1;
-}
-
-struct SeqPos {
-    uint32_t l, stage, i;   // stage: 0 QKV, 1 attention, 2 O, 3 GU, 4 D; i = chunk index inside the stage
-    bool done;
-};
-__device__ __forceinline__ void seq_normalize(const SeqPlan& q, SeqPos& r) {
-    if (q.per_layer == 0) {
-        r.done = true;
-        return;
-    }
-    while (r.i >= q.cnt[r.stage]) {
-        r.i -= q.cnt[r.stage];
-        if (++r.stage == 5) {
-            r.stage = 0;
-            if (++r.l >= q.l1) {
-                r.done = true;
-                return;
-            }
-        }
-    }
-}
-struct ChunkSrc {
-    const uint8_t* src0;
-    const uint8_t* src1;
-    uint32_t bytes0, bytes1;
-};
-__device__ __forceinline__ ChunkSrc seq_chunk(const SeqPlan& q, const SeqPos& r) {
-    ChunkSrc c;
-    c.src1 = nullptr;
-    c.bytes1 = 0;
-    if (r.stage == 1) {
-        const uint32_t t = r.i * q.pb;
-        const uint32_t np = min(q.pb, q.attn_len - t);
-        c.bytes0 = c.bytes1 = np * q.row_bytes;
-        c.src0 = q.k0 + (size_t)r.l * q.kv_layer_bytes + (size_t)t * q.row_bytes;
-        c.src1 = q.v0 + (size_t)r.l * q.kv_layer_bytes + (size_t)t * q.row_bytes;
-    } else {
-        const uint32_t m = r.stage == 0 ? 0u : r.stage - 1u;
-        const StageStream& st = q.st[m];
-        uint64_t off;
-        if (st.period == 1) {
-            off = (uint64_t)r.i * st.bytes_a;
-            c.bytes0 = (r.i == st.nch - 1) ? st.bytes_last : st.bytes_a;
-        } else {
-            const uint32_t row = r.i / st.period, j = r.i % st.period;
-            off = (uint64_t)row * ((st.period - 1) * st.bytes_a + st.bytes_b) + (uint64_t)j * st.bytes_a;
-            c.bytes0 = (j == st.period - 1) ? st.bytes_b : st.bytes_a;
-        }
-        c.src0 = q.base[m] + (size_t)r.l * q.layer_bytes + st.byte_off + off;
-    }
-    return c;
-}
-
-__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
-
-// Everything lane 0 needs to start the copies of a chunk, worked out ahead of time.
-struct ChunkIssue {
-    const uint8_t* src0;   // linear copies: sources; tensor boxes: unused
-    const uint8_t* src1;
-    uint32_t bytes0, bytes1;
-    int32_t yk, yv;        // tensor boxes: first cache row of the K and of the V boxes
-    bool boxes;
-};
-__device__ __forceinline__ ChunkIssue seq_issue_info(const SeqPlan& q, const SeqPos& r) {
-    ChunkIssue c;
-    c.boxes = (r.stage == 1 && q.tc != 0);
-    c.yk = c.yv = 0;
-    if (c.boxes) {
-        const AttnWindow w = attn_window(q.c0, q.cend, q.pb, r.i);
-        c.yk = (int32_t)(q.k_row0 + r.l * q.rows_per_layer + w.w0);
-        c.yv = c.yk + (int32_t)q.v_row_delta;
-        c.src0 = c.src1 = nullptr;
-        c.bytes0 = c.bytes1 = SLOT_BYTES / 2;
-    } else {
-        const ChunkSrc l = seq_chunk(q, r);
-        c.src0 = l.src0;
-        c.src1 = l.src1;
-        c.bytes0 = l.bytes0;
-        c.bytes1 = l.bytes1;
-    }
-    return c;
-}
-
-// State of a warp's slot: the next chunk it will issue, the chunk it will prefetch into L2, and the use counts.
+// Consumer side of the ring: which of its nsw slots the warp reads next and with which barrier phase.
 struct WarpRing {
-    SeqPos pos;             // next chunk to issue
-    ChunkIssue nx;          // how to issue pos (precomputed)
-    SeqPos ahead;           // chunk to prefetch into L2 at the next issue (pos + prefetch_chunks turns)
-    uint32_t n;             // global index of pos (for the optional chunk log)
-    uint32_t issued;        // copies armed on this warp's barrier so far
-    uint32_t uses;          // chunks taken from the slot so far; (uses & 1) is the phase to wait for
+    uint32_t cslot;         // slot (0..nsw-1) the next chunk is consumed from
+    uint32_t cphase;        // barrier phase of that slot to wait for
+    uint32_t rslot;         // slot consumed last (the one to release)
 };
-
-// Arms the warp's barrier and starts the copies of its next chunk (lane 0) from the precomputed description, then
-// steps nslots chunks ahead and works out the following chunk -- that arithmetic overlaps with the copy just
-// started.  Called once the whole warp has finished reading the slot (after __syncwarp).
-// With Params::prefetch_chunks = k > 0 the warp also asks L2 to fetch the chunk it will issue k turns later.
-__device__ __forceinline__ void ring_issue_next(const Params& p, const Smem& s, WarpRing& r, uint32_t warp, uint32_t lane,
-                                                uint64_t pol) {
-    if (r.pos.done || *s.abort_flag) return;
-    if (lane == 0) {
-        const ChunkIssue& c = r.nx;
-        const uint32_t bar = smem_u32(&s.full[warp]);
-        const uint32_t dst = smem_u32(s.ring) + warp * SLOT_BYTES;
-        // the slot was read through the generic proxy; the copies write it through the async proxy
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        chunk_stamp(p, blockIdx.x, r.n, 0);
-        mbar_arrive_expect_tx(bar, c.bytes0 + c.bytes1);
-        if (c.boxes) {
-            // K/V rows as swizzled boxes of the cache tensor: [pb rows] x [64 columns] per box, K boxes in the first
-            // half of the slot, V boxes in the second; a box is always written whole (rows outside the chunk's own
-            // positions are ignored by the consumer)
-            const uint32_t box_bytes = SLOT_BYTES / 2 / (p.hd / 64u);
-            for (uint32_t bx = 0; bx < p.hd / 64u; ++bx) {
-                tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), c.yk, bar, pol);
-                tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), c.yv, bar, pol);
-            }
-        } else {
-            tma_bulk_g2s(dst, c.src0, c.bytes0, bar, pol);
-            if (c.bytes1) tma_bulk_g2s(dst + SLOT_BYTES / 2, c.src1, c.bytes1, bar, pol);
-        }
-    }
-    ++r.issued;
-    const SeqPlan& q = *s.plan;
-    r.pos.i += p.nslots;
-    r.n += p.nslots;
-    seq_normalize(q, r.pos);
-    if (!r.pos.done) r.nx = seq_issue_info(q, r.pos);
-    if (p.prefetch_chunks && !r.ahead.done && !(r.ahead.stage == 1 && q.tc)) {
-        const ChunkSrc f = seq_chunk(q, r.ahead);
-        for (uint32_t o = lane * 128u; o < f.bytes0; o += 32u * 128u)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(f.src0 + o));
-        for (uint32_t o = lane * 128u; o < f.bytes1; o += 32u * 128u)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(f.src1 + o));
-        r.ahead.i += p.nslots;
-        seq_normalize(q, r.ahead);
+// The warp takes a chunk from its current slot and moves to the next one (call after the wait).
+__device__ __forceinline__ void ring_advance_consume(const Params& p, WarpRing& r) {
+    r.rslot = r.cslot;
+    if (++r.cslot == p.nsw) {
+        r.cslot = 0;
+        r.cphase ^= 1u;
     }
 }
-
-__device__ __forceinline__ WarpRing ring_begin(const Params& p, const Smem& s, uint32_t warp, uint32_t l0) {
+// The whole warp has finished reading the slot it consumed last (call after __syncwarp): hand it back.
+__device__ __forceinline__ void ring_release(const Params& p, const Smem& s, const WarpRing& r, uint32_t warp, uint32_t lane) {
+    if (lane == 0) mbar_arrive(smem_u32(&s.empty[warp * p.nsw + r.rslot]));
+}
+__device__ __forceinline__ WarpRing ring_begin() {
     WarpRing r;
-    r.pos.l = l0;
-    r.pos.stage = 0;
-    r.pos.i = warp;
-    r.pos.done = warp >= p.nslots || l0 >= s.plan->l1;
-    r.n = warp;
-    r.issued = 0;
-    r.uses = 0;
-    if (!r.pos.done) seq_normalize(*s.plan, r.pos);
-    if (!r.pos.done) r.nx = seq_issue_info(*s.plan, r.pos);
-    r.ahead = r.pos;
-    if (!r.ahead.done) {
-        r.ahead.i += p.prefetch_chunks * p.nslots;
-        seq_normalize(*s.plan, r.ahead);
-    }
+    r.cslot = 0;
+    r.cphase = 0;
+    r.rslot = 0;
     return r;
 }
 
-// Before the CTA exits no bulk copy may still be writing its shared memory: wait (bounded) for the last copy this
-// warp armed.  On the normal path that copy was consumed long ago and the wait returns at once.
-__device__ __forceinline__ void ring_finish(const Params& p, const Smem& s, const WarpRing& r, uint32_t warp) {
-    if (r.issued == 0) return;
-    const uint32_t bar = smem_u32(&s.full[warp]);
-    const uint32_t parity = (r.issued - 1u) & 1u;
-    const uint64_t t0 = globaltimer_ns();
-    while (!mbar_try_wait(bar, parity)) {
-        if (globaltimer_ns() - t0 > p.wait_ns) return;
+// Producer state: where the next chunk goes.
+struct RingProd {
+    uint32_t c, k, use, n;   // consumer, slot of that consumer, use count of that slot, chunk index (for the log)
+    uint64_t pol;
+    bool aborted;
+};
+
+// Waits for the slot of the next chunk, arms its barrier and starts one or two linear copies into it.
+__device__ __forceinline__ void prod_issue(const Params& p, const Smem& s, RingProd& r, const uint8_t* src0, uint32_t bytes0,
+                                           const uint8_t* src1, uint32_t bytes1, uint32_t dst1) {
+    if (r.aborted) return;
+    const uint32_t slot = r.c * p.nsw + r.k;
+    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty[slot]), (r.use - 1u) & 1u)) {
+        r.aborted = true;
+        return;
     }
+    const uint32_t bar = smem_u32(&s.full[slot]);
+    const uint32_t dst = smem_u32(s.ring) + slot * SLOT_BYTES;
+    chunk_stamp(p, blockIdx.x, r.n, 0);
+    mbar_arrive_expect_tx(bar, bytes0 + bytes1);
+    tma_bulk_g2s(dst, src0, bytes0, bar, r.pol);
+    if (bytes1) tma_bulk_g2s(dst + dst1, src1, bytes1, bar, r.pol);
+    ++r.n;
+    if (++r.c == p.nslots) {
+        r.c = 0;
+        if (++r.k == p.nsw) {
+            r.k = 0;
+            ++r.use;
+        }
+    }
+}
+// Same for a chunk of K/V rows as swizzled boxes of the cache tensor: [pb rows] x [64 columns] per box, K boxes in
+// the first half of the slot, V boxes in the second; a box is always written whole (rows outside the chunk's own
+// positions are ignored by the consumer).
+__device__ __forceinline__ void prod_issue_boxes(const Params& p, const Smem& s, RingProd& r, int32_t yk, int32_t yv) {
+    if (r.aborted) return;
+    const uint32_t slot = r.c * p.nsw + r.k;
+    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty[slot]), (r.use - 1u) & 1u)) {
+        r.aborted = true;
+        return;
+    }
+    const uint32_t bar = smem_u32(&s.full[slot]);
+    const uint32_t dst = smem_u32(s.ring) + slot * SLOT_BYTES;
+    chunk_stamp(p, blockIdx.x, r.n, 0);
+    mbar_arrive_expect_tx(bar, (uint32_t)SLOT_BYTES);
+    const uint32_t box_bytes = SLOT_BYTES / 2 / (p.hd / 64u);
+    for (uint32_t bx = 0; bx < p.hd / 64u; ++bx) {
+        tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yk, bar, r.pol);
+        tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yv, bar, r.pol);
+    }
+    ++r.n;
+    if (++r.c == p.nslots) {
+        r.c = 0;
+        if (++r.k == p.nsw) {
+            r.k = 0;
+            ++r.use;
+        }
+    }
+}
+
+// Streams this CTA's share of one matrix (units [u0, u1) of the plan): one linear run of bytes cut into chunks,
+// per chunk only pointer increments.
+__device__ __forceinline__ void produce_matrix(const Params& p, const Smem& s, RingProd& r, const GemvPlan& pl,
+                                               const __nv_bfloat16* base, uint32_t cta) {
+    const CtaRange cr = cta_units(pl, cta, p.P);
+    const uint8_t* ptr = reinterpret_cast<const uint8_t*>(base) + (size_t)cr.u0 * pl.rpc * pl.K * 2u;
+    const uint32_t last_len = pl.K - (pl.npieces - 1) * pl.kp;
+    for (uint32_t u = cr.u0; u < cr.u1; ++u) {
+        const uint32_t rows = min(pl.rpc, pl.R - u * pl.rpc);   // only the matrix's last unit can be short
+        for (uint32_t j = 0; j < pl.npieces; ++j) {
+            const uint32_t bytes = rows * ((j == pl.npieces - 1) ? last_len : pl.kp) * 2u;
+            prod_issue(p, s, r, ptr, bytes, nullptr, 0u, 0u);
+            ptr += bytes;
+        }
+    }
+}
+
+// Streams the cached K/V rows of this CTA's attention unit for one layer.
+__device__ __forceinline__ void produce_attention(const Params& p, const Smem& s, RingProd& r, const AttnUnit& u,
+                                                  uint32_t layer) {
+    if (!u.active) return;
+    const uint32_t pb = attn_positions_per_chunk(p);
+    if (p.attn_tc) {
+        const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
+        const uint32_t row0 = layer * 2u * vdelta + (u.b * p.nkv + u.g) * p.max_ctx;
+        for (uint32_t i = 0; i < u.nring; ++i) {
+            const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
+            prod_issue_boxes(p, s, r, (int32_t)(row0 + w.w0), (int32_t)(row0 + w.w0 + vdelta));
+        }
+    } else {
+        const uint32_t row_bytes = p.hd * 2u;
+        const uint8_t* ks = reinterpret_cast<const uint8_t*>(kv_head(p, layer, 0, u.b, u.g)) + (size_t)u.c0 * row_bytes;
+        const uint8_t* vs = reinterpret_cast<const uint8_t*>(kv_head(p, layer, 1, u.b, u.g)) + (size_t)u.c0 * row_bytes;
+        uint32_t left = u.cend - u.c0;
+        for (uint32_t i = 0; i < u.nring; ++i) {
+            const uint32_t np = left < pb ? left : pb;
+            prod_issue(p, s, r, ks, np * row_bytes, vs, np * row_bytes, SLOT_BYTES / 2);
+            ks += np * row_bytes;
+            vs += np * row_bytes;
+            left -= np;
+        }
+    }
+}
+
+// After an abandoned run no bulk copy may still be writing this CTA's shared memory when it exits: wait (bounded)
+// for the last copy armed on every slot.
+__device__ __forceinline__ void produce_drain(const Params& p, const Smem& s, const RingProd& r) {
+    if (!r.aborted) return;
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t cc = 0; cc < p.nslots; ++cc) {
+        for (uint32_t kk = 0; kk < p.nsw; ++kk) {
+            const uint32_t cnt = r.use + ((kk < r.k || (kk == r.k && cc < r.c)) ? 1u : 0u);  // uses of this slot so far
+            if (cnt == 0) continue;
+            const uint32_t bar = smem_u32(&s.full[cc * p.nsw + kk]);
+            while (!mbar_try_wait(bar, (cnt - 1u) & 1u)) {
+                if (globaltimer_ns() - t0 > p.wait_ns) return;
+            }
+        }
+    }
+}
+
+// The producer thread of the decoder kernel: layers [l0, l1).
+__device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, uint32_t cta, uint32_t l0, uint32_t l1) {
+    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+    const AttnUnit u = attn_unit(p, cta);
+    for (uint32_t l = l0; l < l1 && !r.aborted; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
+        produce_attention(p, s, r, u, l);
+        produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+        produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
+        produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+    }
+    produce_drain(p, s, r);
+}
+// ... and of the classifier kernel.
+__device__ __forceinline__ void produce_classifier(const Params& p, const Smem& s, uint32_t cta) {
+    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+    produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
+    produce_drain(p, s, r);
 }
 
 // ------------------------------------------------------------------------------------------------ consumers
@@ -688,60 +585,131 @@ __device__ __forceinline__ void load_vec(const Params& p, const Smem& s, const f
 }
 
 // acc[r] += sum over this lane's columns of W[r][k] * vec[k]; W rows in shared memory, row pitch rowbytes.
-// One 256-column block of the dot products: this lane's 8 columns of NR rows against its 8 vector elements,
-// into two accumulators per row (even and odd columns) so that the FMA chains stay short.
-template <int NR>
-__device__ __forceinline__ void dot_block(const uint4 (&q)[NR], const float4& xa, const float4& xb, float (&e)[NR],
-                                          float (&o)[NR]) {
+// This lane's share of a slice of the input vector: for block b of 256 columns the 8 columns b*256 + lane*8 .. +7.
+struct XRegs {
+    float v[MAX_XB][8];
+};
+// Loads columns [kofs, kofs + klen) of the shared input vector (lane-permuted layout, see vec_perm) into registers;
+// columns beyond klen read as zero.  kofs is a multiple of 256.
+__device__ __forceinline__ void load_xregs(XRegs& x, const float* vec, uint32_t kofs, uint32_t klen, uint32_t lane) {
+    const float4* v4 = reinterpret_cast<const float4*>(vec) + (kofs >> 8) * 64;
 #pragma unroll
-    for (int r = 0; r < NR; ++r) {
-        e[r] = fmaf(bf_lo(q[r].x), xa.x, e[r]);
-        o[r] = fmaf(bf_hi(q[r].x), xa.y, o[r]);
-        e[r] = fmaf(bf_lo(q[r].y), xa.z, e[r]);
-        o[r] = fmaf(bf_hi(q[r].y), xa.w, o[r]);
-        e[r] = fmaf(bf_lo(q[r].z), xb.x, e[r]);
-        o[r] = fmaf(bf_hi(q[r].z), xb.y, o[r]);
-        e[r] = fmaf(bf_lo(q[r].w), xb.z, e[r]);
-        o[r] = fmaf(bf_hi(q[r].w), xb.w, o[r]);
+    for (int b = 0; b < MAX_XB; ++b) {
+        float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+        if ((uint32_t)b * 256u + lane * 8u < klen) {
+            lo = v4[b * 64 + lane];
+            hi = v4[b * 64 + 32 + lane];
+        }
+        x.v[b][0] = lo.x; x.v[b][1] = lo.y; x.v[b][2] = lo.z; x.v[b][3] = lo.w;
+        x.v[b][4] = hi.x; x.v[b][5] = hi.y; x.v[b][6] = hi.z; x.v[b][7] = hi.w;
     }
 }
 
-// acc[r] += sum over this lane's columns of W[r][k] * vec[k]; W rows in shared memory, row pitch rowbytes.
-// Four blocks are loaded before any is used, so the shared-memory latency overlaps with the arithmetic.
+// Same slice taken straight from global memory (a vector written by other CTAs: read through L2), for input
+// vectors that are not staged in shared memory.  src points at column 0 of the whole vector.
+__device__ __forceinline__ void load_xregs_global(XRegs& x, const float* src, uint32_t kofs, uint32_t klen, uint32_t lane) {
+    float4 lo[MAX_XB], hi[MAX_XB];
+#pragma unroll
+    for (int b = 0; b < MAX_XB; ++b) {
+        lo[b] = make_float4(0.f, 0.f, 0.f, 0.f);
+        hi[b] = lo[b];
+        const uint32_t k = (uint32_t)b * 256u + lane * 8u;
+        if (k < klen) {
+            lo[b] = __ldcg(reinterpret_cast<const float4*>(src + kofs + k));
+            hi[b] = __ldcg(reinterpret_cast<const float4*>(src + kofs + k + 4));
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < MAX_XB; ++b) {
+        x.v[b][0] = lo[b].x; x.v[b][1] = lo[b].y; x.v[b][2] = lo[b].z; x.v[b][3] = lo[b].w;
+        x.v[b][4] = hi[b].x; x.v[b][5] = hi[b].y; x.v[b][6] = hi[b].z; x.v[b][7] = hi[b].w;
+    }
+}
+
+// acc[r] = sum over this lane's columns of W[r][k] * x[k] for NR rows held in shared memory (row pitch `pitch`
+// bytes, klen columns each).  The vector comes from registers, so the only shared-memory traffic is the weights.
+// Two accumulators per row (even and odd columns) keep the FMA chains short; the order of the sums is fixed.
 template <int NR>
-__device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t rowbytes, const float* vec, uint32_t len,
-                                         uint32_t lane, float (&acc)[NR]) {
-    const float4* v4 = reinterpret_cast<const float4*>(vec);
+__device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane, const XRegs& x,
+                                         float (&acc)[NR]) {
     float e[NR], o[NR];
 #pragma unroll
     for (int r = 0; r < NR; ++r) e[r] = o[r] = 0.f;
-    const uint32_t nblk = len >> 8;  // full 256-column blocks
-    uint32_t blk = 0;
-    for (; blk + 4 <= nblk; blk += 4) {
-        float4 xa[4], xb[4];
-        uint4 q[4][NR];
+    // blocks in groups of four: the (predicated) loads of a group are all issued before its arithmetic, so the
+    // shared-memory latency is paid once per group, not once per block
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            xa[u] = v4[(blk + u) * 64 + lane];
-            xb[u] = v4[(blk + u) * 64 + 32 + lane];
+    for (int b0 = 0; b0 < MAX_XB; b0 += 4) {
+        if ((uint32_t)b0 * 256u < klen) {                   // uniform over the warp
+            uint4 q[4][NR];
 #pragma unroll
-            for (int r = 0; r < NR; ++r)
-                q[u][r] = *reinterpret_cast<const uint4*>(w + (size_t)r * rowbytes + (size_t)((blk + u) * 256 + lane * 8) * 2);
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t k = (uint32_t)(b0 + u) * 256u + lane * 8u;
+                const bool in = k < klen;                   // false only in or after the last, partial block
+                const uint32_t kk = in ? k : 0u;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    q[u][r] = *reinterpret_cast<const uint4*>(w + (size_t)r * pitch + (size_t)kk * 2);
+                    if (!in) q[u][r] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int b = b0 + u;
+#pragma unroll
+                for (int r = 0; r < NR; ++r) {
+                    e[r] = fmaf(bf_lo(q[u][r].x), x.v[b][0], e[r]);
+                    o[r] = fmaf(bf_hi(q[u][r].x), x.v[b][1], o[r]);
+                    e[r] = fmaf(bf_lo(q[u][r].y), x.v[b][2], e[r]);
+                    o[r] = fmaf(bf_hi(q[u][r].y), x.v[b][3], o[r]);
+                    e[r] = fmaf(bf_lo(q[u][r].z), x.v[b][4], e[r]);
+                    o[r] = fmaf(bf_hi(q[u][r].z), x.v[b][5], o[r]);
+                    e[r] = fmaf(bf_lo(q[u][r].w), x.v[b][6], e[r]);
+                    o[r] = fmaf(bf_hi(q[u][r].w), x.v[b][7], o[r]);
+                }
+            }
         }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) dot_block<NR>(q[u], xa[u], xb[u], e, o);
-    }
-    for (uint32_t k = blk * 256 + lane * 8; k < len; k += 256) {  // remaining blocks, the last possibly partial
-        const uint32_t bk = k >> 8;
-        const float4 xa = v4[bk * 64 + lane];
-        const float4 xb = v4[bk * 64 + 32 + lane];
-        uint4 q[NR];
-#pragma unroll
-        for (int r = 0; r < NR; ++r) q[r] = *reinterpret_cast<const uint4*>(w + (size_t)r * rowbytes + (size_t)k * 2);
-        dot_block<NR>(q, xa, xb, e, o);
     }
 #pragma unroll
-    for (int r = 0; r < NR; ++r) acc[r] += e[r] + o[r];
+    for (int r = 0; r < NR; ++r) acc[r] = e[r] + o[r];
+}
+
+// Branch-free variant for pieces of exactly NB full blocks (the common sizes): no predicates, so the compiler is
+// free to software-pipeline the shared-memory loads against the arithmetic.  Same order of operations as dot_rows.
+template <int NR, int NB>
+__device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, uint32_t lane, const XRegs& x,
+                                              float (&acc)[NR]) {
+    float e[NR], o[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) e[r] = o[r] = 0.f;
+    const uint8_t* wl = w + (size_t)lane * 16;
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+            const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)b * 512);
+            e[r] = fmaf(bf_lo(q.x), x.v[b][0], e[r]);
+            o[r] = fmaf(bf_hi(q.x), x.v[b][1], o[r]);
+            e[r] = fmaf(bf_lo(q.y), x.v[b][2], e[r]);
+            o[r] = fmaf(bf_hi(q.y), x.v[b][3], o[r]);
+            e[r] = fmaf(bf_lo(q.z), x.v[b][4], e[r]);
+            o[r] = fmaf(bf_hi(q.z), x.v[b][5], o[r]);
+            e[r] = fmaf(bf_lo(q.w), x.v[b][6], e[r]);
+            o[r] = fmaf(bf_hi(q.w), x.v[b][7], o[r]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) acc[r] = e[r] + o[r];
+}
+// NR rows: picks the branch-free variant when the piece is a whole number of blocks of a common size.
+template <int NR>
+__device__ __forceinline__ void dot_n(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane, const XRegs& x,
+                                      float (&acc)[NR]) {
+    switch (klen) {
+        case 4096: dot_rows_full<NR, 16>(w, pitch, lane, x, acc); break;
+        case 2560: dot_rows_full<NR, 10>(w, pitch, lane, x, acc); break;
+        case 2048: dot_rows_full<NR, 8>(w, pitch, lane, x, acc); break;
+        default: dot_rows<NR>(w, pitch, klen, lane, x, acc); break;
+    }
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -775,104 +743,141 @@ struct RingCursor {
 // same warp, in order, so a parity wait can never be satisfied by a phase two uses old.  (With free chunk-to-warp
 // assignment a fast warp can test the barrier of use k while use k-1 is still in flight, and parity k&1 then
 // reads as complete.)
-__device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, float* out,
-                                           uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
-                                           uint64_t pol) {
+__device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, float* out,
+                                        uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
+                                        const float* xsrc) {
+    // xsrc == nullptr: the input vector is staged in s.vec; otherwise it is read from global memory per piece
     const CtaRange r = cta_units(pl, cta, p.P);
-    const uint32_t nch = (r.u1 - r.u0) * pl.chunks_per_unit;
+    const uint32_t nch = (r.u1 - r.u0) * pl.npieces;
     const uint32_t first = rc.first_chunk(warp, p.nslots);
-    for (uint32_t i = (warp < p.nslots ? first : nch); i < nch; i += p.nslots) {
-        const uint32_t slot = warp;
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
-        mbar_wait(p, s, smem_u32(&s.full[slot]), wr.uses & 1u);
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
-        ++wr.uses;
-        const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
+    XRegs x;
+    uint32_t x_piece = 0xffffffffu;
+    for (uint32_t i = first; i < nch; i += p.nslots) {
         const ChunkGeom g = chunk_geom(pl, r.u0, i);
-        if (pl.rpc) {
-            const uint32_t rowbytes = pl.K * 2u;
-            for (uint32_t rr = 0; rr < g.nrows; rr += 2) {
-                float y0, y1 = 0.f;
-                float res0 = 0.f, res1 = 0.f;  // residual inputs, fetched before the dot products hide their latency
-                if (ep == EP_RESIDUAL && lane == 0) {
-                    res0 = __ldcg(out + g.row + rr);
-                    if (rr + 1 < g.nrows) res1 = __ldcg(out + g.row + rr + 1);
+        if (g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
+            if (xsrc) load_xregs_global(x, xsrc, g.kofs, g.klen, lane);
+            else load_xregs(x, s.vec, g.kofs, g.klen, lane);
+            x_piece = g.piece;
+        }
+        const uint32_t slot = warp * p.nsw + wr.cslot;
+        const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
+        const uint32_t pitch = g.klen * 2u;
+        if (pl.rpc <= MAX_RPC_SPLIT) {
+            // one unit piece of up to four rows: the common case.  Residual inputs are fetched before the wait, their
+            // L2 latency hides behind it.
+            float res = 0.f;
+            if (ep == EP_RESIDUAL && lane < g.nrows) res = __ldcg(out + g.row + lane);
+            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            ring_advance_consume(p, wr);
+            float y[MAX_RPC_SPLIT] = {0.f, 0.f, 0.f, 0.f};
+            if (g.nrows == 2) {
+                float acc[2];
+                dot_n<2>(sp, pitch, g.klen, lane, x, acc);
+                y[0] = acc[0]; y[1] = acc[1];
+            } else if (g.nrows == 3) {
+                float acc[3];
+                dot_n<3>(sp, pitch, g.klen, lane, x, acc);
+                y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2];
+            } else if (g.nrows == 4) {
+                float acc[4];
+                dot_n<4>(sp, pitch, g.klen, lane, x, acc);
+                y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2]; y[3] = acc[3];
+            } else {
+                float acc[1];
+                dot_n<1>(sp, pitch, g.klen, lane, x, acc);
+                y[0] = acc[0];
+            }
+            __syncwarp();
+            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+            ring_release(p, s, wr, warp, lane);   // the slot has been read for the last time
+#pragma unroll
+            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = warp_sum(y[rr]);
+            float rs[MAX_RPC_SPLIT];
+#pragma unroll
+            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) rs[rr] = __shfl_sync(0xffffffffu, res, rr);
+            if (lane == 0) {
+                bool emit = true;
+                if (pl.npieces > 1) {
+                    // partial sums of the unit's pieces meet in shared memory; the last piece to arrive adds them in
+                    // piece order and emits the rows
+                    const uint32_t us = (g.unit - r.u0) % UNIT_SLOTS;
+                    volatile float* part = s.unit_part + us * (MAX_PIECES * MAX_RPC_SPLIT);
+#pragma unroll
+                    for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) part[g.piece * MAX_RPC_SPLIT + rr] = y[rr];
+                    __threadfence_block();
+                    const int old = atomicAdd(&s.unit_cnt[us], 1);
+                    emit = (old == (int)pl.npieces - 1);
+                    if (emit) {
+                        __threadfence_block();
+                        s.unit_cnt[us] = 0;
+#pragma unroll
+                        for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = 0.f;
+                        for (uint32_t j = 0; j < pl.npieces; ++j) {
+#pragma unroll
+                            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] += part[j * MAX_RPC_SPLIT + rr];
+                        }
+                    }
                 }
-                if (rr + 1 < g.nrows) {
-                    float acc[2] = {0.f, 0.f};
-                    dot_rows<2>(sp + (size_t)rr * rowbytes, rowbytes, s.vec, pl.K, lane, acc);
+                if (emit) {
+                    if (ep == EP_SWIGLU) {
+                        out[g.row >> 1] = silu(y[0]) * y[1];
+                        if (g.nrows == 4) out[(g.row >> 1) + 1] = silu(y[2]) * y[3];
+                    } else {
+#pragma unroll
+                        for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
+                            if ((uint32_t)rr < g.nrows) out[g.row + rr] = (ep == EP_RESIDUAL ? rs[rr] : 0.f) + y[rr];
+                    }
+                }
+            }
+        } else {
+            // many short rows in one chunk (small hidden sizes): pair after pair, whole rows (npieces == 1)
+            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            ring_advance_consume(p, wr);
+            for (uint32_t rr = 0; rr < g.nrows; rr += 2) {
+                const bool two = rr + 1 < g.nrows;
+                float rs0 = 0.f, rs1 = 0.f;
+                if (ep == EP_RESIDUAL && lane == 0) {
+                    rs0 = __ldcg(out + g.row + rr);
+                    if (two) rs1 = __ldcg(out + g.row + rr + 1);
+                }
+                float y0, y1 = 0.f;
+                if (two) {
+                    float acc[2];
+                    dot_rows<2>(sp + (size_t)rr * pitch, pitch, g.klen, lane, x, acc);
                     y0 = warp_sum(acc[0]);
                     y1 = warp_sum(acc[1]);
                 } else {
-                    float acc[1] = {0.f};
-                    dot_rows<1>(sp + (size_t)rr * rowbytes, rowbytes, s.vec, pl.K, lane, acc);
+                    float acc[1];
+                    dot_rows<1>(sp + (size_t)rr * pitch, pitch, g.klen, lane, x, acc);
                     y0 = warp_sum(acc[0]);
                 }
                 if (lane == 0) {
                     const uint32_t row = g.row + rr;
                     if (ep == EP_STORE) {
                         out[row] = y0;
-                        if (rr + 1 < g.nrows) out[row + 1] = y1;
+                        if (two) out[row + 1] = y1;
                     } else if (ep == EP_RESIDUAL) {
-                        out[row] = res0 + y0;
-                        if (rr + 1 < g.nrows) out[row + 1] = res1 + y1;
+                        out[row] = rs0 + y0;
+                        if (two) out[row + 1] = rs1 + y1;
                     } else {
                         out[row >> 1] = silu(y0) * y1;
                     }
                 }
             }
             __syncwarp();
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
-            ring_issue_next(p, s, wr, warp, lane, pol);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
-        } else {
-            float resb[2] = {0.f, 0.f};
-            if (ep == EP_RESIDUAL && lane == 0) {
-                resb[0] = __ldcg(out + g.unit * pl.rows_per_unit);
-                if (pl.rows_per_unit == 2) resb[1] = __ldcg(out + g.unit * pl.rows_per_unit + 1);
-            }
-            float acc[1] = {0.f};
-            dot_rows<1>(sp, 0, s.vec + g.kofs, g.elems, lane, acc);
-            const float y = warp_sum(acc[0]);
-            if (lane == 0) {
-                const uint32_t us = (g.unit - r.u0) % UNIT_SLOTS;
-                volatile float* part = s.unit_part + us * MAX_PIECES;
-                part[g.piece] = y;
-                __threadfence_block();
-                const int old = atomicAdd(&s.unit_cnt[us], 1);
-                if (old == (int)pl.chunks_per_unit - 1) {
-                    __threadfence_block();
-                    s.unit_cnt[us] = 0;
-                    float row_y[2] = {0.f, 0.f};
-                    for (uint32_t rr = 0; rr < pl.rows_per_unit; ++rr) {
-                        float t = 0.f;
-                        for (uint32_t j = 0; j < pl.ksplit; ++j) t += part[rr * pl.ksplit + j];
-                        row_y[rr] = t;
-                    }
-                    const uint32_t row = g.unit * pl.rows_per_unit;
-                    if (ep == EP_STORE) {
-                        out[row] = row_y[0];
-                        if (pl.rows_per_unit == 2) out[row + 1] = row_y[1];
-                    } else if (ep == EP_RESIDUAL) {
-                        out[row] = resb[0] + row_y[0];
-                        if (pl.rows_per_unit == 2) out[row + 1] = resb[1] + row_y[1];
-                    } else {
-                        out[row >> 1] = silu(row_y[0]) * row_y[1];
-                    }
-                }
-            }
-            __syncwarp();
-            ring_issue_next(p, s, wr, warp, lane, pol);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
+            ring_release(p, s, wr, warp, lane);
         }
+        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
     }
     rc.advance(nch, p.nslots);
 }
 
 // End of a stage: all consumer warps have written their outputs; one thread publishes the CTA's arrival.
-__device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool skip) {
+__device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool skip, uint32_t weight = 1u) {
     consumer_bar();
-    if (ctid == 0 && !skip) red_release_add(ctr, 1u);  // release: cumulative over the CTA barrier above
+    if (ctid == 0 && !skip && weight) red_release_add(ctr, weight);  // release: cumulative over the CTA barrier above
 }
 
 // Waits (bounded) until `target` CTAs have signalled.  Replaces the grid-wide barrier of a kernel boundary.
@@ -972,9 +977,9 @@ __device__ __forceinline__ void attn_batch(AttnAcc<G>& st, const float (&q)[G][8
 template <int HD>
 __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, const AttnUnit& u, uint32_t cta,
                                                uint32_t warp, uint32_t lane, uint32_t first, const RingCursor& rc,
-                                               WarpRing& wr, uint64_t pol, const float* q_s, float* comb,
+                                               WarpRing& wr, const float* q_s, float* comb,
                                                const uint8_t* stage_k, const uint8_t* stage_v) {
-    constexpr int NKB = HD / 16, NNT = HD / 8;
+    constexpr int NKB = HD / 16, NMT = HD / 16;
     const uint32_t G = p.G, g = lane >> 2, t = lane & 3u;
     AttnTcState<HD> st;
 #pragma unroll
@@ -989,41 +994,112 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
         }
     }
 #pragma unroll
-    for (int n = 0; n < NNT; ++n) st.o[n][0] = st.o[n][1] = st.o[n][2] = st.o[n][3] = 0.f;
-    st.m = -INFINITY;
-    st.l = 0.f;
+    for (int n = 0; n < NMT; ++n) st.o[n][0] = st.o[n][1] = st.o[n][2] = st.o[n][3] = 0.f;
+    st.m[0] = st.m[1] = -INFINITY;
+    st.l[0] = st.l[1] = 0.f;
 
     const uint32_t pb = attn_positions_per_chunk(p);
     const uint32_t box_bytes = pb * 128u;
-    for (uint32_t i = (warp < p.nslots ? first : u.nring); i < u.nring; i += p.nslots) {
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
-        mbar_wait(p, s, smem_u32(&s.full[warp]), wr.uses & 1u);
+    for (uint32_t i = first; i < u.nring; i += p.nslots) {
+        const uint32_t slot = warp * p.nsw + wr.cslot;
+        mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
         if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
-        ++wr.uses;
-        const uint32_t kbase = smem_u32(s.ring) + warp * SLOT_BYTES;
+        ring_advance_consume(p, wr);
+        const uint32_t kbase = smem_u32(s.ring) + slot * SLOT_BYTES;
         const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
         for (uint32_t row0 = 0; row0 < pb; row0 += 16)
             if (row0 + 16 > w.lo && row0 < w.hi) attn_tc_tile<HD>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, row0, w.lo, w.hi, lane);
         __syncwarp();
-        ring_issue_next(p, s, wr, warp, lane, pol);
+        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+        ring_release(p, s, wr, warp, lane);
         if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
     }
     if (u.has_new && first == 0)  // the position written by this step sits in row 0 of the staging tile
-        attn_tc_tile<HD>(st, smem_u32(stage_k), smem_u32(stage_v), 16u * 128u, 0u, 0u, 1u, lane);
+        attn_tc_tile<HD>(st, smem_u32(stage_k), smem_u32(stage_v), 128u, 0u, 0u, 1u, lane);
 
-    float l = st.l;
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (g < G) {
-        float* dst = comb + ((size_t)first * G + g) * (HD + 2);
+    // row sums: add the parts held by the lanes that share the heads (same lane % 4)
+    float l0 = st.l[0], l1 = st.l[1];
 #pragma unroll
-        for (int n = 0; n < NNT; ++n) {
-            dst[n * 8 + 2 * t] = st.o[n][0];
-            dst[n * 8 + 2 * t + 1] = st.o[n][1];
+    for (int o = 4; o < 32; o <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const uint32_t h = 2 * t + hh;
+        if (h < G) {
+            float* dst = comb + ((size_t)first * G + h) * (HD + 2);
+#pragma unroll
+            for (int n = 0; n < NMT; ++n) {
+                dst[n * 16 + g] = st.o[n][hh];
+                dst[n * 16 + g + 8] = st.o[n][2 + hh];
+            }
+            if (g == 0) {
+                dst[HD] = st.m[hh];
+                dst[HD + 1] = hh ? l1 : l0;
+            }
         }
-        if (t == 0) {
-            dst[HD] = st.m;
-            dst[HD + 1] = l;
+    }
+}
+
+// Merges the split-K partial results of one (sequence, kv head) into the attention output o (run by the unit that
+// arrived last, after every other unit of the group has published its partial result).
+__device__ __noinline__ void attn_merge(const Params& p, const AttnUnit& u, uint32_t G, uint32_t ctid, float* comb) {
+    const uint32_t hd = p.hd, b = u.b, g = u.g, nchunk = u.nchunk;
+    const uint32_t unit0 = u.bg * p.cps;
+    // Merge in two L2 round trips.  First the (max, sum) pairs of every (head, chunk): one per thread, turned into
+    // weights w[h][c] = exp2(m_c - M_h) / L_h in shared memory.  Then the weighted sum of the partial outputs, with
+    // all the loads of up to three outputs per thread in flight at once.  The orders of all sums are fixed.
+    float* wtab = comb;   // [2][G][nchunk]; the per-warp partials in comb are no longer needed
+    for (uint32_t t = ctid; t < G * nchunk; t += NCT) {
+        const uint32_t h = t / nchunk, c = t % nchunk;
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(unit0 + c) * G + h) * 2));
+        wtab[t] = ml.x;
+        wtab[G * nchunk + t] = ml.y;
+    }
+    consumer_bar();
+    if (ctid < G) {
+        const uint32_t h = ctid;
+        float Mx = -INFINITY;
+        for (uint32_t c = 0; c < nchunk; ++c) Mx = fmaxf(Mx, wtab[h * nchunk + c]);
+        float Lx = 0.f;
+        for (uint32_t c = 0; c < nchunk; ++c) {
+            const float sc = rescale(wtab[h * nchunk + c], Mx);
+            Lx += wtab[G * nchunk + h * nchunk + c] * sc;
+            wtab[h * nchunk + c] = sc;
+        }
+        const float inv = 1.0f / Lx;
+        for (uint32_t c = 0; c < nchunk; ++c) wtab[h * nchunk + c] *= inv;
+    }
+    consumer_bar();
+    constexpr int MC = 24;   // chunks per pass
+    constexpr int ME = 3;    // outputs per thread and pass
+    for (uint32_t t0 = 0; t0 < G * hd; t0 += NCT * ME) {
+        for (uint32_t c0 = 0; c0 < nchunk; c0 += MC) {
+            float aa[ME][MC];
+#pragma unroll
+            for (int e = 0; e < ME; ++e) {
+                const uint32_t t = t0 + ctid + e * NCT;
+                const uint32_t h = t / hd, d = t % hd;
+#pragma unroll
+                for (int c = 0; c < MC; ++c) {
+                    aa[e][c] = 0.f;
+                    if (t < G * hd && c0 + c < nchunk) aa[e][c] = __ldcg(p.part + ((size_t)(unit0 + c0 + c) * G + h) * hd + d);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < ME; ++e) {
+                const uint32_t t = t0 + ctid + e * NCT;
+                if (t < G * hd) {
+                    const uint32_t h = t / hd, d = t % hd;
+                    float Ax = 0.f;
+#pragma unroll
+                    for (int c = 0; c < MC; ++c)
+                        if (c0 + c < nchunk) Ax += aa[e][c] * wtab[h * nchunk + c0 + c];
+                    float* dst = p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d;
+                    *dst = (c0 == 0 ? 0.f : *dst) + Ax;
+                }
+            }
         }
     }
 }
@@ -1032,12 +1108,14 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
 // arrive through the ring (in flight while the QKV stage and its counter wait were still running); the last CTA
 // to finish a (b, g) merges its chunks.  Scores use q pre-multiplied by log2(e)/sqrt(hd): the softmax runs in
 // base 2.  GT > 0 selects the CUDA-core inner loop for GT query heads per KV head; GT == 0 the tensor-core loop.
+// Returns the weight with which this CTA signals the end of the stage: the last unit of a (sequence, kv head) to
+// arrive merges the chunks and signals for all of them; the other units of that group do not signal at all (their
+// only fence is the ticket), CTAs without a unit and single-chunk units signal for themselves.
 template <int GT>
-__device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
-                                                uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
-                                                uint64_t pol) {
+__device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+                                                 uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
     const AttnUnit u = attn_unit(p, cta);
-    if (!u.active) return;
+    if (!u.active) return 1u;
     const uint32_t G = GT > 0 ? (uint32_t)GT : p.G;
     const uint32_t hd = p.hd, half = hd >> 1;
     const uint32_t b = u.b, g = u.g, pos = u.pos, nchunk = u.nchunk;
@@ -1046,15 +1124,14 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     float* q_s = s.vec;                         // [G][hd]
     float* new_k = q_s + G * hd;                // [hd]
     float* new_v = new_k + hd;                  // [hd]
-    float* comb = new_v + hd;                   // [NCW][G][hd + 2]
-    uint8_t* stage_k = reinterpret_cast<uint8_t*>(comb + (size_t)NCW * G * (hd + 2));  // [hd/64][16 rows][128 B]
-    uint8_t* stage_v = stage_k + hd * 32u;
+    // Staging "tile" of the position written by this step: only row 0 of each 64-column box is ever valid, so the
+    // boxes are packed 128 bytes apart; the 15 ignored rows the tile loop also reads overlap whatever follows.
+    uint8_t* stage_k = reinterpret_cast<uint8_t*>(new_v + hd);   // [hd/64][128 B]
+    uint8_t* stage_v = stage_k + 256;
+    float* comb = reinterpret_cast<float*>(stage_v + 256);       // [NCW][G][hd + 2]
 
     const float* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
     const float* cs = p.rope_cs + (size_t)b * hd;  // [half][2]
-    __nv_bfloat16* Kc = const_cast<__nv_bfloat16*>(kv_head(p, layer, 0, b, g));
-    __nv_bfloat16* Vc = const_cast<__nv_bfloat16*>(kv_head(p, layer, 1, b, g));
-
     const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
     for (uint32_t idx = ctid; idx < G * half; idx += NCT) {
         const uint32_t h = idx / half, i = idx % half;
@@ -1067,27 +1144,24 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     if (u.has_new) {
         const float* kr = qkv + p.QD + (size_t)g * hd;
         const float* vr = qkv + p.QD + p.KVD + (size_t)g * hd;
-        // row 0 of a swizzled box is stored unswizzled: column k of box k/64 sits at byte (k % 64) * 2
+            // row 0 of a swizzled box is stored unswizzled: column k of box k/64 sits at byte (k % 64) * 2 of the box
         for (uint32_t i = ctid; i < half; i += NCT) {
             const float a = __ldcg(kr + i), bb = __ldcg(kr + i + half);
             const float c = cs[2 * i], sn = cs[2 * i + 1];
             const __nv_bfloat16 k0 = __float2bfloat16_rn(a * c - bb * sn);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(bb * c + a * sn);
-            Kc[(size_t)pos * hd + i] = k0;
-            Kc[(size_t)pos * hd + i + half] = k1;
-            new_k[i] = __bfloat162float(k0);
+            new_k[i] = __bfloat162float(k0);   // the cache row itself is written after the stage (attention_flush_new_row)
             new_k[i + half] = __bfloat162float(k1);
             if (GT == 0) {
                 const uint32_t j = i + half;
-                *reinterpret_cast<__nv_bfloat16*>(stage_k + (i >> 6) * 2048u + (i & 63u) * 2u) = k0;
-                *reinterpret_cast<__nv_bfloat16*>(stage_k + (j >> 6) * 2048u + (j & 63u) * 2u) = k1;
+                *reinterpret_cast<__nv_bfloat16*>(stage_k + (i >> 6) * 128u + (i & 63u) * 2u) = k0;
+                *reinterpret_cast<__nv_bfloat16*>(stage_k + (j >> 6) * 128u + (j & 63u) * 2u) = k1;
             }
         }
         for (uint32_t d = ctid; d < hd; d += NCT) {
             const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(vr + d));
-            Vc[(size_t)pos * hd + d] = v0;
             new_v[d] = __bfloat162float(v0);
-            if (GT == 0) *reinterpret_cast<__nv_bfloat16*>(stage_v + (d >> 6) * 2048u + (d & 63u) * 2u) = v0;
+            if (GT == 0) *reinterpret_cast<__nv_bfloat16*>(stage_v + (d >> 6) * 128u + (d & 63u) * 2u) = v0;
         }
     }
     consumer_bar();
@@ -1096,9 +1170,9 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     const uint32_t first = rc.first_chunk(warp, p.nslots);
     if constexpr (GT == 0) {
         if (hd == 128)
-            attn_chunks_tc<128>(p, s, u, cta, warp, lane, first, rc, wr, pol, q_s, comb, stage_k, stage_v);
+            attn_chunks_tc<128>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
         else
-            attn_chunks_tc<64>(p, s, u, cta, warp, lane, first, rc, wr, pol, q_s, comb, stage_k, stage_v);
+            attn_chunks_tc<64>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
     } else {
         constexpr int G_ = GT > 0 ? GT : 1;
         const uint32_t lpp = hd >> 3;           // lanes per position
@@ -1127,10 +1201,11 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
         const uint32_t pb = attn_positions_per_chunk(p);
         for (uint32_t i = (warp < p.nslots ? first : u.nring); i < u.nring; i += p.nslots) {
             if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
-            mbar_wait(p, s, smem_u32(&s.full[warp]), wr.uses & 1u);
+            const uint32_t slot = warp * p.nsw + wr.cslot;
+            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
             if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
-            ++wr.uses;
-            const uint8_t* kp = s.ring + (size_t)warp * SLOT_BYTES;
+            ring_advance_consume(p, wr);
+            const uint8_t* kp = s.ring + (size_t)slot * SLOT_BYTES;
             const uint8_t* vp = kp + SLOT_BYTES / 2;
             const uint32_t np = min(pb, u.cend - (u.c0 + i * pb));
             constexpr int U = (G_ <= 4) ? 4 : 2;
@@ -1148,7 +1223,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
                 attn_batch<G_, U>(st, q, kk, vv, ok, lpp);
             }
             __syncwarp();
-            ring_issue_next(p, s, wr, warp, lane, pol);
+            ring_release(p, s, wr, warp, lane);
             if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
         }
         if (u.has_new && first == 0) {
@@ -1228,7 +1303,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
             }
         }
     }
-    if (nchunk == 1) return;
+    if (nchunk == 1) return 1u;
 
     // ticket: the last unit of (b, g) to arrive merges all chunks
     consumer_bar();
@@ -1237,32 +1312,44 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
         *s.bcast = (old == nchunk - 1) ? 1 : 0;
     }
     consumer_bar();
-    if (*s.bcast == 0) return;
-    const uint32_t unit0 = u.bg * p.cps;
-    for (uint32_t t = ctid; t < G * hd; t += NCT) {
-        const uint32_t h = t / hd, d = t % hd;
-        float Mx = -INFINITY;
-#pragma unroll 8
-        for (uint32_t c = 0; c < nchunk; ++c) Mx = fmaxf(Mx, __ldcg(p.part_ml + ((size_t)(unit0 + c) * G + h) * 2));
-        float Ax = 0.f, Lx = 0.f;
-#pragma unroll 8
-        for (uint32_t c = 0; c < nchunk; ++c) {
-            const size_t uu = (size_t)(unit0 + c) * G + h;
-            const float sc = rescale(__ldcg(p.part_ml + uu * 2), Mx);
-            Ax += __ldcg(p.part + uu * hd + d) * sc;
-            Lx += __ldcg(p.part_ml + uu * 2 + 1) * sc;
-        }
-        p.o[(size_t)b * p.QD + (size_t)(g * G + h) * hd + d] = Ax / Lx;
+    if (*s.bcast == 0) return 0u;
+    attn_merge(p, u, G, ctid, comb);
+    return nchunk;
+}
+
+// Appends the K/V row of the position written by this step to the cache (16-byte stores).  Nothing in the running
+// kernel reads that row from memory -- the unit that owns it works from the shared-memory copy -- so the store is
+// kept off the stage's critical path: it runs after the CTA has signalled, and before the shared-memory copy is
+// overwritten by the next stage's input vector.
+__device__ __forceinline__ void attention_flush_new_row(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+                                                        uint32_t ctid) {
+    const AttnUnit u = attn_unit(p, cta);
+    if (!u.active || !u.has_new) return;
+    const uint32_t hd = p.hd;
+    const float* new_k = s.vec + p.G * hd;
+    const float* new_v = new_k + hd;
+    const uint32_t per = hd / 8;
+    if (ctid < 2 * per) {
+        const uint32_t which = ctid / per, j = (ctid % per) * 8;
+        const float* src = (which ? new_v : new_k) + j;
+        uint4 v;
+        v.x = (__float_as_uint(src[0]) >> 16) | (__float_as_uint(src[1]) & 0xffff0000u);
+        v.y = (__float_as_uint(src[2]) >> 16) | (__float_as_uint(src[3]) & 0xffff0000u);
+        v.z = (__float_as_uint(src[4]) >> 16) | (__float_as_uint(src[5]) & 0xffff0000u);
+        v.w = (__float_as_uint(src[6]) >> 16) | (__float_as_uint(src[7]) & 0xffff0000u);
+        __nv_bfloat16* row = const_cast<__nv_bfloat16*>(kv_head(p, layer, which, u.b, u.g)) + (size_t)u.pos * hd + j;
+        *reinterpret_cast<uint4*>(row) = v;
     }
 }
 
 // Runs the attention stage and moves the ring cursor past the unit's chunks (also for CTAs without a unit).
 template <int GT>
-__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
-                                                            uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
-                                                            WarpRing& wr, uint64_t pol) {
-    attention_stage<GT>(p, s, layer, cta, ctid, warp, lane, rc, wr, pol);
+__device__ __forceinline__ uint32_t attention_stage_and_advance(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+                                                                uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
+                                                                WarpRing& wr) {
+    const uint32_t weight = attention_stage<GT>(p, s, layer, cta, ctid, warp, lane, rc, wr);
     rc.advance(attn_unit(p, cta).nring, p.nslots);
+    return weight;
 }
 
 }  // namespace kl
