@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libkl.so"
 SOURCES = [CSRC / "kl.cu"]
-HEADERS = [CSRC / "kl_device.cuh", PKG.parent / "include" / "kl.h"]
+HEADERS = [CSRC / "kl_device.cuh", CSRC / "kl_attention_tc.cuh", PKG.parent / "include" / "kl.h"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
@@ -27,7 +27,8 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, "-o", str(tmp), *map(str, SOURCES)]
+    extra = os.environ.get("KL_NVCC_FLAGS", "").split()   # e.g. -DKL_MAX_KP=4096 for tuning experiments
+    cmd = [nvcc, *NVCC_FLAGS, *extra, "-o", str(tmp), *map(str, SOURCES)]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

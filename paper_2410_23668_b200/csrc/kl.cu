@@ -32,7 +32,8 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
         atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
     if (tok < 0 || tok >= (int32_t)p.V) tok = 0;
     const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
-    for (uint32_t i = tid; i < p.H; i += blockDim.x) p.x[(size_t)b * p.H + i] = __bfloat162float(row[i]);
+    const uint32_t xtag = tag_of(p, 0, TG_XA);
+    for (uint32_t i = tid; i < p.H; i += blockDim.x) st_tw(p.xa + (size_t)b * p.H + i, __bfloat162float(row[i]), xtag);
     // RoPE table of this step: angle in double so that large positions keep their phase
     for (uint32_t i = tid; i < p.hd / 2; i += blockDim.x) {
         double sn, cs;
@@ -40,10 +41,8 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
         p.rope_cs[((size_t)b * (p.hd / 2) + i) * 2] = (float)cs;
         p.rope_cs[((size_t)b * (p.hd / 2) + i) * 2 + 1] = (float)sn;
     }
-    if (b == 0) {
-        const uint32_t nw = p.L * 8 + p.L * p.B * p.nkv;  // counters, then tickets (contiguous)
-        for (uint32_t i = tid; i < nw; i += blockDim.x) p.counters[i] = 0u;
-    }
+    if (b == 0)
+        for (uint32_t i = tid; i < p.L; i += blockDim.x) p.counters[i] = 0u;
 }
 
 // Layers [l0, l1) of the decoder.  l1 - l0 == L is the looped kernel; l1 - l0 == 1 the per-layer launch.
@@ -78,54 +77,60 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     RingCursor rc = {0u, 0u};
     for (uint32_t l = l0; l < l1; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
-        uint32_t* ctr = p.counters + (size_t)l * 8;
+        // test hook: the results of one stage of layer 0 get a tag nobody waits for
         const int skip = (l == 0) ? p.skip_stage : -1;
-        // S1: RMSNorm + QKV projection.  The hidden state of the previous layer must be complete.
-        if (l > l0) stage_wait(p, s, p.counters + (size_t)(l - 1) * 8 + ST_D, p.P, ctid);
+        const uint32_t bad = 0x2u;
+        // S1: RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the embedding).
         trace_stamp(p, cta, l, 0, ctid);
-        load_vec(p, s, p.x, p.H, true, p.g1 + lo, ctid);
+        load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
         trace_stamp(p, cta, l, 1, ctid);
-        gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, p.qkv, cta, warp, lane, rc, wr, nullptr);
-        stage_signal(ctr + ST_QKV, ctid, skip == ST_QKV);
-        trace_stamp(p, cta, l, 2, ctid);
-        // S2: RoPE, KV append, split-K attention, merge
-        stage_wait(p, s, ctr + ST_QKV, p.P, ctid);
-        trace_stamp(p, cta, l, 3, ctid);
-        uint32_t aw;
-        if (p.attn_tc) {
-            aw = attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
-        } else switch (p.G) {
-            case 1: aw = attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            case 2: aw = attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            case 4: aw = attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            default: aw = attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        {
+            const GemvOut out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
+            gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, out, cta, warp, lane, rc, wr, nullptr);
         }
-        stage_signal(ctr + ST_ATTN, ctid, skip == ST_ATTN, aw);
+        trace_stamp(p, cta, l, 2, ctid);
+        trace_stamp(p, cta, l, 3, ctid);
+        // S2: RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
+        if (p.attn_tc) {
+            attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
+        } else switch (p.G) {
+            case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+            default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        }
+        consumer_bar();
         attention_flush_new_row(p, s, l, cta, ctid);
         trace_stamp(p, cta, l, 4, ctid);
-        // S3: output projection + residual
-        stage_wait(p, s, ctr + ST_ATTN, p.P, ctid);
+        // S3: output projection + residual (xa -> xb).  The poll on o's tags waits for the mergers.
+        load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
         trace_stamp(p, cta, l, 5, ctid);
-        load_vec(p, s, p.o, p.QD, false, nullptr, ctid);
         trace_stamp(p, cta, l, 6, ctid);
-        gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, nullptr);
-        stage_signal(ctr + ST_O, ctid, skip == ST_O);
+        {
+            const GemvOut out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, l, TG_XB)};
+            gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, out, cta, warp, lane, rc, wr, nullptr);
+        }
         trace_stamp(p, cta, l, 7, ctid);
         // S4: RMSNorm + gate/up projections + SwiGLU
-        stage_wait(p, s, ctr + ST_O, p.P, ctid);
+        load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
         trace_stamp(p, cta, l, 8, ctid);
-        load_vec(p, s, p.x, p.H, true, p.g2 + lo, ctid);
         trace_stamp(p, cta, l, 9, ctid);
-        gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, p.h, cta, warp, lane, rc, wr, nullptr);
-        stage_signal(ctr + ST_GU, ctid, skip == ST_GU);
+        {
+            const GemvOut out = {nullptr, p.h, nullptr, 0u};
+            gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, out, cta, warp, lane, rc, wr, nullptr);
+        }
+        // h is plain fp32 read per warp and per column piece straight from L2 into registers (too wide for tagged
+        // words): its readiness is a counter, signalled with release and awaited with acquire
+        stage_signal(p.counters + l, ctid, skip == ST_GU);
         trace_stamp(p, cta, l, 10, ctid);
-        // S5: down projection + residual
-        stage_wait(p, s, ctr + ST_GU, p.P, ctid);
+        stage_wait(p, s, p.counters + l, p.P, ctid);
         trace_stamp(p, cta, l, 11, ctid);
         trace_stamp(p, cta, l, 12, ctid);
-        // h is read per warp and per column piece straight from L2 into registers (no shared-memory staging)
-        gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, p.x, cta, warp, lane, rc, wr, p.h);
-        stage_signal(ctr + ST_D, ctid, skip == ST_D);
+        // S5: down projection + residual (xb -> xa of the next layer)
+        {
+            const GemvOut out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
+            gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, out, cta, warp, lane, rc, wr, p.h);
+        }
         trace_stamp(p, cta, l, 13, ctid);
     }
 }
@@ -155,8 +160,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     const uint64_t pol = 0;
     WarpRing wr = ring_begin();
     RingCursor rc = {0u, 0u};
-    load_vec(p, s, p.x, p.H, true, p.gf, tid);
-    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, p.logits, cta, warp, lane, rc, wr, nullptr);
+    load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, tid);
+    const GemvOut out = {nullptr, p.logits, nullptr, 0u};
+    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr);
 }
 
 // Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per
@@ -258,7 +264,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sx, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, scratch_bytes;
     uint32_t cps;
 };
 
@@ -297,15 +303,17 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     const uint32_t G = d.n_q_heads / d.n_kv_heads;
     const size_t units = (size_t)num_sms;  // at most one attention unit per CTA
     size_t s = 0;
-    y.sx = s;        s += align_up(B * H * 4);
-    y.sqkv = s;      s += align_up(B * (QD + 2 * KVD) * 4);
-    y.so = s;        s += align_up(B * QD * 4);
+    // tagged words (8 bytes each): xa, xb, qkv, o, split-K partials; h is plain fp32
+    y.sxa = s;       s += align_up(B * H * 8);
+    y.sxb = s;       s += align_up(B * H * 8);
+    y.sqkv = s;      s += align_up(B * (QD + 2 * KVD) * 8);
+    y.so = s;        s += align_up(B * QD * 8);
     y.sh = s;        s += align_up(B * F * 4);
-    y.spart = s;     s += align_up(units * G * d.head_dim * 4);
-    y.spart_ml = s;  s += align_up(units * G * 2 * 4);
+    y.spart = s;     s += align_up(units * G * d.head_dim * 8);
+    y.spart_ml = s;  s += align_up(units * G * 2 * 8);
     y.srope = s;     s += align_up(B * d.head_dim * 4);
     y.sinvf = s;     s += align_up((size_t)(d.head_dim / 2) * 8);
-    y.scounters = s; s += align_up(((size_t)d.n_layers * 8 + (size_t)d.n_layers * B * d.n_kv_heads) * 4);
+    y.scounters = s; s += align_up((size_t)d.n_layers * 4);
     y.sstatus = s;   s += ALIGN;
     y.stok = s;      s += align_up(B * 4);
     y.spos = s;      s += align_up(B * 4);
@@ -348,7 +356,7 @@ GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t alig
         pl.npieces = ceil_div(K, pl.kp);
         uint32_t rpc = SLOT_BYTES / (pl.kp * 2);
         if (rpc > (uint32_t)MAX_RPC_SPLIT) rpc = MAX_RPC_SPLIT;
-        if (pairs) rpc = 2;
+        if (pairs) rpc &= ~1u;
         while (align && rpc > 1 && align % rpc) --rpc;
         if (rpc < 1) rpc = 1;
         pl.rpc = rpc;
@@ -364,7 +372,6 @@ bool plans_ok(const Params& p) {
         if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
         if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % 256)) return false;
         if (i == PL_GU && (pl.rpc & 1u)) return false;
-        if (i == PL_GU && pl.npieces > 1 && pl.rpc != 2) return false;
     }
     return true;
 }
@@ -386,9 +393,15 @@ cudaError_t store_rows(const GemvPlan& pl, __nv_bfloat16* mat, const __nv_bfloat
         const size_t c0 = (size_t)j * pl.kp;
         const size_t len = (j == pl.npieces - 1) ? K - c0 : pl.kp;
         if (vstep == 2) {
-            // units of two rows (gate f, up f): this tensor fills row v0 of every unit
-            e = cudaMemcpy2DAsync(mat + rpc * c0 + (size_t)v0 * len, rpc * K * 2, src + c0, K * 2, len * 2, rows,
-                                  cudaMemcpyDefault, st);
+            // units of rpc/2 (gate f, up f) row pairs: source row s of this tensor is row 2 * (s % (rpc/2)) + v0 of
+            // unit s / (rpc/2)
+            const size_t ppu = rpc / 2;
+            for (size_t t = 0; t < ppu && e == cudaSuccess; ++t) {
+                if (rows <= t) break;
+                const size_t cnt = (rows - t + ppu - 1) / ppu;
+                e = cudaMemcpy2DAsync(mat + rpc * c0 + (2 * t + v0) * len, rpc * K * 2, src + t * K + c0, ppu * K * 2,
+                                      len * 2, cnt, cudaMemcpyDefault, st);
+            }
             continue;
         }
         const size_t u_first = v0 / rpc;
@@ -525,11 +538,11 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.wqkv = w + y.off_qkv; p.wo = w + y.off_o; p.wgu = w + y.off_gu; p.wd = w + y.off_d;
     p.g1 = w + y.off_g1; p.g2 = w + y.off_g2; p.gf = w + y.off_gf; p.wlm = w + y.off_lm; p.embed = w + y.off_embed;
     uint8_t* sc = h->scratch;
-    p.x = (float*)(sc + y.sx); p.qkv = (float*)(sc + y.sqkv); p.o = (float*)(sc + y.so); p.h = (float*)(sc + y.sh);
-    p.part = (float*)(sc + y.spart); p.part_ml = (float*)(sc + y.spart_ml); p.rope_cs = (float*)(sc + y.srope);
+    p.xa = (TW*)(sc + y.sxa); p.xb = (TW*)(sc + y.sxb); p.qkv = (TW*)(sc + y.sqkv); p.o = (TW*)(sc + y.so);
+    p.h = (float*)(sc + y.sh);
+    p.part = (TW*)(sc + y.spart); p.part_ml = (TW*)(sc + y.spart_ml); p.rope_cs = (float*)(sc + y.srope);
     p.inv_freq = (const double*)(sc + y.sinvf);
     p.counters = (uint32_t*)(sc + y.scounters);
-    p.tickets = p.counters + (size_t)p.L * 8;
     p.status = (int32_t*)(sc + y.sstatus);
     h->stage_tokens = (int32_t*)(sc + y.stok);
     h->stage_positions = (int32_t*)(sc + y.spos);
@@ -653,6 +666,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     p.logits = logits_d;
     p.skip_stage = h->pending_skip_stage;
     h->pending_skip_stage = -1;
+    p.step = ++h->prm.step;
     p.attn_tc = 0;
     if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
         const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, batch);
@@ -712,7 +726,9 @@ kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens
 
 kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream) {
     if (!h || !hidden_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
-    if (cudaMemcpyAsync(hidden_d, h->prm.x, (size_t)batch * h->prm.H * 4, cudaMemcpyDeviceToDevice, as_stream(stream)) != cudaSuccess)
+    // the hidden state leaving the last layer is an array of tagged words: take the value half of each
+    if (cudaMemcpy2DAsync(hidden_d, 4, h->prm.xa, 8, 4, (size_t)batch * h->prm.H, cudaMemcpyDeviceToDevice, as_stream(stream)) !=
+        cudaSuccess)
         return KL_ERR_CUDA;
     return KL_OK;
 }

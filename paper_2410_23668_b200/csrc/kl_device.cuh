@@ -45,7 +45,10 @@ struct GemvPlan {
     uint32_t npieces;
     uint32_t nunits;
 };
-constexpr uint32_t MAX_KP = 4096;           // columns per chunk piece: 16 blocks of 256, 8 per lane and block
+#ifndef KL_MAX_KP
+#define KL_MAX_KP 2560
+#endif
+constexpr uint32_t MAX_KP = KL_MAX_KP;      // columns per chunk piece: blocks of 256, 8 per lane and block
 constexpr int MAX_XB = MAX_KP / 256;
 
 struct Params {
@@ -66,10 +69,14 @@ struct Params {
     __nv_bfloat16* kv;
     const int32_t* tokens;
     const int32_t* positions;
-    float *x, *qkv, *o, *h, *part, *part_ml, *rope_cs, *logits;
+    // activations that cross CTAs.  xa, xb, qkv, o and the split-K partials are arrays of tagged words (see TW):
+    // xa = hidden state entering a layer, xb = hidden state after the attention half.  h (the MLP's inner vector) is
+    // plain fp32 guarded by a counter.
+    struct TW *xa, *xb, *qkv, *o, *part, *part_ml;
+    float *h, *rope_cs, *logits;
+    uint32_t step;         // decode steps issued on this handle so far (makes the tags of every step distinct)
     const double* inv_freq;
-    uint32_t* counters;    // [L][8]
-    uint32_t* tickets;     // [L][B*nkv]
+    uint32_t* counters;    // [L]: CTAs that have finished the gate/up stage of each layer
     int32_t* status;
     unsigned long long* trace;  // optional [P][L][TRACE_STAMPS] globaltimer stamps of consumer thread 0, or null
     unsigned long long* chunk_trace;  // optional [CHUNK_TRACE_ROWS][4] per-chunk stamps of CTA 0 (issue, wait, full, done)
@@ -148,6 +155,41 @@ __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
                  : "l"(p));
     return v;
 }
+// A value that crosses CTAs travels with its own flag: one aligned 8-byte word {fp32 value, 32-bit tag}, written
+// with a single 64-bit store and read with 64-bit (or 2 x 64-bit) loads that bypass L1.  A reader that sees the
+// tag it expects has the value -- no fence on the writer's side, no counter to poll, one L2 round trip on the
+// reader's side.  Tags are odd numbers built from (decode step, layer, stage), so a word left over from an earlier
+// layer or step never matches, and neither does zero-initialised memory.
+struct __align__(8) TW {
+    float v;
+    uint32_t tag;
+};
+// Every tagged word is moved by one 64-bit access (value in the low half, tag in the high half): a single aligned
+// 64-bit access is never torn, so the tag cannot be seen without its value.  The accesses are strong (relaxed at gpu
+// scope): a weak load inside a polling loop may legally be hoisted out of it by the assembler.
+__device__ __forceinline__ void st_tw(TW* p, float v, uint32_t tag) {
+    const uint64_t w = ((uint64_t)tag << 32) | __float_as_uint(v);
+    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
+}
+__device__ __forceinline__ TW ld_tw(const TW* p) {
+    uint64_t r;
+    asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(r) : "l"(p) : "memory");
+    TW w;
+    w.v = __uint_as_float((uint32_t)r);
+    w.tag = (uint32_t)(r >> 32);
+    return w;
+}
+// two consecutive words (16-byte aligned): x, y = value and tag of the first, z, w of the second
+__device__ __forceinline__ uint4 ld_tw2(const TW* p) {
+    uint64_t a, b;
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+    return make_uint4((uint32_t)a, (uint32_t)(a >> 32), (uint32_t)b, (uint32_t)(b >> 32));
+}
+enum TagSlot { TG_XA = 0, TG_QKV = 1, TG_PART = 2, TG_O = 3, TG_XB = 4 };
+__device__ __forceinline__ uint32_t tag_of(const Params& p, uint32_t layer, uint32_t slot) {
+    return ((((p.step * p.L + layer) << 3) + slot) << 1) | 1u;
+}
+
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
@@ -185,9 +227,16 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
 // Records the first error and tells every waiter of this CTA to give up.  After an abort every wait returns at
 // once but the control flow (stage order, CTA barriers) is unchanged, so no warp is left behind at a barrier; the
 // step's outputs are then meaningless and the status word says so.
-__device__ __forceinline__ void raise_abort(const Params& p, const Smem& s, int code) {
-    atomicCAS(p.status, 0, code);
+__device__ __forceinline__ bool raise_abort(const Params& p, const Smem& s, int code, int where = 0) {
+    bool first = false;
+    if (atomicCAS(p.status, 0, code) == 0) {   // following words: which wait gave up, where (diagnostics)
+        p.status[1] = where;
+        p.status[2] = (int)blockIdx.x;
+        p.status[3] = (int)threadIdx.x;
+        first = true;
+    }
     *s.abort_flag = 1;
+    return first;
 }
 
 // Bounded mbarrier wait.  Returns false when the wait was abandoned (limit reached or abort raised elsewhere).
@@ -200,9 +249,33 @@ __device__ __forceinline__ bool mbar_wait(const Params& p, const Smem& s, uint32
         if ((++it & 63u) == 0) {
             if (*s.abort_flag) return false;
             if (globaltimer_ns() - t0 > p.wait_ns) {
-                raise_abort(p, s, ERR_SYNC_TIMEOUT);
+                raise_abort(p, s, ERR_SYNC_TIMEOUT, 500);
                 return false;
             }
+        }
+    }
+    return true;
+}
+
+// Bookkeeping of a bounded polling loop on tagged words or counters.  poll_continue() returns false when the loop
+// must be abandoned: another waiter of the CTA gave up, a kernel of this step flagged an error, or the limit ran out.
+struct PollGuard {
+    uint64_t t0;
+    uint32_t it;
+    int where;
+};
+__device__ __forceinline__ bool poll_continue(const Params& p, const Smem& s, PollGuard& g) {
+    if (g.it == 0) g.t0 = globaltimer_ns();
+    __nanosleep(64);   // keeps the polling traffic of a waiting CTA off the L2 ports the late CTAs still need
+    if ((++g.it & 7u) == 0) {
+        if (*s.abort_flag) return false;
+        if (__ldcg(p.status) != 0) {
+            *s.abort_flag = 1;
+            return false;
+        }
+        if (globaltimer_ns() - g.t0 > p.wait_ns) {
+            raise_abort(p, s, ERR_SYNC_TIMEOUT, g.where);
+            return false;
         }
     }
     return true;
@@ -500,65 +573,57 @@ __device__ __forceinline__ uint32_t vec_perm(uint32_t e) {
     return (e & ~255u) + (((e >> 2) & 1u) << 7) + (((e >> 3) & 31u) << 2) + (e & 3u);
 }
 
-// Loads src[0..n) (fp32, produced by other CTAs: read through L2) into the shared vector area, optionally
-// applying RMSNorm with bf16 gains.  Every CTA recomputes the norm; the summation order is fixed.
-__device__ __forceinline__ void load_vec(const Params& p, const Smem& s, const float* src, uint32_t n, bool norm,
+// Loads the tagged vector src[0..n) (produced by other CTAs) into the shared vector area, polling until every word
+// carries `tag`, and optionally applies RMSNorm with bf16 gains.  Every CTA recomputes the norm; the summation
+// order is fixed.  This poll is what replaces the grid-wide barrier of a kernel boundary: the first read that finds
+// all tags in place already holds the data.
+__device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
                                          const __nv_bfloat16* gain, uint32_t ctid) {
-    constexpr int NB = 8;  // float4 loads kept in flight per thread: one L2 round trip per NB * NCT * 4 elements
-    if (norm && n <= (uint32_t)(NB * NCT * 4)) {
-        // whole vector in registers: x and gains are fetched together, one round trip before the reduction
-        float4 v[NB];
-        uint2 gb[NB];
-#pragma unroll
-        for (int i = 0; i < NB; ++i) {
-            const uint32_t e = (ctid + i * NCT) * 4;
-            v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            gb[i] = make_uint2(0u, 0u);
-            if (e < n) {
-                v[i] = __ldcg(reinterpret_cast<const float4*>(src + e));
-                gb[i] = __ldg(reinterpret_cast<const uint2*>(gain + e));
-            }
-        }
-        float ss = 0.f;
-#pragma unroll
-        for (int i = 0; i < NB; ++i) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if ((ctid & 31) == 0) s.red[ctid >> 5] = ss;
-        consumer_bar();
-        float tot = 0.f;
-#pragma unroll
-        for (int w = 0; w < NCW; ++w) tot += s.red[w];
-        const float inv = rsqrtf(tot / (float)n + p.eps);
-#pragma unroll
-        for (int i = 0; i < NB; ++i) {
-            const uint32_t e = (ctid + i * NCT) * 4;
-            if (e < n) {
-                float4 o;
-                o.x = v[i].x * inv * bf_lo(gb[i].x);
-                o.y = v[i].y * inv * bf_hi(gb[i].x);
-                o.z = v[i].z * inv * bf_lo(gb[i].y);
-                o.w = v[i].w * inv * bf_hi(gb[i].y);
-                *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = o;
-            }
-        }
-        consumer_bar();
-        return;
-    }
+    constexpr int NB = 6;  // groups of four values kept in flight per thread (two 16-byte loads each)
     float ss = 0.f;
+    const bool single = n <= (uint32_t)(NB * NCT * 4);
+    float4 keep[NB];
+    uint2 gkeep[NB];
     for (uint32_t base = 0; base < n; base += NB * NCT * 4) {
         float4 v[NB];
+        if (norm && single) {
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+                const uint32_t e = (ctid + i * NCT) * 4;
+                gkeep[i] = make_uint2(0u, 0u);
+                if (e < n) gkeep[i] = __ldg(reinterpret_cast<const uint2*>(gain + e));
+            }
+        }
+        // Only the groups whose tags are not all in place yet are read again: the words that are late come from the
+        // few CTAs that finish the previous stage last, and re-reading the whole vector from every waiting CTA
+        // floods the L2 slices those late CTAs stream their weights through.
+        uint32_t pend = 0u;
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
-            const uint32_t e = base + (ctid + i * NCT) * 4;
             v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (e < n) v[i] = __ldcg(reinterpret_cast<const float4*>(src + e));
+            if (base + (ctid + i * NCT) * 4 < n) pend |= 1u << i;
+        }
+        PollGuard pg = {0ull, 0u, (int)(tag & 15u) + 100};
+        for (;;) {
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+                if ((pend >> i) & 1u) {
+                    const uint32_t e = base + (ctid + i * NCT) * 4;
+                    const uint4 a = ld_tw2(src + e), b = ld_tw2(src + e + 2);
+                    if (a.y == tag && a.w == tag && b.y == tag && b.w == tag) {
+                        v[i] = make_float4(__uint_as_float(a.x), __uint_as_float(a.z), __uint_as_float(b.x), __uint_as_float(b.z));
+                        pend &= ~(1u << i);
+                    }
+                }
+            }
+            if (pend == 0u || !poll_continue(p, s, pg)) break;
         }
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
             const uint32_t e = base + (ctid + i * NCT) * 4;
             ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
-            if (e < n) *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = v[i];
+            if (norm && single) keep[i] = v[i];
+            else if (e < n) *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = v[i];
         }
     }
     if (norm) {
@@ -570,21 +635,35 @@ __device__ __forceinline__ void load_vec(const Params& p, const Smem& s, const f
 #pragma unroll
         for (int w = 0; w < NCW; ++w) tot += s.red[w];
         const float inv = rsqrtf(tot / (float)n + p.eps);
-        for (uint32_t e = ctid * 4; e < n; e += NCT * 4) {
-            float4* q = reinterpret_cast<float4*>(s.vec + vec_perm(e));
-            const uint2 gb = __ldg(reinterpret_cast<const uint2*>(gain + e));
-            float4 v = *q;
-            v.x *= inv * bf_lo(gb.x);
-            v.y *= inv * bf_hi(gb.x);
-            v.z *= inv * bf_lo(gb.y);
-            v.w *= inv * bf_hi(gb.y);
-            *q = v;
+        if (single) {
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+                const uint32_t e = (ctid + i * NCT) * 4;
+                if (e < n) {
+                    float4 o;
+                    o.x = keep[i].x * inv * bf_lo(gkeep[i].x);
+                    o.y = keep[i].y * inv * bf_hi(gkeep[i].x);
+                    o.z = keep[i].z * inv * bf_lo(gkeep[i].y);
+                    o.w = keep[i].w * inv * bf_hi(gkeep[i].y);
+                    *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = o;
+                }
+            }
+        } else {
+            for (uint32_t e = ctid * 4; e < n; e += NCT * 4) {
+                float4* q = reinterpret_cast<float4*>(s.vec + vec_perm(e));
+                const uint2 gb = __ldg(reinterpret_cast<const uint2*>(gain + e));
+                float4 v = *q;
+                v.x *= inv * bf_lo(gb.x);
+                v.y *= inv * bf_hi(gb.x);
+                v.z *= inv * bf_lo(gb.y);
+                v.w *= inv * bf_hi(gb.y);
+                *q = v;
+            }
         }
     }
     consumer_bar();
 }
 
-// acc[r] += sum over this lane's columns of W[r][k] * vec[k]; W rows in shared memory, row pitch rowbytes.
 // This lane's share of a slice of the input vector: for block b of 256 columns the 8 columns b*256 + lane*8 .. +7.
 struct XRegs {
     float v[MAX_XB][8];
@@ -644,7 +723,7 @@ __device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t pitch, uint3
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const uint32_t k = (uint32_t)(b0 + u) * 256u + lane * 8u;
-                const bool in = k < klen;                   // false only in or after the last, partial block
+                const bool in = b0 + u < MAX_XB && k < klen;   // false only in or after the last, partial block
                 const uint32_t kk = in ? k : 0u;
 #pragma unroll
                 for (int r = 0; r < NR; ++r) {
@@ -654,7 +733,7 @@ __device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t pitch, uint3
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int b = b0 + u;
+                const int b = b0 + u < MAX_XB ? b0 + u : MAX_XB - 1;   // blocks past the end hold zero weights
 #pragma unroll
                 for (int r = 0; r < NR; ++r) {
                     e[r] = fmaf(bf_lo(q[u][r].x), x.v[b][0], e[r]);
@@ -704,8 +783,13 @@ __device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, 
 template <int NR>
 __device__ __forceinline__ void dot_n(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane, const XRegs& x,
                                       float (&acc)[NR]) {
+    if constexpr (MAX_XB >= 16) {
+        if (klen == 4096) {
+            dot_rows_full<NR, (MAX_XB >= 16 ? 16 : 1)>(w, pitch, lane, x, acc);
+            return;
+        }
+    }
     switch (klen) {
-        case 4096: dot_rows_full<NR, 16>(w, pitch, lane, x, acc); break;
         case 2560: dot_rows_full<NR, 10>(w, pitch, lane, x, acc); break;
         case 2048: dot_rows_full<NR, 8>(w, pitch, lane, x, acc); break;
         default: dot_rows<NR>(w, pitch, klen, lane, x, acc); break;
@@ -743,7 +827,21 @@ struct RingCursor {
 // same warp, in order, so a parity wait can never be satisfied by a phase two uses old.  (With free chunk-to-warp
 // assignment a fast warp can test the barrier of use k while use k-1 is still in flight, and parity k&1 then
 // reads as complete.)
-__device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, float* out,
+// Where a stage's results go.  Tagged outputs (`tw`) are read by other CTAs of the running kernel; `plain` outputs are
+// only read after the kernel (logits) or are guarded by a counter (h).  `res` is the tagged vector the residual is
+// taken from: this CTA validated all of its tags when it loaded the vector at the start of an earlier stage.
+struct GemvOut {
+    TW* tw;
+    float* plain;
+    const TW* res;
+    uint32_t tag;
+};
+__device__ __forceinline__ void emit_value(const GemvOut& o, uint32_t idx, float v) {
+    if (o.tw) st_tw(o.tw + idx, v, o.tag);
+    else o.plain[idx] = v;
+}
+
+__device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
                                         uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
                                         const float* xsrc) {
     // xsrc == nullptr: the input vector is staged in s.vec; otherwise it is read from global memory per piece
@@ -766,7 +864,7 @@ __device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const Ge
             // one unit piece of up to four rows: the common case.  Residual inputs are fetched before the wait, their
             // L2 latency hides behind it.
             float res = 0.f;
-            if (ep == EP_RESIDUAL && lane < g.nrows) res = __ldcg(out + g.row + lane);
+            if (ep == EP_RESIDUAL && lane < g.nrows) res = ld_tw(out.res + g.row + lane).v;
             mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
             if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
@@ -821,12 +919,12 @@ __device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const Ge
                 }
                 if (emit) {
                     if (ep == EP_SWIGLU) {
-                        out[g.row >> 1] = silu(y[0]) * y[1];
-                        if (g.nrows == 4) out[(g.row >> 1) + 1] = silu(y[2]) * y[3];
+                        emit_value(out, g.row >> 1, silu(y[0]) * y[1]);
+                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2]) * y[3]);
                     } else {
 #pragma unroll
                         for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
-                            if ((uint32_t)rr < g.nrows) out[g.row + rr] = (ep == EP_RESIDUAL ? rs[rr] : 0.f) + y[rr];
+                            if ((uint32_t)rr < g.nrows) emit_value(out, g.row + rr, (ep == EP_RESIDUAL ? rs[rr] : 0.f) + y[rr]);
                     }
                 }
             }
@@ -839,8 +937,8 @@ __device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const Ge
                 const bool two = rr + 1 < g.nrows;
                 float rs0 = 0.f, rs1 = 0.f;
                 if (ep == EP_RESIDUAL && lane == 0) {
-                    rs0 = __ldcg(out + g.row + rr);
-                    if (two) rs1 = __ldcg(out + g.row + rr + 1);
+                    rs0 = ld_tw(out.res + g.row + rr).v;
+                    if (two) rs1 = ld_tw(out.res + g.row + rr + 1).v;
                 }
                 float y0, y1 = 0.f;
                 if (two) {
@@ -856,13 +954,13 @@ __device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const Ge
                 if (lane == 0) {
                     const uint32_t row = g.row + rr;
                     if (ep == EP_STORE) {
-                        out[row] = y0;
-                        if (two) out[row + 1] = y1;
+                        emit_value(out, row, y0);
+                        if (two) emit_value(out, row + 1, y1);
                     } else if (ep == EP_RESIDUAL) {
-                        out[row] = rs0 + y0;
-                        if (two) out[row + 1] = rs1 + y1;
+                        emit_value(out, row, rs0 + y0);
+                        if (two) emit_value(out, row + 1, rs1 + y1);
                     } else {
-                        out[row >> 1] = silu(y0) * y1;
+                        emit_value(out, row >> 1, silu(y0) * y1);
                     }
                 }
             }
@@ -895,7 +993,7 @@ __device__ __forceinline__ void stage_wait(const Params& p, const Smem& s, const
                         break;
                     }
                     if (globaltimer_ns() - t0 > p.wait_ns) {
-                        raise_abort(p, s, ERR_SYNC_TIMEOUT);
+                        raise_abort(p, s, ERR_SYNC_TIMEOUT, 600);
                         break;
                     }
                 }
@@ -1042,20 +1140,41 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
     }
 }
 
-// Merges the split-K partial results of one (sequence, kv head) into the attention output o (run by the unit that
-// arrived last, after every other unit of the group has published its partial result).
-__device__ __noinline__ void attn_merge(const Params& p, const AttnUnit& u, uint32_t G, uint32_t ctid, float* comb) {
+// Two tagged words that may lie apart, polled until both carry `tag` (bounded).
+__device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const TW* a, const TW* b, uint32_t tag, float& va,
+                                          float& vb) {
+    PollGuard pg = {0ull, 0u, 200 + (int)(tag >> 4) * 1000};
+    for (;;) {
+        const TW x = ld_tw(a), y = ld_tw(b);
+        va = x.v;
+        vb = y.v;
+        if ((x.tag == tag && y.tag == tag) || !poll_continue(p, s, pg)) return;
+    }
+}
+
+// Merges the split-K partial results of one (sequence, kv head) into the attention output o.  Run by the unit that
+// holds the group's last chunk; the partial results of the other units are tagged words, polled until they are all
+// there.  Two passes: the (max, sum) pairs of every (head, chunk), turned into weights
+// w[h][c] = exp2(m_c - M_h) / L_h in shared memory; then the weighted sum of the partial outputs, with the loads of up
+// to three outputs per thread in flight at once.  The orders of all sums are fixed.
+__device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const AttnUnit& u, uint32_t layer, uint32_t G,
+                                        uint32_t ctid, float* comb) {
     const uint32_t hd = p.hd, b = u.b, g = u.g, nchunk = u.nchunk;
     const uint32_t unit0 = u.bg * p.cps;
-    // Merge in two L2 round trips.  First the (max, sum) pairs of every (head, chunk): one per thread, turned into
-    // weights w[h][c] = exp2(m_c - M_h) / L_h in shared memory.  Then the weighted sum of the partial outputs, with
-    // all the loads of up to three outputs per thread in flight at once.  The orders of all sums are fixed.
+    const uint32_t tag = tag_of(p, layer, TG_PART), otag = tag_of(p, layer, TG_O);
     float* wtab = comb;   // [2][G][nchunk]; the per-warp partials in comb are no longer needed
+    consumer_bar();
     for (uint32_t t = ctid; t < G * nchunk; t += NCT) {
         const uint32_t h = t / nchunk, c = t % nchunk;
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(unit0 + c) * G + h) * 2));
-        wtab[t] = ml.x;
-        wtab[G * nchunk + t] = ml.y;
+        const TW* src = p.part_ml + ((size_t)(unit0 + c) * G + h) * 2;
+        uint4 ml;
+        PollGuard pg = {0ull, 0u, 300};
+        for (;;) {
+            ml = ld_tw2(src);
+            if ((ml.y == tag && ml.w == tag) || !poll_continue(p, s, pg)) break;
+        }
+        wtab[t] = __uint_as_float(ml.x);
+        wtab[G * nchunk + t] = __uint_as_float(ml.z);
     }
     consumer_bar();
     if (ctid < G) {
@@ -1072,33 +1191,50 @@ __device__ __noinline__ void attn_merge(const Params& p, const AttnUnit& u, uint
         for (uint32_t c = 0; c < nchunk; ++c) wtab[h * nchunk + c] *= inv;
     }
     consumer_bar();
-    constexpr int MC = 24;   // chunks per pass
+    constexpr int MC = 12;   // chunks per pass
     constexpr int ME = 3;    // outputs per thread and pass
     for (uint32_t t0 = 0; t0 < G * hd; t0 += NCT * ME) {
+        float acc[ME];
+#pragma unroll
+        for (int e = 0; e < ME; ++e) acc[e] = 0.f;
         for (uint32_t c0 = 0; c0 < nchunk; c0 += MC) {
             float aa[ME][MC];
+            PollGuard pg = {0ull, 0u, 400};
+            for (;;) {
+                bool ok = true;
 #pragma unroll
-            for (int e = 0; e < ME; ++e) {
-                const uint32_t t = t0 + ctid + e * NCT;
-                const uint32_t h = t / hd, d = t % hd;
+                for (int e = 0; e < ME; ++e) {
+                    const uint32_t t = t0 + ctid + e * NCT;
+                    const uint32_t h = t / hd, d = t % hd;
 #pragma unroll
-                for (int c = 0; c < MC; ++c) {
-                    aa[e][c] = 0.f;
-                    if (t < G * hd && c0 + c < nchunk) aa[e][c] = __ldcg(p.part + ((size_t)(unit0 + c0 + c) * G + h) * hd + d);
+                    for (int c = 0; c < MC; ++c) {
+                        aa[e][c] = 0.f;
+                        if (t < G * hd && c0 + c < nchunk) {
+                            const TW w = ld_tw(p.part + ((size_t)(unit0 + c0 + c) * G + h) * hd + d);
+                            aa[e][c] = w.v;
+                            ok = ok && w.tag == tag;
+                        }
+                    }
                 }
+                if (ok || !poll_continue(p, s, pg)) break;
             }
 #pragma unroll
             for (int e = 0; e < ME; ++e) {
                 const uint32_t t = t0 + ctid + e * NCT;
                 if (t < G * hd) {
-                    const uint32_t h = t / hd, d = t % hd;
-                    float Ax = 0.f;
+                    const uint32_t h = t / hd;
 #pragma unroll
                     for (int c = 0; c < MC; ++c)
-                        if (c0 + c < nchunk) Ax += aa[e][c] * wtab[h * nchunk + c0 + c];
-                    float* dst = p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d;
-                    *dst = (c0 == 0 ? 0.f : *dst) + Ax;
+                        if (c0 + c < nchunk) acc[e] += aa[e][c] * wtab[h * nchunk + c0 + c];
                 }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < ME; ++e) {
+            const uint32_t t = t0 + ctid + e * NCT;
+            if (t < G * hd) {
+                const uint32_t h = t / hd, d = t % hd;
+                st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, acc[e], otag);
             }
         }
     }
@@ -1130,23 +1266,28 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
     uint8_t* stage_v = stage_k + 256;
     float* comb = reinterpret_cast<float*>(stage_v + 256);       // [NCW][G][hd + 2]
 
-    const float* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
+    // q (and, for the unit that owns the new position, k and v) of this step: tagged words written by whichever CTAs
+    // own those rows of the QKV projection.  The unit waits for exactly the rows it needs, not for the whole stage.
+    const TW* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
+    const uint32_t qtag = tag_of(p, layer, TG_QKV);
     const float* cs = p.rope_cs + (size_t)b * hd;  // [half][2]
     const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
     for (uint32_t idx = ctid; idx < G * half; idx += NCT) {
         const uint32_t h = idx / half, i = idx % half;
-        const float* qr = qkv + (size_t)(g * G + h) * hd;
-        const float a = __ldcg(qr + i), bb = __ldcg(qr + i + half);
+        const TW* qr = qkv + (size_t)(g * G + h) * hd;
+        float a, bb;
+        poll_pair(p, s, qr + i, qr + i + half, qtag, a, bb);
         const float c = cs[2 * i], sn = cs[2 * i + 1];
         q_s[h * hd + i] = (a * c - bb * sn) * qscale;
         q_s[h * hd + i + half] = (bb * c + a * sn) * qscale;
     }
     if (u.has_new) {
-        const float* kr = qkv + p.QD + (size_t)g * hd;
-        const float* vr = qkv + p.QD + p.KVD + (size_t)g * hd;
-            // row 0 of a swizzled box is stored unswizzled: column k of box k/64 sits at byte (k % 64) * 2 of the box
+        const TW* kr = qkv + p.QD + (size_t)g * hd;
+        const TW* vr = qkv + p.QD + p.KVD + (size_t)g * hd;
+        // row 0 of a swizzled box is stored unswizzled: column k of box k/64 sits at byte (k % 64) * 2 of the box
         for (uint32_t i = ctid; i < half; i += NCT) {
-            const float a = __ldcg(kr + i), bb = __ldcg(kr + i + half);
+            float a, bb;
+            poll_pair(p, s, kr + i, kr + i + half, qtag, a, bb);
             const float c = cs[2 * i], sn = cs[2 * i + 1];
             const __nv_bfloat16 k0 = __float2bfloat16_rn(a * c - bb * sn);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(bb * c + a * sn);
@@ -1159,7 +1300,9 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
             }
         }
         for (uint32_t d = ctid; d < hd; d += NCT) {
-            const __nv_bfloat16 v0 = __float2bfloat16_rn(__ldcg(vr + d));
+            float va, vb;
+            poll_pair(p, s, vr + d, vr + d, qtag, va, vb);
+            const __nv_bfloat16 v0 = __float2bfloat16_rn(va);
             new_v[d] = __bfloat162float(v0);
             if (GT == 0) *reinterpret_cast<__nv_bfloat16*>(stage_v + (d >> 6) * 128u + (d & 63u) * 2u) = v0;
         }
@@ -1294,27 +1437,21 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
             Lsum += src[hd + 1] * c;
         }
         if (nchunk == 1) {
-            p.o[(size_t)b * p.QD + (size_t)(g * G + h) * hd + d] = A / Lsum;
+            st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, A / Lsum, tag_of(p, layer, TG_O));
         } else {
-            p.part[((size_t)unit * G + h) * hd + d] = A;
+            const uint32_t ptag = tag_of(p, layer, TG_PART);
+            st_tw(p.part + ((size_t)unit * G + h) * hd + d, A, ptag);
             if (d == 0) {
-                p.part_ml[((size_t)unit * G + h) * 2] = M;
-                p.part_ml[((size_t)unit * G + h) * 2 + 1] = Lsum;
+                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, M, ptag);
+                st_tw(p.part_ml + ((size_t)unit * G + h) * 2 + 1, Lsum, ptag);
             }
         }
     }
-    if (nchunk == 1) return 1u;
-
-    // ticket: the last unit of (b, g) to arrive merges all chunks
-    consumer_bar();
-    if (ctid == 0) {
-        const uint32_t old = atom_add_acq_rel(p.tickets + (size_t)layer * p.B * p.nkv + u.bg, 1u);
-        *s.bcast = (old == nchunk - 1) ? 1 : 0;
-    }
-    consumer_bar();
-    if (*s.bcast == 0) return 0u;
-    attn_merge(p, u, G, ctid, comb);
-    return nchunk;
+    // The unit that holds the group's last chunk (the one with the new position) merges; the others are done: their
+    // partial results carry their own flags, there is nothing to signal and nothing to wait for.
+    if (nchunk == 1 || u.ch != nchunk - 1) return 0u;
+    attn_merge(p, s, u, layer, G, ctid, comb);
+    return 0u;
 }
 
 // Appends the K/V row of the position written by this step to the cache (16-byte stores).  Nothing in the running
