@@ -36,7 +36,8 @@ enum {
     KL_ERR_NOT_LOADED = -3,        /* kl_decode_step before every tensor was loaded */
     KL_ERR_CUDA = -4,              /* a CUDA runtime call failed */
     KL_ERR_SYNC_TIMEOUT = -5,      /* a bounded device-side wait ran out (reported by kl_last_status) */
-    KL_ERR_OUT_OF_RANGE = -6       /* token >= vocab or position >= max_ctx seen on the device */
+    KL_ERR_OUT_OF_RANGE = -6,      /* token >= vocab or position >= max_ctx seen on the device */
+    KL_ERR_TOO_LARGE = -7          /* a size beyond the fixed capacity of kl_argmax_advance_static */
 };
 
 enum { KL_MODE_LOOPED = 0, KL_MODE_PER_LAYER = 1 };
@@ -109,6 +110,28 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
 /* Sampling block (greedy): tokens_d[b] = argmax_v logits_d[b, v] (lowest index on ties); positions_d[b] += 1. */
 kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d,
                             uint32_t batch, void* stream);
+
+/* The same sampling block for callers that cannot give the library any memory to work in and must not cause an
+ * allocation: a sampler that runs on logits produced elsewhere and holds no kl_handle (so there is no scratch arena
+ * to carve from), or a serving loop in which a device allocation would synchronise the device or fail because the
+ * process has already committed all device memory to its own pools.  The paper has no counterpart of this entry
+ * point; it describes the sampling block only as one of the calls around the looped decoder (Section 3.2).
+ *
+ * The per-block partial results and the completion tickets live in a fixed array that is part of the library
+ * image (KL_STATIC_ARGMAX_MAX_BATCH sequences, about 130 KB per device); nothing is allocated or freed, here or
+ * inside the CUDA runtime routines this call uses (a symbol-address query, a memset node and a kernel launch).
+ *   logits_d    [batch, vocab] fp32 on the current device
+ *   tokens_d    [batch] int32, written: argmax (lowest index on ties)
+ *   positions_d [batch] int32, incremented
+ *   batch       1..KL_STATIC_ARGMAX_MAX_BATCH; larger -> KL_ERR_TOO_LARGE, nothing is launched
+ * The first call on a device looks up the array's address (with that device current): make that first call outside
+ * any stream capture, before the latency-critical part of the program.  Every call on a device shares the one
+ * array, which keeps whatever the previous call left; the call itself clears the tickets it is about to use, in
+ * stream order.  Two calls that may run at the same time on one device (different streams, or different host
+ * threads without ordering) would race on the array: order them. */
+#define KL_STATIC_ARGMAX_MAX_BATCH 256
+kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_t* tokens_d, int32_t* positions_d,
+                                   uint32_t batch, void* stream);
 
 /* Copies the hidden state after the last decoder layer (before the final RMSNorm) of the latest step:
  * hidden_d [batch, hidden] fp32. */

@@ -18,6 +18,8 @@ KL_ERR_NOT_LOADED = -3
 KL_ERR_CUDA = -4
 KL_ERR_SYNC_TIMEOUT = -5
 KL_ERR_OUT_OF_RANGE = -6
+KL_ERR_TOO_LARGE = -7
+KL_STATIC_ARGMAX_MAX_BATCH = 256
 KL_MODE_LOOPED = 0
 KL_MODE_PER_LAYER = 1
 
@@ -28,7 +30,7 @@ TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup":
 EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_bytes", "kl_set_mode", "kl_decode_step",
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
-           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention")
+           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static")
 
 
 class ModelDesc(C.Structure):
@@ -67,6 +69,8 @@ def lib():
     l.kl_decode_step_host.restype = i32
     l.kl_argmax_advance.argtypes = [vp, vp, vp, vp, u32, vp]
     l.kl_argmax_advance.restype = i32
+    l.kl_argmax_advance_static.argtypes = [vp, u32, vp, vp, u32, vp]
+    l.kl_argmax_advance_static.restype = i32
     l.kl_read_hidden.argtypes = [vp, vp, u32, vp]
     l.kl_read_hidden.restype = i32
     l.kl_last_status.argtypes = [vp]
@@ -125,6 +129,12 @@ def _ptr(t) -> int:
 
 def _stream_ptr(stream) -> int:
     return 0 if stream is None else int(stream.cuda_stream)
+
+
+def kl_argmax_advance_static(logits_d, tokens_d, positions_d, batch: int, stream=None) -> None:
+    """Sampling block without a handle: scratch in a fixed array inside the library, nothing is allocated."""
+    _check(lib().kl_argmax_advance_static(_ptr(logits_d), int(logits_d.shape[-1]), _ptr(tokens_d), _ptr(positions_d), batch,
+                                          _stream_ptr(stream)), "kl_argmax_advance_static")
 
 
 class Decoder:

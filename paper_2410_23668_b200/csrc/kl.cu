@@ -16,6 +16,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "../../include/kl.h"
@@ -432,6 +433,7 @@ const char* kl_status_string(kl_status s) {
         case KL_ERR_CUDA: return "KL_ERR_CUDA";
         case KL_ERR_SYNC_TIMEOUT: return "KL_ERR_SYNC_TIMEOUT";
         case KL_ERR_OUT_OF_RANGE: return "KL_ERR_OUT_OF_RANGE";
+        case KL_ERR_TOO_LARGE: return "KL_ERR_TOO_LARGE";
         default: return "KL_ERR_UNKNOWN";
     }
 }
@@ -721,6 +723,51 @@ kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens
                                                                                  h->argmax_val, h->argmax_idx, h->argmax_tickets);
     if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
     ++h->launches;
+    return KL_OK;
+}
+
+// ---- sampling block without a handle and without any allocation.
+// Some callers have no arena to lend: a sampler working on logits that came from elsewhere owns no kl_handle, and a
+// serving process that has handed all device memory to its own pools can neither afford the device-wide
+// synchronisation of an allocation nor expect it to succeed.  For them the partial results and the tickets of the
+// argmax kernel sit in the array below, which is part of the module image on every device that loads it.
+// Layout: [MAX_BATCH][ARGMAX_BLOCKS] fp32 maxima | [MAX_BATCH][ARGMAX_BLOCKS] u32 indices | [MAX_BATCH] u32 tickets.
+namespace {
+constexpr size_t STATIC_ARGMAX_PART = (size_t)KL_STATIC_ARGMAX_MAX_BATCH * ARGMAX_BLOCKS * 4;
+constexpr size_t STATIC_ARGMAX_BYTES = 2 * STATIC_ARGMAX_PART + (size_t)KL_STATIC_ARGMAX_MAX_BATCH * 4;
+constexpr int STATIC_MAX_DEVICES = 64;
+}  // namespace
+static __device__ __align__(256) unsigned char kl_static_argmax_scratch[STATIC_ARGMAX_BYTES];
+static unsigned char* g_static_argmax_ptr[STATIC_MAX_DEVICES];   // per device; written once under the mutex
+static std::mutex g_static_argmax_mutex;
+
+kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_t* tokens_d, int32_t* positions_d,
+                                   uint32_t batch, void* stream) {
+    if (!logits_d || !tokens_d || !positions_d || batch == 0 || vocab == 0) return KL_ERR_INVALID_ARG;
+    if (batch > (uint32_t)KL_STATIC_ARGMAX_MAX_BATCH) return KL_ERR_TOO_LARGE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KL_ERR_CUDA;
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return KL_ERR_INVALID_ARG;
+    unsigned char* base;
+    {
+        // set-up, once per device, with that device current: the address of this device's copy of the array
+        std::lock_guard<std::mutex> lock(g_static_argmax_mutex);
+        if (!g_static_argmax_ptr[dev]) {
+            unsigned char* ptr = nullptr;
+            if (cudaGetSymbolAddress((void**)&ptr, kl_static_argmax_scratch) != cudaSuccess || !ptr) return KL_ERR_CUDA;
+            g_static_argmax_ptr[dev] = ptr;
+        }
+        base = g_static_argmax_ptr[dev];
+    }
+    float* part_val = reinterpret_cast<float*>(base);
+    uint32_t* part_idx = reinterpret_cast<uint32_t*>(base + STATIC_ARGMAX_PART);
+    uint32_t* tickets = reinterpret_cast<uint32_t*>(base + 2 * STATIC_ARGMAX_PART);
+    cudaStream_t st = as_stream(stream);
+    // the array keeps what the previous call left; only the tickets have to start at zero
+    if (cudaMemsetAsync(tickets, 0, (size_t)batch * 4, st) != cudaSuccess) return KL_ERR_CUDA;
+    kl_argmax_kernel<<<dim3(ARGMAX_BLOCKS, batch), 256, 0, st>>>(logits_d, vocab, tokens_d, positions_d, part_val, part_idx,
+                                                                  tickets);
+    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
 }
 
