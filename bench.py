@@ -337,7 +337,10 @@ def run_ours(args, shape, batch, context):
                 "d2h_bytes_per_step": 4 * shape.vocab * batch},
         "roofline": {"bound": "hbm", "kernel": "kl_decoder_kernel (looped, all layers)", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": None, "bytes_per_launch": bytes_dec,
+                     "peak_source": peaks["source"], "traffic": ncu_traffic(shape, batch, context),
+                     "traffic_source": "ncu dram bytes read+written of a 4-layer launch, scaled by layers/4 "
+                                       "(profiles/kl_decoder_kernel_llama31_8b_4layers_b1_ctx4096.txt)",
+                     "bytes_per_launch": bytes_dec,
                      "ms_per_launch": dec_avg_ms, "classifier_ms": statistics.mean(cls_ms)},
         "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_looped / K * 1e-3) / 1e9,
                        "frac_of_measured_copy": bytes_step / (ms_looped / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -357,6 +360,20 @@ def run_ours(args, shape, batch, context):
         print(json.dumps(line))
     if world > 1:
         torch.distributed.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one looped launch over 4 layers of the 8B shape at batch 1,
+# context 4096 (ncu capture summarised under profiles/), per layer.  Every layer streams its own weights and KV once,
+# so a full launch is this times the layer count.
+NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813641e9 + 27.529728e6) / 4
+
+
+def ncu_traffic(shape, batch, context):
+    """Bytes per looped launch, from the committed ncu capture; None for workloads that were not captured."""
+    if batch == 1 and context == 4096 and (shape.hidden, shape.ffn, shape.n_q_heads, shape.n_kv_heads, shape.head_dim) == \
+            (4096, 14336, 32, 8, 128):
+        return NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 * shape.n_layers
+    return None
 
 
 def main():
