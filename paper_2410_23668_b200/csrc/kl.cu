@@ -46,6 +46,21 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
         for (uint32_t i = tid; i < p.L; i += blockDim.x) p.counters[i] = 0u;
 }
 
+// The attention half of a layer as one call: RoPE, the unit's ring chunks, the merges, the deferred cache append.
+__device__ __noinline__ void attention_block(const Params& p, const Smem& s, uint32_t l, uint32_t cta, uint32_t ctid,
+                                             uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
+    if (p.attn_tc) {
+        attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
+    } else switch (p.G) {
+        case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+    }
+    consumer_bar();
+    attention_flush_new_row(p, s, l, cta, ctid);
+}
+
 // Layers [l0, l1) of the decoder.  l1 - l0 == L is the looped kernel; l1 - l0 == 1 the per-layer launch.
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -76,61 +91,59 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     // ---------------- consumers
     const uint32_t ctid = tid;
     RingCursor rc = {0u, 0u};
+    // One call site for the GEMV stage, inlined here: the hot loop lives in the kernel's own frame and the cold parts
+    // (vector loads with their polls, the attention block) are calls made between stages, when nothing is live.
     for (uint32_t l = l0; l < l1; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         // test hook: the results of one stage of layer 0 get a tag nobody waits for
         const int skip = (l == 0) ? p.skip_stage : -1;
         const uint32_t bad = 0x2u;
-        // S1: RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the embedding).
-        trace_stamp(p, cta, l, 0, ctid);
-        load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
-        trace_stamp(p, cta, l, 1, ctid);
-        {
-            const GemvOut out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
-            gemv_stage(p, s, p.plan[PL_QKV], EP_STORE, out, cta, warp, lane, rc, wr, nullptr);
-        }
-        trace_stamp(p, cta, l, 2, ctid);
-        trace_stamp(p, cta, l, 3, ctid);
-        // S2: RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
-        if (p.attn_tc) {
-            attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
-        } else switch (p.G) {
-            case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-            default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-        }
-        consumer_bar();
-        attention_flush_new_row(p, s, l, cta, ctid);
-        trace_stamp(p, cta, l, 4, ctid);
-        // S3: output projection + residual (xa -> xb).  The poll on o's tags waits for the mergers.
-        load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
-        trace_stamp(p, cta, l, 5, ctid);
-        trace_stamp(p, cta, l, 6, ctid);
-        {
-            const GemvOut out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, l, TG_XB)};
-            gemv_stage(p, s, p.plan[PL_O], EP_RESIDUAL, out, cta, warp, lane, rc, wr, nullptr);
-        }
-        trace_stamp(p, cta, l, 7, ctid);
-        // S4: RMSNorm + gate/up projections + SwiGLU
-        load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
-        trace_stamp(p, cta, l, 8, ctid);
-        trace_stamp(p, cta, l, 9, ctid);
-        {
-            const GemvOut out = {nullptr, p.h, nullptr, 0u};
-            gemv_stage(p, s, p.plan[PL_GU], EP_SWIGLU, out, cta, warp, lane, rc, wr, nullptr);
-        }
-        // h is plain fp32 read per warp and per column piece straight from L2 into registers (too wide for tagged
-        // words): its readiness is a counter, signalled with release and awaited with acquire
-        stage_signal(p.counters + l, ctid, skip == ST_GU);
-        trace_stamp(p, cta, l, 10, ctid);
-        stage_wait(p, s, p.counters + l, p.P, ctid);
-        trace_stamp(p, cta, l, 11, ctid);
-        trace_stamp(p, cta, l, 12, ctid);
-        // S5: down projection + residual (xb -> xa of the next layer)
-        {
-            const GemvOut out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
-            gemv_stage(p, s, p.plan[PL_D], EP_RESIDUAL, out, cta, warp, lane, rc, wr, p.h);
+        for (int st = 0; st < 4; ++st) {
+            GemvOut out;
+            int plan, ep;
+            const float* xsrc = nullptr;
+            if (st == 0) {
+                // S1: RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the
+                // embedding).
+                trace_stamp(p, cta, l, 0, ctid);
+                load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
+                trace_stamp(p, cta, l, 1, ctid);
+                out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
+                plan = PL_QKV;
+                ep = EP_STORE;
+            } else if (st == 1) {
+                trace_stamp(p, cta, l, 2, ctid); trace_stamp(p, cta, l, 3, ctid);
+                // S2: RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
+                attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
+                trace_stamp(p, cta, l, 4, ctid); trace_stamp(p, cta, l, 5, ctid);
+                // S3: output projection + residual (xa -> xb).  The poll on o's tags waits for the mergers.
+                load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
+                trace_stamp(p, cta, l, 6, ctid);
+                out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, l, TG_XB)};
+                plan = PL_O;
+                ep = EP_RESIDUAL;
+            } else if (st == 2) {
+                trace_stamp(p, cta, l, 7, ctid); trace_stamp(p, cta, l, 8, ctid);
+                // S4: RMSNorm + gate/up projections + SwiGLU
+                load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
+                trace_stamp(p, cta, l, 9, ctid);
+                out = {nullptr, p.h, nullptr, 0u};
+                plan = PL_GU;
+                ep = EP_SWIGLU;
+            } else {
+                // h is plain fp32 read per warp and per column piece straight from L2 into registers (too wide for
+                // tagged words): its readiness is a counter, signalled with release and awaited with acquire
+                stage_signal(p.counters + l, ctid, skip == ST_GU);
+                trace_stamp(p, cta, l, 10, ctid);
+                stage_wait(p, s, p.counters + l, p.P, ctid);
+                trace_stamp(p, cta, l, 11, ctid); trace_stamp(p, cta, l, 12, ctid);
+                // S5: down projection + residual (xb -> xa of the next layer)
+                out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
+                plan = PL_D;
+                ep = EP_RESIDUAL;
+                xsrc = p.h;
+            }
+            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc);
         }
         trace_stamp(p, cta, l, 13, ctid);
     }
@@ -527,12 +540,14 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.nslots = NCW;
     p.nsw = (uint32_t)nsw;
     h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
-    if (cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) != cudaSuccess) {
-        free(h->loaded); delete h; return KL_ERR_CUDA;
-    }
+    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
+    if (ce == cudaSuccess)
+        ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes) != cudaSuccess || occ < 1) {
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes);
+    if (ce != cudaSuccess || occ < 1) {
+        fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
+                        "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
         free(h->loaded); delete h; return KL_ERR_CUDA;
     }
 

@@ -841,7 +841,7 @@ __device__ __forceinline__ void emit_value(const GemvOut& o, uint32_t idx, float
     else o.plain[idx] = v;
 }
 
-__device__ __noinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
+__device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
                                         uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
                                         const float* xsrc) {
     // xsrc == nullptr: the input vector is staged in s.vec; otherwise it is read from global memory per piece
