@@ -526,7 +526,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     uint32_t vecf = p.H > p.QD ? p.H : p.QD;  // the down projection reads its input from L2, not from this area
     vecf = ceil_div(vecf, 256) * 256;
     // attention workspace: rotated q, the new K/V row, per-warp partial results, the staging tile of the new row
-    const uint32_t attnf = p.G * p.hd + 2 * p.hd + 128 + NCW * p.G * (p.hd + 2);
+    // (the same area then holds the merge tables: 2 * G * nchunk pairs and the unit's slice of every partial output)
+    const uint32_t comb_f = NCW * p.G * (p.hd + 2), merge_f = 2 * p.G * (p.P / p.nkv) + p.G * p.hd + 2 * (p.P / p.nkv);  // batch 1 has the most chunks
+    const uint32_t attnf = p.G * p.hd + 2 * p.hd + 128 + (comb_f > merge_f ? comb_f : merge_f);
     if (attnf > vecf) vecf = ceil_div(attnf, 256) * 256;
     p.vec_floats = vecf;
     int max_optin = 0;

@@ -1152,29 +1152,61 @@ __device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const 
     }
 }
 
-// Merges the split-K partial results of one (sequence, kv head) into the attention output o.  Run by the unit that
-// holds the group's last chunk; the partial results of the other units are tagged words, polled until they are all
-// there.  Two passes: the (max, sum) pairs of every (head, chunk), turned into weights
-// w[h][c] = exp2(m_c - M_h) / L_h in shared memory; then the weighted sum of the partial outputs, with the loads of up
-// to three outputs per thread in flight at once.  The orders of all sums are fixed.
+// Merges the split-K partial results of one (sequence, kv head) into the attention output o.  Every unit of the
+// group merges its own slice of the G * hd outputs (unit c takes outputs [c*S, (c+1)*S), S = ceil(G*hd / nchunk)), so
+// the merge costs each unit a handful of loads that are all in flight at once -- one L2 round trip after the last
+// unit of the group has published its partial result -- instead of one unit reading everything in several passes.
+// The partial results are tagged words, polled until they are there.  Steps: the (max, sum) pairs of every
+// (head, chunk) and the unit's slice of every chunk's partial output go to shared memory; the pairs become weights
+// w[h][c] = exp2(m_c - M_h) / L_h; thread j adds its output's nchunk terms in chunk order.  The orders of all sums
+// are fixed.
 __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const AttnUnit& u, uint32_t layer, uint32_t G,
                                         uint32_t ctid, float* comb) {
     const uint32_t hd = p.hd, b = u.b, g = u.g, nchunk = u.nchunk;
     const uint32_t unit0 = u.bg * p.cps;
     const uint32_t tag = tag_of(p, layer, TG_PART), otag = tag_of(p, layer, TG_O);
-    float* wtab = comb;   // [2][G][nchunk]; the per-warp partials in comb are no longer needed
-    consumer_bar();
-    for (uint32_t t = ctid; t < G * nchunk; t += NCT) {
-        const uint32_t h = t / nchunk, c = t % nchunk;
-        const TW* src = p.part_ml + ((size_t)(unit0 + c) * G + h) * 2;
-        uint4 ml;
+    const uint32_t total = G * hd;
+    const uint32_t S = (total + nchunk - 1) / nchunk;
+    const uint32_t t_lo = min(total, u.ch * S), t_hi = min(total, t_lo + S);
+    const uint32_t ns = t_hi - t_lo;
+    float* wtab = comb;                      // [2][G][nchunk]: maxima, sums; then weights in the first half
+    float* pv = wtab + 2 * G * nchunk;       // [ns][nchunk] partial outputs of this unit's slice
+    consumer_bar();                          // the per-warp partials in comb are no longer needed
+    // all loads of a thread are issued before it waits on any of them; only those that are late are repeated
+    constexpr int NL = 4;
+    const uint32_t nml = G * nchunk, npv = ns * nchunk;
+    for (uint32_t i0 = 0; i0 < max(nml, (npv + NL - 1) / NL); i0 += NCT) {
+        const uint32_t i = i0 + ctid;
+        bool ml_pend = i < nml;
+        uint32_t pend = 0u;
+#pragma unroll
+        for (int k = 0; k < NL; ++k)
+            if (i * NL + k < npv) pend |= 1u << k;
         PollGuard pg = {0ull, 0u, 300};
-        for (;;) {
-            ml = ld_tw2(src);
-            if ((ml.y == tag && ml.w == tag) || !poll_continue(p, s, pg)) break;
+        while (ml_pend || pend) {
+            if (ml_pend) {
+                const uint32_t h = i / nchunk, c = i % nchunk;
+                const uint4 ml = ld_tw2(p.part_ml + ((size_t)(unit0 + c) * G + h) * 2);
+                if (ml.y == tag && ml.w == tag) {
+                    wtab[i] = __uint_as_float(ml.x);
+                    wtab[nml + i] = __uint_as_float(ml.z);
+                    ml_pend = false;
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < NL; ++k) {
+                if ((pend >> k) & 1u) {
+                    const uint32_t j = i * NL + k;
+                    const uint32_t t = t_lo + j / nchunk, c = j % nchunk;
+                    const TW w = ld_tw(p.part + (size_t)(unit0 + c) * total + t);
+                    if (w.tag == tag) {
+                        pv[j] = w.v;
+                        pend &= ~(1u << k);
+                    }
+                }
+            }
+            if ((ml_pend || pend) && !poll_continue(p, s, pg)) break;
         }
-        wtab[t] = __uint_as_float(ml.x);
-        wtab[G * nchunk + t] = __uint_as_float(ml.z);
     }
     consumer_bar();
     if (ctid < G) {
@@ -1184,59 +1216,18 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
         float Lx = 0.f;
         for (uint32_t c = 0; c < nchunk; ++c) {
             const float sc = rescale(wtab[h * nchunk + c], Mx);
-            Lx += wtab[G * nchunk + h * nchunk + c] * sc;
+            Lx += wtab[nml + h * nchunk + c] * sc;
             wtab[h * nchunk + c] = sc;
         }
         const float inv = 1.0f / Lx;
         for (uint32_t c = 0; c < nchunk; ++c) wtab[h * nchunk + c] *= inv;
     }
     consumer_bar();
-    constexpr int MC = 12;   // chunks per pass
-    constexpr int ME = 3;    // outputs per thread and pass
-    for (uint32_t t0 = 0; t0 < G * hd; t0 += NCT * ME) {
-        float acc[ME];
-#pragma unroll
-        for (int e = 0; e < ME; ++e) acc[e] = 0.f;
-        for (uint32_t c0 = 0; c0 < nchunk; c0 += MC) {
-            float aa[ME][MC];
-            PollGuard pg = {0ull, 0u, 400};
-            for (;;) {
-                bool ok = true;
-#pragma unroll
-                for (int e = 0; e < ME; ++e) {
-                    const uint32_t t = t0 + ctid + e * NCT;
-                    const uint32_t h = t / hd, d = t % hd;
-#pragma unroll
-                    for (int c = 0; c < MC; ++c) {
-                        aa[e][c] = 0.f;
-                        if (t < G * hd && c0 + c < nchunk) {
-                            const TW w = ld_tw(p.part + ((size_t)(unit0 + c0 + c) * G + h) * hd + d);
-                            aa[e][c] = w.v;
-                            ok = ok && w.tag == tag;
-                        }
-                    }
-                }
-                if (ok || !poll_continue(p, s, pg)) break;
-            }
-#pragma unroll
-            for (int e = 0; e < ME; ++e) {
-                const uint32_t t = t0 + ctid + e * NCT;
-                if (t < G * hd) {
-                    const uint32_t h = t / hd;
-#pragma unroll
-                    for (int c = 0; c < MC; ++c)
-                        if (c0 + c < nchunk) acc[e] += aa[e][c] * wtab[h * nchunk + c0 + c];
-                }
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < ME; ++e) {
-            const uint32_t t = t0 + ctid + e * NCT;
-            if (t < G * hd) {
-                const uint32_t h = t / hd, d = t % hd;
-                st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, acc[e], otag);
-            }
-        }
+    for (uint32_t j = ctid; j < ns; j += NCT) {
+        const uint32_t t = t_lo + j, h = t / hd, d = t % hd;
+        float acc = 0.f;
+        for (uint32_t c = 0; c < nchunk; ++c) acc += pv[j * nchunk + c] * wtab[h * nchunk + c];
+        st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, acc, otag);
     }
 }
 
@@ -1447,10 +1438,8 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
             }
         }
     }
-    // The unit that holds the group's last chunk (the one with the new position) merges; the others are done: their
-    // partial results carry their own flags, there is nothing to signal and nothing to wait for.
-    if (nchunk == 1 || u.ch != nchunk - 1) return 0u;
-    attn_merge(p, s, u, layer, G, ctid, comb);
+    // every unit of the group merges its slice of the outputs
+    if (nchunk > 1) attn_merge(p, s, u, layer, G, ctid, comb);
     return 0u;
 }
 
