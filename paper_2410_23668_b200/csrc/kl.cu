@@ -339,14 +339,15 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
 
 // `align`: units must not straddle multiples of `align` rows (sources that are concatenated row-wise, such as
 // Wq | Wk | Wv, start at multiples of it); 0 = no constraint.
-GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t align) {
+// `x_in_smem`: the stage's input vector is staged in shared memory, so whole rows of any length that fit a slot are fine.
+GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t align, bool x_in_smem) {
     GemvPlan pl;
     memset(&pl, 0, sizeof(pl));
     pl.R = R;
     pl.K = K;
     const uint32_t rowbytes = K * 2;
     const uint32_t minrows = pairs ? 2u : 1u;
-    if (K <= MAX_KP && rowbytes * minrows <= (uint32_t)SLOT_BYTES) {
+    if ((K <= MAX_KP || x_in_smem) && rowbytes * minrows <= (uint32_t)SLOT_BYTES) {
         // whole rows: as many as fit a slot, but keep at least ~2 chunks per CTA on small matrices
         uint32_t rpc = SLOT_BYTES / rowbytes;
         uint32_t cap = R / (2 * P);
@@ -382,7 +383,8 @@ GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t alig
 bool plans_ok(const Params& p) {
     for (int i = 0; i < PL_COUNT; ++i) {
         const GemvPlan& pl = p.plan[i];
-        if (pl.npieces > (uint32_t)MAX_PIECES || pl.kp > MAX_KP || pl.rpc < 1) return false;
+        if (pl.npieces > (uint32_t)MAX_PIECES || pl.rpc < 1) return false;
+        if (pl.kp > MAX_KP && (pl.npieces > 1 || i == PL_D || pl.rpc > (uint32_t)MAX_RPC_SPLIT)) return false;
         if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
         if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % 256)) return false;
         if (i == PL_GU && (pl.rpc & 1u)) return false;
@@ -515,11 +517,11 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.skip_stage = -1;
     p.wait_ns = 2000000000ull;
     p.layer_stride = y.layer_stride;
-    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD);  // KVD divides QD: Wq | Wk | Wv stay aligned
-    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P, 0);
-    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P, 0);
-    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0);
-    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0);
+    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD, true);  // KVD divides QD: Wq | Wk | Wv stay aligned
+    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P, 0, true);
+    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P, 0, true);
+    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0, false);
+    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0, true);
     if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
 
     // shared memory: input vector area (also the attention workspace), then as many ring slots as fit

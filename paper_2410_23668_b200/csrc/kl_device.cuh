@@ -796,6 +796,53 @@ __device__ __forceinline__ void dot_n(const uint8_t* w, uint32_t pitch, uint32_t
     }
 }
 
+// Whole rows with the input vector read from shared memory block by block (lane-permuted layout, see vec_perm):
+// for rows too long for a register-resident slice.  Per block of 256 columns a lane loads its 8 vector elements
+// (two conflict-free 16-byte loads) and one 16-byte piece of every row.  klen is a multiple of 8.
+template <int NR>
+__device__ __forceinline__ void dot_rows_smemx(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane,
+                                               const float* vec, float (&acc)[NR]) {
+    float e[NR], o[NR];
+#pragma unroll
+    for (int r = 0; r < NR; ++r) e[r] = o[r] = 0.f;
+    const float4* v4 = reinterpret_cast<const float4*>(vec) + lane;
+    const uint8_t* wl = w + (size_t)lane * 16;
+    const uint32_t nb = klen >> 8;
+#pragma unroll 4
+    for (uint32_t b = 0; b < nb; ++b) {
+        const float4 lo = v4[b * 64], hi = v4[b * 64 + 32];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+            const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)b * 512);
+            e[r] = fmaf(bf_lo(q.x), lo.x, e[r]);
+            o[r] = fmaf(bf_hi(q.x), lo.y, o[r]);
+            e[r] = fmaf(bf_lo(q.y), lo.z, e[r]);
+            o[r] = fmaf(bf_hi(q.y), lo.w, o[r]);
+            e[r] = fmaf(bf_lo(q.z), hi.x, e[r]);
+            o[r] = fmaf(bf_hi(q.z), hi.y, o[r]);
+            e[r] = fmaf(bf_lo(q.w), hi.z, e[r]);
+            o[r] = fmaf(bf_hi(q.w), hi.w, o[r]);
+        }
+    }
+    if ((klen & 255u) && nb * 256u + lane * 8u < klen) {   // last, partial block
+        const float4 lo = v4[nb * 64], hi = v4[nb * 64 + 32];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) {
+            const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)nb * 512);
+            e[r] = fmaf(bf_lo(q.x), lo.x, e[r]);
+            o[r] = fmaf(bf_hi(q.x), lo.y, o[r]);
+            e[r] = fmaf(bf_lo(q.y), lo.z, e[r]);
+            o[r] = fmaf(bf_hi(q.y), lo.w, o[r]);
+            e[r] = fmaf(bf_lo(q.z), hi.x, e[r]);
+            o[r] = fmaf(bf_hi(q.z), hi.y, o[r]);
+            e[r] = fmaf(bf_lo(q.w), hi.z, e[r]);
+            o[r] = fmaf(bf_hi(q.w), hi.w, o[r]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < NR; ++r) acc[r] = e[r] + o[r];
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -850,9 +897,11 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
     const uint32_t first = rc.first_chunk(warp, p.nslots);
     XRegs x;
     uint32_t x_piece = 0xffffffffu;
+    // rows that come whole and find their vector in shared memory are multiplied against it block by block
+    const bool smemx = xsrc == nullptr && pl.npieces == 1u && pl.rpc <= (uint32_t)MAX_RPC_SPLIT;
     for (uint32_t i = first; i < nch; i += p.nslots) {
         const ChunkGeom g = chunk_geom(pl, r.u0, i);
-        if (g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
+        if (!smemx && g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
             if (xsrc) load_xregs_global(x, xsrc, g.kofs, g.klen, lane);
             else load_xregs(x, s.vec, g.kofs, g.klen, lane);
             x_piece = g.piece;
@@ -860,7 +909,46 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
         const uint32_t slot = warp * p.nsw + wr.cslot;
         const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
         const uint32_t pitch = g.klen * 2u;
-        if (pl.rpc <= MAX_RPC_SPLIT) {
+        if (smemx) {
+            // Whole rows, the vector taken from shared memory block by block: no cross-warp combine, the warp that
+            // multiplied the rows emits them.
+            float res = 0.f;
+            if (ep == EP_RESIDUAL && lane < g.nrows) res = ld_tw(out.res + g.row + lane).v;
+            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            ring_advance_consume(p, wr);
+            float y[MAX_RPC_SPLIT] = {0.f, 0.f, 0.f, 0.f};
+            if (g.nrows == 2) {
+                float acc[2];
+                dot_rows_smemx<2>(sp, pitch, g.klen, lane, s.vec, acc);
+                y[0] = acc[0]; y[1] = acc[1];
+            } else if (g.nrows == 4) {
+                float acc[4];
+                dot_rows_smemx<4>(sp, pitch, g.klen, lane, s.vec, acc);
+                y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2]; y[3] = acc[3];
+            } else if (g.nrows == 3) {
+                float acc[3];
+                dot_rows_smemx<3>(sp, pitch, g.klen, lane, s.vec, acc);
+                y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2];
+            } else {
+                float acc[1];
+                dot_rows_smemx<1>(sp, pitch, g.klen, lane, s.vec, acc);
+                y[0] = acc[0];
+            }
+            __syncwarp();
+            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+            ring_release(p, s, wr, warp, lane);
+#pragma unroll
+            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = warp_sum(y[rr]);
+            if (ep == EP_SWIGLU) {
+                if (lane == 0) emit_value(out, g.row >> 1, silu(y[0]) * y[1]);
+                if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2]) * y[3]);
+            } else if (lane < g.nrows) {
+                // lane rr emits row rr (every lane holds all sums after the butterfly)
+                const float v = lane == 0 ? y[0] : lane == 1 ? y[1] : lane == 2 ? y[2] : y[3];
+                emit_value(out, g.row + lane, (ep == EP_RESIDUAL ? res : 0.f) + v);
+            }
+        } else if (pl.rpc <= MAX_RPC_SPLIT) {
             // one unit piece of up to four rows: the common case.  Residual inputs are fetched before the wait, their
             // L2 latency hides behind it.
             float res = 0.f;
