@@ -112,10 +112,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
                 plan = PL_QKV;
                 ep = EP_STORE;
             } else if (st == 1) {
-                trace_stamp(p, cta, l, 2, ctid); trace_stamp(p, cta, l, 3, ctid);
+                trace_stamp(p, cta, l, 2, ctid);
                 // S2: RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
                 attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
-                trace_stamp(p, cta, l, 4, ctid); trace_stamp(p, cta, l, 5, ctid);
+                trace_stamp(p, cta, l, 4, ctid);
                 // S3: output projection + residual (xa -> xb).  The poll on o's tags waits for the mergers.
                 load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
                 trace_stamp(p, cta, l, 6, ctid);

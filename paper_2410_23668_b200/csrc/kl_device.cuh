@@ -1296,19 +1296,25 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
             if ((ml_pend || pend) && !poll_continue(p, s, pg)) break;
         }
     }
+    trace_stamp(p, blockIdx.x, layer, 5, ctid);
     consumer_bar();
-    if (ctid < G) {
-        const uint32_t h = ctid;
+    // one warp per head: maximum and normaliser by butterfly reductions (every lane ends with the same value)
+    for (uint32_t h = ctid >> 5; h < G; h += NCW) {
+        const uint32_t lane = ctid & 31u;
         float Mx = -INFINITY;
-        for (uint32_t c = 0; c < nchunk; ++c) Mx = fmaxf(Mx, wtab[h * nchunk + c]);
+        for (uint32_t c = lane; c < nchunk; c += 32) Mx = fmaxf(Mx, wtab[h * nchunk + c]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Mx = fmaxf(Mx, __shfl_xor_sync(0xffffffffu, Mx, o));
         float Lx = 0.f;
-        for (uint32_t c = 0; c < nchunk; ++c) {
+        for (uint32_t c = lane; c < nchunk; c += 32) {
             const float sc = rescale(wtab[h * nchunk + c], Mx);
             Lx += wtab[nml + h * nchunk + c] * sc;
             wtab[h * nchunk + c] = sc;
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) Lx += __shfl_xor_sync(0xffffffffu, Lx, o);
         const float inv = 1.0f / Lx;
-        for (uint32_t c = 0; c < nchunk; ++c) wtab[h * nchunk + c] *= inv;
+        for (uint32_t c = lane; c < nchunk; c += 32) wtab[h * nchunk + c] *= inv;
     }
     consumer_bar();
     for (uint32_t j = ctid; j < ns; j += NCT) {
@@ -1526,6 +1532,7 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
             }
         }
     }
+    trace_stamp(p, cta, layer, 3, ctid);
     // every unit of the group merges its slice of the outputs
     if (nchunk > 1) attn_merge(p, s, u, layer, G, ctid, comb);
     return 0u;
