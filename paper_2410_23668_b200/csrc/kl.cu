@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
                 plan = PL_O;
                 ep = EP_RESIDUAL;
             } else if (st == 2) {
-                trace_stamp(p, cta, l, 7, ctid); trace_stamp(p, cta, l, 8, ctid);
+                trace_stamp(p, cta, l, 7, ctid);
                 // S4: RMSNorm + gate/up projections + SwiGLU
                 load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
                 trace_stamp(p, cta, l, 9, ctid);
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
                 stage_signal(p.counters + l, ctid, skip == ST_GU);
                 trace_stamp(p, cta, l, 10, ctid);
                 stage_wait(p, s, p.counters + l, p.P, ctid);
-                trace_stamp(p, cta, l, 11, ctid); trace_stamp(p, cta, l, 12, ctid);
+                trace_stamp(p, cta, l, 12, ctid);
                 // S5: down projection + residual (xb -> xa of the next layer)
                 out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
                 plan = PL_D;

@@ -626,6 +626,10 @@ __device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* 
             else if (e < n) *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = v[i];
         }
     }
+    if (norm && p.trace != nullptr && ctid == 0) {   // stamp 8: thread 0 holds valid data (diagnostic)
+        const uint32_t layer = ((tag >> 4) - p.step * p.L);
+        if (layer < p.L) p.trace[((size_t)blockIdx.x * p.L + layer) * TRACE_STAMPS + (((tag >> 1) & 7u) == TG_XA ? 8 : 11)] = globaltimer_ns();
+    }
     if (norm) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);

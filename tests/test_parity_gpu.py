@@ -61,6 +61,24 @@ def test_llama31_8b_shape_16_greedy_steps():
     print("oracle top-1/top-2 logit margins:", ["%.3f" % m for m in margins])
 
 
+def test_llama31_8b_shape_context_65536():
+    """Config 3 by sampled layers: the 8B shape at context 65536 (attention-heavy: every split-K unit streams ~3640
+    positions), the first two layers and the classifier, two decode steps.  The oracle streams the same layers."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_8B, n_layers=2)
+    rep = helpers.run_parity(shape, context=65536, steps=2, seed=0, max_ctx=65536 + 8, check_cache=False)
+    helpers.assert_parity(rep, 2, check_cache=False)
+
+
+def test_llama31_70b_shape_two_layers():
+    """Config 5 by sampled layers: the 70B shape (hidden 8192, 64 / 8 heads, FFN 28672) at context 4096, the first two
+    layers and the classifier, two decode steps."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_70B, n_layers=2)
+    rep = helpers.run_parity(shape, context=4096, steps=2, seed=0, max_ctx=4096 + 8, check_cache=False)
+    helpers.assert_parity(rep, 2, check_cache=False)
+
+
 def test_bounded_wait_reports_timeout_and_recovers():
     """A stage end that is never signalled makes the waits on it run out: the step reports KL_ERR_SYNC_TIMEOUT
     (no hang, no trap) and the next step on the same handle is correct again."""
