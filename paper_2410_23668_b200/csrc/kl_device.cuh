@@ -580,6 +580,9 @@ __device__ __forceinline__ uint32_t vec_perm(uint32_t e) {
 __device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
                                          const __nv_bfloat16* gain, uint32_t ctid) {
     constexpr int NB = 6;  // groups of four values kept in flight per thread (two 16-byte loads each)
+    // The vector area is about to be overwritten: every warp of the CTA must be done with what the previous stage
+    // kept there (the stage's input vector, read block by block until a warp's last chunk; the attention workspace).
+    consumer_bar();
     float ss = 0.f;
     const bool single = n <= (uint32_t)(NB * NCT * 4);
     float4 keep[NB];
@@ -1357,6 +1360,7 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
 
     // q (and, for the unit that owns the new position, k and v) of this step: tagged words written by whichever CTAs
     // own those rows of the QKV projection.  The unit waits for exactly the rows it needs, not for the whole stage.
+    consumer_bar();   // the workspace below overlays the QKV stage's input vector: wait for this CTA's last QKV chunk
     const TW* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
     const uint32_t qtag = tag_of(p, layer, TG_QKV);
     const float* cs = p.rope_cs + (size_t)b * hd;  // [half][2]
