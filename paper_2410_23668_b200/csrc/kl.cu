@@ -367,7 +367,10 @@ GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t alig
         const uint32_t cand[5] = {1, 2, 3, NCW, 2 * NCW};
         for (int q = 0; q < 5; ++q)
             if (cand[q] >= np) { np = cand[q]; break; }
-        pl.kp = ceil_div(ceil_div(K, np), 256) * 256;
+        // a piece multiplied against shared memory starts at a block of 256 columns; one read from global memory
+        // only needs 16-byte pieces per lane
+        const uint32_t gran = x_in_smem ? 256u : 8u;
+        pl.kp = ceil_div(ceil_div(K, np), gran) * gran;
         pl.npieces = ceil_div(K, pl.kp);
         uint32_t rpc = SLOT_BYTES / (pl.kp * 2);
         if (rpc > (uint32_t)MAX_RPC_SPLIT) rpc = MAX_RPC_SPLIT;
@@ -386,7 +389,7 @@ bool plans_ok(const Params& p) {
         if (pl.npieces > (uint32_t)MAX_PIECES || pl.rpc < 1) return false;
         if (pl.kp > MAX_KP && (pl.npieces > 1 || i == PL_D || pl.rpc > (uint32_t)MAX_RPC_SPLIT)) return false;
         if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
-        if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % 256)) return false;
+        if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % (i == PL_D ? 8 : 256))) return false;
         if (i == PL_GU && (pl.rpc & 1u)) return false;
     }
     return true;

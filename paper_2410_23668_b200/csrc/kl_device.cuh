@@ -10,19 +10,23 @@
 
 namespace kl {
 
-constexpr int NCW = 6;                     // consumer warps per CTA; consumer c takes chunks c, c + NCW, ... and so
+#ifndef KL_NCW
+#define KL_NCW 10
+#endif
+
+constexpr int NCW = KL_NCW;                     // consumer warps per CTA; consumer c takes chunks c, c + NCW, ... and so
                                            // always meets the same nsw ring slots, in order
 constexpr int NCT = NCW * 32;              // consumer threads (they take part in the CTA-wide steps)
 constexpr int NTHREADS = NCT + 32;         // + the producer warp (the last warp; 7 warps leave 255 registers each)
 constexpr int SLOT_BYTES = 16384;          // one ring slot = one chunk (one or two TMA copies)
-constexpr int MAX_NSW = 4;                 // ring slots per consumer warp
+constexpr int MAX_NSW = 24 / NCW;          // ring slots per consumer warp (the barrier arrays hold 24 slots)
 constexpr int MAX_SLOTS = NCW * MAX_NSW;
-constexpr int MAX_PIECES = 16;             // chunks per unit when a unit spans several chunks
-constexpr int UNIT_SLOTS = 16;             // in-flight multi-chunk units tracked per CTA
+constexpr int MAX_PIECES = 2 * NCW;            // chunks per unit when a unit spans several chunks
+constexpr int UNIT_SLOTS = 8;             // in-flight multi-chunk units tracked per CTA
 constexpr int MAX_RPC_SPLIT = 4;           // rows per unit when units are split into column pieces
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
 constexpr int MAX_G = 8;                   // query heads per KV head
-constexpr int SMEM_MISC_BYTES = 8192;  // barriers, chunk-sequence plan, reduction scratch, unit table (see carve_smem)
+constexpr int SMEM_MISC_BYTES = 6656;  // barriers, chunk-sequence plan, reduction scratch, unit table (see carve_smem)
 
 enum StageId { ST_QKV = 0, ST_ATTN = 1, ST_O = 2, ST_GU = 3, ST_D = 4, ST_LM = 5 };
 enum EpilogueKind { EP_STORE = 0, EP_RESIDUAL = 1, EP_SWIGLU = 2 };
@@ -46,7 +50,7 @@ struct GemvPlan {
     uint32_t nunits;
 };
 #ifndef KL_MAX_KP
-#define KL_MAX_KP 2560
+#define KL_MAX_KP 1536
 #endif
 constexpr uint32_t MAX_KP = KL_MAX_KP;      // columns per chunk piece: blocks of 256, 8 per lane and block
 constexpr int MAX_XB = MAX_KP / 256;
@@ -759,10 +763,11 @@ __device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t pitch, uint3
     for (int r = 0; r < NR; ++r) acc[r] = e[r] + o[r];
 }
 
-// Branch-free variant for pieces of exactly NB full blocks (the common sizes): no predicates, so the compiler is
-// free to software-pipeline the shared-memory loads against the arithmetic.  Same order of operations as dot_rows.
+// Variant for pieces of NB full blocks plus, possibly, one partial block: no predicates on the full blocks, so the
+// compiler is free to software-pipeline the shared-memory loads against the arithmetic.  Same order of operations as
+// dot_rows.
 template <int NR, int NB>
-__device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, uint32_t lane, const XRegs& x,
+__device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane, const XRegs& x,
                                               float (&acc)[NR]) {
     float e[NR], o[NR];
 #pragma unroll
@@ -783,22 +788,32 @@ __device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, 
             o[r] = fmaf(bf_hi(q.w), x.v[b][7], o[r]);
         }
     }
+    if constexpr (NB < MAX_XB) {
+        if ((uint32_t)NB * 256u + lane * 8u < klen) {   // the partial block (klen is a multiple of 8)
+#pragma unroll
+            for (int r = 0; r < NR; ++r) {
+                const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)NB * 512);
+                e[r] = fmaf(bf_lo(q.x), x.v[NB][0], e[r]);
+                o[r] = fmaf(bf_hi(q.x), x.v[NB][1], o[r]);
+                e[r] = fmaf(bf_lo(q.y), x.v[NB][2], e[r]);
+                o[r] = fmaf(bf_hi(q.y), x.v[NB][3], o[r]);
+                e[r] = fmaf(bf_lo(q.z), x.v[NB][4], e[r]);
+                o[r] = fmaf(bf_hi(q.z), x.v[NB][5], o[r]);
+                e[r] = fmaf(bf_lo(q.w), x.v[NB][6], e[r]);
+                o[r] = fmaf(bf_hi(q.w), x.v[NB][7], o[r]);
+            }
+        }
+    }
 #pragma unroll
     for (int r = 0; r < NR; ++r) acc[r] = e[r] + o[r];
 }
-// NR rows: picks the branch-free variant when the piece is a whole number of blocks of a common size.
+// NR rows: picks the variant by the number of full blocks of the piece.
 template <int NR>
 __device__ __forceinline__ void dot_n(const uint8_t* w, uint32_t pitch, uint32_t klen, uint32_t lane, const XRegs& x,
                                       float (&acc)[NR]) {
-    if constexpr (MAX_XB >= 16) {
-        if (klen == 4096) {
-            dot_rows_full<NR, (MAX_XB >= 16 ? 16 : 1)>(w, pitch, lane, x, acc);
-            return;
-        }
-    }
-    switch (klen) {
-        case 2560: dot_rows_full<NR, 10>(w, pitch, lane, x, acc); break;
-        case 2048: dot_rows_full<NR, 8>(w, pitch, lane, x, acc); break;
+    switch (klen >> 8) {
+        case 5: dot_rows_full<NR, (MAX_XB >= 5 ? 5 : MAX_XB)>(w, pitch, klen, lane, x, acc); break;
+        case 6: dot_rows_full<NR, (MAX_XB >= 6 ? 6 : MAX_XB)>(w, pitch, klen, lane, x, acc); break;
         default: dot_rows<NR>(w, pitch, klen, lane, x, acc); break;
     }
 }

@@ -79,6 +79,33 @@ def test_llama31_70b_shape_two_layers():
     helpers.assert_parity(rep, 2, check_cache=False)
 
 
+def test_repeated_steps_are_bit_identical():
+    """The same step from the same state, several times and in both schedules: identical logits and hidden state.
+    Any race between the warps of a CTA or between CTAs (a buffer reused too early) shows up here as run-to-run
+    noise long before it breaks the oracle tolerance."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_8B, n_layers=4)
+    context, max_ctx = 4096, 4096 + 8
+    dec = helpers.make_decoder(shape, 1, max_ctx, 0)
+    cache0 = gen.make_kv_cache(shape, 1, context, max_ctx, 0, "cuda")
+    tok = gen.make_tokens(shape, 1, 0).cuda()
+    pos = torch.tensor([context], dtype=torch.int32, device="cuda")
+    outs = []
+    for mode in (binding.KL_MODE_LOOPED,) * 4 + (binding.KL_MODE_PER_LAYER,) * 2:
+        dec.kl_set_mode(mode)
+        cache = cache0.clone()
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        hidden = torch.empty(1, shape.hidden, device="cuda")
+        dec.kl_decode_step(tok, pos, cache, logits, 1)
+        dec.kl_read_hidden(hidden, 1)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        outs.append((logits.cpu(), hidden.cpu(), cache.cpu().view(torch.uint16)))
+    for lg, hd, ch in outs[1:]:
+        assert torch.equal(lg, outs[0][0]) and torch.equal(hd, outs[0][1]) and torch.equal(ch, outs[0][2])
+    dec.close()
+
+
 def test_bounded_wait_reports_timeout_and_recovers():
     """A stage end that is never signalled makes the waits on it run out: the step reports KL_ERR_SYNC_TIMEOUT
     (no hang, no trap) and the next step on the same handle is correct again."""
