@@ -8,6 +8,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#ifndef KL_ST_TW
+#define KL_ST_TW "st.relaxed.gpu.global.b64"
+#endif
+
 namespace kl {
 
 #ifndef KL_NCW
@@ -173,7 +177,7 @@ struct __align__(8) TW {
 // scope): a weak load inside a polling loop may legally be hoisted out of it by the assembler.
 __device__ __forceinline__ void st_tw(TW* p, float v, uint32_t tag) {
     const uint64_t w = ((uint64_t)tag << 32) | __float_as_uint(v);
-    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
+    asm volatile(KL_ST_TW " [%0], %1;" ::"l"(p), "l"(w) : "memory");
 }
 __device__ __forceinline__ TW ld_tw(const TW* p) {
     uint64_t r;
@@ -960,8 +964,12 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             __syncwarp();
             if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
             ring_release(p, s, wr, warp, lane);
-#pragma unroll
-            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = warp_sum(y[rr]);
+            y[0] = warp_sum(y[0]);
+            y[1] = warp_sum(y[1]);
+            if (g.nrows > 2) {   // uniform over the warp
+                y[2] = warp_sum(y[2]);
+                y[3] = warp_sum(y[3]);
+            }
             if (ep == EP_SWIGLU) {
                 if (lane == 0) emit_value(out, g.row >> 1, silu(y[0]) * y[1]);
                 if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2]) * y[3]);
@@ -1195,7 +1203,9 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const uint32_t k = kb * 16 + hf * 8 + 2 * t;
-            const float x0 = g < G ? q_s[g * HD + k] : 0.f, x1 = g < G ? q_s[g * HD + k + 1] : 0.f;
+            float2 xx = make_float2(0.f, 0.f);
+            if (g < G) xx = *reinterpret_cast<const float2*>(q_s + g * HD + k);   // k is even: 8-byte aligned
+            const float x0 = xx.x, x1 = xx.y;
             const uint32_t hi = pack_bf16(x0, x1);
             st.qh[kb][hf] = hi;
             st.ql[kb][hf] = pack_bf16(x0 - bf_lo(hi), x1 - bf_hi(hi));
@@ -1529,18 +1539,31 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
     trace_stamp(p, cta, layer, 15, ctid);
     consumer_bar();
 
-    // merge the warps; thread t owns (head, column)
+    // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h),
+    // in place; then thread t owns (head, column) and adds the NCW weighted terms in warp order.
     const uint32_t unit = u.bg * p.cps + u.ch;
+    {
+        float fw = 0.f, Mh = -INFINITY;
+        const uint32_t w = ctid / G, h = ctid % G;
+        if (ctid < NCW * G) {
+#pragma unroll
+            for (int ww = 0; ww < NCW; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (hd + 2) + hd]);
+            fw = rescale(comb[((size_t)w * G + h) * (hd + 2) + hd], Mh);
+        }
+        consumer_bar();
+        if (ctid < NCW * G) {
+            comb[((size_t)w * G + h) * (hd + 2) + hd] = fw;
+            if (w == 0) s.red[h] = Mh;
+        }
+        consumer_bar();
+    }
     for (uint32_t t = ctid; t < G * hd; t += NCT) {
         const uint32_t h = t / hd, d = t % hd;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < NCW; ++w) M = fmaxf(M, comb[((size_t)w * G + h) * (hd + 2) + hd]);
         float A = 0.f, Lsum = 0.f;
 #pragma unroll
         for (int w = 0; w < NCW; ++w) {
             const float* src = comb + ((size_t)w * G + h) * (hd + 2);
-            const float c = rescale(src[hd], M);
+            const float c = src[hd];
             A += src[d] * c;
             Lsum += src[hd + 1] * c;
         }
@@ -1550,7 +1573,7 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
             const uint32_t ptag = tag_of(p, layer, TG_PART);
             st_tw(p.part + ((size_t)unit * G + h) * hd + d, A, ptag);
             if (d == 0) {
-                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, M, ptag);
+                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, s.red[h], ptag);
                 st_tw(p.part_ml + ((size_t)unit * G + h) * 2 + 1, Lsum, ptag);
             }
         }
