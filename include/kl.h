@@ -155,26 +155,32 @@ kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* c
 
 /* Stage timeline of the decoder kernel (the analogue of the paper's per-socket HBM-bandwidth trace, Section 4).
  * trace_d: DEVICE buffer of n_ctas * n_layers * n_stamps + 8192 * 4 uint64 (zero it first), or NULL to switch
- * tracing off; the three sizes
- * are returned through the out pointers (each may be NULL).  While set, consumer thread 0 of every CTA stores the
- * GPU global timer (ns) at fixed points of every layer: 0 previous layer complete, 1 input normalised, 2 QKV rows
- * done and signalled, 3 all QKV seen, 4 attention unit done and signalled, 5 all attention seen, 6 o loaded,
- * 7 O-projection done, 8 all O seen, 9 input normalised, 10 gate/up done, 11 all gate/up seen, 12 h loaded,
- * 13 down-projection done, 14 attention prologue done, 15 attention ring chunks consumed.  The trailing
- * 8192 x 4 block logs the first 8192 ring chunks of CTA 0: issue by the producer, consumer starts waiting, chunk
- * landed, chunk consumed and released.  Stamps of the latest step overwrite earlier ones. */
+ * tracing off; the three sizes are returned through the out pointers (each may be NULL).  While set, consumer
+ * thread 0 of every CTA stores the GPU global timer (ns) at fixed points of every layer:
+ *    0 layer entered (starts polling the hidden state)      8 thread 0 holds valid words of it
+ *    1 input normalised                                     2 QKV rows of this CTA done
+ *   14 attention prologue done (q, k, v polled, rotated)   15 this warp's ring chunks of the unit consumed
+ *    3 partial result of the unit written                   5 thread 0's loads for the slice merge complete
+ *    4 attention block done                                 6 attention output loaded
+ *    7 O-projection rows done                              11 thread 0 holds valid words of x'
+ *    9 x' normalised                                       10 gate/up rows done
+ *   12 counter of the gate/up stage passed                 13 down-projection rows done
+ * The trailing 8192 x 4 block logs the first 8192 ring chunks of CTA 0: [0] issue by the producer, [2] chunk seen
+ * landed by its consumer warp, [1] dot product done, [3] results emitted.  Stamps of the latest step overwrite
+ * earlier ones. */
 kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32_t* n_layers, uint32_t* n_stamps);
 
 /* Attention inner loop.  on = 1 (default when head_dim is 64 or 128): tensor-core loop (mma.sync on 128-byte
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
-/* Limit, in nanoseconds, of every device-side wait (flag, counter or mbarrier).  Default 2e9. */
+/* Limit, in nanoseconds, of every device-side wait (tagged word, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
 
-/* Test hook for the bounded waits: when stage >= 0 the CTAs of the persistent kernel do not signal the end of
- * that stage (0..4) of layer 0 on the NEXT kl_decode_step only, so the waits on it run out and the step reports
- * KL_ERR_SYNC_TIMEOUT.  No fault, trap or endless loop is involved. */
+/* Test hook for the bounded waits: when stage >= 0 the results of that stage (0 QKV, 1 attention, 2 O, 3 gate/up,
+ * 4 down) of layer 0 are published with a tag nobody waits for (stage 3: its counter is not incremented) on the
+ * NEXT kl_decode_step only, so the waits on them run out and the step reports KL_ERR_SYNC_TIMEOUT.  No fault, trap
+ * or endless loop is involved. */
 kl_status kl_debug_skip_signal_once(kl_handle* h, int stage);
 
 const char* kl_status_string(kl_status s);
