@@ -38,6 +38,9 @@ WORKLOADS = {
     "llama31_8b_4layers_b1_ctx4096": (gen.ModelShape(4, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 1, 4096, 8),
     "llama31_8b_b1_ctx65536": (gen.LLAMA31_8B, 1, 65536, 64),
     "llama31_70b_b1_ctx4096": (gen.LLAMA31_70B, 1, 4096, 32),
+    # batches run sequence after sequence through the batch-1 kernels (weights streamed once per sequence): functional,
+    # not the batched roofline
+    "llama31_8b_b32_ctx4096": (gen.LLAMA31_8B, 32, 4096, 4),
 }
 DEFAULT_WORKLOAD = "llama31_8b_b1_ctx4096"
 NOMINAL_HBM_GBS = 8000.0

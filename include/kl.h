@@ -96,6 +96,10 @@ kl_status kl_set_mode(kl_handle* h, int mode);
  *                  attention covers positions 0..positions_d[b] inclusive
  *   kv_cache_d     cache in the layout above; row positions_d[b] of every layer is written
  *   logits_d       [batch, vocab] fp32, written
+ * Sequences of a batch are independent (ragged positions are fine).  They are decoded one after another by the
+ * batch-1 kernels -- the weights are streamed once per SEQUENCE; projections as M = batch tensor-core contractions,
+ * which would stream them once per step, are not built.  Tokens and positions of the whole batch are checked
+ * before the first sequence is decoded.
  * Merged-call argument rule of Section 3.2: weights (grouped, all layers) come from the handle, the hidden
  * state enters once (from the embedding) and leaves once (kl_read_hidden / the classifier), the KV cache is the
  * grouped in/out parameter.  Device-detected errors make the step a no-op and are reported by kl_last_status. */
@@ -134,7 +138,7 @@ kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_
                                    uint32_t batch, void* stream);
 
 /* Copies the hidden state after the last decoder layer (before the final RMSNorm) of the latest step:
- * hidden_d [batch, hidden] fp32. */
+ * hidden_d [batch, hidden] fp32; batch must be the latest step's. */
 kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream);
 
 /* Synchronises nothing: call after the stream has been synchronised.  Reads and clears the device status word

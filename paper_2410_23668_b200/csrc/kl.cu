@@ -26,11 +26,16 @@ namespace kl {
 // ------------------------------------------------------------------------------------------------ kernels
 
 __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
-    const uint32_t b = blockIdx.x, tid = threadIdx.x;
-    int32_t tok = p.tokens[b];
-    const int32_t pos = p.positions[b];
-    if (tid == 0 && (tok < 0 || tok >= (int32_t)p.V || pos < 0 || pos >= (int32_t)p.max_ctx))
-        atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+    const uint32_t b = 0u, tid = threadIdx.x;   // b: slot of the sequence in the scratch vectors
+    int32_t tok = p.tokens[p.b0];
+    const int32_t pos = p.positions[p.b0];
+    // the launch for the first sequence checks the whole batch, so that a bad entry anywhere makes the step a no-op
+    // before any sequence has been decoded
+    if (p.b0 == 0u)
+        for (uint32_t i = tid; i < p.B; i += blockDim.x) {
+            const int32_t t = p.tokens[i], q = p.positions[i];
+            if (t < 0 || t >= (int32_t)p.V || q < 0 || q >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+        }
     if (tok < 0 || tok >= (int32_t)p.V) tok = 0;
     const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
     const uint32_t xtag = tag_of(p, 0, TG_XA);
@@ -253,6 +258,8 @@ struct kl_handle {
     int32_t* stage_positions;
     float* stage_logits;
     float* argmax_val;
+    float* hidden_all;     // [max_batch][H] hidden states of the sequences of the latest batched step
+    uint32_t last_batch;
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
     uint64_t launches;
@@ -278,7 +285,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, shid, scratch_bytes;
     uint32_t cps;
 };
 
@@ -290,7 +297,7 @@ bool shape_supported(const kl_model_desc& d, int num_sms) {
     if (d.n_q_heads % d.n_kv_heads) return false;
     const uint32_t G = d.n_q_heads / d.n_kv_heads;
     if (G != 1 && G != 2 && G != 4 && G != 8) return false;
-    if ((uint64_t)d.max_batch * d.n_kv_heads > (uint64_t)num_sms) return false;
+    if ((uint64_t)d.n_kv_heads > (uint64_t)num_sms) return false;
     if (!(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f)) return false;
     return true;
 }
@@ -333,6 +340,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.spos = s;      s += align_up(B * 4);
     y.slogits = s;   s += align_up(B * V * 4);
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
+    y.shid = s;      s += align_up(B * H * 4);
     y.scratch_bytes = s;
     return y;
 }
@@ -572,6 +580,8 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->stage_positions = (int32_t*)(sc + y.spos);
     h->stage_logits = (float*)(sc + y.slogits);
     h->argmax_val = (float*)(sc + y.samax);
+    h->hidden_all = (float*)(sc + y.shid);
+    h->last_batch = 1;
     h->argmax_idx = (uint32_t*)(h->argmax_val + (size_t)d.max_batch * ARGMAX_BLOCKS);
     h->argmax_tickets = h->argmax_idx + (size_t)d.max_batch * ARGMAX_BLOCKS;
 
@@ -678,48 +688,59 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
                          float* logits_d, uint32_t batch, void* stream) {
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
-    if (batch != 1) return KL_ERR_UNSUPPORTED_SHAPE;  // batched tensor-core path not built yet
     if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
     cudaStream_t st = as_stream(stream);
     Params p = h->prm;
     p.B = batch;
-    p.cps = (uint32_t)h->num_sms / (batch * p.nkv);
+    p.cps = (uint32_t)h->num_sms / p.nkv;
     p.tokens = tokens_d;
     p.positions = positions_d;
     p.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
-    p.logits = logits_d;
     p.skip_stage = h->pending_skip_stage;
     h->pending_skip_stage = -1;
-    p.step = ++h->prm.step;
     p.attn_tc = 0;
     if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
         const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, batch);
         if (trc != KL_OK) return trc;
         p.attn_tc = 1;
     }
-
-    kl_embed_kernel<<<batch, 256, 0, st>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
-    ++h->launches;
-    kl_status rc;
+    h->last_batch = batch;
     cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
-    if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
-    if (h->mode == KL_MODE_LOOPED) {
-        uint32_t l0 = 0, l1 = p.L;
-        void* args[] = {&p, &l0, &l1};
-        if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
-    } else {
-        for (uint32_t l = 0; l < p.L; ++l) {
-            uint32_t l0 = l, l1 = l + 1;
+    // Sequences of a batch are independent.  The batch-1 kernels decode them one after another (the weights are
+    // streamed once per sequence); the M = batch tensor-core projections that would stream them once per step are
+    // not built.
+    for (uint32_t b = 0; b < batch; ++b) {
+        p.b0 = b;
+        p.logits = logits_d + (size_t)b * p.V;
+        p.step = ++h->prm.step;
+        kl_embed_kernel<<<1, 256, 0, st>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+        ++h->launches;
+        kl_status rc;
+        if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+        if (h->mode == KL_MODE_LOOPED) {
+            uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1};
             if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+        } else {
+            for (uint32_t l = 0; l < p.L; ++l) {
+                uint32_t l0 = l, l1 = l + 1;
+                void* args[] = {&p, &l0, &l1};
+                if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+            }
+        }
+        if (ev && b == 0 && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
+        Params pc = p;
+        pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
+        void* cargs[] = {&pc};
+        if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
+        if (ev && b == 0 && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
+        if (batch > 1) {
+            // keep this sequence's hidden state (the value half of every tagged word) for kl_read_hidden
+            if (cudaMemcpy2DAsync(h->hidden_all + (size_t)b * p.H, 4, p.xa, 8, 4, p.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return KL_ERR_CUDA;
         }
     }
-    if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
-    p.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
-    void* cargs[] = {&p};
-    if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
-    if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
 }
 
@@ -795,10 +816,13 @@ kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_
 
 kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream) {
     if (!h || !hidden_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
-    // the hidden state leaving the last layer is an array of tagged words: take the value half of each
-    if (cudaMemcpy2DAsync(hidden_d, 4, h->prm.xa, 8, 4, (size_t)batch * h->prm.H, cudaMemcpyDeviceToDevice, as_stream(stream)) !=
-        cudaSuccess)
-        return KL_ERR_CUDA;
+    if (batch != h->last_batch) return KL_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (batch == 1)   // the hidden state leaving the last layer is an array of tagged words: take the value half of each
+        e = cudaMemcpy2DAsync(hidden_d, 4, h->prm.xa, 8, 4, h->prm.H, cudaMemcpyDeviceToDevice, as_stream(stream));
+    else
+        e = cudaMemcpyAsync(hidden_d, h->hidden_all, (size_t)batch * h->prm.H * 4, cudaMemcpyDeviceToDevice, as_stream(stream));
+    if (e != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
 }
 

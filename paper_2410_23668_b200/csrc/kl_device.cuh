@@ -62,7 +62,8 @@ constexpr int MAX_XB = MAX_KP / 256;
 struct Params {
     CUtensorMap kv_map;    // the whole KV cache as a 2-D tensor [rows, head_dim], 128-byte swizzle (64-byte aligned)
     uint32_t attn_tc;      // 1: tensor-core attention loop fed by kv_map boxes; 0: CUDA-core loop fed by linear copies
-    uint32_t L, H, nq, nkv, hd, F, V, G, QD, KVD, max_ctx, B;
+    uint32_t L, H, nq, nkv, hd, F, V, G, QD, KVD, max_ctx, B;   // B: sequences in the KV cache of this step
+    uint32_t b0;           // the sequence this launch decodes (batches run one sequence after another)
     uint32_t P;            // CTAs in the persistent grid
     uint32_t nslots;       // ways of the ring = consumer warps (chunk n belongs to consumer n % nslots)
     uint32_t nsw;          // slots per consumer (chunk n sits in slot (n % nslots) * nsw + (n / nslots) % nsw)
@@ -341,9 +342,9 @@ __device__ __forceinline__ AttnUnit attn_unit(const Params& p, uint32_t cta) {
     u.nring = 0;
     u.bg = cta / p.cps;
     u.ch = cta % p.cps;
-    if (u.bg >= p.B * p.nkv) return u;
-    u.b = u.bg / p.nkv;
-    u.g = u.bg % p.nkv;
+    if (u.bg >= p.nkv) return u;
+    u.b = p.b0;
+    u.g = u.bg;
     u.pos = (uint32_t)p.positions[u.b];
     const uint32_t n = u.pos + 1;
     uint32_t nchunk = min(p.cps, (n + MIN_POS_PER_CHUNK - 1) / MIN_POS_PER_CHUNK);
@@ -1282,7 +1283,7 @@ __device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const 
 // are fixed.
 __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const AttnUnit& u, uint32_t layer, uint32_t G,
                                         uint32_t ctid, float* comb) {
-    const uint32_t hd = p.hd, b = u.b, g = u.g, nchunk = u.nchunk;
+    const uint32_t hd = p.hd, b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
     const uint32_t unit0 = u.bg * p.cps;
     const uint32_t tag = tag_of(p, layer, TG_PART), otag = tag_of(p, layer, TG_O);
     const uint32_t total = G * hd;
@@ -1371,7 +1372,7 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
     if (!u.active) return 1u;
     const uint32_t G = GT > 0 ? (uint32_t)GT : p.G;
     const uint32_t hd = p.hd, half = hd >> 1;
-    const uint32_t b = u.b, g = u.g, pos = u.pos, nchunk = u.nchunk;
+    const uint32_t b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
 
     // shared workspace inside the vector area
     float* q_s = s.vec;                         // [G][hd]

@@ -79,6 +79,30 @@ def test_llama31_70b_shape_two_layers():
     helpers.assert_parity(rep, 2, check_cache=False)
 
 
+def test_batch_of_sequences_ragged_positions():
+    """Batches are decoded one sequence after another by the batch-1 kernels: three sequences at different
+    positions, four steps, both schedules; every sequence matches the oracle and its cache rows land in its own
+    slab of the [L][2][B][nkv][max_ctx][hd] cache."""
+    rep = helpers.run_parity(gen.TINY, context=128, steps=4, seed=3, batch=3, positions0=[5, 64, 128])
+    helpers.assert_parity(rep, 4, batch=3)
+
+
+def test_batch_bad_entry_makes_the_whole_step_a_no_op():
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 2, 200, 0)
+    cache = gen.make_kv_cache(shape, 2, 128, 200, 0, "cuda")
+    before = cache.clone()
+    tok = torch.tensor([1, shape.vocab + 7], dtype=torch.int32, device="cuda")   # the SECOND sequence is bad
+    pos = torch.tensor([128, 128], dtype=torch.int32, device="cuda")
+    logits = torch.full((2, shape.vocab), 7.0, device="cuda")
+    dec.kl_decode_step(tok, pos, cache, logits, 2)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE
+    assert torch.equal(cache.view(torch.uint16), before.view(torch.uint16))       # nothing appended, not even for sequence 0
+    assert bool((logits == 7.0).all())
+    dec.close()
+
+
 def test_repeated_steps_are_bit_identical():
     """The same step from the same state, several times and in both schedules: identical logits and hidden state.
     Any race between the warps of a CTA or between CTAs (a buffer reused too early) shows up here as run-to-run
