@@ -7,8 +7,8 @@
 // The decoder kernel is persistent: one CTA per SM, one producer warp that streams this CTA's share of every
 // weight matrix through a shared-memory ring with TMA bulk copies, and NCW consumer warps.  Weight addresses do
 // not depend on activations, so the producer runs ahead of the consumers across stage boundaries and, in looped
-// mode, across layer boundaries: while the CTAs wait on the acquire/release counter that replaces a kernel
-// boundary, HBM keeps streaming the next stage's (next layer's) tiles.
+// mode, across layer boundaries: while the CTAs poll the tagged words that replace a kernel boundary, HBM keeps
+// streaming the next stage's (next layer's) chunks until the ring is full.
 #include "kl_device.cuh"
 
 #include <math.h>
@@ -77,7 +77,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
             mbar_init(smem_u32(&s.empty[i]), 1);
         }
         *s.abort_flag = 0;
-        *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -90,7 +89,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
         if (lane == 0) produce_decoder(p, s, cta, l0, l1);
         return;
     }
-    const uint64_t pol = 0;
     WarpRing wr = ring_begin();
 
     // ---------------- consumers
@@ -165,7 +163,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
             mbar_init(smem_u32(&s.empty[i]), 1);
         }
         *s.abort_flag = 0;
-        *s.bcast = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -176,7 +173,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
         if (lane == 0) produce_classifier(p, s, cta);
         return;
     }
-    const uint64_t pol = 0;
     WarpRing wr = ring_begin();
     RingCursor rc = {0u, 0u};
     load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, tid);

@@ -1,6 +1,6 @@
-// Device-side building blocks of the kernel-looped decoder: PTX wrappers (mbarrier, TMA bulk copy,
-// acquire/release counters), the shared-memory weight ring, the GEMV stage consumer and the split-K
-// attention stage.  sm_100a only.
+// Device-side building blocks of the kernel-looped decoder: PTX wrappers (mbarrier, TMA bulk and tensor copies,
+// tagged 64-bit words, one acquire/release counter), the shared-memory weight ring, the GEMV stage consumer and
+// the split-K attention stage.  sm_100a only.
 #pragma once
 
 #include <cuda.h>
@@ -215,7 +215,6 @@ struct Smem {
     float* unit_part;       // [UNIT_SLOTS][MAX_PIECES]
     int* unit_cnt;          // [UNIT_SLOTS]
     volatile int* abort_flag;
-    volatile int* bcast;
 };
 
 __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
@@ -229,7 +228,6 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
     s.unit_part = reinterpret_cast<float*>(misc + 2048);           // [UNIT_SLOTS][MAX_PIECES][MAX_RPC_SPLIT] 4 KB
     s.unit_cnt = reinterpret_cast<int*>(misc + 6144);              // [UNIT_SLOTS]
     s.abort_flag = s.unit_cnt + UNIT_SLOTS;
-    s.bcast = s.abort_flag + 1;
     return s;
 }
 
@@ -1092,9 +1090,9 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
 }
 
 // End of a stage: all consumer warps have written their outputs; one thread publishes the CTA's arrival.
-__device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool skip, uint32_t weight = 1u) {
+__device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool skip) {
     consumer_bar();
-    if (ctid == 0 && !skip && weight) red_release_add(ctr, weight);  // release: cumulative over the CTA barrier above
+    if (ctid == 0 && !skip) red_release_add(ctr, 1u);  // release: cumulative over the CTA barrier above
 }
 
 // Waits (bounded) until `target` CTAs have signalled.  Replaces the grid-wide barrier of a kernel boundary.
@@ -1358,18 +1356,17 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
     }
 }
 
-// Split-K decode attention of one layer (flash-decoding): CTA `cta` owns at most one unit; its cached K/V rows
-// arrive through the ring (in flight while the QKV stage and its counter wait were still running); the last CTA
-// to finish a (b, g) merges its chunks.  Scores use q pre-multiplied by log2(e)/sqrt(hd): the softmax runs in
-// base 2.  GT > 0 selects the CUDA-core inner loop for GT query heads per KV head; GT == 0 the tensor-core loop.
-// Returns the weight with which this CTA signals the end of the stage: the last unit of a (sequence, kv head) to
-// arrive merges the chunks and signals for all of them; the other units of that group do not signal at all (their
-// only fence is the ticket), CTAs without a unit and single-chunk units signal for themselves.
+// Split-K decode attention of one layer (flash-decoding): CTA `cta` owns at most one unit (kv head, chunk of the
+// cached positions); its cached K/V rows arrive through the ring, requested while the QKV stage was still running.
+// The unit polls the q (and, for the chunk that ends with the new position, k and v) rows it needs, runs its ring
+// chunks, merges its warps and publishes the partial result; then every unit of the kv head merges its slice of
+// the outputs (attn_merge).  Scores use q pre-multiplied by log2(e)/sqrt(hd): the softmax runs in base 2.
+// GT > 0 selects the CUDA-core inner loop for GT query heads per KV head; GT == 0 the tensor-core loop.
 template <int GT>
-__device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+__device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
                                                  uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
     const AttnUnit u = attn_unit(p, cta);
-    if (!u.active) return 1u;
+    if (!u.active) return;
     const uint32_t G = GT > 0 ? (uint32_t)GT : p.G;
     const uint32_t hd = p.hd, half = hd >> 1;
     const uint32_t b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
@@ -1582,7 +1579,6 @@ __device__ __noinline__ uint32_t attention_stage(const Params& p, const Smem& s,
     trace_stamp(p, cta, layer, 3, ctid);
     // every unit of the group merges its slice of the outputs
     if (nchunk > 1) attn_merge(p, s, u, layer, G, ctid, comb);
-    return 0u;
 }
 
 // Appends the K/V row of the position written by this step to the cache (16-byte stores).  Nothing in the running
@@ -1612,12 +1608,11 @@ __device__ __forceinline__ void attention_flush_new_row(const Params& p, const S
 
 // Runs the attention stage and moves the ring cursor past the unit's chunks (also for CTAs without a unit).
 template <int GT>
-__device__ __forceinline__ uint32_t attention_stage_and_advance(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
-                                                                uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
-                                                                WarpRing& wr) {
-    const uint32_t weight = attention_stage<GT>(p, s, layer, cta, ctid, warp, lane, rc, wr);
+__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+                                                            uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
+                                                            WarpRing& wr) {
+    attention_stage<GT>(p, s, layer, cta, ctid, warp, lane, rc, wr);
     rc.advance(attn_unit(p, cta).nring, p.nslots);
-    return weight;
 }
 
 }  // namespace kl
