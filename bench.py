@@ -164,6 +164,47 @@ def run_device_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
     return e0.elapsed_time(e1)
 
 
+def run_graph_loop(dec, cache, tok0, context, batch, warmup, steps):
+    """The same greedy steps with ONE decode step (all its launches + sampling) captured in a CUDA graph and replayed:
+    the launch-overhead-free version of a schedule.  Returns ms for the K timed replays, or None with the reason when
+    the capture is refused."""
+    tok = tok0.clone()
+    pos = torch.full((batch,), context, dtype=torch.int32, device="cuda")
+    logits = torch.empty(batch, dec.shape.vocab, dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    try:
+        with torch.cuda.stream(side):
+            dec.kl_decode_step(tok, pos, cache, logits, batch, side)       # set-up outside the capture
+            dec.kl_argmax_advance(logits, tok, pos, batch, side)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                dec.kl_decode_step(tok, pos, cache, logits, batch, side)
+                dec.kl_argmax_advance(logits, tok, pos, batch, side)
+    except Exception as exc:  # capture not possible on this driver: report it, the plain launches stand
+        torch.cuda.synchronize()
+        return None, f"{type(exc).__name__}: {exc}".splitlines()[0][:200]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(side):
+        for _ in range(warmup):
+            graph.replay()
+        side.synchronize()
+        barrier()
+        e0.record(side)
+        for _ in range(steps):
+            graph.replay()
+        e1.record(side)
+        side.synchronize()
+    barrier()
+    st = dec.kl_last_status()
+    if st != 0:
+        return None, f"device status {st} after the replays"
+    if int(pos[0]) != context + 1 + warmup + steps:
+        return None, f"positions advanced to {int(pos[0])}, expected {context + 1 + warmup + steps}"
+    return e0.elapsed_time(e1), None
+
+
 def run_host_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
     """End to end through the host-buffer entry point: every step copies tokens and positions host->device,
     runs the step, copies the logits device->host, and the host picks the next token."""
@@ -347,6 +388,14 @@ def run_ours(args, shape, batch, context):
     # 2. the synchronisation-boundary schedule: one launch per layer
     dec.kl_set_mode(binding.KL_MODE_PER_LAYER)
     ms_layer = max_over_ranks(run_device_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    # 2b. both schedules again with one step captured in a CUDA graph (no per-launch host cost): the per-layer
+    #     baseline at its best, so that the looped kernel is not compared with a strawman
+    graph_ms, graph_err = {}, {}
+    for name, mode in (("looped", binding.KL_MODE_LOOPED), ("per_layer", binding.KL_MODE_PER_LAYER)):
+        dec.kl_set_mode(mode)
+        ms, err = run_graph_loop(dec, fresh_cache(), tok0, context, batch, W, K)
+        graph_ms[name] = max_over_ranks(ms) if ms is not None and not _DIST["on"] else ms
+        graph_err[name] = err
     # 3. roofline of the dominant kernel: events around the decoder launch inside the timed steps
     dec.kl_set_mode(binding.KL_MODE_LOOPED)
     dec.kl_profile_enable(K)
@@ -391,6 +440,8 @@ def run_ours(args, shape, batch, context):
         "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_looped / K * 1e-3) / 1e9,
                        "frac_of_measured_copy": bytes_step / (ms_looped / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
                        "frac_of_8tbs": bytes_step / (ms_looped / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+        "cuda_graph": {k: ({"value": tokens / (graph_ms[k] * 1e-3), "ms_per_step": graph_ms[k] / K} if graph_ms[k]
+                           else {"value": None, "why": graph_err[k]}) for k in graph_ms},
         "per_layer": {"value": tokens / (ms_layer * 1e-3), "ms_per_step": ms_layer / K,
                       "launches_per_step": shape.n_layers + 3,
                       "looped_speedup": ms_layer / ms_looped},

@@ -100,6 +100,8 @@ kl_status kl_set_mode(kl_handle* h, int mode);
  * batch-1 kernels -- the weights are streamed once per SEQUENCE; projections as M = batch tensor-core contractions,
  * which would stream them once per step, are not built.  Tokens and positions of the whole batch are checked
  * before the first sequence is decoded.
+ * The step reads tokens and positions on the device and keeps its own step counter there, so a stream capture of
+ * kl_decode_step + kl_argmax_advance can be replayed step after step (same buffers).
  * Merged-call argument rule of Section 3.2: weights (grouped, all layers) come from the handle, the hidden
  * state enters once (from the embedding) and leaves once (kl_read_hidden / the classifier), the KV cache is the
  * grouped in/out parameter.  Device-detected errors make the step a no-op and are reported by kl_last_status. */

@@ -38,7 +38,14 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
         }
     if (tok < 0 || tok >= (int32_t)p.V) tok = 0;
     const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
-    const uint32_t xtag = tag_of(p, 0, TG_XA);
+    // one more sequence on this handle: every tag of this launch sequence differs from all earlier ones
+    __shared__ uint32_t step_s;
+    if (tid == 0) {
+        step_s = *p.step_dev + 1u;
+        *p.step_dev = step_s;
+    }
+    __syncthreads();
+    const uint32_t xtag = tag_from(step_s, p.L, 0, TG_XA);
     for (uint32_t i = tid; i < p.H; i += blockDim.x) st_tw(p.xa + (size_t)b * p.H + i, __bfloat162float(row[i]), xtag);
     // RoPE table of this step: angle in double so that large positions keep their phase
     for (uint32_t i = tid; i < p.hd / 2; i += blockDim.x) {
@@ -281,7 +288,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, stok, spos, slogits, samax, shid, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, scratch_bytes;
     uint32_t cps;
 };
 
@@ -332,6 +339,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.sinvf = s;     s += align_up((size_t)(d.head_dim / 2) * 8);
     y.scounters = s; s += align_up((size_t)d.n_layers * 4);
     y.sstatus = s;   s += ALIGN;
+    y.sstep = s;     s += ALIGN;
     y.stok = s;      s += align_up(B * 4);
     y.spos = s;      s += align_up(B * 4);
     y.slogits = s;   s += align_up(B * V * 4);
@@ -571,6 +579,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.part = (TW*)(sc + y.spart); p.part_ml = (TW*)(sc + y.spart_ml); p.rope_cs = (float*)(sc + y.srope);
     p.inv_freq = (const double*)(sc + y.sinvf);
     p.counters = (uint32_t*)(sc + y.scounters);
+    p.step_dev = (uint32_t*)(sc + y.sstep);
     p.status = (int32_t*)(sc + y.sstatus);
     h->stage_tokens = (int32_t*)(sc + y.stok);
     h->stage_positions = (int32_t*)(sc + y.spos);
@@ -708,7 +717,6 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     for (uint32_t b = 0; b < batch; ++b) {
         p.b0 = b;
         p.logits = logits_d + (size_t)b * p.V;
-        p.step = ++h->prm.step;
         kl_embed_kernel<<<1, 256, 0, st>>>(p);
         if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
         ++h->launches;

@@ -83,7 +83,8 @@ struct Params {
     // plain fp32 guarded by a counter.
     struct TW *xa, *xb, *qkv, *o, *part, *part_ml;
     float *h, *rope_cs, *logits;
-    uint32_t step;         // decode steps issued on this handle so far (makes the tags of every step distinct)
+    uint32_t* step_dev;    // device word: sequences decoded on this handle so far (makes the tags of every launch
+                           // distinct).  The embedding kernel increments it, so a captured step can be replayed.
     const double* inv_freq;
     uint32_t* counters;    // [L]: CTAs that have finished the gate/up stage of each layer
     int32_t* status;
@@ -195,8 +196,12 @@ __device__ __forceinline__ uint4 ld_tw2(const TW* p) {
     return make_uint4((uint32_t)a, (uint32_t)(a >> 32), (uint32_t)b, (uint32_t)(b >> 32));
 }
 enum TagSlot { TG_XA = 0, TG_QKV = 1, TG_PART = 2, TG_O = 3, TG_XB = 4 };
+__device__ __forceinline__ uint32_t tag_from(uint32_t step, uint32_t L, uint32_t layer, uint32_t slot) {
+    return ((((step * L + layer) << 3) + slot) << 1) | 1u;
+}
+// The step word was written by the embedding kernel of this sequence, an earlier launch: a read-only load is fine.
 __device__ __forceinline__ uint32_t tag_of(const Params& p, uint32_t layer, uint32_t slot) {
-    return ((((p.step * p.L + layer) << 3) + slot) << 1) | 1u;
+    return tag_from(__ldg(p.step_dev), p.L, layer, slot);
 }
 
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
@@ -637,7 +642,7 @@ __device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* 
         }
     }
     if (norm && p.trace != nullptr && ctid == 0) {   // stamp 8: thread 0 holds valid data (diagnostic)
-        const uint32_t layer = ((tag >> 4) - p.step * p.L);
+        const uint32_t layer = (tag >> 4) % p.L;
         if (layer < p.L) p.trace[((size_t)blockIdx.x * p.L + layer) * TRACE_STAMPS + (((tag >> 1) & 7u) == TG_XA ? 8 : 11)] = globaltimer_ns();
     }
     if (norm) {

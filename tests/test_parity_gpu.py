@@ -103,6 +103,57 @@ def test_batch_bad_entry_makes_the_whole_step_a_no_op():
     dec.close()
 
 
+def test_captured_step_replays_like_plain_launches():
+    """One decode step + sampling captured in a CUDA graph and replayed gives the same tokens and logits as the same
+    steps launched one by one: nothing in a step depends on host state that a replay would not advance (the step
+    counter behind the tags lives on the device)."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 1, 200, 0)
+    cache0 = gen.make_kv_cache(shape, 1, 128, 200, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+
+    def plain(n):
+        cache, tok = cache0.clone(), tok0.clone()
+        pos = torch.tensor([128], dtype=torch.int32, device="cuda")
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        toks = []
+        for _ in range(n):
+            dec.kl_decode_step(tok, pos, cache, logits, 1)
+            dec.kl_argmax_advance(logits, tok, pos, 1)
+            toks.append(int(tok[0]))
+        torch.cuda.synchronize()
+        return toks, logits.cpu(), cache.cpu().view(torch.uint16)
+
+    ref_toks, ref_logits, ref_cache = plain(5)
+    cache, tok = cache0.clone(), tok0.clone()
+    pos = torch.tensor([128], dtype=torch.int32, device="cuda")
+    logits = torch.empty(1, shape.vocab, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    toks = []
+    with torch.cuda.stream(side):
+        dec.kl_decode_step(tok, pos, cache, logits, 1, side)   # first step outside the capture
+        dec.kl_argmax_advance(logits, tok, pos, 1, side)
+        side.synchronize()
+        toks.append(int(tok[0]))
+        graph = torch.cuda.CUDAGraph()
+        try:
+            with torch.cuda.graph(graph, stream=side):
+                dec.kl_decode_step(tok, pos, cache, logits, 1, side)
+                dec.kl_argmax_advance(logits, tok, pos, 1, side)
+        except Exception as exc:
+            pytest.skip(f"stream capture of the cooperative launches refused: {exc}")
+        for _ in range(4):
+            graph.replay()
+            side.synchronize()
+            toks.append(int(tok[0]))
+    assert dec.kl_last_status() == binding.KL_OK
+    assert toks == ref_toks
+    assert torch.equal(logits.cpu(), ref_logits)
+    assert torch.equal(cache.cpu().view(torch.uint16), ref_cache)
+    dec.close()
+
+
 def test_repeated_steps_are_bit_identical():
     """The same step from the same state, several times and in both schedules: identical logits and hidden state.
     Any race between the warps of a CTA or between CTAs (a buffer reused too early) shows up here as run-to-run
