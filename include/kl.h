@@ -40,7 +40,7 @@ enum {
     KL_ERR_TOO_LARGE = -7          /* a size beyond the fixed capacity of kl_argmax_advance_static */
 };
 
-enum { KL_MODE_LOOPED = 0, KL_MODE_PER_LAYER = 1 };
+enum { KL_MODE_LOOPED = 0, KL_MODE_PER_LAYER = 1, KL_MODE_PER_STAGE = 2 };
 
 /* Tensors accepted by kl_load_weights; all bf16, row-major [out_features, in_features] (gains: [hidden]). */
 enum {
@@ -87,7 +87,10 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
  * bf16.  Cached keys are stored already rotated.  The cache is caller-owned and updated in place. */
 size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch);
 
-/* KL_MODE_LOOPED (default): one persistent kernel runs all layers.  KL_MODE_PER_LAYER: one launch per layer. */
+/* KL_MODE_LOOPED (default): one persistent kernel runs all layers (4 launches per token with embedding, classifier
+ * and sampling).  KL_MODE_PER_LAYER: one launch per layer (L + 3).  KL_MODE_PER_STAGE: one launch per operator group
+ * of every layer -- QKV, attention, O, gate/up, down (5 L + 3): the three call schedules of Section 3.2, from the
+ * same stage code. */
 kl_status kl_set_mode(kl_handle* h, int mode);
 
 /* One decode step for `batch` sequences, asynchronous on `stream`.

@@ -22,6 +22,7 @@ KL_ERR_TOO_LARGE = -7
 KL_STATIC_ARGMAX_MAX_BATCH = 256
 KL_MODE_LOOPED = 0
 KL_MODE_PER_LAYER = 1
+KL_MODE_PER_STAGE = 2
 
 TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup": 6, "wdown": 7,
               "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11}

@@ -73,8 +73,11 @@ __device__ __noinline__ void attention_block(const Params& p, const Smem& s, uin
     attention_flush_new_row(p, s, l, cta, ctid);
 }
 
-// Layers [l0, l1) of the decoder.  l1 - l0 == L is the looped kernel; l1 - l0 == 1 the per-layer launch.
-__global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1) {
+// Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
+// stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
+// boundary after every operator group).
+__global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
+                                                                 uint32_t sbeg, uint32_t send) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
@@ -93,7 +96,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
 
     if (warp == NCW) {
         // producer warp: one thread streams the CTA's chunk sequence into the ring
-        if (lane == 0) produce_decoder(p, s, cta, l0, l1);
+        if (lane == 0) produce_decoder(p, s, cta, l0, l1, sbeg, send);
         return;
     }
     WarpRing wr = ring_begin();
@@ -108,12 +111,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
         // test hook: the results of one stage of layer 0 get a tag nobody waits for
         const int skip = (l == 0) ? p.skip_stage : -1;
         const uint32_t bad = 0x2u;
-        for (int st = 0; st < 4; ++st) {
-            GemvOut out;
-            int plan, ep;
+        for (uint32_t st = sbeg; st < send; ++st) {
+            GemvOut out = {nullptr, nullptr, nullptr, 0u};
+            int plan = PL_QKV, ep = EP_STORE;
             const float* xsrc = nullptr;
-            if (st == 0) {
-                // S1: RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the
+            if (st == ST_QKV) {
+                // RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the
                 // embedding).
                 trace_stamp(p, cta, l, 0, ctid);
                 load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
@@ -121,39 +124,43 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
                 out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
                 plan = PL_QKV;
                 ep = EP_STORE;
-            } else if (st == 1) {
+            } else if (st == ST_ATTN) {
                 trace_stamp(p, cta, l, 2, ctid);
-                // S2: RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
+                // RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
                 attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
                 trace_stamp(p, cta, l, 4, ctid);
-                // S3: output projection + residual (xa -> xb).  The poll on o's tags waits for the mergers.
+                continue;
+            } else if (st == ST_O) {
+                // output projection + residual (xa -> xb).  The poll on o's tags waits for the attention units.
                 load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
                 trace_stamp(p, cta, l, 6, ctid);
                 out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, l, TG_XB)};
                 plan = PL_O;
                 ep = EP_RESIDUAL;
-            } else if (st == 2) {
+            } else if (st == ST_GU) {
                 trace_stamp(p, cta, l, 7, ctid);
-                // S4: RMSNorm + gate/up projections + SwiGLU
+                // RMSNorm + gate/up projections + SwiGLU
                 load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
                 trace_stamp(p, cta, l, 9, ctid);
                 out = {nullptr, p.h, nullptr, 0u};
                 plan = PL_GU;
                 ep = EP_SWIGLU;
             } else {
-                // h is plain fp32 read per warp and per column piece straight from L2 into registers (too wide for
-                // tagged words): its readiness is a counter, signalled with release and awaited with acquire
-                stage_signal(p.counters + l, ctid, skip == ST_GU);
-                trace_stamp(p, cta, l, 10, ctid);
+                // down projection + residual (xb -> xa of the next layer).  h is plain fp32 read per warp and per
+                // column piece straight from L2 into registers (too wide for shared memory): its readiness is a
+                // counter, signalled with release at the end of the gate/up stage and awaited with acquire here
                 stage_wait(p, s, p.counters + l, p.P, ctid);
                 trace_stamp(p, cta, l, 12, ctid);
-                // S5: down projection + residual (xb -> xa of the next layer)
                 out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
                 plan = PL_D;
                 ep = EP_RESIDUAL;
                 xsrc = p.h;
             }
             gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc);
+            if (st == ST_GU) {
+                stage_signal(p.counters + l, ctid, skip == ST_GU);
+                trace_stamp(p, cta, l, 10, ctid);
+            }
         }
         trace_stamp(p, cta, l, 13, ctid);
     }
@@ -676,7 +683,7 @@ size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch) {
 }
 
 kl_status kl_set_mode(kl_handle* h, int mode) {
-    if (!h || (mode != KL_MODE_LOOPED && mode != KL_MODE_PER_LAYER)) return KL_ERR_INVALID_ARG;
+    if (!h || (mode != KL_MODE_LOOPED && mode != KL_MODE_PER_LAYER && mode != KL_MODE_PER_STAGE)) return KL_ERR_INVALID_ARG;
     h->mode = mode;
     return KL_OK;
 }
@@ -722,16 +729,24 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         ++h->launches;
         kl_status rc;
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+        uint32_t sbeg = 0, send = 5;
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
-            void* args[] = {&p, &l0, &l1};
+            void* args[] = {&p, &l0, &l1, &sbeg, &send};
             if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
-        } else {
+        } else if (h->mode == KL_MODE_PER_LAYER) {
             for (uint32_t l = 0; l < p.L; ++l) {
                 uint32_t l0 = l, l1 = l + 1;
-                void* args[] = {&p, &l0, &l1};
+                void* args[] = {&p, &l0, &l1, &sbeg, &send};
                 if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
             }
+        } else {
+            for (uint32_t l = 0; l < p.L; ++l)
+                for (uint32_t sg = 0; sg < 5; ++sg) {
+                    uint32_t l0 = l, l1 = l + 1, s0 = sg, s1 = sg + 1;
+                    void* args[] = {&p, &l0, &l1, &s0, &s1};
+                    if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+                }
         }
         if (ev && b == 0 && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
         Params pc = p;

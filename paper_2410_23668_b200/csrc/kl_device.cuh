@@ -556,16 +556,19 @@ __device__ __forceinline__ void produce_drain(const Params& p, const Smem& s, co
 }
 
 // The producer thread of the decoder kernel: layers [l0, l1).
-__device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, uint32_t cta, uint32_t l0, uint32_t l1) {
+__device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, uint32_t cta, uint32_t l0, uint32_t l1,
+                                                uint32_t sbeg, uint32_t send) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     const AttnUnit u = attn_unit(p, cta);
     for (uint32_t l = l0; l < l1 && !r.aborted; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
-        produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
-        produce_attention(p, s, r, u, l);
-        produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
-        produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
-        produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+        for (uint32_t st = sbeg; st < send; ++st) {
+            if (st == ST_QKV) produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
+            else if (st == ST_ATTN) produce_attention(p, s, r, u, l);
+            else if (st == ST_O) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+            else if (st == ST_GU) produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
+            else produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+        }
     }
     produce_drain(p, s, r);
 }

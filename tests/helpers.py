@@ -75,7 +75,8 @@ def bf16_decode(u16: np.ndarray) -> np.ndarray:
     return (u16.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
 
 
-def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None, modes=(binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER),
+def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
+               modes=(binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER, binding.KL_MODE_PER_STAGE),
                overrides=None, positions0=None, stream_layers=False, check_cache=True):
     """Teacher-forced greedy decode: the oracle runs `steps` steps on its own tokens; each CUDA mode consumes the
     oracle's token of the previous step.  Returns a report dict; asserts nothing."""
@@ -144,9 +145,9 @@ def assert_parity(report, steps, batch=1, check_cache=True):
             assert np.all(np.abs(g - e) <= 2.0 ** -7 * np.abs(e) + 1e-3 * np.abs(e).max()), mode
             assert (got[changed] != exp[changed]).mean() < 0.02, mode
     modes = list(report["modes"].values())
-    if len(modes) == 2:  # the transformation preserves semantics: both schedules run the same arithmetic
+    for other in modes[1:]:  # the transformation preserves semantics: all schedules run the same arithmetic
         for s in range(steps):
-            assert np.array_equal(modes[0]["steps"][s]["logits"], modes[1]["steps"][s]["logits"]), s
-            assert np.array_equal(modes[0]["steps"][s]["hidden"], modes[1]["steps"][s]["hidden"]), s
+            assert np.array_equal(modes[0]["steps"][s]["logits"], other["steps"][s]["logits"]), s
+            assert np.array_equal(modes[0]["steps"][s]["hidden"], other["steps"][s]["hidden"]), s
         if modes[0]["cache"] is not None:
-            assert np.array_equal(modes[0]["cache"], modes[1]["cache"])
+            assert np.array_equal(modes[0]["cache"], other["cache"])

@@ -21,7 +21,7 @@ def test_generator_is_bit_identical_on_cpu_and_cuda():
     assert torch.equal(a, b)
 
 
-def test_tiny_16_greedy_steps_both_modes():
+def test_tiny_16_greedy_steps_all_schedules():
     """Config 1: 4 layers, hidden 256, 4/2 heads of 64, FFN 512, vocab 1024, 128 cached positions, 16 steps."""
     rep = helpers.run_parity(gen.TINY, context=128, steps=16, seed=0)
     helpers.assert_parity(rep, 16)
@@ -166,7 +166,7 @@ def test_repeated_steps_are_bit_identical():
     tok = gen.make_tokens(shape, 1, 0).cuda()
     pos = torch.tensor([context], dtype=torch.int32, device="cuda")
     outs = []
-    for mode in (binding.KL_MODE_LOOPED,) * 4 + (binding.KL_MODE_PER_LAYER,) * 2:
+    for mode in (binding.KL_MODE_LOOPED,) * 4 + (binding.KL_MODE_PER_LAYER,) * 2 + (binding.KL_MODE_PER_STAGE,) * 2:
         dec.kl_set_mode(mode)
         cache = cache0.clone()
         logits = torch.empty(1, shape.vocab, device="cuda")
