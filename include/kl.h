@@ -6,7 +6,8 @@
  * (Section 2, call-schedule figure).  In KL_MODE_LOOPED the L consecutive calls to the decoder-layer
  * kernel are one call to a persistent kernel with an outer loop over layers (Section 3.2, rules
  * (1)-(10)); in KL_MODE_PER_LAYER the same kernel body is launched once per layer, which is the
- * synchronisation-boundary schedule the transformation removes (Section 2, schedule (ii)).
+ * synchronisation-boundary schedule the transformation removes (Section 2, schedule (ii)); in
+ * KL_MODE_PER_STAGE once per operator group of every layer (schedule (i)).
  *
  * Conventions
  *   - All pointers named *_d are DEVICE pointers, *_h are HOST pointers.  Nothing here allocates or frees
@@ -147,7 +148,8 @@ kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_
 kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream);
 
 /* Synchronises nothing: call after the stream has been synchronised.  Reads and clears the device status word
- * (KL_OK, KL_ERR_SYNC_TIMEOUT or KL_ERR_OUT_OF_RANGE). */
+ * (KL_OK, KL_ERR_SYNC_TIMEOUT or KL_ERR_OUT_OF_RANGE).  The word is sticky: once a step has set it, every later
+ * step on the handle is a no-op until this call has read (and thereby cleared) it. */
 kl_status kl_last_status(kl_handle* h);
 
 /* Number of kernels this handle has launched so far (for reporting). */
