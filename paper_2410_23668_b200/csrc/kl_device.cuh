@@ -594,7 +594,7 @@ __device__ __forceinline__ uint32_t vec_perm(uint32_t e) {
 // all tags in place already holds the data.
 __device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
                                          const __nv_bfloat16* gain, uint32_t ctid) {
-    constexpr int NB = 6;  // groups of four values kept in flight per thread (two 16-byte loads each)
+    constexpr int NB = 4;  // groups of four values kept in flight per thread (two 16-byte loads each)
     // The vector area is about to be overwritten: every warp of the CTA must be done with what the previous stage
     // kept there (the stage's input vector, read block by block until a warp's last chunk; the attention workspace).
     consumer_bar();
