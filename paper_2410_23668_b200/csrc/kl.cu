@@ -115,11 +115,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
             GemvOut out = {nullptr, nullptr, nullptr, 0u};
             int plan = PL_QKV, ep = EP_STORE;
             const float* xsrc = nullptr;
+            float xscale = 1.f;   // RMSNorm's normaliser of the stage's input vector, applied to the stage's outputs
             if (st == ST_QKV) {
                 // RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the
                 // embedding).
                 trace_stamp(p, cta, l, 0, ctid);
-                load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
+                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
                 trace_stamp(p, cta, l, 1, ctid);
                 out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
                 plan = PL_QKV;
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
             } else if (st == ST_GU) {
                 trace_stamp(p, cta, l, 7, ctid);
                 // RMSNorm + gate/up projections + SwiGLU
-                load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
+                xscale = load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
                 trace_stamp(p, cta, l, 9, ctid);
                 out = {nullptr, p.h, nullptr, 0u};
                 plan = PL_GU;
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
                 ep = EP_RESIDUAL;
                 xsrc = p.h;
             }
-            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc);
+            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
             if (st == ST_GU) {
                 stage_signal(p.counters + l, ctid, skip == ST_GU);
                 trace_stamp(p, cta, l, 10, ctid);
@@ -189,9 +190,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     }
     WarpRing wr = ring_begin();
     RingCursor rc = {0u, 0u};
-    load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, tid);
+    const float xscale = load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, tid);
     const GemvOut out = {nullptr, p.logits, nullptr, 0u};
-    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr);
+    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr, xscale);
 }
 
 // Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per

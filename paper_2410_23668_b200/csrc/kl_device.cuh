@@ -8,6 +8,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#ifndef KL_POLL_NS
+#define KL_POLL_NS 64
+#endif
 #ifndef KL_ST_TW
 #define KL_ST_TW "st.relaxed.gpu.global.b64"
 #endif
@@ -278,7 +281,7 @@ struct PollGuard {
 };
 __device__ __forceinline__ bool poll_continue(const Params& p, const Smem& s, PollGuard& g) {
     if (g.it == 0) g.t0 = globaltimer_ns();
-    __nanosleep(64);   // keeps the polling traffic of a waiting CTA off the L2 ports the late CTAs still need
+    if (KL_POLL_NS) __nanosleep(KL_POLL_NS);   // keeps the polling traffic of a waiting CTA off the L2 ports the late CTAs still need
     if ((++g.it & 7u) == 0) {
         if (*s.abort_flag) return false;
         if (__ldcg(p.status) != 0) {
@@ -589,37 +592,34 @@ __device__ __forceinline__ uint32_t vec_perm(uint32_t e) {
 }
 
 // Loads the tagged vector src[0..n) (produced by other CTAs) into the shared vector area, polling until every word
-// carries `tag`, and optionally applies RMSNorm with bf16 gains.  Every CTA recomputes the norm; the summation
-// order is fixed.  This poll is what replaces the grid-wide barrier of a kernel boundary: the first read that finds
+// carries `tag`.  With `norm` the values are multiplied by the bf16 gains on the way in and the function returns
+// rsqrt(mean(x^2) + eps): RMSNorm's normaliser is one number for the whole vector, so the stage applies it to its
+// outputs instead of to its 4096 inputs (one pass and one barrier less).  Every CTA recomputes it; the summation
+// order is fixed.  Without `norm` the function returns 1.  This poll is what replaces the grid-wide barrier of a kernel boundary: the first read that finds
 // all tags in place already holds the data.
-__device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
-                                         const __nv_bfloat16* gain, uint32_t ctid) {
+__device__ __noinline__ float load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
+                                          const __nv_bfloat16* gain, uint32_t ctid) {
     constexpr int NB = 4;  // groups of four values kept in flight per thread (two 16-byte loads each)
     // The vector area is about to be overwritten: every warp of the CTA must be done with what the previous stage
     // kept there (the stage's input vector, read block by block until a warp's last chunk; the attention workspace).
     consumer_bar();
     float ss = 0.f;
-    const bool single = n <= (uint32_t)(NB * NCT * 4);
-    float4 keep[NB];
-    uint2 gkeep[NB];
     for (uint32_t base = 0; base < n; base += NB * NCT * 4) {
         float4 v[NB];
-        if (norm && single) {
-#pragma unroll
-            for (int i = 0; i < NB; ++i) {
-                const uint32_t e = (ctid + i * NCT) * 4;
-                gkeep[i] = make_uint2(0u, 0u);
-                if (e < n) gkeep[i] = __ldg(reinterpret_cast<const uint2*>(gain + e));
-            }
-        }
+        uint2 gk[NB];
         // Only the groups whose tags are not all in place yet are read again: the words that are late come from the
         // few CTAs that finish the previous stage last, and re-reading the whole vector from every waiting CTA
         // floods the L2 slices those late CTAs stream their weights through.
         uint32_t pend = 0u;
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
+            const uint32_t e = base + (ctid + i * NCT) * 4;
             v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (base + (ctid + i * NCT) * 4 < n) pend |= 1u << i;
+            gk[i] = make_uint2(0x3f803f80u, 0x3f803f80u);   // bf16 ones
+            if (e < n) {
+                pend |= 1u << i;
+                if (norm) gk[i] = __ldg(reinterpret_cast<const uint2*>(gain + e));
+            }
         }
         PollGuard pg = {0ull, 0u, (int)(tag & 15u) + 100};
         for (;;) {
@@ -640,50 +640,32 @@ __device__ __noinline__ void load_vec(const Params& p, const Smem& s, const TW* 
         for (int i = 0; i < NB; ++i) {
             const uint32_t e = base + (ctid + i * NCT) * 4;
             ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
-            if (norm && single) keep[i] = v[i];
-            else if (e < n) *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = v[i];
+            if (e < n) {
+                // the gains go in now, the normaliser (one number for the whole vector) is applied to the stage's outputs
+                const float4 o = make_float4(v[i].x * bf_lo(gk[i].x), v[i].y * bf_hi(gk[i].x), v[i].z * bf_lo(gk[i].y),
+                                             v[i].w * bf_hi(gk[i].y));
+                *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = o;
+            }
         }
     }
-    if (norm && p.trace != nullptr && ctid == 0) {   // stamp 8: thread 0 holds valid data (diagnostic)
+    if (norm && p.trace != nullptr && ctid == 0) {   // stamps 8 / 11: thread 0 holds valid data (diagnostic)
         const uint32_t layer = (tag >> 4) % p.L;
-        if (layer < p.L) p.trace[((size_t)blockIdx.x * p.L + layer) * TRACE_STAMPS + (((tag >> 1) & 7u) == TG_XA ? 8 : 11)] = globaltimer_ns();
+        p.trace[((size_t)blockIdx.x * p.L + layer) * TRACE_STAMPS + (((tag >> 1) & 7u) == TG_XA ? 8 : 11)] = globaltimer_ns();
     }
+    float inv = 1.f;
     if (norm) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if ((ctid & 31) == 0) s.red[ctid >> 5] = ss;
-        consumer_bar();
+    }
+    consumer_bar();
+    if (norm) {
         float tot = 0.f;
 #pragma unroll
         for (int w = 0; w < NCW; ++w) tot += s.red[w];
-        const float inv = rsqrtf(tot / (float)n + p.eps);
-        if (single) {
-#pragma unroll
-            for (int i = 0; i < NB; ++i) {
-                const uint32_t e = (ctid + i * NCT) * 4;
-                if (e < n) {
-                    float4 o;
-                    o.x = keep[i].x * inv * bf_lo(gkeep[i].x);
-                    o.y = keep[i].y * inv * bf_hi(gkeep[i].x);
-                    o.z = keep[i].z * inv * bf_lo(gkeep[i].y);
-                    o.w = keep[i].w * inv * bf_hi(gkeep[i].y);
-                    *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = o;
-                }
-            }
-        } else {
-            for (uint32_t e = ctid * 4; e < n; e += NCT * 4) {
-                float4* q = reinterpret_cast<float4*>(s.vec + vec_perm(e));
-                const uint2 gb = __ldg(reinterpret_cast<const uint2*>(gain + e));
-                float4 v = *q;
-                v.x *= inv * bf_lo(gb.x);
-                v.y *= inv * bf_hi(gb.x);
-                v.z *= inv * bf_lo(gb.y);
-                v.w *= inv * bf_hi(gb.y);
-                *q = v;
-            }
-        }
+        inv = rsqrtf(tot / (float)n + p.eps);
     }
-    consumer_bar();
+    return inv;
 }
 
 // This lane's share of a slice of the input vector: for block b of 256 columns the 8 columns b*256 + lane*8 .. +7.
@@ -923,7 +905,7 @@ __device__ __forceinline__ void emit_value(const GemvOut& o, uint32_t idx, float
 
 __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
                                         uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
-                                        const float* xsrc) {
+                                        const float* xsrc, float xscale) {
     // xsrc == nullptr: the input vector is staged in s.vec; otherwise it is read from global memory per piece
     const CtaRange r = cta_units(pl, cta, p.P);
     const uint32_t nch = (r.u1 - r.u0) * pl.npieces;
@@ -978,12 +960,12 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
                 y[3] = warp_sum(y[3]);
             }
             if (ep == EP_SWIGLU) {
-                if (lane == 0) emit_value(out, g.row >> 1, silu(y[0]) * y[1]);
-                if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2]) * y[3]);
+                if (lane == 0) emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
+                if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
             } else if (lane < g.nrows) {
                 // lane rr emits row rr (every lane holds all sums after the butterfly)
                 const float v = lane == 0 ? y[0] : lane == 1 ? y[1] : lane == 2 ? y[2] : y[3];
-                emit_value(out, g.row + lane, (ep == EP_RESIDUAL ? res : 0.f) + v);
+                emit_value(out, g.row + lane, (ep == EP_RESIDUAL ? res : 0.f) + v * xscale);
             }
         } else if (pl.rpc <= MAX_RPC_SPLIT) {
             // one unit piece of up to four rows: the common case.  Residual inputs are fetched before the wait, their
@@ -1044,12 +1026,12 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
                 }
                 if (emit) {
                     if (ep == EP_SWIGLU) {
-                        emit_value(out, g.row >> 1, silu(y[0]) * y[1]);
-                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2]) * y[3]);
+                        emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
+                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
                     } else {
 #pragma unroll
                         for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
-                            if ((uint32_t)rr < g.nrows) emit_value(out, g.row + rr, (ep == EP_RESIDUAL ? rs[rr] : 0.f) + y[rr]);
+                            if ((uint32_t)rr < g.nrows) emit_value(out, g.row + rr, (ep == EP_RESIDUAL ? rs[rr] : 0.f) + y[rr] * xscale);
                     }
                 }
             }
@@ -1079,13 +1061,13 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
                 if (lane == 0) {
                     const uint32_t row = g.row + rr;
                     if (ep == EP_STORE) {
-                        emit_value(out, row, y0);
-                        if (two) emit_value(out, row + 1, y1);
+                        emit_value(out, row, y0 * xscale);
+                        if (two) emit_value(out, row + 1, y1 * xscale);
                     } else if (ep == EP_RESIDUAL) {
-                        emit_value(out, row, rs0 + y0);
-                        if (two) emit_value(out, row + 1, rs1 + y1);
+                        emit_value(out, row, rs0 + y0 * xscale);
+                        if (two) emit_value(out, row + 1, rs1 + y1 * xscale);
                     } else {
-                        emit_value(out, row >> 1, silu(y0) * y1);
+                        emit_value(out, row >> 1, silu(y0 * xscale) * (y1 * xscale));
                     }
                 }
             }
