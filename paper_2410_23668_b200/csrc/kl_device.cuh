@@ -1282,7 +1282,7 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
     float* pv = wtab + 2 * G * nchunk;       // [ns][nchunk] partial outputs of this unit's slice
     consumer_bar();                          // the per-warp partials in comb are no longer needed
     // all loads of a thread are issued before it waits on any of them; only those that are late are repeated
-    constexpr int NL = 4;
+    constexpr int NL = 2;
     const uint32_t nml = G * nchunk, npv = ns * nchunk;
     for (uint32_t i0 = 0; i0 < max(nml, (npv + NL - 1) / NL); i0 += NCT) {
         const uint32_t i = i0 + ctid;
@@ -1530,28 +1530,23 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h),
     // in place; then thread t owns (head, column) and adds the NCW weighted terms in warp order.
     const uint32_t unit = u.bg * p.cps + u.ch;
-    {
-        float fw = 0.f, Mh = -INFINITY;
+    float* ftab = s.unit_part;   // [NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
+    if (ctid < NCW * G) {
         const uint32_t w = ctid / G, h = ctid % G;
-        if (ctid < NCW * G) {
+        float Mh = -INFINITY;
 #pragma unroll
-            for (int ww = 0; ww < NCW; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (hd + 2) + hd]);
-            fw = rescale(comb[((size_t)w * G + h) * (hd + 2) + hd], Mh);
-        }
-        consumer_bar();
-        if (ctid < NCW * G) {
-            comb[((size_t)w * G + h) * (hd + 2) + hd] = fw;
-            if (w == 0) s.red[h] = Mh;
-        }
-        consumer_bar();
+        for (int ww = 0; ww < NCW; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (hd + 2) + hd]);
+        ftab[w * G + h] = rescale(comb[((size_t)w * G + h) * (hd + 2) + hd], Mh);
+        if (w == 0) ftab[NCW * G + h] = Mh;
     }
+    consumer_bar();
     for (uint32_t t = ctid; t < G * hd; t += NCT) {
         const uint32_t h = t / hd, d = t % hd;
         float A = 0.f, Lsum = 0.f;
 #pragma unroll
         for (int w = 0; w < NCW; ++w) {
             const float* src = comb + ((size_t)w * G + h) * (hd + 2);
-            const float c = src[hd];
+            const float c = ftab[w * G + h];
             A += src[d] * c;
             Lsum += src[hd + 1] * c;
         }
@@ -1561,7 +1556,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
             const uint32_t ptag = tag_of(p, layer, TG_PART);
             st_tw(p.part + ((size_t)unit * G + h) * hd + d, A, ptag);
             if (d == 0) {
-                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, s.red[h], ptag);
+                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, ftab[NCW * G + h], ptag);
                 st_tw(p.part_ml + ((size_t)unit * G + h) * 2 + 1, Lsum, ptag);
             }
         }
