@@ -69,7 +69,8 @@ __device__ __noinline__ void attention_block(const Params& p, const Smem& s, uin
         case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
         default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
     }
-    consumer_bar();
+    // the row written by this step is copied from the workspace to the cache here; the next vector load starts with
+    // a CTA barrier, so the workspace is not overwritten before this copy has read it
     attention_flush_new_row(p, s, l, cta, ctid);
 }
 
@@ -551,9 +552,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     uint32_t vecf = p.H > p.QD ? p.H : p.QD;  // the down projection reads its input from L2, not from this area
     vecf = ceil_div(vecf, 256) * 256;
     // attention workspace: rotated q, the new K/V row, per-warp partial results, the staging tile of the new row
-    // (the same area then holds the merge tables: 2 * G * nchunk pairs and the unit's slice of every partial output)
+    // and, behind them, the merge tables: 2 * G * nchunk pairs and the unit's slice of every partial output
     const uint32_t comb_f = NCW * p.G * (p.hd + 2), merge_f = 2 * p.G * (p.P / p.nkv) + p.G * p.hd + 2 * (p.P / p.nkv);  // batch 1 has the most chunks
-    const uint32_t attnf = p.G * p.hd + 2 * p.hd + 128 + (comb_f > merge_f ? comb_f : merge_f);
+    const uint32_t attnf = p.G * p.hd + 2 * p.hd + 128 + comb_f + merge_f;
     if (attnf > vecf) vecf = ceil_div(attnf, 256) * 256;
     p.vec_floats = vecf;
     int max_optin = 0;

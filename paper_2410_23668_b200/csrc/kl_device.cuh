@@ -1278,9 +1278,9 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
     const uint32_t S = (total + nchunk - 1) / nchunk;
     const uint32_t t_lo = min(total, u.ch * S), t_hi = min(total, t_lo + S);
     const uint32_t ns = t_hi - t_lo;
-    float* wtab = comb;                      // [2][G][nchunk]: maxima, sums; then weights in the first half
-    float* pv = wtab + 2 * G * nchunk;       // [ns][nchunk] partial outputs of this unit's slice
-    consumer_bar();                          // the per-warp partials in comb are no longer needed
+    // the tables sit behind the per-warp partials, which other threads of the CTA may still be reading
+    float* wtab = comb + (size_t)NCW * G * (hd + 2);   // [2][G][nchunk]: maxima, sums; then weights in the first half
+    float* pv = wtab + 2 * G * nchunk;                 // [ns][nchunk] partial outputs of this unit's slice
     // all loads of a thread are issued before it waits on any of them; only those that are late are repeated
     constexpr int NL = 2;
     const uint32_t nml = G * nchunk, npv = ns * nchunk;
@@ -1527,8 +1527,8 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     trace_stamp(p, cta, layer, 15, ctid);
     consumer_bar();
 
-    // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h),
-    // in place; then thread t owns (head, column) and adds the NCW weighted terms in warp order.
+    // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h);
+    // then thread t owns (head, column) and adds the NCW weighted terms in warp order.
     const uint32_t unit = u.bg * p.cps + u.ch;
     float* ftab = s.unit_part;   // [NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
     if (ctid < NCW * G) {
