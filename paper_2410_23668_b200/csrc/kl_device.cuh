@@ -242,7 +242,7 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
 // Records the first error and tells every waiter of this CTA to give up.  After an abort every wait returns at
 // once but the control flow (stage order, CTA barriers) is unchanged, so no warp is left behind at a barrier; the
 // step's outputs are then meaningless and the status word says so.
-__device__ __forceinline__ bool raise_abort(const Params& p, const Smem& s, int code, int where = 0) {
+__device__ __noinline__ bool raise_abort(const Params& p, const Smem& s, int code, int where = 0) {
     bool first = false;
     if (atomicCAS(p.status, 0, code) == 0) {   // following words: which wait gave up, where (diagnostics)
         p.status[1] = where;
@@ -264,7 +264,7 @@ __device__ __forceinline__ bool mbar_wait(const Params& p, const Smem& s, uint32
         if ((++it & 63u) == 0) {
             if (*s.abort_flag) return false;
             if (globaltimer_ns() - t0 > p.wait_ns) {
-                raise_abort(p, s, ERR_SYNC_TIMEOUT, 500);
+                raise_abort(p, s, ERR_SYNC_TIMEOUT, 500);   // out of line: it runs once, if ever
                 return false;
             }
         }
