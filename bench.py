@@ -474,7 +474,7 @@ def run_ours(args, shape, batch, context):
 # dram__bytes_read.sum + dram__bytes_write.sum of one looped launch over 4 layers of the 8B shape at batch 1,
 # context 4096 (ncu capture summarised under profiles/), per layer.  Every layer streams its own weights and KV once,
 # so a full launch is this times the layer count.
-NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813762e9 + 28.287744e6) / 4
+NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813534e9 + 15.228672e6) / 4
 
 
 def ncu_traffic(shape, batch, context):
