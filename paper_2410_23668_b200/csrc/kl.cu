@@ -383,7 +383,9 @@ GemvPlan make_plan(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t alig
         // units cut into column pieces.  A piece count that divides the consumer count (or is a multiple of it)
         // keeps every consumer on the same column piece for a whole stage, so its share of the input vector
         // stays in registers.
-        const uint32_t kp_max = MAX_KP / 256u * 256u;
+        // pieces multiplied against shared memory may be as long as a slot allows; pieces whose vector slice lives in
+        // registers are capped
+        const uint32_t kp_max = x_in_smem ? (uint32_t)SLOT_BYTES / (2u * minrows) / 256u * 256u : MAX_KP / 256u * 256u;
         uint32_t np = ceil_div(K, kp_max);
         const uint32_t cand[5] = {1, 2, 3, NCW, 2 * NCW};
         for (int q = 0; q < 5; ++q)
@@ -408,7 +410,7 @@ bool plans_ok(const Params& p) {
     for (int i = 0; i < PL_COUNT; ++i) {
         const GemvPlan& pl = p.plan[i];
         if (pl.npieces > (uint32_t)MAX_PIECES || pl.rpc < 1) return false;
-        if (pl.kp > MAX_KP && (pl.npieces > 1 || i == PL_D || pl.rpc > (uint32_t)MAX_RPC_SPLIT)) return false;
+        if (pl.kp > MAX_KP && (i == PL_D || pl.rpc > (uint32_t)MAX_RPC_SPLIT)) return false;
         if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
         if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % (i == PL_D ? 8 : 256))) return false;
         if (i == PL_GU && (pl.rpc & 1u)) return false;

@@ -903,6 +903,28 @@ __device__ __forceinline__ void emit_value(const GemvOut& o, uint32_t idx, float
     else o.plain[idx] = v;
 }
 
+// Partial sums of a unit's column pieces meet in shared memory; the last piece to arrive adds them in piece order.
+// Called by one lane per chunk.  Returns true for that last piece, with the unit's complete sums in y.
+__device__ __forceinline__ bool unit_combine(const Smem& s, const GemvPlan& pl, const ChunkGeom& g, uint32_t u0,
+                                             float (&y)[MAX_RPC_SPLIT]) {
+    const uint32_t us = (g.unit - u0) % UNIT_SLOTS;
+    volatile float* part = s.unit_part + us * (MAX_PIECES * MAX_RPC_SPLIT);
+#pragma unroll
+    for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) part[g.piece * MAX_RPC_SPLIT + rr] = y[rr];
+    __threadfence_block();
+    const int old = atomicAdd(&s.unit_cnt[us], 1);
+    if (old != (int)pl.npieces - 1) return false;
+    __threadfence_block();
+    s.unit_cnt[us] = 0;
+#pragma unroll
+    for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = 0.f;
+    for (uint32_t j = 0; j < pl.npieces; ++j) {
+#pragma unroll
+        for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] += part[j * MAX_RPC_SPLIT + rr];
+    }
+    return true;
+}
+
 __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
                                         uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
                                         const float* xsrc, float xscale) {
@@ -913,7 +935,7 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
     XRegs x;
     uint32_t x_piece = 0xffffffffu;
     // rows that come whole and find their vector in shared memory are multiplied against it block by block
-    const bool smemx = xsrc == nullptr && pl.npieces == 1u && pl.rpc <= (uint32_t)MAX_RPC_SPLIT;
+    const bool smemx = xsrc == nullptr && pl.rpc <= (uint32_t)MAX_RPC_SPLIT;
     for (uint32_t i = first; i < nch; i += p.nslots) {
         const ChunkGeom g = chunk_geom(pl, r.u0, i);
         if (!smemx && g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
@@ -925,8 +947,9 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
         const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
         const uint32_t pitch = g.klen * 2u;
         if (smemx) {
-            // Whole rows, the vector taken from shared memory block by block: no cross-warp combine, the warp that
-            // multiplied the rows emits them.
+            // Rows (or, for rows longer than a slot, column pieces starting at a block of 256) multiplied against the
+            // vector in shared memory block by block.  Whole rows need no cross-warp combine: the warp that
+            // multiplied them emits them.
             float res = 0.f;
             if (ep == EP_RESIDUAL && lane < g.nrows) res = ld_tw(out.res + g.row + lane).v;
             mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
@@ -935,19 +958,19 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             float y[MAX_RPC_SPLIT] = {0.f, 0.f, 0.f, 0.f};
             if (g.nrows == 2) {
                 float acc[2];
-                dot_rows_smemx<2>(sp, pitch, g.klen, lane, s.vec, acc);
+                dot_rows_smemx<2>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1];
             } else if (g.nrows == 4) {
                 float acc[4];
-                dot_rows_smemx<4>(sp, pitch, g.klen, lane, s.vec, acc);
+                dot_rows_smemx<4>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2]; y[3] = acc[3];
             } else if (g.nrows == 3) {
                 float acc[3];
-                dot_rows_smemx<3>(sp, pitch, g.klen, lane, s.vec, acc);
+                dot_rows_smemx<3>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2];
             } else {
                 float acc[1];
-                dot_rows_smemx<1>(sp, pitch, g.klen, lane, s.vec, acc);
+                dot_rows_smemx<1>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
                 y[0] = acc[0];
             }
             __syncwarp();
@@ -959,7 +982,19 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
                 y[2] = warp_sum(y[2]);
                 y[3] = warp_sum(y[3]);
             }
-            if (ep == EP_SWIGLU) {
+            if (pl.npieces > 1) {
+                if (lane == 0 && unit_combine(s, pl, g, r.u0, y)) {
+                    if (ep == EP_SWIGLU) {
+                        emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
+                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
+                    } else {
+#pragma unroll
+                        for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
+                            if ((uint32_t)rr < g.nrows)
+                                emit_value(out, g.row + rr, (ep == EP_RESIDUAL ? ld_tw(out.res + g.row + rr).v : 0.f) + y[rr] * xscale);
+                    }
+                }
+            } else if (ep == EP_SWIGLU) {
                 if (lane == 0) emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
                 if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
             } else if (lane < g.nrows) {
@@ -1003,27 +1038,7 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) rs[rr] = __shfl_sync(0xffffffffu, res, rr);
             if (lane == 0) {
                 bool emit = true;
-                if (pl.npieces > 1) {
-                    // partial sums of the unit's pieces meet in shared memory; the last piece to arrive adds them in
-                    // piece order and emits the rows
-                    const uint32_t us = (g.unit - r.u0) % UNIT_SLOTS;
-                    volatile float* part = s.unit_part + us * (MAX_PIECES * MAX_RPC_SPLIT);
-#pragma unroll
-                    for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) part[g.piece * MAX_RPC_SPLIT + rr] = y[rr];
-                    __threadfence_block();
-                    const int old = atomicAdd(&s.unit_cnt[us], 1);
-                    emit = (old == (int)pl.npieces - 1);
-                    if (emit) {
-                        __threadfence_block();
-                        s.unit_cnt[us] = 0;
-#pragma unroll
-                        for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = 0.f;
-                        for (uint32_t j = 0; j < pl.npieces; ++j) {
-#pragma unroll
-                            for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] += part[j * MAX_RPC_SPLIT + rr];
-                        }
-                    }
-                }
+                if (pl.npieces > 1) emit = unit_combine(s, pl, g, r.u0, y);
                 if (emit) {
                     if (ep == EP_SWIGLU) {
                         emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
