@@ -11,6 +11,12 @@
 //
 // Precision: q and the probabilities are each split into two bf16 numbers (x = hi + lo to ~2^-17), K and V are
 // bf16 values by definition, all accumulation is fp32: the result matches an fp32 CUDA-core loop to ~1e-5.
+//
+// PACK (G <= 4): the eight columns of an MMA hold the hi halves of the (up to four) heads in columns 0..3 and their lo
+// halves in columns 4..7, so one MMA does the work of two.  The two partial scores of a head then sit in lanes
+// t and t ^ 2 of a quad and are added with one shuffle; the hi and lo parts of O^T are accumulated in separate
+// columns and added once, when the unit's chunks are done.  (mma.sync is slow on this part -- about 70 cycles per
+// instruction from a single warp -- so the instruction count is what the loop costs.)
 #pragma once
 
 // Included by kl_device.cuh once its PTX helpers, ex2() and rescale() are defined.
@@ -55,14 +61,16 @@ struct AttnTcState {
     static constexpr int NKB = HD / 16;  // k blocks of the score product
     static constexpr int NMT = HD / 16;  // m tiles (16 value columns each) of the value product
     uint32_t qh[NKB][2], ql[NKB][2];     // B fragments of Q for head lane/4 (zero beyond G), hi and lo bf16 halves
+                                         // (PACK: qh holds column lane/4 of the packed operand, ql is unused)
     float o[NMT][4];                     // O^T accumulators: value columns mt*16 + lane/4 (+8), heads 2*(lane%4), +1
+                                         // (PACK: columns 2*(lane%4), +1 of the packed result)
     float m[2], l[2];                    // running maximum (base-2 scores) and this lane's part of the row sums, for
-                                         // heads 2*(lane%4) and 2*(lane%4)+1
+                                         // heads 2*(lane%4) and 2*(lane%4)+1 (PACK: heads 2*(lane%2), +1)
 };
 
 // One tile of 16 positions starting at row `row0` of the box set at (kbase, vbase); rows j with lo <= j < hi hold
 // valid positions, every other row is ignored whatever it contains.
-template <int HD>
+template <int HD, bool PACK>
 __device__ __forceinline__ void attn_tc_tile(AttnTcState<HD>& st, uint32_t kbase, uint32_t vbase, uint32_t box_bytes,
                                              uint32_t row0, uint32_t lo, uint32_t hi, uint32_t lane) {
     constexpr int NKB = HD / 16, NMT = HD / 16;
@@ -77,17 +85,23 @@ __device__ __forceinline__ void attn_tc_tile(AttnTcState<HD>& st, uint32_t kbase
             ldmatrix_x4(a, kbase + swz_off(box_bytes, r, 2u * kb + (mi >> 1)));
             if (kb & 1) {
                 mma_16816(s1, a, st.qh[kb][0], st.qh[kb][1]);
-                mma_16816(s1, a, st.ql[kb][0], st.ql[kb][1]);
+                if (!PACK) mma_16816(s1, a, st.ql[kb][0], st.ql[kb][1]);
             } else {
                 mma_16816(s0, a, st.qh[kb][0], st.qh[kb][1]);
-                mma_16816(s0, a, st.ql[kb][0], st.ql[kb][1]);
+                if (!PACK) mma_16816(s0, a, st.ql[kb][0], st.ql[kb][1]);
             }
         }
     }
     // this lane holds the scores of positions row0 + g and row0 + g + 8 for heads 2t and 2t + 1
     const uint32_t j0 = row0 + g;
     const bool v0 = j0 >= lo && j0 < hi, v1 = j0 + 8 >= lo && j0 + 8 < hi;
-    const float sa0 = s0[0] + s1[0], sa1 = s0[1] + s1[1], sb0 = s0[2] + s1[2], sb1 = s0[3] + s1[3];
+    float sa0 = s0[0] + s1[0], sa1 = s0[1] + s1[1], sb0 = s0[2] + s1[2], sb1 = s0[3] + s1[3];
+    if (PACK) {   // hi and lo partial scores of a head sit in lanes t and t ^ 2
+        sa0 += __shfl_xor_sync(0xffffffffu, sa0, 2);
+        sa1 += __shfl_xor_sync(0xffffffffu, sa1, 2);
+        sb0 += __shfl_xor_sync(0xffffffffu, sb0, 2);
+        sb1 += __shfl_xor_sync(0xffffffffu, sb1, 2);
+    }
     float mx0 = fmaxf(v0 ? sa0 : -INFINITY, v1 ? sb0 : -INFINITY);
     float mx1 = fmaxf(v0 ? sa1 : -INFINITY, v1 ? sb1 : -INFINITY);
 #pragma unroll
@@ -114,8 +128,17 @@ __device__ __forceinline__ void attn_tc_tile(AttnTcState<HD>& st, uint32_t kbase
     // transposed into the B-operand layout (rows = two positions, column = head)
     const uint32_t ph0 = pack_bf16(p00, p01), ph1 = pack_bf16(p10, p11);
     const uint32_t pl0 = pack_bf16(p00 - bf_lo(ph0), p01 - bf_hi(ph0)), pl1 = pack_bf16(p10 - bf_lo(ph1), p11 - bf_hi(ph1));
-    const uint32_t bh0 = movmatrix_trans(ph0), bh1 = movmatrix_trans(ph1);
-    const uint32_t bl0 = movmatrix_trans(pl0), bl1 = movmatrix_trans(pl1);
+    uint32_t bh0, bh1, bl0 = 0u, bl1 = 0u;
+    if (PACK) {   // columns 0..3 (lanes t < 2) carry the hi halves, columns 4..7 the lo halves
+        const bool lo_cols = (lane & 2u) != 0u;
+        bh0 = movmatrix_trans(lo_cols ? pl0 : ph0);
+        bh1 = movmatrix_trans(lo_cols ? pl1 : ph1);
+    } else {
+        bh0 = movmatrix_trans(ph0);
+        bh1 = movmatrix_trans(ph1);
+        bl0 = movmatrix_trans(pl0);
+        bl1 = movmatrix_trans(pl1);
+    }
     // V rows of ignored positions may hold anything (even NaN payloads): clear them, 0 * NaN would poison O.
     // The A fragment of V^T holds positions row0 + 2t, +1 (registers 0, 1) and row0 + 8 + 2t, +1 (registers 2, 3).
     const uint32_t t = lane & 3u;
@@ -136,7 +159,7 @@ __device__ __forceinline__ void attn_tc_tile(AttnTcState<HD>& st, uint32_t kbase
                 a[3] &= mhi;
             }
             mma_16816(st.o[mt], a, bh0, bh1);
-            mma_16816(st.o[mt], a, bl0, bl1);
+            if (!PACK) mma_16816(st.o[mt], a, bl0, bl1);
         }
     }
 }

@@ -1194,7 +1194,7 @@ __device__ __forceinline__ void attn_batch(AttnAcc<G>& st, const float (&q)[G][8
 }
 
 // Ring chunks of the unit through the tensor-core loop; leaves this warp's partial result in comb[first].
-template <int HD>
+template <int HD, bool PACK>
 __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, const AttnUnit& u, uint32_t cta,
                                                uint32_t warp, uint32_t lane, uint32_t first, const RingCursor& rc,
                                                WarpRing& wr, const float* q_s, float* comb,
@@ -1207,12 +1207,14 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const uint32_t k = kb * 16 + hf * 8 + 2 * t;
+            const uint32_t head = PACK ? (g & 3u) : g;   // PACK: column g = hi (g < 4) or lo (g >= 4) half of head g % 4
             float2 xx = make_float2(0.f, 0.f);
-            if (g < G) xx = *reinterpret_cast<const float2*>(q_s + g * HD + k);   // k is even: 8-byte aligned
+            if (head < G) xx = *reinterpret_cast<const float2*>(q_s + head * HD + k);   // k is even: 8-byte aligned
             const float x0 = xx.x, x1 = xx.y;
             const uint32_t hi = pack_bf16(x0, x1);
-            st.qh[kb][hf] = hi;
-            st.ql[kb][hf] = pack_bf16(x0 - bf_lo(hi), x1 - bf_hi(hi));
+            const uint32_t lo = pack_bf16(x0 - bf_lo(hi), x1 - bf_hi(hi));
+            st.qh[kb][hf] = (PACK && g >= 4u) ? lo : hi;
+            st.ql[kb][hf] = lo;
         }
     }
 #pragma unroll
@@ -1230,14 +1232,14 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
         const uint32_t kbase = smem_u32(s.ring) + slot * SLOT_BYTES;
         const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
         for (uint32_t row0 = 0; row0 < pb; row0 += 16)
-            if (row0 + 16 > w.lo && row0 < w.hi) attn_tc_tile<HD>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, row0, w.lo, w.hi, lane);
+            if (row0 + 16 > w.lo && row0 < w.hi) attn_tc_tile<HD, PACK>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, row0, w.lo, w.hi, lane);
         __syncwarp();
         if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
         ring_release(p, s, wr, warp, lane);
         if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
     }
     if (u.has_new && first == 0)  // the position written by this step sits in row 0 of the staging tile
-        attn_tc_tile<HD>(st, smem_u32(stage_k), smem_u32(stage_v), 128u, 0u, 0u, 1u, lane);
+        attn_tc_tile<HD, PACK>(st, smem_u32(stage_k), smem_u32(stage_v), 128u, 0u, 0u, 1u, lane);
 
     // row sums: add the parts held by the lanes that share the heads (same lane % 4)
     float l0 = st.l[0], l1 = st.l[1];
@@ -1246,10 +1248,16 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
         l0 += __shfl_xor_sync(0xffffffffu, l0, o);
         l1 += __shfl_xor_sync(0xffffffffu, l1, o);
     }
+    if (PACK) {   // columns 0..3 hold the hi parts of O^T, columns 4..7 the lo parts: lanes t and t ^ 2 of a quad
+#pragma unroll
+        for (int n = 0; n < NMT; ++n)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) st.o[n][j] += __shfl_xor_sync(0xffffffffu, st.o[n][j], 2);
+    }
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
         const uint32_t h = 2 * t + hh;
-        if (h < G) {
+        if (h < G && (!PACK || t < 2u)) {
             float* dst = comb + ((size_t)first * G + h) * (HD + 2);
 #pragma unroll
             for (int n = 0; n < NMT; ++n) {
@@ -1433,10 +1441,13 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
 
     const uint32_t first = rc.first_chunk(warp, p.nslots);
     if constexpr (GT == 0) {
-        if (hd == 128)
-            attn_chunks_tc<128>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
-        else
-            attn_chunks_tc<64>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
+        if (hd == 128) {
+            if (G <= 4) attn_chunks_tc<128, true>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
+            else attn_chunks_tc<128, false>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
+        } else {
+            if (G <= 4) attn_chunks_tc<64, true>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
+            else attn_chunks_tc<64, false>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
+        }
     } else {
         constexpr int G_ = GT > 0 ? GT : 1;
         const uint32_t lpp = hd >> 3;           // lanes per position
