@@ -185,6 +185,14 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
+/* Classifier of a batched step (batch > 1).  on = 1 (default when available): one pass over the classifier matrix
+ * for the whole batch on the tcgen05 tensor cores (M = 128 vocabulary rows x N = 64 = 32 sequences x (hi, lo bf16
+ * halves of the normalised hidden state), fp32 accumulators in TMEM) -- at batch 32 this projection is a dense
+ * contraction (Table 1 of the paper).  on = 0: the batch-1 GEMV kernel, sequence after sequence.  Available when
+ * max_batch is 2..32, hidden is a multiple of 64 and the driver exports cuTensorMapEncodeTiled; otherwise
+ * KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
+kl_status kl_set_batched_classifier(kl_handle* h, int on);
+
 /* Limit, in nanoseconds, of every device-side wait (tagged word, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
 

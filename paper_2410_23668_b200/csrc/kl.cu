@@ -10,6 +10,7 @@
 // mode, across layer boundaries: while the CTAs poll the tagged words that replace a kernel boundary, HBM keeps
 // streaming the next stage's (next layer's) chunks until the ring is full.
 #include "kl_device.cuh"
+#include "kl_batched_classifier.cuh"
 
 #include <math.h>
 #include <stdio.h>
@@ -271,6 +272,10 @@ struct kl_handle {
     float* stage_logits;
     float* argmax_val;
     float* hidden_all;     // [max_batch][H] hidden states of the sequences of the latest batched step
+    __nv_bfloat16* bc_x;   // [64][H] normalised inputs of the batched classifier (hi and lo halves)
+    BcParams bc;           // tensor maps and sizes of the batched classifier
+    int bc_ok;             // 1: the tensor-core classifier for batches is available
+    int use_bc;            // 1 (default): use it for batches; 0: classify sequence by sequence
     uint32_t last_batch;
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
@@ -297,7 +302,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbcx, scratch_bytes;
     uint32_t cps;
 };
 
@@ -354,6 +359,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.slogits = s;   s += align_up(B * V * 4);
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
     y.shid = s;      s += align_up(B * H * 4);
+    y.sbcx = s;      s += align_up((size_t)64 * H * 2 + 1024);
     y.scratch_bytes = s;
     return y;
 }
@@ -487,6 +493,22 @@ static int query_sms(int* dev_out) {
     return sms;
 }
 
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// A row-major bf16 matrix [rows, cols] as a 2-D tensor with boxes of [box_rows] x [64 columns] and the 128-byte swizzle.
+static bool encode_bf16_2d(void* encode_fn, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+    if (!encode_fn || ((uintptr_t)base & 15u) || (cols * 2) % 16) return false;
+    const cuuint64_t gdim[2] = {cols, rows};
+    const cuuint64_t gstride[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return ((encode_tiled_fn)encode_fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 kl_status kl_workspace_bytes(const kl_model_desc* desc, size_t* weight_bytes, size_t* scratch_bytes) {
     if (!desc || !weight_bytes || !scratch_bytes) return KL_ERR_INVALID_ARG;
     int sms = query_sms(nullptr);
@@ -598,6 +620,19 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->argmax_val = (float*)(sc + y.samax);
     h->hidden_all = (float*)(sc + y.shid);
     h->last_batch = 1;
+    // tensor-core classifier for batches: W_lm must be plain row-major (whole-row plan) and H a multiple of 64
+    h->bc_x = (__nv_bfloat16*)(((uintptr_t)(sc + y.sbcx) + 1023u) & ~(uintptr_t)1023u);
+    h->bc_ok = 0;
+    h->use_bc = 1;
+    if (p.plan[PL_LM].npieces == 1 && p.H % BC_TILE_K == 0 && d.max_batch > 1 && d.max_batch <= 32 &&
+        encode_bf16_2d(h->encode_tiled, &h->bc.map_w, p.wlm, p.V, p.H, BC_TILE_M) &&
+        encode_bf16_2d(h->encode_tiled, &h->bc.map_x, h->bc_x, 64, p.H, BC_TILE_N) &&
+        cudaFuncSetAttribute(kl_bc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BC_SMEM_BYTES) == cudaSuccess) {
+        h->bc.V = p.V;
+        h->bc.H = p.H;
+        h->bc.status = p.status;
+        h->bc_ok = 1;
+    }
     h->argmax_idx = (uint32_t*)(h->argmax_val + (size_t)d.max_batch * ARGMAX_BLOCKS);
     h->argmax_tickets = h->argmax_idx + (size_t)d.max_batch * ARGMAX_BLOCKS;
 
@@ -650,10 +685,6 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
 
 // The KV cache as a 2-D bf16 tensor [n_layers*2*batch*n_kv_heads*max_ctx rows, head_dim columns]; boxes of
 // [positions per chunk] x [64 columns] with the 128-byte swizzle.  Encoded per call because the cache is the caller's.
-typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch) {
     if (!h->encode_tiled) return KL_ERR_CUDA;
     if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
@@ -753,16 +784,33 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
                 }
         }
         if (ev && b == 0 && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
-        Params pc = p;
-        pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
-        void* cargs[] = {&pc};
-        if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
+        const bool batched_classifier = batch > 1 && h->bc_ok && h->use_bc;
+        if (!batched_classifier) {
+            Params pc = p;
+            pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
+            void* cargs[] = {&pc};
+            if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
+        }
         if (ev && b == 0 && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
         if (batch > 1) {
             // keep this sequence's hidden state (the value half of every tagged word) for kl_read_hidden
             if (cudaMemcpy2DAsync(h->hidden_all + (size_t)b * p.H, 4, p.xa, 8, 4, p.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
                 return KL_ERR_CUDA;
         }
+    }
+    if (batch > 1 && h->bc_ok && h->use_bc) {
+        // one pass over W_lm for the whole batch, on the tensor cores
+        kl_bc_prepare_kernel<<<32, 256, 0, st>>>(h->hidden_all, p.gf, h->bc_x, p.H, batch, p.eps);
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+        BcParams bp = h->bc;
+        bp.logits = logits_d;
+        bp.B = batch;
+        bp.wait_ns = p.wait_ns;
+        const uint32_t ntiles = (p.V + BC_TILE_M - 1) / BC_TILE_M;
+        const uint32_t grid = ntiles < (uint32_t)h->num_sms ? ntiles : (uint32_t)h->num_sms;
+        kl_bc_kernel<<<grid, BC_THREADS, BC_SMEM_BYTES, st>>>(bp);
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+        h->launches += 2;
     }
     return KL_OK;
 }
@@ -920,6 +968,13 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
     if (on && !h->encode_tiled) return KL_ERR_CUDA;
     h->use_tc_attention = on ? 1 : 0;
+    return KL_OK;
+}
+
+kl_status kl_set_batched_classifier(kl_handle* h, int on) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    if (on && !h->bc_ok) return KL_ERR_UNSUPPORTED_SHAPE;
+    h->use_bc = on ? 1 : 0;
     return KL_OK;
 }
 
