@@ -41,6 +41,8 @@ WORKLOADS = {
     # batches run sequence after sequence through the batch-1 kernels (weights streamed once per sequence): functional,
     # not the batched roofline
     "llama31_8b_b32_ctx4096": (gen.LLAMA31_8B, 32, 4096, 4),
+    # one layer, short context, 32 sequences: 2 GB on the device, for profiler captures of the batched classifier
+    "llama31_8b_1layer_b32_ctx64": (gen.ModelShape(1, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 32, 64, 4),
 }
 DEFAULT_WORKLOAD = "llama31_8b_b1_ctx4096"
 NOMINAL_HBM_GBS = 8000.0
