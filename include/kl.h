@@ -185,13 +185,16 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
-/* Classifier of a batched step (batch > 1).  on = 1 (default when available): one pass over the classifier matrix
- * for the whole batch on the tcgen05 tensor cores (M = 128 vocabulary rows x N = 64 = 32 sequences x (hi, lo bf16
- * halves of the normalised hidden state), fp32 accumulators in TMEM) -- at batch 32 this projection is a dense
- * contraction (Table 1 of the paper).  on = 0: the batch-1 GEMV kernel, sequence after sequence.  Available when
- * max_batch is 2..32, hidden is a multiple of 64 and the driver exports cuTensorMapEncodeTiled; otherwise
- * KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
-kl_status kl_set_batched_classifier(kl_handle* h, int on);
+/* Decode steps of a batch (batch > 1).  on = 1 (default when available): the tensor-core path -- every projection
+ * of the step (QKV, O, gate/up, down, classifier) is one dense contraction for the whole batch on the tcgen05 tensor
+ * cores (M = 128 weight rows x N = 64 = 32 sequences x (hi, lo bf16 halves of the fp32 input), fp32 accumulators in
+ * TMEM), so the weights are streamed once per step instead of once per sequence -- at batch 32 the projections are
+ * dense contractions (Table 1 of the paper); attention runs as split-K units over (sequence, kv head, split).  The
+ * step is a sequence of launches, one per operator group (Section 3.1's per-operator calls); kl_set_mode does not
+ * apply to it.  on = 0: the batch-1 kernels in the mode of kl_set_mode, sequence after sequence.  Available when
+ * max_batch is 2..32, head_dim is 64 or 128, hidden / q width / ffn are multiples of 8, every projection has at
+ * least 128 rows and the driver exports cuTensorMapEncodeTiled; otherwise KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
+kl_status kl_set_batched_path(kl_handle* h, int on);
 
 /* Limit, in nanoseconds, of every device-side wait (tagged word, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);

@@ -10,7 +10,7 @@
 // mode, across layer boundaries: while the CTAs poll the tagged words that replace a kernel boundary, HBM keeps
 // streaming the next stage's (next layer's) chunks until the ring is full.
 #include "kl_device.cuh"
-#include "kl_batched_classifier.cuh"
+#include "kl_batched.cuh"
 
 #include <math.h>
 #include <stdio.h>
@@ -272,10 +272,20 @@ struct kl_handle {
     float* stage_logits;
     float* argmax_val;
     float* hidden_all;     // [max_batch][H] hidden states of the sequences of the latest batched step
-    __nv_bfloat16* bc_x;   // [64][H] normalised inputs of the batched classifier (hi and lo halves)
-    BcParams bc;           // tensor maps and sizes of the batched classifier
-    int bc_ok;             // 1: the tensor-core classifier for batches is available
-    int use_bc;            // 1 (default): use it for batches; 0: classify sequence by sequence
+    // batched (tensor-core) path
+    int bt_ok;             // 1: available for this shape
+    int use_bt;            // 1 (default): batches take it; 0: sequence after sequence on the batch-1 kernels
+    float* bx;             // [32][H] hidden states of the batch (== hidden_all)
+    __nv_bfloat16* bxop;   // [64][Kmax] operand of the next projection (hi and lo halves)
+    float* bpart;          // partial sums of the projection in flight
+    float* bq;             // [32][QD] rotated queries
+    float* bao;            // attention partial outputs
+    float* baml;           // attention partial (max, sum) pairs
+    CUtensorMap bmap_x[3];   // operand buffer seen as [64][H], [64][QD], [64][F]
+    CUtensorMap bmap_w[5];   // QKV, O, gate/up, down, classifier
+    CUtensorMap bmap_wl[5];  // last column piece of the matrices stored in chunk order
+    uint32_t bsplit[5];      // K splits of the five projections
+    uint32_t battn_splits;   // attention splits per (sequence, kv head) at the largest batch
     uint32_t last_batch;
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
@@ -302,7 +312,8 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbcx, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbpart, sbq, sbao, sbaml, scratch_bytes;
+    uint32_t bsplit[5], battn_splits;
     uint32_t cps;
 };
 
@@ -317,6 +328,47 @@ bool shape_supported(const kl_model_desc& d, int num_sms) {
     if ((uint64_t)d.n_kv_heads > (uint64_t)num_sms) return false;
     if (!(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f)) return false;
     return true;
+}
+
+static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
+
+// K splits of a batched projection: the (row tile, split) items are dealt round-robin to the CTAs; pick the count that
+// wastes the least of the last round, with at least four K blocks per split and at most eight splits.
+static uint32_t pick_split(uint32_t tiles, uint32_t nkb, uint32_t P) {
+    uint32_t best = 1;
+    double best_eff = 0.0;
+    for (uint32_t sp = 1; sp <= 8 && nkb / sp >= 4; ++sp) {
+        const uint32_t items = tiles * sp;
+        const double eff = (double)items / (double)(((items + P - 1) / P) * P);
+        if (eff > best_eff + 1e-9) {
+            best_eff = eff;
+            best = sp;
+        }
+    }
+    return best;
+}
+
+// Dynamic shared memory of kl_b_attn_kernel: alignment slack, the warps' ring slots, barriers, the queries, the warps'
+// partial results, the rescale table and the abort flag.
+static size_t batched_attn_smem(uint32_t G, uint32_t hd) {
+    return 1024 + (size_t)BA_WARPS * BA_SLOTS * SLOT_BYTES + 128 + (size_t)G * hd * 4 + (size_t)BA_WARPS * G * (hd + 2) * 4 +
+           (size_t)(BA_WARPS * MAX_G + MAX_G) * 4 + 16;
+}
+
+// Attention splits per (sequence, kv head) for a batch: the count (at most max_splits) whose units fill whole rounds
+// of one CTA per SM best, the smallest such count on a tie.
+static uint32_t pick_attn_splits(uint32_t batch, uint32_t nkv, uint32_t P, uint32_t max_splits) {
+    uint32_t best = 1;
+    double best_eff = 0.0;
+    for (uint32_t sa = 1; sa <= max_splits; ++sa) {
+        const uint32_t units = batch * nkv * sa;
+        const double eff = (double)units / (double)(((units + P - 1) / P) * P);
+        if (eff > best_eff + 0.02) {
+            best_eff = eff;
+            best = sa;
+        }
+    }
+    return best;
 }
 
 Layout make_layout(const kl_model_desc& d, int num_sms) {
@@ -358,8 +410,27 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.spos = s;      s += align_up(B * 4);
     y.slogits = s;   s += align_up(B * V * 4);
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
-    y.shid = s;      s += align_up(B * H * 4);
-    y.sbcx = s;      s += align_up((size_t)64 * H * 2 + 1024);
+    y.shid = s;      s += align_up((B > 1 ? 32 : B) * H * 4);
+    // batched path (max_batch > 1): operand, partial sums, queries, attention partials
+    {
+        const size_t QR = QD + 2 * KVD;
+        const uint32_t tiles[5] = {(uint32_t)ceil_div(QR, 128), (uint32_t)ceil_div(H, 128), (uint32_t)ceil_div(2 * F, 128),
+                                   (uint32_t)ceil_div(H, 128), (uint32_t)ceil_div(V, 128)};
+        const size_t rows[5] = {QR, H, 2 * F, H, V}, ks[5] = {H, QD, H, F, H};
+        size_t part_max = 0;
+        for (int i = 0; i < 5; ++i) {
+            y.bsplit[i] = i == 4 ? 1u : pick_split(tiles[i], (uint32_t)ceil_div(ks[i], 64), (uint32_t)num_sms);
+            if (i < 4 && y.bsplit[i] * rows[i] > part_max) part_max = y.bsplit[i] * rows[i];
+        }
+        y.battn_splits = 16;
+        const size_t kmax = H > QD ? (H > F ? H : F) : (QD > F ? QD : F);
+        const bool on = B > 1;
+        y.sbxop = s;  s += on ? align_up(64 * kmax * 2 + 1024) : 0;
+        y.sbpart = s; s += on ? align_up(part_max * 32 * 4) : 0;
+        y.sbq = s;    s += on ? align_up(32 * QD * 4) : 0;
+        y.sbao = s;   s += on ? align_up(B * d.n_kv_heads * y.battn_splits * G * d.head_dim * 4) : 0;
+        y.sbaml = s;  s += on ? align_up(B * d.n_kv_heads * y.battn_splits * G * 2 * 4) : 0;
+    }
     y.scratch_bytes = s;
     return y;
 }
@@ -509,6 +580,48 @@ static bool encode_bf16_2d(void* encode_fn, CUtensorMap* map, const void* base, 
                                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A bf16 tensor of rank `rank` (dimensions innermost first, byte strides of dimensions 1 .. rank-1), 128-byte swizzle,
+// zeros outside the tensor.
+static bool encode_bf16_nd(void* encode_fn, CUtensorMap* map, const void* base, uint32_t rank, const cuuint64_t* dims,
+                           const cuuint64_t* strides, const cuuint32_t* box) {
+    if (!encode_fn || ((uintptr_t)base & 15u)) return false;
+    for (uint32_t i = 0; i + 1 < rank; ++i)
+        if (strides[i] % 16) return false;
+    const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    return ((encode_tiled_fn)encode_fn)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
+                                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor maps of one weight matrix (R rows, plan pl, `layers` copies layer_stride elements apart) for the batched
+// projections: tiles of 128 rows x 64 columns.  A matrix stored whole-row is a rank-3 tensor (column, row, layer).  One
+// stored in chunk order (units of rpc rows, each cut into column pieces of kp) is a rank-5 tensor (column in piece, row
+// in unit, piece, unit, layer) for the full pieces and a rank-4 one for the last, shorter piece.
+static bool encode_weight_maps(void* fn, CUtensorMap* map, CUtensorMap* map_last, const __nv_bfloat16* mat, const GemvPlan& pl,
+                               uint32_t R, uint32_t layers, uint64_t layer_stride) {
+    const uint64_t K = pl.K;
+    if (R < (uint32_t)BG_TILE_M || K < (uint64_t)BG_TILE_K || K % 8) return false;
+    const uint64_t lbytes = layers > 1 ? layer_stride * 2 : (((uint64_t)R * K * 2 + 15) & ~15ull);
+    if (pl.npieces == 1) {
+        const cuuint64_t dims[3] = {K, R, layers};
+        const cuuint64_t strides[2] = {K * 2, lbytes};
+        const cuuint32_t box[3] = {(cuuint32_t)BG_TILE_K, (cuuint32_t)BG_TILE_M, 1};
+        return encode_bf16_nd(fn, map, mat, 3, dims, strides, box);
+    }
+    const uint64_t rpc = pl.rpc, kp = pl.kp, np = pl.npieces, last = K - (np - 1) * kp;
+    if (R % rpc || BG_TILE_M % rpc || kp % 8 || last % 8 || kp < (uint64_t)BG_TILE_K || last == 0) return false;
+    {
+        const cuuint64_t dims[5] = {kp, rpc, np - 1, R / rpc, layers};
+        const cuuint64_t strides[4] = {kp * 2, rpc * kp * 2, rpc * K * 2, lbytes};
+        const cuuint32_t box[5] = {(cuuint32_t)BG_TILE_K, (cuuint32_t)rpc, 1, (cuuint32_t)(BG_TILE_M / rpc), 1};
+        if (!encode_bf16_nd(fn, map, mat, 5, dims, strides, box)) return false;
+    }
+    const cuuint64_t dims[4] = {last, rpc, R / rpc, layers};
+    const cuuint64_t strides[3] = {last * 2, rpc * K * 2, lbytes};
+    const cuuint32_t box[4] = {(cuuint32_t)BG_TILE_K, (cuuint32_t)rpc, (cuuint32_t)(BG_TILE_M / rpc), 1};
+    return encode_bf16_nd(fn, map_last, mat + rpc * (np - 1) * kp, 4, dims, strides, box);
+}
+
 kl_status kl_workspace_bytes(const kl_model_desc* desc, size_t* weight_bytes, size_t* scratch_bytes) {
     if (!desc || !weight_bytes || !scratch_bytes) return KL_ERR_INVALID_ARG;
     int sms = query_sms(nullptr);
@@ -620,18 +733,33 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->argmax_val = (float*)(sc + y.samax);
     h->hidden_all = (float*)(sc + y.shid);
     h->last_batch = 1;
-    // tensor-core classifier for batches: W_lm must be plain row-major (whole-row plan) and H a multiple of 64
-    h->bc_x = (__nv_bfloat16*)(((uintptr_t)(sc + y.sbcx) + 1023u) & ~(uintptr_t)1023u);
-    h->bc_ok = 0;
-    h->use_bc = 1;
-    if (p.plan[PL_LM].npieces == 1 && p.H % BC_TILE_K == 0 && d.max_batch > 1 && d.max_batch <= 32 &&
-        encode_bf16_2d(h->encode_tiled, &h->bc.map_w, p.wlm, p.V, p.H, BC_TILE_M) &&
-        encode_bf16_2d(h->encode_tiled, &h->bc.map_x, h->bc_x, 64, p.H, BC_TILE_N) &&
-        cudaFuncSetAttribute(kl_bc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BC_SMEM_BYTES) == cudaSuccess) {
-        h->bc.V = p.V;
-        h->bc.H = p.H;
-        h->bc.status = p.status;
-        h->bc_ok = 1;
+    // tensor-core path for batches of up to 32 sequences
+    h->bx = h->hidden_all;
+    h->bxop = (__nv_bfloat16*)(((uintptr_t)(sc + y.sbxop) + 1023u) & ~(uintptr_t)1023u);
+    h->bpart = (float*)(sc + y.sbpart);
+    h->bq = (float*)(sc + y.sbq);
+    h->bao = (float*)(sc + y.sbao);
+    h->baml = (float*)(sc + y.sbaml);
+    for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
+    h->battn_splits = y.battn_splits;
+    h->use_bt = 1;
+    h->bt_ok = 0;
+    if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
+        p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
+        const uint32_t QR = p.QD + 2 * p.KVD;
+        const size_t ba_smem = batched_attn_smem(p.G, p.hd);
+        bool ok = encode_weight_maps(h->encode_tiled, &h->bmap_w[0], &h->bmap_wl[0], p.wqkv, p.plan[PL_QKV], QR, p.L, p.layer_stride) &&
+                  encode_weight_maps(h->encode_tiled, &h->bmap_w[1], &h->bmap_wl[1], p.wo, p.plan[PL_O], p.H, p.L, p.layer_stride) &&
+                  encode_weight_maps(h->encode_tiled, &h->bmap_w[2], &h->bmap_wl[2], p.wgu, p.plan[PL_GU], 2 * p.F, p.L, p.layer_stride) &&
+                  encode_weight_maps(h->encode_tiled, &h->bmap_w[3], &h->bmap_wl[3], p.wd, p.plan[PL_D], p.H, p.L, p.layer_stride) &&
+                  encode_weight_maps(h->encode_tiled, &h->bmap_w[4], &h->bmap_wl[4], p.wlm, p.plan[PL_LM], p.V, 1, 0) &&
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[0], h->bxop, 64, p.H, BG_TILE_N) &&
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[1], h->bxop, 64, p.QD, BG_TILE_N) &&
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[2], h->bxop, 64, p.F, BG_TILE_N);
+        ok = ok && cudaFuncSetAttribute(kl_bgemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BG_SMEM_BYTES) == cudaSuccess &&
+             cudaFuncSetAttribute(kl_b_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ba_smem) == cudaSuccess;
+        (void)cudaGetLastError();
+        h->bt_ok = ok ? 1 : 0;
     }
     h->argmax_idx = (uint32_t*)(h->argmax_val + (size_t)d.max_batch * ARGMAX_BLOCKS);
     h->argmax_tickets = h->argmax_idx + (size_t)d.max_batch * ARGMAX_BLOCKS;
@@ -731,12 +859,124 @@ static kl_status launch_persistent(kl_handle* h, const void* func, void** args, 
     return KL_OK;
 }
 
+// One projection of the batched path: out[s][b][r] = partial sums over K split s of W[idx](layer) . operand.
+static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out, uint32_t batch, cudaStream_t st) {
+    const Params& p = h->prm;
+    static const int plan_of[5] = {PL_QKV, PL_O, PL_GU, PL_D, PL_LM};
+    static const int xmap_of[5] = {0, 1, 0, 2, 0};
+    const uint32_t rows[5] = {p.QD + 2 * p.KVD, p.H, 2 * p.F, p.H, p.V};
+    const GemvPlan& pl = p.plan[plan_of[idx]];
+    BgemmParams g;
+    g.map_w = h->bmap_w[idx];
+    g.map_wl = h->bmap_wl[idx];
+    g.map_x = h->bmap_x[xmap_of[idx]];
+    g.out = out;
+    g.R = rows[idx];
+    g.K = pl.K;
+    g.B = batch;
+    g.S = h->bsplit[idx];
+    g.layer = layer;
+    g.kp = pl.kp;
+    g.rpc = pl.rpc;
+    g.kb_piece = ceil_div(pl.kp, (uint32_t)BG_TILE_K);
+    if (pl.npieces == 1) {
+        g.pieces = 0;
+        g.nkb = ceil_div(pl.K, (uint32_t)BG_TILE_K);
+    } else {
+        g.pieces = pl.npieces;
+        g.nkb = (pl.npieces - 1) * g.kb_piece + ceil_div(pl.K - (pl.npieces - 1) * pl.kp, (uint32_t)BG_TILE_K);
+    }
+    g.status = p.status;
+    g.wait_ns = p.wait_ns;
+    const uint32_t items = ceil_div(g.R, (uint32_t)BG_TILE_M) * g.S;
+    const uint32_t grid = items < (uint32_t)h->num_sms ? items : (uint32_t)h->num_sms;
+    kl_bgemm_kernel<<<grid, BG_THREADS, BG_SMEM_BYTES, st>>>(g);
+    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+    ++h->launches;
+    return KL_OK;
+}
+
+// Decode step of a batch on the tensor-core path: one launch per operator group, every weight matrix streamed once.
+static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
+                                     float* logits_d, uint32_t batch, cudaStream_t st) {
+    const Params& p = h->prm;
+    BAttnParams a;
+    const kl_status trc = encode_kv_map(h, &a.kv_map, kv_cache_d, batch);
+    if (trc != KL_OK) return trc;
+    a.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
+    a.positions = positions_d;
+    a.inv_freq = p.inv_freq;
+    a.qkv_part = h->bpart;
+    a.q = h->bq;
+    a.part_o = h->bao;
+    a.part_ml = h->baml;
+    a.xop = h->bxop;
+    a.S = h->bsplit[0];
+    a.QR = p.QD + 2 * p.KVD;
+    a.QD = p.QD; a.KVD = p.KVD; a.nq = p.nq; a.nkv = p.nkv; a.G = p.G; a.hd = p.hd;
+    a.B = batch;
+    a.max_ctx = h->desc.max_ctx;
+    a.Sa = pick_attn_splits(batch, p.nkv, (uint32_t)h->num_sms, h->battn_splits);
+    a.status = p.status;
+    a.wait_ns = p.wait_ns;
+    const size_t ba_smem = batched_attn_smem(p.G, p.hd);
+    cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
+    kl_status rc;
+#define KL_B_CHECK()                                          \
+    do {                                                      \
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA; \
+        ++h->launches;                                        \
+    } while (0)
+    kl_b_embed_kernel<<<batch, 256, 0, st>>>(tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, batch, p.status);
+    KL_B_CHECK();
+    if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+    uint32_t s_prev = 0;   // splits of the down projection whose sums are still to be added to the residual stream
+    for (uint32_t l = 0; l < p.L; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        a.layer = l;
+        // x += down projection of the previous layer; operand = RMSNorm(x; g1)
+        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, p.eps, 0, p.H, batch, h->bxop, p.status);
+        KL_B_CHECK();
+        if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st)) != KL_OK) return rc;
+        kl_b_rope_kernel<<<batch, 256, 0, st>>>(a);
+        KL_B_CHECK();
+        kl_b_attn_kernel<<<dim3(a.Sa, p.nkv, batch), BA_THREADS, ba_smem, st>>>(a);
+        KL_B_CHECK();
+        kl_b_attn_merge_kernel<<<dim3(p.nkv, 32), 256, 0, st>>>(a);
+        KL_B_CHECK();
+        if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st)) != KL_OK) return rc;
+        // x += attention output projection; operand = RMSNorm(x; g2)
+        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, p.eps, 0, p.H, batch, h->bxop,
+                                               p.status);
+        KL_B_CHECK();
+        if ((rc = launch_bgemm(h, 2, l, h->bpart, batch, st)) != KL_OK) return rc;
+        // operand = silu(gate) * up
+        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, p.eps, 1, p.F, batch,
+                                               h->bxop, p.status);
+        KL_B_CHECK();
+        if ((rc = launch_bgemm(h, 3, l, h->bpart, batch, st)) != KL_OK) return rc;
+        s_prev = h->bsplit[3];
+    }
+    if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
+    // x += last down projection (kept for kl_read_hidden); operand = RMSNorm(x; gf); logits = W_lm . operand
+    kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, p.eps, 0, p.H, batch, h->bxop, p.status);
+    KL_B_CHECK();
+    if ((rc = launch_bgemm(h, 4, 0, logits_d, batch, st)) != KL_OK) return rc;
+    if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
+#undef KL_B_CHECK
+    return KL_OK;
+}
+
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                          float* logits_d, uint32_t batch, void* stream) {
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
     cudaStream_t st = as_stream(stream);
+    if (batch > 1 && h->bt_ok && h->use_bt) {
+        h->last_batch = batch;
+        return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
+    }
     Params p = h->prm;
     p.B = batch;
     p.cps = (uint32_t)h->num_sms / p.nkv;
@@ -753,9 +993,8 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     }
     h->last_batch = batch;
     cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
-    // Sequences of a batch are independent.  The batch-1 kernels decode them one after another (the weights are
-    // streamed once per sequence); the M = batch tensor-core projections that would stream them once per step are
-    // not built.
+    // Sequences of a batch are independent: without the batched path the batch-1 kernels decode them one after
+    // another (the weights are streamed once per sequence).
     for (uint32_t b = 0; b < batch; ++b) {
         p.b0 = b;
         p.logits = logits_d + (size_t)b * p.V;
@@ -784,8 +1023,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
                 }
         }
         if (ev && b == 0 && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
-        const bool batched_classifier = batch > 1 && h->bc_ok && h->use_bc;
-        if (!batched_classifier) {
+        {
             Params pc = p;
             pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
             void* cargs[] = {&pc};
@@ -797,20 +1035,6 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
             if (cudaMemcpy2DAsync(h->hidden_all + (size_t)b * p.H, 4, p.xa, 8, 4, p.H, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
                 return KL_ERR_CUDA;
         }
-    }
-    if (batch > 1 && h->bc_ok && h->use_bc) {
-        // one pass over W_lm for the whole batch, on the tensor cores
-        kl_bc_prepare_kernel<<<32, 256, 0, st>>>(h->hidden_all, p.gf, h->bc_x, p.H, batch, p.eps);
-        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
-        BcParams bp = h->bc;
-        bp.logits = logits_d;
-        bp.B = batch;
-        bp.wait_ns = p.wait_ns;
-        const uint32_t ntiles = (p.V + BC_TILE_M - 1) / BC_TILE_M;
-        const uint32_t grid = ntiles < (uint32_t)h->num_sms ? ntiles : (uint32_t)h->num_sms;
-        kl_bc_kernel<<<grid, BC_THREADS, BC_SMEM_BYTES, st>>>(bp);
-        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
-        h->launches += 2;
     }
     return KL_OK;
 }
@@ -971,10 +1195,10 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     return KL_OK;
 }
 
-kl_status kl_set_batched_classifier(kl_handle* h, int on) {
+kl_status kl_set_batched_path(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
-    if (on && !h->bc_ok) return KL_ERR_UNSUPPORTED_SHAPE;
-    h->use_bc = on ? 1 : 0;
+    if (on && !h->bt_ok) return KL_ERR_UNSUPPORTED_SHAPE;
+    h->use_bt = on ? 1 : 0;
     return KL_OK;
 }
 

@@ -1,0 +1,632 @@
+// Decode step for a BATCH of sequences: every projection is a dense contraction [rows x K] x [K x batch] on the
+// 5th-generation tensor cores (tcgen05, accumulators in TMEM), so the weights are streamed once per step for all
+// sequences (the paper's Table 1: ~20 FLOP/B at batch 32 -- still far below the ridge, i.e. HBM-bound, which is why the
+// tiling is chosen for streaming and balance, not for tensor throughput).
+//
+// One projection = kl_bgemm_kernel:  part[s][b][r] = sum over the K blocks of split s of W[r, k] * x[b, k].
+//   * M = 128 weight rows per tile; the inputs enter as the N operand split into bf16 hi and lo halves that sit in
+//     columns 0..31 and 32..63 of ONE N = 64 operand: a single MMA per 16 columns of K yields W.x_hi and W.x_lo side by
+//     side and the epilogue adds them (fp32-accurate inputs on a bf16 tensor pipe).
+//   * Work items are (row tile, K split); 148 persistent CTAs take items round-robin.  The split count is chosen on the
+//     host so that the items balance over the SMs; the partial sums of the splits are added, in split order, by the
+//     kernel that consumes them (kl_b_finish_kernel / kl_b_rope_kernel) -- no atomics, the result is reproducible.
+//   * Per 64 columns of K one ring stage holds a [128 x 64] weight tile (16 KB) and the [64 x 64] input tile (8 KB),
+//     written by TMA with the 128-byte swizzle the MMA's shared-memory descriptors expect.  Row-major matrices are read
+//     through a 3-D tensor (column, row, layer); the down projection, which is stored in chunk order for the batch-1
+//     kernel (unit of rpc rows x column piece), through a 5-D tensor (column, row in unit, piece, unit, layer) plus a
+//     4-D one for its shorter last piece.
+//   * Roles (192 threads): warp 0 lane 0 issues the TMA loads, warp 1 owns TMEM and its lane 0 issues tcgen05.mma and
+//     the commits, warps 2..5 read the accumulators (tcgen05.ld) and store.  Two accumulator buffers overlap the
+//     epilogue of one item with the MMAs of the next.  Every mbarrier wait is bounded.
+//
+// Between the projections small kernels do the per-sequence vector work (sum of the splits, residual, RMSNorm, SwiGLU,
+// RoPE, cache append) and write the next projection's bf16 operand; attention is a split-K flash-decoding kernel over
+// (sequence, kv head, split) units with the same mma.sync tiles as the batch-1 kernel.
+#pragma once
+
+namespace kl {
+
+constexpr int BG_THREADS = 192;
+constexpr int BG_STAGES = 6;
+constexpr int BG_TILE_M = 128;
+constexpr int BG_TILE_N = 64;   // 32 sequences x (hi, lo)
+constexpr int BG_TILE_K = 64;   // bf16 columns per stage = one 128-byte swizzle row
+constexpr int BG_A_BYTES = BG_TILE_M * BG_TILE_K * 2;
+constexpr int BG_B_BYTES = BG_TILE_N * BG_TILE_K * 2;
+constexpr int BG_STAGE_BYTES = BG_A_BYTES + BG_B_BYTES;
+constexpr int BG_TMEM_COLS = 128;   // two accumulator buffers of 64 fp32 columns
+constexpr size_t BG_SMEM_BYTES = (size_t)BG_STAGES * BG_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int BG_MAX_BATCH = 32;
+
+struct BgemmParams {
+    CUtensorMap map_w;     // weights: rank 3 (column, row, layer) or, for chunk-ordered matrices, rank 5
+    CUtensorMap map_wl;    // chunk-ordered matrices: the last (shorter) column piece, rank 4 (column, row in unit, unit, layer)
+    CUtensorMap map_x;     // inputs [64 rows, K] bf16: rows 0..31 hi halves, 32..63 lo halves
+    float* out;            // [S][32][R] partial sums (S = 1: the result itself)
+    uint32_t R, K, B, S, layer;
+    uint32_t nkb;          // K blocks of 64 columns in all (a block may reach past the end of K or of a piece: TMA fills zeros)
+    uint32_t pieces;       // 0: row-major weights; otherwise the number of column pieces of the chunk order
+    uint32_t kp;           // columns per full piece
+    uint32_t kb_piece;     // K blocks per full piece = ceil(kp / 64)
+    uint32_t rpc;          // rows per unit of the chunk order
+    int32_t* status;
+    uint64_t wait_ns;
+};
+
+// ---- PTX wrappers (tcgen05 / TMEM / higher-rank TMA)
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]; M, N and the operand types are in the instruction descriptor.
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier gets one arrival when all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives lane (row) i.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_tensor_3d_g2s(uint32_t dst, const void* tmap, int32_t c0, int32_t c1, int32_t c2, uint32_t bar,
+                                                  uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ void tma_tensor_4d_g2s(uint32_t dst, const void* tmap, int32_t c0, int32_t c1, int32_t c2, int32_t c3,
+                                                  uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(pol)
+        : "memory");
+}
+__device__ __forceinline__ void tma_tensor_5d_g2s(uint32_t dst, const void* tmap, int32_t c0, int32_t c1, int32_t c2, int32_t c3,
+                                                  int32_t c4, uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar), "l"(pol)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the 128-byte swizzle
+// (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B; the tile starts on a 1024-byte boundary): start address / 16 in
+// bits 0..13, leading byte offset (unused for this layout) 1 in bits 16..29, stride between groups of eight rows
+// 1024 / 16 in bits 32..45, descriptor version 1 in bits 46..47, layout type 2 (128-byte swizzle) in bits 61..63.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor for kind::f16: fp32 accumulator (bits 4..5 = 1), bf16 A and B (bits 7..9 and 10..12 = 1),
+// both K-major (bits 15, 16 = 0), N / 8 in bits 17..22, M / 16 in bits 24..28.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(uint32_t M, uint32_t N) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
+}
+
+__device__ __forceinline__ bool bg_wait(uint32_t bar, uint32_t parity, int32_t* status, uint64_t wait_ns, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > wait_ns) {
+                atomicCAS(status, 0, ERR_SYNC_TIMEOUT);
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_constant__ BgemmParams p) {
+    extern __shared__ uint8_t bg_smem_raw[];
+    // tiles on 1024-byte boundaries (the swizzle pattern repeats every 1024 bytes)
+    const uint32_t raw = smem_u32(bg_smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    uint8_t* misc = bg_smem_raw + (tiles - raw) + (size_t)BG_STAGES * BG_STAGE_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(misc);            // [BG_STAGES] tile pair landed
+    uint64_t* empty = full + BG_STAGES;                             // [BG_STAGES] MMAs that read the stage are done
+    uint64_t* acc_full = empty + BG_STAGES;                         // [2] accumulator buffer complete
+    uint64_t* acc_empty = acc_full + 2;                             // [2] epilogue has read the buffer
+    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_s + 1);
+
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int i = 0; i < BG_STAGES; ++i) {
+            mbar_init(smem_u32(&full[i]), 1);
+            mbar_init(smem_u32(&empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&acc_full[i]), 1);
+            mbar_init(smem_u32(&acc_empty[i]), 4);   // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(tmem_base_s), BG_TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_base_s;
+
+    const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
+    const uint32_t nkb = p.nkb;
+    const uint32_t nitems = ntiles * p.S;
+    const bool skip = *p.status != 0;   // an earlier kernel of this step flagged an error: the step is a no-op
+
+    if (!skip && warp == 0 && lane == 0) {
+        // ---- producer: TMA loads of the weight tile and the input tile of every (row tile, K block) of this CTA's items
+        const uint64_t pol = l2_policy_evict_first();
+        uint32_t stage = 0, use = 0;
+        for (uint32_t item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x) {
+            const uint32_t t = item / p.S, sp = item % p.S;
+            const uint32_t kb0 = (uint32_t)(((uint64_t)sp * nkb) / p.S), kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / p.S);
+            for (uint32_t kb = kb0; kb < kb1; ++kb) {
+                if (use > 0 && !bg_wait(smem_u32(&empty[stage]), (use - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
+                const uint32_t bar = smem_u32(&full[stage]);
+                const uint32_t dst = tiles + stage * BG_STAGE_BYTES;
+                mbar_arrive_expect_tx(bar, (uint32_t)BG_STAGE_BYTES);
+                uint32_t xcol = kb * BG_TILE_K;
+                if (p.pieces == 0u) {
+                    tma_tensor_3d_g2s(dst, &p.map_w, (int32_t)xcol, (int32_t)(t * BG_TILE_M), (int32_t)p.layer, bar, pol);
+                } else {
+                    // a block that reaches past the end of its piece gets zeros there from TMA, so whatever the input
+                    // tile holds in those columns (the next piece's values) does not count
+                    const uint32_t j = kb / p.kb_piece, cin = (kb - j * p.kb_piece) * BG_TILE_K, unit0 = t * BG_TILE_M / p.rpc;
+                    xcol = j * p.kp + cin;
+                    if (j + 1u < p.pieces)
+                        tma_tensor_5d_g2s(dst, &p.map_w, (int32_t)cin, 0, (int32_t)j, (int32_t)unit0, (int32_t)p.layer, bar, pol);
+                    else
+                        tma_tensor_4d_g2s(dst, &p.map_wl, (int32_t)cin, 0, (int32_t)unit0, (int32_t)p.layer, bar, pol);
+                }
+                tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, pol);
+                if (++stage == BG_STAGES) {
+                    stage = 0;
+                    ++use;
+                }
+            }
+        }
+        if (*abort_flag) {
+            // no copy may still be writing this CTA's shared memory when it exits: wait (bounded) for the last copy
+            // armed on every stage
+            const uint64_t t0 = globaltimer_ns();
+            for (uint32_t sidx = 0; sidx < (uint32_t)BG_STAGES; ++sidx) {
+                const uint32_t cnt = use + (sidx < stage ? 1u : 0u);
+                if (cnt == 0) continue;
+                while (!mbar_try_wait(smem_u32(&full[sidx]), (cnt - 1u) & 1u))
+                    if (globaltimer_ns() - t0 > p.wait_ns) break;
+            }
+        }
+    } else if (!skip && warp == 1 && lane == 0) {
+        // ---- MMA issuer
+        const uint32_t idesc = umma_idesc_bf16(BG_TILE_M, BG_TILE_N);
+        uint32_t stage = 0, use = 0, it = 0;
+        for (uint32_t item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++it) {
+            const uint32_t sp = item % p.S;
+            const uint32_t kb0 = (uint32_t)(((uint64_t)sp * nkb) / p.S), kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / p.S);
+            const uint32_t buf = it & 1u, buse = it >> 1;
+            if (buse > 0 && !bg_wait(smem_u32(&acc_empty[buf]), (buse - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * BG_TILE_N;
+            for (uint32_t kb = kb0; kb < kb1; ++kb) {
+                if (!bg_wait(smem_u32(&full[stage]), use & 1u, p.status, p.wait_ns, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t a_addr = tiles + stage * BG_STAGE_BYTES;
+                const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + BG_A_BYTES);
+#pragma unroll
+                for (uint32_t k = 0; k < BG_TILE_K / 16; ++k)   // 16 bf16 = 32 bytes further along the swizzled row
+                    umma_f16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb != kb0 || k != 0u) ? 1u : 0u);
+                umma_commit(smem_u32(&empty[stage]));   // the stage may be refilled when these MMAs are done
+                if (++stage == BG_STAGES) {
+                    stage = 0;
+                    ++use;
+                }
+            }
+            umma_commit(smem_u32(&acc_full[buf]));
+        }
+    } else if (!skip && warp >= 2) {
+        // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 = rows of the tile
+        const uint32_t quarter = warp & 3u;
+        uint32_t it = 0;
+        for (uint32_t item = blockIdx.x; item < nitems; item += gridDim.x, ++it) {
+            const uint32_t t = item / p.S, sp = item % p.S;
+            const uint32_t buf = it & 1u, buse = it >> 1;
+            if (!bg_wait(smem_u32(&acc_full[buf]), buse & 1u, p.status, p.wait_ns, abort_flag)) break;
+            tc_fence_after();
+            uint32_t hi[32], lo[32];
+            const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BG_TILE_N;
+            tmem_ld32(taddr, hi);
+            tmem_ld32(taddr + 32u, lo);
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+            const uint32_t row = t * BG_TILE_M + quarter * 32u + lane;
+            if (row < p.R) {
+                float* dst = p.out + (size_t)sp * BG_MAX_BATCH * p.R + row;
+#pragma unroll
+                for (uint32_t b = 0; b < 32; ++b)
+                    if (b < p.B) dst[(size_t)b * p.R] = __uint_as_float(hi[b]) + __uint_as_float(lo[b]);
+            }
+        }
+    }
+    // ---- common exit: nobody may still be using TMEM when it is freed
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, BG_TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ vector kernels
+
+// Writes row b of the N operand of the next projection: xop[b][k] = hi half, xop[32 + b][k] = lo half of v (bf16).
+__device__ __forceinline__ void put_operand(__nv_bfloat16* xop, uint32_t K, uint32_t b, uint32_t k, float v) {
+    const __nv_bfloat16 h16 = __float2bfloat16_rn(v);
+    xop[(size_t)b * K + k] = h16;
+    xop[(size_t)(32 + b) * K + k] = __float2bfloat16_rn(v - __bfloat162float(h16));
+}
+
+// One block per sequence slot (grid 32).  v[k] = res[b][k] + sum_s part[s][b][k]  (res or part may be absent);
+// SWIGLU: v[f] = silu(sum_s part[s][b][2f]) * (sum_s part[s][b][2f+1]).  Optionally stores v (xout), then writes the
+// operand of the next projection: v itself, or RMSNorm(v; gain).  Slots b >= B get a zero operand.
+// The sums over the splits run in split order: reproducible.
+__global__ void __launch_bounds__(256) kl_b_finish_kernel(const float* part, uint32_t S, uint32_t Rpart, const float* res, float* xout,
+                                                          const __nv_bfloat16* gain, float eps, int swiglu, uint32_t K, uint32_t B,
+                                                          __nv_bfloat16* xop, const int32_t* status) {
+    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    __shared__ float red[8];
+    if (*status != 0) return;
+    if (b >= B) {
+        for (uint32_t k = tid; k < K; k += blockDim.x) put_operand(xop, K, b, k, 0.f);
+        return;
+    }
+    float ss = 0.f;
+    for (uint32_t k = tid; k < K; k += blockDim.x) {
+        float v;
+        if (swiglu) {
+            float g = 0.f, u = 0.f;
+            for (uint32_t s = 0; s < S; ++s) {
+                const float2 gu = *reinterpret_cast<const float2*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + 2 * k);
+                g += gu.x;
+                u += gu.y;
+            }
+            v = g / (1.0f + __expf(-g)) * u;
+        } else {
+            v = res ? res[(size_t)b * K + k] : 0.f;
+            for (uint32_t s = 0; s < S; ++s) v += part[((size_t)s * BG_MAX_BATCH + b) * Rpart + k];
+        }
+        if (xout) xout[(size_t)b * K + k] = v;
+        if (gain) ss += v * v;
+        else put_operand(xop, K, b, k, v);
+    }
+    if (!gain) return;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();   // also orders this block's xout stores before the re-reads below
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)K + eps);
+    for (uint32_t k = tid; k < K; k += blockDim.x)
+        put_operand(xop, K, b, k, xout[(size_t)b * K + k] * __bfloat162float(gain[k]) * inv);
+}
+
+// Token embedding of every sequence of the batch, and the check of the whole batch: x[b] = E[token_b].
+__global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, const int32_t* positions, const __nv_bfloat16* embed,
+                                                         float* x, uint32_t H, uint32_t V, uint32_t max_ctx, uint32_t B, int32_t* status) {
+    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    if (b >= B) return;
+    int32_t tok = tokens[b];
+    const int32_t pos = positions[b];
+    if (tid == 0 && (tok < 0 || tok >= (int32_t)V || pos < 0 || pos >= (int32_t)max_ctx)) atomicCAS(status, 0, ERR_OUT_OF_RANGE);
+    if (tok < 0 || tok >= (int32_t)V) tok = 0;
+    const __nv_bfloat16* row = embed + (size_t)tok * H;
+    for (uint32_t i = tid; i < H; i += blockDim.x) x[(size_t)b * H + i] = __bfloat162float(row[i]);
+}
+
+struct BAttnParams {
+    CUtensorMap kv_map;       // the whole KV cache as [rows, head_dim] (same map as the batch-1 kernel)
+    __nv_bfloat16* kv;
+    const int32_t* positions;
+    const double* inv_freq;
+    const float* qkv_part;    // [S][32][QR] partial sums of the QKV projection
+    float* q;                 // [32][QD] rotated, pre-scaled queries
+    float* part_o;            // [B * nkv * Sa][G][hd]
+    float* part_ml;           // [B * nkv * Sa][G][2]
+    __nv_bfloat16* xop;       // operand of the O projection [64][QD]
+    uint32_t S, QR, QD, KVD, nq, nkv, G, hd, B, max_ctx, layer, Sa;
+    int32_t* status;
+    uint64_t wait_ns;
+};
+
+// RoPE and cache append for one sequence per block: sums the splits of the QKV projection, rotates q (and scales it
+// by log2(e) / sqrt(hd) for the base-2 softmax) and k at the sequence's position, rounds k and v to bf16 and writes
+// them into row `position` of the sequence's cache slabs.  The attention kernel that follows reads that row from
+// the cache like any other.
+__global__ void __launch_bounds__(256) kl_b_rope_kernel(const BAttnParams p) {
+    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    __shared__ float cs[256];   // [hd / 2][2]
+    if (*p.status != 0 || b >= p.B) return;
+    const uint32_t hd = p.hd, half = hd >> 1;
+    const int32_t pos = p.positions[b];
+    for (uint32_t i = tid; i < half; i += blockDim.x) {
+        double sn, c;
+        sincos((double)pos * p.inv_freq[i], &sn, &c);
+        cs[2 * i] = (float)c;
+        cs[2 * i + 1] = (float)sn;
+    }
+    __syncthreads();
+    auto val = [&](uint32_t r) {
+        float v = 0.f;
+        for (uint32_t s = 0; s < p.S; ++s) v += p.qkv_part[((size_t)s * BG_MAX_BATCH + b) * p.QR + r];
+        return v;
+    };
+    const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
+    for (uint32_t idx = tid; idx < p.nq * half; idx += blockDim.x) {
+        const uint32_t h = idx / half, i = idx % half;
+        const float a = val(h * hd + i), bb = val(h * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+        p.q[(size_t)b * p.QD + h * hd + i] = (a * c - bb * sn) * qscale;
+        p.q[(size_t)b * p.QD + h * hd + i + half] = (bb * c + a * sn) * qscale;
+    }
+    const size_t slab = (size_t)p.max_ctx * hd;
+    for (uint32_t idx = tid; idx < p.nkv * half; idx += blockDim.x) {
+        const uint32_t g = idx / half, i = idx % half;
+        const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+        __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 0) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
+        row[i] = __float2bfloat16_rn(a * c - bb * sn);
+        row[i + half] = __float2bfloat16_rn(bb * c + a * sn);
+    }
+    for (uint32_t idx = tid; idx < p.nkv * hd; idx += blockDim.x) {
+        const uint32_t g = idx / hd, d = idx % hd;
+        __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 1) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
+        row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
+    }
+}
+
+constexpr int BA_WARPS = 6;
+constexpr int BA_THREADS = BA_WARPS * 32;
+constexpr int BA_SLOTS = 2;   // ring slots per warp
+
+// Split-K flash-decoding over (split, kv head, sequence) units.  Every warp streams its own chunks of 32 (head size
+// 128) or 64 (head size 64) cached positions through a two-slot ring of its own (lane 0 issues the TMA box loads two
+// chunks ahead) and runs the mma.sync tiles of kl_attention_tc.cuh on them; the warps' results are merged in shared
+// memory and written as the unit's partial result (O^T unnormalised, running maximum, sum).
+template <int HD, bool PACK>
+__device__ __forceinline__ void b_attn_unit(const BAttnParams& p, uint8_t* smem_raw) {
+    const uint32_t sp = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t G = p.G;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;
+    uint8_t* after = smem_raw + (ring - raw) + (size_t)BA_WARPS * BA_SLOTS * SLOT_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(after);                          // [BA_WARPS * BA_SLOTS]
+    float* q_s = reinterpret_cast<float*>(after + 128);                           // [G][HD]
+    float* comb = q_s + G * HD;                                                   // [BA_WARPS][G][HD + 2]
+    float* ftab = comb + (size_t)BA_WARPS * G * (HD + 2);                         // [BA_WARPS][G] + [G]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ftab + BA_WARPS * MAX_G + MAX_G);
+
+    if (tid == 0) {
+        for (int i = 0; i < BA_WARPS * BA_SLOTS; ++i) mbar_init(smem_u32(&full[i]), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    for (uint32_t i = tid; i < G * HD; i += blockDim.x) q_s[i] = p.q[(size_t)b * p.QD + (size_t)g * G * HD + i];
+    __syncthreads();
+
+    // positions of this unit: split sp of 0 .. position (the row appended by this step included)
+    const uint32_t n = (uint32_t)p.positions[b] + 1u;
+    const uint32_t clen = (n + p.Sa - 1) / p.Sa;
+    const uint32_t c0 = min(n, sp * clen), cend = min(n, c0 + clen);
+    const uint32_t pb = SLOT_BYTES / (4u * HD);
+    const uint32_t nring = (cend - c0 + pb - 1) / pb;
+    const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
+    const uint32_t row0 = p.layer * 2u * vdelta + (b * p.nkv + g) * p.max_ctx;
+    const uint32_t box_bytes = pb * 128u;
+    const uint64_t pol = l2_policy_evict_first();
+
+    auto issue = [&](uint32_t i, uint32_t slot) {   // lane 0: chunk i of the unit into this warp's slot
+        const AttnWindow w = attn_window(c0, cend, pb, i);
+        const uint32_t bar = smem_u32(&full[warp * BA_SLOTS + slot]);
+        const uint32_t dst = ring + (warp * BA_SLOTS + slot) * SLOT_BYTES;
+        mbar_arrive_expect_tx(bar, (uint32_t)SLOT_BYTES);
+#pragma unroll
+        for (uint32_t bx = 0; bx < HD / 64u; ++bx) {
+            tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + w.w0), bar, pol);
+            tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + w.w0 + vdelta), bar, pol);
+        }
+    };
+    if (lane == 0) {
+        if (warp < nring) issue(warp, 0);
+        if (warp + BA_WARPS < nring) issue(warp + BA_WARPS, 1);
+    }
+
+    constexpr int NKB = HD / 16, NMT = HD / 16;
+    const uint32_t gq = lane >> 2, t = lane & 3u;
+    AttnTcState<HD> st;
+#pragma unroll
+    for (int kb = 0; kb < NKB; ++kb) {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const uint32_t k = kb * 16 + hf * 8 + 2 * t;
+            const uint32_t head = PACK ? (gq & 3u) : gq;
+            float2 xx = make_float2(0.f, 0.f);
+            if (head < G) xx = *reinterpret_cast<const float2*>(q_s + head * HD + k);
+            const uint32_t hi = pack_bf16(xx.x, xx.y);
+            const uint32_t lo = pack_bf16(xx.x - bf_lo(hi), xx.y - bf_hi(hi));
+            st.qh[kb][hf] = (PACK && gq >= 4u) ? lo : hi;
+            st.ql[kb][hf] = lo;
+        }
+    }
+#pragma unroll
+    for (int nn = 0; nn < NMT; ++nn) st.o[nn][0] = st.o[nn][1] = st.o[nn][2] = st.o[nn][3] = 0.f;
+    st.m[0] = st.m[1] = -INFINITY;
+    st.l[0] = st.l[1] = 0.f;
+
+    // chunk c of this warp (c = 0, 1, ...) sits in slot c % BA_SLOTS and completes phase (c / BA_SLOTS) % 2 of its barrier
+    uint32_t consumed = 0;
+    uint32_t issued = (warp < nring ? 1u : 0u) + (warp + BA_WARPS < nring ? 1u : 0u);
+    for (uint32_t i = warp; i < nring; i += BA_WARPS, ++consumed) {
+        const uint32_t slot = consumed % BA_SLOTS, phase = (consumed / BA_SLOTS) & 1u;
+        if (!bg_wait(smem_u32(&full[warp * BA_SLOTS + slot]), phase, p.status, p.wait_ns, abort_flag)) break;
+        const uint32_t kbase = ring + (warp * BA_SLOTS + slot) * SLOT_BYTES;
+        const AttnWindow w = attn_window(c0, cend, pb, i);
+        for (uint32_t r0 = 0; r0 < pb; r0 += 16)
+            if (r0 + 16 > w.lo && r0 < w.hi) attn_tc_tile<HD, PACK>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, r0, w.lo, w.hi, lane);
+        __syncwarp();
+        if (i + BA_SLOTS * BA_WARPS < nring) {
+            if (lane == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the slot was read through the generic proxy
+                issue(i + BA_SLOTS * BA_WARPS, slot);
+            }
+            ++issued;
+        }
+    }
+    // after a time-out copies may still be in flight: wait (bounded) for every chunk issued but not consumed
+    if (consumed < issued && lane == 0) {
+        const uint64_t t0 = globaltimer_ns();
+        for (uint32_t c = consumed; c < issued; ++c)
+            while (!mbar_try_wait(smem_u32(&full[warp * BA_SLOTS + c % BA_SLOTS]), (c / BA_SLOTS) & 1u))
+                if (globaltimer_ns() - t0 > p.wait_ns) break;
+    }
+
+    // this warp's result into shared memory (same layout as the batch-1 kernel)
+    float l0 = st.l[0], l1 = st.l[1];
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) {
+        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+    }
+    if (PACK) {
+#pragma unroll
+        for (int nn = 0; nn < NMT; ++nn)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) st.o[nn][j] += __shfl_xor_sync(0xffffffffu, st.o[nn][j], 2);
+    }
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const uint32_t h = 2 * t + hh;
+        if (h < G && (!PACK || t < 2u)) {
+            float* dst = comb + ((size_t)warp * G + h) * (HD + 2);
+#pragma unroll
+            for (int nn = 0; nn < NMT; ++nn) {
+                dst[nn * 16 + gq] = st.o[nn][hh];
+                dst[nn * 16 + gq + 8] = st.o[nn][2 + hh];
+            }
+            if (gq == 0) {
+                dst[HD] = st.m[hh];
+                dst[HD + 1] = hh ? l1 : l0;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < BA_WARPS * G) {
+        const uint32_t w = tid / G, h = tid % G;
+        float Mh = -INFINITY;
+#pragma unroll
+        for (int ww = 0; ww < BA_WARPS; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (HD + 2) + HD]);
+        ftab[w * G + h] = rescale(comb[((size_t)w * G + h) * (HD + 2) + HD], Mh);
+        if (w == 0) ftab[BA_WARPS * G + h] = Mh;
+    }
+    __syncthreads();
+    const uint32_t unit = (b * p.nkv + g) * p.Sa + sp;
+    for (uint32_t x = tid; x < G * HD; x += blockDim.x) {
+        const uint32_t h = x / HD, d = x % HD;
+        float A = 0.f, Ls = 0.f;
+#pragma unroll
+        for (int w = 0; w < BA_WARPS; ++w) {
+            const float* src = comb + ((size_t)w * G + h) * (HD + 2);
+            const float c = ftab[w * G + h];
+            A += src[d] * c;
+            Ls += src[HD + 1] * c;
+        }
+        p.part_o[((size_t)unit * G + h) * HD + d] = A;
+        if (d == 0) {
+            p.part_ml[((size_t)unit * G + h) * 2] = ftab[BA_WARPS * G + h];
+            p.part_ml[((size_t)unit * G + h) * 2 + 1] = Ls;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_constant__ BAttnParams p) {
+    extern __shared__ uint8_t ba_smem_raw[];
+    if (*p.status != 0) return;
+    if (p.hd == 128) {
+        if (p.G <= 4) b_attn_unit<128, true>(p, ba_smem_raw);
+        else b_attn_unit<128, false>(p, ba_smem_raw);
+    } else {
+        if (p.G <= 4) b_attn_unit<64, true>(p, ba_smem_raw);
+        else b_attn_unit<64, false>(p, ba_smem_raw);
+    }
+}
+
+// Merges the Sa partial results of every (sequence, kv head) and writes the attention output straight into the
+// operand of the O projection (bf16 hi and lo halves).  Grid (nkv, 32): slots b >= B get zeros.
+__global__ void __launch_bounds__(256) kl_b_attn_merge_kernel(const BAttnParams p) {
+    const uint32_t g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const uint32_t G = p.G, hd = p.hd;
+    if (*p.status != 0) return;
+    for (uint32_t x = tid; x < G * hd; x += blockDim.x) {
+        const uint32_t h = x / hd, d = x % hd;
+        float v = 0.f;
+        if (b < p.B) {
+            const size_t u0 = (size_t)(b * p.nkv + g) * p.Sa;
+            float M = -INFINITY;
+            for (uint32_t s = 0; s < p.Sa; ++s) M = fmaxf(M, p.part_ml[((u0 + s) * G + h) * 2]);
+            float L = 0.f, A = 0.f;
+            for (uint32_t s = 0; s < p.Sa; ++s) {
+                const float c = rescale(p.part_ml[((u0 + s) * G + h) * 2], M);
+                L += p.part_ml[((u0 + s) * G + h) * 2 + 1] * c;
+                A += p.part_o[((u0 + s) * G + h) * hd + d] * c;
+            }
+            v = A / L;
+        }
+        put_operand(p.xop, p.QD, b, (g * G + h) * hd + d, v);
+    }
+}
+
+}  // namespace kl

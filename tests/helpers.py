@@ -77,9 +77,11 @@ def bf16_decode(u16: np.ndarray) -> np.ndarray:
 
 def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
                modes=(binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER, binding.KL_MODE_PER_STAGE),
-               overrides=None, positions0=None, stream_layers=False, check_cache=True):
+               overrides=None, positions0=None, stream_layers=False, check_cache=True, batched_path=None):
     """Teacher-forced greedy decode: the oracle runs `steps` steps on its own tokens; each CUDA mode consumes the
-    oracle's token of the previous step.  Returns a report dict; asserts nothing."""
+    oracle's token of the previous step.  Returns a report dict; asserts nothing.  batched_path: None leaves the
+    library's default (batches take the tensor-core path when the shape allows), True / False forces the choice
+    (True raises when the shape has no such path)."""
     max_ctx = max_ctx or (context + steps + 8)
     host = HostWeights(shape, seed, stream_layers, overrides)
     orc = ko.Oracle(shape, max_ctx, host.layer, host.globals())
@@ -99,6 +101,8 @@ def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
 
     report = dict(ref=ref, modes={}, cache_ref=cache_or, cache0=cache0.cpu().view(torch.uint16).numpy())
     dec = make_decoder(shape, batch, max_ctx, seed, overrides)
+    if batched_path is not None:
+        dec.kl_set_batched_path(batched_path)
     for mode in modes:
         dec.kl_set_mode(mode)
         cache = cache0.clone().cuda()
@@ -123,7 +127,7 @@ def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
     return report
 
 
-def assert_parity(report, steps, batch=1, check_cache=True):
+def assert_parity(report, steps, batch=1, check_cache=True, flip_tol=0.02):
     ref = report["ref"]
     for mode, res in report["modes"].items():
         for s in range(steps):
@@ -143,7 +147,7 @@ def assert_parity(report, steps, batch=1, check_cache=True):
             assert np.array_equal(got[~changed], exp[~changed]), mode
             g, e = bf16_decode(got[changed]), bf16_decode(exp[changed])
             assert np.all(np.abs(g - e) <= 2.0 ** -7 * np.abs(e) + 1e-3 * np.abs(e).max()), mode
-            assert (got[changed] != exp[changed]).mean() < 0.02, mode
+            assert (got[changed] != exp[changed]).mean() < flip_tol, mode
     modes = list(report["modes"].values())
     for other in modes[1:]:  # the transformation preserves semantics: all schedules run the same arithmetic
         for s in range(steps):

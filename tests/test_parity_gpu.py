@@ -80,16 +80,87 @@ def test_llama31_70b_shape_two_layers():
 
 
 def test_batch_of_sequences_ragged_positions():
-    """Batches are decoded one sequence after another by the batch-1 kernels: three sequences at different
-    positions, four steps, both schedules; every sequence matches the oracle and its cache rows land in its own
-    slab of the [L][2][B][nkv][max_ctx][hd] cache."""
-    rep = helpers.run_parity(gen.TINY, context=128, steps=4, seed=3, batch=3, positions0=[5, 64, 128])
+    """Without the batched path a batch is decoded one sequence after another by the batch-1 kernels: three sequences
+    at different positions, four steps, all schedules; every sequence matches the oracle and its cache rows land in
+    its own slab of the [L][2][B][nkv][max_ctx][hd] cache."""
+    rep = helpers.run_parity(gen.TINY, context=128, steps=4, seed=3, batch=3, positions0=[5, 64, 128], batched_path=False)
     helpers.assert_parity(rep, 4, batch=3)
 
 
-def test_batch_bad_entry_makes_the_whole_step_a_no_op():
+BATCHED = {
+    # name: (shape, batch, context, first positions)
+    "tiny_b3": (gen.TINY, 3, 128, [5, 64, 128]),
+    # a full batch with every length from an empty cache up: attention units with no position, one position, ragged tails
+    "tiny_b32": (gen.TINY, 32, 330, [0, 1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129] + list(range(130, 330, 10))),
+    # rows and columns that are no multiples of the 128 x 64 tiles (TMA fills the tile edges with zeros), head size 128
+    "odd_rows_hd128_b5": (SHAPES["odd_rows_hd128"], 5, 150, [0, 17, 64, 149, 150]),
+    # gate/up stored in chunk order (units of two rows cut into two column pieces): the rank-5 / rank-4 tensor maps; G = 8
+    "wide_hidden_g8_b4": (SHAPES["wide_hidden_g8"], 4, 150, [3, 77, 128, 150]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(BATCHED))
+def test_batched_tensor_core_path(name):
+    """Batches on the tcgen05 path (every projection one dense contraction for the whole batch; the default for
+    batch > 1): every sequence matches the oracle within the same tolerances as the batch-1 kernels, greedy tokens
+    included, and the appended cache rows land in the right slabs.
+
+    The projections take their fp32 inputs as two bf16 halves (16 significant bits instead of 24), so a k or v value
+    that lies within ~2^-17 of a bf16 rounding boundary may round the other way than in the oracle; for a sequence
+    with a single cached position that one-step difference reaches the next layer undiluted and flips more there.
+    Every appended value is still within one bf16 step of the oracle's (checked); only the share of values that
+    differ at all is allowed to be larger than for the fp32 batch-1 kernels."""
+    shape, batch, context, pos0 = BATCHED[name]
+    rep = helpers.run_parity(shape, context=context, steps=3, seed=3, batch=batch, positions0=pos0,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True)
+    helpers.assert_parity(rep, 3, batch=batch, flip_tol=0.05)
+
+
+def test_batched_path_llama31_8b_shape_b32():
+    """Config 4 by sampled layers: the 8B shape (down projection in chunk order with ten column pieces), batch 32,
+    ragged contexts up to 1024, the first two layers and the classifier, two decode steps."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_8B, n_layers=2)
+    pos0 = [1024 - 29 * i for i in range(32)]
+    rep = helpers.run_parity(shape, context=1024, steps=2, seed=0, batch=32, positions0=pos0, max_ctx=1024 + 8,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True, check_cache=False)
+    helpers.assert_parity(rep, 2, batch=32, check_cache=False)
+
+
+def test_batched_path_is_reproducible_and_optional():
+    """The split sums are added in a fixed order: the same batched step twice gives identical bits.  A shape without
+    the path (head size 32) refuses to switch it on and decodes batches on the batch-1 kernels."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 4, 200, 0)
+    cache0 = gen.make_kv_cache(shape, 4, 128, 200, 0, "cuda")
+    tok = gen.make_tokens(shape, 4, 0).cuda()
+    pos = torch.tensor([128, 7, 64, 0], dtype=torch.int32, device="cuda")
+    outs = []
+    for _ in range(3):
+        cache = cache0.clone()
+        logits = torch.empty(4, shape.vocab, device="cuda")
+        hidden = torch.empty(4, shape.hidden, device="cuda")
+        dec.kl_decode_step(tok, pos, cache, logits, 4)
+        dec.kl_read_hidden(hidden, 4)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        outs.append((logits.cpu(), hidden.cpu(), cache.cpu().view(torch.uint16)))
+    for lg, hd, ch in outs[1:]:
+        assert torch.equal(lg, outs[0][0]) and torch.equal(hd, outs[0][1]) and torch.equal(ch, outs[0][2])
+    dec.close()
+    dec = binding.Decoder(SHAPES["split_k_down"], 2, 64)
+    with pytest.raises(binding.KlError) as e:
+        dec.kl_set_batched_path(True)
+    assert e.value.code == binding.KL_ERR_UNSUPPORTED_SHAPE
+    dec.kl_set_batched_path(False)
+    dec.close()
+
+
+@pytest.mark.parametrize("batched", [True, False])
+def test_batch_bad_entry_makes_the_whole_step_a_no_op(batched):
     shape = gen.TINY
     dec = helpers.make_decoder(shape, 2, 200, 0)
+    dec.kl_set_batched_path(batched)
     cache = gen.make_kv_cache(shape, 2, 128, 200, 0, "cuda")
     before = cache.clone()
     tok = torch.tensor([1, shape.vocab + 7], dtype=torch.int32, device="cuda")   # the SECOND sequence is bad
@@ -100,6 +171,12 @@ def test_batch_bad_entry_makes_the_whole_step_a_no_op():
     assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE
     assert torch.equal(cache.view(torch.uint16), before.view(torch.uint16))       # nothing appended, not even for sequence 0
     assert bool((logits == 7.0).all())
+    # the handle stays usable: the same step with valid tokens runs
+    tok[1] = 2
+    dec.kl_decode_step(tok, pos, cache, logits, 2)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    assert bool(torch.isfinite(logits).all()) and not bool((logits == 7.0).all())
     dec.close()
 
 
