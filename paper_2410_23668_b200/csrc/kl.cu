@@ -276,7 +276,8 @@ struct kl_handle {
     int bt_ok;             // 1: available for this shape
     int use_bt;            // 1 (default): batches take it; 0: sequence after sequence on the batch-1 kernels
     float* bx;             // [32][H] hidden states of the batch (== hidden_all)
-    __nv_bfloat16* bxop;   // [64][Kmax] operand of the next projection (hi and lo halves)
+    __nv_bfloat16* bxop[3];   // operands [64][H], [64][QD], [64][F]: rows 0..31 hi halves, 32..63 lo halves
+    float* bssq;           // [32][BV_MAX_CHUNKS] partial sums of squares of the residual stream
     float* bpart;          // partial sums of the projection in flight
     float* bq;             // [32][QD] rotated queries
     float* bao;            // attention partial outputs
@@ -312,7 +313,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbpart, sbq, sbao, sbaml, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
     uint32_t bsplit[5], battn_splits;
     uint32_t cps;
 };
@@ -330,18 +331,20 @@ bool shape_supported(const kl_model_desc& d, int num_sms) {
     return true;
 }
 
-static size_t ceil_div(size_t a, size_t b) { return (a + b - 1) / b; }
-
-// K splits of a batched projection: the (row tile, split) items are dealt round-robin to the CTAs; pick the count that
-// wastes the least of the last round, with at least four K blocks per split and at most eight splits.
-static uint32_t pick_split(uint32_t tiles, uint32_t nkb, uint32_t P) {
+// K splits of a batched projection [R x K]: the (row tile, split) items are dealt round-robin to the P CTAs.  More
+// splits fill the last round better but every split writes and the consumer re-reads a [32 x R] fp32 partial result;
+// pick the count that minimises streamed bytes (idle CTAs of the last round counted as if they streamed) plus that
+// partial traffic, with at least four K blocks per split and at most eight splits.
+static uint32_t pick_split(uint32_t R, uint32_t K, uint32_t P) {
+    const uint32_t tiles = (R + 127) / 128, nkb = (K + 63) / 64;
     uint32_t best = 1;
-    double best_eff = 0.0;
-    for (uint32_t sp = 1; sp <= 8 && nkb / sp >= 4; ++sp) {
+    double best_cost = 0.0;
+    for (uint32_t sp = 1; sp <= 8 && (sp == 1 || nkb / sp >= 4); ++sp) {
         const uint32_t items = tiles * sp;
-        const double eff = (double)items / (double)(((items + P - 1) / P) * P);
-        if (eff > best_eff + 1e-9) {
-            best_eff = eff;
+        const double stream = (double)((items + P - 1) / P) * P * (128.0 * K * 2.0 / sp);
+        const double cost = stream + 2.0 * sp * R * 32.0 * 4.0;
+        if (sp == 1 || cost < best_cost) {
+            best_cost = cost;
             best = sp;
         }
     }
@@ -401,7 +404,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.sh = s;        s += align_up(B * F * 4);
     y.spart = s;     s += align_up(units * G * d.head_dim * 8);
     y.spart_ml = s;  s += align_up(units * G * 2 * 8);
-    y.srope = s;     s += align_up(B * d.head_dim * 4);
+    y.srope = s;     s += align_up((B > 1 ? 32 : B) * d.head_dim * 4);
     y.sinvf = s;     s += align_up((size_t)(d.head_dim / 2) * 8);
     y.scounters = s; s += align_up((size_t)d.n_layers * 4);
     y.sstatus = s;   s += ALIGN;
@@ -414,18 +417,17 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     // batched path (max_batch > 1): operand, partial sums, queries, attention partials
     {
         const size_t QR = QD + 2 * KVD;
-        const uint32_t tiles[5] = {(uint32_t)ceil_div(QR, 128), (uint32_t)ceil_div(H, 128), (uint32_t)ceil_div(2 * F, 128),
-                                   (uint32_t)ceil_div(H, 128), (uint32_t)ceil_div(V, 128)};
         const size_t rows[5] = {QR, H, 2 * F, H, V}, ks[5] = {H, QD, H, F, H};
         size_t part_max = 0;
         for (int i = 0; i < 5; ++i) {
-            y.bsplit[i] = i == 4 ? 1u : pick_split(tiles[i], (uint32_t)ceil_div(ks[i], 64), (uint32_t)num_sms);
+            y.bsplit[i] = i == 4 ? 1u : pick_split((uint32_t)rows[i], (uint32_t)ks[i], (uint32_t)num_sms);
             if (i < 4 && y.bsplit[i] * rows[i] > part_max) part_max = y.bsplit[i] * rows[i];
         }
         y.battn_splits = 16;
-        const size_t kmax = H > QD ? (H > F ? H : F) : (QD > F ? QD : F);
         const bool on = B > 1;
-        y.sbxop = s;  s += on ? align_up(64 * kmax * 2 + 1024) : 0;
+        // one operand buffer per input width (hidden, q width, ffn), each on a 1024-byte boundary
+        y.sbxop = s;  s += on ? align_up(64 * H * 2 + 1024) + align_up(64 * QD * 2 + 1024) + align_up(64 * F * 2 + 1024) : 0;
+        y.sbssq = s;  s += on ? align_up((size_t)32 * BV_MAX_CHUNKS * 4) : 0;
         y.sbpart = s; s += on ? align_up(part_max * 32 * 4) : 0;
         y.sbq = s;    s += on ? align_up(32 * QD * 4) : 0;
         y.sbao = s;   s += on ? align_up(B * d.n_kv_heads * y.battn_splits * G * d.head_dim * 4) : 0;
@@ -735,7 +737,15 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->last_batch = 1;
     // tensor-core path for batches of up to 32 sequences
     h->bx = h->hidden_all;
-    h->bxop = (__nv_bfloat16*)(((uintptr_t)(sc + y.sbxop) + 1023u) & ~(uintptr_t)1023u);
+    {
+        uintptr_t a = ((uintptr_t)(sc + y.sbxop) + 1023u) & ~(uintptr_t)1023u;
+        const size_t widths[3] = {p.H, p.QD, p.F};
+        for (int i = 0; i < 3; ++i) {
+            h->bxop[i] = (__nv_bfloat16*)a;
+            a = (a + 64 * widths[i] * 2 + 1023u) & ~(uintptr_t)1023u;
+        }
+    }
+    h->bssq = (float*)(sc + y.sbssq);
     h->bpart = (float*)(sc + y.sbpart);
     h->bq = (float*)(sc + y.sbq);
     h->bao = (float*)(sc + y.sbao);
@@ -753,9 +763,10 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
                   encode_weight_maps(h->encode_tiled, &h->bmap_w[2], &h->bmap_wl[2], p.wgu, p.plan[PL_GU], 2 * p.F, p.L, p.layer_stride) &&
                   encode_weight_maps(h->encode_tiled, &h->bmap_w[3], &h->bmap_wl[3], p.wd, p.plan[PL_D], p.H, p.L, p.layer_stride) &&
                   encode_weight_maps(h->encode_tiled, &h->bmap_w[4], &h->bmap_wl[4], p.wlm, p.plan[PL_LM], p.V, 1, 0) &&
-                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[0], h->bxop, 64, p.H, BG_TILE_N) &&
-                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[1], h->bxop, 64, p.QD, BG_TILE_N) &&
-                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[2], h->bxop, 64, p.F, BG_TILE_N);
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[0], h->bxop[0], 64, p.H, BG_TILE_N) &&
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[1], h->bxop[1], 64, p.QD, BG_TILE_N) &&
+                  encode_bf16_2d(h->encode_tiled, &h->bmap_x[2], h->bxop[2], 64, p.F, BG_TILE_N);
+        ok = ok && p.H <= (uint32_t)(BV_CHUNK * BV_MAX_CHUNKS);
         ok = ok && cudaFuncSetAttribute(kl_bgemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BG_SMEM_BYTES) == cudaSuccess &&
              cudaFuncSetAttribute(kl_b_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ba_smem) == cudaSuccess;
         (void)cudaGetLastError();
@@ -886,6 +897,10 @@ static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out,
         g.pieces = pl.npieces;
         g.nkb = (pl.npieces - 1) * g.kb_piece + ceil_div(pl.K - (pl.npieces - 1) * pl.kp, (uint32_t)BG_TILE_K);
     }
+    const bool normed = idx == 0 || idx == 2 || idx == 4;   // inputs that are RMSNorm outputs: the factor is applied here
+    g.ssq = normed ? h->bssq : nullptr;
+    g.ssq_n = ceil_div(p.H, (uint32_t)BV_CHUNK);
+    g.eps = p.eps;
     g.status = p.status;
     g.wait_ns = p.wait_ns;
     const uint32_t items = ceil_div(g.R, (uint32_t)BG_TILE_M) * g.S;
@@ -905,12 +920,12 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     if (trc != KL_OK) return trc;
     a.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
     a.positions = positions_d;
-    a.inv_freq = p.inv_freq;
+    a.cs = p.rope_cs;
     a.qkv_part = h->bpart;
     a.q = h->bq;
     a.part_o = h->bao;
     a.part_ml = h->baml;
-    a.xop = h->bxop;
+    a.xop = h->bxop[1];
     a.S = h->bsplit[0];
     a.QR = p.QD + 2 * p.KVD;
     a.QD = p.QD; a.KVD = p.KVD; a.nq = p.nq; a.nkv = p.nkv; a.G = p.G; a.hd = p.hd;
@@ -927,39 +942,41 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
         if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA; \
         ++h->launches;                                        \
     } while (0)
-    kl_b_embed_kernel<<<batch, 256, 0, st>>>(tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, batch, p.status);
+    kl_b_embed_kernel<<<batch, 256, 0, st>>>(tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, p.inv_freq, p.rope_cs,
+                                             p.hd / 2, p.status);
     KL_B_CHECK();
     if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+    const dim3 grid_h(batch, ceil_div(p.H, (uint32_t)BV_CHUNK)), grid_f(batch, ceil_div(p.F, (uint32_t)BV_CHUNK));
     uint32_t s_prev = 0;   // splits of the down projection whose sums are still to be added to the residual stream
     for (uint32_t l = 0; l < p.L; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         a.layer = l;
-        // x += down projection of the previous layer; operand = RMSNorm(x; g1)
-        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, p.eps, 0, p.H, batch, h->bxop, p.status);
+        // x += down projection of the previous layer; operand = g1 * x, sums of squares for the RMSNorm factor
+        kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);
         KL_B_CHECK();
         if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st)) != KL_OK) return rc;
-        kl_b_rope_kernel<<<batch, 256, 0, st>>>(a);
+        kl_b_rope_kernel<<<dim3(batch, p.nq + 2 * p.nkv), 128, 0, st>>>(a);
         KL_B_CHECK();
         kl_b_attn_kernel<<<dim3(a.Sa, p.nkv, batch), BA_THREADS, ba_smem, st>>>(a);
         KL_B_CHECK();
-        kl_b_attn_merge_kernel<<<dim3(p.nkv, 32), 256, 0, st>>>(a);
+        kl_b_attn_merge_kernel<<<dim3(p.nkv, batch), 256, 0, st>>>(a);
         KL_B_CHECK();
         if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st)) != KL_OK) return rc;
-        // x += attention output projection; operand = RMSNorm(x; g2)
-        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, p.eps, 0, p.H, batch, h->bxop,
-                                               p.status);
+        // x += attention output projection; operand = g2 * x
+        kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq,
+                                                   p.status);
         KL_B_CHECK();
         if ((rc = launch_bgemm(h, 2, l, h->bpart, batch, st)) != KL_OK) return rc;
         // operand = silu(gate) * up
-        kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, p.eps, 1, p.F, batch,
-                                               h->bxop, p.status);
+        kl_b_finish_kernel<<<grid_f, 256, 0, st>>>(h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, 1, p.F, h->bxop[2],
+                                                   nullptr, p.status);
         KL_B_CHECK();
         if ((rc = launch_bgemm(h, 3, l, h->bpart, batch, st)) != KL_OK) return rc;
         s_prev = h->bsplit[3];
     }
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
-    // x += last down projection (kept for kl_read_hidden); operand = RMSNorm(x; gf); logits = W_lm . operand
-    kl_b_finish_kernel<<<32, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, p.eps, 0, p.H, batch, h->bxop, p.status);
+    // x += last down projection (kept for kl_read_hidden); operand = gf * x; logits = RMSNorm factor * W_lm . operand
+    kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, 0, p.H, h->bxop[0], h->bssq, p.status);
     KL_B_CHECK();
     if ((rc = launch_bgemm(h, 4, 0, logits_d, batch, st)) != KL_OK) return rc;
     if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;

@@ -49,9 +49,17 @@ struct BgemmParams {
     uint32_t kp;           // columns per full piece
     uint32_t kb_piece;     // K blocks per full piece = ceil(kp / 64)
     uint32_t rpc;          // rows per unit of the chunk order
+    // RMSNorm folded behind the contraction: when ssq is set the operand holds gain * x (not normalised) and the epilogue
+    // multiplies column b by rsqrt(sum_c ssq[b][c] / K + eps); ssq[b][c] are the partial sums of squares of x[b]
+    const float* ssq;
+    uint32_t ssq_n;        // partial sums per sequence
+    float eps;
     int32_t* status;
     uint64_t wait_ns;
 };
+
+constexpr int BV_CHUNK = 512;        // elements per block of the vector kernels (256 threads x 2)
+constexpr int BV_MAX_CHUNKS = 64;    // partial sums of squares per sequence: hidden <= 32768
 
 // ---- PTX wrappers (tcgen05 / TMEM / higher-rank TMA)
 
@@ -269,6 +277,12 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
         // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 = rows of the tile
         const uint32_t quarter = warp & 3u;
         uint32_t it = 0;
+        float inv = 1.0f;   // lane b: the RMSNorm factor of sequence b
+        if (p.ssq != nullptr && lane < p.B) {
+            float ss = 0.f;
+            for (uint32_t c = 0; c < p.ssq_n; ++c) ss += p.ssq[lane * BV_MAX_CHUNKS + c];
+            inv = rsqrtf(ss / (float)p.K + p.eps);
+        }
         for (uint32_t item = blockIdx.x; item < nitems; item += gridDim.x, ++it) {
             const uint32_t t = item / p.S, sp = item % p.S;
             const uint32_t buf = it & 1u, buse = it >> 1;
@@ -283,11 +297,11 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
             const uint32_t row = t * BG_TILE_M + quarter * 32u + lane;
-            if (row < p.R) {
-                float* dst = p.out + (size_t)sp * BG_MAX_BATCH * p.R + row;
+            float* dst = p.out + (size_t)sp * BG_MAX_BATCH * p.R + row;
 #pragma unroll
-                for (uint32_t b = 0; b < 32; ++b)
-                    if (b < p.B) dst[(size_t)b * p.R] = __uint_as_float(hi[b]) + __uint_as_float(lo[b]);
+            for (uint32_t b = 0; b < 32; ++b) {
+                const float sc = __shfl_sync(0xffffffffu, inv, b);   // all lanes take part, also those past the last row
+                if (row < p.R && b < p.B) dst[(size_t)b * p.R] = (__uint_as_float(hi[b]) + __uint_as_float(lo[b])) * sc;
             }
         }
     }
@@ -302,68 +316,81 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
 
 // ------------------------------------------------------------------------------------------------ vector kernels
 
-// Writes row b of the N operand of the next projection: xop[b][k] = hi half, xop[32 + b][k] = lo half of v (bf16).
-__device__ __forceinline__ void put_operand(__nv_bfloat16* xop, uint32_t K, uint32_t b, uint32_t k, float v) {
-    const __nv_bfloat16 h16 = __float2bfloat16_rn(v);
-    xop[(size_t)b * K + k] = h16;
-    xop[(size_t)(32 + b) * K + k] = __float2bfloat16_rn(v - __bfloat162float(h16));
+// Row b of the N operand of a projection: xop[b][k] = hi half, xop[32 + b][k] = lo half (bf16) of the fp32 value.
+// Every projection input width has an operand buffer of its own; rows of sequences beyond the batch keep whatever
+// finite values they last held (the MMA columns they feed are never stored).
+__device__ __forceinline__ void put_operand2(__nv_bfloat16* xop, uint32_t K, uint32_t b, uint32_t k, float v0, float v1) {
+    const uint32_t hi = pack_bf16(v0, v1);
+    const uint32_t lo = pack_bf16(v0 - bf_lo(hi), v1 - bf_hi(hi));
+    *reinterpret_cast<uint32_t*>(xop + (size_t)b * K + k) = hi;
+    *reinterpret_cast<uint32_t*>(xop + (size_t)(32 + b) * K + k) = lo;
 }
 
-// One block per sequence slot (grid 32).  v[k] = res[b][k] + sum_s part[s][b][k]  (res or part may be absent);
-// SWIGLU: v[f] = silu(sum_s part[s][b][2f]) * (sum_s part[s][b][2f+1]).  Optionally stores v (xout), then writes the
-// operand of the next projection: v itself, or RMSNorm(v; gain).  Slots b >= B get a zero operand.
-// The sums over the splits run in split order: reproducible.
+// Vector work between two projections; grid (batch, ceil(K / BV_CHUNK)), 256 threads x 2 elements.
+//   swiglu = 0:  v[k] = res[b][k] + sum_s part[s][b][k];  xout[b][k] = v[k];  operand = gain[k] * v[k] (the RMSNorm
+//                factor is applied behind the next contraction);  ssq[b][chunk] = sum of v[k]^2 over the chunk.
+//   swiglu = 1:  v[f] = silu(sum_s part[s][b][2f]) * (sum_s part[s][b][2f+1]);  operand = v.
+// The sums over the splits run in split order and the sum of squares in a fixed tree: reproducible.
 __global__ void __launch_bounds__(256) kl_b_finish_kernel(const float* part, uint32_t S, uint32_t Rpart, const float* res, float* xout,
-                                                          const __nv_bfloat16* gain, float eps, int swiglu, uint32_t K, uint32_t B,
-                                                          __nv_bfloat16* xop, const int32_t* status) {
-    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+                                                          const __nv_bfloat16* gain, int swiglu, uint32_t K, __nv_bfloat16* xop,
+                                                          float* ssq, const int32_t* status) {
+    const uint32_t b = blockIdx.x, c = blockIdx.y, tid = threadIdx.x;
     __shared__ float red[8];
     if (*status != 0) return;
-    if (b >= B) {
-        for (uint32_t k = tid; k < K; k += blockDim.x) put_operand(xop, K, b, k, 0.f);
-        return;
-    }
-    float ss = 0.f;
-    for (uint32_t k = tid; k < K; k += blockDim.x) {
-        float v;
+    const uint32_t k = c * BV_CHUNK + 2 * tid;
+    float v0 = 0.f, v1 = 0.f;
+    if (k < K) {   // K is even
         if (swiglu) {
-            float g = 0.f, u = 0.f;
+            float g0 = 0.f, u0 = 0.f, g1 = 0.f, u1 = 0.f;
             for (uint32_t s = 0; s < S; ++s) {
-                const float2 gu = *reinterpret_cast<const float2*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + 2 * k);
-                g += gu.x;
-                u += gu.y;
+                const float4 gu = *reinterpret_cast<const float4*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + 2 * k);
+                g0 += gu.x; u0 += gu.y; g1 += gu.z; u1 += gu.w;
             }
-            v = g / (1.0f + __expf(-g)) * u;
+            v0 = g0 / (1.0f + __expf(-g0)) * u0;
+            v1 = g1 / (1.0f + __expf(-g1)) * u1;
+            put_operand2(xop, K, b, k, v0, v1);
         } else {
-            v = res ? res[(size_t)b * K + k] : 0.f;
-            for (uint32_t s = 0; s < S; ++s) v += part[((size_t)s * BG_MAX_BATCH + b) * Rpart + k];
+            const float2 r = *reinterpret_cast<const float2*>(res + (size_t)b * K + k);
+            v0 = r.x; v1 = r.y;
+            for (uint32_t s = 0; s < S; ++s) {
+                const float2 a = *reinterpret_cast<const float2*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + k);
+                v0 += a.x; v1 += a.y;
+            }
+            *reinterpret_cast<float2*>(xout + (size_t)b * K + k) = make_float2(v0, v1);
+            const uint32_t gg = *reinterpret_cast<const uint32_t*>(gain + k);
+            put_operand2(xop, K, b, k, v0 * bf_lo(gg), v1 * bf_hi(gg));
         }
-        if (xout) xout[(size_t)b * K + k] = v;
-        if (gain) ss += v * v;
-        else put_operand(xop, K, b, k, v);
     }
-    if (!gain) return;
+    if (swiglu) return;
+    float ss = v0 * v0 + v1 * v1;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if ((tid & 31) == 0) red[tid >> 5] = ss;
-    __syncthreads();   // also orders this block's xout stores before the re-reads below
-    float tot = 0.f;
+    __syncthreads();
+    if (tid == 0) {
+        float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
-    const float inv = rsqrtf(tot / (float)K + eps);
-    for (uint32_t k = tid; k < K; k += blockDim.x)
-        put_operand(xop, K, b, k, xout[(size_t)b * K + k] * __bfloat162float(gain[k]) * inv);
+        for (int w = 0; w < 8; ++w) tot += red[w];
+        ssq[b * BV_MAX_CHUNKS + c] = tot;
+    }
 }
 
-// Token embedding of every sequence of the batch, and the check of the whole batch: x[b] = E[token_b].
+// Token embedding of every sequence of the batch, the check of the whole batch, and the step's rotary table:
+// x[b] = E[token_b]; cs[b][i] = (cos, sin)(position_b * inv_freq[i]).  Grid (batch), 256 threads.
 __global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, const int32_t* positions, const __nv_bfloat16* embed,
-                                                         float* x, uint32_t H, uint32_t V, uint32_t max_ctx, uint32_t B, int32_t* status) {
+                                                         float* x, uint32_t H, uint32_t V, uint32_t max_ctx, const double* inv_freq,
+                                                         float* cs, uint32_t half, int32_t* status) {
     const uint32_t b = blockIdx.x, tid = threadIdx.x;
-    if (b >= B) return;
     int32_t tok = tokens[b];
     const int32_t pos = positions[b];
     if (tid == 0 && (tok < 0 || tok >= (int32_t)V || pos < 0 || pos >= (int32_t)max_ctx)) atomicCAS(status, 0, ERR_OUT_OF_RANGE);
     if (tok < 0 || tok >= (int32_t)V) tok = 0;
+    for (uint32_t i = tid; i < half; i += blockDim.x) {
+        double sn, c;
+        sincos((double)pos * inv_freq[i], &sn, &c);
+        cs[(size_t)b * 2 * half + 2 * i] = (float)c;
+        cs[(size_t)b * 2 * half + 2 * i + 1] = (float)sn;
+    }
     const __nv_bfloat16* row = embed + (size_t)tok * H;
     for (uint32_t i = tid; i < H; i += blockDim.x) x[(size_t)b * H + i] = __bfloat162float(row[i]);
 }
@@ -372,7 +399,7 @@ struct BAttnParams {
     CUtensorMap kv_map;       // the whole KV cache as [rows, head_dim] (same map as the batch-1 kernel)
     __nv_bfloat16* kv;
     const int32_t* positions;
-    const double* inv_freq;
+    const float* cs;          // [32][hd / 2][2] (cos, sin) of the step's positions
     const float* qkv_part;    // [S][32][QR] partial sums of the QKV projection
     float* q;                 // [32][QD] rotated, pre-scaled queries
     float* part_o;            // [B * nkv * Sa][G][hd]
@@ -383,47 +410,41 @@ struct BAttnParams {
     uint64_t wait_ns;
 };
 
-// RoPE and cache append for one sequence per block: sums the splits of the QKV projection, rotates q (and scales it
-// by log2(e) / sqrt(hd) for the base-2 softmax) and k at the sequence's position, rounds k and v to bf16 and writes
-// them into row `position` of the sequence's cache slabs.  The attention kernel that follows reads that row from
-// the cache like any other.
-__global__ void __launch_bounds__(256) kl_b_rope_kernel(const BAttnParams p) {
-    const uint32_t b = blockIdx.x, tid = threadIdx.x;
-    __shared__ float cs[256];   // [hd / 2][2]
-    if (*p.status != 0 || b >= p.B) return;
+// RoPE and cache append; grid (batch, n_q_heads + 2 * n_kv_heads), one head of one sequence per block of 128
+// threads: sums the splits of the QKV projection, rotates a q head (and scales it by log2(e) / sqrt(hd) for the base-2
+// softmax) or a k head at the sequence's position, rounds k and v to bf16 and writes them into row `position` of the
+// sequence's cache slabs.  The attention kernel that follows reads that row from the cache like any other.
+__global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
+    const uint32_t b = blockIdx.x, head = blockIdx.y, tid = threadIdx.x;
+    if (*p.status != 0) return;
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
-    for (uint32_t i = tid; i < half; i += blockDim.x) {
-        double sn, c;
-        sincos((double)pos * p.inv_freq[i], &sn, &c);
-        cs[2 * i] = (float)c;
-        cs[2 * i + 1] = (float)sn;
-    }
-    __syncthreads();
+    const float* cs = p.cs + (size_t)b * hd;
     auto val = [&](uint32_t r) {
         float v = 0.f;
         for (uint32_t s = 0; s < p.S; ++s) v += p.qkv_part[((size_t)s * BG_MAX_BATCH + b) * p.QR + r];
         return v;
     };
-    const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
-    for (uint32_t idx = tid; idx < p.nq * half; idx += blockDim.x) {
-        const uint32_t h = idx / half, i = idx % half;
-        const float a = val(h * hd + i), bb = val(h * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
-        p.q[(size_t)b * p.QD + h * hd + i] = (a * c - bb * sn) * qscale;
-        p.q[(size_t)b * p.QD + h * hd + i + half] = (bb * c + a * sn) * qscale;
-    }
     const size_t slab = (size_t)p.max_ctx * hd;
-    for (uint32_t idx = tid; idx < p.nkv * half; idx += blockDim.x) {
-        const uint32_t g = idx / half, i = idx % half;
-        const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+    if (head < p.nq) {
+        const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
+        for (uint32_t i = tid; i < half; i += blockDim.x) {
+            const float a = val(head * hd + i), bb = val(head * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+            p.q[(size_t)b * p.QD + head * hd + i] = (a * c - bb * sn) * qscale;
+            p.q[(size_t)b * p.QD + head * hd + i + half] = (bb * c + a * sn) * qscale;
+        }
+    } else if (head < p.nq + p.nkv) {
+        const uint32_t g = head - p.nq;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 0) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        row[i] = __float2bfloat16_rn(a * c - bb * sn);
-        row[i + half] = __float2bfloat16_rn(bb * c + a * sn);
-    }
-    for (uint32_t idx = tid; idx < p.nkv * hd; idx += blockDim.x) {
-        const uint32_t g = idx / hd, d = idx % hd;
+        for (uint32_t i = tid; i < half; i += blockDim.x) {
+            const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+            row[i] = __float2bfloat16_rn(a * c - bb * sn);
+            row[i + half] = __float2bfloat16_rn(bb * c + a * sn);
+        }
+    } else {
+        const uint32_t g = head - p.nq - p.nkv;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 1) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
+        for (uint32_t d = tid; d < hd; d += blockDim.x) row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
     }
 }
 
@@ -605,27 +626,26 @@ __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_c
 }
 
 // Merges the Sa partial results of every (sequence, kv head) and writes the attention output straight into the
-// operand of the O projection (bf16 hi and lo halves).  Grid (nkv, 32): slots b >= B get zeros.
+// operand of the O projection (bf16 hi and lo halves).  Grid (nkv, batch), 256 threads x 2 outputs.
 __global__ void __launch_bounds__(256) kl_b_attn_merge_kernel(const BAttnParams p) {
     const uint32_t g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const uint32_t G = p.G, hd = p.hd;
     if (*p.status != 0) return;
-    for (uint32_t x = tid; x < G * hd; x += blockDim.x) {
+    const size_t u0 = (size_t)(b * p.nkv + g) * p.Sa;
+    for (uint32_t x = 2 * tid; x < G * hd; x += 2 * blockDim.x) {   // hd is even: both outputs belong to head h
         const uint32_t h = x / hd, d = x % hd;
-        float v = 0.f;
-        if (b < p.B) {
-            const size_t u0 = (size_t)(b * p.nkv + g) * p.Sa;
-            float M = -INFINITY;
-            for (uint32_t s = 0; s < p.Sa; ++s) M = fmaxf(M, p.part_ml[((u0 + s) * G + h) * 2]);
-            float L = 0.f, A = 0.f;
-            for (uint32_t s = 0; s < p.Sa; ++s) {
-                const float c = rescale(p.part_ml[((u0 + s) * G + h) * 2], M);
-                L += p.part_ml[((u0 + s) * G + h) * 2 + 1] * c;
-                A += p.part_o[((u0 + s) * G + h) * hd + d] * c;
-            }
-            v = A / L;
+        float M = -INFINITY;
+        for (uint32_t s = 0; s < p.Sa; ++s) M = fmaxf(M, p.part_ml[((u0 + s) * G + h) * 2]);
+        float L = 0.f, A0 = 0.f, A1 = 0.f;
+        for (uint32_t s = 0; s < p.Sa; ++s) {
+            const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((u0 + s) * G + h) * 2);
+            const float c = rescale(ml.x, M);
+            const float2 o = *reinterpret_cast<const float2*>(p.part_o + ((u0 + s) * G + h) * hd + d);
+            L += ml.y * c;
+            A0 += o.x * c;
+            A1 += o.y * c;
         }
-        put_operand(p.xop, p.QD, b, (g * G + h) * hd + d, v);
+        put_operand2(p.xop, p.QD, b, (g * G + h) * hd + d, A0 / L, A1 / L);
     }
 }
 
