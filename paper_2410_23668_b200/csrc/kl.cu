@@ -19,6 +19,7 @@
 
 #include <mutex>
 #include <new>
+#include <utility>
 
 #include "../../include/kl.h"
 
@@ -286,7 +287,6 @@ struct kl_handle {
     CUtensorMap bmap_w[5];   // QKV, O, gate/up, down, classifier
     CUtensorMap bmap_wl[5];  // last column piece of the matrices stored in chunk order
     uint32_t bsplit[5];      // K splits of the five projections
-    uint32_t battn_splits;   // attention splits per (sequence, kv head) at the largest batch
     uint32_t last_batch;
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
@@ -314,7 +314,7 @@ struct Layout {
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
     size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
-    uint32_t bsplit[5], battn_splits;
+    uint32_t bsplit[5];
     uint32_t cps;
 };
 
@@ -351,28 +351,8 @@ static uint32_t pick_split(uint32_t R, uint32_t K, uint32_t P) {
     return best;
 }
 
-// Dynamic shared memory of kl_b_attn_kernel: alignment slack, the warps' ring slots, barriers, the queries, the warps'
-// partial results, the rescale table and the abort flag.
-static size_t batched_attn_smem(uint32_t G, uint32_t hd) {
-    return 1024 + (size_t)BA_WARPS * BA_SLOTS * SLOT_BYTES + 128 + (size_t)G * hd * 4 + (size_t)BA_WARPS * G * (hd + 2) * 4 +
-           (size_t)(BA_WARPS * MAX_G + MAX_G) * 4 + 16;
-}
-
-// Attention splits per (sequence, kv head) for a batch: the count (at most max_splits) whose units fill whole rounds
-// of one CTA per SM best, the smallest such count on a tie.
-static uint32_t pick_attn_splits(uint32_t batch, uint32_t nkv, uint32_t P, uint32_t max_splits) {
-    uint32_t best = 1;
-    double best_eff = 0.0;
-    for (uint32_t sa = 1; sa <= max_splits; ++sa) {
-        const uint32_t units = batch * nkv * sa;
-        const double eff = (double)units / (double)(((units + P - 1) / P) * P);
-        if (eff > best_eff + 0.02) {
-            best_eff = eff;
-            best = sa;
-        }
-    }
-    return best;
-}
+// Dynamic shared memory of kl_b_attn_kernel: alignment slack, the warps' ring slots, their barriers, the abort flag.
+static size_t batched_attn_smem() { return 1024 + (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES + (size_t)BA_WARPS * BA_SLOTS * 8 + 16; }
 
 Layout make_layout(const kl_model_desc& d, int num_sms) {
     Layout y;
@@ -423,15 +403,15 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
             y.bsplit[i] = i == 4 ? 1u : pick_split((uint32_t)rows[i], (uint32_t)ks[i], (uint32_t)num_sms);
             if (i < 4 && y.bsplit[i] * rows[i] > part_max) part_max = y.bsplit[i] * rows[i];
         }
-        y.battn_splits = 16;
         const bool on = B > 1;
         // one operand buffer per input width (hidden, q width, ffn), each on a 1024-byte boundary
         y.sbxop = s;  s += on ? align_up(64 * H * 2 + 1024) + align_up(64 * QD * 2 + 1024) + align_up(64 * F * 2 + 1024) : 0;
         y.sbssq = s;  s += on ? align_up((size_t)32 * BV_MAX_CHUNKS * 4) : 0;
         y.sbpart = s; s += on ? align_up(part_max * 32 * 4) : 0;
         y.sbq = s;    s += on ? align_up(32 * QD * 4) : 0;
-        y.sbao = s;   s += on ? align_up(B * d.n_kv_heads * y.battn_splits * G * d.head_dim * 4) : 0;
-        y.sbaml = s;  s += on ? align_up(B * d.n_kv_heads * y.battn_splits * G * 2 * 4) : 0;
+        const size_t aslots = B * d.n_kv_heads + (size_t)num_sms * BA_WARPS;   // attention partial results: pair + warp
+        y.sbao = s;   s += on ? align_up(aslots * G * d.head_dim * 4) : 0;
+        y.sbaml = s;  s += on ? align_up(aslots * G * 2 * 4) : 0;
     }
     y.scratch_bytes = s;
     return y;
@@ -539,6 +519,23 @@ cudaError_t store_rows(const GemvPlan& pl, __nv_bfloat16* mat, const __nv_bfloat
 }
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+// Launch with programmatic stream serialisation: the kernel may start while its predecessor in the stream still runs
+// and orders itself behind it with griddepcontrol.wait (see griddep_wait in kl_batched.cuh).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 }  // namespace
 
@@ -751,13 +748,12 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->bao = (float*)(sc + y.sbao);
     h->baml = (float*)(sc + y.sbaml);
     for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
-    h->battn_splits = y.battn_splits;
     h->use_bt = 1;
     h->bt_ok = 0;
     if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
         p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
         const uint32_t QR = p.QD + 2 * p.KVD;
-        const size_t ba_smem = batched_attn_smem(p.G, p.hd);
+        const size_t ba_smem = batched_attn_smem();
         bool ok = encode_weight_maps(h->encode_tiled, &h->bmap_w[0], &h->bmap_wl[0], p.wqkv, p.plan[PL_QKV], QR, p.L, p.layer_stride) &&
                   encode_weight_maps(h->encode_tiled, &h->bmap_w[1], &h->bmap_wl[1], p.wo, p.plan[PL_O], p.H, p.L, p.layer_stride) &&
                   encode_weight_maps(h->encode_tiled, &h->bmap_w[2], &h->bmap_wl[2], p.wgu, p.plan[PL_GU], 2 * p.F, p.L, p.layer_stride) &&
@@ -824,7 +820,7 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
 
 // The KV cache as a 2-D bf16 tensor [n_layers*2*batch*n_kv_heads*max_ctx rows, head_dim columns]; boxes of
 // [positions per chunk] x [64 columns] with the 128-byte swizzle.  Encoded per call because the cache is the caller's.
-static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch) {
+static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch, uint32_t slot_bytes = SLOT_BYTES) {
     if (!h->encode_tiled) return KL_ERR_CUDA;
     if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
     const kl_model_desc& d = h->desc;
@@ -832,7 +828,7 @@ static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d,
     if (rows > 0x7fffffffull) return KL_ERR_UNSUPPORTED_SHAPE;  // box coordinates are 32-bit signed
     const cuuint64_t gdim[2] = {d.head_dim, rows};
     const cuuint64_t gstride[1] = {(cuuint64_t)d.head_dim * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)(SLOT_BYTES / (4 * d.head_dim))};
+    const cuuint32_t box[2] = {64, (cuuint32_t)(slot_bytes / (4 * d.head_dim))};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = ((encode_tiled_fn)h->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, kv_cache_d, gdim, gstride, box,
                                                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -905,8 +901,7 @@ static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out,
     g.wait_ns = p.wait_ns;
     const uint32_t items = ceil_div(g.R, (uint32_t)BG_TILE_M) * g.S;
     const uint32_t grid = items < (uint32_t)h->num_sms ? items : (uint32_t)h->num_sms;
-    kl_bgemm_kernel<<<grid, BG_THREADS, BG_SMEM_BYTES, st>>>(g);
-    if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+    if (launch_dependent(kl_bgemm_kernel, dim3(grid), dim3(BG_THREADS), BG_SMEM_BYTES, st, g) != cudaSuccess) return KL_ERR_CUDA;
     ++h->launches;
     return KL_OK;
 }
@@ -916,7 +911,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
                                      float* logits_d, uint32_t batch, cudaStream_t st) {
     const Params& p = h->prm;
     BAttnParams a;
-    const kl_status trc = encode_kv_map(h, &a.kv_map, kv_cache_d, batch);
+    const kl_status trc = encode_kv_map(h, &a.kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
     if (trc != KL_OK) return trc;
     a.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
     a.positions = positions_d;
@@ -931,20 +926,19 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     a.QD = p.QD; a.KVD = p.KVD; a.nq = p.nq; a.nkv = p.nkv; a.G = p.G; a.hd = p.hd;
     a.B = batch;
     a.max_ctx = h->desc.max_ctx;
-    a.Sa = pick_attn_splits(batch, p.nkv, (uint32_t)h->num_sms, h->battn_splits);
+    a.NW = (uint32_t)h->num_sms * BA_WARPS;
     a.status = p.status;
     a.wait_ns = p.wait_ns;
-    const size_t ba_smem = batched_attn_smem(p.G, p.hd);
+    const size_t ba_smem = batched_attn_smem();
     cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
     kl_status rc;
-#define KL_B_CHECK()                                          \
-    do {                                                      \
-        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA; \
-        ++h->launches;                                        \
+#define KL_B_LAUNCH(kernel, grid, block, smem, ...)                                                              \
+    do {                                                                                                         \
+        if (launch_dependent(kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__) != cudaSuccess) return KL_ERR_CUDA; \
+        ++h->launches;                                                                                           \
     } while (0)
-    kl_b_embed_kernel<<<batch, 256, 0, st>>>(tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, p.inv_freq, p.rope_cs,
-                                             p.hd / 2, p.status);
-    KL_B_CHECK();
+    KL_B_LAUNCH(kl_b_embed_kernel, batch, 256, 0, tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, p.inv_freq,
+                p.rope_cs, p.hd / 2, p.status);
     if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
     const dim3 grid_h(batch, ceil_div(p.H, (uint32_t)BV_CHUNK)), grid_f(batch, ceil_div(p.F, (uint32_t)BV_CHUNK));
     uint32_t s_prev = 0;   // splits of the down projection whose sums are still to be added to the residual stream
@@ -952,35 +946,29 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
         const size_t lo = (size_t)l * p.layer_stride;
         a.layer = l;
         // x += down projection of the previous layer; operand = g1 * x, sums of squares for the RMSNorm factor
-        kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);
-        KL_B_CHECK();
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq,
+                    p.status);
         if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st)) != KL_OK) return rc;
-        kl_b_rope_kernel<<<dim3(batch, p.nq + 2 * p.nkv), 128, 0, st>>>(a);
-        KL_B_CHECK();
-        kl_b_attn_kernel<<<dim3(a.Sa, p.nkv, batch), BA_THREADS, ba_smem, st>>>(a);
-        KL_B_CHECK();
-        kl_b_attn_merge_kernel<<<dim3(p.nkv, batch), 256, 0, st>>>(a);
-        KL_B_CHECK();
+        KL_B_LAUNCH(kl_b_rope_kernel, dim3(batch, p.nq + 2 * p.nkv), 128, 0, a);
+        KL_B_LAUNCH(kl_b_attn_kernel, (uint32_t)h->num_sms, BA_THREADS, ba_smem, a);
+        KL_B_LAUNCH(kl_b_attn_merge_kernel, dim3(p.nkv, batch), 256, 0, a);
         if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st)) != KL_OK) return rc;
         // x += attention output projection; operand = g2 * x
-        kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq,
-                                                   p.status);
-        KL_B_CHECK();
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq,
+                    p.status);
         if ((rc = launch_bgemm(h, 2, l, h->bpart, batch, st)) != KL_OK) return rc;
         // operand = silu(gate) * up
-        kl_b_finish_kernel<<<grid_f, 256, 0, st>>>(h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, 1, p.F, h->bxop[2],
-                                                   nullptr, p.status);
-        KL_B_CHECK();
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_f, 256, 0, h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, 1, p.F, h->bxop[2],
+                    nullptr, p.status);
         if ((rc = launch_bgemm(h, 3, l, h->bpart, batch, st)) != KL_OK) return rc;
         s_prev = h->bsplit[3];
     }
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
     // x += last down projection (kept for kl_read_hidden); operand = gf * x; logits = RMSNorm factor * W_lm . operand
-    kl_b_finish_kernel<<<grid_h, 256, 0, st>>>(h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, 0, p.H, h->bxop[0], h->bssq, p.status);
-    KL_B_CHECK();
+    KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, 0, p.H, h->bxop[0], h->bssq, p.status);
     if ((rc = launch_bgemm(h, 4, 0, logits_d, batch, st)) != KL_OK) return rc;
     if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
-#undef KL_B_CHECK
+#undef KL_B_LAUNCH
     return KL_OK;
 }
 

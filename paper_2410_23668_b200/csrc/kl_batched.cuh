@@ -126,6 +126,14 @@ __device__ __forceinline__ void tma_tensor_5d_g2s(uint32_t dst, const void* tmap
         : "memory");
 }
 
+// Programmatic dependent launch: the kernels of a step are launched with programmatic stream serialisation, so a
+// kernel may start while its predecessor still runs.  griddep_wait() returns when the predecessor has completed and
+// its writes are visible -- everything a kernel reads from or writes to buffers shared with other kernels comes after
+// it; before it a kernel only sets itself up and prefetches data no kernel of the step writes (weights, cache rows of
+// earlier steps).  griddep_launch() lets the successor start its own set-up.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the 128-byte swizzle
 // (what TMA writes with CU_TENSOR_MAP_SWIZZLE_128B; the tile starts on a 1024-byte boundary): start address / 16 in
 // bits 0..13, leading byte offset (unused for this layout) 1 in bits 16..29, stride between groups of eight rows
@@ -201,16 +209,34 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
     const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
     const uint32_t nkb = p.nkb;
     const uint32_t nitems = ntiles * p.S;
-    const bool skip = *p.status != 0;   // an earlier kernel of this step flagged an error: the step is a no-op
+    griddep_launch();
+    bool skip = false;
+    if (!(warp == 0 && lane == 0)) {
+        griddep_wait();
+        skip = *p.status != 0;   // an earlier kernel of this step flagged an error: the step is a no-op
+    }
 
-    if (!skip && warp == 0 && lane == 0) {
-        // ---- producer: TMA loads of the weight tile and the input tile of every (row tile, K block) of this CTA's items
+    if (warp == 0 && lane == 0) {
+        // ---- producer: TMA loads of the weight tile and the input tile of every (row tile, K block) of this CTA's items.
+        // The weight tiles of the first ring round are requested before the predecessor kernel has finished (nothing
+        // writes weights); their input tiles follow once it has.
         const uint64_t pol = l2_policy_evict_first();
-        uint32_t stage = 0, use = 0;
-        for (uint32_t item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x) {
+        uint32_t stage = 0, use = 0, n = 0;
+        uint32_t xcols[BG_STAGES];
+        bool waited = false;
+        auto after_predecessor = [&]() {
+            griddep_wait();
+            waited = true;
+            skip = *p.status != 0;
+            for (uint32_t i = 0; i < n; ++i)   // n <= BG_STAGES: stage i holds iteration i
+                tma_tensor_2d_g2s(tiles + i * BG_STAGE_BYTES + BG_A_BYTES, &p.map_x, (int32_t)xcols[i], 0, smem_u32(&full[i]), pol);
+        };
+        for (uint32_t item = blockIdx.x; item < nitems && !skip && !*abort_flag; item += gridDim.x) {
             const uint32_t t = item / p.S, sp = item % p.S;
             const uint32_t kb0 = (uint32_t)(((uint64_t)sp * nkb) / p.S), kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / p.S);
-            for (uint32_t kb = kb0; kb < kb1; ++kb) {
+            for (uint32_t kb = kb0; kb < kb1; ++kb, ++n) {
+                if (!waited && n == (uint32_t)BG_STAGES) after_predecessor();
+                if (skip) break;
                 if (use > 0 && !bg_wait(smem_u32(&empty[stage]), (use - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
                 const uint32_t bar = smem_u32(&full[stage]);
                 const uint32_t dst = tiles + stage * BG_STAGE_BYTES;
@@ -228,14 +254,16 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
                     else
                         tma_tensor_4d_g2s(dst, &p.map_wl, (int32_t)cin, 0, (int32_t)unit0, (int32_t)p.layer, bar, pol);
                 }
-                tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, pol);
+                if (waited) tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, pol);
+                else xcols[stage] = xcol;
                 if (++stage == BG_STAGES) {
                     stage = 0;
                     ++use;
                 }
             }
         }
-        if (*abort_flag) {
+        if (!waited) after_predecessor();
+        if (skip || *abort_flag) {
             // no copy may still be writing this CTA's shared memory when it exits: wait (bounded) for the last copy
             // armed on every stage
             const uint64_t t0 = globaltimer_ns();
@@ -336,6 +364,8 @@ __global__ void __launch_bounds__(256) kl_b_finish_kernel(const float* part, uin
                                                           float* ssq, const int32_t* status) {
     const uint32_t b = blockIdx.x, c = blockIdx.y, tid = threadIdx.x;
     __shared__ float red[8];
+    griddep_launch();
+    griddep_wait();
     if (*status != 0) return;
     const uint32_t k = c * BV_CHUNK + 2 * tid;
     float v0 = 0.f, v1 = 0.f;
@@ -381,6 +411,8 @@ __global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, 
                                                          float* x, uint32_t H, uint32_t V, uint32_t max_ctx, const double* inv_freq,
                                                          float* cs, uint32_t half, int32_t* status) {
     const uint32_t b = blockIdx.x, tid = threadIdx.x;
+    griddep_launch();
+    griddep_wait();
     int32_t tok = tokens[b];
     const int32_t pos = positions[b];
     if (tid == 0 && (tok < 0 || tok >= (int32_t)V || pos < 0 || pos >= (int32_t)max_ctx)) atomicCAS(status, 0, ERR_OUT_OF_RANGE);
@@ -402,10 +434,10 @@ struct BAttnParams {
     const float* cs;          // [32][hd / 2][2] (cos, sin) of the step's positions
     const float* qkv_part;    // [S][32][QR] partial sums of the QKV projection
     float* q;                 // [32][QD] rotated, pre-scaled queries
-    float* part_o;            // [B * nkv * Sa][G][hd]
-    float* part_ml;           // [B * nkv * Sa][G][2]
+    float* part_o;            // [B * nkv + NW][G][hd] partial results, slot = pair + warp
+    float* part_ml;           // [B * nkv + NW][G][2]
     __nv_bfloat16* xop;       // operand of the O projection [64][QD]
-    uint32_t S, QR, QD, KVD, nq, nkv, G, hd, B, max_ctx, layer, Sa;
+    uint32_t S, QR, QD, KVD, nq, nkv, G, hd, B, max_ctx, layer, NW;   // NW: warps of the attention grid
     int32_t* status;
     uint64_t wait_ns;
 };
@@ -416,6 +448,8 @@ struct BAttnParams {
 // sequence's cache slabs.  The attention kernel that follows reads that row from the cache like any other.
 __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     const uint32_t b = blockIdx.x, head = blockIdx.y, tid = threadIdx.x;
+    griddep_launch();
+    griddep_wait();
     if (*p.status != 0) return;
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
@@ -448,199 +482,244 @@ __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     }
 }
 
-constexpr int BA_WARPS = 6;
+constexpr int BA_WARPS = 12;     // independent warps per CTA; one persistent CTA per SM
 constexpr int BA_THREADS = BA_WARPS * 32;
-constexpr int BA_SLOTS = 2;   // ring slots per warp
+constexpr int BA_SLOTS = 2;      // ring slots per warp
+constexpr int BA_SLOT_BYTES = 8192;   // K rows | V rows of 16 (head size 128) or 32 (head size 64) cached positions
 
-// Split-K flash-decoding over (split, kv head, sequence) units.  Every warp streams its own chunks of 32 (head size
-// 128) or 64 (head size 64) cached positions through a two-slot ring of its own (lane 0 issues the TMA box loads two
-// chunks ahead) and runs the mma.sync tiles of kl_attention_tc.cuh on them; the warps' results are merged in shared
-// memory and written as the unit's partial result (O^T unnormalised, running maximum, sum).
+// Chunks of cached positions a sequence at position `pos` holds after this step's append (pb positions per chunk).
+__device__ __forceinline__ uint32_t ba_chunks(int32_t pos, uint32_t pb) { return ((uint32_t)pos + 1u + pb - 1u) / pb; }
+
+// First chunk of warp w when W chunks are dealt in contiguous, equally long ranges to NW warps.
+__device__ __forceinline__ uint32_t ba_range_lo(uint32_t w, uint32_t W, uint32_t NW) { return (uint32_t)(((uint64_t)w * W) / NW); }
+
+// Walks the chunk list of the step: (sequence b, kv head g, chunk c of the sequence's nch chunks), in that order.
+struct BaCursor {
+    uint32_t b, g, c, nch;
+};
+
+// Attention of a batch as ONE balanced stream.  The chunks (16 or 32 cached positions of one kv head of one sequence:
+// an 8 KB K|V tile pair) of all (sequence, kv head) pairs form one list; every warp of the persistent grid takes a
+// contiguous range of W / NW chunks of it, streams them through a two-slot TMA ring of its own (loads run two chunks
+// ahead, across pair boundaries) and runs the mma.sync tiles of kl_attention_tc.cuh on them.  Whenever its range
+// leaves a pair the warp writes its flash-decoding partial result for that pair (O^T unnormalised, running maximum,
+// sum) to slot (pair + warp) -- unique, because along the list either the pair or the warp advances from one segment
+// to the next.  kl_b_attn_merge_kernel combines the segments of every pair.  No warp waits for another one, every
+// warp streams the same number of bytes (+- one chunk), and a sequence's length only decides how many warps share it.
 template <int HD, bool PACK>
-__device__ __forceinline__ void b_attn_unit(const BAttnParams& p, uint8_t* smem_raw) {
-    const uint32_t sp = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+__device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* smem_raw) {
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t G = p.G;
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t ring = (raw + 1023u) & ~1023u;
-    uint8_t* after = smem_raw + (ring - raw) + (size_t)BA_WARPS * BA_SLOTS * SLOT_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(after);                          // [BA_WARPS * BA_SLOTS]
-    float* q_s = reinterpret_cast<float*>(after + 128);                           // [G][HD]
-    float* comb = q_s + G * HD;                                                   // [BA_WARPS][G][HD + 2]
-    float* ftab = comb + (size_t)BA_WARPS * G * (HD + 2);                         // [BA_WARPS][G] + [G]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(ftab + BA_WARPS * MAX_G + MAX_G);
+    const uint32_t ring = ((raw + 1023u) & ~1023u) + warp * BA_SLOTS * BA_SLOT_BYTES;   // this warp's slots
+    uint8_t* after = smem_raw + (((raw + 1023u) & ~1023u) - raw) + (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(after) + warp * BA_SLOTS;        // [BA_WARPS][BA_SLOTS]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(after + BA_WARPS * BA_SLOTS * 8);
 
-    if (tid == 0) {
-        for (int i = 0; i < BA_WARPS * BA_SLOTS; ++i) mbar_init(smem_u32(&full[i]), 1);
-        *abort_flag = 0;
+    if (tid == 0) *abort_flag = 0;
+    if (lane == 0) {
+        for (int i = 0; i < BA_SLOTS; ++i) mbar_init(smem_u32(&full[i]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    for (uint32_t i = tid; i < G * HD; i += blockDim.x) q_s[i] = p.q[(size_t)b * p.QD + (size_t)g * G * HD + i];
     __syncthreads();
 
-    // positions of this unit: split sp of 0 .. position (the row appended by this step included)
-    const uint32_t n = (uint32_t)p.positions[b] + 1u;
-    const uint32_t clen = (n + p.Sa - 1) / p.Sa;
-    const uint32_t c0 = min(n, sp * clen), cend = min(n, c0 + clen);
-    const uint32_t pb = SLOT_BYTES / (4u * HD);
-    const uint32_t nring = (cend - c0 + pb - 1) / pb;
-    const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
-    const uint32_t row0 = p.layer * 2u * vdelta + (b * p.nkv + g) * p.max_ctx;
-    const uint32_t box_bytes = pb * 128u;
-    const uint64_t pol = l2_policy_evict_first();
-
-    auto issue = [&](uint32_t i, uint32_t slot) {   // lane 0: chunk i of the unit into this warp's slot
-        const AttnWindow w = attn_window(c0, cend, pb, i);
-        const uint32_t bar = smem_u32(&full[warp * BA_SLOTS + slot]);
-        const uint32_t dst = ring + (warp * BA_SLOTS + slot) * SLOT_BYTES;
-        mbar_arrive_expect_tx(bar, (uint32_t)SLOT_BYTES);
+    constexpr uint32_t pb = BA_SLOT_BYTES / (4u * HD);
+    constexpr uint32_t box_bytes = pb * 128u;
+    // lane b keeps the chunk count of sequence b; W = chunks of the whole step
+    const uint32_t my_nch = lane < p.B ? ba_chunks(p.positions[lane], pb) : 0u;
+    uint32_t W = my_nch;
 #pragma unroll
-        for (uint32_t bx = 0; bx < HD / 64u; ++bx) {
-            tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + w.w0), bar, pol);
-            tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + w.w0 + vdelta), bar, pol);
+    for (int o = 16; o > 0; o >>= 1) W += __shfl_xor_sync(0xffffffffu, W, o);
+    W *= p.nkv;
+    const uint32_t NW = min(p.NW, W), gw = blockIdx.x * BA_WARPS + warp;   // at least one chunk per working warp
+    if (gw >= NW) return;
+    const uint32_t lo = ba_range_lo(gw, W, NW), hi = ba_range_lo(gw + 1, W, NW);
+
+    // cursor at chunk `lo`
+    BaCursor cur = {0u, 0u, 0u, __shfl_sync(0xffffffffu, my_nch, 0)};
+    {
+        uint32_t skip = lo;
+        while (skip >= cur.nch * p.nkv) {   // whole sequences before the range (sequences have at least one chunk)
+            skip -= cur.nch * p.nkv;
+            ++cur.b;
+            cur.nch = __shfl_sync(0xffffffffu, my_nch, cur.b & 31u);
+        }
+        cur.g = skip / cur.nch;
+        cur.c = skip % cur.nch;
+    }
+    auto advance = [&](BaCursor& x) {   // warp-uniform
+        if (++x.c == x.nch) {
+            x.c = 0;
+            if (++x.g == p.nkv) {
+                x.g = 0;
+                ++x.b;
+                x.nch = __shfl_sync(0xffffffffu, my_nch, x.b & 31u);
+            }
         }
     };
-    if (lane == 0) {
-        if (warp < nring) issue(warp, 0);
-        if (warp + BA_WARPS < nring) issue(warp + BA_WARPS, 1);
+    const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
+    const uint64_t pol = l2_policy_evict_first();
+    auto issue = [&](const BaCursor& x, uint32_t slot) {   // lane 0: the chunk under cursor x into this warp's slot
+        const uint32_t n = (uint32_t)p.positions[x.b] + 1u;
+        const AttnWindow w = attn_window(0u, n, pb, x.c);
+        const uint32_t row0 = p.layer * 2u * vdelta + (x.b * p.nkv + x.g) * p.max_ctx + w.w0;
+        const uint32_t bar = smem_u32(&full[slot]);
+        const uint32_t dst = ring + slot * BA_SLOT_BYTES;
+        mbar_arrive_expect_tx(bar, (uint32_t)BA_SLOT_BYTES);
+#pragma unroll
+        for (uint32_t bx = 0; bx < HD / 64u; ++bx) {
+            tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)row0, bar, pol);
+            tma_tensor_2d_g2s(dst + BA_SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + vdelta), bar, pol);
+        }
+    };
+
+    // the first chunks of the range go out before anything else
+    BaCursor nxt = cur;   // cursor of the next chunk to request
+    uint32_t issued = 0;
+    for (; issued < (uint32_t)BA_SLOTS && lo + issued < hi; ++issued) {
+        if (lane == 0) issue(nxt, issued);
+        advance(nxt);
     }
 
     constexpr int NKB = HD / 16, NMT = HD / 16;
     const uint32_t gq = lane >> 2, t = lane & 3u;
     AttnTcState<HD> st;
+    auto begin_pair = [&](const BaCursor& x) {   // Q fragments of the pair's heads, empty accumulators
+        const float* q = p.q + (size_t)x.b * p.QD + (size_t)x.g * G * HD;
 #pragma unroll
-    for (int kb = 0; kb < NKB; ++kb) {
+        for (int kb = 0; kb < NKB; ++kb) {
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const uint32_t k = kb * 16 + hf * 8 + 2 * t;
-            const uint32_t head = PACK ? (gq & 3u) : gq;
-            float2 xx = make_float2(0.f, 0.f);
-            if (head < G) xx = *reinterpret_cast<const float2*>(q_s + head * HD + k);
-            const uint32_t hi = pack_bf16(xx.x, xx.y);
-            const uint32_t lo = pack_bf16(xx.x - bf_lo(hi), xx.y - bf_hi(hi));
-            st.qh[kb][hf] = (PACK && gq >= 4u) ? lo : hi;
-            st.ql[kb][hf] = lo;
+            for (int hf = 0; hf < 2; ++hf) {
+                const uint32_t k = kb * 16 + hf * 8 + 2 * t;
+                const uint32_t head = PACK ? (gq & 3u) : gq;   // PACK: column gq = hi (gq < 4) or lo half of head gq % 4
+                float2 xx = make_float2(0.f, 0.f);
+                if (head < G) xx = *reinterpret_cast<const float2*>(q + head * HD + k);
+                const uint32_t qhi = pack_bf16(xx.x, xx.y);
+                const uint32_t qlo = pack_bf16(xx.x - bf_lo(qhi), xx.y - bf_hi(qhi));
+                st.qh[kb][hf] = (PACK && gq >= 4u) ? qlo : qhi;
+                st.ql[kb][hf] = qlo;
+            }
         }
-    }
 #pragma unroll
-    for (int nn = 0; nn < NMT; ++nn) st.o[nn][0] = st.o[nn][1] = st.o[nn][2] = st.o[nn][3] = 0.f;
-    st.m[0] = st.m[1] = -INFINITY;
-    st.l[0] = st.l[1] = 0.f;
+        for (int nn = 0; nn < NMT; ++nn) st.o[nn][0] = st.o[nn][1] = st.o[nn][2] = st.o[nn][3] = 0.f;
+        st.m[0] = st.m[1] = -INFINITY;
+        st.l[0] = st.l[1] = 0.f;
+    };
+    auto end_pair = [&](const BaCursor& x) {   // this warp's partial result of the pair to slot (pair + warp)
+        float l0 = st.l[0], l1 = st.l[1];
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {   // the lanes that share the heads (same lane % 4) hold parts of the row sums
+            l0 += __shfl_xor_sync(0xffffffffu, l0, o);
+            l1 += __shfl_xor_sync(0xffffffffu, l1, o);
+        }
+        if (PACK) {   // columns 0..3 hold the hi parts of O^T, columns 4..7 the lo parts: lanes t and t ^ 2 of a quad
+#pragma unroll
+            for (int nn = 0; nn < NMT; ++nn)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) st.o[nn][j] += __shfl_xor_sync(0xffffffffu, st.o[nn][j], 2);
+        }
+        const size_t slot = (size_t)(x.b * p.nkv + x.g) + gw;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const uint32_t h = 2 * t + hh;
+            if (h < G && (!PACK || t < 2u)) {
+                float* dst = p.part_o + (slot * G + h) * HD;
+#pragma unroll
+                for (int nn = 0; nn < NMT; ++nn) {
+                    dst[nn * 16 + gq] = st.o[nn][hh];
+                    dst[nn * 16 + gq + 8] = st.o[nn][2 + hh];
+                }
+                if (gq == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + h) * 2) = make_float2(st.m[hh], hh ? l1 : l0);
+            }
+        }
+    };
 
-    // chunk c of this warp (c = 0, 1, ...) sits in slot c % BA_SLOTS and completes phase (c / BA_SLOTS) % 2 of its barrier
-    uint32_t consumed = 0;
-    uint32_t issued = (warp < nring ? 1u : 0u) + (warp + BA_WARPS < nring ? 1u : 0u);
-    for (uint32_t i = warp; i < nring; i += BA_WARPS, ++consumed) {
-        const uint32_t slot = consumed % BA_SLOTS, phase = (consumed / BA_SLOTS) & 1u;
-        if (!bg_wait(smem_u32(&full[warp * BA_SLOTS + slot]), phase, p.status, p.wait_ns, abort_flag)) break;
-        const uint32_t kbase = ring + (warp * BA_SLOTS + slot) * SLOT_BYTES;
-        const AttnWindow w = attn_window(c0, cend, pb, i);
+    begin_pair(cur);
+    uint32_t k = lo;
+    for (; k < hi; ++k) {
+        const uint32_t slot = (k - lo) % BA_SLOTS, phase = ((k - lo) / BA_SLOTS) & 1u;
+        if (!bg_wait(smem_u32(&full[slot]), phase, p.status, p.wait_ns, abort_flag)) break;
+        const uint32_t kbase = ring + slot * BA_SLOT_BYTES;
+        const AttnWindow w = attn_window(0u, (uint32_t)p.positions[cur.b] + 1u, pb, cur.c);
+#pragma unroll
         for (uint32_t r0 = 0; r0 < pb; r0 += 16)
-            if (r0 + 16 > w.lo && r0 < w.hi) attn_tc_tile<HD, PACK>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, r0, w.lo, w.hi, lane);
+            if (r0 + 16 > w.lo && r0 < w.hi) attn_tc_tile<HD, PACK>(st, kbase, kbase + BA_SLOT_BYTES / 2, box_bytes, r0, w.lo, w.hi, lane);
         __syncwarp();
-        if (i + BA_SLOTS * BA_WARPS < nring) {
+        if (lo + issued < hi) {   // refill the slot just read
             if (lane == 0) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the slot was read through the generic proxy
-                issue(i + BA_SLOTS * BA_WARPS, slot);
+                issue(nxt, slot);
             }
+            advance(nxt);
             ++issued;
         }
+        const BaCursor done = cur;
+        advance(cur);
+        if (k + 1 == hi || cur.c == 0) {   // the pair ends here for this warp
+            end_pair(done);
+            if (k + 1 < hi) begin_pair(cur);
+        }
     }
-    // after a time-out copies may still be in flight: wait (bounded) for every chunk issued but not consumed
-    if (consumed < issued && lane == 0) {
+    // after a time-out copies may still be in flight: wait (bounded) for every chunk requested but not consumed
+    if (k < hi && lane == 0) {
         const uint64_t t0 = globaltimer_ns();
-        for (uint32_t c = consumed; c < issued; ++c)
-            while (!mbar_try_wait(smem_u32(&full[warp * BA_SLOTS + c % BA_SLOTS]), (c / BA_SLOTS) & 1u))
+        for (uint32_t c = k - lo; c < issued; ++c)
+            while (!mbar_try_wait(smem_u32(&full[c % BA_SLOTS]), (c / BA_SLOTS) & 1u))
                 if (globaltimer_ns() - t0 > p.wait_ns) break;
-    }
-
-    // this warp's result into shared memory (same layout as the batch-1 kernel)
-    float l0 = st.l[0], l1 = st.l[1];
-#pragma unroll
-    for (int o = 4; o < 32; o <<= 1) {
-        l0 += __shfl_xor_sync(0xffffffffu, l0, o);
-        l1 += __shfl_xor_sync(0xffffffffu, l1, o);
-    }
-    if (PACK) {
-#pragma unroll
-        for (int nn = 0; nn < NMT; ++nn)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) st.o[nn][j] += __shfl_xor_sync(0xffffffffu, st.o[nn][j], 2);
-    }
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
-        const uint32_t h = 2 * t + hh;
-        if (h < G && (!PACK || t < 2u)) {
-            float* dst = comb + ((size_t)warp * G + h) * (HD + 2);
-#pragma unroll
-            for (int nn = 0; nn < NMT; ++nn) {
-                dst[nn * 16 + gq] = st.o[nn][hh];
-                dst[nn * 16 + gq + 8] = st.o[nn][2 + hh];
-            }
-            if (gq == 0) {
-                dst[HD] = st.m[hh];
-                dst[HD + 1] = hh ? l1 : l0;
-            }
-        }
-    }
-    __syncthreads();
-    if (tid < BA_WARPS * G) {
-        const uint32_t w = tid / G, h = tid % G;
-        float Mh = -INFINITY;
-#pragma unroll
-        for (int ww = 0; ww < BA_WARPS; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (HD + 2) + HD]);
-        ftab[w * G + h] = rescale(comb[((size_t)w * G + h) * (HD + 2) + HD], Mh);
-        if (w == 0) ftab[BA_WARPS * G + h] = Mh;
-    }
-    __syncthreads();
-    const uint32_t unit = (b * p.nkv + g) * p.Sa + sp;
-    for (uint32_t x = tid; x < G * HD; x += blockDim.x) {
-        const uint32_t h = x / HD, d = x % HD;
-        float A = 0.f, Ls = 0.f;
-#pragma unroll
-        for (int w = 0; w < BA_WARPS; ++w) {
-            const float* src = comb + ((size_t)w * G + h) * (HD + 2);
-            const float c = ftab[w * G + h];
-            A += src[d] * c;
-            Ls += src[HD + 1] * c;
-        }
-        p.part_o[((size_t)unit * G + h) * HD + d] = A;
-        if (d == 0) {
-            p.part_ml[((size_t)unit * G + h) * 2] = ftab[BA_WARPS * G + h];
-            p.part_ml[((size_t)unit * G + h) * 2 + 1] = Ls;
-        }
     }
 }
 
 __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_constant__ BAttnParams p) {
     extern __shared__ uint8_t ba_smem_raw[];
+    griddep_launch();
+    griddep_wait();
     if (*p.status != 0) return;
     if (p.hd == 128) {
-        if (p.G <= 4) b_attn_unit<128, true>(p, ba_smem_raw);
-        else b_attn_unit<128, false>(p, ba_smem_raw);
+        if (p.G <= 4) b_attn_stream<128, true>(p, ba_smem_raw);
+        else b_attn_stream<128, false>(p, ba_smem_raw);
     } else {
-        if (p.G <= 4) b_attn_unit<64, true>(p, ba_smem_raw);
-        else b_attn_unit<64, false>(p, ba_smem_raw);
+        if (p.G <= 4) b_attn_stream<64, true>(p, ba_smem_raw);
+        else b_attn_stream<64, false>(p, ba_smem_raw);
     }
 }
 
-// Merges the Sa partial results of every (sequence, kv head) and writes the attention output straight into the
-// operand of the O projection (bf16 hi and lo halves).  Grid (nkv, batch), 256 threads x 2 outputs.
+// Combines the segments of every (sequence, kv head) pair and writes the attention output straight into the operand
+// of the O projection (bf16 hi and lo halves).  The pair's chunks [first, first + nch) were processed by the warps
+// whose ranges meet them; warp w left its part in slot (pair + w).  Grid (nkv, batch), 256 threads x 2 outputs.
 __global__ void __launch_bounds__(256) kl_b_attn_merge_kernel(const BAttnParams p) {
     const uint32_t g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     const uint32_t G = p.G, hd = p.hd;
+    griddep_launch();
+    griddep_wait();
     if (*p.status != 0) return;
-    const size_t u0 = (size_t)(b * p.nkv + g) * p.Sa;
+    __shared__ uint32_t seg[2];
+    if (tid == 0) {
+        const uint32_t pb = BA_SLOT_BYTES / (4u * hd);
+        uint32_t W = 0, first = 0;
+        for (uint32_t bb = 0; bb < p.B; ++bb) {
+            const uint32_t n = ba_chunks(p.positions[bb], pb) * p.nkv;
+            if (bb < b) first += n;
+            W += n;
+        }
+        const uint32_t nch = ba_chunks(p.positions[b], pb), NW = min(p.NW, W);
+        first += g * nch;
+        // the warp whose range holds chunk x: floor(((x + 1) * NW - 1) / W)  (every range holds at least one chunk)
+        seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
+        seg[1] = (uint32_t)((((uint64_t)first + nch) * NW - 1u) / W);
+    }
+    __syncthreads();
+    const uint32_t w_first = seg[0], w_last = seg[1];
+    const size_t pair = (size_t)b * p.nkv + g;
     for (uint32_t x = 2 * tid; x < G * hd; x += 2 * blockDim.x) {   // hd is even: both outputs belong to head h
         const uint32_t h = x / hd, d = x % hd;
         float M = -INFINITY;
-        for (uint32_t s = 0; s < p.Sa; ++s) M = fmaxf(M, p.part_ml[((u0 + s) * G + h) * 2]);
+        for (uint32_t w = w_first; w <= w_last; ++w) M = fmaxf(M, p.part_ml[((pair + w) * G + h) * 2]);
         float L = 0.f, A0 = 0.f, A1 = 0.f;
-        for (uint32_t s = 0; s < p.Sa; ++s) {
-            const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((u0 + s) * G + h) * 2);
+        for (uint32_t w = w_first; w <= w_last; ++w) {
+            const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((pair + w) * G + h) * 2);
             const float c = rescale(ml.x, M);
-            const float2 o = *reinterpret_cast<const float2*>(p.part_o + ((u0 + s) * G + h) * hd + d);
+            const float2 o = *reinterpret_cast<const float2*>(p.part_o + ((pair + w) * G + h) * hd + d);
             L += ml.y * c;
             A0 += o.x * c;
             A1 += o.y * c;
