@@ -276,6 +276,7 @@ struct kl_handle {
     // batched (tensor-core) path
     int bt_ok;             // 1: available for this shape
     int use_bt;            // 1 (default): batches take it; 0: sequence after sequence on the batch-1 kernels
+    int use_stream;        // 1 (default): stream schedule for the projections of the layers; 0: (row tile, K split) items
     float* bx;             // [32][H] hidden states of the batch (== hidden_all)
     __nv_bfloat16* bxop[3];   // operands [64][H], [64][QD], [64][F]: rows 0..31 hi halves, 32..63 lo halves
     float* bssq;           // [32][BV_MAX_CHUNKS] partial sums of squares of the residual stream
@@ -407,6 +408,9 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
         // one operand buffer per input width (hidden, q width, ffn), each on a 1024-byte boundary
         y.sbxop = s;  s += on ? align_up(64 * H * 2 + 1024) + align_up(64 * QD * 2 + 1024) + align_up(64 * F * 2 + 1024) : 0;
         y.sbssq = s;  s += on ? align_up((size_t)32 * BV_MAX_CHUNKS * 4) : 0;
+        // stream schedule: one partial tile [32][128] per (row tile + CTA)
+        const size_t stream_max = (ceil_div((uint32_t)(2 * F > QR ? 2 * F : QR), 128u) + (size_t)num_sms) * 128;
+        if (stream_max > part_max) part_max = stream_max;
         y.sbpart = s; s += on ? align_up(part_max * 32 * 4) : 0;
         y.sbq = s;    s += on ? align_up(32 * QD * 4) : 0;
         const size_t aslots = B * d.n_kv_heads + (size_t)num_sms * BA_WARPS;   // attention partial results: pair + warp
@@ -749,6 +753,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->baml = (float*)(sc + y.sbaml);
     for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
     h->use_bt = 1;
+    h->use_stream = 1;
     h->bt_ok = 0;
     if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
         p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
@@ -867,7 +872,8 @@ static kl_status launch_persistent(kl_handle* h, const void* func, void** args, 
 }
 
 // One projection of the batched path: out[s][b][r] = partial sums over K split s of W[idx](layer) . operand.
-static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out, uint32_t batch, cudaStream_t st) {
+static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out, uint32_t batch, cudaStream_t st,
+                              BgPartials* parts = nullptr) {
     const Params& p = h->prm;
     static const int plan_of[5] = {PL_QKV, PL_O, PL_GU, PL_D, PL_LM};
     static const int xmap_of[5] = {0, 1, 0, 2, 0};
@@ -899,8 +905,21 @@ static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out,
     g.eps = p.eps;
     g.status = p.status;
     g.wait_ns = p.wait_ns;
-    const uint32_t items = ceil_div(g.R, (uint32_t)BG_TILE_M) * g.S;
+    // the projections of the layers run on the stream schedule (every CTA the same share of the K blocks of all
+    // tiles); the classifier writes its result directly and keeps whole tiles
+    const uint32_t ntiles = ceil_div(g.R, (uint32_t)BG_TILE_M), T = ntiles * g.nkb;
+    g.stream = (idx != 4 && h->use_stream && T >= (uint32_t)h->num_sms) ? 1u : 0u;
+    const uint32_t items = g.stream ? T : ntiles * g.S;
     const uint32_t grid = items < (uint32_t)h->num_sms ? items : (uint32_t)h->num_sms;
+    if (parts) {
+        parts->part = out;
+        parts->R = g.R;
+        parts->S = g.S;
+        parts->stream = g.stream;
+        parts->nkb = g.nkb;
+        parts->T = T;
+        parts->P = grid;
+    }
     if (launch_dependent(kl_bgemm_kernel, dim3(grid), dim3(BG_THREADS), BG_SMEM_BYTES, st, g) != cudaSuccess) return KL_ERR_CUDA;
     ++h->launches;
     return KL_OK;
@@ -916,14 +935,12 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     a.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
     a.positions = positions_d;
     a.cs = p.rope_cs;
-    a.qkv_part = h->bpart;
     a.q = h->bq;
     a.part_o = h->bao;
     a.part_ml = h->baml;
     a.xop = h->bxop[1];
-    a.S = h->bsplit[0];
-    a.QR = p.QD + 2 * p.KVD;
     a.QD = p.QD; a.KVD = p.KVD; a.nq = p.nq; a.nkv = p.nkv; a.G = p.G; a.hd = p.hd;
+    BgPartials parts = {};   // of the latest projection; part == nullptr: nothing to add
     a.B = batch;
     a.max_ctx = h->desc.max_ctx;
     a.NW = (uint32_t)h->num_sms * BA_WARPS;
@@ -941,31 +958,26 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
                 p.rope_cs, p.hd / 2, p.status);
     if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
     const dim3 grid_h(batch, ceil_div(p.H, (uint32_t)BV_CHUNK)), grid_f(batch, ceil_div(p.F, (uint32_t)BV_CHUNK));
-    uint32_t s_prev = 0;   // splits of the down projection whose sums are still to be added to the residual stream
     for (uint32_t l = 0; l < p.L; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         a.layer = l;
         // x += down projection of the previous layer; operand = g1 * x, sums of squares for the RMSNorm factor
-        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, s_prev, p.H, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq,
-                    p.status);
-        if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st)) != KL_OK) return rc;
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, parts, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);
+        if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st, &a.qkv)) != KL_OK) return rc;
         KL_B_LAUNCH(kl_b_rope_kernel, dim3(batch, p.nq + 2 * p.nkv), 128, 0, a);
         KL_B_LAUNCH(kl_b_attn_kernel, (uint32_t)h->num_sms, BA_THREADS, ba_smem, a);
         KL_B_LAUNCH(kl_b_attn_merge_kernel, dim3(p.nkv, batch), 256, 0, a);
-        if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st)) != KL_OK) return rc;
+        if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st, &parts)) != KL_OK) return rc;
         // x += attention output projection; operand = g2 * x
-        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, h->bsplit[1], p.H, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq,
-                    p.status);
-        if ((rc = launch_bgemm(h, 2, l, h->bpart, batch, st)) != KL_OK) return rc;
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, parts, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);
+        if ((rc = launch_bgemm(h, 2, l, h->bpart, batch, st, &parts)) != KL_OK) return rc;
         // operand = silu(gate) * up
-        KL_B_LAUNCH(kl_b_finish_kernel, grid_f, 256, 0, h->bpart, h->bsplit[2], 2 * p.F, nullptr, nullptr, nullptr, 1, p.F, h->bxop[2],
-                    nullptr, p.status);
-        if ((rc = launch_bgemm(h, 3, l, h->bpart, batch, st)) != KL_OK) return rc;
-        s_prev = h->bsplit[3];
+        KL_B_LAUNCH(kl_b_finish_kernel, grid_f, 256, 0, parts, nullptr, nullptr, nullptr, 1, p.F, h->bxop[2], nullptr, p.status);
+        if ((rc = launch_bgemm(h, 3, l, h->bpart, batch, st, &parts)) != KL_OK) return rc;
     }
     if (ev && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;
     // x += last down projection (kept for kl_read_hidden); operand = gf * x; logits = RMSNorm factor * W_lm . operand
-    KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, h->bpart, s_prev, p.H, h->bx, h->bx, p.gf, 0, p.H, h->bxop[0], h->bssq, p.status);
+    KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, parts, h->bx, h->bx, p.gf, 0, p.H, h->bxop[0], h->bssq, p.status);
     if ((rc = launch_bgemm(h, 4, 0, logits_d, batch, st)) != KL_OK) return rc;
     if (ev && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
 #undef KL_B_LAUNCH

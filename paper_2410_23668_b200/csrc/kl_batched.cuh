@@ -3,25 +3,36 @@
 // sequences (the paper's Table 1: ~20 FLOP/B at batch 32 -- still far below the ridge, i.e. HBM-bound, which is why the
 // tiling is chosen for streaming and balance, not for tensor throughput).
 //
-// One projection = kl_bgemm_kernel:  part[s][b][r] = sum over the K blocks of split s of W[r, k] * x[b, k].
+// One projection = kl_bgemm_kernel:  result[b][r] = sum_k W[r, k] * x[b, k], left as partial results.
 //   * M = 128 weight rows per tile; the inputs enter as the N operand split into bf16 hi and lo halves that sit in
 //     columns 0..31 and 32..63 of ONE N = 64 operand: a single MMA per 16 columns of K yields W.x_hi and W.x_lo side by
 //     side and the epilogue adds them (fp32-accurate inputs on a bf16 tensor pipe).
-//   * Work items are (row tile, K split); 148 persistent CTAs take items round-robin.  The split count is chosen on the
-//     host so that the items balance over the SMs; the partial sums of the splits are added, in split order, by the
-//     kernel that consumes them (kl_b_finish_kernel / kl_b_rope_kernel) -- no atomics, the result is reproducible.
+//   * Schedule (see BgIter): the K blocks (64 columns) of all row tiles form one list and each of the 148 persistent
+//     CTAs takes a contiguous, equally long range of it, so every CTA streams the same number of bytes whatever the
+//     tile count; a tile cut by a range boundary is left as partial tiles, one per CTA that shares it.  Small
+//     projections (fewer blocks than CTAs) and the classifier use whole (row tile, K split) items instead.  The
+//     partial results are added, in a fixed order, by the kernel that consumes them (kl_b_finish_kernel /
+//     kl_b_rope_kernel) -- no floating-point atomics, the result is reproducible.
+//   * The RMSNorm factor is applied behind the contraction (W.(g*x) * rsqrt(mean x^2 + eps)): the operand holds
+//     g * x, the epilogue scales column b by the factor of sequence b, so no kernel waits for a whole-vector reduction.
 //   * Per 64 columns of K one ring stage holds a [128 x 64] weight tile (16 KB) and the [64 x 64] input tile (8 KB),
 //     written by TMA with the 128-byte swizzle the MMA's shared-memory descriptors expect.  Row-major matrices are read
-//     through a 3-D tensor (column, row, layer); the down projection, which is stored in chunk order for the batch-1
-//     kernel (unit of rpc rows x column piece), through a 5-D tensor (column, row in unit, piece, unit, layer) plus a
-//     4-D one for its shorter last piece.
+//     through a 3-D tensor (column, row, layer); matrices stored in chunk order for the batch-1 kernel (unit of rpc
+//     rows x column piece) through a 5-D tensor (column, row in unit, piece, unit, layer) plus a 4-D one for the
+//     shorter last piece.
 //   * Roles (192 threads): warp 0 lane 0 issues the TMA loads, warp 1 owns TMEM and its lane 0 issues tcgen05.mma and
 //     the commits, warps 2..5 read the accumulators (tcgen05.ld) and store.  Two accumulator buffers overlap the
-//     epilogue of one item with the MMAs of the next.  Every mbarrier wait is bounded.
+//     epilogue of one segment with the MMAs of the next.  Every mbarrier wait is bounded.
+//   * The kernels of a step are launched with programmatic stream serialisation: a projection requests the weight
+//     tiles of its first ring round while its predecessor still runs (see griddep_wait).
 //
-// Between the projections small kernels do the per-sequence vector work (sum of the splits, residual, RMSNorm, SwiGLU,
-// RoPE, cache append) and write the next projection's bf16 operand; attention is a split-K flash-decoding kernel over
-// (sequence, kv head, split) units with the same mma.sync tiles as the batch-1 kernel.
+// Between the projections small kernels, spread over (sequence, chunk) blocks, do the vector work (sum of the partial
+// results, residual, gain and sums of squares for the RMSNorm, SwiGLU, RoPE, cache append) and write the next
+// projection's bf16 operand.  Doing this work in the projection's epilogue instead (the CTA that completes a tile,
+// found by a ticket, finishes it) was measured and is slower: fence, ticket, re-read and store form a latency chain
+// of ~10 us per tile on four warps, more than a separate kernel over hundreds of blocks costs.
+// Attention is one balanced stream of K|V chunks over a persistent grid (kl_b_attn_kernel) followed by a merge per
+// (sequence, kv head) that writes the operand of the O projection.
 #pragma once
 
 namespace kl {
@@ -42,8 +53,10 @@ struct BgemmParams {
     CUtensorMap map_w;     // weights: rank 3 (column, row, layer) or, for chunk-ordered matrices, rank 5
     CUtensorMap map_wl;    // chunk-ordered matrices: the last (shorter) column piece, rank 4 (column, row in unit, unit, layer)
     CUtensorMap map_x;     // inputs [64 rows, K] bf16: rows 0..31 hi halves, 32..63 lo halves
-    float* out;            // [S][32][R] partial sums (S = 1: the result itself)
+    float* out;            // tile schedule: [S][32][R] partial sums (S = 1: the result itself);
+                           // stream schedule: [row tiles + CTAs][32][128] partial tiles, slot = tile + CTA
     uint32_t R, K, B, S, layer;
+    uint32_t stream;       // 0: tile schedule, items (row tile, K split) dealt round-robin; 1: stream schedule, see BgIter
     uint32_t nkb;          // K blocks of 64 columns in all (a block may reach past the end of K or of a piece: TMA fills zeros)
     uint32_t pieces;       // 0: row-major weights; otherwise the number of column pieces of the chunk order
     uint32_t kp;           // columns per full piece
@@ -153,6 +166,95 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(uint32_t M, uint32_t N) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((N >> 3) << 17) | ((M >> 4) << 24);
 }
 
+// The work of one CTA as a list of segments (row tile t, K blocks [kb0, kb1), partial-result slot).
+//   tile schedule:   items (t, split) dealt round-robin; slot = split.
+//   stream schedule: the K blocks of all tiles form one list of T = tiles * nkb blocks; CTA c takes the contiguous range
+//                    [c * T / P, (c + 1) * T / P) of it, so every CTA streams the same number of bytes (+- one block of
+//                    24 KB) whatever the tile count.  A tile cut by a range boundary is finished by the consumer
+//                    kernel, which adds up the partial tiles of the CTAs that share it (slot = tile + CTA is unique,
+//                    because along the list either the tile or the CTA advances from one segment to the next).
+struct BgSeg {
+    uint32_t t, kb0, kb1, slot;
+};
+struct BgIter {
+    uint32_t stream, nkb, S, nitems, item;   // tile schedule
+    uint32_t g0, g1;                         // stream schedule: blocks of the list still to do
+    __device__ __forceinline__ BgIter(const BgemmParams& p, uint32_t ntiles)
+        : stream(p.stream), nkb(p.nkb), S(p.S), nitems(ntiles * p.S), item(blockIdx.x) {
+        const uint32_t T = ntiles * p.nkb;
+        g0 = (uint32_t)(((uint64_t)blockIdx.x * T) / gridDim.x);
+        g1 = (uint32_t)(((uint64_t)(blockIdx.x + 1) * T) / gridDim.x);
+    }
+    __device__ __forceinline__ bool next(BgSeg& sg) {
+        if (stream) {
+            if (g0 >= g1) return false;
+            sg.t = g0 / nkb;
+            sg.kb0 = g0 - sg.t * nkb;
+            sg.kb1 = min(nkb, sg.kb0 + (g1 - g0));
+            sg.slot = sg.t + blockIdx.x;
+            g0 += sg.kb1 - sg.kb0;
+            return true;
+        }
+        if (item >= nitems) return false;
+        const uint32_t sp = item % S;
+        sg.t = item / S;
+        sg.kb0 = (uint32_t)(((uint64_t)sp * nkb) / S);
+        sg.kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / S);
+        sg.slot = sp;
+        item += gridDim.x;
+        return true;
+    }
+};
+
+// CTAs [first, last] whose ranges of the stream schedule meet row tile t (T = tiles * nkb blocks over P CTAs, T >= P).
+__device__ __forceinline__ void bg_stream_sharers(uint32_t t, uint32_t nkb, uint32_t T, uint32_t P, uint32_t& first, uint32_t& last) {
+    first = (uint32_t)((((uint64_t)t * nkb + 1u) * P - 1u) / T);
+    last = (uint32_t)((((uint64_t)(t + 1u) * nkb) * P - 1u) / T);
+}
+
+// Where the partial results of a projection lie, for the kernels that consume them.
+struct BgPartials {
+    const float* part;
+    uint32_t R;        // rows of the projection
+    uint32_t S;        // tile schedule: K splits
+    uint32_t stream;   // 1: stream schedule
+    uint32_t nkb, T, P;   // stream schedule: K blocks per tile, blocks in all, CTAs
+};
+
+// v[i] = sum of the partial results of rows row .. row + N - 1 (one row tile; row % N == 0) of sequence b, added in
+// split order (tile schedule) or CTA order (stream schedule): the same sum on every run.
+template <int N>
+__device__ __forceinline__ void bg_sum_partials(const BgPartials& q, uint32_t b, uint32_t row, float (&v)[N]) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = 0.f;
+    const float* src;
+    size_t stride;
+    uint32_t n;
+    if (q.stream) {
+        const uint32_t t = row / BG_TILE_M;
+        uint32_t first, last;
+        bg_stream_sharers(t, q.nkb, q.T, q.P, first, last);
+        src = q.part + ((size_t)(t + first) * BG_MAX_BATCH + b) * BG_TILE_M + (row - t * BG_TILE_M);
+        stride = (size_t)BG_MAX_BATCH * BG_TILE_M;
+        n = last - first + 1u;
+    } else {
+        src = q.part + (size_t)b * q.R + row;
+        stride = (size_t)BG_MAX_BATCH * q.R;
+        n = q.S;
+    }
+    for (uint32_t s = 0; s < n; ++s, src += stride) {
+        if (N == 4) {
+            const float4 a = *reinterpret_cast<const float4*>(src);
+            v[0] += a.x; v[1] += a.y; v[2 % N] += a.z; v[3 % N] += a.w;
+        } else if (N == 2) {
+            const float2 a = *reinterpret_cast<const float2*>(src);
+            v[0] += a.x; v[1 % N] += a.y;
+        } else {
+            v[0] += *src;
+        }
+    }
+}
+
 __device__ __forceinline__ bool bg_wait(uint32_t bar, uint32_t parity, int32_t* status, uint64_t wait_ns, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
@@ -207,8 +309,6 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
     const uint32_t tmem_base = *tmem_base_s;
 
     const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
-    const uint32_t nkb = p.nkb;
-    const uint32_t nitems = ntiles * p.S;
     griddep_launch();
     bool skip = false;
     if (!(warp == 0 && lane == 0)) {
@@ -231,10 +331,11 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
             for (uint32_t i = 0; i < n; ++i)   // n <= BG_STAGES: stage i holds iteration i
                 tma_tensor_2d_g2s(tiles + i * BG_STAGE_BYTES + BG_A_BYTES, &p.map_x, (int32_t)xcols[i], 0, smem_u32(&full[i]), pol);
         };
-        for (uint32_t item = blockIdx.x; item < nitems && !skip && !*abort_flag; item += gridDim.x) {
-            const uint32_t t = item / p.S, sp = item % p.S;
-            const uint32_t kb0 = (uint32_t)(((uint64_t)sp * nkb) / p.S), kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / p.S);
-            for (uint32_t kb = kb0; kb < kb1; ++kb, ++n) {
+        BgIter iter(p, ntiles);
+        BgSeg sg;
+        while (!skip && !*abort_flag && iter.next(sg)) {
+            const uint32_t t = sg.t;
+            for (uint32_t kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
                 if (!waited && n == (uint32_t)BG_STAGES) after_predecessor();
                 if (skip) break;
                 if (use > 0 && !bg_wait(smem_u32(&empty[stage]), (use - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
@@ -278,9 +379,10 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
         // ---- MMA issuer
         const uint32_t idesc = umma_idesc_bf16(BG_TILE_M, BG_TILE_N);
         uint32_t stage = 0, use = 0, it = 0;
-        for (uint32_t item = blockIdx.x; item < nitems && !*abort_flag; item += gridDim.x, ++it) {
-            const uint32_t sp = item % p.S;
-            const uint32_t kb0 = (uint32_t)(((uint64_t)sp * nkb) / p.S), kb1 = (uint32_t)(((uint64_t)(sp + 1) * nkb) / p.S);
+        BgIter iter(p, ntiles);
+        BgSeg sg;
+        for (; !*abort_flag && iter.next(sg); ++it) {
+            const uint32_t kb0 = sg.kb0, kb1 = sg.kb1;
             const uint32_t buf = it & 1u, buse = it >> 1;
             if (buse > 0 && !bg_wait(smem_u32(&acc_empty[buf]), (buse - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
             tc_fence_after();
@@ -311,8 +413,10 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
             for (uint32_t c = 0; c < p.ssq_n; ++c) ss += p.ssq[lane * BV_MAX_CHUNKS + c];
             inv = rsqrtf(ss / (float)p.K + p.eps);
         }
-        for (uint32_t item = blockIdx.x; item < nitems; item += gridDim.x, ++it) {
-            const uint32_t t = item / p.S, sp = item % p.S;
+        BgIter iter(p, ntiles);
+        BgSeg sg;
+        for (; iter.next(sg); ++it) {
+            const uint32_t t = sg.t;
             const uint32_t buf = it & 1u, buse = it >> 1;
             if (!bg_wait(smem_u32(&acc_full[buf]), buse & 1u, p.status, p.wait_ns, abort_flag)) break;
             tc_fence_after();
@@ -325,11 +429,14 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
             const uint32_t row = t * BG_TILE_M + quarter * 32u + lane;
-            float* dst = p.out + (size_t)sp * BG_MAX_BATCH * p.R + row;
+            // tile schedule: [slot][b][R rows]; stream schedule: [slot][b][128 rows of the tile]
+            float* dst = p.stream ? p.out + (size_t)sg.slot * BG_MAX_BATCH * BG_TILE_M + quarter * 32u + lane
+                                  : p.out + (size_t)sg.slot * BG_MAX_BATCH * p.R + row;
+            const size_t bstride = p.stream ? (size_t)BG_TILE_M : (size_t)p.R;
 #pragma unroll
             for (uint32_t b = 0; b < 32; ++b) {
                 const float sc = __shfl_sync(0xffffffffu, inv, b);   // all lanes take part, also those past the last row
-                if (row < p.R && b < p.B) dst[(size_t)b * p.R] = (__uint_as_float(hi[b]) + __uint_as_float(lo[b])) * sc;
+                if (row < p.R && b < p.B) dst[(size_t)b * bstride] = (__uint_as_float(hi[b]) + __uint_as_float(lo[b])) * sc;
             }
         }
     }
@@ -359,7 +466,7 @@ __device__ __forceinline__ void put_operand2(__nv_bfloat16* xop, uint32_t K, uin
 //                factor is applied behind the next contraction);  ssq[b][chunk] = sum of v[k]^2 over the chunk.
 //   swiglu = 1:  v[f] = silu(sum_s part[s][b][2f]) * (sum_s part[s][b][2f+1]);  operand = v.
 // The sums over the splits run in split order and the sum of squares in a fixed tree: reproducible.
-__global__ void __launch_bounds__(256) kl_b_finish_kernel(const float* part, uint32_t S, uint32_t Rpart, const float* res, float* xout,
+__global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part, const float* res, float* xout,
                                                           const __nv_bfloat16* gain, int swiglu, uint32_t K, __nv_bfloat16* xop,
                                                           float* ssq, const int32_t* status) {
     const uint32_t b = blockIdx.x, c = blockIdx.y, tid = threadIdx.x;
@@ -371,21 +478,18 @@ __global__ void __launch_bounds__(256) kl_b_finish_kernel(const float* part, uin
     float v0 = 0.f, v1 = 0.f;
     if (k < K) {   // K is even
         if (swiglu) {
-            float g0 = 0.f, u0 = 0.f, g1 = 0.f, u1 = 0.f;
-            for (uint32_t s = 0; s < S; ++s) {
-                const float4 gu = *reinterpret_cast<const float4*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + 2 * k);
-                g0 += gu.x; u0 += gu.y; g1 += gu.z; u1 += gu.w;
-            }
-            v0 = g0 / (1.0f + __expf(-g0)) * u0;
-            v1 = g1 / (1.0f + __expf(-g1)) * u1;
+            float gu[4];   // gate f, up f, gate f + 1, up f + 1
+            bg_sum_partials<4>(part, b, 2 * k, gu);
+            v0 = gu[0] / (1.0f + __expf(-gu[0])) * gu[1];
+            v1 = gu[2] / (1.0f + __expf(-gu[2])) * gu[3];
             put_operand2(xop, K, b, k, v0, v1);
         } else {
             const float2 r = *reinterpret_cast<const float2*>(res + (size_t)b * K + k);
-            v0 = r.x; v1 = r.y;
-            for (uint32_t s = 0; s < S; ++s) {
-                const float2 a = *reinterpret_cast<const float2*>(part + ((size_t)s * BG_MAX_BATCH + b) * Rpart + k);
-                v0 += a.x; v1 += a.y;
-            }
+            float a[2];
+            if (part.part != nullptr) bg_sum_partials<2>(part, b, k, a);
+            else a[0] = a[1] = 0.f;
+            v0 = r.x + a[0];
+            v1 = r.y + a[1];
             *reinterpret_cast<float2*>(xout + (size_t)b * K + k) = make_float2(v0, v1);
             const uint32_t gg = *reinterpret_cast<const uint32_t*>(gain + k);
             put_operand2(xop, K, b, k, v0 * bf_lo(gg), v1 * bf_hi(gg));
@@ -432,12 +536,12 @@ struct BAttnParams {
     __nv_bfloat16* kv;
     const int32_t* positions;
     const float* cs;          // [32][hd / 2][2] (cos, sin) of the step's positions
-    const float* qkv_part;    // [S][32][QR] partial sums of the QKV projection
+    BgPartials qkv;           // partial results of the QKV projection
     float* q;                 // [32][QD] rotated, pre-scaled queries
     float* part_o;            // [B * nkv + NW][G][hd] partial results, slot = pair + warp
     float* part_ml;           // [B * nkv + NW][G][2]
     __nv_bfloat16* xop;       // operand of the O projection [64][QD]
-    uint32_t S, QR, QD, KVD, nq, nkv, G, hd, B, max_ctx, layer, NW;   // NW: warps of the attention grid
+    uint32_t QD, KVD, nq, nkv, G, hd, B, max_ctx, layer, NW;   // NW: warps of the attention grid
     int32_t* status;
     uint64_t wait_ns;
 };
@@ -455,9 +559,9 @@ __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     const int32_t pos = p.positions[b];
     const float* cs = p.cs + (size_t)b * hd;
     auto val = [&](uint32_t r) {
-        float v = 0.f;
-        for (uint32_t s = 0; s < p.S; ++s) v += p.qkv_part[((size_t)s * BG_MAX_BATCH + b) * p.QR + r];
-        return v;
+        float v[1];
+        bg_sum_partials<1>(p.qkv, b, r, v);
+        return v[0];
     };
     const size_t slab = (size_t)p.max_ctx * hd;
     if (head < p.nq) {
