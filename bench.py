@@ -534,7 +534,11 @@ def run_ours_batched(args, shape, batch, context):
         "roofline": {"bound": "hbm", "kernel": "all launches of the decoder layers (kl_bgemm_kernel x4, kl_b_attn_kernel and "
                                                "the vector kernels, per layer)", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                     "peak_source": peaks["source"], "traffic": None, "bytes_per_launch": bytes_dec,
+                     "peak_source": peaks["source"], "traffic": ncu_traffic(shape, batch, context),
+                     "traffic_source": ("ncu dram bytes read+written of the ten launches of one layer, scaled by the layer count "
+                                        "(profiles/batched_path_llama31_8b_2layers_b32_ctx4096.txt)"
+                                        if ncu_traffic(shape, batch, context) else None),
+                     "bytes_per_launch": bytes_dec,
                      "ms_per_launch": dec_avg_ms, "classifier_ms": statistics.mean(cls_ms)},
         "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_batched / K * 1e-3) / 1e9,
                        "frac_of_measured_copy": bytes_step / (ms_batched / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -569,8 +573,16 @@ def run_ours_batched(args, shape, batch, context):
 NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813534e9 + 15.228672e6) / 4
 
 
+# the same for the ten launches of one layer of the batched path at batch 32, context 4096
+NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1002.0e6
+
+
 def ncu_traffic(shape, batch, context):
-    """Bytes per looped launch, from the committed ncu capture; None for workloads that were not captured."""
+    """Bytes per looped launch (batch 1) or per step's decoder layers (batch 32), from the committed ncu captures; None
+    for workloads that were not captured."""
+    if batch == 32 and context == 4096 and (shape.hidden, shape.ffn, shape.n_q_heads, shape.n_kv_heads, shape.head_dim) == \
+            (4096, 14336, 32, 8, 128):
+        return NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 * shape.n_layers
     if batch == 1 and context == 4096 and (shape.hidden, shape.ffn, shape.n_q_heads, shape.n_kv_heads, shape.head_dim) == \
             (4096, 14336, 32, 8, 128):
         return NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 * shape.n_layers
