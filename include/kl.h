@@ -100,10 +100,11 @@ kl_status kl_set_mode(kl_handle* h, int mode);
  *                  attention covers positions 0..positions_d[b] inclusive
  *   kv_cache_d     cache in the layout above; row positions_d[b] of every layer is written
  *   logits_d       [batch, vocab] fp32, written
- * Sequences of a batch are independent (ragged positions are fine).  They are decoded one after another by the
- * batch-1 kernels -- the weights are streamed once per SEQUENCE; projections as M = batch tensor-core contractions,
- * which would stream them once per step, are not built.  Tokens and positions of the whole batch are checked
- * before the first sequence is decoded.
+ * Sequences of a batch are independent (ragged positions are fine).  A batch of 2..32 sequences takes the
+ * tensor-core path when the shape allows (kl_set_batched_path): every projection is one contraction for the whole
+ * batch, the weights are streamed once per step.  Otherwise the sequences are decoded one after another by the
+ * batch-1 kernels (weights streamed once per sequence).  Tokens and positions of the whole batch are checked before
+ * anything is written: one bad entry makes the step a no-op for every sequence.
  * The step reads tokens and positions on the device and keeps its own step counter there, so a stream capture of
  * kl_decode_step + kl_argmax_advance can be replayed step after step (same buffers).
  * Merged-call argument rule of Section 3.2: weights (grouped, all layers) come from the handle, the hidden
@@ -113,7 +114,12 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
                          float* logits_d, uint32_t batch, void* stream);
 
 /* Same step with HOST token / position / logit buffers: copies tokens and positions to the device, runs the
- * step, copies the logits back and synchronises `stream` before returning.  The KV cache stays on the device. */
+ * step, copies the logits back and synchronises `stream` before returning.  The KV cache stays on the device.
+ * A step of the batched tensor-core path is a few hundred launches whose host cost would otherwise sit between two
+ * synchronisations of every step; this entry point therefore captures it once per (kv_cache_d, batch) into a CUDA
+ * graph on a stream of its own (nothing executes there) and replays the graph on `stream` afterwards -- same
+ * kernels, same arguments, same results.  The graph is dropped by kl_set_batched_path, kl_set_wait_limit_ns and
+ * kl_destroy; with kl_profile_enable active, or if the capture is refused, the step is launched kernel by kernel. */
 kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
                               float* logits_h, uint32_t batch, void* stream);
 

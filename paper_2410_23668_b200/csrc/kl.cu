@@ -288,6 +288,13 @@ struct kl_handle {
     CUtensorMap bmap_w[5];   // QKV, O, gate/up, down, classifier
     CUtensorMap bmap_wl[5];  // last column piece of the matrices stored in chunk order
     uint32_t bsplit[5];      // K splits of the five projections
+    // kl_decode_step_host: one batched step (323 launches at 32 layers) kept as an instantiated CUDA graph, so that the
+    // host cost of the launches is paid once and not between two synchronisations of every step
+    cudaStream_t cap_stream;       // capture only; nothing ever executes on it
+    cudaGraphExec_t bgraph;        // null: none cached
+    void* bgraph_kv;               // the cache the graph was captured for
+    uint32_t bgraph_batch;
+    uint64_t bgraph_launches;      // kernels per replay
     uint32_t last_batch;
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
@@ -754,6 +761,11 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
     h->use_bt = 1;
     h->use_stream = 1;
+    h->cap_stream = nullptr;
+    h->bgraph = nullptr;
+    h->bgraph_kv = nullptr;
+    h->bgraph_batch = 0;
+    h->bgraph_launches = 0;
     h->bt_ok = 0;
     if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
         p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
@@ -925,6 +937,13 @@ static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out,
     return KL_OK;
 }
 
+static void drop_batched_graph(kl_handle* h) {
+    if (h->bgraph) cudaGraphExecDestroy(h->bgraph);
+    h->bgraph = nullptr;
+    h->bgraph_kv = nullptr;
+    h->bgraph_batch = 0;
+}
+
 // Decode step of a batch on the tensor-core path: one launch per operator group, every weight matrix streamed once.
 static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                                      float* logits_d, uint32_t batch, cudaStream_t st) {
@@ -1063,7 +1082,39 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
     cudaStream_t st = as_stream(stream);
     if (cudaMemcpyAsync(h->stage_tokens, tokens_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
     if (cudaMemcpyAsync(h->stage_positions, positions_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
-    const kl_status rc = kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
+    kl_status rc = KL_OK;
+    bool replayed = false;
+    if (batch > 1 && h->bt_ok && h->use_bt && !h->prof_capacity && all_loaded(h)) {
+        // the batched step reads and writes only the library's staging buffers and the caller's cache: captured once
+        // per (cache, batch), replayed afterwards
+        if (!h->bgraph || h->bgraph_kv != kv_cache_d || h->bgraph_batch != batch) {
+            drop_batched_graph(h);
+            if (!h->cap_stream && cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess) h->cap_stream = nullptr;
+            if (h->cap_stream && cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+                const uint64_t l0 = h->launches;
+                const kl_status crc = decode_step_batched(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch,
+                                                          h->cap_stream);
+                cudaGraph_t graph = nullptr;
+                const cudaError_t e = cudaStreamEndCapture(h->cap_stream, &graph);
+                h->bgraph_launches = h->launches - l0;
+                h->launches = l0;   // captured, not launched
+                if (crc == KL_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&h->bgraph, graph, 0) == cudaSuccess) {
+                    h->bgraph_kv = kv_cache_d;
+                    h->bgraph_batch = batch;
+                } else {
+                    h->bgraph = nullptr;
+                }
+                if (graph) cudaGraphDestroy(graph);
+            }
+            (void)cudaGetLastError();   // a refused capture is not an error: the step is launched kernel by kernel below
+        }
+        if (h->bgraph && cudaGraphLaunch(h->bgraph, st) == cudaSuccess) {
+            h->launches += h->bgraph_launches;
+            h->last_batch = batch;
+            replayed = true;
+        }
+    }
+    if (!replayed) rc = kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
     if (rc != KL_OK) return rc;
     if (cudaMemcpyAsync(logits_h, h->stage_logits, (size_t)batch * h->prm.V * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return KL_ERR_CUDA;
@@ -1191,6 +1242,7 @@ kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* c
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns) {
     if (!h || ns == 0) return KL_ERR_INVALID_ARG;
     h->prm.wait_ns = ns;
+    drop_batched_graph(h);   // the limit is a kernel argument
     return KL_OK;
 }
 
@@ -1216,6 +1268,7 @@ kl_status kl_set_batched_path(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
     if (on && !h->bt_ok) return KL_ERR_UNSUPPORTED_SHAPE;
     h->use_bt = on ? 1 : 0;
+    drop_batched_graph(h);
     return KL_OK;
 }
 
@@ -1228,6 +1281,8 @@ kl_status kl_debug_skip_signal_once(kl_handle* h, int stage) {
 void kl_destroy(kl_handle* h) {
     if (!h) return;
     kl_profile_enable(h, 0);
+    drop_batched_graph(h);
+    if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
     free(h->loaded);
     delete h;
 }

@@ -317,3 +317,37 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     dec.kl_decode_step_host(tok.pin_memory(), pos.pin_memory(), c2, logits_h, 1)
     assert torch.equal(logits_h, logits_d.cpu()) and torch.equal(c1, c2)
     dec.close()
+
+
+def test_host_buffer_entry_point_batched_graph_replay():
+    """kl_decode_step_host keeps a batched step as an instantiated CUDA graph per (cache, batch): the first call
+    captures, later calls replay, a different cache or batch captures again.  Every call gives the bits of the
+    device-pointer entry point, and a bad token still makes the whole step a no-op that the status word reports."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 4, 200, 0)
+    cache0 = gen.make_kv_cache(shape, 4, 128, 200, 0, "cuda")
+    for batch, caches in ((4, 2), (3, 1)):
+        tok = gen.make_tokens(shape, 4, 0)[:batch].contiguous()
+        for c in range(caches):
+            ref_cache, cache = cache0.clone(), cache0.clone()   # a new tensor: a new cache address
+            logits_d = torch.empty(batch, shape.vocab, device="cuda")
+            logits_h = torch.empty(batch, shape.vocab).pin_memory()
+            for step in range(3):   # capture, replay, replay
+                pos = torch.tensor([128, 7, 64, 0][:batch], dtype=torch.int32) + step
+                n0 = dec.kl_launch_count()
+                dec.kl_decode_step(tok.cuda(), pos.cuda(), ref_cache, logits_d, batch)
+                n1 = dec.kl_launch_count()
+                dec.kl_decode_step_host(tok.pin_memory(), pos.pin_memory(), cache, logits_h, batch)
+                assert dec.kl_launch_count() - n1 == n1 - n0   # a replay counts the kernels it launches
+                torch.cuda.synchronize()
+                assert dec.kl_last_status() == binding.KL_OK
+                assert torch.equal(logits_h, logits_d.cpu()), (batch, c, step)
+                assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+            bad = tok.clone()
+            bad[batch - 1] = shape.vocab + 3
+            before = cache.clone()
+            logits_h.fill_(7.0)
+            dec.kl_decode_step_host(bad.pin_memory(), pos.pin_memory(), cache, logits_h, batch)
+            assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE
+            assert torch.equal(cache.view(torch.uint16), before.view(torch.uint16))
+    dec.close()
