@@ -127,6 +127,17 @@ def test_batched_path_llama31_8b_shape_b32():
     helpers.assert_parity(rep, 2, batch=32, check_cache=False)
 
 
+def test_batched_path_llama31_70b_shape_b8():
+    """The 70B layer shape (hidden 8192: gate/up in chunk order with two column pieces, down with twenty) at batch 8,
+    ragged contexts up to 2048, the first two layers and the classifier, two decode steps."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_70B, n_layers=2)
+    pos0 = [2048, 1500, 1024, 777, 300, 64, 1, 0]
+    rep = helpers.run_parity(shape, context=2048, steps=2, seed=0, batch=8, positions0=pos0, max_ctx=2048 + 8,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True, check_cache=False)
+    helpers.assert_parity(rep, 2, batch=8, check_cache=False)
+
+
 def test_batched_path_is_reproducible_and_optional():
     """The split sums are added in a fixed order: the same batched step twice gives identical bits.  A shape without
     the path (head size 32) refuses to switch it on and decodes batches on the batch-1 kernels."""
