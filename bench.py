@@ -44,6 +44,7 @@ WORKLOADS = {
     "llama31_8b_b8_ctx8192": (gen.LLAMA31_8B, 8, 8192, 16),
     "llama31_8b_b16_ctx16384": (gen.LLAMA31_8B, 16, 16384, 16),
     "llama31_70b_b8_ctx4096": (gen.LLAMA31_70B, 8, 4096, 8),
+    "llama31_70b_2layers_b8_ctx4096": (gen.ModelShape(2, 8192, 64, 8, 128, 28672, 128256, 1e-5, 500000.0), 8, 4096, 4),
     # two layers, 32 sequences at the full context: a few GB on the device, for profiler captures of the batched path
     "llama31_8b_2layers_b32_ctx4096": (gen.ModelShape(2, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 32, 4096, 4),
 }

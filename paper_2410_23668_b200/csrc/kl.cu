@@ -985,7 +985,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
         if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st, &a.qkv)) != KL_OK) return rc;
         KL_B_LAUNCH(kl_b_rope_kernel, dim3(batch, p.nq + 2 * p.nkv), 128, 0, a);
         KL_B_LAUNCH(kl_b_attn_kernel, (uint32_t)h->num_sms, BA_THREADS, ba_smem, a);
-        KL_B_LAUNCH(kl_b_attn_merge_kernel, dim3(p.nkv, batch), 256, 0, a);
+        KL_B_LAUNCH(kl_b_attn_merge_kernel, dim3(p.nq, batch), p.hd / 2, 0, a);
         if ((rc = launch_bgemm(h, 1, l, h->bpart, batch, st, &parts)) != KL_OK) return rc;
         // x += attention output projection; operand = g2 * x
         KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, parts, h->bx, h->bx, p.g2 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);

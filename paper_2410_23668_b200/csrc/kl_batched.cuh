@@ -790,46 +790,67 @@ __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_c
 
 // Combines the segments of every (sequence, kv head) pair and writes the attention output straight into the operand
 // of the O projection (bf16 hi and lo halves).  The pair's chunks [first, first + nch) were processed by the warps
-// whose ranges meet them; warp w left its part in slot (pair + w).  Grid (nkv, batch), 256 threads x 2 outputs.
-__global__ void __launch_bounds__(256) kl_b_attn_merge_kernel(const BAttnParams p) {
-    const uint32_t g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    const uint32_t G = p.G, hd = p.hd;
+// whose ranges meet them; warp w left its part in slot (pair + w).  Grid (query heads, batch), hd / 2 threads x 2
+// outputs: the threads first turn the segments' (maximum, sum) pairs into one weight per segment (in shared memory,
+// segments beyond BA_MERGE_SEGS in further rounds), then every thread adds up its two outputs over the segments --
+// independent loads, the additions in segment order.
+constexpr int BA_MERGE_SEGS = 64;
+__global__ void __launch_bounds__(64) kl_b_attn_merge_kernel(const BAttnParams p) {
+    const uint32_t hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    const uint32_t G = p.G, hd = p.hd, g = hq / G, h = hq % G;
+    __shared__ uint32_t seg[2];
+    __shared__ float wgt[BA_MERGE_SEGS];
+    __shared__ float red[4];
     griddep_launch();
     griddep_wait();
     if (*p.status != 0) return;
-    __shared__ uint32_t seg[2];
-    if (tid == 0) {
+    if (tid < 32) {   // lane bb: chunks of sequence bb; W = all chunks, first = chunks before this pair
         const uint32_t pb = BA_SLOT_BYTES / (4u * hd);
-        uint32_t W = 0, first = 0;
-        for (uint32_t bb = 0; bb < p.B; ++bb) {
-            const uint32_t n = ba_chunks(p.positions[bb], pb) * p.nkv;
-            if (bb < b) first += n;
-            W += n;
+        const uint32_t n = tid < p.B ? ba_chunks(p.positions[tid], pb) * p.nkv : 0u;
+        uint32_t W = n, first = tid < b ? n : 0u;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            W += __shfl_xor_sync(0xffffffffu, W, o);
+            first += __shfl_xor_sync(0xffffffffu, first, o);
         }
-        const uint32_t nch = ba_chunks(p.positions[b], pb), NW = min(p.NW, W);
-        first += g * nch;
-        // the warp whose range holds chunk x: floor(((x + 1) * NW - 1) / W)  (every range holds at least one chunk)
-        seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
-        seg[1] = (uint32_t)((((uint64_t)first + nch) * NW - 1u) / W);
+        if (tid == 0) {
+            const uint32_t nch = ba_chunks(p.positions[b], pb), NW = min(p.NW, W);
+            first += g * nch;
+            // the warp whose range holds chunk x: floor(((x + 1) * NW - 1) / W)  (every range holds at least one chunk)
+            seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
+            seg[1] = (uint32_t)((((uint64_t)first + nch) * NW - 1u) / W);
+        }
     }
     __syncthreads();
-    const uint32_t w_first = seg[0], w_last = seg[1];
+    const uint32_t w_first = seg[0], nseg = seg[1] - seg[0] + 1u;
     const size_t pair = (size_t)b * p.nkv + g;
-    for (uint32_t x = 2 * tid; x < G * hd; x += 2 * blockDim.x) {   // hd is even: both outputs belong to head h
-        const uint32_t h = x / hd, d = x % hd;
-        float M = -INFINITY;
-        for (uint32_t w = w_first; w <= w_last; ++w) M = fmaxf(M, p.part_ml[((pair + w) * G + h) * 2]);
-        float L = 0.f, A0 = 0.f, A1 = 0.f;
-        for (uint32_t w = w_first; w <= w_last; ++w) {
-            const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((pair + w) * G + h) * 2);
-            const float c = rescale(ml.x, M);
-            const float2 o = *reinterpret_cast<const float2*>(p.part_o + ((pair + w) * G + h) * hd + d);
-            L += ml.y * c;
+    const float* ml = p.part_ml + ((pair + w_first) * G + h) * 2;   // segment s: ml[s * G * 2], o[s * G * hd]
+    const float* po = p.part_o + ((pair + w_first) * G + h) * hd;
+    // running maximum over all segments
+    float M = -INFINITY;
+    for (uint32_t s = tid; s < nseg; s += blockDim.x) M = fmaxf(M, ml[(size_t)s * G * 2]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if ((tid & 31) == 0) red[tid >> 5] = M;
+    __syncthreads();
+    M = fmaxf(red[0], blockDim.x > 32 ? red[1] : -INFINITY);
+    float L = 0.f, A0 = 0.f, A1 = 0.f;
+    const uint32_t d = 2 * tid;   // hd is even; blockDim.x = hd / 2
+    for (uint32_t s0 = 0; s0 < nseg; s0 += BA_MERGE_SEGS) {
+        const uint32_t ns = min((uint32_t)BA_MERGE_SEGS, nseg - s0);
+        __syncthreads();   // the previous round's weights have been used
+        for (uint32_t s = tid; s < ns; s += blockDim.x) wgt[s] = rescale(ml[(size_t)(s0 + s) * G * 2], M);
+        __syncthreads();
+#pragma unroll 4
+        for (uint32_t s = 0; s < ns; ++s) {   // every thread also sums the segments' row sums itself, in segment order
+            const float c = wgt[s];
+            const float2 o = *reinterpret_cast<const float2*>(po + (size_t)(s0 + s) * G * hd + d);
+            L += __ldg(ml + (size_t)(s0 + s) * G * 2 + 1) * c;
             A0 += o.x * c;
             A1 += o.y * c;
         }
-        put_operand2(p.xop, p.QD, b, (g * G + h) * hd + d, A0 / L, A1 / L);
     }
+    if (d < hd) put_operand2(p.xop, p.QD, b, hq * hd + d, A0 / L, A1 / L);
 }
 
 }  // namespace kl
