@@ -493,7 +493,7 @@ def run_ours_batched(args, shape, batch, context):
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
     Ks = max(1, min(K, 4))   # the sequential schedule takes batch times longer per step: fewer steps
-    dec, cache, max_ctx = build_model(shape, batch, context, 4 * (K + W) + Ks + 3, seed=rank)
+    dec, cache, max_ctx = build_model(shape, batch, context, 5 * (K + W) + Ks + 3, seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
@@ -512,6 +512,10 @@ def run_ours_batched(args, shape, batch, context):
     dec.kl_profile_enable(0)
     clocks = sampler.stop()
     ms_e2e = max_over_ranks(run_host_loop(dec, cache, tok0, context, batch, W, K, stream))
+    # the same launches in plain stream order (no programmatic dependent launch): what the launch boundaries cost
+    dec.kl_set_dependent_launch(False)
+    ms_plain = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
+    dec.kl_set_dependent_launch(True)
     dec.kl_set_batched_path(False)
     dec.kl_set_mode(binding.KL_MODE_LOOPED)
     ms_seq = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, 3, Ks, stream))
@@ -551,6 +555,8 @@ def run_ours_batched(args, shape, batch, context):
                        "best_frac_of_measured_copy": bytes_step / (best_ms / K * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "cuda_graph": ({"value": tokens / (ms_graph * 1e-3), "ms_per_step": ms_graph / K} if ms_graph
                        else {"value": None, "why": graph_err}),
+        "plain_stream_order": {"value": tokens / (ms_plain * 1e-3), "ms_per_step": ms_plain / K,
+                               "launches_per_step": int(launches) // K},
         "sequential_looped": {"value": Ks * batch * world / (ms_seq * 1e-3), "ms_per_step": ms_seq / Ks, "steps": Ks,
                               "batched_speedup": (ms_seq / Ks) / (ms_batched / K)},
     }

@@ -202,6 +202,13 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
  * least 128 rows and the driver exports cuTensorMapEncodeTiled; otherwise KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
 kl_status kl_set_batched_path(kl_handle* h, int on);
 
+/* How the kernels of a batched step (ten per layer: the per-operator call schedule of Section 3.2) follow one
+ * another.  on = 1 (default): programmatic dependent launch -- a kernel may start while its predecessor still runs,
+ * sets itself up and requests weight tiles, and waits for the predecessor only before it touches the step's
+ * buffers.  on = 0: plain stream order, every kernel starts when the one before it has ended.  Same results; the
+ * switch exists so that the cost of the launch boundaries can be measured. */
+kl_status kl_set_dependent_launch(kl_handle* h, int on);
+
 /* Limit, in nanoseconds, of every device-side wait (tagged word, counter or mbarrier).  Default 2e9. */
 kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
 

@@ -31,7 +31,8 @@ TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup":
 EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_bytes", "kl_set_mode", "kl_decode_step",
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
-           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path")
+           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
+           "kl_set_dependent_launch")
 
 
 class ModelDesc(C.Structure):
@@ -92,6 +93,8 @@ def lib():
     l.kl_set_tensor_core_attention.restype = i32
     l.kl_set_batched_path.argtypes = [vp, C.c_int]
     l.kl_set_batched_path.restype = i32
+    l.kl_set_dependent_launch.argtypes = [vp, C.c_int]
+    l.kl_set_dependent_launch.restype = i32
     l.kl_status_string.argtypes = [i32]
     l.kl_status_string.restype = C.c_char_p
     l.kl_destroy.argtypes = [vp]
@@ -223,6 +226,9 @@ class Decoder:
 
     def kl_set_batched_path(self, on: bool) -> None:
         _check(lib().kl_set_batched_path(self.handle, 1 if on else 0), "kl_set_batched_path")
+
+    def kl_set_dependent_launch(self, on: bool) -> None:
+        _check(lib().kl_set_dependent_launch(self.handle, 1 if on else 0), "kl_set_dependent_launch")
 
     def kl_set_wait_limit_ns(self, ns: int) -> None:
         _check(lib().kl_set_wait_limit_ns(self.handle, ns), "kl_set_wait_limit_ns")

@@ -276,6 +276,7 @@ struct kl_handle {
     // batched (tensor-core) path
     int bt_ok;             // 1: available for this shape
     int use_bt;            // 1 (default): batches take it; 0: sequence after sequence on the batch-1 kernels
+    int use_pdl;           // 1 (default): the kernels of a batched step are launched with programmatic stream serialisation
     int use_stream;        // 1 (default): stream schedule for the projections of the layers; 0: (row tile, K split) items
     float* bx;             // [32][H] hidden states of the batch (== hidden_all)
     __nv_bfloat16* bxop[3];   // operands [64][H], [64][QD], [64][F]: rows 0..31 hi halves, 32..63 lo halves
@@ -534,7 +535,8 @@ inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s
 // Launch with programmatic stream serialisation: the kernel may start while its predecessor in the stream still runs
 // and orders itself behind it with griddepcontrol.wait (see griddep_wait in kl_batched.cuh).
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+static cudaError_t launch_dependent(int allowed, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -542,7 +544,7 @@ static cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = allowed ? 1 : 0;   // 0: the kernel starts when its predecessor has ended
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
@@ -761,6 +763,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
     h->use_bt = 1;
     h->use_stream = 1;
+    h->use_pdl = 1;
     h->cap_stream = nullptr;
     h->bgraph = nullptr;
     h->bgraph_kv = nullptr;
@@ -932,7 +935,7 @@ static kl_status launch_bgemm(kl_handle* h, int idx, uint32_t layer, float* out,
         parts->T = T;
         parts->P = grid;
     }
-    if (launch_dependent(kl_bgemm_kernel, dim3(grid), dim3(BG_THREADS), BG_SMEM_BYTES, st, g) != cudaSuccess) return KL_ERR_CUDA;
+    if (launch_dependent(h->use_pdl, kl_bgemm_kernel, dim3(grid), dim3(BG_THREADS), BG_SMEM_BYTES, st, g) != cudaSuccess) return KL_ERR_CUDA;
     ++h->launches;
     return KL_OK;
 }
@@ -970,7 +973,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     kl_status rc;
 #define KL_B_LAUNCH(kernel, grid, block, smem, ...)                                                              \
     do {                                                                                                         \
-        if (launch_dependent(kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__) != cudaSuccess) return KL_ERR_CUDA; \
+        if (launch_dependent(h->use_pdl, kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__) != cudaSuccess) return KL_ERR_CUDA; \
         ++h->launches;                                                                                           \
     } while (0)
     KL_B_LAUNCH(kl_b_embed_kernel, batch, 256, 0, tokens_d, positions_d, p.embed, h->bx, p.H, p.V, h->desc.max_ctx, p.inv_freq,
@@ -1268,6 +1271,13 @@ kl_status kl_set_batched_path(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
     if (on && !h->bt_ok) return KL_ERR_UNSUPPORTED_SHAPE;
     h->use_bt = on ? 1 : 0;
+    drop_batched_graph(h);
+    return KL_OK;
+}
+
+kl_status kl_set_dependent_launch(kl_handle* h, int on) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    h->use_pdl = on ? 1 : 0;
     drop_batched_graph(h);
     return KL_OK;
 }

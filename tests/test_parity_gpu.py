@@ -139,7 +139,8 @@ def test_batched_path_llama31_70b_shape_b8():
 
 
 def test_batched_path_is_reproducible_and_optional():
-    """The split sums are added in a fixed order: the same batched step twice gives identical bits.  A shape without
+    """The partial results are added in a fixed order: the same batched step again gives identical bits, with and
+    without programmatic dependent launch.  A shape without
     the path (head size 32) refuses to switch it on and decodes batches on the batch-1 kernels."""
     shape = gen.TINY
     dec = helpers.make_decoder(shape, 4, 200, 0)
@@ -147,7 +148,8 @@ def test_batched_path_is_reproducible_and_optional():
     tok = gen.make_tokens(shape, 4, 0).cuda()
     pos = torch.tensor([128, 7, 64, 0], dtype=torch.int32, device="cuda")
     outs = []
-    for _ in range(3):
+    for run in range(4):
+        dec.kl_set_dependent_launch(run < 3)   # the last run in plain stream order: same kernels, same bits
         cache = cache0.clone()
         logits = torch.empty(4, shape.vocab, device="cuda")
         hidden = torch.empty(4, shape.hidden, device="cuda")
