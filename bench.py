@@ -238,6 +238,32 @@ def run_host_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
     return e0.elapsed_time(e1)
 
 
+def run_greedy_host_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
+    """End to end greedy decoding through kl_decode_greedy_host: every step copies tokens and positions host->device
+    from pinned memory, runs the step and the sampling on the device, and reads the next tokens back to the host."""
+    tok_h = tok0.cpu().pin_memory()
+    pos_h = torch.full((batch,), context, dtype=torch.int32).pin_memory()
+    nxt_h = torch.empty(batch, dtype=torch.int32).pin_memory()
+
+    def one():
+        dec.kl_decode_greedy_host(tok_h, pos_h, cache, nxt_h, batch, stream)
+        tok_h.copy_(nxt_h)
+        pos_h.add_(1)
+
+    for _ in range(warmup):
+        one()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        one()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)
+
+
 _DIST = {"on": False}
 
 
@@ -373,7 +399,7 @@ def run_ours(args, shape, batch, context):
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
-    passes = 5  # looped, per-layer, per-stage, profiled, end-to-end (the graph passes restart from the context too)
+    passes = 6  # looped, per-layer, per-stage, profiled, two end-to-end passes (the graph passes restart from the context too)
     dec, cache, max_ctx = build_model(shape, batch, context, passes * (K + W), seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
@@ -414,7 +440,8 @@ def run_ours(args, shape, batch, context):
     dec.kl_profile_enable(0)
     clocks = sampler.stop()
     # 4. end to end through the host-buffer entry point
-    ms_e2e = max_over_ranks(run_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    ms_e2e_logits = max_over_ranks(run_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    ms_e2e = max_over_ranks(run_greedy_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
 
     tokens = K * batch * world
     value = tokens / (ms_looped * 1e-3)   # ms_looped is already the maximum over the replicas (replica_throughput)
@@ -438,7 +465,10 @@ def run_ours(args, shape, batch, context):
                    "l2": "inputs larger than L2 (weights streamed once per step)", "max_ctx": max_ctx},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
-                "d2h_bytes_per_step": 4 * shape.vocab * batch},
+                "d2h_bytes_per_step": 4 * batch, "call": "kl_decode_greedy_host (tokens and positions in, next tokens out)"},
+        "e2e_logits": {"value": tokens / (ms_e2e_logits * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
+                       "d2h_bytes_per_step": 4 * shape.vocab * batch,
+                       "call": "kl_decode_step_host (logits copied back, the host picks the next token)"},
         "roofline": {"bound": "hbm", "kernel": "kl_decoder_kernel (looped, all layers)", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                      "peak_source": peaks["source"], "traffic": ncu_traffic(shape, batch, context),
@@ -493,7 +523,7 @@ def run_ours_batched(args, shape, batch, context):
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
     Ks = max(1, min(K, 4))   # the sequential schedule takes batch times longer per step: fewer steps
-    dec, cache, max_ctx = build_model(shape, batch, context, 5 * (K + W) + Ks + 3, seed=rank)
+    dec, cache, max_ctx = build_model(shape, batch, context, 6 * (K + W) + Ks + 3, seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
@@ -511,7 +541,8 @@ def run_ours_batched(args, shape, batch, context):
     dec_ms, cls_ms = dec.kl_profile_read(K)
     dec.kl_profile_enable(0)
     clocks = sampler.stop()
-    ms_e2e = max_over_ranks(run_host_loop(dec, cache, tok0, context, batch, W, K, stream))
+    ms_e2e_logits = max_over_ranks(run_host_loop(dec, cache, tok0, context, batch, W, K, stream))
+    ms_e2e = max_over_ranks(run_greedy_host_loop(dec, cache, tok0, context, batch, W, K, stream))
     # the same launches in plain stream order (no programmatic dependent launch): what the launch boundaries cost
     dec.kl_set_dependent_launch(False)
     ms_plain = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
@@ -539,7 +570,10 @@ def run_ours_batched(args, shape, batch, context):
                    "l2": "inputs larger than L2 (weights and KV streamed once per step)", "max_ctx": max_ctx},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
-                "d2h_bytes_per_step": 4 * shape.vocab * batch},
+                "d2h_bytes_per_step": 4 * batch, "call": "kl_decode_greedy_host (tokens and positions in, next tokens out)"},
+        "e2e_logits": {"value": tokens / (ms_e2e_logits * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
+                       "d2h_bytes_per_step": 4 * shape.vocab * batch,
+                       "call": "kl_decode_step_host (logits copied back, the host picks the next token)"},
         "roofline": {"bound": "hbm", "kernel": "all launches of the decoder layers (kl_bgemm_kernel x4, kl_b_attn_kernel and "
                                                "the vector kernels, per layer)", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],

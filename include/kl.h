@@ -123,6 +123,14 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
 kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
                               float* logits_h, uint32_t batch, void* stream);
 
+/* One greedy decode step with HOST buffers: tokens and positions in, the next token of every sequence out
+ * (next_tokens_h[b] = lowest index among the maxima of sequence b's logits; Section 3.2's embedding, decoder,
+ * classifier and sampling calls in one entry point).  Copies tokens and positions to the device, runs the step as
+ * kl_decode_step_host does, samples on the device (kl_argmax_advance on the library's staging buffers), copies the
+ * batch x 4 bytes of tokens back and synchronises `stream`.  The logits stay on the device. */
+kl_status kl_decode_greedy_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
+                                int32_t* next_tokens_h, uint32_t batch, void* stream);
+
 /* Sampling block (greedy): tokens_d[b] = argmax_v logits_d[b, v] (lowest index on ties); positions_d[b] += 1. */
 kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d,
                             uint32_t batch, void* stream);

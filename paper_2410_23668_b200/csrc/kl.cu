@@ -1078,15 +1078,13 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     return KL_OK;
 }
 
-kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
-                              float* logits_h, uint32_t batch, void* stream) {
-    if (!h || !tokens_h || !positions_h || !kv_cache_d || !logits_h) return KL_ERR_INVALID_ARG;
-    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+// Tokens and positions from the host into the staging buffers, then one step into the staging logits (a batched
+// step replayed from its cached graph).
+static kl_status host_step(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d, uint32_t batch,
+                           void* stream) {
     cudaStream_t st = as_stream(stream);
     if (cudaMemcpyAsync(h->stage_tokens, tokens_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
     if (cudaMemcpyAsync(h->stage_positions, positions_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
-    kl_status rc = KL_OK;
-    bool replayed = false;
     if (batch > 1 && h->bt_ok && h->use_bt && !h->prof_capacity && all_loaded(h)) {
         // the batched step reads and writes only the library's staging buffers and the caller's cache: captured once
         // per (cache, batch), replayed afterwards
@@ -1114,13 +1112,35 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
         if (h->bgraph && cudaGraphLaunch(h->bgraph, st) == cudaSuccess) {
             h->launches += h->bgraph_launches;
             h->last_batch = batch;
-            replayed = true;
+            return KL_OK;
         }
     }
-    if (!replayed) rc = kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
+    return kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
+}
+
+kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
+                              float* logits_h, uint32_t batch, void* stream) {
+    if (!h || !tokens_h || !positions_h || !kv_cache_d || !logits_h) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    const kl_status rc = host_step(h, tokens_h, positions_h, kv_cache_d, batch, stream);
     if (rc != KL_OK) return rc;
     if (cudaMemcpyAsync(logits_h, h->stage_logits, (size_t)batch * h->prm.V * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return KL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KL_ERR_CUDA;
+    return KL_OK;
+}
+
+kl_status kl_decode_greedy_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
+                                int32_t* next_tokens_h, uint32_t batch, void* stream) {
+    if (!h || !tokens_h || !positions_h || !kv_cache_d || !next_tokens_h) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    kl_status rc = host_step(h, tokens_h, positions_h, kv_cache_d, batch, stream);
+    if (rc != KL_OK) return rc;
+    // greedy sampling on the device: the staging tokens become the next tokens (the staging positions advance too)
+    if ((rc = kl_argmax_advance(h, h->stage_logits, h->stage_tokens, h->stage_positions, batch, stream)) != KL_OK) return rc;
+    if (cudaMemcpyAsync(next_tokens_h, h->stage_tokens, batch * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
 }

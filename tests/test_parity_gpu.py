@@ -364,3 +364,28 @@ def test_host_buffer_entry_point_batched_graph_replay():
             assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE
             assert torch.equal(cache.view(torch.uint16), before.view(torch.uint16))
     dec.close()
+
+
+@pytest.mark.parametrize("batch", [1, 4])
+def test_greedy_host_entry_point(batch):
+    """kl_decode_greedy_host (host tokens and positions in, next tokens out) gives the tokens that kl_decode_step +
+    kl_argmax_advance give on device buffers, step after step, for the batch-1 kernels and for the batched path."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, batch, 200, 0)
+    cache0 = gen.make_kv_cache(shape, batch, 128, 200, 0, "cuda")
+    tok0 = gen.make_tokens(shape, batch, 0)
+    pos0 = torch.tensor([128, 7, 64, 0][:batch], dtype=torch.int32)
+    ref_cache, tok_d, pos_d = cache0.clone(), tok0.cuda(), pos0.cuda()
+    logits = torch.empty(batch, shape.vocab, device="cuda")
+    cache, tok_h, pos_h = cache0.clone(), tok0.clone().pin_memory(), pos0.clone().pin_memory()
+    nxt_h = torch.empty(batch, dtype=torch.int32).pin_memory()
+    for step in range(4):
+        dec.kl_decode_step(tok_d, pos_d, ref_cache, logits, batch)
+        dec.kl_argmax_advance(logits, tok_d, pos_d, batch)
+        dec.kl_decode_greedy_host(tok_h, pos_h, cache, nxt_h, batch)
+        assert dec.kl_last_status() == binding.KL_OK
+        assert torch.equal(nxt_h, tok_d.cpu()), step
+        tok_h.copy_(nxt_h)
+        pos_h.add_(1)
+    assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    dec.close()
