@@ -127,6 +127,15 @@ def test_batched_path_llama31_8b_shape_b32():
     helpers.assert_parity(rep, 2, batch=32, check_cache=False)
 
 
+def test_batched_path_llama31_8b_full_depth():
+    """All 32 layers of the 8B shape on the batched path (the layer coordinate of every tensor map, the residual
+    stream carried through 128 projections), four sequences with ragged contexts up to 512, two decode steps."""
+    pos0 = [512, 300, 77, 0]
+    rep = helpers.run_parity(gen.LLAMA31_8B, context=512, steps=2, seed=0, batch=4, positions0=pos0, max_ctx=512 + 8,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True, check_cache=False, stream_layers=True)
+    helpers.assert_parity(rep, 2, batch=4, check_cache=False)
+
+
 def test_batched_path_llama31_70b_shape_b8():
     """The 70B layer shape (hidden 8192: gate/up in chunk order with two column pieces, down with twenty) at batch 8,
     ragged contexts up to 2048, the first two layers and the classifier, two decode steps."""
