@@ -44,6 +44,9 @@ WORKLOADS = {
     "llama31_8b_b8_ctx8192": (gen.LLAMA31_8B, 8, 8192, 16),
     "llama31_8b_b16_ctx16384": (gen.LLAMA31_8B, 16, 16384, 16),
     "llama31_70b_b8_ctx4096": (gen.LLAMA31_70B, 8, 4096, 8),
+    # the 3B decoder of Table 2 by its public dimensions
+    "llama32_3b_b1_ctx4096": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 1, 4096, 64),
+    "llama32_3b_b16_ctx8192": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 16, 8192, 16),
     "llama31_70b_2layers_b8_ctx4096": (gen.ModelShape(2, 8192, 64, 8, 128, 28672, 128256, 1e-5, 500000.0), 8, 4096, 4),
     # two layers, 32 sequences at the full context: a few GB on the device, for profiler captures of the batched path
     "llama31_8b_2layers_b32_ctx4096": (gen.ModelShape(2, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 32, 4096, 4),

@@ -59,6 +59,10 @@ enum {
     KL_LM_HEAD = 11 /* [vocab, hidden]                  layer = -1 */
 };
 
+/* Shapes the kernels cover (anything else: KL_ERR_UNSUPPORTED_SHAPE): head_dim 32, 64, 128 or 256; hidden and ffn
+ * multiples of 8; n_q_heads a multiple of n_kv_heads with 1, 2, 4 or 8 query heads per kv head -- any group size up
+ * to 8 (3 and 6 included) when head_dim is 64 or 128, where attention runs on the tensor-core loop; at most as many
+ * kv heads as the device has SMs. */
 typedef struct {
     uint32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     float rms_eps;    /* added to the mean of squares, inside the root */
@@ -196,7 +200,8 @@ kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* c
 kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32_t* n_layers, uint32_t* n_stamps);
 
 /* Attention inner loop.  on = 1 (default when head_dim is 64 or 128): tensor-core loop (mma.sync on 128-byte
- * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes). */
+ * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes;
+ * built for 1, 2, 4 and 8 query heads per kv head: KL_ERR_UNSUPPORTED_SHAPE for other group sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
 /* Decode steps of a batch (batch > 1).  on = 1 (default when available): the tensor-core path -- every projection

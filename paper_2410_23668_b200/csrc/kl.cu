@@ -334,7 +334,10 @@ bool shape_supported(const kl_model_desc& d, int num_sms) {
     if (d.hidden % 8 || d.ffn % 8) return false;
     if (d.n_q_heads % d.n_kv_heads) return false;
     const uint32_t G = d.n_q_heads / d.n_kv_heads;
-    if (G != 1 && G != 2 && G != 4 && G != 8) return false;
+    // the CUDA-core attention loop is instantiated for 1, 2, 4 and 8 query heads per kv head; the tensor-core loop
+    // (head size 64 or 128) takes any group size up to 8
+    const bool pow2 = G == 1 || G == 2 || G == 4 || G == 8;
+    if (!pow2 && !(G <= 8 && (d.head_dim == 64 || d.head_dim == 128))) return false;
     if ((uint64_t)d.n_kv_heads > (uint64_t)num_sms) return false;
     if (!(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f)) return false;
     return true;
@@ -684,6 +687,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.L = d.n_layers; p.H = d.hidden; p.nq = d.n_q_heads; p.nkv = d.n_kv_heads; p.hd = d.head_dim; p.F = d.ffn;
     p.V = d.vocab; p.G = d.n_q_heads / d.n_kv_heads; p.QD = d.n_q_heads * d.head_dim; p.KVD = d.n_kv_heads * d.head_dim;
     p.max_ctx = d.max_ctx; p.B = 1;
+    if (!h->use_tc_attention && p.G != 1 && p.G != 2 && p.G != 4 && p.G != 8) {   // only the tensor-core loop takes this group size
+        free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE;
+    }
     p.P = (uint32_t)sms;
     p.cps = y.cps;
     p.eps = d.rms_eps;
@@ -1283,6 +1289,8 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
     if (on && !h->encode_tiled) return KL_ERR_CUDA;
+    const uint32_t G = h->prm.G;
+    if (!on && G != 1 && G != 2 && G != 4 && G != 8) return KL_ERR_UNSUPPORTED_SHAPE;   // no CUDA-core loop for this group size
     h->use_tc_attention = on ? 1 : 0;
     return KL_OK;
 }

@@ -147,6 +147,26 @@ def test_batched_path_llama31_70b_shape_b8():
     helpers.assert_parity(rep, 2, batch=8, check_cache=False)
 
 
+# Decoder shape of the 3B model of the paper's Table 2 (public hyper-parameters: 28 layers, hidden 3072, 24 query and
+# 8 kv heads of 128, FFN 8192); two layers of it here.
+LLAMA32_3B_2L = gen.ModelShape(2, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0)
+
+
+def test_llama32_3b_shape_two_layers():
+    """A second decoder shape by its dimensions (G = 3 query heads per kv head, hidden 3072): the batch-1 kernel in its
+    three schedules, context 2048, two steps."""
+    rep = helpers.run_parity(LLAMA32_3B_2L, context=2048, steps=2, seed=0, max_ctx=2048 + 8, check_cache=False)
+    helpers.assert_parity(rep, 2, check_cache=False)
+
+
+def test_batched_path_llama32_3b_shape_b16():
+    """The same shape on the batched path: 16 sequences, ragged contexts up to 2048, two steps."""
+    pos0 = [2048 - 131 * i for i in range(16)]
+    rep = helpers.run_parity(LLAMA32_3B_2L, context=2048, steps=2, seed=0, batch=16, positions0=pos0, max_ctx=2048 + 8,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True, check_cache=False)
+    helpers.assert_parity(rep, 2, batch=16, check_cache=False)
+
+
 def test_batched_path_is_reproducible_and_optional():
     """The partial results are added in a fixed order: the same batched step again gives identical bits, with and
     without programmatic dependent launch.  A shape without
