@@ -54,6 +54,7 @@ typedef struct {
 
 typedef struct {
     const uint16_t *wq, *wk, *wv, *wo, *wgate, *wup, *wdown, *norm1, *norm2;
+    const uint16_t *bq, *bk, *bv; /* optional biases of the q, k, v projections (NULL: none), bf16 */
 } ko_layer_weights;
 
 /* ---------------------------------------------------------------- bf16 */
@@ -208,6 +209,11 @@ int ko_decoder_layer(const ko_desc *d, const ko_layer_weights *w, uint16_t *kcac
     ko_matvec(w->wq, nq * hd, H, a, q, c, count_only);
     ko_matvec(w->wk, nkv * hd, H, a, k, c, count_only);
     ko_matvec(w->wv, nkv * hd, H, a, v, c, count_only);
+    /* q, k, v = W a + b for decoders with projection biases; the bias is added before the rotation */
+    if (w->bq && !count_only) for (int i = 0; i < nq * hd; ++i) q[i] += ko_bf16_to_double(w->bq[i]);
+    if (w->bk && !count_only) for (int i = 0; i < nkv * hd; ++i) k[i] += ko_bf16_to_double(w->bk[i]);
+    if (w->bv && !count_only) for (int i = 0; i < nkv * hd; ++i) v[i] += ko_bf16_to_double(w->bv[i]);
+    if (c && w->bq) c->weight_bytes += (uint64_t)2 * (uint64_t)(nq + 2 * nkv) * hd;
     if (c) {
         c->kv_write_bytes += (uint64_t)2 * nkv * hd * 2u;
         c->kv_read_bytes += (uint64_t)2 * nkv * (uint64_t)n * hd * 2u; /* each cached row once */

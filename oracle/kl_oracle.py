@@ -42,7 +42,8 @@ class Counters(C.Structure):
 
 
 class LayerWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "norm1", "norm2")]
+    _fields_ = [(n, C.c_void_p) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "norm1", "norm2",
+                                           "bq", "bk", "bv")]   # the biases are optional (null: none)
 
 
 _lib = None
@@ -185,7 +186,8 @@ def argmax(logits: np.ndarray) -> int:
 class Oracle:
     """Decode steps of one model, one sequence at a time, with optional layer streaming.
 
-    layer_weights(l) -> dict name -> bf16 buffer for layer l (wq wk wv wo wgate wup wdown norm1 norm2);
+    layer_weights(l) -> dict name -> bf16 buffer for layer l (wq wk wv wo wgate wup wdown norm1 norm2, and
+    bq bk bv for decoders whose q, k, v projections carry a bias);
     globals_: dict with 'norm_f', 'lm_head' and either 'embed' (the table) or a callable
     'embed_row'(token) -> bf16 row.
     """
@@ -201,7 +203,7 @@ class Oracle:
     def _layer_struct(self, l: int):
         w = self._layer_weights(l)
         keep = {k: as_u16(v) for k, v in w.items()}
-        s = LayerWeights(*[C.c_void_p(keep[n].ctypes.data) for n, _ in LayerWeights._fields_])
+        s = LayerWeights(*[C.c_void_p(keep[n].ctypes.data) if n in keep else None for n, _ in LayerWeights._fields_])
         return s, keep
 
     def embed(self, token: int) -> np.ndarray:

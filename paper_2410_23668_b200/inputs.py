@@ -51,6 +51,7 @@ class ModelShape:
     vocab: int
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
+    qkv_bias: bool = False   # q, k, v = W a + b (the 72B decoder of the paper's Table 2 has such biases)
 
     @property
     def q_dim(self) -> int:
@@ -71,6 +72,7 @@ LLAMA31_70B = ModelShape(80, 8192, 64, 8, 128, 28672, 128256, 1e-5, 500000.0)
 # name -> (rows, cols) of each tensor as handed to the library (row-major [out, in]).
 MATRIX_NAMES = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown")
 LAYER_TENSORS = MATRIX_NAMES + ("norm1", "norm2")
+BIAS_TENSORS = ("bq", "bk", "bv")   # only for shapes with qkv_bias
 GLOBAL_TENSORS = ("embed", "norm_f", "lm_head")
 
 
@@ -84,6 +86,9 @@ def tensor_shape(shape: ModelShape, name: str) -> tuple[int, ...]:
         "wgate": (s.ffn, s.hidden),
         "wup": (s.ffn, s.hidden),
         "wdown": (s.hidden, s.ffn),
+        "bq": (s.q_dim,),
+        "bk": (s.kv_dim,),
+        "bv": (s.kv_dim,),
         "norm1": (s.hidden,),
         "norm2": (s.hidden,),
         "norm_f": (s.hidden,),
@@ -176,13 +181,16 @@ def make_tensor(shape: ModelShape, name: str, layer: int = -1, seed: int = 0, de
     key = tensor_key(seed, name, layer)
     if name.startswith("norm"):
         t = normal_bf16(key, numel, 0.02, 1.0, device)
+    elif name in BIAS_TENSORS:
+        t = normal_bf16(key, numel, 0.1, 0.0, device)   # about a third of the scale of W a: visible, not dominant
     else:
         t = normal_bf16(key, numel, 0.02, 0.0, device)
     return t.view(*dims)
 
 
 def make_layer(shape: ModelShape, layer: int, seed: int = 0, device="cpu") -> dict[str, torch.Tensor]:
-    return {n: make_tensor(shape, n, layer, seed, device) for n in LAYER_TENSORS}
+    names = LAYER_TENSORS + (BIAS_TENSORS if shape.qkv_bias else ())
+    return {n: make_tensor(shape, n, layer, seed, device) for n in names}
 
 
 def make_globals(shape: ModelShape, seed: int = 0, device="cpu", with_embed_table: bool = True) -> dict[str, torch.Tensor]:

@@ -7,6 +7,8 @@ from pathlib import Path
 
 import numpy as np
 import pytest
+import dataclasses
+
 import torch
 
 from oracle import kl_oracle as ko
@@ -217,6 +219,54 @@ def test_gqa_head_mapping_constant_values():
     assert np.allclose(out, consts[1], rtol=1e-14)
 
 
+TINY_BIAS = dataclasses.replace(gen.TINY, qkv_bias=True)
+
+
+def test_qkv_bias_against_torch_restatement_and_closed_form():
+    """Decoders whose q, k, v projections carry a bias (the 72B decoder of Table 2).  (1) Four greedy steps agree with
+    the torch restatement, which adds the bias with library operators (torch rounds the new cache row through
+    float32, so a longer run eventually meets a double-rounding tie that differs by one bf16 step).  (2) W_q = W_k = W_v = 0: the cached rows are
+    the biases themselves, v row = bf16(b_v) and k row = bf16(rope(b_k)) at every position -- a bias added after the
+    rotation, to the wrong one of q / k / v, or dropped, fails.  (3) Zero biases give the bits of the model without
+    biases."""
+    shape, layers, glob, cache = _tiny_setup(shape=TINY_BIAS)
+    assert all(n in layers[0] for n in ("bq", "bk", "bv"))
+    orc = ko.Oracle(shape, cache.shape[4], lambda l: layers[l], glob)
+    c_or, c_t = u16(cache).copy(), cache.clone()
+    tok, p = int(gen.make_tokens(shape, 1, 0)[0]), 128
+    for step in range(4):
+        hidden, logits, nxt = orc.step(c_or, [tok], [p])
+        h_ref, l_ref = _torch_reference_step(shape, layers, glob, c_t, tok, p)
+        assert np.allclose(hidden[0], h_ref, rtol=1e-9, atol=1e-11), step
+        assert np.allclose(logits[0], l_ref, rtol=1e-9, atol=1e-11), step
+        c_t[:, :, :, :, p, :] = torch.from_numpy(c_or[:, :, :, :, p, :].copy()).view(torch.bfloat16)
+        tok, p = int(nxt[0]), p + 1
+    # (2)
+    zl = [{k: v.clone() for k, v in lw.items()} for lw in layers]
+    for lw in zl:
+        for n in ("wq", "wk", "wv"):
+            lw[n].zero_()
+    c16 = u16(cache).copy()
+    p = 131
+    ko.Oracle(shape, cache.shape[4], lambda l: zl[l], glob).step(c16, [5], [p])
+    hd, half = shape.head_dim, shape.head_dim // 2
+    ang = p * shape.rope_theta ** (-2.0 * np.arange(half) / hd)
+    for l in range(shape.n_layers):
+        bv = zl[l]["bv"].to(torch.float64).numpy().reshape(shape.n_kv_heads, hd)
+        assert np.array_equal(ko.bf16_to_double(c16[l, 1, 0, :, p, :]), bv)   # bf16 values: stored exactly
+        bk = zl[l]["bk"].to(torch.float64).numpy().reshape(shape.n_kv_heads, hd)
+        rot = np.concatenate([bk[:, :half] * np.cos(ang) - bk[:, half:] * np.sin(ang),
+                              bk[:, half:] * np.cos(ang) + bk[:, :half] * np.sin(ang)], axis=1)
+        assert np.allclose(ko.bf16_to_double(c16[l, 0, 0, :, p, :]), rot, rtol=2.0 ** -8, atol=1e-30)
+    # (3)
+    nb = [{k: (torch.zeros_like(v) if k in ("bq", "bk", "bv") else v) for k, v in lw.items()} for lw in layers]
+    plain = [{k: v for k, v in lw.items() if k not in ("bq", "bk", "bv")} for lw in layers]
+    ca, cb = u16(cache).copy(), u16(cache).copy()
+    ha, la, _ = ko.Oracle(shape, cache.shape[4], lambda l: nb[l], glob).step(ca, [9], [128])
+    hb, lb, _ = ko.Oracle(gen.TINY, cache.shape[4], lambda l: plain[l], glob).step(cb, [9], [128])
+    assert np.array_equal(ha, hb) and np.array_equal(la, lb) and np.array_equal(ca, cb)
+
+
 def test_zero_output_projections_pass_residual_through():
     """W_o = W_down = 0: x is unchanged by every layer, so logits = W_lm rmsnorm(E[tok]) in closed form,
     and the cache still receives bf16(rope(W_k a)) and bf16(W_v a)."""
@@ -267,9 +317,10 @@ def _torch_reference_step(shape, layers, glob, cache_bf16, token, p):
 
     for l, w in enumerate(layers):
         a = norm(x, w["norm1"])
-        q = rope((w["wq"].to(f64) @ a).view(nq, hd))
-        k = rope((w["wk"].to(f64) @ a).view(nkv, hd))
-        v = (w["wv"].to(f64) @ a).view(nkv, hd)
+        bias = {n: w[n].to(f64) if n in w else 0.0 for n in ("bq", "bk", "bv")}
+        q = rope((w["wq"].to(f64) @ a + bias["bq"]).view(nq, hd))
+        k = rope((w["wk"].to(f64) @ a + bias["bk"]).view(nkv, hd))
+        v = (w["wv"].to(f64) @ a + bias["bv"]).view(nkv, hd)
         cache_bf16[l, 0, 0, :, p, :] = k.to(torch.float32).to(torch.bfloat16)
         cache_bf16[l, 1, 0, :, p, :] = v.to(torch.float32).to(torch.bfloat16)
         K = cache_bf16[l, 0, 0, :, : p + 1, :].to(f64).repeat_interleave(nq // nkv, dim=0)  # [nq, n, hd]
