@@ -44,6 +44,9 @@ WORKLOADS = {
     "llama31_8b_b8_ctx8192": (gen.LLAMA31_8B, 8, 8192, 16),
     "llama31_8b_b16_ctx16384": (gen.LLAMA31_8B, 16, 16384, 16),
     "llama31_70b_b8_ctx4096": (gen.LLAMA31_70B, 8, 4096, 8),
+    # the 72B decoder of Table 2 by its public dimensions (biases on the q, k, v projections)
+    "qwen25_72b_shape_b1_ctx4096": (gen.ModelShape(80, 8192, 64, 8, 128, 29568, 152064, 1e-6, 1000000.0, True), 1, 4096, 16),
+    "qwen25_72b_shape_b8_ctx4096": (gen.ModelShape(80, 8192, 64, 8, 128, 29568, 152064, 1e-6, 1000000.0, True), 8, 4096, 8),
     # the 3B decoder of Table 2 by its public dimensions
     "llama32_3b_b1_ctx4096": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 1, 4096, 64),
     "llama32_3b_b16_ctx8192": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 16, 8192, 16),

@@ -56,8 +56,16 @@ enum {
     KL_NORM1 = 8,   /* [hidden]  gain of the RMSNorm before attention */
     KL_NORM2 = 9,   /* [hidden]  gain of the RMSNorm before the MLP */
     KL_NORM_F = 10, /* [hidden]  final gain              layer = -1 */
-    KL_LM_HEAD = 11 /* [vocab, hidden]                  layer = -1 */
+    KL_LM_HEAD = 11,/* [vocab, hidden]                  layer = -1 */
+    /* only for models created with KL_FLAG_QKV_BIAS: q, k, v = W a + b, the bias added before the rotation */
+    KL_BQ = 12,     /* [n_q_heads*head_dim] */
+    KL_BK = 13,     /* [n_kv_heads*head_dim] */
+    KL_BV = 14      /* [n_kv_heads*head_dim] */
 };
+
+/* kl_model_desc.flags: the q, k, v projections carry biases (KL_BQ, KL_BK, KL_BV must be loaded for every layer).
+ * The paper's operator list has no such term; its Table 2 includes a 72B decoder that does. */
+#define KL_FLAG_QKV_BIAS 1u
 
 /* Shapes the kernels cover (anything else: KL_ERR_UNSUPPORTED_SHAPE): head_dim 32, 64, 128 or 256; hidden and ffn
  * multiples of 8; n_q_heads a multiple of n_kv_heads with 1, 2, 4 or 8 query heads per kv head -- any group size up
@@ -69,7 +77,7 @@ typedef struct {
     float rope_theta; /* RoPE base; pair (i, i + head_dim/2) rotates by position * theta^(-2i/head_dim) */
     uint32_t max_batch;
     uint32_t max_ctx; /* capacity of the KV cache in positions */
-    uint32_t flags;   /* reserved, must be 0 */
+    uint32_t flags;   /* 0 or KL_FLAG_QKV_BIAS */
 } kl_model_desc;
 
 /* Sizes of the two device arenas the caller must provide to kl_create (both 256-byte aligned).

@@ -25,7 +25,8 @@ KL_MODE_PER_LAYER = 1
 KL_MODE_PER_STAGE = 2
 
 TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup": 6, "wdown": 7,
-              "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11}
+              "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11, "bq": 12, "bk": 13, "bv": 14}
+KL_FLAG_QKV_BIAS = 1
 
 # every symbol include/kl.h declares
 EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_bytes", "kl_set_mode", "kl_decode_step",
@@ -122,7 +123,8 @@ def _check(code: int, where: str) -> None:
 
 def make_desc(shape, max_batch: int, max_ctx: int) -> ModelDesc:
     return ModelDesc(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
-                     shape.vocab, float(shape.rms_eps), float(shape.rope_theta), max_batch, max_ctx, 0)
+                     shape.vocab, float(shape.rms_eps), float(shape.rope_theta), max_batch, max_ctx,
+                     KL_FLAG_QKV_BIAS if getattr(shape, "qkv_bias", False) else 0)
 
 
 def kl_workspace_bytes(desc: ModelDesc) -> tuple[int, int]:

@@ -319,7 +319,7 @@ inline uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
 
 struct Layout {
     // weight arena, element offsets (bf16)
-    size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, layer_stride;
+    size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
     size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
@@ -329,7 +329,7 @@ struct Layout {
 
 bool shape_supported(const kl_model_desc& d, int num_sms) {
     if (!d.n_layers || !d.hidden || !d.n_q_heads || !d.n_kv_heads || !d.head_dim || !d.ffn || !d.vocab) return false;
-    if (!d.max_batch || !d.max_ctx || d.flags != 0) return false;
+    if (!d.max_batch || !d.max_ctx || (d.flags & ~(uint32_t)KL_FLAG_QKV_BIAS) != 0) return false;
     if (d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128 && d.head_dim != 256) return false;
     if (d.hidden % 8 || d.ffn % 8) return false;
     if (d.n_q_heads % d.n_kv_heads) return false;
@@ -377,6 +377,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.off_d = o;   o += H * F;
     y.off_g1 = o;  o += H;
     y.off_g2 = o;  o += H;
+    y.off_bqkv = o; o += (d.flags & KL_FLAG_QKV_BIAS) ? align_up((QD + 2 * KVD) * 2, 16) / 2 : 0;
     y.layer_stride = align_up(o * 2, ALIGN) / 2;
     o = y.layer_stride * d.n_layers;
     y.off_gf = o;    o += align_up(H * 2, ALIGN) / 2;
@@ -680,7 +681,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
         else
             h->use_tc_attention = 0;
     }
-    h->loaded = (uint8_t*)calloc(12 * (size_t)d.n_layers, 1);
+    h->loaded = (uint8_t*)calloc((size_t)(KL_BV + 1) * (size_t)d.n_layers, 1);
     if (!h->loaded) { delete h; return KL_ERR_INVALID_ARG; }
 
     Params& p = h->prm;
@@ -736,6 +737,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
 
     const __nv_bfloat16* w = reinterpret_cast<const __nv_bfloat16*>(h->weights);
     p.wqkv = w + y.off_qkv; p.wo = w + y.off_o; p.wgu = w + y.off_gu; p.wd = w + y.off_d;
+    p.bqkv = (d.flags & KL_FLAG_QKV_BIAS) ? w + y.off_bqkv : nullptr;
     p.g1 = w + y.off_g1; p.g2 = w + y.off_g2; p.gf = w + y.off_gf; p.wlm = w + y.off_lm; p.embed = w + y.off_embed;
     uint8_t* sc = h->scratch;
     p.xa = (TW*)(sc + y.sxa); p.xb = (TW*)(sc + y.sxb); p.qkv = (TW*)(sc + y.sqkv); p.o = (TW*)(sc + y.so);
@@ -812,7 +814,8 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
     const Params& p = h->prm;
     const Layout y = make_layout(h->desc, h->num_sms);
     const bool global_t = (tensor == KL_EMBED || tensor == KL_NORM_F || tensor == KL_LM_HEAD);
-    if (tensor < 0 || tensor > KL_LM_HEAD) return KL_ERR_INVALID_ARG;
+    if (tensor < 0 || tensor > KL_BV) return KL_ERR_INVALID_ARG;
+    if (tensor > KL_LM_HEAD && !(h->desc.flags & KL_FLAG_QKV_BIAS)) return KL_ERR_INVALID_ARG;   // this model has no biases
     if (global_t ? (layer != -1) : (layer < 0 || layer >= (int)p.L)) return KL_ERR_INVALID_ARG;
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(h->weights);
     const size_t lo = global_t ? 0 : (size_t)layer * y.layer_stride;
@@ -833,6 +836,9 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
         case KL_WDOWN: rows = p.H; cols = p.F; dst = lo + y.off_d; pl = &p.plan[PL_D]; break;
         case KL_NORM1: rows = 1; cols = p.H; dst = lo + y.off_g1; break;
         case KL_NORM2: rows = 1; cols = p.H; dst = lo + y.off_g2; break;
+        case KL_BQ: rows = 1; cols = p.QD; dst = lo + y.off_bqkv; break;
+        case KL_BK: rows = 1; cols = p.KVD; dst = lo + y.off_bqkv + p.QD; break;
+        case KL_BV: rows = 1; cols = p.KVD; dst = lo + y.off_bqkv + p.QD + p.KVD; break;
         default: return KL_ERR_INVALID_ARG;
     }
     if (bytes != rows * cols * 2) return KL_ERR_INVALID_ARG;
@@ -864,7 +870,8 @@ static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d,
 
 static bool all_loaded(const kl_handle* h) {
     const uint32_t L = h->prm.L;
-    for (int t = 0; t <= KL_LM_HEAD; ++t) {
+    const int last = (h->desc.flags & KL_FLAG_QKV_BIAS) ? KL_BV : KL_LM_HEAD;
+    for (int t = 0; t <= last; ++t) {
         const bool global_t = (t == KL_EMBED || t == KL_NORM_F || t == KL_LM_HEAD);
         for (uint32_t l = 0; l < (global_t ? 1u : L); ++l)
             if (!h->loaded[(size_t)t * L + l]) return false;
@@ -968,6 +975,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     a.part_ml = h->baml;
     a.xop = h->bxop[1];
     a.QD = p.QD; a.KVD = p.KVD; a.nq = p.nq; a.nkv = p.nkv; a.G = p.G; a.hd = p.hd;
+    a.bias = nullptr;
     BgPartials parts = {};   // of the latest projection; part == nullptr: nothing to add
     a.B = batch;
     a.max_ctx = h->desc.max_ctx;
@@ -989,6 +997,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     for (uint32_t l = 0; l < p.L; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         a.layer = l;
+        a.bias = p.bqkv ? p.bqkv + lo : nullptr;
         // x += down projection of the previous layer; operand = g1 * x, sums of squares for the RMSNorm factor
         KL_B_LAUNCH(kl_b_finish_kernel, grid_h, 256, 0, parts, h->bx, h->bx, p.g1 + lo, 0, p.H, h->bxop[0], h->bssq, p.status);
         if ((rc = launch_bgemm(h, 0, l, h->bpart, batch, st, &a.qkv)) != KL_OK) return rc;

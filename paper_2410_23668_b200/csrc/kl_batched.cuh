@@ -537,6 +537,7 @@ struct BAttnParams {
     const int32_t* positions;
     const float* cs;          // [32][hd / 2][2] (cos, sin) of the step's positions
     BgPartials qkv;           // partial results of the QKV projection
+    const __nv_bfloat16* bias;   // biases of this layer's q, k, v projections [QD + 2 KVD], or null
     float* q;                 // [32][QD] rotated, pre-scaled queries
     float* part_o;            // [B * nkv + NW][G][hd] partial results, slot = pair + warp
     float* part_ml;           // [B * nkv + NW][G][2]
@@ -558,10 +559,10 @@ __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
     const float* cs = p.cs + (size_t)b * hd;
-    auto val = [&](uint32_t r) {
+    auto val = [&](uint32_t r) {   // row r of [q | k | v]: sum of the partial results, plus the projection's bias if any
         float v[1];
         bg_sum_partials<1>(p.qkv, b, r, v);
-        return v[0];
+        return p.bias ? v[0] + __bfloat162float(p.bias[r]) : v[0];
     };
     const size_t slab = (size_t)p.max_ctx * hd;
     if (head < p.nq) {

@@ -76,6 +76,7 @@ struct Params {
     int32_t skip_stage;    // test hook: stage of layer 0 whose end is not signalled (-1 = none)
     uint64_t wait_ns;
     uint64_t layer_stride; // elements between consecutive layers of any per-layer tensor
+    const __nv_bfloat16* bqkv;   // biases of the q, k, v projections [L][QD + 2 KVD] (layer_stride apart), or null
     GemvPlan plan[PL_COUNT];
     const __nv_bfloat16 *wqkv, *wo, *wgu, *wd, *g1, *g2, *gf, *wlm, *embed;
     __nv_bfloat16* kv;
@@ -1401,11 +1402,17 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     const uint32_t qtag = tag_of(p, layer, TG_QKV);
     const float* cs = p.rope_cs + (size_t)b * hd;  // [half][2]
     const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
+    // biases of the projections (decoders that have them): added to the polled values, before the rotation
+    const __nv_bfloat16* bias = p.bqkv ? p.bqkv + (size_t)layer * p.layer_stride : nullptr;
     for (uint32_t idx = ctid; idx < G * half; idx += NCT) {
         const uint32_t h = idx / half, i = idx % half;
         const TW* qr = qkv + (size_t)(g * G + h) * hd;
         float a, bb;
         poll_pair(p, s, qr + i, qr + i + half, qtag, a, bb);
+        if (bias) {
+            a += __bfloat162float(bias[(g * G + h) * hd + i]);
+            bb += __bfloat162float(bias[(g * G + h) * hd + i + half]);
+        }
         const float c = cs[2 * i], sn = cs[2 * i + 1];
         q_s[h * hd + i] = (a * c - bb * sn) * qscale;
         q_s[h * hd + i + half] = (bb * c + a * sn) * qscale;
@@ -1417,6 +1424,10 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
         for (uint32_t i = ctid; i < half; i += NCT) {
             float a, bb;
             poll_pair(p, s, kr + i, kr + i + half, qtag, a, bb);
+            if (bias) {
+                a += __bfloat162float(bias[p.QD + g * hd + i]);
+                bb += __bfloat162float(bias[p.QD + g * hd + i + half]);
+            }
             const float c = cs[2 * i], sn = cs[2 * i + 1];
             const __nv_bfloat16 k0 = __float2bfloat16_rn(a * c - bb * sn);
             const __nv_bfloat16 k1 = __float2bfloat16_rn(bb * c + a * sn);
@@ -1431,6 +1442,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
         for (uint32_t d = ctid; d < hd; d += NCT) {
             float va, vb;
             poll_pair(p, s, vr + d, vr + d, qtag, va, vb);
+            if (bias) va += __bfloat162float(bias[p.QD + p.KVD + g * hd + d]);
             const __nv_bfloat16 v0 = __float2bfloat16_rn(va);
             new_v[d] = __bfloat162float(v0);
             if (GT == 0) *reinterpret_cast<__nv_bfloat16*>(stage_v + (d >> 6) * 128u + (d & 63u) * 2u) = v0;

@@ -167,6 +167,51 @@ def test_batched_path_llama32_3b_shape_b16():
     helpers.assert_parity(rep, 2, batch=16, check_cache=False)
 
 
+def test_qwen25_72b_shape_two_layers_both_paths():
+    """The 72B decoder of the paper's Table 2 by its public dimensions (hidden 8192, 64 / 8 heads of 128, FFN 29568,
+    vocabulary 152064, biases on q, k, v), two layers: the looped batch-1 kernel and the batched path, two steps."""
+    shape = gen.ModelShape(2, 8192, 64, 8, 128, 29568, 152064, 1e-6, 1000000.0, True)
+    rep = helpers.run_parity(shape, context=1024, steps=2, seed=0, max_ctx=1024 + 8, check_cache=False,
+                             modes=(binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER))
+    helpers.assert_parity(rep, 2, check_cache=False)
+    rep = helpers.run_parity(shape, context=1024, steps=2, seed=0, batch=4, positions0=[1024, 700, 33, 0], max_ctx=1024 + 8,
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True, check_cache=False)
+    helpers.assert_parity(rep, 2, batch=4, check_cache=False)
+
+
+def test_qkv_bias_both_paths():
+    """A decoder whose q, k, v projections carry biases (flag KL_FLAG_QKV_BIAS, tensors bq / bk / bv): the batch-1 kernel
+    in its three schedules and the batched path against the oracle; and the flag is checked -- a model without it
+    refuses bias tensors, a model with it does not run before they are loaded."""
+    import dataclasses
+    shape = dataclasses.replace(gen.TINY, qkv_bias=True)
+    rep = helpers.run_parity(shape, context=128, steps=4, seed=5)
+    helpers.assert_parity(rep, 4)
+    rep = helpers.run_parity(shape, context=128, steps=3, seed=5, batch=5, positions0=[0, 17, 64, 127, 128],
+                             modes=(binding.KL_MODE_LOOPED,), batched_path=True)
+    helpers.assert_parity(rep, 3, batch=5, flip_tol=0.05)
+    wide = dataclasses.replace(LLAMA32_3B_2L, qkv_bias=True)   # head size 128, G = 3
+    rep = helpers.run_parity(wide, context=300, steps=2, seed=5, max_ctx=308, check_cache=False)
+    helpers.assert_parity(rep, 2, check_cache=False)
+    dec = binding.Decoder(gen.TINY, 1, 64)
+    with pytest.raises(binding.KlError) as e:
+        dec.kl_load_weights("bq", 0, torch.zeros(gen.TINY.q_dim, dtype=torch.bfloat16, device="cuda"))
+    assert e.value.code == binding.KL_ERR_INVALID_ARG
+    dec.close()
+    dec = binding.Decoder(shape, 1, 64)
+    for l in range(shape.n_layers):
+        for name, t in gen.make_layer(gen.TINY, l, 0, "cuda").items():   # everything but the biases
+            dec.kl_load_weights(name, l, t)
+    for name, t in gen.make_globals(shape, 0, "cuda").items():
+        dec.kl_load_weights(name, -1, t)
+    cache = gen.make_kv_cache(shape, 1, 8, 64, 0, "cuda")
+    with pytest.raises(binding.KlError) as e:
+        dec.kl_decode_step(torch.zeros(1, dtype=torch.int32, device="cuda"), torch.full((1,), 8, dtype=torch.int32, device="cuda"),
+                           cache, torch.empty(1, shape.vocab, device="cuda"), 1)
+    assert e.value.code == binding.KL_ERR_NOT_LOADED
+    dec.close()
+
+
 def test_batched_path_is_reproducible_and_optional():
     """The partial results are added in a fixed order: the same batched step again gives identical bits, with and
     without programmatic dependent launch.  A shape without
