@@ -47,6 +47,23 @@ def test_workspace_sizes_and_shape_validation(lib):
     bad = binding.make_desc(gen.ModelShape(2, 128, 6, 4, 64, 512, 1000), 1, 64)  # heads not divisible
     assert lib.kl_workspace_bytes(C.byref(bad), C.byref(w), C.byref(sc)) == binding.KL_ERR_UNSUPPORTED_SHAPE
     assert lib.kl_workspace_bytes(None, C.byref(w), C.byref(sc)) == binding.KL_ERR_INVALID_ARG
+    # group sizes: three query heads per kv head only where the tensor-core attention loop exists (head size 64 / 128)
+    ok = binding.make_desc(gen.ModelShape(2, 3072, 24, 8, 128, 8192, 1000), 1, 64)
+    assert lib.kl_workspace_bytes(C.byref(ok), C.byref(w), C.byref(sc)) == binding.KL_OK
+    bad = binding.make_desc(gen.ModelShape(2, 768, 24, 8, 32, 1024, 1000), 1, 64)
+    assert lib.kl_workspace_bytes(C.byref(bad), C.byref(w), C.byref(sc)) == binding.KL_ERR_UNSUPPORTED_SHAPE
+    # flags: the projection biases add their vectors to every layer; unknown flags are refused
+    import dataclasses
+    sb_shape = dataclasses.replace(s, qkv_bias=True)
+    wb2, _ = binding.kl_workspace_bytes(binding.make_desc(sb_shape, 1, 4096 + 256))
+    qr = s.q_dim + 2 * s.kv_dim
+    assert s.n_layers * qr * 2 <= wb2 - wb <= s.n_layers * (qr * 2 + 256)
+    bad = binding.make_desc(s, 1, 64)
+    bad.flags = 2
+    assert lib.kl_workspace_bytes(C.byref(bad), C.byref(w), C.byref(sc)) == binding.KL_ERR_UNSUPPORTED_SHAPE
+    # a batched handle (max_batch > 1) carries the operand, partial-result and attention buffers of the batched path
+    _, sb32 = binding.kl_workspace_bytes(binding.make_desc(s, 32, 4096 + 256))
+    assert sb < sb32 < 256 << 20
 
 
 def test_null_handle_calls_are_rejected(lib):
