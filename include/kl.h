@@ -102,7 +102,7 @@ size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch);
 
 /* KL_MODE_LOOPED (default): one persistent kernel runs all layers (4 launches per token with embedding, classifier
  * and sampling).  KL_MODE_PER_LAYER: one launch per layer (L + 3).  KL_MODE_PER_STAGE: one launch per operator group
- * of every layer -- QKV, attention, O, gate/up, down (5 L + 3): the three call schedules of Section 3.2, from the
+ * of every layer -- QKV, attention, O, gate/up, down (5 L + 3): the three call schedules of Section 2, from the
  * same stage code. */
 kl_status kl_set_mode(kl_handle* h, int mode);
 
@@ -136,7 +136,7 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
                               float* logits_h, uint32_t batch, void* stream);
 
 /* One greedy decode step with HOST buffers: tokens and positions in, the next token of every sequence out
- * (next_tokens_h[b] = lowest index among the maxima of sequence b's logits; Section 3.2's embedding, decoder,
+ * (next_tokens_h[b] = lowest index among the maxima of sequence b's logits; Section 2's embedding, decoder,
  * classifier and sampling calls in one entry point).  Copies tokens and positions to the device, runs the step as
  * kl_decode_step_host does, samples on the device (kl_argmax_advance on the library's staging buffers), copies the
  * batch x 4 bytes of tokens back and synchronises `stream`.  The logits stay on the device. */
@@ -151,7 +151,7 @@ kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens
  * allocation: a sampler that runs on logits produced elsewhere and holds no kl_handle (so there is no scratch arena
  * to carve from), or a serving loop in which a device allocation would synchronise the device or fail because the
  * process has already committed all device memory to its own pools.  The paper has no counterpart of this entry
- * point; it describes the sampling block only as one of the calls around the looped decoder (Section 3.2).
+ * point; it describes the sampling block only as one of the calls around the looped decoder (Section 2).
  *
  * The per-block partial results and the completion tickets live in a fixed array that is part of the library
  * image (KL_STATIC_ARGMAX_MAX_BATCH sequences, about 130 KB per device); nothing is allocated or freed, here or
@@ -217,13 +217,13 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
  * cores (M = 128 weight rows x N = 64 = 32 sequences x (hi, lo bf16 halves of the fp32 input), fp32 accumulators in
  * TMEM), so the weights are streamed once per step instead of once per sequence -- at batch 32 the projections are
  * dense contractions (Table 1 of the paper); attention runs as split-K units over (sequence, kv head, split).  The
- * step is a sequence of launches, one per operator group (Section 3.1's per-operator calls); kl_set_mode does not
+ * step is a sequence of launches, one per operator group (Section 2's per-operator calls); kl_set_mode does not
  * apply to it.  on = 0: the batch-1 kernels in the mode of kl_set_mode, sequence after sequence.  Available when
  * max_batch is 2..32, head_dim is 64 or 128, hidden / q width / ffn are multiples of 8, every projection has at
  * least 128 rows and the driver exports cuTensorMapEncodeTiled; otherwise KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
 kl_status kl_set_batched_path(kl_handle* h, int on);
 
-/* How the kernels of a batched step (ten per layer: the per-operator call schedule of Section 3.2) follow one
+/* How the kernels of a batched step (ten per layer: the per-operator call schedule of Section 2) follow one
  * another.  on = 1 (default): programmatic dependent launch -- a kernel may start while its predecessor still runs,
  * sets itself up and requests weight tiles, and waits for the predecessor only before it touches the step's
  * buffers.  on = 0: plain stream order, every kernel starts when the one before it has ended.  Same results; the
