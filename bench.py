@@ -625,7 +625,7 @@ NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813534e9 + 15.228672e6) / 4
 
 
 # the same for the ten launches of one layer of the batched path at batch 32, context 4096
-NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1002.0e6
+NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1002.2e6
 
 
 def ncu_traffic(shape, batch, context):
