@@ -41,6 +41,10 @@ WORKLOADS = {
     # batches take the tensor-core path: every projection one dense contraction for the whole batch
     "llama31_8b_b32_ctx4096": (gen.LLAMA31_8B, 32, 4096, 16),
     # batch sizes and context lengths of the paper's Table 2 (8 and 16 sequences, 8K and 16K tokens), same decoder shape
+    "llama31_8b_b2_ctx4096": (gen.LLAMA31_8B, 2, 4096, 32),
+    "llama31_8b_b4_ctx4096": (gen.LLAMA31_8B, 4, 4096, 32),
+    "llama31_8b_b8_ctx4096": (gen.LLAMA31_8B, 8, 4096, 32),
+    "llama31_8b_b16_ctx4096": (gen.LLAMA31_8B, 16, 4096, 16),
     "llama31_8b_b8_ctx8192": (gen.LLAMA31_8B, 8, 8192, 16),
     "llama31_8b_b16_ctx16384": (gen.LLAMA31_8B, 16, 16384, 16),
     "llama31_70b_b8_ctx4096": (gen.LLAMA31_70B, 8, 4096, 8),

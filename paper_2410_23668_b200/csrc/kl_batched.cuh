@@ -598,6 +598,12 @@ __device__ __forceinline__ uint32_t ba_chunks(int32_t pos, uint32_t pb) { return
 // First chunk of warp w when W chunks are dealt in contiguous, equally long ranges to NW warps.
 __device__ __forceinline__ uint32_t ba_range_lo(uint32_t w, uint32_t W, uint32_t NW) { return (uint32_t)(((uint64_t)w * W) / NW); }
 
+// Warps that share the W chunks of a step: all NW of the grid when there is enough to stream, fewer for a small batch or
+// short contexts -- at least BA_MIN_CHUNKS chunks per working warp, so that a (sequence, kv head) pair is not cut into
+// more segments than the merge can add up cheaply.  Every working warp gets at least one chunk.
+constexpr uint32_t BA_MIN_CHUNKS = 8;
+__device__ __forceinline__ uint32_t ba_workers(uint32_t W, uint32_t NW) { return max(1u, min(NW, W / BA_MIN_CHUNKS)); }
+
 // Walks the chunk list of the step: (sequence b, kv head g, chunk c of the sequence's nch chunks), in that order.
 struct BaCursor {
     uint32_t b, g, c, nch;
@@ -637,7 +643,8 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) W += __shfl_xor_sync(0xffffffffu, W, o);
     W *= p.nkv;
-    const uint32_t NW = min(p.NW, W), gw = blockIdx.x * BA_WARPS + warp;   // at least one chunk per working warp
+    // worker w = warp (w / CTAs) of CTA (w % CTAs): when fewer warps than the grid has are at work, they spread over all SMs
+    const uint32_t NW = ba_workers(W, p.NW), gw = warp * gridDim.x + blockIdx.x;
     if (gw >= NW) return;
     const uint32_t lo = ba_range_lo(gw, W, NW), hi = ba_range_lo(gw + 1, W, NW);
 
@@ -815,7 +822,7 @@ __global__ void __launch_bounds__(64) kl_b_attn_merge_kernel(const BAttnParams p
             first += __shfl_xor_sync(0xffffffffu, first, o);
         }
         if (tid == 0) {
-            const uint32_t nch = ba_chunks(p.positions[b], pb), NW = min(p.NW, W);
+            const uint32_t nch = ba_chunks(p.positions[b], pb), NW = ba_workers(W, p.NW);
             first += g * nch;
             // the warp whose range holds chunk x: floor(((x + 1) * NW - 1) / W)  (every range holds at least one chunk)
             seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
