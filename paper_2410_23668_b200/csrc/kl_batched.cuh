@@ -30,9 +30,11 @@
 // results, residual, gain and sums of squares for the RMSNorm, SwiGLU, RoPE, cache append) and write the next
 // projection's bf16 operand.  Doing this work in the projection's epilogue instead (the CTA that completes a tile,
 // found by a ticket, finishes it) was measured and is slower: fence, ticket, re-read and store form a latency chain
-// of ~10 us per tile on four warps, more than a separate kernel over hundreds of blocks costs.
+// of ~10 us per tile on four warps, more than a separate kernel over hundreds of blocks costs.  Doing it as the
+// prologue of the consuming kernel (shares of the work, then a grid barrier) was measured too and is no faster than a
+// small kernel that is already resident, through programmatic dependent launch, when its predecessor ends.
 // Attention is one balanced stream of K|V chunks over a persistent grid (kl_b_attn_kernel) followed by a merge per
-// (sequence, kv head) that writes the operand of the O projection.
+// (sequence, query head) that writes the operand of the O projection.
 #pragma once
 
 namespace kl {
