@@ -125,6 +125,20 @@ kl_status kl_set_mode(kl_handle* h, int mode);
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                          float* logits_d, uint32_t batch, void* stream);
 
+/* One greedy decode step, sampling included, on device buffers: decodes tokens_d at positions_d, writes the logits,
+ * replaces tokens_d[b] by the next token (lowest index among the maxima) and adds one to positions_d[b].
+ * For batch 1 this is ONE launch per token instead of the four of Section 2's looped schedule (embedding, looped
+ * decoder, classifier, sampling): the classifier runs as one more stage of the persistent kernel, every CTA reduces
+ * the logits rows it produced, and the last CTA to finish picks the token, advances the position, keeps the final
+ * hidden state for kl_read_hidden and writes the next token's embedding, rotary table and step counter.  Calls are
+ * therefore CHAINED: pass restart != 0 on the first call of a chain and whenever tokens_d / positions_d were changed
+ * by anyone else since the previous call (the embedding is then computed from tokens_d first, one more launch);
+ * restart = 0 continues the chain and must see the buffers as the previous call left them.  kl_set_mode does not
+ * apply.  For batch > 1 the call is kl_decode_step followed by kl_argmax_advance.  When the new position reaches
+ * max_ctx the status word is set to KL_ERR_OUT_OF_RANGE and the next step is a no-op. */
+kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                           uint32_t batch, int restart, void* stream);
+
 /* Same step with HOST token / position / logit buffers: copies tokens and positions to the device, runs the
  * step, copies the logits back and synchronises `stream` before returning.  The KV cache stays on the device.
  * A step of the batched tensor-core path is a few hundred launches whose host cost would otherwise sit between two

@@ -33,7 +33,7 @@ EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_by
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
            "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
-           "kl_set_dependent_launch", "kl_decode_greedy_host")
+           "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy")
 
 
 class ModelDesc(C.Structure):
@@ -72,6 +72,8 @@ def lib():
     l.kl_decode_step_host.restype = i32
     l.kl_decode_greedy_host.argtypes = [vp, vp, vp, vp, vp, u32, vp]
     l.kl_decode_greedy_host.restype = i32
+    l.kl_decode_greedy.argtypes = [vp, vp, vp, vp, vp, u32, C.c_int, vp]
+    l.kl_decode_greedy.restype = i32
     l.kl_argmax_advance.argtypes = [vp, vp, vp, vp, u32, vp]
     l.kl_argmax_advance.restype = i32
     l.kl_argmax_advance_static.argtypes = [vp, u32, vp, vp, u32, vp]
@@ -197,6 +199,10 @@ class Decoder:
     def kl_decode_step_host(self, tokens_h, positions_h, kv_cache_d, logits_h, batch: int, stream=None) -> None:
         _check(lib().kl_decode_step_host(self.handle, _ptr(tokens_h), _ptr(positions_h), _ptr(kv_cache_d),
                                          _ptr(logits_h), batch, _stream_ptr(stream)), "kl_decode_step_host")
+
+    def kl_decode_greedy(self, tokens_d, positions_d, kv_cache_d, logits_d, batch: int, restart: bool, stream=None) -> None:
+        _check(lib().kl_decode_greedy(self.handle, _ptr(tokens_d), _ptr(positions_d), _ptr(kv_cache_d), _ptr(logits_d),
+                                      batch, 1 if restart else 0, _stream_ptr(stream)), "kl_decode_greedy")
 
     def kl_decode_greedy_host(self, tokens_h, positions_h, kv_cache_d, next_tokens_h, batch: int, stream=None) -> None:
         _check(lib().kl_decode_greedy_host(self.handle, _ptr(tokens_h), _ptr(positions_h), _ptr(kv_cache_d),

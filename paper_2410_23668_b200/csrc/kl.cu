@@ -251,6 +251,164 @@ __global__ void __launch_bounds__(256) kl_argmax_kernel(const float* logits, uin
     }
 }
 
+// ------------------------------------------------------------------------------------------------ one launch per token
+// The paper's looped schedule still pays four calls per token: embedding, the looped decoder, classifier, sampling
+// (Section 2).  kl_token_kernel is all four for one sequence: the decoder layers and the classifier as consecutive
+// stages of one persistent kernel (the ring runs on from the last down projection into W_lm), then greedy sampling --
+// every CTA reduces the logits rows it has just produced, the last CTA to finish (ticket) reduces the per-CTA results,
+// advances token and position, keeps the final hidden state for kl_read_hidden and writes the NEXT token's embedding,
+// rotary table and step counter, so that the next launch starts at its first layer at once.
+struct TokenParams {
+    int32_t* tokens;        // [1] in: the token this step decodes (already embedded); out: the next token
+    int32_t* positions;     // [1] advanced by one
+    float* part_val;        // [P] per-CTA maxima
+    uint32_t* part_idx;     // [P] and their indices
+    uint32_t* ticket;       // zero between launches
+    float* hidden;          // [H] final hidden state of this step
+};
+
+__device__ __forceinline__ void produce_token(const Params& p, const Smem& s, uint32_t cta) {
+    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+    const AttnUnit u = attn_unit(p, cta);
+    for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
+        produce_attention(p, s, r, u, l);
+        produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+        produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
+        produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+    }
+    if (!r.aborted) produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
+    produce_drain(p, s, r);
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const TokenParams t) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, p);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    if (tid == 0) {
+        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    __syncthreads();
+    if (*p.status != 0) return;
+    if (warp == NCW) {
+        if (lane == 0) produce_token(p, s, cta);
+        return;
+    }
+    WarpRing wr = ring_begin();
+    const uint32_t ctid = tid;
+    RingCursor rc = {0u, 0u};
+    // ---- the decoder layers: the stage sequence of kl_decoder_kernel (kept as a copy so that the looped kernel's
+    // own code stays exactly as tuned)
+    for (uint32_t l = 0; l < p.L; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        for (uint32_t st = 0; st < 5; ++st) {
+            GemvOut out = {nullptr, nullptr, nullptr, 0u};
+            int plan = PL_QKV, ep = EP_STORE;
+            const float* xsrc = nullptr;
+            float xscale = 1.f;
+            if (st == ST_QKV) {
+                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
+                out = {p.qkv, nullptr, nullptr, tag_of(p, l, TG_QKV)};
+            } else if (st == ST_ATTN) {
+                attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
+                continue;
+            } else if (st == ST_O) {
+                load_vec(p, s, p.o, p.QD, tag_of(p, l, TG_O), false, nullptr, ctid);
+                out = {p.xb, nullptr, p.xa, tag_of(p, l, TG_XB)};
+                plan = PL_O;
+                ep = EP_RESIDUAL;
+            } else if (st == ST_GU) {
+                xscale = load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
+                out = {nullptr, p.h, nullptr, 0u};
+                plan = PL_GU;
+                ep = EP_SWIGLU;
+            } else {
+                stage_wait(p, s, p.counters + l, p.P, ctid);
+                out = {p.xa, nullptr, p.xb, tag_of(p, l + 1, TG_XA)};
+                plan = PL_D;
+                ep = EP_RESIDUAL;
+                xsrc = p.h;
+            }
+            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+            if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
+        }
+    }
+    // ---- classifier: one more stage on the same ring
+    {
+        const float xscale = load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, ctid);
+        const GemvOut out = {nullptr, p.logits, nullptr, 0u};
+        gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr, xscale);
+    }
+    // ---- greedy sampling: this CTA's rows first
+    consumer_bar();   // the rows this CTA stored are visible to all of its threads
+    const GemvPlan& pl = p.plan[PL_LM];
+    const CtaRange cr = cta_units(pl, cta, p.P);
+    const uint32_t r0 = cr.u0 * pl.rpc, r1 = min(cr.u1 * pl.rpc, p.V);
+    float bv = -INFINITY;
+    uint32_t bi = 0xffffffffu;
+    for (uint32_t i = r0 + ctid; i < r1; i += NCT) argmax_merge(bv, bi, p.logits[i], i);
+    for (int o = 16; o > 0; o >>= 1)
+        argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
+    float* sv = s.unit_part;                                           // [NCW] maxima, then [NCW] indices, then flags
+    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part) + NCW;
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part) + 2 * NCW;   // [0] last CTA, [1] token, [2] position, [3] step
+    if (lane == 0) {
+        sv[warp] = bv;
+        si[warp] = bi;
+    }
+    consumer_bar();
+    if (ctid == 0) {
+        for (uint32_t w = 1; w < (uint32_t)NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
+        t.part_val[cta] = bv;
+        t.part_idx[cta] = bi;
+        sh[0] = (atom_add_acq_rel(t.ticket, 1u) == p.P - 1u) ? 1u : 0u;
+    }
+    consumer_bar();
+    if (sh[0] == 0u) return;
+    // ---- the last CTA: all logits are written.  Next token, next position, and everything the next launch needs.
+    if (warp == 0) {
+        bv = -INFINITY;
+        bi = 0xffffffffu;
+        for (uint32_t j = lane; j < p.P; j += 32) argmax_merge(bv, bi, __ldcg(t.part_val + j), __ldcg(t.part_idx + j));
+        for (int o = 16; o > 0; o >>= 1)
+            argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
+        if (lane == 0) {
+            const uint32_t tok = bi == 0xffffffffu ? 0u : bi;
+            const int32_t pos = t.positions[0] + 1;
+            t.tokens[0] = (int32_t)tok;
+            t.positions[0] = pos;
+            *t.ticket = 0u;   // ready for the next launch
+            if (pos >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);   // the next step would leave the cache
+            sh[1] = tok;
+            sh[2] = (uint32_t)pos;
+            sh[3] = __ldg(p.step_dev) + 1u;
+        }
+    }
+    consumer_bar();
+    for (uint32_t i = ctid; i < p.H; i += NCT) t.hidden[i] = ld_tw(p.xa + i).v;   // before xa is overwritten below
+    consumer_bar();
+    const uint32_t tok = sh[1], pos = sh[2], step = sh[3];
+    const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
+    const uint32_t xtag = tag_from(step, p.L, 0, TG_XA);
+    for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
+    for (uint32_t i = ctid; i < p.hd / 2; i += NCT) {
+        double sn, cs;
+        sincos((double)pos * p.inv_freq[i], &sn, &cs);
+        p.rope_cs[2 * i] = (float)cs;
+        p.rope_cs[2 * i + 1] = (float)sn;
+    }
+    for (uint32_t i = ctid; i < p.L; i += NCT) p.counters[i] = 0u;
+    if (ctid == 0) *p.step_dev = step;
+}
+
 }  // namespace kl
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -297,6 +455,11 @@ struct kl_handle {
     uint32_t bgraph_batch;
     uint64_t bgraph_launches;      // kernels per replay
     uint32_t last_batch;
+    int hidden_is_copy;    // 1: the latest step left its final hidden state in hidden_all (kl_decode_greedy, batch 1)
+    float* tok_val;        // [P] per-CTA maxima of kl_token_kernel
+    uint32_t* tok_idx;     // [P]
+    uint32_t* tok_ticket;
+    int token_ok;          // kl_token_kernel can be resident
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
     uint64_t launches;
@@ -322,7 +485,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
     uint32_t bsplit[5];
     uint32_t cps;
 };
@@ -407,6 +570,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.slogits = s;   s += align_up(B * V * 4);
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
     y.shid = s;      s += align_up((B > 1 ? 32 : B) * H * 4);
+    y.stokp = s;     s += align_up((size_t)num_sms * 8 + ALIGN);
     // batched path (max_batch > 1): operand, partial sums, queries, attention partials
     {
         const size_t QR = QD + 2 * KVD;
@@ -727,6 +891,12 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
     if (ce == cudaSuccess)
         ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
+    {
+        int tocc = 0;
+        h->token_ok = cudaFuncSetAttribute(kl_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) == cudaSuccess &&
+                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+        (void)cudaGetLastError();
+    }
     int occ = 0;
     if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
@@ -752,6 +922,10 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->stage_logits = (float*)(sc + y.slogits);
     h->argmax_val = (float*)(sc + y.samax);
     h->hidden_all = (float*)(sc + y.shid);
+    h->tok_val = (float*)(sc + y.stokp);
+    h->tok_idx = (uint32_t*)(h->tok_val + sms);
+    h->tok_ticket = h->tok_idx + sms;
+    h->hidden_is_copy = 0;
     h->last_batch = 1;
     // tensor-core path for batches of up to 32 sequences
     h->bx = h->hidden_all;
@@ -1046,6 +1220,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         p.attn_tc = 1;
     }
     h->last_batch = batch;
+    h->hidden_is_copy = 0;
     cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
     // Sequences of a batch are independent: without the batched path the batch-1 kernels decode them one after
     // another (the weights are streamed once per sequence).
@@ -1090,6 +1265,48 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
                 return KL_ERR_CUDA;
         }
     }
+    return KL_OK;
+}
+
+kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                           uint32_t batch, int restart, void* stream) {
+    if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    if (batch > 1 || !h->token_ok) {
+        // batches (and devices on which the one-launch kernel cannot be resident): the step, then the sampling kernel
+        const kl_status rc = kl_decode_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, stream);
+        return rc != KL_OK ? rc : kl_argmax_advance(h, logits_d, tokens_d, positions_d, batch, stream);
+    }
+    if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
+    cudaStream_t st = as_stream(stream);
+    Params p = h->prm;
+    p.B = 1;
+    p.b0 = 0;
+    p.cps = (uint32_t)h->num_sms / p.nkv;
+    p.tokens = tokens_d;
+    p.positions = positions_d;
+    p.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
+    p.logits = logits_d;
+    p.skip_stage = -1;
+    p.trace = nullptr;
+    p.chunk_trace = nullptr;
+    p.attn_tc = 0;
+    if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
+        const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, 1);
+        if (trc != KL_OK) return trc;
+        p.attn_tc = 1;
+    }
+    if (restart) {   // a chain starts: embedding, rotary table and step counter as in kl_decode_step
+        kl_embed_kernel<<<1, 256, 0, st>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+        ++h->launches;
+    }
+    TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all};
+    void* args[] = {&p, &t};
+    const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
+    if (rc != KL_OK) return rc;
+    h->last_batch = 1;
+    h->hidden_is_copy = 1;
     return KL_OK;
 }
 
@@ -1151,10 +1368,19 @@ kl_status kl_decode_greedy_host(kl_handle* h, const int32_t* tokens_h, const int
     if (!h || !tokens_h || !positions_h || !kv_cache_d || !next_tokens_h) return KL_ERR_INVALID_ARG;
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     cudaStream_t st = as_stream(stream);
-    kl_status rc = host_step(h, tokens_h, positions_h, kv_cache_d, batch, stream);
-    if (rc != KL_OK) return rc;
-    // greedy sampling on the device: the staging tokens become the next tokens (the staging positions advance too)
-    if ((rc = kl_argmax_advance(h, h->stage_logits, h->stage_tokens, h->stage_positions, batch, stream)) != KL_OK) return rc;
+    kl_status rc;
+    if (batch == 1 && h->token_ok) {
+        // one sequence: embedding, then decoder layers + classifier + sampling as one kernel (the tokens come from the
+        // host every call, so every call starts a chain)
+        if (cudaMemcpyAsync(h->stage_tokens, tokens_h, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+        if (cudaMemcpyAsync(h->stage_positions, positions_h, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+        if ((rc = kl_decode_greedy(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, 1, 1, stream)) != KL_OK)
+            return rc;
+    } else {
+        if ((rc = host_step(h, tokens_h, positions_h, kv_cache_d, batch, stream)) != KL_OK) return rc;
+        // greedy sampling on the device: the staging tokens become the next tokens (the staging positions advance too)
+        if ((rc = kl_argmax_advance(h, h->stage_logits, h->stage_tokens, h->stage_positions, batch, stream)) != KL_OK) return rc;
+    }
     if (cudaMemcpyAsync(next_tokens_h, h->stage_tokens, batch * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KL_ERR_CUDA;
     if (cudaStreamSynchronize(st) != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
@@ -1219,7 +1445,7 @@ kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* st
     if (!h || !hidden_d || batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     if (batch != h->last_batch) return KL_ERR_INVALID_ARG;
     cudaError_t e;
-    if (batch == 1)   // the hidden state leaving the last layer is an array of tagged words: take the value half of each
+    if (batch == 1 && !h->hidden_is_copy)   // the hidden state leaving the last layer is an array of tagged words: the value halves
         e = cudaMemcpy2DAsync(hidden_d, 4, h->prm.xa, 8, 4, h->prm.H, cudaMemcpyDeviceToDevice, as_stream(stream));
     else
         e = cudaMemcpyAsync(hidden_d, h->hidden_all, (size_t)batch * h->prm.H * 4, cudaMemcpyDeviceToDevice, as_stream(stream));

@@ -463,3 +463,58 @@ def test_greedy_host_entry_point(batch):
         pos_h.add_(1)
     assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
     dec.close()
+
+
+@pytest.mark.parametrize("name", ["tiny", "odd_rows_hd128", "llama31_8b_4layers"])
+def test_one_launch_per_token_matches_four_launches(name):
+    """kl_decode_greedy at batch 1 (decoder layers, classifier and sampling in one persistent kernel, the next token's
+    embedding prepared by its last CTA) gives, step after step in a chain, the bits of embedding + looped decoder +
+    classifier + sampling launched one by one: tokens, positions, logits, final hidden state and cache."""
+    import dataclasses
+    shape, ctx, steps = {"tiny": (gen.TINY, 128, 8), "odd_rows_hd128": (SHAPES["odd_rows_hd128"], 150, 5),
+                         "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 1024, 4)}[name]
+    dec = helpers.make_decoder(shape, 1, ctx + steps + 8, 0)
+    cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + steps + 8, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+    ref_cache, tok, pos = cache0.clone(), tok0.clone(), torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    cache, tok1, pos1 = cache0.clone(), tok0.clone(), pos.clone()
+    logits, logits1 = torch.empty(1, shape.vocab, device="cuda"), torch.empty(1, shape.vocab, device="cuda")
+    hid, hid1 = torch.empty(1, shape.hidden, device="cuda"), torch.empty(1, shape.hidden, device="cuda")
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    for step in range(steps):
+        dec.kl_decode_step(tok, pos, ref_cache, logits, 1)
+        dec.kl_read_hidden(hid, 1)
+        dec.kl_argmax_advance(logits, tok, pos, 1)
+        torch.cuda.synchronize()
+        ref = (tok.clone(), pos.clone(), logits.clone(), hid.clone())
+        n0 = dec.kl_launch_count()
+        # the reference calls in between overwrite the library's activation buffers: the chain restarts every step
+        # except where the two runs are kept apart below
+        dec.kl_decode_greedy(tok1, pos1, cache, logits1, 1, True)
+        assert dec.kl_launch_count() - n0 == 2      # embedding + the one kernel
+        dec.kl_read_hidden(hid1, 1)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        assert torch.equal(tok1, ref[0]) and torch.equal(pos1, ref[1]), step
+        assert torch.equal(logits1, ref[2]) and torch.equal(hid1, ref[3]), step
+    assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    # an uninterrupted chain: one launch per token, the same tokens as the step-by-step run from the same start
+    cache2, tok2, pos2 = cache0.clone(), tok0.clone(), torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    cache3, tok3, pos3 = cache0.clone(), tok0.clone(), pos2.clone()
+    want = []
+    for step in range(steps):
+        dec.kl_decode_step(tok3, pos3, cache3, logits, 1)
+        dec.kl_argmax_advance(logits, tok3, pos3, 1)
+        want.append(int(tok3[0]))
+    torch.cuda.synchronize()
+    got = []
+    n0 = dec.kl_launch_count()
+    for step in range(steps):
+        dec.kl_decode_greedy(tok2, pos2, cache2, logits1, 1, step == 0)
+        got.append(tok2.clone())
+    torch.cuda.synchronize()
+    assert dec.kl_launch_count() - n0 == steps + 1
+    assert dec.kl_last_status() == binding.KL_OK
+    assert [int(t[0]) for t in got] == want and int(pos2[0]) == ctx + steps
+    assert torch.equal(logits1, logits) and torch.equal(cache2.view(torch.uint16), cache3.view(torch.uint16))
+    dec.close()
