@@ -132,7 +132,8 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
  * the logits rows it produced, and the last CTA to finish picks the token, advances the position, keeps the final
  * hidden state for kl_read_hidden and writes the next token's embedding, rotary table and step counter.  Calls are
  * therefore CHAINED: pass restart != 0 on the first call of a chain and whenever tokens_d / positions_d were changed
- * by anyone else since the previous call (the embedding is then computed from tokens_d first, one more launch);
+ * by anyone else, or another decode call was made on this handle, since the previous call (the embedding is then
+ * computed from tokens_d first, one more launch);
  * restart = 0 continues the chain and must see the buffers as the previous call left them.  kl_set_mode does not
  * apply.  For batch > 1 the call is kl_decode_step followed by kl_argmax_advance.  When the new position reaches
  * max_ctx the status word is set to KL_ERR_OUT_OF_RANGE and the next step is a no-op. */
