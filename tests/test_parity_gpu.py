@@ -518,3 +518,44 @@ def test_one_launch_per_token_matches_four_launches(name):
     assert [int(t[0]) for t in got] == want and int(pos2[0]) == ctx + steps
     assert torch.equal(logits1, logits) and torch.equal(cache2.view(torch.uint16), cache3.view(torch.uint16))
     dec.close()
+
+
+def test_one_launch_per_token_edge_cases():
+    """The chained one-launch step from an empty cache (the first token attends to itself only), on a shape with three
+    query heads per kv head and projection biases, against the oracle; and the end of the cache: the step that fills the
+    last position succeeds and reports that the next one would not fit, which is then a no-op."""
+    import dataclasses
+    shape = dataclasses.replace(LLAMA32_3B_2L, qkv_bias=True)
+    steps, max_ctx = 3, 16
+    host = helpers.HostWeights(shape, 0)
+    from oracle import kl_oracle as ko
+    orc = ko.Oracle(shape, max_ctx, host.layer, host.globals())
+    cache_or = gen.make_kv_cache(shape, 1, 0, max_ctx, 0, "cpu").view(torch.uint16).numpy().copy()
+    dec = helpers.make_decoder(shape, 1, max_ctx, 0)
+    cache = gen.make_kv_cache(shape, 1, 0, max_ctx, 0, "cuda")
+    tok = gen.make_tokens(shape, 1, 0).cuda()
+    pos = torch.zeros(1, dtype=torch.int32, device="cuda")
+    logits = torch.empty(1, shape.vocab, device="cuda")
+    hid = torch.empty(1, shape.hidden, device="cuda")
+    t, p = [int(tok[0])], [0]
+    for step in range(steps):
+        hidden, ref_logits, nxt = orc.step(cache_or, t, p)
+        dec.kl_decode_greedy(tok, pos, cache, logits, 1, step == 0)
+        dec.kl_read_hidden(hid, 1)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        assert helpers.rel_l2(hid.cpu().numpy()[0], hidden[0]) <= helpers.REL_L2_TOL
+        assert helpers.rel_l2(logits.cpu().numpy()[0], ref_logits[0]) <= helpers.REL_L2_TOL
+        assert int(tok[0]) == int(nxt[0]) and int(pos[0]) == step + 1
+        t, p = [int(nxt[0])], [step + 1]
+    # run on to the last position of the cache
+    while int(pos[0]) < max_ctx - 1:
+        dec.kl_decode_greedy(tok, pos, cache, logits, 1, False)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+    before, tok_before = cache.clone(), tok.clone()
+    dec.kl_decode_greedy(tok, pos, cache, logits, 1, False)     # fills position max_ctx - 1
+    torch.cuda.synchronize()
+    assert int(pos[0]) == max_ctx and not torch.equal(cache.view(torch.uint16), before.view(torch.uint16))
+    assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE   # ... and says that the cache is full
+    dec.close()
