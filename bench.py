@@ -204,7 +204,7 @@ def run_token_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
     return e0.elapsed_time(e1)
 
 
-def run_graph_loop(dec, cache, tok0, context, batch, warmup, steps):
+def run_graph_loop(dec, cache, tok0, context, batch, warmup, steps, greedy=False):
     """The same greedy steps with ONE decode step (all its launches + sampling) captured in a CUDA graph and replayed:
     the launch-overhead-free version of a schedule.  Returns ms for the K timed replays, or None with the reason when
     the capture is refused."""
@@ -214,14 +214,18 @@ def run_graph_loop(dec, cache, tok0, context, batch, warmup, steps):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     try:
+        def one(first):
+            if greedy:   # the chained one-launch step: the graph holds the single kernel
+                dec.kl_decode_greedy(tok, pos, cache, logits, batch, first, side)
+            else:
+                dec.kl_decode_step(tok, pos, cache, logits, batch, side)
+                dec.kl_argmax_advance(logits, tok, pos, batch, side)
         with torch.cuda.stream(side):
-            dec.kl_decode_step(tok, pos, cache, logits, batch, side)       # set-up outside the capture
-            dec.kl_argmax_advance(logits, tok, pos, batch, side)
+            one(True)                                                      # set-up outside the capture
             side.synchronize()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph, stream=side):
-                dec.kl_decode_step(tok, pos, cache, logits, batch, side)
-                dec.kl_argmax_advance(logits, tok, pos, batch, side)
+                one(False)
     except Exception as exc:  # capture not possible on this driver: report it, the plain launches stand
         torch.cuda.synchronize()
         return None, f"{type(exc).__name__}: {exc}".splitlines()[0][:200]
@@ -433,7 +437,7 @@ def run_ours(args, shape, batch, context):
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
-    passes = 7  # looped, per-layer, per-stage, one launch per token, profiled, two end-to-end passes
+    passes = 8  # looped, per-layer, per-stage, one launch per token, profiled, two end-to-end passes, graph replays
     dec, cache, max_ctx = build_model(shape, batch, context, passes * (K + W), seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
@@ -470,6 +474,9 @@ def run_ours(args, shape, batch, context):
         ms, err = run_graph_loop(dec, fresh_cache(), tok0, context, batch, W, K)
         graph_ms[name] = max_over_ranks(ms) if ms is not None and not _DIST["on"] else ms
         graph_err[name] = err
+    ms, err = run_graph_loop(dec, fresh_cache(), tok0, context, batch, W, K, greedy=True)
+    graph_ms["one_launch_per_token"] = max_over_ranks(ms) if ms is not None and not _DIST["on"] else ms
+    graph_err["one_launch_per_token"] = err
     # 3. roofline of the dominant kernel: events around the decoder launch inside the timed steps
     dec.kl_set_mode(binding.KL_MODE_LOOPED)
     dec.kl_profile_enable(K)
