@@ -585,7 +585,7 @@ def run_ours_batched(args, shape, batch, context):
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
     Ks = max(1, min(K, 4))   # the sequential schedule takes batch times longer per step: fewer steps
-    dec, cache, max_ctx = build_model(shape, batch, context, 6 * (K + W) + Ks + 3, seed=rank)
+    dec, cache, max_ctx = build_model(shape, batch, context, 7 * (K + W) + Ks + 3, seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
@@ -595,6 +595,8 @@ def run_ours_batched(args, shape, batch, context):
     l0 = dec.kl_launch_count()
     ms_batched = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
     launches = (dec.kl_launch_count() - l0) * K // (K + W)
+    # the same greedy steps through kl_decode_greedy: the library replays the step from the CUDA graph it keeps
+    ms_greedy = max_over_ranks(run_token_loop(dec, cache, tok0, context, batch, W, K, stream))
     ms_graph, graph_err = run_graph_loop(dec, cache, tok0, context, batch, W, K)
     if ms_graph is not None and _DIST["on"]:
         ms_graph = max_over_ranks(ms_graph)
@@ -620,12 +622,12 @@ def run_ours_batched(args, shape, batch, context):
     peaks = measured_peaks()
     dec_avg_ms = statistics.mean(dec_ms)
     achieved = bytes_dec / (dec_avg_ms * 1e-3) / 1e9
-    best_ms = ms_batched if ms_graph is None else min(ms_batched, ms_graph)
     line = {
-        "metric": "decode tokens/s", "value": tokens / (ms_batched * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": K,
-        "warmup": W, "ms_per_step": ms_batched / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        # headline: greedy decoding through kl_decode_greedy (the step replayed from the library's own CUDA graph)
+        "metric": "decode tokens/s", "value": tokens / (ms_greedy * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms_greedy / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": batch, "context": context, "mode": "batched tensor-core path",
+        "config": {"workload": args.workload, "batch": batch, "context": context, "mode": "batched tensor-core path, kl_decode_greedy chained on the device",
                    "storage": "bf16 weights and KV; fp32 activations enter the tcgen05 MMAs as two bf16 halves, fp32 accumulation",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "batch_schedule": "all sequences per launch (weights streamed once per step)",
@@ -645,16 +647,17 @@ def run_ours_batched(args, shape, batch, context):
                                         if ncu_traffic(shape, batch, context) else None),
                      "bytes_per_launch": bytes_dec,
                      "ms_per_launch": dec_avg_ms, "classifier_ms": statistics.mean(cls_ms)},
-        "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_batched / K * 1e-3) / 1e9,
-                       "frac_of_measured_copy": bytes_step / (ms_batched / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                       "frac_of_8tbs": bytes_step / (ms_batched / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-                       "best_frac_of_measured_copy": bytes_step / (best_ms / K * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "whole_step": {"bytes_per_step": bytes_step, "gbs": bytes_step / (ms_greedy / K * 1e-3) / 1e9,
+                       "frac_of_measured_copy": bytes_step / (ms_greedy / K * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "frac_of_8tbs": bytes_step / (ms_greedy / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
         "cuda_graph": ({"value": tokens / (ms_graph * 1e-3), "ms_per_step": ms_graph / K} if ms_graph
                        else {"value": None, "why": graph_err}),
+        "launch_by_launch": {"value": tokens / (ms_batched * 1e-3), "ms_per_step": ms_batched / K,
+                             "call": "kl_decode_step + kl_argmax_advance, every kernel launched from the host (dependent launch on)"},
         "plain_stream_order": {"value": tokens / (ms_plain * 1e-3), "ms_per_step": ms_plain / K,
                                "launches_per_step": int(launches) // K},
         "sequential_looped": {"value": Ks * batch * world / (ms_seq * 1e-3), "ms_per_step": ms_seq / Ks, "steps": Ks,
-                              "batched_speedup": (ms_seq / Ks) / (ms_batched / K)},
+                              "batched_speedup": (ms_seq / Ks) / (ms_greedy / K)},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import kl_oracle as ko

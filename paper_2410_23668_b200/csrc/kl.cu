@@ -451,7 +451,10 @@ struct kl_handle {
     // host cost of the launches is paid once and not between two synchronisations of every step
     cudaStream_t cap_stream;       // capture only; nothing ever executes on it
     cudaGraphExec_t bgraph;        // null: none cached
-    void* bgraph_kv;               // the cache the graph was captured for
+    void* bgraph_kv;               // the buffers the graph was captured for
+    const void* bgraph_tok;
+    const void* bgraph_pos;
+    void* bgraph_logits;
     uint32_t bgraph_batch;
     uint64_t bgraph_launches;      // kernels per replay
     uint32_t last_batch;
@@ -949,6 +952,8 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->cap_stream = nullptr;
     h->bgraph = nullptr;
     h->bgraph_kv = nullptr;
+    h->bgraph_tok = h->bgraph_pos = nullptr;
+    h->bgraph_logits = nullptr;
     h->bgraph_batch = 0;
     h->bgraph_launches = 0;
     h->bt_ok = 0;
@@ -1131,6 +1136,8 @@ static void drop_batched_graph(kl_handle* h) {
     if (h->bgraph) cudaGraphExecDestroy(h->bgraph);
     h->bgraph = nullptr;
     h->bgraph_kv = nullptr;
+    h->bgraph_tok = h->bgraph_pos = nullptr;
+    h->bgraph_logits = nullptr;
     h->bgraph_batch = 0;
 }
 
@@ -1268,13 +1275,58 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     return KL_OK;
 }
 
+// A batched step replayed from the handle's cached CUDA graph: captured once per set of buffers (tokens, positions,
+// cache, logits, batch) on a stream of its own, where nothing executes.  False: not replayed (profiling is on, `st`
+// is itself being captured, or the capture was refused) -- the caller launches the step kernel by kernel.
+static bool replay_batched(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                           uint32_t batch, cudaStream_t st) {
+    if (!(batch > 1 && h->bt_ok && h->use_bt && !h->prof_capacity && all_loaded(h))) return false;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    if (!h->bgraph || h->bgraph_kv != kv_cache_d || h->bgraph_batch != batch || h->bgraph_tok != tokens_d ||
+        h->bgraph_pos != positions_d || h->bgraph_logits != logits_d) {
+        drop_batched_graph(h);
+        if (!h->cap_stream && cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess) h->cap_stream = nullptr;
+        if (h->cap_stream && cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+            const uint64_t l0 = h->launches;
+            const kl_status crc = decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, h->cap_stream);
+            cudaGraph_t graph = nullptr;
+            const cudaError_t e = cudaStreamEndCapture(h->cap_stream, &graph);
+            h->bgraph_launches = h->launches - l0;
+            h->launches = l0;   // captured, not launched
+            if (crc == KL_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&h->bgraph, graph, 0) == cudaSuccess) {
+                h->bgraph_kv = kv_cache_d;
+                h->bgraph_batch = batch;
+                h->bgraph_tok = tokens_d;
+                h->bgraph_pos = positions_d;
+                h->bgraph_logits = logits_d;
+            } else {
+                h->bgraph = nullptr;
+            }
+            if (graph) cudaGraphDestroy(graph);
+        }
+        (void)cudaGetLastError();   // a refused capture is not an error
+    }
+    if (h->bgraph && cudaGraphLaunch(h->bgraph, st) == cudaSuccess) {
+        h->launches += h->bgraph_launches;
+        h->last_batch = batch;
+        return true;
+    }
+    return false;
+}
+
 kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
                            uint32_t batch, int restart, void* stream) {
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     if (batch > 1 || !h->token_ok) {
         // batches (and devices on which the one-launch kernel cannot be resident): the step, then the sampling kernel
-        const kl_status rc = kl_decode_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, stream);
+        kl_status rc = KL_OK;
+        if (!replay_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, as_stream(stream)))
+            rc = kl_decode_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, stream);
         return rc != KL_OK ? rc : kl_argmax_advance(h, logits_d, tokens_d, positions_d, batch, stream);
     }
     if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
@@ -1317,36 +1369,7 @@ static kl_status host_step(kl_handle* h, const int32_t* tokens_h, const int32_t*
     cudaStream_t st = as_stream(stream);
     if (cudaMemcpyAsync(h->stage_tokens, tokens_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
     if (cudaMemcpyAsync(h->stage_positions, positions_h, batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
-    if (batch > 1 && h->bt_ok && h->use_bt && !h->prof_capacity && all_loaded(h)) {
-        // the batched step reads and writes only the library's staging buffers and the caller's cache: captured once
-        // per (cache, batch), replayed afterwards
-        if (!h->bgraph || h->bgraph_kv != kv_cache_d || h->bgraph_batch != batch) {
-            drop_batched_graph(h);
-            if (!h->cap_stream && cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess) h->cap_stream = nullptr;
-            if (h->cap_stream && cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
-                const uint64_t l0 = h->launches;
-                const kl_status crc = decode_step_batched(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch,
-                                                          h->cap_stream);
-                cudaGraph_t graph = nullptr;
-                const cudaError_t e = cudaStreamEndCapture(h->cap_stream, &graph);
-                h->bgraph_launches = h->launches - l0;
-                h->launches = l0;   // captured, not launched
-                if (crc == KL_OK && e == cudaSuccess && graph && cudaGraphInstantiate(&h->bgraph, graph, 0) == cudaSuccess) {
-                    h->bgraph_kv = kv_cache_d;
-                    h->bgraph_batch = batch;
-                } else {
-                    h->bgraph = nullptr;
-                }
-                if (graph) cudaGraphDestroy(graph);
-            }
-            (void)cudaGetLastError();   // a refused capture is not an error: the step is launched kernel by kernel below
-        }
-        if (h->bgraph && cudaGraphLaunch(h->bgraph, st) == cudaSuccess) {
-            h->launches += h->bgraph_launches;
-            h->last_batch = batch;
-            return KL_OK;
-        }
-    }
+    if (replay_batched(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, st)) return KL_OK;
     return kl_decode_step(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, batch, stream);
 }
 

@@ -559,3 +559,43 @@ def test_one_launch_per_token_edge_cases():
     assert int(pos[0]) == max_ctx and not torch.equal(cache.view(torch.uint16), before.view(torch.uint16))
     assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE   # ... and says that the cache is full
     dec.close()
+
+
+def test_greedy_chain_of_a_batch_replays_the_cached_graph():
+    """kl_decode_greedy for a batch: kl_decode_step + kl_argmax_advance with the step replayed from the graph the handle
+    keeps per set of buffers -- same tokens, logits and cache as the two calls made one by one, also after the buffers
+    change (a new capture) and inside a caller's own stream capture (no nested replay)."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 4, 200, 0)
+    cache0 = gen.make_kv_cache(shape, 4, 128, 200, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 4, 0).cuda()
+    pos0 = torch.tensor([128, 7, 64, 0], dtype=torch.int32, device="cuda")
+    ref_cache, tok, pos = cache0.clone(), tok0.clone(), pos0.clone()
+    logits = torch.empty(4, shape.vocab, device="cuda")
+    want = []
+    for _ in range(4):
+        dec.kl_decode_step(tok, pos, ref_cache, logits, 4)
+        dec.kl_argmax_advance(logits, tok, pos, 4)
+        want.append(tok.clone())
+    torch.cuda.synchronize()
+    for attempt in range(2):   # the second attempt uses new buffers: the graph is captured again
+        cache, tok1, pos1, logits1 = cache0.clone(), tok0.clone(), pos0.clone(), torch.empty(4, shape.vocab, device="cuda")
+        for step in range(4):
+            dec.kl_decode_greedy(tok1, pos1, cache, logits1, 4, step == 0)
+            assert torch.equal(tok1, want[step]), (attempt, step)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        assert torch.equal(logits1, logits) and torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    # inside a caller's capture the step is captured kernel by kernel and replays like any other graph
+    cache, tok1, pos1 = cache0.clone(), tok0.clone(), pos0.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            dec.kl_decode_greedy(tok1, pos1, cache, logits1, 4, False, side)
+        for step in range(4):
+            graph.replay()
+        side.synchronize()
+    assert torch.equal(tok1, want[3]) and torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    dec.close()
