@@ -134,7 +134,9 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
  * therefore CHAINED: pass restart != 0 on the first call of a chain and whenever tokens_d / positions_d were changed
  * by anyone else, or another decode call was made on this handle, since the previous call (the embedding is then
  * computed from tokens_d first, one more launch);
- * restart = 0 continues the chain and must see the buffers as the previous call left them.  kl_set_mode does not
+ * restart = 0 continues the chain and must see the buffers as the previous call left them (when the handle knows
+ * that there is no chain to continue -- first call, another decode call in between, another tokens_d -- it starts
+ * one as if restart were set).  kl_set_mode does not
  * apply.  For batch > 1 the call is kl_decode_step followed by kl_argmax_advance, the step replayed from a CUDA graph
  * that the handle keeps per set of buffers (see kl_decode_step_host) unless `stream` is itself being captured.  When the new position reaches
  * max_ctx the status word is set to KL_ERR_OUT_OF_RANGE and the next step is a no-op. */

@@ -459,6 +459,8 @@ struct kl_handle {
     uint64_t bgraph_launches;      // kernels per replay
     uint32_t last_batch;
     int hidden_is_copy;    // 1: the latest step left its final hidden state in hidden_all (kl_decode_greedy, batch 1)
+    const void* chain_tok; // kl_decode_greedy, batch 1: the token buffer whose next embedding the latest launch prepared
+                           // (null: no chain to continue -- another decode call came in between)
     float* tok_val;        // [P] per-CTA maxima of kl_token_kernel
     uint32_t* tok_idx;     // [P]
     uint32_t* tok_ticket;
@@ -929,6 +931,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->tok_idx = (uint32_t*)(h->tok_val + sms);
     h->tok_ticket = h->tok_idx + sms;
     h->hidden_is_copy = 0;
+    h->chain_tok = nullptr;
     h->last_batch = 1;
     // tensor-core path for batches of up to 32 sequences
     h->bx = h->hidden_all;
@@ -1208,6 +1211,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
     cudaStream_t st = as_stream(stream);
+    h->chain_tok = nullptr;   // whatever kl_decode_greedy prepared for its next launch is overwritten by this step
     if (batch > 1 && h->bt_ok && h->use_bt) {
         h->last_batch = batch;
         return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
@@ -1228,6 +1232,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     }
     h->last_batch = batch;
     h->hidden_is_copy = 0;
+    h->chain_tok = nullptr;
     cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
     // Sequences of a batch are independent: without the batched path the batch-1 kernels decode them one after
     // another (the weights are streamed once per sequence).
@@ -1313,6 +1318,7 @@ static bool replay_batched(kl_handle* h, const int32_t* tokens_d, const int32_t*
     if (h->bgraph && cudaGraphLaunch(h->bgraph, st) == cudaSuccess) {
         h->launches += h->bgraph_launches;
         h->last_batch = batch;
+        h->chain_tok = nullptr;
         return true;
     }
     return false;
@@ -1348,7 +1354,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
         if (trc != KL_OK) return trc;
         p.attn_tc = 1;
     }
-    if (restart) {   // a chain starts: embedding, rotary table and step counter as in kl_decode_step
+    if (restart || h->chain_tok != tokens_d) {   // a chain starts: embedding, rotary table and step counter as in kl_decode_step
         kl_embed_kernel<<<1, 256, 0, st>>>(p);
         if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
         ++h->launches;
@@ -1359,6 +1365,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     if (rc != KL_OK) return rc;
     h->last_batch = 1;
     h->hidden_is_copy = 1;
+    h->chain_tok = tokens_d;
     return KL_OK;
 }
 

@@ -517,6 +517,12 @@ def test_one_launch_per_token_matches_four_launches(name):
     assert dec.kl_last_status() == binding.KL_OK
     assert [int(t[0]) for t in got] == want and int(pos2[0]) == ctx + steps
     assert torch.equal(logits1, logits) and torch.equal(cache2.view(torch.uint16), cache3.view(torch.uint16))
+    # a call without restart after other decode calls on the handle finds no chain and starts one by itself
+    cache4, tok4, pos4 = cache0.clone(), tok0.clone(), torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    dec.kl_decode_step(tok3, pos3, cache3, logits, 1)
+    dec.kl_decode_greedy(tok4, pos4, cache4, logits1, 1, False)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK and int(tok4[0]) == want[0]
     dec.close()
 
 
