@@ -323,6 +323,9 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
         // The weight tiles of the first ring round are requested before the predecessor kernel has finished (nothing
         // writes weights); their input tiles follow once it has.
         const uint64_t pol = l2_policy_evict_first();
+        // the input tiles are read again by every row tile: they should outlive the weights in L2
+        uint64_t polx;
+        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(polx));
         uint32_t stage = 0, use = 0, n = 0;
         uint32_t xcols[BG_STAGES];
         bool waited = false;
@@ -331,7 +334,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
             waited = true;
             skip = *p.status != 0;
             for (uint32_t i = 0; i < n; ++i)   // n <= BG_STAGES: stage i holds iteration i
-                tma_tensor_2d_g2s(tiles + i * BG_STAGE_BYTES + BG_A_BYTES, &p.map_x, (int32_t)xcols[i], 0, smem_u32(&full[i]), pol);
+                tma_tensor_2d_g2s(tiles + i * BG_STAGE_BYTES + BG_A_BYTES, &p.map_x, (int32_t)xcols[i], 0, smem_u32(&full[i]), polx);
         };
         BgIter iter(p, ntiles);
         BgSeg sg;
@@ -357,7 +360,7 @@ __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_co
                     else
                         tma_tensor_4d_g2s(dst, &p.map_wl, (int32_t)cin, 0, (int32_t)unit0, (int32_t)p.layer, bar, pol);
                 }
-                if (waited) tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, pol);
+                if (waited) tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, polx);
                 else xcols[stage] = xcol;
                 if (++stage == BG_STAGES) {
                     stage = 0;
