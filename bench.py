@@ -204,6 +204,42 @@ def run_token_loop(dec, cache, tok0, context, batch, warmup, steps, stream):
     return e0.elapsed_time(e1)
 
 
+def run_tokens_per_launch(dec, cache, tok0, context, warmup, steps, stream, host=False):
+    """Batch 1: the K timed steps as ONE call of kl_decode_greedy_tokens (the loop over layers extended to a loop over
+    tokens: up to 256 tokens per launch) behind `warmup` chained one-token launches.  host=True: through the host-buffer
+    entry point instead (token and position in, K tokens out, synchronised), timed by the host clock."""
+    tok = tok0.clone()
+    pos = torch.full((1,), context, dtype=torch.int32, device="cuda")
+    logits = torch.empty(1, dec.shape.vocab, dtype=torch.float32, device="cuda")
+    out = torch.empty(steps, dtype=torch.int32, device="cuda")
+    out_h = torch.empty(steps, dtype=torch.int32).pin_memory()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(warmup):
+        dec.kl_decode_greedy(tok, pos, cache, logits, 1, i == 0, stream)
+    torch.cuda.synchronize()
+    barrier()
+    if host:
+        t0 = time.perf_counter()
+        done, token, position = 0, int(tok[0]), context + warmup
+        while done < steps:
+            n = min(256, steps - done)
+            dec.kl_decode_greedy_tokens_host(token, position, cache, out_h[done:], n, stream)
+            done, token, position = done + n, int(out_h[done + n - 1]), position + n
+        ms = (time.perf_counter() - t0) * 1e3
+    else:
+        e0.record(stream)
+        dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, steps, 1, False, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        assert int(pos[0]) == context + warmup + steps
+    barrier()
+    st = dec.kl_last_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} after kl_decode_greedy_tokens")
+    return ms
+
+
 def run_graph_loop(dec, cache, tok0, context, batch, warmup, steps, greedy=False):
     """The same greedy steps with ONE decode step (all its launches + sampling) captured in a CUDA graph and replayed:
     the launch-overhead-free version of a schedule.  Returns ms for the K timed replays, or None with the reason when
@@ -437,7 +473,7 @@ def run_ours(args, shape, batch, context):
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local))
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
-    passes = 8  # looped, per-layer, per-stage, one launch per token, profiled, two end-to-end passes, graph replays
+    passes = 10  # looped, per-layer, per-stage, one launch per token, profiled, two end-to-end passes, graph replays
     dec, cache, max_ctx = build_model(shape, batch, context, passes * (K + W), seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
@@ -465,6 +501,10 @@ def run_ours(args, shape, batch, context):
     l0t = dec.kl_launch_count()
     ms_token = max_over_ranks(run_token_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
     token_launches = (dec.kl_launch_count() - l0t - 1) / (K + W)
+    # 2d. the K timed tokens in one launch (kl_decode_greedy_tokens)
+    l0k = dec.kl_launch_count()
+    ms_tokens = max_over_ranks(run_tokens_per_launch(dec, fresh_cache(), tok0, context, W, K, stream))
+    tokens_launches = dec.kl_launch_count() - l0k - 1 - W
     # 2b. both schedules again with one step captured in a CUDA graph (no per-launch host cost): the per-layer
     #     baseline at its best, so that the looped kernel is not compared with a strawman
     graph_ms, graph_err = {}, {}
@@ -487,6 +527,7 @@ def run_ours(args, shape, batch, context):
     # 4. end to end through the host-buffer entry point
     ms_e2e_logits = max_over_ranks(run_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
     ms_e2e = max_over_ranks(run_greedy_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
+    ms_e2e_tokens = max_over_ranks(run_tokens_per_launch(dec, fresh_cache(), tok0, context, W, K, stream, host=True))
 
     tokens = K * batch * world
     # headline: the fastest schedule of the same work -- one launch per token (decoder layers, classifier and sampling in
@@ -546,6 +587,10 @@ def run_ours(args, shape, batch, context):
                       "launches_per_step": 5 * shape.n_layers + 3, "looped_speedup": ms_stage / ms_looped},
         "one_launch_per_token": {"value": tokens / (ms_token * 1e-3), "ms_per_step": ms_token / K,
                                  "launches_per_step": token_launches, "vs_four_launches": ms_looped / ms_token},
+        "tokens_per_launch": {"value": tokens / (ms_tokens * 1e-3), "ms_per_step": ms_tokens / K, "launches": tokens_launches,
+                              "call": "kl_decode_greedy_tokens: the K timed tokens in one call (up to 256 tokens per launch)",
+                              "e2e": {"value": tokens / (ms_e2e_tokens * 1e-3), "h2d_bytes_per_call": 8, "d2h_bytes_per_call": 4 * K,
+                                      "call": "kl_decode_greedy_tokens_host, host clock"}},
         "per_layer": {"value": tokens / (ms_layer * 1e-3), "ms_per_step": ms_layer / K,
                       "launches_per_step": shape.n_layers + 3,
                       "looped_speedup": ms_layer / ms_looped},

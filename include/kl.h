@@ -143,6 +143,27 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
 kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
                            uint32_t batch, int restart, void* stream);
 
+/* n_tokens greedy steps in a row: after the call tokens_d / positions_d hold what n_tokens calls of kl_decode_greedy
+ * would have left, and out_tokens_d[k * batch + b] (device, n_tokens * batch int32) the token sequence b picked after
+ * step k.  logits_d holds the last step's logits.
+ * For batch 1 the loop over the decoder layers (Section 3.3) is extended to a loop over TOKENS: one launch of the
+ * persistent kernel decodes up to 256 consecutive tokens (longer runs are cut into launches of 256), with a small
+ * launch before it that lays out what changes from token to token (position, step number of the tags, rotary table).
+ * Inside the launch the CTA that finishes a token's sampling writes the next embedding while every other CTA already
+ * holds the next token's first weight tiles: neither a launch boundary nor a pipeline restart between tokens.
+ * The launch needs position + n_tokens <= max_ctx (checked on the device before anything is decoded: otherwise the
+ * status word is set to KL_ERR_OUT_OF_RANGE and nothing is decoded).  restart as in kl_decode_greedy; the call continues and is
+ * continued by chains of kl_decode_greedy on the same buffers.  For batch > 1 the call is a loop of kl_decode_greedy
+ * with the picked tokens copied to out_tokens_d after every step. */
+kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                                  int32_t* out_tokens_d, uint32_t n_tokens, uint32_t batch, int restart, void* stream);
+
+/* The same for one sequence with HOST buffers: decodes n_tokens (1..256) tokens starting from `token` at `position`,
+ * copies the picked tokens to out_tokens_h (n_tokens int32) and synchronises `stream` before returning.  Always starts
+ * a chain. */
+kl_status kl_decode_greedy_tokens_host(kl_handle* h, int32_t token, int32_t position, void* kv_cache_d, int32_t* out_tokens_h,
+                                       uint32_t n_tokens, void* stream);
+
 /* Same step with HOST token / position / logit buffers: copies tokens and positions to the device, runs the
  * step, copies the logits back and synchronises `stream` before returning.  The KV cache stays on the device.
  * A step of the batched tensor-core path is a few hundred launches whose host cost would otherwise sit between two

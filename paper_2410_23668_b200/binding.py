@@ -33,7 +33,8 @@ EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_by
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
            "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
-           "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy")
+           "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy", "kl_decode_greedy_tokens",
+           "kl_decode_greedy_tokens_host")
 
 
 class ModelDesc(C.Structure):
@@ -74,6 +75,10 @@ def lib():
     l.kl_decode_greedy_host.restype = i32
     l.kl_decode_greedy.argtypes = [vp, vp, vp, vp, vp, u32, C.c_int, vp]
     l.kl_decode_greedy.restype = i32
+    l.kl_decode_greedy_tokens.argtypes = [vp, vp, vp, vp, vp, vp, u32, u32, C.c_int, vp]
+    l.kl_decode_greedy_tokens.restype = i32
+    l.kl_decode_greedy_tokens_host.argtypes = [vp, i32, i32, vp, vp, u32, vp]
+    l.kl_decode_greedy_tokens_host.restype = i32
     l.kl_argmax_advance.argtypes = [vp, vp, vp, vp, u32, vp]
     l.kl_argmax_advance.restype = i32
     l.kl_argmax_advance_static.argtypes = [vp, u32, vp, vp, u32, vp]
@@ -203,6 +208,16 @@ class Decoder:
     def kl_decode_greedy(self, tokens_d, positions_d, kv_cache_d, logits_d, batch: int, restart: bool, stream=None) -> None:
         _check(lib().kl_decode_greedy(self.handle, _ptr(tokens_d), _ptr(positions_d), _ptr(kv_cache_d), _ptr(logits_d),
                                       batch, 1 if restart else 0, _stream_ptr(stream)), "kl_decode_greedy")
+
+    def kl_decode_greedy_tokens(self, tokens_d, positions_d, kv_cache_d, logits_d, out_tokens_d, n_tokens: int, batch: int,
+                                restart: bool, stream=None) -> None:
+        _check(lib().kl_decode_greedy_tokens(self.handle, _ptr(tokens_d), _ptr(positions_d), _ptr(kv_cache_d), _ptr(logits_d),
+                                             _ptr(out_tokens_d), n_tokens, batch, 1 if restart else 0, _stream_ptr(stream)),
+               "kl_decode_greedy_tokens")
+
+    def kl_decode_greedy_tokens_host(self, token: int, position: int, kv_cache_d, out_tokens_h, n_tokens: int, stream=None) -> None:
+        _check(lib().kl_decode_greedy_tokens_host(self.handle, token, position, _ptr(kv_cache_d), _ptr(out_tokens_h), n_tokens,
+                                                  _stream_ptr(stream)), "kl_decode_greedy_tokens_host")
 
     def kl_decode_greedy_host(self, tokens_h, positions_h, kv_cache_d, next_tokens_h, batch: int, stream=None) -> None:
         _check(lib().kl_decode_greedy_host(self.handle, _ptr(tokens_h), _ptr(positions_h), _ptr(kv_cache_d),

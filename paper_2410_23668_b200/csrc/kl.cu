@@ -307,16 +307,22 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_cons
     RingCursor rc = {0u, 0u};
     // ---- the decoder layers: the stage sequence of kl_decoder_kernel (kept as a copy so that the looped kernel's
     // own code stays exactly as tuned)
-    for (uint32_t l = 0; l < p.L; ++l) {
+    for (uint32_t l = 0; l <= p.L; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
-        for (uint32_t st = 0; st < 5; ++st) {
+        const bool cls = l == p.L;
+        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st) {
             GemvOut out = {nullptr, nullptr, nullptr, 0u};
             int plan = PL_QKV, ep = EP_STORE;
             const float* xsrc = nullptr;
             float xscale = 1.f;
             if (st == ST_QKV) {
-                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
-                out = {p.qkv, nullptr, nullptr, tag_of(p, l, TG_QKV)};
+                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, cls ? p.gf : p.g1 + lo, ctid);
+                if (cls) {
+                    out = {nullptr, p.logits, nullptr, 0u};
+                    plan = PL_LM;
+                } else {
+                    out = {p.qkv, nullptr, nullptr, tag_of(p, l, TG_QKV)};
+                }
             } else if (st == ST_ATTN) {
                 attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
                 continue;
@@ -340,12 +346,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_cons
             gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
             if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
         }
-    }
-    // ---- classifier: one more stage on the same ring
-    {
-        const float xscale = load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, ctid);
-        const GemvOut out = {nullptr, p.logits, nullptr, 0u};
-        gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr, xscale);
     }
     // ---- greedy sampling: this CTA's rows first
     consumer_bar();   // the rows this CTA stored are visible to all of its threads
@@ -409,6 +409,256 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_cons
     if (ctid == 0) *p.step_dev = step;
 }
 
+// ------------------------------------------------------------------------------------------------ K tokens per launch
+// The loop over layers extended to a loop over TOKENS: one launch decodes K consecutive tokens of one sequence.  What
+// changes from token to token inside the launch -- the position, the step number the tags are built from, the rotary
+// table -- is laid out beforehand, one entry per token, by kl_token_plan_kernel (the values are known: position and
+// step advance by one); entry k also holds a copy of the kernel parameters that points at them, which is what the
+// attention code (out of line, parameters by reference) is given for token k.  Counters that were zeroed between
+// launches count on instead: the gate/up counter of a layer reaches P * (k + 1) during token k, and so does the
+// sampling ticket.  The CTA that draws the last ticket of token k picks the token, records it, and writes the next
+// embedding under the tags of step + 1; all other CTAs are by then polling for exactly those words, with the first
+// weight tiles of the next token already in their rings -- no launch boundary, no pipeline restart.
+// Tag slot of an embedding written INSIDE the launch.  The hidden state that enters the classifier carries
+// (step, layer L, TG_XA), which is the same number as (step + 1, layer 0, TG_XA): across a launch boundary that is
+// harmless, inside the launch the CTAs polling for the next embedding would take the old hidden state for it.
+constexpr uint32_t TG_NEXT = 5;
+struct TokenLoopParams {
+    TokenParams t;
+    int32_t* out_tokens;       // [K] the token picked after each step
+    uint32_t K;
+    const Params* params;      // [K] parameters of token k (positions, step_dev and rope_cs point at entry k below)
+    const uint32_t* steps;     // [K] step number of token k
+};
+
+__global__ void kl_token_plan_kernel(const __grid_constant__ Params p, Params* params, uint32_t* steps, int32_t* pos_arr,
+                                     float* rope_arr, uint32_t K) {
+    const uint32_t step0 = *p.step_dev;
+    const int32_t pos0 = p.positions[0];
+    if (pos0 < 0 || (uint32_t)pos0 + K > p.max_ctx) {   // every position of the launch has to be inside the cache
+        if (threadIdx.x == 0) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+        return;
+    }
+    for (uint32_t k = threadIdx.x; k < K; k += blockDim.x) {
+        steps[k] = step0 + k;
+        pos_arr[k] = pos0 + (int32_t)k;
+        Params q = p;
+        q.positions = pos_arr + k;
+        q.step_dev = steps + k;
+        q.rope_cs = rope_arr + (size_t)k * p.hd;
+        params[k] = q;
+    }
+    const uint32_t half = p.hd / 2;
+    for (uint32_t i = threadIdx.x; i < K * half; i += blockDim.x) {
+        const uint32_t k = i / half, j = i % half;
+        double sn, cs;
+        sincos((double)(pos0 + (int32_t)k) * p.inv_freq[j], &sn, &cs);
+        rope_arr[(size_t)k * p.hd + 2 * j] = (float)cs;
+        rope_arr[(size_t)k * p.hd + 2 * j + 1] = (float)sn;
+    }
+}
+
+__device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, uint32_t cta, const TokenLoopParams& t) {
+    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+    for (uint32_t k = 0; k < t.K && !r.aborted; ++k) {
+        const AttnUnit u = attn_unit(t.params[k], cta);
+        for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
+            const size_t lo = (size_t)l * p.layer_stride;
+            produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
+            if (k > 0 && l == 0) {
+                // The cache rows of the previous token are read by this token's copies: none is requested before the
+                // previous token is complete in every CTA, which the first word of this token's embedding says (it
+                // keeps its tag until the first down projection of this token, which cannot start before this point
+                // has been passed in every CTA).  Weight tiles do not wait: the ring is full of them by now.
+                const uint32_t want = tag_from(__ldg(t.steps + k), p.L, 0, TG_NEXT);
+                PollGuard g = {0ull, 0u, 700};
+                while (ld_tw(p.xa).tag != want) {
+                    if (!poll_continue(p, s, g)) {
+                        r.aborted = true;
+                        break;
+                    }
+                }
+                __threadfence();
+                asm volatile("fence.proxy.async;" ::: "memory");
+                if (r.aborted) break;
+            }
+            produce_attention(p, s, r, u, l);
+            produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+            produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
+            produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+        }
+        if (!r.aborted) produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
+    }
+    produce_drain(p, s, r);
+}
+
+// Sampling at the end of token k, out of line (once per token; inlined, its address arithmetic would be hoisted out of
+// the loop over tokens and held in registers through the stage code).  Every CTA reduces the logits rows it has just
+// produced; the CTA that draws the token's last ticket reduces the per-CTA results, records the token and writes the
+// next embedding.  false: that was the last token of the launch, or a wait gave up.
+__device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const TokenLoopParams& t, const uint32_t k,
+                                          uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane) {
+    auto tk = [&]() -> uint32_t { return k; };
+    const uint32_t step = __ldg(p.step_dev) + k;   // read once, here: the last CTA of the last token advances the word below
+    auto tstep = [&]() -> uint32_t { return step; };
+    auto tfinal = [&]() -> bool { return k + 1u == t.K; };
+    // ---- greedy sampling: this CTA's rows first
+    const GemvPlan& plm = p.plan[PL_LM];
+    asm volatile("fence.proxy.async;" ::: "memory");   // the cache rows this thread appended: readable by later bulk copies
+    consumer_bar();
+    float* sv = s.unit_part;                                           // [NCW] maxima, then [NCW] indices, then flags
+    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part) + NCW;
+    // [0] this CTA drew the last ticket, [1] token, [2] position, [4] stop: a wait of this launch gave up
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part) + 2 * NCW;
+    const CtaRange cr = cta_units(plm, cta, p.P);
+    const uint32_t r0 = cr.u0 * plm.rpc, r1 = min(cr.u1 * plm.rpc, p.V);
+    float bv = -INFINITY;
+    uint32_t bi = 0xffffffffu;
+    for (uint32_t i = r0 + ctid; i < r1; i += NCT) argmax_merge(bv, bi, p.logits[i], i);
+    for (int o = 16; o > 0; o >>= 1)
+        argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
+    if (lane == 0) {
+        sv[warp] = bv;
+        si[warp] = bi;
+    }
+    consumer_bar();
+    if (ctid == 0) {
+        for (uint32_t w = 1; w < (uint32_t)NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
+        t.t.part_val[cta] = bv;
+        t.t.part_idx[cta] = bi;
+        sh[0] = (atom_add_acq_rel(t.t.ticket, 1u) == p.P * (tk() + 1u) - 1u) ? 1u : 0u;
+        sh[4] = (*s.abort_flag != 0 || __ldcg(p.status) != 0) ? 1u : 0u;
+    }
+    consumer_bar();
+    const bool last_cta = sh[0] != 0u, stop = sh[4] != 0u;
+    if (last_cta) {
+        // all logits of this token are written.  Next token, next position, the next embedding.
+        if (warp == 0) {
+            bv = -INFINITY;
+            bi = 0xffffffffu;
+            for (uint32_t j = lane; j < p.P; j += 32) argmax_merge(bv, bi, __ldcg(t.t.part_val + j), __ldcg(t.t.part_idx + j));
+            for (int o = 16; o > 0; o >>= 1)
+                argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
+            if (lane == 0) {
+                const uint32_t tok = bi == 0xffffffffu ? 0u : bi;
+                const int32_t pos = __ldg(t.params[tk()].positions) + 1;
+                t.t.tokens[0] = (int32_t)tok;
+                t.t.positions[0] = pos;
+                t.out_tokens[tk()] = (int32_t)tok;
+                if (tfinal() || stop) *p.step_dev = tstep() + 1u;
+                if (tfinal() || stop) *t.t.ticket = 0u;   // ready for the next launch
+                if (tfinal() && pos >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+                sh[1] = tok;
+                sh[2] = (uint32_t)pos;
+            }
+        }
+        consumer_bar();
+        if (tfinal() || stop) {   // what the next launch needs: hidden state kept, rotary table, counters at zero
+            for (uint32_t i = ctid; i < p.H; i += NCT) t.t.hidden[i] = ld_tw(p.xa + i).v;
+            for (uint32_t i = ctid; i < p.hd / 2; i += NCT) {
+                double sn, cs;
+                sincos((double)sh[2] * p.inv_freq[i], &sn, &cs);
+                p.rope_cs[2 * i] = (float)cs;
+                p.rope_cs[2 * i + 1] = (float)sn;
+            }
+            for (uint32_t i = ctid; i < p.L; i += NCT) p.counters[i] = 0u;
+            consumer_bar();
+        }
+        const __nv_bfloat16* row = p.embed + (size_t)sh[1] * p.H;
+        // the next launch expects the usual tag, the next token of this launch the one of its own
+        const uint32_t xtag = tag_from(tstep() + 1u, p.L, 0, tfinal() || stop ? (uint32_t)TG_XA : TG_NEXT);
+        __threadfence();   // release side of the token boundary (see the fence behind the first load_vec)
+        for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
+    }
+    consumer_bar();   // the flags above are read before the next stage reuses the area
+    return !stop && !tfinal();
+}
+
+
+// Token k of the launch on the consumer warps; false: it was the last one (or a wait gave up).  The step number (for the
+// tags) and the parameter copy of the token are fetched where they are needed rather than kept, so that the loop over
+// tokens costs the stage code no registers: k itself is uniform.
+__device__ __forceinline__ bool consume_token(const Params& p, const Smem& s, const TokenLoopParams& t, const uint32_t k,
+                                              uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
+                                              WarpRing& wr) {
+    auto tk = [&]() -> uint32_t { return k; };
+    auto tstep = [&]() -> uint32_t { return __ldg(p.step_dev) + k; };   // the word changes behind the launch's last token only
+    auto tfinal = [&]() -> bool { return k + 1u == t.K; };
+    // ---- the decoder layers, and the classifier as the only stage of a layer behind them (one copy of the stage code:
+    // a second one behind the loop would have its loop-invariant values held in registers through the first)
+    for (uint32_t l = 0; l <= p.L; ++l) {
+        const size_t lo = (size_t)l * p.layer_stride;
+        const bool cls = l == p.L;
+        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st) {
+            GemvOut out = {nullptr, nullptr, nullptr, 0u};
+            int plan = PL_QKV, ep = EP_STORE;
+            const float* xsrc = nullptr;
+            float xscale = 1.f;
+            if (st == ST_QKV) {
+                xscale = load_vec(p, s, p.xa, p.H, tag_from(tstep(), p.L, l, tk() > 0 && l == 0 ? TG_NEXT : (uint32_t)TG_XA), true,
+                                  cls ? p.gf : p.g1 + lo, ctid);
+                if (cls) {
+                    out = {nullptr, p.logits, nullptr, 0u};
+                    plan = PL_LM;
+                } else {
+                    out = {p.qkv, nullptr, nullptr, tag_from(tstep(), p.L, l, TG_QKV)};
+                }
+            } else if (st == ST_ATTN) {
+                attention_block(tk() == 0 ? p : t.params[tk()], s, l, cta, ctid, warp, lane, rc, wr);
+                continue;
+            } else if (st == ST_O) {
+                load_vec(p, s, p.o, p.QD, tag_from(tstep(), p.L, l, TG_O), false, nullptr, ctid);
+                out = {p.xb, nullptr, p.xa, tag_from(tstep(), p.L, l, TG_XB)};
+                plan = PL_O;
+                ep = EP_RESIDUAL;
+            } else if (st == ST_GU) {
+                xscale = load_vec(p, s, p.xb, p.H, tag_from(tstep(), p.L, l, TG_XB), true, p.g2 + lo, ctid);
+                out = {nullptr, p.h, nullptr, 0u};
+                plan = PL_GU;
+                ep = EP_SWIGLU;
+            } else {
+                stage_wait(p, s, p.counters + l, p.P * (tk() + 1u), ctid);
+                out = {p.xa, nullptr, p.xb, tag_from(tstep(), p.L, l + 1, TG_XA)};
+                plan = PL_D;
+                ep = EP_RESIDUAL;
+                xsrc = p.h;
+            }
+            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+            if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
+        }
+    }
+    return sample_token(p, s, t, k, cta, ctid, warp, lane);
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1) kl_token_loop_kernel(const __grid_constant__ Params p,
+                                                                    const __grid_constant__ TokenLoopParams t) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, p);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    if (tid == 0) {
+        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    __syncthreads();
+    if (*p.status != 0) return;
+    if (warp == NCW) {
+        if (lane == 0) produce_tokens(p, s, cta, t);
+        return;
+    }
+    WarpRing wr = ring_begin();
+    const uint32_t ctid = tid;
+    RingCursor rc = {0u, 0u};
+
+#pragma unroll 1
+    for (uint32_t k = 0; consume_token(p, s, t, k, cta, ctid, warp, lane, rc, wr); ++k) {}
+}
+
 }  // namespace kl
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -465,6 +715,12 @@ struct kl_handle {
     uint32_t* tok_idx;     // [P]
     uint32_t* tok_ticket;
     int token_ok;          // kl_token_kernel can be resident
+    int loop_ok;           // kl_token_loop_kernel can be resident
+    Params* plan_params;   // [TOKENS_PER_LAUNCH] per-token parameter copies of kl_token_loop_kernel, written by kl_token_plan_kernel
+    uint32_t* plan_steps;  // [TOKENS_PER_LAUNCH]
+    int32_t* plan_pos;     // [TOKENS_PER_LAUNCH]
+    int32_t* plan_out;     // [TOKENS_PER_LAUNCH] picked tokens of the host-buffer entry point
+    float* plan_rope;      // [TOKENS_PER_LAUNCH][head_dim]
     uint32_t* argmax_idx;
     uint32_t* argmax_tickets;
     uint64_t launches;
@@ -482,6 +738,7 @@ struct kl_handle {
 namespace {
 
 constexpr size_t ALIGN = 256;
+constexpr size_t TOKENS_PER_LAUNCH = 256;   // most tokens one launch of kl_token_loop_kernel decodes
 inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
 inline uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
 
@@ -490,7 +747,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, stplan, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
     uint32_t bsplit[5];
     uint32_t cps;
 };
@@ -576,6 +833,8 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
     y.shid = s;      s += align_up((B > 1 ? 32 : B) * H * 4);
     y.stokp = s;     s += align_up((size_t)num_sms * 8 + ALIGN);
+    y.stplan = s;    s += align_up(TOKENS_PER_LAUNCH * align_up(sizeof(Params))) + 3 * align_up(TOKENS_PER_LAUNCH * 4) +
+                          align_up((size_t)TOKENS_PER_LAUNCH * d.head_dim * 4);
     // batched path (max_batch > 1): operand, partial sums, queries, attention partials
     {
         const size_t QR = QD + 2 * KVD;
@@ -901,6 +1160,10 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
         h->token_ok = cudaFuncSetAttribute(kl_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) == cudaSuccess &&
                       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
+        h->loop_ok = h->token_ok &&
+                     cudaFuncSetAttribute(kl_token_loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) == cudaSuccess &&
+                     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_loop_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+        (void)cudaGetLastError();
     }
     int occ = 0;
     if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes);
@@ -930,6 +1193,11 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->tok_val = (float*)(sc + y.stokp);
     h->tok_idx = (uint32_t*)(h->tok_val + sms);
     h->tok_ticket = h->tok_idx + sms;
+    h->plan_params = (Params*)(sc + y.stplan);
+    h->plan_steps = (uint32_t*)(sc + y.stplan + align_up(TOKENS_PER_LAUNCH * align_up(sizeof(Params))));
+    h->plan_pos = (int32_t*)((uint8_t*)h->plan_steps + align_up(TOKENS_PER_LAUNCH * 4));
+    h->plan_out = (int32_t*)((uint8_t*)h->plan_pos + align_up(TOKENS_PER_LAUNCH * 4));
+    h->plan_rope = (float*)((uint8_t*)h->plan_out + align_up(TOKENS_PER_LAUNCH * 4));
     h->hidden_is_copy = 0;
     h->chain_tok = nullptr;
     h->last_batch = 1;
@@ -1324,19 +1592,10 @@ static bool replay_batched(kl_handle* h, const int32_t* tokens_d, const int32_t*
     return false;
 }
 
-kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
-                           uint32_t batch, int restart, void* stream) {
-    if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
-    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
-    if (batch > 1 || !h->token_ok) {
-        // batches (and devices on which the one-launch kernel cannot be resident): the step, then the sampling kernel
-        kl_status rc = KL_OK;
-        if (!replay_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, as_stream(stream)))
-            rc = kl_decode_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, stream);
-        return rc != KL_OK ? rc : kl_argmax_advance(h, logits_d, tokens_d, positions_d, batch, stream);
-    }
-    if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
-    cudaStream_t st = as_stream(stream);
+// Parameters of a batch-1 launch that samples on the device; starts a chain (embedding, rotary table, step counter as
+// in kl_decode_step; sampling ticket at zero) unless the latest launch already prepared this token buffer's next step.
+static kl_status token_chain_params(kl_handle* h, Params* out, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d,
+                                    float* logits_d, int restart, cudaStream_t st) {
     Params p = h->prm;
     p.B = 1;
     p.b0 = 0;
@@ -1354,11 +1613,32 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
         if (trc != KL_OK) return trc;
         p.attn_tc = 1;
     }
-    if (restart || h->chain_tok != tokens_d) {   // a chain starts: embedding, rotary table and step counter as in kl_decode_step
+    if (restart || h->chain_tok != tokens_d) {
+        if (cudaMemsetAsync(h->tok_ticket, 0, 4, st) != cudaSuccess) return KL_ERR_CUDA;   // a launch that gave up may have left it anywhere
         kl_embed_kernel<<<1, 256, 0, st>>>(p);
         if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
         ++h->launches;
     }
+    *out = p;
+    return KL_OK;
+}
+
+kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                           uint32_t batch, int restart, void* stream) {
+    if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    if (batch > 1 || !h->token_ok) {
+        // batches (and devices on which the one-launch kernel cannot be resident): the step, then the sampling kernel
+        kl_status rc = KL_OK;
+        if (!replay_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, as_stream(stream)))
+            rc = kl_decode_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, stream);
+        return rc != KL_OK ? rc : kl_argmax_advance(h, logits_d, tokens_d, positions_d, batch, stream);
+    }
+    if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
+    cudaStream_t st = as_stream(stream);
+    Params p;
+    const kl_status prc = token_chain_params(h, &p, tokens_d, positions_d, kv_cache_d, logits_d, restart, st);
+    if (prc != KL_OK) return prc;
     TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all};
     void* args[] = {&p, &t};
     const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
@@ -1366,6 +1646,57 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     h->last_batch = 1;
     h->hidden_is_copy = 1;
     h->chain_tok = tokens_d;
+    return KL_OK;
+}
+
+kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                                  int32_t* out_tokens_d, uint32_t n_tokens, uint32_t batch, int restart, void* stream) {
+    if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d || !out_tokens_d) return KL_ERR_INVALID_ARG;
+    if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (batch > 1 || !h->loop_ok) {
+        // batches: token after token (each step replayed from the handle's graph), the picked tokens copied out
+        for (uint32_t k = 0; k < n_tokens; ++k) {
+            const kl_status rc = kl_decode_greedy(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, restart && k == 0, stream);
+            if (rc != KL_OK) return rc;
+            if (cudaMemcpyAsync(out_tokens_d + (size_t)k * batch, tokens_d, (size_t)batch * 4, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                return KL_ERR_CUDA;
+        }
+        return KL_OK;
+    }
+    if (!all_loaded(h)) return KL_ERR_NOT_LOADED;
+    for (uint32_t done = 0; done < n_tokens;) {
+        const uint32_t K = n_tokens - done < TOKENS_PER_LAUNCH ? n_tokens - done : (uint32_t)TOKENS_PER_LAUNCH;
+        Params p;
+        const kl_status prc = token_chain_params(h, &p, tokens_d, positions_d, kv_cache_d, logits_d, restart && done == 0, st);
+        if (prc != KL_OK) return prc;
+        kl_token_plan_kernel<<<1, 256, 0, st>>>(p, h->plan_params, h->plan_steps, h->plan_pos, h->plan_rope, K);
+        if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
+        ++h->launches;
+        TokenLoopParams t = {{tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all},
+                             out_tokens_d + done, K, h->plan_params, h->plan_steps};
+        void* args[] = {&p, &t};
+        const kl_status rc = launch_persistent(h, (const void*)kl_token_loop_kernel, args, st);
+        if (rc != KL_OK) return rc;
+        h->last_batch = 1;
+        h->hidden_is_copy = 1;
+        h->chain_tok = tokens_d;
+        done += K;
+    }
+    return KL_OK;
+}
+
+kl_status kl_decode_greedy_tokens_host(kl_handle* h, int32_t token, int32_t position, void* kv_cache_d, int32_t* out_tokens_h,
+                                       uint32_t n_tokens, void* stream) {
+    if (!h || !kv_cache_d || !out_tokens_h || n_tokens == 0 || n_tokens > TOKENS_PER_LAUNCH) return KL_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(h->stage_tokens, &token, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+    if (cudaMemcpyAsync(h->stage_positions, &position, 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return KL_ERR_CUDA;
+    int32_t* out_d = h->plan_out;
+    const kl_status rc = kl_decode_greedy_tokens(h, h->stage_tokens, h->stage_positions, kv_cache_d, h->stage_logits, out_d, n_tokens, 1, 1, stream);
+    if (rc != KL_OK) return rc;
+    if (cudaMemcpyAsync(out_tokens_h, out_d, (size_t)n_tokens * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return KL_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KL_ERR_CUDA;
     return KL_OK;
 }
 

@@ -567,6 +567,119 @@ def test_one_launch_per_token_edge_cases():
     dec.close()
 
 
+@pytest.mark.parametrize("name", ["tiny", "odd_rows_hd128", "llama31_8b_4layers", "llama32_3b_2layers_bias"])
+def test_tokens_per_launch_match_the_chain_of_single_launches(name):
+    """kl_decode_greedy_tokens at batch 1 (the loop over layers extended to a loop over tokens: K tokens in one launch)
+    gives the bits of K chained one-token launches: picked tokens, final token / position, logits and hidden state of
+    the last step, cache.  A second call continues the chain (restart = 0), a one-token launch continues that, and the
+    host-buffer entry point returns the same tokens."""
+    import dataclasses
+    shape, ctx, K = {"tiny": (gen.TINY, 128, 9), "odd_rows_hd128": (SHAPES["odd_rows_hd128"], 150, 5),
+                     "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 1024, 6),
+                     "llama32_3b_2layers_bias": (dataclasses.replace(LLAMA32_3B_2L, qkv_bias=True), 0, 7)}[name]
+    total = 2 * K + 1
+    dec = helpers.make_decoder(shape, 1, ctx + total + 8, 0)
+    cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + total + 8, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+    pos0 = torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    # K + K + 1 chained one-token launches
+    ref_cache, tok, pos = cache0.clone(), tok0.clone(), pos0.clone()
+    logits, hid = torch.empty(1, shape.vocab, device="cuda"), torch.empty(1, shape.hidden, device="cuda")
+    want, want_logits, want_hid = [], [], []
+    for step in range(total):
+        dec.kl_decode_greedy(tok, pos, ref_cache, logits, 1, step == 0)
+        dec.kl_read_hidden(hid, 1)
+        want.append(int(tok[0]))
+        want_logits.append(logits.clone())
+        want_hid.append(hid.clone())
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    # the same as K tokens in one launch, K more in a second one, and a one-token launch behind them
+    cache, tok1, pos1 = cache0.clone(), tok0.clone(), pos0.clone()
+    logits1, hid1 = torch.empty(1, shape.vocab, device="cuda"), torch.empty(1, shape.hidden, device="cuda")
+    out = torch.full((total,), -1, dtype=torch.int32, device="cuda")
+    n0 = dec.kl_launch_count()
+    dec.kl_decode_greedy_tokens(tok1, pos1, cache, logits1, out, K, 1, True)
+    assert dec.kl_launch_count() - n0 == 3            # embedding, the per-token table, the one kernel
+    dec.kl_read_hidden(hid1, 1)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    assert out[:K].tolist() == want[:K] and int(tok1[0]) == want[K - 1] and int(pos1[0]) == ctx + K
+    assert torch.equal(logits1, want_logits[K - 1]) and torch.equal(hid1, want_hid[K - 1])
+    n0 = dec.kl_launch_count()
+    dec.kl_decode_greedy_tokens(tok1, pos1, cache, logits1, out[K:], K, 1, False)
+    assert dec.kl_launch_count() - n0 == 2            # the chain goes on: no embedding launch
+    dec.kl_decode_greedy(tok1, pos1, cache, logits1, 1, False)
+    dec.kl_read_hidden(hid1, 1)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    assert out[:2 * K].tolist() == want[:2 * K] and int(tok1[0]) == want[-1] and int(pos1[0]) == ctx + total
+    assert torch.equal(logits1, want_logits[-1]) and torch.equal(hid1, want_hid[-1])
+    assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    # host buffers
+    cache2 = cache0.clone()
+    out_h = torch.empty(K, dtype=torch.int32).pin_memory()
+    dec.kl_decode_greedy_tokens_host(int(tok0[0]), ctx, cache2, out_h, K)
+    assert dec.kl_last_status() == binding.KL_OK
+    assert out_h.tolist() == want[:K]
+    dec.close()
+
+
+def test_tokens_per_launch_edge_cases():
+    """K tokens per launch against the oracle from an empty cache; a run that would leave the cache is refused on the
+    device before anything is decoded; a run that ends exactly at the last position succeeds and reports the full
+    cache; batches go through the step-by-step path with the same interface."""
+    shape = gen.TINY
+    K, max_ctx = 6, 16
+    host = helpers.HostWeights(shape, 0)
+    from oracle import kl_oracle as ko
+    orc = ko.Oracle(shape, max_ctx, host.layer, host.globals())
+    cache_or = gen.make_kv_cache(shape, 1, 0, max_ctx, 0, "cpu").view(torch.uint16).numpy().copy()
+    dec = helpers.make_decoder(shape, 2, max_ctx, 0)
+    cache = gen.make_kv_cache(shape, 1, 0, max_ctx, 0, "cuda")
+    tok = gen.make_tokens(shape, 1, 0).cuda()
+    pos = torch.zeros(1, dtype=torch.int32, device="cuda")
+    logits = torch.empty(1, shape.vocab, device="cuda")
+    out = torch.full((max_ctx,), -1, dtype=torch.int32, device="cuda")
+    t, p, want = [int(tok[0])], [0], []
+    for step in range(K):
+        hidden, ref_logits, nxt = orc.step(cache_or, t, p)
+        want.append(int(nxt[0]))
+        t, p = [int(nxt[0])], [step + 1]
+    dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, K, 1, True)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    assert out[:K].tolist() == want and int(pos[0]) == K
+    assert helpers.rel_l2(logits.cpu().numpy()[0], ref_logits[0]) <= helpers.REL_L2_TOL
+    # position K, max_ctx - K + 1 more tokens: one too many
+    before = cache.clone()
+    dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, max_ctx - K + 1, 1, False)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE
+    assert int(pos[0]) == K and torch.equal(cache.view(torch.uint16), before.view(torch.uint16))
+    # exactly to the end of the cache
+    dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, max_ctx - K, 1, True)
+    torch.cuda.synchronize()
+    assert int(pos[0]) == max_ctx
+    assert dec.kl_last_status() == binding.KL_ERR_OUT_OF_RANGE   # the cache is full
+    # a batch: the same interface, one step after the other
+    cache_b0 = gen.make_kv_cache(shape, 2, 5, max_ctx, 1, "cuda")
+    tok_b0 = gen.make_tokens(shape, 2, 1).cuda()
+    pos_b0 = torch.tensor([5, 2], dtype=torch.int32, device="cuda")
+    logits_b = torch.empty(2, shape.vocab, device="cuda")
+    ref_cache, tok_b, pos_b, want_b = cache_b0.clone(), tok_b0.clone(), pos_b0.clone(), []
+    for _ in range(4):
+        dec.kl_decode_greedy(tok_b, pos_b, ref_cache, logits_b, 2, False)
+        want_b.append(tok_b.clone())
+    cache_b, tok_b, pos_b = cache_b0.clone(), tok_b0.clone(), pos_b0.clone()
+    out_b = torch.empty(4, 2, dtype=torch.int32, device="cuda")
+    dec.kl_decode_greedy_tokens(tok_b, pos_b, cache_b, logits_b, out_b, 4, 2, True)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    assert torch.equal(out_b, torch.stack(want_b)) and torch.equal(cache_b.view(torch.uint16), ref_cache.view(torch.uint16))
+    dec.close()
+
+
 def test_greedy_chain_of_a_batch_replays_the_cached_graph():
     """kl_decode_greedy for a batch: kl_decode_step + kl_argmax_advance with the step replayed from the graph the handle
     keeps per set of buffers -- same tokens, logits and cache as the two calls made one by one, also after the buffers
