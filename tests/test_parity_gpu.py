@@ -625,6 +625,41 @@ def test_tokens_per_launch_match_the_chain_of_single_launches(name):
     dec.close()
 
 
+@pytest.mark.parametrize("name,n_tokens", [("tiny", 700), ("llama31_8b_4layers", 300)])
+def test_tokens_per_launch_long_runs(name, n_tokens):
+    """Runs longer than one launch holds (256 tokens): the call cuts them into launches that continue one another.  The
+    tiny shape is the hard case for the token boundary inside a launch -- a whole token's weight tiles fit into the
+    rings, so the copies of a token are requested while the previous token is still being computed and only the wait
+    of the producer threads keeps them from reading cache rows that are not written yet."""
+    import dataclasses
+    shape, ctx = {"tiny": (gen.TINY, 40), "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 512)}[name]
+    dec = helpers.make_decoder(shape, 1, ctx + n_tokens + 8, 0)
+    cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + n_tokens + 8, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+    pos0 = torch.tensor([ctx], dtype=torch.int32, device="cuda")
+    ref_cache, tok, pos = cache0.clone(), tok0.clone(), pos0.clone()
+    logits = torch.empty(1, shape.vocab, device="cuda")
+    want = torch.empty(n_tokens, dtype=torch.int32, device="cuda")
+    for step in range(n_tokens):
+        dec.kl_decode_greedy(tok, pos, ref_cache, logits, 1, step == 0)
+        want[step] = tok[0]
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    for attempt in range(2):
+        cache, tok1, pos1 = cache0.clone(), tok0.clone(), pos0.clone()
+        logits1 = torch.empty(1, shape.vocab, device="cuda")
+        out = torch.full((n_tokens,), -1, dtype=torch.int32, device="cuda")
+        n0 = dec.kl_launch_count()
+        dec.kl_decode_greedy_tokens(tok1, pos1, cache, logits1, out, n_tokens, 1, True)
+        torch.cuda.synchronize()
+        assert dec.kl_launch_count() - n0 == 1 + 2 * ((n_tokens + 255) // 256)
+        assert dec.kl_last_status() == binding.KL_OK
+        assert torch.equal(out, want), (attempt, int((out != want).nonzero()[0]))
+        assert int(pos1[0]) == ctx + n_tokens and torch.equal(logits1, logits)
+        assert torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
+    dec.close()
+
+
 def test_tokens_per_launch_edge_cases():
     """K tokens per launch against the oracle from an empty cache; a run that would leave the cache is refused on the
     device before anything is decoded; a run that ends exactly at the last position succeeds and reports the full
