@@ -306,7 +306,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_cons
     const uint32_t ctid = tid;
     RingCursor rc = {0u, 0u};
     // ---- the decoder layers: the stage sequence of kl_decoder_kernel (kept as a copy so that the looped kernel's
-    // own code stays exactly as tuned)
+    // own code stays exactly as tuned), and the classifier as the only stage of one more pass: one more stage on the
+    // same ring, and ONE copy of the stage code (a second one behind the loop would have its loop-invariant values held
+    // in registers through the first)
     for (uint32_t l = 0; l <= p.L; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         const bool cls = l == p.L;
@@ -1821,6 +1823,7 @@ kl_status kl_last_status(kl_handle* h) {
     if (v != 0) {
         const int32_t zero = 0;
         if (cudaMemcpy(h->prm.status, &zero, 4, cudaMemcpyHostToDevice) != cudaSuccess) return KL_ERR_CUDA;
+        h->chain_tok = nullptr;   // whatever a chain of kl_decode_greedy had prepared is not to be trusted: the next call starts one
     }
     return (kl_status)v;
 }

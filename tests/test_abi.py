@@ -70,6 +70,9 @@ def test_null_handle_calls_are_rejected(lib):
     assert lib.kl_set_mode(None, 0) == binding.KL_ERR_INVALID_ARG
     assert lib.kl_decode_step(None, None, None, None, None, 1, None) == binding.KL_ERR_INVALID_ARG
     assert lib.kl_last_status(None) == binding.KL_ERR_INVALID_ARG
+    assert lib.kl_decode_greedy(None, None, None, None, None, 1, 1, None) == binding.KL_ERR_INVALID_ARG
+    assert lib.kl_decode_greedy_tokens(None, None, None, None, None, None, 4, 1, 1, None) == binding.KL_ERR_INVALID_ARG
+    assert lib.kl_decode_greedy_tokens_host(None, 0, 0, None, None, 4, None) == binding.KL_ERR_INVALID_ARG
     assert lib.kl_kv_cache_bytes(None, 1) == 0
     assert lib.kl_launch_count(None) == 0
     lib.kl_destroy(None)
