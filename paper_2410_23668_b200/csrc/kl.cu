@@ -577,18 +577,18 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
 }
 
 
-// Token k of the launch on the consumer warps; false: it was the last one (or a wait gave up).  The step number (for the
-// tags) and the parameter copy of the token are fetched where they are needed rather than kept, so that the loop over
-// tokens costs the stage code no registers: k itself is uniform.
-__device__ __forceinline__ bool consume_token(const Params& p, const Smem& s, const TokenLoopParams& t, const uint32_t k,
-                                              uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
-                                              WarpRing& wr) {
+// All tokens of the launch on the consumer warps.  ONE loop over (token, layer) pairs, the classifier being the only
+// stage of a layer L behind the decoder layers and the sampling a call behind that: with a loop over tokens around the
+// loop over layers the compiler holds more in registers through the stage code (and a second copy of the stage code
+// for the classifier would have its loop-invariant values held through the first).  The step number (for the tags) and
+// the parameter copy of the token are fetched where they are needed rather than kept.
+__device__ __forceinline__ void consume_tokens(const Params& p, const Smem& s, const TokenLoopParams& t, uint32_t cta,
+                                               uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
+    uint32_t k = 0, l = 0;
     auto tk = [&]() -> uint32_t { return k; };
     auto tstep = [&]() -> uint32_t { return __ldg(p.step_dev) + k; };   // the word changes behind the launch's last token only
-    auto tfinal = [&]() -> bool { return k + 1u == t.K; };
-    // ---- the decoder layers, and the classifier as the only stage of a layer behind them (one copy of the stage code:
-    // a second one behind the loop would have its loop-invariant values held in registers through the first)
-    for (uint32_t l = 0; l <= p.L; ++l) {
+#pragma unroll 1
+    for (;;) {
         const size_t lo = (size_t)l * p.layer_stride;
         const bool cls = l == p.L;
         for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st) {
@@ -628,8 +628,14 @@ __device__ __forceinline__ bool consume_token(const Params& p, const Smem& s, co
             gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
             if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
         }
+        if (cls) {
+            if (!sample_token(p, s, t, k, cta, ctid, warp, lane)) break;
+            ++k;
+            l = 0;
+        } else {
+            ++l;
+        }
     }
-    return sample_token(p, s, t, k, cta, ctid, warp, lane);
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_loop_kernel(const __grid_constant__ Params p,
@@ -657,8 +663,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_token_loop_kernel(const __grid
     const uint32_t ctid = tid;
     RingCursor rc = {0u, 0u};
 
-#pragma unroll 1
-    for (uint32_t k = 0; consume_token(p, s, t, k, cta, ctid, warp, lane, rc, wr); ++k) {}
+    consume_tokens(p, s, t, cta, ctid, warp, lane, rc, wr);
 }
 
 }  // namespace kl
