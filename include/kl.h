@@ -81,23 +81,30 @@ typedef struct {
 } kl_model_desc;
 
 /* Sizes of the two device arenas the caller must provide to kl_create (both 256-byte aligned).
- * weight_bytes holds the library's own copy of every tensor, grouped per layer and laid out linearly in the
- * order the persistent kernel streams it (Section 3.2: grouped parameters [N x S], "linear in memory").
+ * weight_bytes holds the library's own copy of every tensor, grouped per layer (the [N x S] parameters that Eq. 3 /
+ * Group(p) of Section 3.2 yields) and stored as one contiguous run per layer in the order the persistent kernel
+ * streams it -- the second representation of grouped tensors that the end of Section 3.2 describes.
  * scratch_bytes holds activations, split-K attention partials, synchronisation counters, the status word and
  * staging buffers for the host-buffer entry point. */
 kl_status kl_workspace_bytes(const kl_model_desc* desc, size_t* weight_bytes, size_t* scratch_bytes);
 
 /* Creates a handle over caller-owned arenas (device pointers, sizes as reported by kl_workspace_bytes).
+ * The handle is the merged kernel's parameter list of Section 3.2 (rules (2)-(5) and Eq. 3): per-layer tensors become
+ * grouped parameters with a leading layer dimension and one constant layer stride, constants (shape, eps, RoPE base)
+ * are kept once.  Several handles may be alive at once (one stream each).
  * Uses the current CUDA device.  The scratch arena is cleared synchronously.  *out is set on success only. */
 kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scratch_arena_d, kl_handle** out);
 
 /* Copies one tensor into the weight arena (host or device source, any pageable/pinned/device memory), in the
- * library's streaming layout.  `bytes` must equal the tensor's size.  layer = -1 for KL_EMBED, KL_NORM_F,
+ * library's streaming layout: slot `layer` of a grouped parameter (Section 3.2, rule (3): a grouped parameter is indexed
+ * by the loop variable; the closing paragraph of that section: grouped tensors stored contiguously, in loop order).  `bytes` must equal the tensor's size.  layer = -1 for KL_EMBED, KL_NORM_F,
  * KL_LM_HEAD.  The copy is ordered on `stream`; the source may be released once the stream has passed it. */
 kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, size_t bytes, void* stream);
 
 /* Bytes of a KV cache for `batch` sequences: layout [n_layers][2 (K,V)][batch][n_kv_heads][max_ctx][head_dim]
- * bf16.  Cached keys are stored already rotated.  The cache is caller-owned and updated in place. */
+ * bf16.  The cache is read, written and live after the call, i.e. element (6) {In, Live, Out} of the lattice of
+ * Section 3.1: a grouped in/out parameter with a leading layer dimension (Eq. 3), sized as Table 1's KV column
+ * (batch x context x layers x 2 x kv heads x head size x 2 bytes).  Cached keys are stored already rotated.  The cache is caller-owned and updated in place. */
 size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch);
 
 /* KL_MODE_LOOPED (default): one persistent kernel runs all layers (4 launches per token with embedding, classifier
@@ -121,7 +128,11 @@ kl_status kl_set_mode(kl_handle* h, int mode);
  * kl_decode_step + kl_argmax_advance can be replayed step after step (same buffers).
  * Merged-call argument rule of Section 3.2: weights (grouped, all layers) come from the handle, the hidden
  * state enters once (from the embedding) and leaves once (kl_read_hidden / the classifier), the KV cache is the
- * grouped in/out parameter.  Device-detected errors make the step a no-op and are reported by kl_last_status. */
+ * grouped in/out parameter.  Device-detected errors are reported by kl_last_status.  KL_ERR_OUT_OF_RANGE (a bad
+ * token or position) is found before anything is written and makes the step a no-op.  KL_ERR_SYNC_TIMEOUT (a
+ * bounded wait ran out in the middle of the step) leaves the step's logits, its cache row and the hidden state
+ * undefined; the greedy entry points then leave tokens_d and positions_d as they were, and the next call starts a
+ * new chain. */
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                          float* logits_d, uint32_t batch, void* stream);
 
@@ -182,7 +193,9 @@ kl_status kl_decode_step_host(kl_handle* h, const int32_t* tokens_h, const int32
 kl_status kl_decode_greedy_host(kl_handle* h, const int32_t* tokens_h, const int32_t* positions_h, void* kv_cache_d,
                                 int32_t* next_tokens_h, uint32_t batch, void* stream);
 
-/* Sampling block (greedy): tokens_d[b] = argmax_v logits_d[b, v] (lowest index on ties); positions_d[b] += 1. */
+/* Sampling block, the last of the four calls per token of Section 2's looped schedule (Embedding, looped Decoder,
+ * Classifier, Sampling), as greedy sampling: tokens_d[b] = argmax_v logits_d[b, v] (lowest index on ties);
+ * positions_d[b] += 1. */
 kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens_d, int32_t* positions_d,
                             uint32_t batch, void* stream);
 
@@ -208,11 +221,16 @@ kl_status kl_argmax_advance(kl_handle* h, const float* logits_d, int32_t* tokens
 kl_status kl_argmax_advance_static(const float* logits_d, uint32_t vocab, int32_t* tokens_d, int32_t* positions_d,
                                    uint32_t batch, void* stream);
 
-/* Copies the hidden state after the last decoder layer (before the final RMSNorm) of the latest step:
+/* The hidden state is the loop-carried {In, Local} / {Local, Out} pair of the merged kernel: it lives in the kernel's
+ * own buffers for all L iterations and is stored once after the loop (Section 3.2, rules (6) and (10)); this call
+ * returns that single store.
+ * Copies the hidden state after the last decoder layer (before the final RMSNorm) of the latest step:
  * hidden_d [batch, hidden] fp32; batch must be the latest step's. */
 kl_status kl_read_hidden(kl_handle* h, float* hidden_d, uint32_t batch, void* stream);
 
-/* Synchronises nothing: call after the stream has been synchronised.  Reads and clears the device status word
+/* No counterpart in the paper (its kernels report no errors): the bounded device-side waits and the range checks of
+ * this library report through one status word.
+ * Synchronises nothing: call after the stream has been synchronised.  Reads and clears the device status word
  * (KL_OK, KL_ERR_SYNC_TIMEOUT or KL_ERR_OUT_OF_RANGE).  The word is sticky: once a step has set it, every later
  * step on the handle is a no-op until this call has read (and thereby cleared) it. */
 kl_status kl_last_status(kl_handle* h);
@@ -277,6 +295,14 @@ kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
  * NEXT kl_decode_step only, so the waits on them run out and the step reports KL_ERR_SYNC_TIMEOUT.  No fault, trap
  * or endless loop is involved. */
 kl_status kl_debug_skip_signal_once(kl_handle* h, int stage);
+
+/* Test hook for the step numbers behind the tags.  Every decoded token takes one step number; the tags hold 28 bits of
+ * (step x n_layers + layer), so after *wrap_at steps (about 2^28 / n_layers: 8.4 million tokens at 32 layers) the
+ * library clears its tagged scratch areas at the next launch boundary and starts numbering again at 1 -- a tagged word
+ * left over from the previous use of a number can therefore never be taken for a fresh one.  This call sets the
+ * counter (device word; synchronous; the stream must be idle) so that a test can step across the wrap;
+ * step = 0xffffffff only queries.  wrap_at may be NULL. */
+kl_status kl_debug_set_step(kl_handle* h, uint32_t step, uint32_t* wrap_at);
 
 const char* kl_status_string(kl_status s);
 

@@ -27,6 +27,28 @@ namespace kl {
 
 // ------------------------------------------------------------------------------------------------ kernels
 
+// Step numbers behind the tags.  A tag holds (step * L + layer) in 28 bits, so step numbers are reused after
+// 2^28 / L steps; a tagged word that is not rewritten in every step (a split-K slot above the current split count)
+// could then meet its own old tag.  Before that can happen -- when the next step number reaches step_wrap(L), at a
+// launch boundary -- every tagged area is cleared and the numbering restarts at 1.  The margin covers the steps one
+// launch may take without passing such a boundary (TOKENS_PER_LAUNCH) and the look-ahead of the tags (step + 1).
+constexpr uint32_t STEP_WRAP_MARGIN = 260u;
+__host__ __device__ __forceinline__ uint32_t step_wrap(uint32_t L) { return (1u << 28) / L - STEP_WRAP_MARGIN; }
+
+// All tagged words of the handle to zero (zero is no tag).  Called by every thread of ONE block at a launch boundary of
+// the chain: nothing else reads or writes these areas then.  The caller puts a block barrier behind it.
+__device__ __noinline__ void clear_tagged(const Params& p, uint32_t tid, uint32_t nthreads) {
+    const uint32_t nq = p.QD + 2u * p.KVD, npart = p.P * p.G * p.hd, nml = p.P * p.G * 2u;
+    for (uint32_t i = tid; i < p.H; i += nthreads) {
+        st_tw(p.xa + i, 0.f, 0u);
+        st_tw(p.xb + i, 0.f, 0u);
+    }
+    for (uint32_t i = tid; i < nq; i += nthreads) st_tw(p.qkv + i, 0.f, 0u);
+    for (uint32_t i = tid; i < p.QD; i += nthreads) st_tw(p.o + i, 0.f, 0u);
+    for (uint32_t i = tid; i < npart; i += nthreads) st_tw(p.part + i, 0.f, 0u);
+    for (uint32_t i = tid; i < nml; i += nthreads) st_tw(p.part_ml + i, 0.f, 0u);
+}
+
 __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
     const uint32_t b = 0u, tid = threadIdx.x;   // b: slot of the sequence in the scratch vectors
     int32_t tok = p.tokens[p.b0];
@@ -41,13 +63,15 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
     if (tok < 0 || tok >= (int32_t)p.V) tok = 0;
     const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
     // one more sequence on this handle: every tag of this launch sequence differs from all earlier ones
-    __shared__ uint32_t step_s;
-    if (tid == 0) {
-        step_s = *p.step_dev + 1u;
-        *p.step_dev = step_s;
+    uint32_t step = *p.step_dev + 1u;   // every thread reads the word; thread 0 writes it behind the barrier
+    const bool wrap = step >= step_wrap(p.L);
+    if (wrap) {
+        clear_tagged(p, tid, blockDim.x);
+        step = 1u;
     }
     __syncthreads();
-    const uint32_t xtag = tag_from(step_s, p.L, 0, TG_XA);
+    if (tid == 0) *p.step_dev = step;
+    const uint32_t xtag = tag_from(step, p.L, 0, TG_XA);
     for (uint32_t i = tid; i < p.H; i += blockDim.x) st_tw(p.xa + (size_t)b * p.H + i, __bfloat162float(row[i]), xtag);
     // RoPE table of this step: angle in double so that large positions keep their phase
     for (uint32_t i = tid; i < p.hd / 2; i += blockDim.x) {
@@ -61,19 +85,113 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
 }
 
 // The attention half of a layer as one call: RoPE, the unit's ring chunks, the merges, the deferred cache append.
-__device__ __noinline__ void attention_block(const Params& p, const Smem& s, uint32_t l, uint32_t cta, uint32_t ctid,
-                                             uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
+__device__ __noinline__ void attention_block(const Params& p, const Smem& s, const StepCtx& cx, uint32_t l, uint32_t cta,
+                                             uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
     if (p.attn_tc) {
-        attention_stage_and_advance<0>(p, s, l, cta, ctid, warp, lane, rc, wr);
+        attention_stage_and_advance<0>(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
     } else switch (p.G) {
-        case 1: attention_stage_and_advance<1>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-        case 2: attention_stage_and_advance<2>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-        case 4: attention_stage_and_advance<4>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
-        default: attention_stage_and_advance<8>(p, s, l, cta, ctid, warp, lane, rc, wr); break;
+        case 1: attention_stage_and_advance<1>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
+        case 2: attention_stage_and_advance<2>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
+        case 4: attention_stage_and_advance<4>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
+        default: attention_stage_and_advance<8>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
     }
     // the row written by this step is copied from the workspace to the cache here; the next vector load starts with
     // a CTA barrier, so the workspace is not overwritten before this copy has read it
-    attention_flush_new_row(p, s, l, cta, ctid);
+    attention_flush_new_row(p, s, cx, l, cta, ctid);
+}
+
+// Set-up every persistent kernel starts with: the ring's barriers, the abort flag, the unit table.  False: an earlier
+// kernel of this step flagged bad input and the launch is a no-op.
+__device__ __forceinline__ bool cta_begin(const Params& p, const Smem& s, uint32_t tid, const float* rope) {
+    if (tid == 0) {
+        // step number and position as the launch finds them: read before any CTA can have finished a token
+        s.ctx->step = ld_step(p.step_dev);
+        s.ctx->pos = (uint32_t)p.positions[p.b0];
+        s.ctx->rope_cs = rope;
+        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
+            mbar_init(smem_u32(&s.full[i]), 1);
+            mbar_init(smem_u32(&s.empty[i]), 1);
+        }
+        *s.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    __syncthreads();
+    return *p.status == 0;
+}
+
+// ONE stage of one layer on the consumer warps -- the only copy of the stage sequence; every persistent kernel calls
+// it from the single call site of its loop, so the GEMV loop is inlined into the kernel's own frame and the cold
+// parts (vector loads with their polls, the attention block) are calls made between stages, when nothing is live.
+//   l < L : stage st of decoder layer l (QKV, attention, O, gate/up, down)
+//   l == L: the classifier, as stage 0 of one more pass (one more stage on the same ring, same code)
+// xa_slot: tag slot under which the hidden state entering stage 0 was published (TG_XA; TG_NEXT for an embedding
+// written inside the running launch).  ctr_target: value of the layer's gate/up counter when all CTAs have signalled.
+__device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32_t l, uint32_t st,
+                                          uint32_t xa_slot, uint32_t ctr_target, uint32_t cta, uint32_t ctid, uint32_t warp,
+                                          uint32_t lane, RingCursor& rc, WarpRing& wr) {
+    const StepCtx& cx = *s.ctx;
+    const size_t lo = (size_t)l * p.layer_stride;
+    const bool cls = l == p.L;
+    // test hook: the results of one stage of layer 0 get a tag nobody waits for
+    const int skip = (l == 0) ? p.skip_stage : -1;
+    const uint32_t bad = 0x2u;
+    GemvOut out = {nullptr, nullptr, nullptr, 0u};
+    int plan = PL_QKV, ep = EP_STORE;
+    const float* xsrc = nullptr;
+    float xscale = 1.f;   // RMSNorm's normaliser of the stage's input vector, applied to the stage's outputs
+    if (st == ST_QKV) {
+        // RMSNorm + QKV projection (classifier: final RMSNorm + W_lm).  The poll on xa's tags is the wait for the
+        // previous layer (or the embedding).
+        trace_stamp(p, cta, l, 0, ctid);
+        xscale = load_vec(p, s, p.xa, p.H, tag_of(p, cx, l, xa_slot), true, cls ? p.gf : p.g1 + lo, ctid);
+        trace_stamp(p, cta, l, 1, ctid);
+        if (cls) {
+            out = {nullptr, p.logits, nullptr, 0u};
+            plan = PL_LM;
+        } else {
+            out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, cx, l, TG_QKV)};
+        }
+    } else if (st == ST_ATTN) {
+        trace_stamp(p, cta, l, 2, ctid);
+        // RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
+        attention_block(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
+        trace_stamp(p, cta, l, 4, ctid);
+        return;
+    } else if (st == ST_O) {
+        // output projection + residual (xa -> xb).  The poll on o's tags waits for the attention units.
+        load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, cx, l, TG_O), false, nullptr, ctid);
+        trace_stamp(p, cta, l, 6, ctid);
+        out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, cx, l, TG_XB)};
+        plan = PL_O;
+        ep = EP_RESIDUAL;
+    } else if (st == ST_GU) {
+        trace_stamp(p, cta, l, 7, ctid);
+        // RMSNorm + gate/up projections + SwiGLU
+        xscale = load_vec(p, s, p.xb, p.H, tag_of(p, cx, l, TG_XB), true, p.g2 + lo, ctid);
+        trace_stamp(p, cta, l, 9, ctid);
+        out = {nullptr, p.h, nullptr, 0u};
+        plan = PL_GU;
+        ep = EP_SWIGLU;
+    } else {
+        // down projection + residual (xb -> xa of the next layer).  h is plain fp32 read per warp and per column piece
+        // straight from L2 into registers (too wide for shared memory): its readiness is a counter, signalled with
+        // release at the end of the gate/up stage and awaited with acquire here
+        stage_wait(p, s, p.counters + l, ctr_target, ctid);
+        trace_stamp(p, cta, l, 12, ctid);
+        out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, cx, l + 1, TG_XA)};
+        plan = PL_D;
+        ep = EP_RESIDUAL;
+        xsrc = p.h;
+    }
+    gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+    if (st == ST_GU) {
+        stage_signal(p.counters + l, ctid, skip == ST_GU);
+        trace_stamp(p, cta, l, 10, ctid);
+    } else if (st == ST_D) {
+        trace_stamp(p, cta, l, 13, ctid);
+    }
 }
 
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
@@ -84,90 +202,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
-    if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
-        *s.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
-    __syncthreads();
-    if (*p.status != 0) return;  // an earlier kernel of this step flagged bad input: the step is a no-op
-
+    if (!cta_begin(p, s, tid, p.rope_cs)) return;   // an earlier kernel of this step flagged bad input: the step is a no-op
     if (warp == NCW) {
         // producer warp: one thread streams the CTA's chunk sequence into the ring
         if (lane == 0) produce_decoder(p, s, cta, l0, l1, sbeg, send);
         return;
     }
     WarpRing wr = ring_begin();
-
-    // ---------------- consumers
-    const uint32_t ctid = tid;
     RingCursor rc = {0u, 0u};
-    // One call site for the GEMV stage, inlined here: the hot loop lives in the kernel's own frame and the cold parts
-    // (vector loads with their polls, the attention block) are calls made between stages, when nothing is live.
-    for (uint32_t l = l0; l < l1; ++l) {
-        const size_t lo = (size_t)l * p.layer_stride;
-        // test hook: the results of one stage of layer 0 get a tag nobody waits for
-        const int skip = (l == 0) ? p.skip_stage : -1;
-        const uint32_t bad = 0x2u;
-        for (uint32_t st = sbeg; st < send; ++st) {
-            GemvOut out = {nullptr, nullptr, nullptr, 0u};
-            int plan = PL_QKV, ep = EP_STORE;
-            const float* xsrc = nullptr;
-            float xscale = 1.f;   // RMSNorm's normaliser of the stage's input vector, applied to the stage's outputs
-            if (st == ST_QKV) {
-                // RMSNorm + QKV projection.  The poll on xa's tags is the wait for the previous layer (or the
-                // embedding).
-                trace_stamp(p, cta, l, 0, ctid);
-                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, p.g1 + lo, ctid);
-                trace_stamp(p, cta, l, 1, ctid);
-                out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, l, TG_QKV)};
-                plan = PL_QKV;
-                ep = EP_STORE;
-            } else if (st == ST_ATTN) {
-                trace_stamp(p, cta, l, 2, ctid);
-                // RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
-                attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
-                trace_stamp(p, cta, l, 4, ctid);
-                continue;
-            } else if (st == ST_O) {
-                // output projection + residual (xa -> xb).  The poll on o's tags waits for the attention units.
-                load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, l, TG_O), false, nullptr, ctid);
-                trace_stamp(p, cta, l, 6, ctid);
-                out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, l, TG_XB)};
-                plan = PL_O;
-                ep = EP_RESIDUAL;
-            } else if (st == ST_GU) {
-                trace_stamp(p, cta, l, 7, ctid);
-                // RMSNorm + gate/up projections + SwiGLU
-                xscale = load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
-                trace_stamp(p, cta, l, 9, ctid);
-                out = {nullptr, p.h, nullptr, 0u};
-                plan = PL_GU;
-                ep = EP_SWIGLU;
-            } else {
-                // down projection + residual (xb -> xa of the next layer).  h is plain fp32 read per warp and per
-                // column piece straight from L2 into registers (too wide for shared memory): its readiness is a
-                // counter, signalled with release at the end of the gate/up stage and awaited with acquire here
-                stage_wait(p, s, p.counters + l, p.P, ctid);
-                trace_stamp(p, cta, l, 12, ctid);
-                out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, l + 1, TG_XA)};
-                plan = PL_D;
-                ep = EP_RESIDUAL;
-                xsrc = p.h;
-            }
-            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
-            if (st == ST_GU) {
-                stage_signal(p.counters + l, ctid, skip == ST_GU);
-                trace_stamp(p, cta, l, 10, ctid);
-            }
-        }
-        trace_stamp(p, cta, l, 13, ctid);
-    }
+    for (uint32_t l = l0; l < l1; ++l)
+        for (uint32_t st = sbeg; st < send; ++st) run_stage(p, s, l, st, TG_XA, p.P, cta, tid, warp, lane, rc, wr);
 }
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
@@ -175,27 +219,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const Smem s = carve_smem(smem_raw, p);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
-    if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
-        *s.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
-    __syncthreads();
-    if (*p.status != 0) return;
+    if (!cta_begin(p, s, tid, p.rope_cs)) return;
     if (warp == NCW) {
         if (lane == 0) produce_classifier(p, s, cta);
         return;
     }
     WarpRing wr = ring_begin();
     RingCursor rc = {0u, 0u};
-    const float xscale = load_vec(p, s, p.xa, p.H, tag_of(p, p.L, TG_XA), true, p.gf, tid);
-    const GemvOut out = {nullptr, p.logits, nullptr, 0u};
-    gemv_stage(p, s, p.plan[PL_LM], EP_STORE, out, cta, warp, lane, rc, wr, nullptr, xscale);
+    run_stage(p, s, p.L, ST_QKV, TG_XA, p.P, cta, tid, warp, lane, rc, wr);
 }
 
 // Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per
@@ -251,204 +282,42 @@ __global__ void __launch_bounds__(256) kl_argmax_kernel(const float* logits, uin
     }
 }
 
-// ------------------------------------------------------------------------------------------------ one launch per token
+// ------------------------------------------------------------------------------------------------ tokens per launch
 // The paper's looped schedule still pays four calls per token: embedding, the looped decoder, classifier, sampling
-// (Section 2).  kl_token_kernel is all four for one sequence: the decoder layers and the classifier as consecutive
-// stages of one persistent kernel (the ring runs on from the last down projection into W_lm), then greedy sampling --
-// every CTA reduces the logits rows it has just produced, the last CTA to finish (ticket) reduces the per-CTA results,
-// advances token and position, keeps the final hidden state for kl_read_hidden and writes the NEXT token's embedding,
-// rotary table and step counter, so that the next launch starts at its first layer at once.
-struct TokenParams {
-    int32_t* tokens;        // [1] in: the token this step decodes (already embedded); out: the next token
-    int32_t* positions;     // [1] advanced by one
-    float* part_val;        // [P] per-CTA maxima
-    uint32_t* part_idx;     // [P] and their indices
-    uint32_t* ticket;       // zero between launches
-    float* hidden;          // [H] final hidden state of this step
-};
-
-__device__ __forceinline__ void produce_token(const Params& p, const Smem& s, uint32_t cta) {
-    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
-    const AttnUnit u = attn_unit(p, cta);
-    for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
-        const size_t lo = (size_t)l * p.layer_stride;
-        produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
-        produce_attention(p, s, r, u, l);
-        produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
-        produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
-        produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
-    }
-    if (!r.aborted) produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
-    produce_drain(p, s, r);
-}
-
-__global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const TokenParams t) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, p);
-    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
-    if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
-        *s.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
-    __syncthreads();
-    if (*p.status != 0) return;
-    if (warp == NCW) {
-        if (lane == 0) produce_token(p, s, cta);
-        return;
-    }
-    WarpRing wr = ring_begin();
-    const uint32_t ctid = tid;
-    RingCursor rc = {0u, 0u};
-    // ---- the decoder layers: the stage sequence of kl_decoder_kernel (kept as a copy so that the looped kernel's
-    // own code stays exactly as tuned), and the classifier as the only stage of one more pass: one more stage on the
-    // same ring, and ONE copy of the stage code (a second one behind the loop would have its loop-invariant values held
-    // in registers through the first)
-    for (uint32_t l = 0; l <= p.L; ++l) {
-        const size_t lo = (size_t)l * p.layer_stride;
-        const bool cls = l == p.L;
-        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st) {
-            GemvOut out = {nullptr, nullptr, nullptr, 0u};
-            int plan = PL_QKV, ep = EP_STORE;
-            const float* xsrc = nullptr;
-            float xscale = 1.f;
-            if (st == ST_QKV) {
-                xscale = load_vec(p, s, p.xa, p.H, tag_of(p, l, TG_XA), true, cls ? p.gf : p.g1 + lo, ctid);
-                if (cls) {
-                    out = {nullptr, p.logits, nullptr, 0u};
-                    plan = PL_LM;
-                } else {
-                    out = {p.qkv, nullptr, nullptr, tag_of(p, l, TG_QKV)};
-                }
-            } else if (st == ST_ATTN) {
-                attention_block(p, s, l, cta, ctid, warp, lane, rc, wr);
-                continue;
-            } else if (st == ST_O) {
-                load_vec(p, s, p.o, p.QD, tag_of(p, l, TG_O), false, nullptr, ctid);
-                out = {p.xb, nullptr, p.xa, tag_of(p, l, TG_XB)};
-                plan = PL_O;
-                ep = EP_RESIDUAL;
-            } else if (st == ST_GU) {
-                xscale = load_vec(p, s, p.xb, p.H, tag_of(p, l, TG_XB), true, p.g2 + lo, ctid);
-                out = {nullptr, p.h, nullptr, 0u};
-                plan = PL_GU;
-                ep = EP_SWIGLU;
-            } else {
-                stage_wait(p, s, p.counters + l, p.P, ctid);
-                out = {p.xa, nullptr, p.xb, tag_of(p, l + 1, TG_XA)};
-                plan = PL_D;
-                ep = EP_RESIDUAL;
-                xsrc = p.h;
-            }
-            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
-            if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
-        }
-    }
-    // ---- greedy sampling: this CTA's rows first
-    consumer_bar();   // the rows this CTA stored are visible to all of its threads
-    const GemvPlan& pl = p.plan[PL_LM];
-    const CtaRange cr = cta_units(pl, cta, p.P);
-    const uint32_t r0 = cr.u0 * pl.rpc, r1 = min(cr.u1 * pl.rpc, p.V);
-    float bv = -INFINITY;
-    uint32_t bi = 0xffffffffu;
-    for (uint32_t i = r0 + ctid; i < r1; i += NCT) argmax_merge(bv, bi, p.logits[i], i);
-    for (int o = 16; o > 0; o >>= 1)
-        argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
-    float* sv = s.unit_part;                                           // [NCW] maxima, then [NCW] indices, then flags
-    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part) + NCW;
-    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part) + 2 * NCW;   // [0] last CTA, [1] token, [2] position, [3] step
-    if (lane == 0) {
-        sv[warp] = bv;
-        si[warp] = bi;
-    }
-    consumer_bar();
-    if (ctid == 0) {
-        for (uint32_t w = 1; w < (uint32_t)NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
-        t.part_val[cta] = bv;
-        t.part_idx[cta] = bi;
-        sh[0] = (atom_add_acq_rel(t.ticket, 1u) == p.P - 1u) ? 1u : 0u;
-    }
-    consumer_bar();
-    if (sh[0] == 0u) return;
-    // ---- the last CTA: all logits are written.  Next token, next position, and everything the next launch needs.
-    if (warp == 0) {
-        bv = -INFINITY;
-        bi = 0xffffffffu;
-        for (uint32_t j = lane; j < p.P; j += 32) argmax_merge(bv, bi, __ldcg(t.part_val + j), __ldcg(t.part_idx + j));
-        for (int o = 16; o > 0; o >>= 1)
-            argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
-        if (lane == 0) {
-            const uint32_t tok = bi == 0xffffffffu ? 0u : bi;
-            const int32_t pos = t.positions[0] + 1;
-            t.tokens[0] = (int32_t)tok;
-            t.positions[0] = pos;
-            *t.ticket = 0u;   // ready for the next launch
-            if (pos >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);   // the next step would leave the cache
-            sh[1] = tok;
-            sh[2] = (uint32_t)pos;
-            sh[3] = __ldg(p.step_dev) + 1u;
-        }
-    }
-    consumer_bar();
-    for (uint32_t i = ctid; i < p.H; i += NCT) t.hidden[i] = ld_tw(p.xa + i).v;   // before xa is overwritten below
-    consumer_bar();
-    const uint32_t tok = sh[1], pos = sh[2], step = sh[3];
-    const __nv_bfloat16* row = p.embed + (size_t)tok * p.H;
-    const uint32_t xtag = tag_from(step, p.L, 0, TG_XA);
-    for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
-    for (uint32_t i = ctid; i < p.hd / 2; i += NCT) {
-        double sn, cs;
-        sincos((double)pos * p.inv_freq[i], &sn, &cs);
-        p.rope_cs[2 * i] = (float)cs;
-        p.rope_cs[2 * i + 1] = (float)sn;
-    }
-    for (uint32_t i = ctid; i < p.L; i += NCT) p.counters[i] = 0u;
-    if (ctid == 0) *p.step_dev = step;
-}
-
-// ------------------------------------------------------------------------------------------------ K tokens per launch
-// The loop over layers extended to a loop over TOKENS: one launch decodes K consecutive tokens of one sequence.  What
-// changes from token to token inside the launch -- the position, the step number the tags are built from, the rotary
-// table -- is laid out beforehand, one entry per token, by kl_token_plan_kernel (the values are known: position and
-// step advance by one); entry k also holds a copy of the kernel parameters that points at them, which is what the
-// attention code (out of line, parameters by reference) is given for token k.  Counters that were zeroed between
+// (Section 2).  kl_token_kernel is all four for one sequence, and for K consecutive tokens: the decoder layers and the
+// classifier as consecutive stages of one persistent kernel (the ring runs on from the last down projection into
+// W_lm), then greedy sampling -- every CTA reduces the logits rows it has just produced, the CTA that draws the token's
+// last ticket reduces the per-CTA results, advances token and position and writes the NEXT token's embedding; all other
+// CTAs are by then polling for exactly those words, with the first weight tiles of the next token already in their
+// rings -- no launch boundary, no pipeline restart.  Behind the launch's last token that CTA also keeps the final hidden
+// state for kl_read_hidden and leaves the rotary table and the step counter of the next token, so that the next launch
+// starts at its first layer at once (K = 1: one launch per token).
+// What changes from token to token inside the launch is arithmetic (position and step number advance by one) except
+// the rotary tables, which kl_token_plan_kernel lays out beforehand, one per token.  Counters that are zeroed between
 // launches count on instead: the gate/up counter of a layer reaches P * (k + 1) during token k, and so does the
-// sampling ticket.  The CTA that draws the last ticket of token k picks the token, records it, and writes the next
-// embedding under the tags of step + 1; all other CTAs are by then polling for exactly those words, with the first
-// weight tiles of the next token already in their rings -- no launch boundary, no pipeline restart.
+// sampling ticket.
 // Tag slot of an embedding written INSIDE the launch.  The hidden state that enters the classifier carries
 // (step, layer L, TG_XA), which is the same number as (step + 1, layer 0, TG_XA): across a launch boundary that is
 // harmless, inside the launch the CTAs polling for the next embedding would take the old hidden state for it.
 constexpr uint32_t TG_NEXT = 5;
-struct TokenLoopParams {
-    TokenParams t;
-    int32_t* out_tokens;       // [K] the token picked after each step
-    uint32_t K;
-    const Params* params;      // [K] parameters of token k (positions, step_dev and rope_cs point at entry k below)
-    const uint32_t* steps;     // [K] step number of token k
+struct TokenParams {
+    int32_t* tokens;        // [1] in: the token the launch starts from (already embedded); out: the token after the last step
+    int32_t* positions;     // [1] advanced by K
+    float* part_val;        // [P] per-CTA maxima
+    uint32_t* part_idx;     // [P] and their indices
+    uint32_t* ticket;       // zero between launches
+    float* hidden;          // [H] final hidden state of the launch's last step
+    int32_t* out_tokens;    // [K] the token picked after each step, or null
+    uint32_t K;             // tokens of this launch
+    const float* rope;      // [K][head_dim] rotary tables of the K positions (K = 1: the handle's own table)
 };
 
-__global__ void kl_token_plan_kernel(const __grid_constant__ Params p, Params* params, uint32_t* steps, int32_t* pos_arr,
-                                     float* rope_arr, uint32_t K) {
-    const uint32_t step0 = *p.step_dev;
+// Rotary tables of the K positions of a launch, and the check that all of them lie inside the cache.
+__global__ void kl_token_plan_kernel(const __grid_constant__ Params p, float* rope_arr, uint32_t K) {
     const int32_t pos0 = p.positions[0];
     if (pos0 < 0 || (uint32_t)pos0 + K > p.max_ctx) {   // every position of the launch has to be inside the cache
         if (threadIdx.x == 0) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
         return;
-    }
-    for (uint32_t k = threadIdx.x; k < K; k += blockDim.x) {
-        steps[k] = step0 + k;
-        pos_arr[k] = pos0 + (int32_t)k;
-        Params q = p;
-        q.positions = pos_arr + k;
-        q.step_dev = steps + k;
-        q.rope_cs = rope_arr + (size_t)k * p.hd;
-        params[k] = q;
     }
     const uint32_t half = p.hd / 2;
     for (uint32_t i = threadIdx.x; i < K * half; i += blockDim.x) {
@@ -460,10 +329,11 @@ __global__ void kl_token_plan_kernel(const __grid_constant__ Params p, Params* p
     }
 }
 
-__device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, uint32_t cta, const TokenLoopParams& t) {
+__device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, uint32_t cta, const TokenParams& t) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+    const uint32_t step0 = ld_step(p.step_dev), pos0 = (uint32_t)p.positions[0];
     for (uint32_t k = 0; k < t.K && !r.aborted; ++k) {
-        const AttnUnit u = attn_unit(t.params[k], cta);
+        const AttnUnit u = attn_unit(p, cta, pos0 + k);
         for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
             const size_t lo = (size_t)l * p.layer_stride;
             produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
@@ -472,7 +342,7 @@ __device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, u
                 // previous token is complete in every CTA, which the first word of this token's embedding says (it
                 // keeps its tag until the first down projection of this token, which cannot start before this point
                 // has been passed in every CTA).  Weight tiles do not wait: the ring is full of them by now.
-                const uint32_t want = tag_from(__ldg(t.steps + k), p.L, 0, TG_NEXT);
+                const uint32_t want = tag_from(step0 + k, p.L, 0, TG_NEXT);
                 PollGuard g = {0ull, 0u, 700};
                 while (ld_tw(p.xa).tag != want) {
                     if (!poll_continue(p, s, g)) {
@@ -494,23 +364,22 @@ __device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, u
     produce_drain(p, s, r);
 }
 
-// Sampling at the end of token k, out of line (once per token; inlined, its address arithmetic would be hoisted out of
-// the loop over tokens and held in registers through the stage code).  Every CTA reduces the logits rows it has just
-// produced; the CTA that draws the token's last ticket reduces the per-CTA results, records the token and writes the
-// next embedding.  false: that was the last token of the launch, or a wait gave up.
-__device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const TokenLoopParams& t, const uint32_t k,
+// Sampling at the end of token k (step cx.step, position cx.pos), out of line: once per token.  Every CTA reduces the
+// logits rows it has just produced; the CTA that draws the token's last ticket reduces the per-CTA results, records the
+// token and writes the next embedding.  false: that was the last token of the launch, or a wait of this launch gave up
+// -- in which case token, position and the next embedding are left alone (the step's outputs are meaningless; the
+// chain has to be restarted).
+__device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const TokenParams& t, uint32_t k,
                                           uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane) {
-    auto tk = [&]() -> uint32_t { return k; };
-    const uint32_t step = __ldg(p.step_dev) + k;   // read once, here: the last CTA of the last token advances the word below
-    auto tstep = [&]() -> uint32_t { return step; };
-    auto tfinal = [&]() -> bool { return k + 1u == t.K; };
+    const bool final = k + 1u == t.K;
+    const StepCtx cx = *s.ctx;   // a copy: the shared one moves on to the next token below
     // ---- greedy sampling: this CTA's rows first
     const GemvPlan& plm = p.plan[PL_LM];
     asm volatile("fence.proxy.async;" ::: "memory");   // the cache rows this thread appended: readable by later bulk copies
-    consumer_bar();
+    consumer_bar();   // the rows this CTA stored are visible to all of its threads
     float* sv = s.unit_part;                                           // [NCW] maxima, then [NCW] indices, then flags
     uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part) + NCW;
-    // [0] this CTA drew the last ticket, [1] token, [2] position, [4] stop: a wait of this launch gave up
+    // [0] this CTA drew the last ticket, [1] token, [2] position, [3] next step number, [4] stop: a wait of this launch gave up
     volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part) + 2 * NCW;
     const CtaRange cr = cta_units(plm, cta, p.P);
     const uint32_t r0 = cr.u0 * plm.rpc, r1 = min(cr.u1 * plm.rpc, p.V);
@@ -526,37 +395,39 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
     consumer_bar();
     if (ctid == 0) {
         for (uint32_t w = 1; w < (uint32_t)NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
-        t.t.part_val[cta] = bv;
-        t.t.part_idx[cta] = bi;
-        sh[0] = (atom_add_acq_rel(t.t.ticket, 1u) == p.P * (tk() + 1u) - 1u) ? 1u : 0u;
+        t.part_val[cta] = bv;
+        t.part_idx[cta] = bi;
+        sh[0] = (atom_add_acq_rel(t.ticket, 1u) == p.P * (k + 1u) - 1u) ? 1u : 0u;
         sh[4] = (*s.abort_flag != 0 || __ldcg(p.status) != 0) ? 1u : 0u;
     }
     consumer_bar();
     const bool last_cta = sh[0] != 0u, stop = sh[4] != 0u;
-    if (last_cta) {
+    if (last_cta && stop) {
+        if (ctid == 0) *t.ticket = 0u;
+    } else if (last_cta) {
         // all logits of this token are written.  Next token, next position, the next embedding.
         if (warp == 0) {
             bv = -INFINITY;
             bi = 0xffffffffu;
-            for (uint32_t j = lane; j < p.P; j += 32) argmax_merge(bv, bi, __ldcg(t.t.part_val + j), __ldcg(t.t.part_idx + j));
+            for (uint32_t j = lane; j < p.P; j += 32) argmax_merge(bv, bi, __ldcg(t.part_val + j), __ldcg(t.part_idx + j));
             for (int o = 16; o > 0; o >>= 1)
                 argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
             if (lane == 0) {
                 const uint32_t tok = bi == 0xffffffffu ? 0u : bi;
-                const int32_t pos = __ldg(t.params[tk()].positions) + 1;
-                t.t.tokens[0] = (int32_t)tok;
-                t.t.positions[0] = pos;
-                t.out_tokens[tk()] = (int32_t)tok;
-                if (tfinal() || stop) *p.step_dev = tstep() + 1u;
-                if (tfinal() || stop) *t.t.ticket = 0u;   // ready for the next launch
-                if (tfinal() && pos >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);
+                const int32_t pos = (int32_t)cx.pos + 1;
+                t.tokens[0] = (int32_t)tok;
+                t.positions[0] = pos;
+                if (t.out_tokens != nullptr) t.out_tokens[k] = (int32_t)tok;
+                if (final) *t.ticket = 0u;   // ready for the next launch
+                if (final && pos >= (int32_t)p.max_ctx) atomicCAS(p.status, 0, ERR_OUT_OF_RANGE);   // the next step would leave the cache
                 sh[1] = tok;
                 sh[2] = (uint32_t)pos;
             }
         }
         consumer_bar();
-        if (tfinal() || stop) {   // what the next launch needs: hidden state kept, rotary table, counters at zero
-            for (uint32_t i = ctid; i < p.H; i += NCT) t.t.hidden[i] = ld_tw(p.xa + i).v;
+        uint32_t next_step = cx.step + 1u;
+        if (final) {   // what the next launch needs: hidden state kept, rotary table, counters at zero, step number
+            for (uint32_t i = ctid; i < p.H; i += NCT) t.hidden[i] = ld_tw(p.xa + i).v;   // before xa is overwritten below
             for (uint32_t i = ctid; i < p.hd / 2; i += NCT) {
                 double sn, cs;
                 sincos((double)sh[2] * p.inv_freq[i], &sn, &cs);
@@ -565,105 +436,56 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
             }
             for (uint32_t i = ctid; i < p.L; i += NCT) p.counters[i] = 0u;
             consumer_bar();
+            if (next_step >= step_wrap(p.L)) {   // every other CTA has left its last stage: the step numbers start over
+                clear_tagged(p, ctid, NCT);
+                next_step = 1u;
+                consumer_bar();
+            }
+            if (ctid == 0) *p.step_dev = next_step;
         }
         const __nv_bfloat16* row = p.embed + (size_t)sh[1] * p.H;
         // the next launch expects the usual tag, the next token of this launch the one of its own
-        const uint32_t xtag = tag_from(tstep() + 1u, p.L, 0, tfinal() || stop ? (uint32_t)TG_XA : TG_NEXT);
-        __threadfence();   // release side of the token boundary (see the fence behind the first load_vec)
+        const uint32_t xtag = tag_from(next_step, p.L, 0, final ? (uint32_t)TG_XA : TG_NEXT);
+        __threadfence();   // release side of the token boundary (the producers' poll above is the acquire side)
         for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
     }
+    if (ctid == 0) {   // the next token of the launch: one step and one position further, the next rotary table
+        s.ctx->step = cx.step + 1u;
+        s.ctx->pos = cx.pos + 1u;
+        s.ctx->rope_cs = cx.rope_cs + p.hd;
+    }
     consumer_bar();   // the flags above are read before the next stage reuses the area
-    return !stop && !tfinal();
+    return !stop && !final;
 }
 
-
-// All tokens of the launch on the consumer warps.  ONE loop over (token, layer) pairs, the classifier being the only
-// stage of a layer L behind the decoder layers and the sampling a call behind that: with a loop over tokens around the
-// loop over layers the compiler holds more in registers through the stage code (and a second copy of the stage code
-// for the classifier would have its loop-invariant values held through the first).  The step number (for the tags) and
-// the parameter copy of the token are fetched where they are needed rather than kept.
-__device__ __forceinline__ void consume_tokens(const Params& p, const Smem& s, const TokenLoopParams& t, uint32_t cta,
-                                               uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
+// K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
+// classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
+// loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
+__global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const Smem s = carve_smem(smem_raw, p);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
+    if (!cta_begin(p, s, tid, t.rope)) return;
+    if (warp == NCW) {
+        if (lane == 0) produce_tokens(p, s, cta, t);
+        return;
+    }
+    WarpRing wr = ring_begin();
+    RingCursor rc = {0u, 0u};
     uint32_t k = 0, l = 0;
-    auto tk = [&]() -> uint32_t { return k; };
-    auto tstep = [&]() -> uint32_t { return __ldg(p.step_dev) + k; };   // the word changes behind the launch's last token only
 #pragma unroll 1
     for (;;) {
-        const size_t lo = (size_t)l * p.layer_stride;
         const bool cls = l == p.L;
-        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st) {
-            GemvOut out = {nullptr, nullptr, nullptr, 0u};
-            int plan = PL_QKV, ep = EP_STORE;
-            const float* xsrc = nullptr;
-            float xscale = 1.f;
-            if (st == ST_QKV) {
-                xscale = load_vec(p, s, p.xa, p.H, tag_from(tstep(), p.L, l, tk() > 0 && l == 0 ? TG_NEXT : (uint32_t)TG_XA), true,
-                                  cls ? p.gf : p.g1 + lo, ctid);
-                if (cls) {
-                    out = {nullptr, p.logits, nullptr, 0u};
-                    plan = PL_LM;
-                } else {
-                    out = {p.qkv, nullptr, nullptr, tag_from(tstep(), p.L, l, TG_QKV)};
-                }
-            } else if (st == ST_ATTN) {
-                attention_block(tk() == 0 ? p : t.params[tk()], s, l, cta, ctid, warp, lane, rc, wr);
-                continue;
-            } else if (st == ST_O) {
-                load_vec(p, s, p.o, p.QD, tag_from(tstep(), p.L, l, TG_O), false, nullptr, ctid);
-                out = {p.xb, nullptr, p.xa, tag_from(tstep(), p.L, l, TG_XB)};
-                plan = PL_O;
-                ep = EP_RESIDUAL;
-            } else if (st == ST_GU) {
-                xscale = load_vec(p, s, p.xb, p.H, tag_from(tstep(), p.L, l, TG_XB), true, p.g2 + lo, ctid);
-                out = {nullptr, p.h, nullptr, 0u};
-                plan = PL_GU;
-                ep = EP_SWIGLU;
-            } else {
-                stage_wait(p, s, p.counters + l, p.P * (tk() + 1u), ctid);
-                out = {p.xa, nullptr, p.xb, tag_from(tstep(), p.L, l + 1, TG_XA)};
-                plan = PL_D;
-                ep = EP_RESIDUAL;
-                xsrc = p.h;
-            }
-            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
-            if (st == ST_GU) stage_signal(p.counters + l, ctid, false);
-        }
+        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st)
+            run_stage(p, s, l, st, (k > 0 && l == 0) ? TG_NEXT : (uint32_t)TG_XA, p.P * (k + 1u), cta, tid, warp, lane, rc, wr);
         if (cls) {
-            if (!sample_token(p, s, t, k, cta, ctid, warp, lane)) break;
+            if (!sample_token(p, s, t, k, cta, tid, warp, lane)) break;
             ++k;
             l = 0;
         } else {
             ++l;
         }
     }
-}
-
-__global__ void __launch_bounds__(NTHREADS, 1) kl_token_loop_kernel(const __grid_constant__ Params p,
-                                                                    const __grid_constant__ TokenLoopParams t) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, p);
-    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
-    if (tid == 0) {
-        for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
-        }
-        *s.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
-    __syncthreads();
-    if (*p.status != 0) return;
-    if (warp == NCW) {
-        if (lane == 0) produce_tokens(p, s, cta, t);
-        return;
-    }
-    WarpRing wr = ring_begin();
-    const uint32_t ctid = tid;
-    RingCursor rc = {0u, 0u};
-
-    consume_tokens(p, s, t, cta, ctid, warp, lane, rc, wr);
 }
 
 }  // namespace kl
@@ -722,10 +544,6 @@ struct kl_handle {
     uint32_t* tok_idx;     // [P]
     uint32_t* tok_ticket;
     int token_ok;          // kl_token_kernel can be resident
-    int loop_ok;           // kl_token_loop_kernel can be resident
-    Params* plan_params;   // [TOKENS_PER_LAUNCH] per-token parameter copies of kl_token_loop_kernel, written by kl_token_plan_kernel
-    uint32_t* plan_steps;  // [TOKENS_PER_LAUNCH]
-    int32_t* plan_pos;     // [TOKENS_PER_LAUNCH]
     int32_t* plan_out;     // [TOKENS_PER_LAUNCH] picked tokens of the host-buffer entry point
     float* plan_rope;      // [TOKENS_PER_LAUNCH][head_dim]
     uint32_t* argmax_idx;
@@ -745,7 +563,7 @@ struct kl_handle {
 namespace {
 
 constexpr size_t ALIGN = 256;
-constexpr size_t TOKENS_PER_LAUNCH = 256;   // most tokens one launch of kl_token_loop_kernel decodes
+constexpr size_t TOKENS_PER_LAUNCH = 256;   // most tokens one launch of kl_token_kernel decodes (see STEP_WRAP_MARGIN)
 inline size_t align_up(size_t v, size_t a = ALIGN) { return (v + a - 1) / a * a; }
 inline uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
 
@@ -840,8 +658,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.samax = s;     s += align_up(B * ARGMAX_BLOCKS * 8 + B * 4);
     y.shid = s;      s += align_up((B > 1 ? 32 : B) * H * 4);
     y.stokp = s;     s += align_up((size_t)num_sms * 8 + ALIGN);
-    y.stplan = s;    s += align_up(TOKENS_PER_LAUNCH * align_up(sizeof(Params))) + 3 * align_up(TOKENS_PER_LAUNCH * 4) +
-                          align_up((size_t)TOKENS_PER_LAUNCH * d.head_dim * 4);
+    y.stplan = s;    s += align_up(TOKENS_PER_LAUNCH * 4) + align_up((size_t)TOKENS_PER_LAUNCH * d.head_dim * 4);
     // batched path (max_batch > 1): operand, partial sums, queries, attention partials
     {
         const size_t QR = QD + 2 * KVD;
@@ -1159,17 +976,14 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.nslots = NCW;
     p.nsw = (uint32_t)nsw;
     h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
-    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
-    if (ce == cudaSuccess)
-        ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes);
+    // The shared-memory limit is an attribute of the kernel, not of a handle: it is raised to the device's opt-in
+    // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
+    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     {
         int tocc = 0;
-        h->token_ok = cudaFuncSetAttribute(kl_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) == cudaSuccess &&
+        h->token_ok = cudaFuncSetAttribute(kl_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
                       cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
-        (void)cudaGetLastError();
-        h->loop_ok = h->token_ok &&
-                     cudaFuncSetAttribute(kl_token_loop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->smem_bytes) == cudaSuccess &&
-                     cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_loop_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
@@ -1200,10 +1014,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->tok_val = (float*)(sc + y.stokp);
     h->tok_idx = (uint32_t*)(h->tok_val + sms);
     h->tok_ticket = h->tok_idx + sms;
-    h->plan_params = (Params*)(sc + y.stplan);
-    h->plan_steps = (uint32_t*)(sc + y.stplan + align_up(TOKENS_PER_LAUNCH * align_up(sizeof(Params))));
-    h->plan_pos = (int32_t*)((uint8_t*)h->plan_steps + align_up(TOKENS_PER_LAUNCH * 4));
-    h->plan_out = (int32_t*)((uint8_t*)h->plan_pos + align_up(TOKENS_PER_LAUNCH * 4));
+    h->plan_out = (int32_t*)(sc + y.stplan);
     h->plan_rope = (float*)((uint8_t*)h->plan_out + align_up(TOKENS_PER_LAUNCH * 4));
     h->hidden_is_copy = 0;
     h->chain_tok = nullptr;
@@ -1611,7 +1422,8 @@ static kl_status token_chain_params(kl_handle* h, Params* out, int32_t* tokens_d
     p.positions = positions_d;
     p.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
     p.logits = logits_d;
-    p.skip_stage = -1;
+    p.skip_stage = h->pending_skip_stage;   // test hook of the bounded waits: applies to the next launch only
+    h->pending_skip_stage = -1;
     p.trace = nullptr;
     p.chunk_trace = nullptr;
     p.attn_tc = 0;
@@ -1646,7 +1458,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     Params p;
     const kl_status prc = token_chain_params(h, &p, tokens_d, positions_d, kv_cache_d, logits_d, restart, st);
     if (prc != KL_OK) return prc;
-    TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all};
+    TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, nullptr, 1u, p.rope_cs};
     void* args[] = {&p, &t};
     const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
     if (rc != KL_OK) return rc;
@@ -1661,7 +1473,7 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d || !out_tokens_d) return KL_ERR_INVALID_ARG;
     if (batch == 0 || batch > h->desc.max_batch) return KL_ERR_INVALID_ARG;
     cudaStream_t st = as_stream(stream);
-    if (batch > 1 || !h->loop_ok) {
+    if (batch > 1 || !h->token_ok) {
         // batches: token after token (each step replayed from the handle's graph), the picked tokens copied out
         for (uint32_t k = 0; k < n_tokens; ++k) {
             const kl_status rc = kl_decode_greedy(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, restart && k == 0, stream);
@@ -1677,13 +1489,12 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
         Params p;
         const kl_status prc = token_chain_params(h, &p, tokens_d, positions_d, kv_cache_d, logits_d, restart && done == 0, st);
         if (prc != KL_OK) return prc;
-        kl_token_plan_kernel<<<1, 256, 0, st>>>(p, h->plan_params, h->plan_steps, h->plan_pos, h->plan_rope, K);
+        kl_token_plan_kernel<<<1, 256, 0, st>>>(p, h->plan_rope, K);
         if (cudaGetLastError() != cudaSuccess) return KL_ERR_CUDA;
         ++h->launches;
-        TokenLoopParams t = {{tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all},
-                             out_tokens_d + done, K, h->plan_params, h->plan_steps};
+        TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, out_tokens_d + done, K, h->plan_rope};
         void* args[] = {&p, &t};
-        const kl_status rc = launch_persistent(h, (const void*)kl_token_loop_kernel, args, st);
+        const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
         if (rc != KL_OK) return rc;
         h->last_batch = 1;
         h->hidden_is_copy = 1;
@@ -1917,6 +1728,15 @@ kl_status kl_set_dependent_launch(kl_handle* h, int on) {
 kl_status kl_debug_skip_signal_once(kl_handle* h, int stage) {
     if (!h || stage < -1 || stage > 4) return KL_ERR_INVALID_ARG;
     h->pending_skip_stage = stage;
+    return KL_OK;
+}
+
+kl_status kl_debug_set_step(kl_handle* h, uint32_t step, uint32_t* wrap_at) {
+    if (!h) return KL_ERR_INVALID_ARG;
+    if (wrap_at) *wrap_at = step_wrap(h->prm.L);
+    if (step == 0xffffffffu) return KL_OK;   // query only
+    if (cudaMemcpy(h->prm.step_dev, &step, 4, cudaMemcpyHostToDevice) != cudaSuccess) return KL_ERR_CUDA;
+    h->chain_tok = nullptr;   // the next greedy call starts a chain (embedding under the new step number)
     return KL_OK;
 }
 

@@ -97,6 +97,15 @@ struct Params {
 };
 constexpr uint32_t CHUNK_TRACE_ROWS = 8192;
 
+// What changes from one decoded token to the next: the step number the tags are built from, the position written by
+// the step, and the rotary table of that position.  One copy per CTA in shared memory, written by one thread at the
+// start of the launch (and behind every token of a launch that decodes several) and read between the stages.
+struct StepCtx {
+    uint32_t step;
+    uint32_t pos;
+    const float* rope_cs;
+};
+
 
 // ------------------------------------------------------------------------------------------------ PTX
 
@@ -203,9 +212,23 @@ enum TagSlot { TG_XA = 0, TG_QKV = 1, TG_PART = 2, TG_O = 3, TG_XB = 4 };
 __device__ __forceinline__ uint32_t tag_from(uint32_t step, uint32_t L, uint32_t layer, uint32_t slot) {
     return ((((step * L + layer) << 3) + slot) << 1) | 1u;
 }
-// The step word was written by the embedding kernel of this sequence, an earlier launch: a read-only load is fine.
-__device__ __forceinline__ uint32_t tag_of(const Params& p, uint32_t layer, uint32_t slot) {
-    return tag_from(__ldg(p.step_dev), p.L, layer, slot);
+__device__ __forceinline__ uint32_t tag_of(const Params& p, const StepCtx& cx, uint32_t layer, uint32_t slot) {
+    return tag_from(cx.step, p.L, layer, slot);
+}
+// The step word as a launch finds it.  The launch that writes it (the last CTA of a sampling kernel, behind every
+// reader's last stage) may still have readers of this load in flight when a bounded wait gave up, so the load is a
+// strong one, not a read-only one.
+__device__ __forceinline__ uint32_t ld_step(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ StepCtx step_ctx(const Params& p) {
+    StepCtx cx;
+    cx.step = ld_step(p.step_dev);
+    cx.pos = (uint32_t)p.positions[p.b0];
+    cx.rope_cs = p.rope_cs;
+    return cx;
 }
 
 __device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
@@ -224,6 +247,7 @@ struct Smem {
     float* unit_part;       // [UNIT_SLOTS][MAX_PIECES]
     int* unit_cnt;          // [UNIT_SLOTS]
     volatile int* abort_flag;
+    StepCtx* ctx;           // step number, position and rotary table of the token being decoded (see StepCtx)
 };
 
 __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
@@ -237,6 +261,7 @@ __device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
     s.unit_part = reinterpret_cast<float*>(misc + 2048);           // [UNIT_SLOTS][MAX_PIECES][MAX_RPC_SPLIT] 4 KB
     s.unit_cnt = reinterpret_cast<int*>(misc + 6144);              // [UNIT_SLOTS]
     s.abort_flag = s.unit_cnt + UNIT_SLOTS;
+    s.ctx = reinterpret_cast<StepCtx*>(misc + 6208);
     return s;
 }
 
@@ -343,7 +368,7 @@ struct AttnUnit {
     uint32_t nring;     // ring chunks of this unit
 };
 __device__ __forceinline__ uint32_t attn_positions_per_chunk(const Params& p) { return SLOT_BYTES / (4u * p.hd); }
-__device__ __forceinline__ AttnUnit attn_unit(const Params& p, uint32_t cta) {
+__device__ __forceinline__ AttnUnit attn_unit(const Params& p, uint32_t cta, uint32_t pos) {
     AttnUnit u;
     u.active = false;
     u.nring = 0;
@@ -352,7 +377,7 @@ __device__ __forceinline__ AttnUnit attn_unit(const Params& p, uint32_t cta) {
     if (u.bg >= p.nkv) return u;
     u.b = p.b0;
     u.g = u.bg;
-    u.pos = (uint32_t)p.positions[u.b];
+    u.pos = pos;
     const uint32_t n = u.pos + 1;
     uint32_t nchunk = min(p.cps, (n + MIN_POS_PER_CHUNK - 1) / MIN_POS_PER_CHUNK);
     const uint32_t clen = (n + nchunk - 1) / nchunk;
@@ -563,7 +588,7 @@ __device__ __forceinline__ void produce_drain(const Params& p, const Smem& s, co
 __device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, uint32_t cta, uint32_t l0, uint32_t l1,
                                                 uint32_t sbeg, uint32_t send) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
-    const AttnUnit u = attn_unit(p, cta);
+    const AttnUnit u = attn_unit(p, cta, (uint32_t)p.positions[p.b0]);
     for (uint32_t l = l0; l < l1 && !r.aborted; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         for (uint32_t st = sbeg; st < send; ++st) {
@@ -1293,11 +1318,11 @@ __device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const 
 // (head, chunk) and the unit's slice of every chunk's partial output go to shared memory; the pairs become weights
 // w[h][c] = exp2(m_c - M_h) / L_h; thread j adds its output's nchunk terms in chunk order.  The orders of all sums
 // are fixed.
-__device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const AttnUnit& u, uint32_t layer, uint32_t G,
-                                        uint32_t ctid, float* comb) {
+__device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const StepCtx& cx, const AttnUnit& u, uint32_t layer,
+                                        uint32_t G, uint32_t ctid, float* comb) {
     const uint32_t hd = p.hd, b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
     const uint32_t unit0 = u.bg * p.cps;
-    const uint32_t tag = tag_of(p, layer, TG_PART), otag = tag_of(p, layer, TG_O);
+    const uint32_t tag = tag_of(p, cx, layer, TG_PART), otag = tag_of(p, cx, layer, TG_O);
     const uint32_t total = G * hd;
     const uint32_t S = (total + nchunk - 1) / nchunk;
     const uint32_t t_lo = min(total, u.ch * S), t_hi = min(total, t_lo + S);
@@ -1377,9 +1402,9 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const At
 // the outputs (attn_merge).  Scores use q pre-multiplied by log2(e)/sqrt(hd): the softmax runs in base 2.
 // GT > 0 selects the CUDA-core inner loop for GT query heads per KV head; GT == 0 the tensor-core loop.
 template <int GT>
-__device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
+__device__ __noinline__ void attention_stage(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer, uint32_t cta,
                                                  uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
-    const AttnUnit u = attn_unit(p, cta);
+    const AttnUnit u = attn_unit(p, cta, cx.pos);
     if (!u.active) return;
     const uint32_t G = GT > 0 ? (uint32_t)GT : p.G;
     const uint32_t hd = p.hd, half = hd >> 1;
@@ -1399,8 +1424,8 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     // own those rows of the QKV projection.  The unit waits for exactly the rows it needs, not for the whole stage.
     consumer_bar();   // the workspace below overlays the QKV stage's input vector: wait for this CTA's last QKV chunk
     const TW* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
-    const uint32_t qtag = tag_of(p, layer, TG_QKV);
-    const float* cs = p.rope_cs + (size_t)b * hd;  // [half][2]
+    const uint32_t qtag = tag_of(p, cx, layer, TG_QKV);
+    const float* cs = cx.rope_cs + (size_t)b * hd;  // [half][2]
     const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
     // biases of the projections (decoders that have them): added to the polled values, before the rotation
     const __nv_bfloat16* bias = p.bqkv ? p.bqkv + (size_t)layer * p.layer_stride : nullptr;
@@ -1589,9 +1614,9 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
             Lsum += src[hd + 1] * c;
         }
         if (nchunk == 1) {
-            st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, A / Lsum, tag_of(p, layer, TG_O));
+            st_tw(p.o + (size_t)b * p.QD + (size_t)(g * G + h) * hd + d, A / Lsum, tag_of(p, cx, layer, TG_O));
         } else {
-            const uint32_t ptag = tag_of(p, layer, TG_PART);
+            const uint32_t ptag = tag_of(p, cx, layer, TG_PART);
             st_tw(p.part + ((size_t)unit * G + h) * hd + d, A, ptag);
             if (d == 0) {
                 st_tw(p.part_ml + ((size_t)unit * G + h) * 2, ftab[NCW * G + h], ptag);
@@ -1601,16 +1626,16 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, uin
     }
     trace_stamp(p, cta, layer, 3, ctid);
     // every unit of the group merges its slice of the outputs
-    if (nchunk > 1) attn_merge(p, s, u, layer, G, ctid, comb);
+    if (nchunk > 1) attn_merge(p, s, cx, u, layer, G, ctid, comb);
 }
 
 // Appends the K/V row of the position written by this step to the cache (16-byte stores).  Nothing in the running
 // kernel reads that row from memory -- the unit that owns it works from the shared-memory copy -- so the store is
 // kept off the stage's critical path: it runs after the CTA has signalled, and before the shared-memory copy is
 // overwritten by the next stage's input vector.
-__device__ __forceinline__ void attention_flush_new_row(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
-                                                        uint32_t ctid) {
-    const AttnUnit u = attn_unit(p, cta);
+__device__ __forceinline__ void attention_flush_new_row(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer,
+                                                        uint32_t cta, uint32_t ctid) {
+    const AttnUnit u = attn_unit(p, cta, cx.pos);
     if (!u.active || !u.has_new) return;
     const uint32_t hd = p.hd;
     const float* new_k = s.vec + p.G * hd;
@@ -1631,11 +1656,11 @@ __device__ __forceinline__ void attention_flush_new_row(const Params& p, const S
 
 // Runs the attention stage and moves the ring cursor past the unit's chunks (also for CTAs without a unit).
 template <int GT>
-__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const Smem& s, uint32_t layer, uint32_t cta,
-                                                            uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc,
-                                                            WarpRing& wr) {
-    attention_stage<GT>(p, s, layer, cta, ctid, warp, lane, rc, wr);
-    rc.advance(attn_unit(p, cta).nring, p.nslots);
+__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer,
+                                                            uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane,
+                                                            RingCursor& rc, WarpRing& wr) {
+    attention_stage<GT>(p, s, cx, layer, cta, ctid, warp, lane, rc, wr);
+    rc.advance(attn_unit(p, cta, cx.pos).nring, p.nslots);
 }
 
 }  // namespace kl

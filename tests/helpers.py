@@ -155,3 +155,65 @@ def assert_parity(report, steps, batch=1, check_cache=True, flip_tol=0.02):
             assert np.array_equal(modes[0]["steps"][s]["hidden"], other["steps"][s]["hidden"]), s
         if modes[0]["cache"] is not None:
             assert np.array_equal(modes[0]["cache"], other["cache"])
+
+
+def run_full_depth(shape, context, steps, batch=1, oracle_rows=None, seed=0, batched_path=None, greedy_chain=False):
+    """Teacher-forced decode through ALL layers of a large model, compared with the layer-streaming oracle.
+
+    The oracle decodes the sequences `oracle_rows` (default: all) of the batch -- sequences are independent, so a subset
+    is exact; the CUDA path decodes the whole batch.  Sequences the oracle does not run continue on the tokens the
+    CUDA path picked itself and are checked for finite logits only.  The cache is compared on the rows appended by the
+    steps (the prefilled rows of a multi-gigabyte cache are not copied back).  greedy_chain: the CUDA path decodes
+    through kl_decode_greedy (one launch per token at batch 1), not kl_decode_step + kl_argmax_advance.
+    Asserts the benchmark spec's tolerances; returns the worst errors seen."""
+    rows = list(range(batch)) if oracle_rows is None else list(oracle_rows)
+    max_ctx = context + steps + 8
+    host = HostWeights(shape, seed, stream_layers=True)
+    orc = ko.Oracle(shape, max_ctx, host.layer, host.globals(with_table=False))
+    cache = gen.make_kv_cache(shape, batch, context, max_ctx, seed, "cuda")
+    cache_or = cache[:, :, rows].cpu().view(torch.uint16).numpy().copy()
+    toks = gen.make_tokens(shape, batch, seed).tolist()
+    ref = []
+    t, p = [toks[r] for r in rows], [context] * len(rows)
+    for s in range(steps):
+        hidden, logits, nxt = orc.step(cache_or, t, p)
+        srt = np.sort(logits, axis=1)
+        ref.append(dict(tokens=list(t), hidden=hidden, logits=logits, next=nxt.tolist(), margin=(srt[:, -1] - srt[:, -2]).tolist()))
+        t, p = nxt.tolist(), [q + 1 for q in p]
+    dec = make_decoder(shape, batch, max_ctx, seed)
+    if batched_path is not None:
+        dec.kl_set_batched_path(batched_path)
+    tok_d = torch.tensor(toks, dtype=torch.int32, device="cuda")
+    pos_d = torch.full((batch,), context, dtype=torch.int32, device="cuda")
+    logits_d = torch.empty(batch, shape.vocab, dtype=torch.float32, device="cuda")
+    hidden_d = torch.empty(batch, shape.hidden, dtype=torch.float32, device="cuda")
+    worst = dict(rel_hidden=0.0, rel_logits=0.0, max_abs_logit=0.0)
+    for s in range(steps):
+        tok_d[rows] = torch.tensor(ref[s]["tokens"], dtype=torch.int32, device="cuda")   # teacher forcing
+        if greedy_chain:
+            dec.kl_decode_greedy(tok_d, pos_d, cache, logits_d, batch, True)
+        else:
+            dec.kl_decode_step(tok_d, pos_d, cache, logits_d, batch)
+            dec.kl_argmax_advance(logits_d, tok_d, pos_d, batch)
+        dec.kl_read_hidden(hidden_d, batch)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == 0, s
+        lg, hd = logits_d.cpu().numpy(), hidden_d.cpu().numpy()
+        assert np.isfinite(lg).all() and np.isfinite(hd).all(), s
+        assert pos_d.cpu().tolist() == [context + s + 1] * batch
+        nxt = tok_d.cpu().tolist()
+        for i, r in enumerate(rows):
+            e = dict(rel_hidden=rel_l2(hd[r], ref[s]["hidden"][i]), rel_logits=rel_l2(lg[r], ref[s]["logits"][i]),
+                     max_abs_logit=float(np.abs(lg[r] - ref[s]["logits"][i]).max()))
+            assert e["rel_hidden"] <= REL_L2_TOL and e["rel_logits"] <= REL_L2_TOL and e["max_abs_logit"] <= ABS_LOGIT_TOL, (s, r, e)
+            assert nxt[r] == ref[s]["next"][i], (s, r, nxt[r], ref[s]["next"][i], ref[s]["margin"][i])
+            for k in worst:
+                worst[k] = max(worst[k], e[k])
+    # rows appended by the steps: within one bf16 rounding step of the oracle's (fp32 here, fp64 there)
+    got = cache[:, :, rows, :, context:context + steps].cpu().view(torch.uint16).numpy()
+    exp = cache_or[:, :, :, :, context:context + steps]
+    g, e = bf16_decode(got), bf16_decode(exp)
+    assert np.all(np.abs(g - e) <= 2.0 ** -7 * np.abs(e) + 1e-3 * np.abs(e).max())
+    worst["cache_values_differing"] = float((got != exp).mean())
+    dec.close()
+    return worst

@@ -141,6 +141,20 @@ def test_silu_values():
     assert abs(ko.silu(-2.0) + 2.0 / (1.0 + math.exp(2.0))) < 1e-15
 
 
+def test_argmax_lowest_index_on_ties():
+    """Sampling block: the largest logit wins, and among equal maxima the LOWEST index (a rule that takes the last
+    of them, i.e. `>=` in place of `>`, fails the first three cases)."""
+    assert ko.argmax(np.array([0.5, 3.0, -1.0, 3.0, 2.0, 3.0])) == 1          # maximum at 1, 3 and 5
+    assert ko.argmax(np.array([7.0, 7.0, 7.0, 7.0])) == 0                       # all equal
+    assert ko.argmax(np.array([-2.0, -1.0, -1.0])) == 1                         # negative values, tie at the end
+    assert ko.argmax(np.array([1.0, 2.0, 5.0])) == 2                            # no tie, maximum last
+    assert ko.argmax(np.array([-0.0, 0.0])) == 0                                # signed zeros compare equal
+    rng = np.random.default_rng(0)
+    for _ in range(50):                                                         # against numpy's first-maximum rule
+        v = rng.integers(-3, 4, size=40).astype(np.float64)
+        assert ko.argmax(v) == int(np.argmax(v))
+
+
 def test_attention_brute_force_and_special_cases():
     rng = np.random.default_rng(7)
     n, hd = 7, 8

@@ -753,3 +753,167 @@ def test_greedy_chain_of_a_batch_replays_the_cached_graph():
         side.synchronize()
     assert torch.equal(tok1, want[3]) and torch.equal(cache.view(torch.uint16), ref_cache.view(torch.uint16))
     dec.close()
+
+
+@pytest.mark.parametrize("name", ["g4_hd128", "g8_hd64", "g4_hd64"])
+def test_cuda_core_attention_loop(name):
+    """The CUDA-core attention loop (kl_set_tensor_core_attention(0)) for four and eight query heads per kv head at the
+    head sizes that default to the tensor-core loop: all three schedules against the oracle, split-K over several
+    chunks with a ragged tail, and -- same arithmetic up to the order of the sums -- close to the tensor-core result."""
+    shape = {"g4_hd128": gen.ModelShape(2, 512, 8, 2, 128, 1024, 1000, 1e-5, 500000.0),
+             "g8_hd64": gen.ModelShape(2, 512, 8, 1, 64, 768, 1000, 1e-5, 10000.0),
+             "g4_hd64": gen.TINY if gen.TINY.n_q_heads // gen.TINY.n_kv_heads == 4 else gen.ModelShape(2, 256, 8, 2, 64, 512, 1024, 1e-5, 10000.0)}[name]
+    context, steps, max_ctx = 700, 3, 720
+    host = helpers.HostWeights(shape, 4)
+    from oracle import kl_oracle as ko
+    orc = ko.Oracle(shape, max_ctx, host.layer, host.globals())
+    cache0 = gen.make_kv_cache(shape, 1, context, max_ctx, 4, "cuda")
+    cache_or = cache0.cpu().view(torch.uint16).numpy().copy()
+    dec = helpers.make_decoder(shape, 1, max_ctx, 4)
+    results = {}
+    for tc in (False, True):
+        dec.kl_set_tensor_core_attention(tc)
+        for mode in (binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER, binding.KL_MODE_PER_STAGE):
+            dec.kl_set_mode(mode)
+            cache = cache0.clone()
+            logits = torch.empty(1, shape.vocab, device="cuda")
+            hidden = torch.empty(1, shape.hidden, device="cuda")
+            t, p = gen.make_tokens(shape, 1, 4).tolist(), [context]
+            cor = cache_or.copy()
+            for s in range(steps):
+                ref_hidden, ref_logits, nxt = orc.step(cor, t, p)
+                tok_d = torch.tensor(t, dtype=torch.int32, device="cuda")
+                pos_d = torch.tensor(p, dtype=torch.int32, device="cuda")
+                dec.kl_decode_step(tok_d, pos_d, cache, logits, 1)
+                dec.kl_read_hidden(hidden, 1)
+                dec.kl_argmax_advance(logits, tok_d, pos_d, 1)
+                torch.cuda.synchronize()
+                assert dec.kl_last_status() == binding.KL_OK
+                lg, hd = logits.cpu().numpy()[0], hidden.cpu().numpy()[0]
+                assert helpers.rel_l2(hd, ref_hidden[0]) <= helpers.REL_L2_TOL, (tc, mode, s)
+                assert helpers.rel_l2(lg, ref_logits[0]) <= helpers.REL_L2_TOL, (tc, mode, s)
+                assert float(np.abs(lg - ref_logits[0]).max()) <= helpers.ABS_LOGIT_TOL, (tc, mode, s)
+                assert int(tok_d[0]) == int(nxt[0]), (tc, mode, s)
+                t, p = nxt.tolist(), [p[0] + 1]
+            results[(tc, mode)] = (logits.cpu(), cache.cpu().view(torch.uint16))
+    for tc in (False, True):   # the schedules of one loop agree bit for bit
+        for mode in (binding.KL_MODE_PER_LAYER, binding.KL_MODE_PER_STAGE):
+            assert torch.equal(results[(tc, mode)][0], results[(tc, binding.KL_MODE_LOOPED)][0])
+            assert torch.equal(results[(tc, mode)][1], results[(tc, binding.KL_MODE_LOOPED)][1])
+    dec.close()
+
+
+def test_two_handles_of_different_shapes_step_alternately():
+    """Two models alive at once (a small one and one with hidden 8192, whose persistent kernels need different amounts of
+    shared memory): creating the second must not take shared memory away from the first.  Both step alternately, on
+    every schedule, and give the bits each gives alone."""
+    small, wide = gen.TINY, SHAPES["wide_hidden_g8"]
+
+    def run(dec, shape, n):
+        cache = gen.make_kv_cache(shape, 1, 100, 120, 0, "cuda")
+        tok = gen.make_tokens(shape, 1, 0).cuda()
+        pos = torch.tensor([100], dtype=torch.int32, device="cuda")
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        outs = []
+        for i in range(n):
+            dec.kl_set_mode(i % 3)
+            dec.kl_decode_step(tok, pos, cache, logits, 1)
+            dec.kl_argmax_advance(logits, tok, pos, 1)
+            outs.append(logits.clone())
+            yield
+        dec.kl_decode_greedy(tok, pos, cache, logits, 1, True)
+        outs.append(logits.clone())
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        run.results[shape.hidden] = outs
+        yield
+
+    def alone(shape):
+        dec = helpers.make_decoder(shape, 1, 120, 0)
+        run.results = {}
+        for _ in run(dec, shape, 3):
+            pass
+        dec.close()
+        return run.results[shape.hidden]
+
+    want_small, want_wide = alone(small), alone(wide)
+    a = helpers.make_decoder(wide, 1, 120, 0)      # the larger shared-memory request first, then the smaller one
+    b = helpers.make_decoder(small, 1, 120, 0)
+    run.results = {}
+    for _ in zip(run(a, wide, 3), run(b, small, 3)):
+        pass
+    for got, want in ((run.results[wide.hidden], want_wide), (run.results[small.hidden], want_small)):
+        assert len(got) == len(want) and all(torch.equal(g, w) for g, w in zip(got, want))
+    a.close()
+    b.close()
+
+
+def test_bounded_wait_on_the_greedy_chain_leaves_token_and_position_alone():
+    """A wait that runs out inside the one-launch-per-token kernel: the call reports KL_ERR_SYNC_TIMEOUT, does not touch
+    the token or the position (the step's logits and cache row are undefined), and the next call starts a new chain that
+    gives the bits of an undisturbed run."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 1, 200, 0)
+    cache0 = gen.make_kv_cache(shape, 1, 128, 200, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+    logits_ok, logits = torch.empty(1, shape.vocab, device="cuda"), torch.empty(1, shape.vocab, device="cuda")
+    c1, tok, pos = cache0.clone(), tok0.clone(), torch.tensor([128], dtype=torch.int32, device="cuda")
+    dec.kl_decode_greedy(tok, pos, c1, logits_ok, 1, True)
+    torch.cuda.synchronize()
+    assert dec.kl_last_status() == binding.KL_OK
+    want_tok = int(tok[0])
+    dec.kl_set_wait_limit_ns(20_000_000)   # 20 ms
+    for stage in (0, 1, 3):
+        c2, tok, pos = cache0.clone(), tok0.clone(), torch.tensor([128], dtype=torch.int32, device="cuda")
+        dec.kl_debug_skip_signal_once(stage)
+        dec.kl_decode_greedy(tok, pos, c2, logits, 1, True)
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_ERR_SYNC_TIMEOUT
+        assert int(tok[0]) == int(tok0[0]) and int(pos[0]) == 128
+        c2 = cache0.clone()
+        dec.kl_decode_greedy(tok, pos, c2, logits, 1, False)    # no restart asked for: the handle starts a chain by itself
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        assert int(tok[0]) == want_tok and int(pos[0]) == 129
+        assert torch.equal(logits, logits_ok) and torch.equal(c1.view(torch.uint16), c2.view(torch.uint16))
+    dec.close()
+
+
+def test_step_numbers_wrap_without_a_stale_tag():
+    """The step numbers behind the tags wrap after about 2^28 / n_layers steps: the tagged scratch areas are cleared at
+    that launch boundary and the numbering restarts.  With the counter preset just below the wrap, a run that crosses
+    it -- step by step, as a greedy chain, and as one multi-token launch -- gives the bits of a run far from it."""
+    shape = gen.TINY
+    dec = helpers.make_decoder(shape, 1, 200, 0)
+    wrap = dec.kl_debug_set_step()
+    assert wrap == (1 << 28) // shape.n_layers - 260
+    cache0 = gen.make_kv_cache(shape, 1, 128, 200, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+    n = 12
+
+    def chain(kind):
+        cache, tok, pos = cache0.clone(), tok0.clone(), torch.tensor([128], dtype=torch.int32, device="cuda")
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        out = torch.empty(n, dtype=torch.int32, device="cuda")
+        if kind == "tokens":
+            dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out[:5], 5, 1, True)
+            dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out[5:], n - 5, 1, False)
+        else:
+            for i in range(n):
+                if kind == "steps":
+                    dec.kl_decode_step(tok, pos, cache, logits, 1)
+                    dec.kl_argmax_advance(logits, tok, pos, 1)
+                else:
+                    dec.kl_decode_greedy(tok, pos, cache, logits, 1, i == 0)
+                out[i] = tok[0]
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        return out.cpu(), logits.cpu(), cache.cpu().view(torch.uint16)
+
+    want = chain("steps")
+    for kind in ("steps", "greedy", "tokens"):
+        for start in (wrap - 4, wrap - 1, wrap - 7):
+            dec.kl_debug_set_step(start)
+            got = chain(kind)
+            assert all(torch.equal(g, w) for g, w in zip(got, want)), (kind, start)
+    dec.close()

@@ -91,3 +91,22 @@ def test_static_argmax_rejects_sizes_beyond_the_array():
     assert "KL_ERR_TOO_LARGE" in str(e.value)
     torch.cuda.synchronize()
     assert int((tok != -7).sum()) == 0 and int(pos.sum()) == 0  # nothing was launched
+
+
+def test_static_argmax_allocates_no_device_memory():
+    """What the entry point is for: after its first call on the device (which looks up the array's address), a call
+    leaves the amount of free device memory exactly where it was -- nothing is allocated, by the library or inside the
+    CUDA runtime on its behalf.  All buffers of the test exist before the measurement starts."""
+    batch, vocab = 4, 4099
+    logits = _logits(batch, vocab, seed=3)
+    tok = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    pos = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    binding.kl_argmax_advance_static(logits, tok, pos, batch)   # the first call on this device may set up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        binding.kl_argmax_advance_static(logits, tok, pos, batch)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.equal(tok, _first_max(logits)) and int((pos != 4).sum()) == 0
