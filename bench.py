@@ -362,10 +362,17 @@ def replica_throughput(steps: int, batch: int, world: int, ms_local: float) -> t
     return steps * batch * world / (ms * 1e-3), ms
 
 
+def oracle_layers_that_fit(shape, budget_bytes=24e9) -> int:
+    """Decoder layers whose weights the oracle's host can hold at once: all of them for models up to the 8B shape (whole
+    decode steps are executed), a bounded sample for the larger ones."""
+    return shape.n_layers if shape.n_layers * layer_weight_bytes(shape) <= budget_bytes else 0
+
+
 class OracleSampler:
-    """The oracle, as it stands, on a bounded sample of one decode step of a workload: `n_layers_sample` decoder
-    layers (weights and cache of those layers only) plus the classifier.  Inputs are generated once; `step()` only
-    times oracle calls and returns seconds per token with the layer part scaled to the full depth."""
+    """The oracle, as it stands, on one decode step of a workload: `n_layers_sample` decoder layers (weights and cache
+    of those layers only) plus the classifier.  With all layers this is the WHOLE step, the hidden state chained
+    through every layer; with fewer it is a bounded sample whose layer time is scaled to the full depth.  Inputs are
+    generated once; `step()` only times oracle calls and returns seconds per token."""
 
     def __init__(self, shape, batch, context, n_layers_sample, seed=0, with_classifier=True):
         from oracle import kl_oracle as ko
@@ -410,6 +417,9 @@ class OracleSampler:
     def describe(self) -> str:
         cls = (f" + classifier executed ({self.t_cls:.2f} s)" if self.with_classifier
                else "; classifier time taken from one separate execution")
+        if self.n == self.shape.n_layers:
+            return (f"one WHOLE decode step at position {self.context}: all {self.n} decoder layers executed "
+                    f"({self.t_layers:.2f} s){cls}, nothing scaled")
         return (f"one decode step at position {self.context}: {self.n} of {self.shape.n_layers} decoder layers "
                 f"executed ({self.t_layers:.2f} s){cls}, layer time scaled to {self.shape.n_layers} layers")
 
@@ -422,39 +432,46 @@ def oracle_sample(shape, batch, context, n_layers_sample, seed=0, device="cpu"):
 
 
 def run_reference(args, shape, batch, context):
-    """Reference arm = the CPU oracle on the host cores.  Every step is a bounded sample of one decode step of the
-    workload: one decoder layer (scaled to the full depth) and, on the first timed step only, the classifier, whose
-    time is then added to every step -- so that K + W steps end within a few minutes."""
+    """Reference arm = the CPU oracle on the host cores.  For models whose weights the host holds at once (up to the 8B
+    shape) every step is a WHOLE decode step of the workload -- all layers, classifier, the hidden state chained
+    through -- executed for as many of the W + K steps as about two minutes allow (the count is reported; steps beyond
+    it take the mean of the executed ones).  For larger models a step is a bounded sample: one decoder layer (scaled to
+    the full depth) plus the classifier."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import kl_oracle as ko
     ko.build()
-    smp = OracleSampler(shape, batch, context, 1, with_classifier=True)
-    sec_first = smp.step()                       # also the calibration: one layer + the classifier
-    t_cls, t_layer = smp.t_cls, smp.t_layers
-    smp.with_classifier = False
+    n = oracle_layers_that_fit(shape) or 1
+    whole = n == shape.n_layers
+    smp = OracleSampler(shape, batch, context, n, with_classifier=True)
+    t_start = time.perf_counter()
+    sec_first = smp.step()                       # untimed warm-up / calibration (pages the weights in)
+    t_one = smp.t_layers + smp.t_cls
     total = args.steps + args.warmup
-    # keep the whole run near 150 s: repeat the layer sample only as often as that allows, reuse the mean after
-    afford = max(1, min(total, int(150.0 / max(t_layer, 1e-3))))
-    times = []
+    afford = max(1, min(total, int(120.0 / max(t_one, 1e-3))))
+    times, executed = [], 0
     for i in range(total):
         if i < afford:
-            sec = smp.step() + t_cls / batch
+            sec = smp.step()
+            executed += 1
         else:
             sec = statistics.mean(times) if times else sec_first
         if i >= args.warmup or not times:
             times.append(sec)
     sec = statistics.mean(times)
     value = 1.0 / sec
-    desc = (f"per step: 1 of {shape.n_layers} decoder layers executed at position {context} ({t_layer:.2f} s, scaled "
-            f"to {shape.n_layers}) + classifier executed once ({t_cls:.2f} s); {min(afford, total)} of {total} steps "
-            f"executed, the rest take their mean")
+    what = (f"WHOLE decode steps at position {context} (all {shape.n_layers} layers + classifier, nothing scaled)" if whole else
+            f"bounded samples of a decode step at position {context}: {n} of {shape.n_layers} decoder layers executed and "
+            f"scaled to {shape.n_layers}, + the classifier")
+    desc = (f"{what}; {executed} of the {total} warm-up + timed steps executed ({time.perf_counter() - t_start:.0f} s of oracle "
+            f"time), the others take the mean of the executed ones")
     line = {
         "impl": "reference", "metric": "decode tokens/s", "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3 * batch, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": batch, "context": context},
+        "config": {"workload": args.workload, "batch": batch, "context": context, "l2": "inputs larger than L2 (weights and KV streamed once per step)"},
+        "steps_executed": executed, "whole_steps": whole,
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": smp.threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -546,12 +563,12 @@ def run_ours(args, shape, batch, context):
         "metric": "decode tokens/s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_token / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": batch, "context": context,
-                   "mode": "looped, one launch per token (kl_decode_greedy: decoder layers + classifier + sampling)",
-                   "storage": "bf16 weights and KV, fp32 activations and accumulation",
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "batch_schedule": "one sequence after another (weights streamed once per sequence)" if batch > 1 else "n/a",
-                   "l2": "inputs larger than L2 (weights streamed once per step)", "max_ctx": max_ctx},
+        "config": {"workload": args.workload, "batch": batch, "context": context, "l2": "inputs larger than L2 (weights and KV streamed once per step)"},
+        "details": {"mode": "looped, one launch per token (kl_decode_greedy: decoder layers + classifier + sampling)",
+                    "storage": "bf16 weights and KV, fp32 activations and accumulation",
+                    "parallelism": "replicas only" if world > 1 else "single GPU",
+                    "batch_schedule": "one sequence after another (weights streamed once per sequence)" if batch > 1 else "n/a",
+                    "max_ctx": max_ctx},
         "clocks": clocks, "gpu_launches": int(round(token_launches * K)),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
                 "d2h_bytes_per_step": 4 * batch, "call": "kl_decode_greedy_host (tokens and positions in, next tokens out)"},
@@ -598,8 +615,9 @@ def run_ours(args, shape, batch, context):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import kl_oracle as ko
         ko.build()
-        # bounded sample: up to 8 layers + the classifier of one step, repeated until about 10 s of CPU work
-        smp = OracleSampler(shape, batch, context, min(8, shape.n_layers))
+        # whole decode steps where the host holds the model (up to the 8B shape), otherwise a bounded sample of up to 8
+        # layers + the classifier; repeated until about 12 s of CPU work
+        smp = OracleSampler(shape, batch, context, oracle_layers_that_fit(shape) or min(8, shape.n_layers))
         secs = [smp.step()]
         t_exec = smp.t_layers + smp.t_cls
         while len(secs) < 40 and t_exec * (len(secs) + 1) < 12.0:
@@ -672,11 +690,12 @@ def run_ours_batched(args, shape, batch, context):
         "metric": "decode tokens/s", "value": tokens / (ms_greedy * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms_greedy / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": args.workload, "batch": batch, "context": context, "mode": "batched tensor-core path, kl_decode_greedy chained on the device",
-                   "storage": "bf16 weights and KV; fp32 activations enter the tcgen05 MMAs as two bf16 halves, fp32 accumulation",
-                   "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "batch_schedule": "all sequences per launch (weights streamed once per step)",
-                   "l2": "inputs larger than L2 (weights and KV streamed once per step)", "max_ctx": max_ctx},
+        "config": {"workload": args.workload, "batch": batch, "context": context, "l2": "inputs larger than L2 (weights and KV streamed once per step)"},
+        "details": {"mode": "batched tensor-core path, kl_decode_greedy chained on the device",
+                    "storage": "bf16 weights and KV; fp32 activations enter the tcgen05 MMAs as two bf16 halves, fp32 accumulation",
+                    "parallelism": "replicas only" if world > 1 else "single GPU",
+                    "batch_schedule": "all sequences per launch (weights streamed once per step)",
+                    "max_ctx": max_ctx},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": tokens / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": 8 * batch,
                 "d2h_bytes_per_step": 4 * batch, "call": "kl_decode_greedy_host (tokens and positions in, next tokens out)"},
@@ -707,7 +726,7 @@ def run_ours_batched(args, shape, batch, context):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import kl_oracle as ko
         ko.build()
-        smp = OracleSampler(shape, batch, context, 1)
+        smp = OracleSampler(shape, batch, context, (oracle_layers_that_fit(shape) or 1) if batch * context <= 16384 else 1)
         secs = [smp.step()]
         t_exec = smp.t_layers + smp.t_cls
         while len(secs) < 40 and t_exec * (len(secs) + 1) < 12.0:
