@@ -85,7 +85,8 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
 }
 
 // The attention half of a layer as one call: RoPE, the unit's ring chunks, the merges, the deferred cache append.
-__device__ __noinline__ void attention_block(const Params& p, const Smem& s, const StepCtx& cx, uint32_t l, uint32_t cta,
+template <class SM>
+__device__ __noinline__ void attention_block(const Params& p, const SM& s, const StepCtx& cx, uint32_t l, uint32_t cta,
                                              uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
     if (p.attn_tc) {
         attention_stage_and_advance<0>(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
@@ -102,21 +103,22 @@ __device__ __noinline__ void attention_block(const Params& p, const Smem& s, con
 
 // Set-up every persistent kernel starts with: the ring's barriers, the abort flag, the unit table.  False: an earlier
 // kernel of this step flagged bad input and the launch is a no-op.
-__device__ __forceinline__ bool cta_begin(const Params& p, const Smem& s, uint32_t tid, const float* rope) {
+template <class SM>
+__device__ __forceinline__ bool cta_begin(const Params& p, const SM& s, uint32_t tid, const float* rope) {
     if (tid == 0) {
         // step number and position as the launch finds them: read before any CTA can have finished a token
-        s.ctx->step = ld_step(p.step_dev);
-        s.ctx->pos = (uint32_t)p.positions[p.b0];
-        s.ctx->rope_cs = rope;
+        s.ctx()->step = ld_step(p.step_dev);
+        s.ctx()->pos = (uint32_t)p.positions[p.b0];
+        s.ctx()->rope_cs = rope;
         for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
-            mbar_init(smem_u32(&s.full[i]), 1);
-            mbar_init(smem_u32(&s.empty[i]), 1);
+            mbar_init(smem_u32(&s.full()[i]), 1);
+            mbar_init(smem_u32(&s.empty()[i]), 1);
         }
-        *s.abort_flag = 0;
+        *s.abort_flag() = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (tid < UNIT_SLOTS) s.unit_cnt[tid] = 0;
+    if (tid < UNIT_SLOTS) s.unit_cnt()[tid] = 0;
     __syncthreads();
     return *p.status == 0;
 }
@@ -128,10 +130,11 @@ __device__ __forceinline__ bool cta_begin(const Params& p, const Smem& s, uint32
 //   l == L: the classifier, as stage 0 of one more pass (one more stage on the same ring, same code)
 // xa_slot: tag slot under which the hidden state entering stage 0 was published (TG_XA; TG_NEXT for an embedding
 // written inside the running launch).  ctr_target: value of the layer's gate/up counter when all CTAs have signalled.
-__device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32_t l, uint32_t st,
+template <class SM>
+__device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t l, uint32_t st,
                                           uint32_t xa_slot, uint32_t ctr_target, uint32_t cta, uint32_t ctid, uint32_t warp,
                                           uint32_t lane, RingCursor& rc, WarpRing& wr) {
-    const StepCtx& cx = *s.ctx;
+    const StepCtx& cx = *s.ctx();
     const size_t lo = (size_t)l * p.layer_stride;
     const bool cls = l == p.L;
     // test hook: the results of one stage of layer 0 get a tag nobody waits for
@@ -144,9 +147,9 @@ __device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32
     if (st == ST_QKV) {
         // RMSNorm + QKV projection (classifier: final RMSNorm + W_lm).  The poll on xa's tags is the wait for the
         // previous layer (or the embedding).
-        trace_stamp(p, cta, l, 0, ctid);
+        trace_stamp(p, s, cta, l, 0, ctid);
         xscale = load_vec(p, s, p.xa, p.H, tag_of(p, cx, l, xa_slot), true, cls ? p.gf : p.g1 + lo, ctid);
-        trace_stamp(p, cta, l, 1, ctid);
+        trace_stamp(p, s, cta, l, 1, ctid);
         if (cls) {
             out = {nullptr, p.logits, nullptr, 0u};
             plan = PL_LM;
@@ -154,23 +157,23 @@ __device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32
             out = {p.qkv, nullptr, nullptr, skip == ST_QKV ? bad : tag_of(p, cx, l, TG_QKV)};
         }
     } else if (st == ST_ATTN) {
-        trace_stamp(p, cta, l, 2, ctid);
+        trace_stamp(p, s, cta, l, 2, ctid);
         // RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
         attention_block(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
-        trace_stamp(p, cta, l, 4, ctid);
+        trace_stamp(p, s, cta, l, 4, ctid);
         return;
     } else if (st == ST_O) {
         // output projection + residual (xa -> xb).  The poll on o's tags waits for the attention units.
         load_vec(p, s, p.o, p.QD, skip == ST_ATTN ? bad : tag_of(p, cx, l, TG_O), false, nullptr, ctid);
-        trace_stamp(p, cta, l, 6, ctid);
+        trace_stamp(p, s, cta, l, 6, ctid);
         out = {p.xb, nullptr, p.xa, skip == ST_O ? bad : tag_of(p, cx, l, TG_XB)};
         plan = PL_O;
         ep = EP_RESIDUAL;
     } else if (st == ST_GU) {
-        trace_stamp(p, cta, l, 7, ctid);
+        trace_stamp(p, s, cta, l, 7, ctid);
         // RMSNorm + gate/up projections + SwiGLU
         xscale = load_vec(p, s, p.xb, p.H, tag_of(p, cx, l, TG_XB), true, p.g2 + lo, ctid);
-        trace_stamp(p, cta, l, 9, ctid);
+        trace_stamp(p, s, cta, l, 9, ctid);
         out = {nullptr, p.h, nullptr, 0u};
         plan = PL_GU;
         ep = EP_SWIGLU;
@@ -179,7 +182,7 @@ __device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32
         // straight from L2 into registers (too wide for shared memory): its readiness is a counter, signalled with
         // release at the end of the gate/up stage and awaited with acquire here
         stage_wait(p, s, p.counters + l, ctr_target, ctid);
-        trace_stamp(p, cta, l, 12, ctid);
+        trace_stamp(p, s, cta, l, 12, ctid);
         out = {p.xa, nullptr, p.xb, skip == ST_D ? bad : tag_of(p, cx, l + 1, TG_XA)};
         plan = PL_D;
         ep = EP_RESIDUAL;
@@ -188,19 +191,19 @@ __device__ __forceinline__ void run_stage(const Params& p, const Smem& s, uint32
     gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
     if (st == ST_GU) {
         stage_signal(p.counters + l, ctid, skip == ST_GU);
-        trace_stamp(p, cta, l, 10, ctid);
+        trace_stamp(p, s, cta, l, 10, ctid);
     } else if (st == ST_D) {
-        trace_stamp(p, cta, l, 13, ctid);
+        trace_stamp(p, s, cta, l, 13, ctid);
     }
 }
 
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
 // stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
 // boundary after every operator group).
+template <bool TR>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
                                                                  uint32_t sbeg, uint32_t send) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, p);
+    const SmemT<TR> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;   // an earlier kernel of this step flagged bad input: the step is a no-op
     if (warp == NCW) {
@@ -216,8 +219,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
 __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid_constant__ Params p) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, p);
+    const SmemT<false> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;
     if (warp == NCW) {
@@ -329,7 +331,8 @@ __global__ void kl_token_plan_kernel(const __grid_constant__ Params p, float* ro
     }
 }
 
-__device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, uint32_t cta, const TokenParams& t) {
+template <class SM>
+__device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uint32_t cta, const TokenParams& t) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     const uint32_t step0 = ld_step(p.step_dev), pos0 = (uint32_t)p.positions[0];
     for (uint32_t k = 0; k < t.K && !r.aborted; ++k) {
@@ -369,18 +372,19 @@ __device__ __forceinline__ void produce_tokens(const Params& p, const Smem& s, u
 // token and writes the next embedding.  false: that was the last token of the launch, or a wait of this launch gave up
 // -- in which case token, position and the next embedding are left alone (the step's outputs are meaningless; the
 // chain has to be restarted).
-__device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const TokenParams& t, uint32_t k,
+template <class SM>
+__device__ __noinline__ bool sample_token(const Params& p, const SM& s, const TokenParams& t, uint32_t k,
                                           uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane) {
     const bool final = k + 1u == t.K;
-    const StepCtx cx = *s.ctx;   // a copy: the shared one moves on to the next token below
+    const StepCtx cx = *s.ctx();   // a copy: the shared one moves on to the next token below
     // ---- greedy sampling: this CTA's rows first
     const GemvPlan& plm = p.plan[PL_LM];
     asm volatile("fence.proxy.async;" ::: "memory");   // the cache rows this thread appended: readable by later bulk copies
     consumer_bar();   // the rows this CTA stored are visible to all of its threads
-    float* sv = s.unit_part;                                           // [NCW] maxima, then [NCW] indices, then flags
-    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part) + NCW;
+    float* sv = s.unit_part();                                           // [NCW] maxima, then [NCW] indices, then flags
+    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part()) + NCW;
     // [0] this CTA drew the last ticket, [1] token, [2] position, [3] next step number, [4] stop: a wait of this launch gave up
-    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part) + 2 * NCW;
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part()) + 2 * NCW;
     const CtaRange cr = cta_units(plm, cta, p.P);
     const uint32_t r0 = cr.u0 * plm.rpc, r1 = min(cr.u1 * plm.rpc, p.V);
     float bv = -INFINITY;
@@ -398,7 +402,7 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
         t.part_val[cta] = bv;
         t.part_idx[cta] = bi;
         sh[0] = (atom_add_acq_rel(t.ticket, 1u) == p.P * (k + 1u) - 1u) ? 1u : 0u;
-        sh[4] = (*s.abort_flag != 0 || __ldcg(p.status) != 0) ? 1u : 0u;
+        sh[4] = (*s.abort_flag() != 0 || __ldcg(p.status) != 0) ? 1u : 0u;
     }
     consumer_bar();
     const bool last_cta = sh[0] != 0u, stop = sh[4] != 0u;
@@ -450,9 +454,9 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
         for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
     }
     if (ctid == 0) {   // the next token of the launch: one step and one position further, the next rotary table
-        s.ctx->step = cx.step + 1u;
-        s.ctx->pos = cx.pos + 1u;
-        s.ctx->rope_cs = cx.rope_cs + p.hd;
+        s.ctx()->step = cx.step + 1u;
+        s.ctx()->pos = cx.pos + 1u;
+        s.ctx()->rope_cs = cx.rope_cs + p.hd;
     }
     consumer_bar();   // the flags above are read before the next stage reuses the area
     return !stop && !final;
@@ -462,8 +466,7 @@ __device__ __noinline__ bool sample_token(const Params& p, const Smem& s, const 
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
-    extern __shared__ __align__(1024) uint8_t smem_raw[];
-    const Smem s = carve_smem(smem_raw, p);
+    const SmemT<false> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, t.rope)) return;
     if (warp == NCW) {
@@ -978,7 +981,8 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
     // The shared-memory limit is an attribute of the kernel, not of a handle: it is raised to the device's opt-in
     // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
-    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     {
         int tocc = 0;
@@ -987,7 +991,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
         (void)cudaGetLastError();
     }
     int occ = 0;
-    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel, NTHREADS, h->smem_bytes);
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true>, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
         fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
                         "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
@@ -1331,22 +1335,24 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         kl_status rc;
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
         uint32_t sbeg = 0, send = 5;
+        // the instantiation with the trace stamps compiled in only while a trace buffer is set
+        const void* decoder_fn = p.trace != nullptr ? (const void*)kl_decoder_kernel<true> : (const void*)kl_decoder_kernel<false>;
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1, &sbeg, &send};
-            if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+            if ((rc = launch_persistent(h, decoder_fn, args, st)) != KL_OK) return rc;
         } else if (h->mode == KL_MODE_PER_LAYER) {
             for (uint32_t l = 0; l < p.L; ++l) {
                 uint32_t l0 = l, l1 = l + 1;
                 void* args[] = {&p, &l0, &l1, &sbeg, &send};
-                if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+                if ((rc = launch_persistent(h, decoder_fn, args, st)) != KL_OK) return rc;
             }
         } else {
             for (uint32_t l = 0; l < p.L; ++l)
                 for (uint32_t sg = 0; sg < 5; ++sg) {
                     uint32_t l0 = l, l1 = l + 1, s0 = sg, s1 = sg + 1;
                     void* args[] = {&p, &l0, &l1, &s0, &s1};
-                    if ((rc = launch_persistent(h, (const void*)kl_decoder_kernel, args, st)) != KL_OK) return rc;
+                    if ((rc = launch_persistent(h, decoder_fn, args, st)) != KL_OK) return rc;
                 }
         }
         if (ev && b == 0 && cudaEventRecord(ev[1], st) != cudaSuccess) return KL_ERR_CUDA;

@@ -33,7 +33,7 @@ constexpr int UNIT_SLOTS = 8;             // in-flight multi-chunk units tracked
 constexpr int MAX_RPC_SPLIT = 4;           // rows per unit when units are split into column pieces
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
 constexpr int MAX_G = 8;                   // query heads per KV head
-constexpr int SMEM_MISC_BYTES = 6656;  // barriers, chunk-sequence plan, reduction scratch, unit table (see carve_smem)
+constexpr int SMEM_MISC_BYTES = 7168;  // barriers, reduction scratch, unit table, step context (see SmemT); a multiple of 1024
 
 enum StageId { ST_QKV = 0, ST_ATTN = 1, ST_O = 2, ST_GU = 3, ST_D = 4, ST_LM = 5 };
 enum EpilogueKind { EP_STORE = 0, EP_RESIDUAL = 1, EP_SWIGLU = 2 };
@@ -118,11 +118,15 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 }
 
 constexpr int TRACE_STAMPS = 16;
-__device__ __forceinline__ void chunk_stamp(const Params& p, uint32_t cta, uint64_t n, int k) {
-    if (p.chunk_trace != nullptr && cta == 0 && n < CHUNK_TRACE_ROWS) p.chunk_trace[n * 4 + k] = globaltimer_ns();
+template <class SM>
+__device__ __forceinline__ void chunk_stamp(const Params& p, const SM&, uint32_t cta, uint64_t n, int k) {
+    if constexpr (SM::kTrace)
+        if (p.chunk_trace != nullptr && cta == 0 && n < CHUNK_TRACE_ROWS) p.chunk_trace[n * 4 + k] = globaltimer_ns();
 }
-__device__ __forceinline__ void trace_stamp(const Params& p, uint32_t cta, uint32_t layer, int k, uint32_t ctid) {
-    if (p.trace != nullptr && ctid == 0) p.trace[((size_t)cta * p.L + layer) * TRACE_STAMPS + k] = globaltimer_ns();
+template <class SM>
+__device__ __forceinline__ void trace_stamp(const Params& p, const SM&, uint32_t cta, uint32_t layer, int k, uint32_t ctid) {
+    if constexpr (SM::kTrace)
+        if (p.trace != nullptr && ctid == 0) p.trace[((size_t)cta * p.L + layer) * TRACE_STAMPS + k] = globaltimer_ns();
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -238,37 +242,37 @@ __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 
 
 // ------------------------------------------------------------------------------------------------ shared state
 
-struct Smem {
-    uint8_t* ring;          // nslots * SLOT_BYTES
-    float* vec;             // input vector of the current GEMV stage (lane-permuted), or attention workspace
-    uint64_t* full;         // [MAX_SLOTS] copy landed
-    uint64_t* empty;        // [MAX_SLOTS] consumer has finished reading
-    float* red;             // [NCW]
-    float* unit_part;       // [UNIT_SLOTS][MAX_PIECES]
-    int* unit_cnt;          // [UNIT_SLOTS]
-    volatile int* abort_flag;
-    StepCtx* ctx;           // step number, position and rotary table of the token being decoded (see StepCtx)
+// Dynamic shared memory of the persistent kernels, at fixed offsets from its start, so that no thread holds a pointer
+// to any part of it in a register: barriers and small tables first (SMEM_MISC_BYTES, a multiple of 1024), then the
+// ring (slots on 1024-byte boundaries, as the swizzled K/V boxes need), then the vector area.
+//   full  [MAX_SLOTS] copy landed                       empty [MAX_SLOTS] consumer has finished reading
+//   red   [NCW] reduction scratch                       unit_part [UNIT_SLOTS][MAX_PIECES][MAX_RPC_SPLIT]
+//   unit_cnt [UNIT_SLOTS], abort flag                   ctx  step number, position and rotary table (see StepCtx)
+//   ring  nslots * nsw * SLOT_BYTES                     vec  input vector of the current GEMV stage (lane-permuted),
+//                                                            or the attention workspace
+// TR selects the instantiation with the trace stamps compiled in (kl_set_trace); the production kernels carry none.
+extern __shared__ __align__(1024) uint8_t kl_smem[];
+template <bool TR>
+struct SmemT {
+    static constexpr bool kTrace = TR;
+    __device__ __forceinline__ static uint64_t* full() { return reinterpret_cast<uint64_t*>(kl_smem); }
+    __device__ __forceinline__ static uint64_t* empty() { return reinterpret_cast<uint64_t*>(kl_smem + 256); }
+    __device__ __forceinline__ static float* red() { return reinterpret_cast<float*>(kl_smem + 1536); }
+    __device__ __forceinline__ static float* unit_part() { return reinterpret_cast<float*>(kl_smem + 2048); }
+    __device__ __forceinline__ static int* unit_cnt() { return reinterpret_cast<int*>(kl_smem + 6144); }
+    __device__ __forceinline__ static volatile int* abort_flag() { return reinterpret_cast<volatile int*>(kl_smem + 6144 + 4 * UNIT_SLOTS); }
+    __device__ __forceinline__ static StepCtx* ctx() { return reinterpret_cast<StepCtx*>(kl_smem + 6208); }
+    __device__ __forceinline__ static uint8_t* ring() { return kl_smem + SMEM_MISC_BYTES; }
+    __device__ __forceinline__ static float* vec(const Params& p) {
+        return reinterpret_cast<float*>(kl_smem + SMEM_MISC_BYTES + (size_t)p.nslots * p.nsw * SLOT_BYTES);
+    }
 };
-
-__device__ __forceinline__ Smem carve_smem(uint8_t* base, const Params& p) {
-    Smem s;
-    s.ring = base;
-    s.vec = reinterpret_cast<float*>(base + (size_t)p.nslots * p.nsw * SLOT_BYTES);
-    uint8_t* misc = reinterpret_cast<uint8_t*>(s.vec) + (size_t)p.vec_floats * 4;
-    s.full = reinterpret_cast<uint64_t*>(misc);                    // [MAX_SLOTS] 192 B
-    s.empty = reinterpret_cast<uint64_t*>(misc + 256);             // [MAX_SLOTS]
-    s.red = reinterpret_cast<float*>(misc + 1536);                 // 128 B
-    s.unit_part = reinterpret_cast<float*>(misc + 2048);           // [UNIT_SLOTS][MAX_PIECES][MAX_RPC_SPLIT] 4 KB
-    s.unit_cnt = reinterpret_cast<int*>(misc + 6144);              // [UNIT_SLOTS]
-    s.abort_flag = s.unit_cnt + UNIT_SLOTS;
-    s.ctx = reinterpret_cast<StepCtx*>(misc + 6208);
-    return s;
-}
 
 // Records the first error and tells every waiter of this CTA to give up.  After an abort every wait returns at
 // once but the control flow (stage order, CTA barriers) is unchanged, so no warp is left behind at a barrier; the
 // step's outputs are then meaningless and the status word says so.
-__device__ __noinline__ bool raise_abort(const Params& p, const Smem& s, int code, int where = 0) {
+template <class SM>
+__device__ __noinline__ bool raise_abort(const Params& p, const SM& s, int code, int where = 0) {
     bool first = false;
     if (atomicCAS(p.status, 0, code) == 0) {   // following words: which wait gave up, where (diagnostics)
         p.status[1] = where;
@@ -276,19 +280,20 @@ __device__ __noinline__ bool raise_abort(const Params& p, const Smem& s, int cod
         p.status[3] = (int)threadIdx.x;
         first = true;
     }
-    *s.abort_flag = 1;
+    *s.abort_flag() = 1;
     return first;
 }
 
 // Bounded mbarrier wait.  Returns false when the wait was abandoned (limit reached or abort raised elsewhere).
-__device__ __forceinline__ bool mbar_wait(const Params& p, const Smem& s, uint32_t bar, uint32_t parity) {
+template <class SM>
+__device__ __forceinline__ bool mbar_wait(const Params& p, const SM& s, uint32_t bar, uint32_t parity) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*s.abort_flag) return false;
+    if (*s.abort_flag()) return false;
     const uint64_t t0 = globaltimer_ns();
     uint32_t it = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++it & 63u) == 0) {
-            if (*s.abort_flag) return false;
+            if (*s.abort_flag()) return false;
             if (globaltimer_ns() - t0 > p.wait_ns) {
                 raise_abort(p, s, ERR_SYNC_TIMEOUT, 500);   // out of line: it runs once, if ever
                 return false;
@@ -305,13 +310,14 @@ struct PollGuard {
     uint32_t it;
     int where;
 };
-__device__ __forceinline__ bool poll_continue(const Params& p, const Smem& s, PollGuard& g) {
+template <class SM>
+__device__ __forceinline__ bool poll_continue(const Params& p, const SM& s, PollGuard& g) {
     if (g.it == 0) g.t0 = globaltimer_ns();
     if (KL_POLL_NS) __nanosleep(KL_POLL_NS);   // keeps the polling traffic of a waiting CTA off the L2 ports the late CTAs still need
     if ((++g.it & 7u) == 0) {
-        if (*s.abort_flag) return false;
+        if (*s.abort_flag()) return false;
         if (__ldcg(p.status) != 0) {
-            *s.abort_flag = 1;
+            *s.abort_flag() = 1;
             return false;
         }
         if (globaltimer_ns() - g.t0 > p.wait_ns) {
@@ -452,8 +458,9 @@ __device__ __forceinline__ void ring_advance_consume(const Params& p, WarpRing& 
     }
 }
 // The whole warp has finished reading the slot it consumed last (call after __syncwarp): hand it back.
-__device__ __forceinline__ void ring_release(const Params& p, const Smem& s, const WarpRing& r, uint32_t warp, uint32_t lane) {
-    if (lane == 0) mbar_arrive(smem_u32(&s.empty[warp * p.nsw + r.rslot]));
+template <class SM>
+__device__ __forceinline__ void ring_release(const Params& p, const SM& s, const WarpRing& r, uint32_t warp, uint32_t lane) {
+    if (lane == 0) mbar_arrive(smem_u32(&s.empty()[warp * p.nsw + r.rslot]));
 }
 __device__ __forceinline__ WarpRing ring_begin() {
     WarpRing r;
@@ -471,17 +478,18 @@ struct RingProd {
 };
 
 // Waits for the slot of the next chunk, arms its barrier and starts one or two linear copies into it.
-__device__ __forceinline__ void prod_issue(const Params& p, const Smem& s, RingProd& r, const uint8_t* src0, uint32_t bytes0,
+template <class SM>
+__device__ __forceinline__ void prod_issue(const Params& p, const SM& s, RingProd& r, const uint8_t* src0, uint32_t bytes0,
                                            const uint8_t* src1, uint32_t bytes1, uint32_t dst1) {
     if (r.aborted) return;
     const uint32_t slot = r.c * p.nsw + r.k;
-    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty[slot]), (r.use - 1u) & 1u)) {
+    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (r.use - 1u) & 1u)) {
         r.aborted = true;
         return;
     }
-    const uint32_t bar = smem_u32(&s.full[slot]);
-    const uint32_t dst = smem_u32(s.ring) + slot * SLOT_BYTES;
-    chunk_stamp(p, blockIdx.x, r.n, 0);
+    const uint32_t bar = smem_u32(&s.full()[slot]);
+    const uint32_t dst = smem_u32(s.ring()) + slot * SLOT_BYTES;
+    chunk_stamp(p, s, blockIdx.x, r.n, 0);
     mbar_arrive_expect_tx(bar, bytes0 + bytes1);
     tma_bulk_g2s(dst, src0, bytes0, bar, r.pol);
     if (bytes1) tma_bulk_g2s(dst + dst1, src1, bytes1, bar, r.pol);
@@ -497,16 +505,17 @@ __device__ __forceinline__ void prod_issue(const Params& p, const Smem& s, RingP
 // Same for a chunk of K/V rows as swizzled boxes of the cache tensor: [pb rows] x [64 columns] per box, K boxes in
 // the first half of the slot, V boxes in the second; a box is always written whole (rows outside the chunk's own
 // positions are ignored by the consumer).
-__device__ __forceinline__ void prod_issue_boxes(const Params& p, const Smem& s, RingProd& r, int32_t yk, int32_t yv) {
+template <class SM>
+__device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, RingProd& r, int32_t yk, int32_t yv) {
     if (r.aborted) return;
     const uint32_t slot = r.c * p.nsw + r.k;
-    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty[slot]), (r.use - 1u) & 1u)) {
+    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (r.use - 1u) & 1u)) {
         r.aborted = true;
         return;
     }
-    const uint32_t bar = smem_u32(&s.full[slot]);
-    const uint32_t dst = smem_u32(s.ring) + slot * SLOT_BYTES;
-    chunk_stamp(p, blockIdx.x, r.n, 0);
+    const uint32_t bar = smem_u32(&s.full()[slot]);
+    const uint32_t dst = smem_u32(s.ring()) + slot * SLOT_BYTES;
+    chunk_stamp(p, s, blockIdx.x, r.n, 0);
     mbar_arrive_expect_tx(bar, (uint32_t)SLOT_BYTES);
     const uint32_t box_bytes = SLOT_BYTES / 2 / (p.hd / 64u);
     for (uint32_t bx = 0; bx < p.hd / 64u; ++bx) {
@@ -525,7 +534,8 @@ __device__ __forceinline__ void prod_issue_boxes(const Params& p, const Smem& s,
 
 // Streams this CTA's share of one matrix (units [u0, u1) of the plan): one linear run of bytes cut into chunks,
 // per chunk only pointer increments.
-__device__ __forceinline__ void produce_matrix(const Params& p, const Smem& s, RingProd& r, const GemvPlan& pl,
+template <class SM>
+__device__ __forceinline__ void produce_matrix(const Params& p, const SM& s, RingProd& r, const GemvPlan& pl,
                                                const __nv_bfloat16* base, uint32_t cta) {
     const CtaRange cr = cta_units(pl, cta, p.P);
     const uint8_t* ptr = reinterpret_cast<const uint8_t*>(base) + (size_t)cr.u0 * pl.rpc * pl.K * 2u;
@@ -541,7 +551,8 @@ __device__ __forceinline__ void produce_matrix(const Params& p, const Smem& s, R
 }
 
 // Streams the cached K/V rows of this CTA's attention unit for one layer.
-__device__ __forceinline__ void produce_attention(const Params& p, const Smem& s, RingProd& r, const AttnUnit& u,
+template <class SM>
+__device__ __forceinline__ void produce_attention(const Params& p, const SM& s, RingProd& r, const AttnUnit& u,
                                                   uint32_t layer) {
     if (!u.active) return;
     const uint32_t pb = attn_positions_per_chunk(p);
@@ -569,14 +580,15 @@ __device__ __forceinline__ void produce_attention(const Params& p, const Smem& s
 
 // After an abandoned run no bulk copy may still be writing this CTA's shared memory when it exits: wait (bounded)
 // for the last copy armed on every slot.
-__device__ __forceinline__ void produce_drain(const Params& p, const Smem& s, const RingProd& r) {
+template <class SM>
+__device__ __forceinline__ void produce_drain(const Params& p, const SM& s, const RingProd& r) {
     if (!r.aborted) return;
     const uint64_t t0 = globaltimer_ns();
     for (uint32_t cc = 0; cc < p.nslots; ++cc) {
         for (uint32_t kk = 0; kk < p.nsw; ++kk) {
             const uint32_t cnt = r.use + ((kk < r.k || (kk == r.k && cc < r.c)) ? 1u : 0u);  // uses of this slot so far
             if (cnt == 0) continue;
-            const uint32_t bar = smem_u32(&s.full[cc * p.nsw + kk]);
+            const uint32_t bar = smem_u32(&s.full()[cc * p.nsw + kk]);
             while (!mbar_try_wait(bar, (cnt - 1u) & 1u)) {
                 if (globaltimer_ns() - t0 > p.wait_ns) return;
             }
@@ -585,7 +597,8 @@ __device__ __forceinline__ void produce_drain(const Params& p, const Smem& s, co
 }
 
 // The producer thread of the decoder kernel: layers [l0, l1).
-__device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, uint32_t cta, uint32_t l0, uint32_t l1,
+template <class SM>
+__device__ __forceinline__ void produce_decoder(const Params& p, const SM& s, uint32_t cta, uint32_t l0, uint32_t l1,
                                                 uint32_t sbeg, uint32_t send) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     const AttnUnit u = attn_unit(p, cta, (uint32_t)p.positions[p.b0]);
@@ -602,7 +615,8 @@ __device__ __forceinline__ void produce_decoder(const Params& p, const Smem& s, 
     produce_drain(p, s, r);
 }
 // ... and of the classifier kernel.
-__device__ __forceinline__ void produce_classifier(const Params& p, const Smem& s, uint32_t cta) {
+template <class SM>
+__device__ __forceinline__ void produce_classifier(const Params& p, const SM& s, uint32_t cta) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
     produce_drain(p, s, r);
@@ -623,7 +637,8 @@ __device__ __forceinline__ uint32_t vec_perm(uint32_t e) {
 // outputs instead of to its 4096 inputs (one pass and one barrier less).  Every CTA recomputes it; the summation
 // order is fixed.  Without `norm` the function returns 1.  This poll is what replaces the grid-wide barrier of a kernel boundary: the first read that finds
 // all tags in place already holds the data.
-__device__ __noinline__ float load_vec(const Params& p, const Smem& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
+template <class SM>
+__device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* src, uint32_t n, uint32_t tag, bool norm,
                                           const __nv_bfloat16* gain, uint32_t ctid) {
     constexpr int NB = 4;  // groups of four values kept in flight per thread (two 16-byte loads each)
     // The vector area is about to be overwritten: every warp of the CTA must be done with what the previous stage
@@ -670,11 +685,11 @@ __device__ __noinline__ float load_vec(const Params& p, const Smem& s, const TW*
                 // the gains go in now, the normaliser (one number for the whole vector) is applied to the stage's outputs
                 const float4 o = make_float4(v[i].x * bf_lo(gk[i].x), v[i].y * bf_hi(gk[i].x), v[i].z * bf_lo(gk[i].y),
                                              v[i].w * bf_hi(gk[i].y));
-                *reinterpret_cast<float4*>(s.vec + vec_perm(e)) = o;
+                *reinterpret_cast<float4*>(s.vec(p) + vec_perm(e)) = o;
             }
         }
     }
-    if (norm && p.trace != nullptr && ctid == 0) {   // stamps 8 / 11: thread 0 holds valid data (diagnostic)
+    if (SM::kTrace && norm && p.trace != nullptr && ctid == 0) {   // stamps 8 / 11: thread 0 holds valid data (diagnostic)
         const uint32_t layer = (tag >> 4) % p.L;
         p.trace[((size_t)blockIdx.x * p.L + layer) * TRACE_STAMPS + (((tag >> 1) & 7u) == TG_XA ? 8 : 11)] = globaltimer_ns();
     }
@@ -682,13 +697,13 @@ __device__ __noinline__ float load_vec(const Params& p, const Smem& s, const TW*
     if (norm) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        if ((ctid & 31) == 0) s.red[ctid >> 5] = ss;
+        if ((ctid & 31) == 0) s.red()[ctid >> 5] = ss;
     }
     consumer_bar();
     if (norm) {
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) tot += s.red[w];
+        for (int w = 0; w < NCW; ++w) tot += s.red()[w];
         inv = rsqrtf(tot / (float)n + p.eps);
     }
     return inv;
@@ -931,17 +946,18 @@ __device__ __forceinline__ void emit_value(const GemvOut& o, uint32_t idx, float
 
 // Partial sums of a unit's column pieces meet in shared memory; the last piece to arrive adds them in piece order.
 // Called by one lane per chunk.  Returns true for that last piece, with the unit's complete sums in y.
-__device__ __forceinline__ bool unit_combine(const Smem& s, const GemvPlan& pl, const ChunkGeom& g, uint32_t u0,
+template <class SM>
+__device__ __forceinline__ bool unit_combine(const SM& s, const GemvPlan& pl, const ChunkGeom& g, uint32_t u0,
                                              float (&y)[MAX_RPC_SPLIT]) {
     const uint32_t us = (g.unit - u0) % UNIT_SLOTS;
-    volatile float* part = s.unit_part + us * (MAX_PIECES * MAX_RPC_SPLIT);
+    volatile float* part = s.unit_part() + us * (MAX_PIECES * MAX_RPC_SPLIT);
 #pragma unroll
     for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) part[g.piece * MAX_RPC_SPLIT + rr] = y[rr];
     __threadfence_block();
-    const int old = atomicAdd(&s.unit_cnt[us], 1);
+    const int old = atomicAdd(&s.unit_cnt()[us], 1);
     if (old != (int)pl.npieces - 1) return false;
     __threadfence_block();
-    s.unit_cnt[us] = 0;
+    s.unit_cnt()[us] = 0;
 #pragma unroll
     for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = 0.f;
     for (uint32_t j = 0; j < pl.npieces; ++j) {
@@ -951,10 +967,11 @@ __device__ __forceinline__ bool unit_combine(const Smem& s, const GemvPlan& pl, 
     return true;
 }
 
-__device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const GemvPlan& pl, int ep, const GemvOut& out,
+template <class SM>
+__device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const GemvPlan& pl, int ep, const GemvOut& out,
                                         uint32_t cta, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr,
                                         const float* xsrc, float xscale) {
-    // xsrc == nullptr: the input vector is staged in s.vec; otherwise it is read from global memory per piece
+    // xsrc == nullptr: the input vector is staged in s.vec(p); otherwise it is read from global memory per piece
     const CtaRange r = cta_units(pl, cta, p.P);
     const uint32_t nch = (r.u1 - r.u0) * pl.npieces;
     const uint32_t first = rc.first_chunk(warp, p.nslots);
@@ -966,11 +983,11 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
         const ChunkGeom g = chunk_geom(pl, r.u0, i);
         if (!smemx && g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
             if (xsrc) load_xregs_global(x, xsrc, g.kofs, g.klen, lane);
-            else load_xregs(x, s.vec, g.kofs, g.klen, lane);
+            else load_xregs(x, s.vec(p), g.kofs, g.klen, lane);
             x_piece = g.piece;
         }
         const uint32_t slot = warp * p.nsw + wr.cslot;
-        const uint8_t* sp = s.ring + (size_t)slot * SLOT_BYTES;
+        const uint8_t* sp = s.ring() + (size_t)slot * SLOT_BYTES;
         const uint32_t pitch = g.klen * 2u;
         if (smemx) {
             // Rows (or, for rows longer than a slot, column pieces starting at a block of 256) multiplied against the
@@ -978,29 +995,29 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             // multiplied them emits them.
             float res = 0.f;
             if (ep == EP_RESIDUAL && lane < g.nrows) res = ld_tw(out.res + g.row + lane).v;
-            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
             float y[MAX_RPC_SPLIT] = {0.f, 0.f, 0.f, 0.f};
             if (g.nrows == 2) {
                 float acc[2];
-                dot_rows_smemx<2>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
+                dot_rows_smemx<2>(sp, pitch, g.klen, lane, s.vec(p) + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1];
             } else if (g.nrows == 4) {
                 float acc[4];
-                dot_rows_smemx<4>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
+                dot_rows_smemx<4>(sp, pitch, g.klen, lane, s.vec(p) + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2]; y[3] = acc[3];
             } else if (g.nrows == 3) {
                 float acc[3];
-                dot_rows_smemx<3>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
+                dot_rows_smemx<3>(sp, pitch, g.klen, lane, s.vec(p) + g.kofs, acc);
                 y[0] = acc[0]; y[1] = acc[1]; y[2] = acc[2];
             } else {
                 float acc[1];
-                dot_rows_smemx<1>(sp, pitch, g.klen, lane, s.vec + g.kofs, acc);
+                dot_rows_smemx<1>(sp, pitch, g.klen, lane, s.vec(p) + g.kofs, acc);
                 y[0] = acc[0];
             }
             __syncwarp();
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 1);
             ring_release(p, s, wr, warp, lane);
             y[0] = warp_sum(y[0]);
             y[1] = warp_sum(y[1]);
@@ -1033,8 +1050,8 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             // L2 latency hides behind it.
             float res = 0.f;
             if (ep == EP_RESIDUAL && lane < g.nrows) res = ld_tw(out.res + g.row + lane).v;
-            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
             float y[MAX_RPC_SPLIT] = {0.f, 0.f, 0.f, 0.f};
             if (g.nrows == 2) {
@@ -1055,7 +1072,7 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
                 y[0] = acc[0];
             }
             __syncwarp();
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 1);
             ring_release(p, s, wr, warp, lane);   // the slot has been read for the last time
 #pragma unroll
             for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = warp_sum(y[rr]);
@@ -1078,8 +1095,8 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             }
         } else {
             // many short rows in one chunk (small hidden sizes): pair after pair, whole rows (npieces == 1)
-            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
             for (uint32_t rr = 0; rr < g.nrows; rr += 2) {
                 const bool two = rr + 1 < g.nrows;
@@ -1115,7 +1132,7 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const Smem& s, const
             __syncwarp();
             ring_release(p, s, wr, warp, lane);
         }
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
+        if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 3);
     }
     rc.advance(nch, p.nslots);
 }
@@ -1127,17 +1144,18 @@ __device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool 
 }
 
 // Waits (bounded) until `target` CTAs have signalled.  Replaces the grid-wide barrier of a kernel boundary.
-__device__ __forceinline__ void stage_wait(const Params& p, const Smem& s, const uint32_t* ctr, uint32_t target,
+template <class SM>
+__device__ __forceinline__ void stage_wait(const Params& p, const SM& s, const uint32_t* ctr, uint32_t target,
                                            uint32_t ctid) {
     if (ctid == 0) {
-        if (*s.abort_flag == 0 && ld_acquire(ctr) < target) {
+        if (*s.abort_flag() == 0 && ld_acquire(ctr) < target) {
             const uint64_t t0 = globaltimer_ns();
             uint32_t it = 0;
             while (ld_acquire(ctr) < target) {
                 if ((++it & 31u) == 0) {
-                    if (*s.abort_flag) break;
+                    if (*s.abort_flag()) break;
                     if (__ldcg(p.status) != 0) {
-                        *s.abort_flag = 1;
+                        *s.abort_flag() = 1;
                         break;
                     }
                     if (globaltimer_ns() - t0 > p.wait_ns) {
@@ -1220,8 +1238,8 @@ __device__ __forceinline__ void attn_batch(AttnAcc<G>& st, const float (&q)[G][8
 }
 
 // Ring chunks of the unit through the tensor-core loop; leaves this warp's partial result in comb[first].
-template <int HD, bool PACK>
-__device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, const AttnUnit& u, uint32_t cta,
+template <int HD, bool PACK, class SM>
+__device__ __forceinline__ void attn_chunks_tc(const Params& p, const SM& s, const AttnUnit& u, uint32_t cta,
                                                uint32_t warp, uint32_t lane, uint32_t first, const RingCursor& rc,
                                                WarpRing& wr, const float* q_s, float* comb,
                                                const uint8_t* stage_k, const uint8_t* stage_v) {
@@ -1252,17 +1270,17 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
     const uint32_t box_bytes = pb * 128u;
     for (uint32_t i = first; i < u.nring; i += p.nslots) {
         const uint32_t slot = warp * p.nsw + wr.cslot;
-        mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+        mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+        if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
         ring_advance_consume(p, wr);
-        const uint32_t kbase = smem_u32(s.ring) + slot * SLOT_BYTES;
+        const uint32_t kbase = smem_u32(s.ring()) + slot * SLOT_BYTES;
         const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
         for (uint32_t row0 = 0; row0 < pb; row0 += 16)
             if (row0 + 16 > w.lo && row0 < w.hi) attn_tc_tile<HD, PACK>(st, kbase, kbase + SLOT_BYTES / 2, box_bytes, row0, w.lo, w.hi, lane);
         __syncwarp();
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+        if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 1);
         ring_release(p, s, wr, warp, lane);
-        if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
+        if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 3);
     }
     if (u.has_new && first == 0)  // the position written by this step sits in row 0 of the staging tile
         attn_tc_tile<HD, PACK>(st, smem_u32(stage_k), smem_u32(stage_v), 128u, 0u, 0u, 1u, lane);
@@ -1299,7 +1317,8 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const Smem& s, c
 }
 
 // Two tagged words that may lie apart, polled until both carry `tag` (bounded).
-__device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const TW* a, const TW* b, uint32_t tag, float& va,
+template <class SM>
+__device__ __forceinline__ void poll_pair(const Params& p, const SM& s, const TW* a, const TW* b, uint32_t tag, float& va,
                                           float& vb) {
     PollGuard pg = {0ull, 0u, 200 + (int)(tag >> 4) * 1000};
     for (;;) {
@@ -1318,7 +1337,8 @@ __device__ __forceinline__ void poll_pair(const Params& p, const Smem& s, const 
 // (head, chunk) and the unit's slice of every chunk's partial output go to shared memory; the pairs become weights
 // w[h][c] = exp2(m_c - M_h) / L_h; thread j adds its output's nchunk terms in chunk order.  The orders of all sums
 // are fixed.
-__device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const StepCtx& cx, const AttnUnit& u, uint32_t layer,
+template <class SM>
+__device__ __noinline__ void attn_merge(const Params& p, const SM& s, const StepCtx& cx, const AttnUnit& u, uint32_t layer,
                                         uint32_t G, uint32_t ctid, float* comb) {
     const uint32_t hd = p.hd, b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
     const uint32_t unit0 = u.bg * p.cps;
@@ -1366,7 +1386,7 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const St
             if ((ml_pend || pend) && !poll_continue(p, s, pg)) break;
         }
     }
-    trace_stamp(p, blockIdx.x, layer, 5, ctid);
+    trace_stamp(p, s, blockIdx.x, layer, 5, ctid);
     consumer_bar();
     // one warp per head: maximum and normaliser by butterfly reductions (every lane ends with the same value)
     for (uint32_t h = ctid >> 5; h < G; h += NCW) {
@@ -1401,8 +1421,8 @@ __device__ __noinline__ void attn_merge(const Params& p, const Smem& s, const St
 // chunks, merges its warps and publishes the partial result; then every unit of the kv head merges its slice of
 // the outputs (attn_merge).  Scores use q pre-multiplied by log2(e)/sqrt(hd): the softmax runs in base 2.
 // GT > 0 selects the CUDA-core inner loop for GT query heads per KV head; GT == 0 the tensor-core loop.
-template <int GT>
-__device__ __noinline__ void attention_stage(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer, uint32_t cta,
+template <int GT, class SM>
+__device__ __noinline__ void attention_stage(const Params& p, const SM& s, const StepCtx& cx, uint32_t layer, uint32_t cta,
                                                  uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
     const AttnUnit u = attn_unit(p, cta, cx.pos);
     if (!u.active) return;
@@ -1411,7 +1431,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
     const uint32_t b = 0u, g = u.g, nchunk = u.nchunk;   // b: slot of the sequence in the scratch vectors
 
     // shared workspace inside the vector area
-    float* q_s = s.vec;                         // [G][hd]
+    float* q_s = s.vec(p);                         // [G][hd]
     float* new_k = q_s + G * hd;                // [hd]
     float* new_v = new_k + hd;                  // [hd]
     // Staging "tile" of the position written by this step: only row 0 of each 64-column box is ever valid, so the
@@ -1474,7 +1494,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
         }
     }
     consumer_bar();
-    trace_stamp(p, cta, layer, 14, ctid);
+    trace_stamp(p, s, cta, layer, 14, ctid);
 
     const uint32_t first = rc.first_chunk(warp, p.nslots);
     if constexpr (GT == 0) {
@@ -1512,12 +1532,12 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
         // (looped and per-layer launches then agree bit for bit).
         const uint32_t pb = attn_positions_per_chunk(p);
         for (uint32_t i = (warp < p.nslots ? first : u.nring); i < u.nring; i += p.nslots) {
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 1);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 1);
             const uint32_t slot = warp * p.nsw + wr.cslot;
-            mbar_wait(p, s, smem_u32(&s.full[slot]), wr.cphase);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 2);
+            mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
-            const uint8_t* kp = s.ring + (size_t)slot * SLOT_BYTES;
+            const uint8_t* kp = s.ring() + (size_t)slot * SLOT_BYTES;
             const uint8_t* vp = kp + SLOT_BYTES / 2;
             const uint32_t np = min(pb, u.cend - (u.c0 + i * pb));
             constexpr int U = (G_ <= 4) ? 4 : 2;
@@ -1536,7 +1556,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
             }
             __syncwarp();
             ring_release(p, s, wr, warp, lane);
-            if (lane == 0) chunk_stamp(p, cta, rc.n0 + i, 3);
+            if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 3);
         }
         if (u.has_new && first == 0) {
             // the position written by this step: its K/V come from shared memory (already rounded to bf16)
@@ -1587,13 +1607,13 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
             }
         }
     }
-    trace_stamp(p, cta, layer, 15, ctid);
+    trace_stamp(p, s, cta, layer, 15, ctid);
     consumer_bar();
 
     // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h);
     // then thread t owns (head, column) and adds the NCW weighted terms in warp order.
     const uint32_t unit = u.bg * p.cps + u.ch;
-    float* ftab = s.unit_part;   // [NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
+    float* ftab = s.unit_part();   // [NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
     if (ctid < NCW * G) {
         const uint32_t w = ctid / G, h = ctid % G;
         float Mh = -INFINITY;
@@ -1624,7 +1644,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
             }
         }
     }
-    trace_stamp(p, cta, layer, 3, ctid);
+    trace_stamp(p, s, cta, layer, 3, ctid);
     // every unit of the group merges its slice of the outputs
     if (nchunk > 1) attn_merge(p, s, cx, u, layer, G, ctid, comb);
 }
@@ -1633,12 +1653,13 @@ __device__ __noinline__ void attention_stage(const Params& p, const Smem& s, con
 // kernel reads that row from memory -- the unit that owns it works from the shared-memory copy -- so the store is
 // kept off the stage's critical path: it runs after the CTA has signalled, and before the shared-memory copy is
 // overwritten by the next stage's input vector.
-__device__ __forceinline__ void attention_flush_new_row(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer,
+template <class SM>
+__device__ __forceinline__ void attention_flush_new_row(const Params& p, const SM& s, const StepCtx& cx, uint32_t layer,
                                                         uint32_t cta, uint32_t ctid) {
     const AttnUnit u = attn_unit(p, cta, cx.pos);
     if (!u.active || !u.has_new) return;
     const uint32_t hd = p.hd;
-    const float* new_k = s.vec + p.G * hd;
+    const float* new_k = s.vec(p) + p.G * hd;
     const float* new_v = new_k + hd;
     const uint32_t per = hd / 8;
     if (ctid < 2 * per) {
@@ -1655,8 +1676,8 @@ __device__ __forceinline__ void attention_flush_new_row(const Params& p, const S
 }
 
 // Runs the attention stage and moves the ring cursor past the unit's chunks (also for CTAs without a unit).
-template <int GT>
-__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const Smem& s, const StepCtx& cx, uint32_t layer,
+template <int GT, class SM>
+__device__ __forceinline__ void attention_stage_and_advance(const Params& p, const SM& s, const StepCtx& cx, uint32_t layer,
                                                             uint32_t cta, uint32_t ctid, uint32_t warp, uint32_t lane,
                                                             RingCursor& rc, WarpRing& wr) {
     attention_stage<GT>(p, s, cx, layer, cta, ctid, warp, lane, rc, wr);
