@@ -246,13 +246,13 @@ __device__ __forceinline__ void bg_sum_partials(const BgPartials& q, uint32_t b,
     }
     for (uint32_t s = 0; s < n; ++s, src += stride) {
         if (N == 4) {
-            const float4 a = *reinterpret_cast<const float4*>(src);
+            const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
             v[0] += a.x; v[1] += a.y; v[2 % N] += a.z; v[3 % N] += a.w;
         } else if (N == 2) {
-            const float2 a = *reinterpret_cast<const float2*>(src);
+            const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
             v[0] += a.x; v[1 % N] += a.y;
         } else {
-            v[0] += *src;
+            v[0] += __ldcg(src);
         }
     }
 }
@@ -274,176 +274,238 @@ __device__ __forceinline__ bool bg_wait(uint32_t bar, uint32_t parity, int32_t* 
     return true;
 }
 
+// Shared memory of the projection pipeline: BG_STAGES tile pairs on 1024-byte boundaries (the swizzle pattern repeats
+// every 1024 bytes), then the barriers.
+struct BgSmem {
+    uint32_t tiles;        // shared-memory address of stage 0
+    uint64_t* full;        // [BG_STAGES] tile pair landed
+    uint64_t* empty;       // [BG_STAGES] MMAs that read the stage are done
+    uint64_t* acc_full;    // [2] accumulator buffer complete
+    uint64_t* acc_empty;   // [2] epilogue has read the buffer
+    uint32_t* tmem_base_s;
+    volatile int* abort_flag;
+};
+__device__ __forceinline__ BgSmem bg_carve(uint8_t* raw_ptr) {
+    BgSmem m;
+    const uint32_t raw = smem_u32(raw_ptr);
+    m.tiles = (raw + 1023u) & ~1023u;
+    uint8_t* misc = raw_ptr + (m.tiles - raw) + (size_t)BG_STAGES * BG_STAGE_BYTES;
+    m.full = reinterpret_cast<uint64_t*>(misc);
+    m.empty = m.full + BG_STAGES;
+    m.acc_full = m.empty + BG_STAGES;
+    m.acc_empty = m.acc_full + 2;
+    m.tmem_base_s = reinterpret_cast<uint32_t*>(m.acc_empty + 2);
+    m.abort_flag = reinterpret_cast<volatile int*>(m.tmem_base_s + 1);
+    return m;
+}
+__device__ __forceinline__ void bg_init_barriers(const BgSmem& m) {   // one thread
+    for (int i = 0; i < BG_STAGES; ++i) {
+        mbar_init(smem_u32(&m.full[i]), 1);
+        mbar_init(smem_u32(&m.empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+        mbar_init(smem_u32(&m.acc_full[i]), 1);
+        mbar_init(smem_u32(&m.acc_empty[i]), 4);   // one arrival per epilogue warp
+    }
+    *m.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Where each of the three roles stands in the pipeline.  One launch of kl_bgemm_kernel starts at zero; the looped
+// kernel carries the state from projection to projection (the ring and the two accumulator buffers never drain).
+struct BgPipe {
+    uint32_t stage, use;   // producer / MMA issuer: ring stage of the next tile pair and how often the ring has wrapped
+    uint32_t it;           // MMA issuer / epilogue: segments so far (accumulator buffer it & 1, its use it >> 1)
+};
+
+// Producer (one thread): TMA loads of the weight tile and the input tile of every (row tile, K block) of this CTA's
+// segments.  Weight tiles never wait for anything but a free stage (nothing writes weights); the input tiles of a
+// projection may only be requested once `ready()` has returned true -- the kernel or phase that writes the operand
+// has completed and its writes are visible.  Until then up to BG_STAGES weight tiles are requested ahead and their
+// input tiles follow afterwards.  Returns false when a wait gave up or `ready` refused (the step is a no-op).
+template <class Ready>
+__device__ __forceinline__ bool bg_produce(const BgemmParams& p, const CUtensorMap* map_w, const CUtensorMap* map_wl,
+                                           const CUtensorMap* map_x, const BgSmem& m, BgPipe& pipe, Ready&& ready) {
+    const uint64_t pol = l2_policy_evict_first();
+    // the input tiles are read again by every row tile: they should outlive the weights in L2
+    uint64_t polx;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(polx));
+    const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
+    uint32_t npend = 0;
+    uint32_t pend_stage[BG_STAGES], pend_col[BG_STAGES];
+    bool waited = false, ok = true;
+    auto flush = [&]() {   // the operand is there: request the input tiles of the stages that went ahead
+        if (!waited) {
+            ok = ready();
+            waited = true;
+        }
+        // (also when the step has turned out to be a no-op: the armed barriers have to complete)
+        for (uint32_t i = 0; i < npend; ++i)
+                tma_tensor_2d_g2s(m.tiles + pend_stage[i] * BG_STAGE_BYTES + BG_A_BYTES, map_x, (int32_t)pend_col[i], 0,
+                                  smem_u32(&m.full[pend_stage[i]]), polx);
+        npend = 0;
+    };
+    BgIter iter(p, ntiles);
+    BgSeg sg;
+    while (ok && !*m.abort_flag && iter.next(sg)) {
+        const uint32_t t = sg.t;
+        for (uint32_t kb = sg.kb0; kb < sg.kb1 && ok; ++kb) {
+            // a stage whose input tile is still pending can never come free: when every stage holds such a tile, the
+            // operand has to be waited for
+            if (!waited && npend == (uint32_t)BG_STAGES) flush();
+            if (!ok) break;
+            if (pipe.use > 0 && !bg_wait(smem_u32(&m.empty[pipe.stage]), (pipe.use - 1u) & 1u, p.status, p.wait_ns, m.abort_flag)) {
+                ok = false;
+                break;
+            }
+            const uint32_t bar = smem_u32(&m.full[pipe.stage]);
+            const uint32_t dst = m.tiles + pipe.stage * BG_STAGE_BYTES;
+            mbar_arrive_expect_tx(bar, (uint32_t)BG_STAGE_BYTES);
+            uint32_t xcol = kb * BG_TILE_K;
+            if (p.pieces == 0u) {
+                tma_tensor_3d_g2s(dst, map_w, (int32_t)xcol, (int32_t)(t * BG_TILE_M), (int32_t)p.layer, bar, pol);
+            } else {
+                // a block that reaches past the end of its piece gets zeros there from TMA, so whatever the input
+                // tile holds in those columns (the next piece's values) does not count
+                const uint32_t j = kb / p.kb_piece, cin = (kb - j * p.kb_piece) * BG_TILE_K, unit0 = t * BG_TILE_M / p.rpc;
+                xcol = j * p.kp + cin;
+                if (j + 1u < p.pieces)
+                    tma_tensor_5d_g2s(dst, map_w, (int32_t)cin, 0, (int32_t)j, (int32_t)unit0, (int32_t)p.layer, bar, pol);
+                else
+                    tma_tensor_4d_g2s(dst, map_wl, (int32_t)cin, 0, (int32_t)unit0, (int32_t)p.layer, bar, pol);
+            }
+            if (waited) {
+                tma_tensor_2d_g2s(dst + BG_A_BYTES, map_x, (int32_t)xcol, 0, bar, polx);
+            } else {
+                pend_stage[npend] = pipe.stage;
+                pend_col[npend] = xcol;
+                ++npend;
+            }
+            if (++pipe.stage == BG_STAGES) {
+                pipe.stage = 0;
+                ++pipe.use;
+            }
+        }
+    }
+    if (!waited || npend) flush();
+    return ok && !*m.abort_flag;
+}
+
+// After an abandoned run no copy may still be writing this CTA's shared memory when it exits: wait (bounded) for the
+// last copy armed on every stage.
+__device__ __forceinline__ void bg_drain(const BgSmem& m, const BgPipe& pipe, uint64_t wait_ns) {
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t sidx = 0; sidx < (uint32_t)BG_STAGES; ++sidx) {
+        const uint32_t cnt = pipe.use + (sidx < pipe.stage ? 1u : 0u);
+        if (cnt == 0) continue;
+        while (!mbar_try_wait(smem_u32(&m.full[sidx]), (cnt - 1u) & 1u))
+            if (globaltimer_ns() - t0 > wait_ns) break;
+    }
+}
+
+// MMA issuer (one thread of the warp that owns TMEM).
+__device__ __forceinline__ void bg_mma(const BgemmParams& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base) {
+    const uint32_t idesc = umma_idesc_bf16(BG_TILE_M, BG_TILE_N);
+    const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
+    BgIter iter(p, ntiles);
+    BgSeg sg;
+    for (; !*m.abort_flag && iter.next(sg); ++pipe.it) {
+        const uint32_t kb0 = sg.kb0, kb1 = sg.kb1;
+        const uint32_t buf = pipe.it & 1u, buse = pipe.it >> 1;
+        if (buse > 0 && !bg_wait(smem_u32(&m.acc_empty[buf]), (buse - 1u) & 1u, p.status, p.wait_ns, m.abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BG_TILE_N;
+        for (uint32_t kb = kb0; kb < kb1; ++kb) {
+            if (!bg_wait(smem_u32(&m.full[pipe.stage]), pipe.use & 1u, p.status, p.wait_ns, m.abort_flag)) break;
+            tc_fence_after();
+            const uint32_t a_addr = m.tiles + pipe.stage * BG_STAGE_BYTES;
+            const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + BG_A_BYTES);
+#pragma unroll
+            for (uint32_t k = 0; k < BG_TILE_K / 16; ++k)   // 16 bf16 = 32 bytes further along the swizzled row
+                umma_f16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb != kb0 || k != 0u) ? 1u : 0u);
+            umma_commit(smem_u32(&m.empty[pipe.stage]));   // the stage may be refilled when these MMAs are done
+            if (++pipe.stage == BG_STAGES) {
+                pipe.stage = 0;
+                ++pipe.use;
+            }
+        }
+        umma_commit(smem_u32(&m.acc_full[buf]));
+    }
+}
+
+// Epilogue warp (one of four): reads TMEM lanes 32 * quarter .. + 31 = rows of the tile, adds the hi and lo halves,
+// applies the RMSNorm factor and stores the partial tile.
+__device__ __forceinline__ void bg_epilogue(const BgemmParams& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base,
+                                            uint32_t quarter, uint32_t lane) {
+    float inv = 1.0f;   // lane b: the RMSNorm factor of sequence b
+    if (p.ssq != nullptr && lane < p.B) {
+        float ss = 0.f;
+        for (uint32_t c = 0; c < p.ssq_n; ++c) ss += __ldcg(p.ssq + lane * BV_MAX_CHUNKS + c);
+        inv = rsqrtf(ss / (float)p.K + p.eps);
+    }
+    const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
+    BgIter iter(p, ntiles);
+    BgSeg sg;
+    for (; iter.next(sg); ++pipe.it) {
+        const uint32_t t = sg.t;
+        const uint32_t buf = pipe.it & 1u, buse = pipe.it >> 1;
+        if (!bg_wait(smem_u32(&m.acc_full[buf]), buse & 1u, p.status, p.wait_ns, m.abort_flag)) break;
+        tc_fence_after();
+        uint32_t hi[32], lo[32];
+        const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BG_TILE_N;
+        tmem_ld32(taddr, hi);
+        tmem_ld32(taddr + 32u, lo);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&m.acc_empty[buf]));
+        const uint32_t row = t * BG_TILE_M + quarter * 32u + lane;
+        // tile schedule: [slot][b][R rows]; stream schedule: [slot][b][128 rows of the tile]
+        float* dst = p.stream ? p.out + (size_t)sg.slot * BG_MAX_BATCH * BG_TILE_M + quarter * 32u + lane
+                              : p.out + (size_t)sg.slot * BG_MAX_BATCH * p.R + row;
+        const size_t bstride = p.stream ? (size_t)BG_TILE_M : (size_t)p.R;
+#pragma unroll
+        for (uint32_t b = 0; b < 32; ++b) {
+            const float sc = __shfl_sync(0xffffffffu, inv, b);   // all lanes take part, also those past the last row
+            if (row < p.R && b < p.B) dst[(size_t)b * bstride] = (__uint_as_float(hi[b]) + __uint_as_float(lo[b])) * sc;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(BG_THREADS, 1) kl_bgemm_kernel(const __grid_constant__ BgemmParams p) {
     extern __shared__ uint8_t bg_smem_raw[];
-    // tiles on 1024-byte boundaries (the swizzle pattern repeats every 1024 bytes)
-    const uint32_t raw = smem_u32(bg_smem_raw);
-    const uint32_t tiles = (raw + 1023u) & ~1023u;
-    uint8_t* misc = bg_smem_raw + (tiles - raw) + (size_t)BG_STAGES * BG_STAGE_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(misc);            // [BG_STAGES] tile pair landed
-    uint64_t* empty = full + BG_STAGES;                             // [BG_STAGES] MMAs that read the stage are done
-    uint64_t* acc_full = empty + BG_STAGES;                         // [2] accumulator buffer complete
-    uint64_t* acc_empty = acc_full + 2;                             // [2] epilogue has read the buffer
-    uint32_t* tmem_base_s = reinterpret_cast<uint32_t*>(acc_empty + 2);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_s + 1);
-
+    const BgSmem m = bg_carve(bg_smem_raw);
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (tid == 0) {
-        for (int i = 0; i < BG_STAGES; ++i) {
-            mbar_init(smem_u32(&full[i]), 1);
-            mbar_init(smem_u32(&empty[i]), 1);
-        }
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(smem_u32(&acc_full[i]), 1);
-            mbar_init(smem_u32(&acc_empty[i]), 4);   // one arrival per epilogue warp
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
+    if (tid == 0) bg_init_barriers(m);
     if (warp == 1) {
-        tmem_alloc(smem_u32(tmem_base_s), BG_TMEM_COLS);
+        tmem_alloc(smem_u32(m.tmem_base_s), BG_TMEM_COLS);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_base_s;
+    const uint32_t tmem_base = *m.tmem_base_s;
 
-    const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
     griddep_launch();
     bool skip = false;
     if (!(warp == 0 && lane == 0)) {
         griddep_wait();
         skip = *p.status != 0;   // an earlier kernel of this step flagged an error: the step is a no-op
     }
-
+    BgPipe pipe = {0u, 0u, 0u};
     if (warp == 0 && lane == 0) {
-        // ---- producer: TMA loads of the weight tile and the input tile of every (row tile, K block) of this CTA's items.
-        // The weight tiles of the first ring round are requested before the predecessor kernel has finished (nothing
-        // writes weights); their input tiles follow once it has.
-        const uint64_t pol = l2_policy_evict_first();
-        // the input tiles are read again by every row tile: they should outlive the weights in L2
-        uint64_t polx;
-        asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(polx));
-        uint32_t stage = 0, use = 0, n = 0;
-        uint32_t xcols[BG_STAGES];
-        bool waited = false;
-        auto after_predecessor = [&]() {
+        // The weight tiles of the first ring round are requested before the predecessor kernel has finished; their
+        // input tiles follow once it has.
+        const bool ok = bg_produce(p, &p.map_w, &p.map_wl, &p.map_x, m, pipe, [&]() {
             griddep_wait();
-            waited = true;
-            skip = *p.status != 0;
-            for (uint32_t i = 0; i < n; ++i)   // n <= BG_STAGES: stage i holds iteration i
-                tma_tensor_2d_g2s(tiles + i * BG_STAGE_BYTES + BG_A_BYTES, &p.map_x, (int32_t)xcols[i], 0, smem_u32(&full[i]), polx);
-        };
-        BgIter iter(p, ntiles);
-        BgSeg sg;
-        while (!skip && !*abort_flag && iter.next(sg)) {
-            const uint32_t t = sg.t;
-            for (uint32_t kb = sg.kb0; kb < sg.kb1; ++kb, ++n) {
-                if (!waited && n == (uint32_t)BG_STAGES) after_predecessor();
-                if (skip) break;
-                if (use > 0 && !bg_wait(smem_u32(&empty[stage]), (use - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
-                const uint32_t bar = smem_u32(&full[stage]);
-                const uint32_t dst = tiles + stage * BG_STAGE_BYTES;
-                mbar_arrive_expect_tx(bar, (uint32_t)BG_STAGE_BYTES);
-                uint32_t xcol = kb * BG_TILE_K;
-                if (p.pieces == 0u) {
-                    tma_tensor_3d_g2s(dst, &p.map_w, (int32_t)xcol, (int32_t)(t * BG_TILE_M), (int32_t)p.layer, bar, pol);
-                } else {
-                    // a block that reaches past the end of its piece gets zeros there from TMA, so whatever the input
-                    // tile holds in those columns (the next piece's values) does not count
-                    const uint32_t j = kb / p.kb_piece, cin = (kb - j * p.kb_piece) * BG_TILE_K, unit0 = t * BG_TILE_M / p.rpc;
-                    xcol = j * p.kp + cin;
-                    if (j + 1u < p.pieces)
-                        tma_tensor_5d_g2s(dst, &p.map_w, (int32_t)cin, 0, (int32_t)j, (int32_t)unit0, (int32_t)p.layer, bar, pol);
-                    else
-                        tma_tensor_4d_g2s(dst, &p.map_wl, (int32_t)cin, 0, (int32_t)unit0, (int32_t)p.layer, bar, pol);
-                }
-                if (waited) tma_tensor_2d_g2s(dst + BG_A_BYTES, &p.map_x, (int32_t)xcol, 0, bar, polx);
-                else xcols[stage] = xcol;
-                if (++stage == BG_STAGES) {
-                    stage = 0;
-                    ++use;
-                }
-            }
-        }
-        if (!waited) after_predecessor();
-        if (skip || *abort_flag) {
-            // no copy may still be writing this CTA's shared memory when it exits: wait (bounded) for the last copy
-            // armed on every stage
-            const uint64_t t0 = globaltimer_ns();
-            for (uint32_t sidx = 0; sidx < (uint32_t)BG_STAGES; ++sidx) {
-                const uint32_t cnt = use + (sidx < stage ? 1u : 0u);
-                if (cnt == 0) continue;
-                while (!mbar_try_wait(smem_u32(&full[sidx]), (cnt - 1u) & 1u))
-                    if (globaltimer_ns() - t0 > p.wait_ns) break;
-            }
-        }
+            return *p.status == 0;
+        });
+        if (!ok) bg_drain(m, pipe, p.wait_ns);
     } else if (!skip && warp == 1 && lane == 0) {
-        // ---- MMA issuer
-        const uint32_t idesc = umma_idesc_bf16(BG_TILE_M, BG_TILE_N);
-        uint32_t stage = 0, use = 0, it = 0;
-        BgIter iter(p, ntiles);
-        BgSeg sg;
-        for (; !*abort_flag && iter.next(sg); ++it) {
-            const uint32_t kb0 = sg.kb0, kb1 = sg.kb1;
-            const uint32_t buf = it & 1u, buse = it >> 1;
-            if (buse > 0 && !bg_wait(smem_u32(&acc_empty[buf]), (buse - 1u) & 1u, p.status, p.wait_ns, abort_flag)) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + buf * BG_TILE_N;
-            for (uint32_t kb = kb0; kb < kb1; ++kb) {
-                if (!bg_wait(smem_u32(&full[stage]), use & 1u, p.status, p.wait_ns, abort_flag)) break;
-                tc_fence_after();
-                const uint32_t a_addr = tiles + stage * BG_STAGE_BYTES;
-                const uint64_t a_desc = umma_desc_sw128(a_addr), b_desc = umma_desc_sw128(a_addr + BG_A_BYTES);
-#pragma unroll
-                for (uint32_t k = 0; k < BG_TILE_K / 16; ++k)   // 16 bf16 = 32 bytes further along the swizzled row
-                    umma_f16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb != kb0 || k != 0u) ? 1u : 0u);
-                umma_commit(smem_u32(&empty[stage]));   // the stage may be refilled when these MMAs are done
-                if (++stage == BG_STAGES) {
-                    stage = 0;
-                    ++use;
-                }
-            }
-            umma_commit(smem_u32(&acc_full[buf]));
-        }
+        bg_mma(p, m, pipe, tmem_base);
     } else if (!skip && warp >= 2) {
-        // ---- epilogue: warp w reads TMEM lanes 32 * (w % 4) .. + 31 = rows of the tile
-        const uint32_t quarter = warp & 3u;
-        uint32_t it = 0;
-        float inv = 1.0f;   // lane b: the RMSNorm factor of sequence b
-        if (p.ssq != nullptr && lane < p.B) {
-            float ss = 0.f;
-            for (uint32_t c = 0; c < p.ssq_n; ++c) ss += p.ssq[lane * BV_MAX_CHUNKS + c];
-            inv = rsqrtf(ss / (float)p.K + p.eps);
-        }
-        BgIter iter(p, ntiles);
-        BgSeg sg;
-        for (; iter.next(sg); ++it) {
-            const uint32_t t = sg.t;
-            const uint32_t buf = it & 1u, buse = it >> 1;
-            if (!bg_wait(smem_u32(&acc_full[buf]), buse & 1u, p.status, p.wait_ns, abort_flag)) break;
-            tc_fence_after();
-            uint32_t hi[32], lo[32];
-            const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + buf * BG_TILE_N;
-            tmem_ld32(taddr, hi);
-            tmem_ld32(taddr + 32u, lo);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
-            const uint32_t row = t * BG_TILE_M + quarter * 32u + lane;
-            // tile schedule: [slot][b][R rows]; stream schedule: [slot][b][128 rows of the tile]
-            float* dst = p.stream ? p.out + (size_t)sg.slot * BG_MAX_BATCH * BG_TILE_M + quarter * 32u + lane
-                                  : p.out + (size_t)sg.slot * BG_MAX_BATCH * p.R + row;
-            const size_t bstride = p.stream ? (size_t)BG_TILE_M : (size_t)p.R;
-#pragma unroll
-            for (uint32_t b = 0; b < 32; ++b) {
-                const float sc = __shfl_sync(0xffffffffu, inv, b);   // all lanes take part, also those past the last row
-                if (row < p.R && b < p.B) dst[(size_t)b * bstride] = (__uint_as_float(hi[b]) + __uint_as_float(lo[b])) * sc;
-            }
-        }
+        bg_epilogue(p, m, pipe, tmem_base, warp & 3u, lane);
     }
     // ---- common exit: nobody may still be using TMEM when it is freed
     tc_fence_before();
@@ -466,19 +528,23 @@ __device__ __forceinline__ void put_operand2(__nv_bfloat16* xop, uint32_t K, uin
     *reinterpret_cast<uint32_t*>(xop + (size_t)(32 + b) * K + k) = lo;
 }
 
-// Vector work between two projections; grid (batch, ceil(K / BV_CHUNK)), 256 threads x 2 elements.
+// Barrier among the NT threads that work on one item together: the whole block of a vector kernel (barrier 0), or a
+// group of warps of the looped kernel (a named barrier of its own).
+template <int BAR, int NT>
+__device__ __forceinline__ void group_bar() {
+    asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
+// Vector work between two projections, one item = (sequence b, chunk c of BV_CHUNK elements), 256 threads x 2 elements.
 //   swiglu = 0:  v[k] = res[b][k] + sum_s part[s][b][k];  xout[b][k] = v[k];  operand = gain[k] * v[k] (the RMSNorm
 //                factor is applied behind the next contraction);  ssq[b][chunk] = sum of v[k]^2 over the chunk.
 //   swiglu = 1:  v[f] = silu(sum_s part[s][b][2f]) * (sum_s part[s][b][2f+1]);  operand = v.
 // The sums over the splits run in split order and the sum of squares in a fixed tree: reproducible.
-__global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part, const float* res, float* xout,
-                                                          const __nv_bfloat16* gain, int swiglu, uint32_t K, __nv_bfloat16* xop,
-                                                          float* ssq, const int32_t* status) {
-    const uint32_t b = blockIdx.x, c = blockIdx.y, tid = threadIdx.x;
-    __shared__ float red[8];
-    griddep_launch();
-    griddep_wait();
-    if (*status != 0) return;
+// red: 8 floats of shared memory owned by the group.
+template <int BAR>
+__device__ __forceinline__ void b_finish_item(const BgPartials& part, const float* res, float* xout, const __nv_bfloat16* gain,
+                                              int swiglu, uint32_t K, __nv_bfloat16* xop, float* ssq, uint32_t b, uint32_t c,
+                                              uint32_t tid, float* red) {
     const uint32_t k = c * BV_CHUNK + 2 * tid;
     float v0 = 0.f, v1 = 0.f;
     if (k < K) {   // K is even
@@ -489,7 +555,7 @@ __global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part,
             v1 = gu[2] / (1.0f + __expf(-gu[2])) * gu[3];
             put_operand2(xop, K, b, k, v0, v1);
         } else {
-            const float2 r = *reinterpret_cast<const float2*>(res + (size_t)b * K + k);
+            const float2 r = __ldcg(reinterpret_cast<const float2*>(res + (size_t)b * K + k));
             float a[2];
             if (part.part != nullptr) bg_sum_partials<2>(part, b, k, a);
             else a[0] = a[1] = 0.f;
@@ -505,7 +571,7 @@ __global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part,
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
     if ((tid & 31) == 0) red[tid >> 5] = ss;
-    __syncthreads();
+    group_bar<BAR, 256>();
     if (tid == 0) {
         float tot = 0.f;
 #pragma unroll
@@ -514,26 +580,43 @@ __global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part,
     }
 }
 
-// Token embedding of every sequence of the batch, the check of the whole batch, and the step's rotary table:
-// x[b] = E[token_b]; cs[b][i] = (cos, sin)(position_b * inv_freq[i]).  Grid (batch), 256 threads.
-__global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, const int32_t* positions, const __nv_bfloat16* embed,
-                                                         float* x, uint32_t H, uint32_t V, uint32_t max_ctx, const double* inv_freq,
-                                                         float* cs, uint32_t half, int32_t* status) {
-    const uint32_t b = blockIdx.x, tid = threadIdx.x;
+// grid (batch, ceil(K / BV_CHUNK)), 256 threads
+__global__ void __launch_bounds__(256) kl_b_finish_kernel(const BgPartials part, const float* res, float* xout,
+                                                          const __nv_bfloat16* gain, int swiglu, uint32_t K, __nv_bfloat16* xop,
+                                                          float* ssq, const int32_t* status) {
+    __shared__ float red[8];
     griddep_launch();
     griddep_wait();
+    if (*status != 0) return;
+    b_finish_item<0>(part, res, xout, gain, swiglu, K, xop, ssq, blockIdx.x, blockIdx.y, threadIdx.x, red);
+}
+
+// Token embedding of every sequence of the batch, the check of the whole batch, and the step's rotary table:
+// x[b] = E[token_b]; cs[b][i] = (cos, sin)(position_b * inv_freq[i]).  Grid (batch), 256 threads.
+template <int NT>
+__device__ __forceinline__ void b_embed_item(const int32_t* tokens, const int32_t* positions, const __nv_bfloat16* embed, float* x,
+                                             uint32_t H, uint32_t V, uint32_t max_ctx, const double* inv_freq, float* cs,
+                                             uint32_t half, int32_t* status, uint32_t b, uint32_t tid) {
     int32_t tok = tokens[b];
     const int32_t pos = positions[b];
     if (tid == 0 && (tok < 0 || tok >= (int32_t)V || pos < 0 || pos >= (int32_t)max_ctx)) atomicCAS(status, 0, ERR_OUT_OF_RANGE);
     if (tok < 0 || tok >= (int32_t)V) tok = 0;
-    for (uint32_t i = tid; i < half; i += blockDim.x) {
+    for (uint32_t i = tid; i < half; i += NT) {
         double sn, c;
         sincos((double)pos * inv_freq[i], &sn, &c);
         cs[(size_t)b * 2 * half + 2 * i] = (float)c;
         cs[(size_t)b * 2 * half + 2 * i + 1] = (float)sn;
     }
     const __nv_bfloat16* row = embed + (size_t)tok * H;
-    for (uint32_t i = tid; i < H; i += blockDim.x) x[(size_t)b * H + i] = __bfloat162float(row[i]);
+    for (uint32_t i = tid; i < H; i += NT) x[(size_t)b * H + i] = __bfloat162float(row[i]);
+}
+
+__global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, const int32_t* positions, const __nv_bfloat16* embed,
+                                                         float* x, uint32_t H, uint32_t V, uint32_t max_ctx, const double* inv_freq,
+                                                         float* cs, uint32_t half, int32_t* status) {
+    griddep_launch();
+    griddep_wait();
+    b_embed_item<256>(tokens, positions, embed, x, H, V, max_ctx, inv_freq, cs, half, status, blockIdx.x, threadIdx.x);
 }
 
 struct BAttnParams {
@@ -556,11 +639,7 @@ struct BAttnParams {
 // threads: sums the splits of the QKV projection, rotates a q head (and scales it by log2(e) / sqrt(hd) for the base-2
 // softmax) or a k head at the sequence's position, rounds k and v to bf16 and writes them into row `position` of the
 // sequence's cache slabs.  The attention kernel that follows reads that row from the cache like any other.
-__global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
-    const uint32_t b = blockIdx.x, head = blockIdx.y, tid = threadIdx.x;
-    griddep_launch();
-    griddep_wait();
-    if (*p.status != 0) return;
+__device__ __forceinline__ void b_rope_item(const BAttnParams& p, uint32_t b, uint32_t head, uint32_t tid) {   // 128 threads
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
     const float* cs = p.cs + (size_t)b * hd;
@@ -572,27 +651,34 @@ __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     const size_t slab = (size_t)p.max_ctx * hd;
     if (head < p.nq) {
         const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
-        for (uint32_t i = tid; i < half; i += blockDim.x) {
-            const float a = val(head * hd + i), bb = val(head * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+        for (uint32_t i = tid; i < half; i += 128u) {
+            const float a = val(head * hd + i), bb = val(head * hd + i + half), c = __ldcg(cs + 2 * i), sn = __ldcg(cs + 2 * i + 1);
             p.q[(size_t)b * p.QD + head * hd + i] = (a * c - bb * sn) * qscale;
             p.q[(size_t)b * p.QD + head * hd + i + half] = (bb * c + a * sn) * qscale;
         }
     } else if (head < p.nq + p.nkv) {
         const uint32_t g = head - p.nq;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 0) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        for (uint32_t i = tid; i < half; i += blockDim.x) {
-            const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
+        for (uint32_t i = tid; i < half; i += 128u) {
+            const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = __ldcg(cs + 2 * i), sn = __ldcg(cs + 2 * i + 1);
             row[i] = __float2bfloat16_rn(a * c - bb * sn);
             row[i + half] = __float2bfloat16_rn(bb * c + a * sn);
         }
     } else {
         const uint32_t g = head - p.nq - p.nkv;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 1) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        for (uint32_t d = tid; d < hd; d += blockDim.x) row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
+        for (uint32_t d = tid; d < hd; d += 128u) row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
     }
 }
 
-constexpr int BA_WARPS = 12;     // independent warps per CTA; one persistent CTA per SM
+__global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
+    griddep_launch();
+    griddep_wait();
+    if (*p.status != 0) return;
+    b_rope_item(p, blockIdx.x, blockIdx.y, threadIdx.x);
+}
+
+constexpr int BA_WARPS = 11;     // independent warps per CTA; one persistent CTA per SM (the looped kernel's twelfth warp streams weights)
 constexpr int BA_THREADS = BA_WARPS * 32;
 constexpr int BA_SLOTS = 2;      // ring slots per warp
 constexpr int BA_SLOT_BYTES = 8192;   // K rows | V rows of 16 (head size 128) or 32 (head size 64) cached positions
@@ -622,24 +708,14 @@ struct BaCursor {
 // sum) to slot (pair + warp) -- unique, because along the list either the pair or the warp advances from one segment
 // to the next.  kl_b_attn_merge_kernel combines the segments of every pair.  No warp waits for another one, every
 // warp streams the same number of bytes (+- one chunk), and a sequence's length only decides how many warps share it.
+// `warp` = index of the calling warp among the BA_WARPS workers of its CTA; `ring` = shared-memory address of its
+// BA_SLOTS slots (1024-byte aligned); `full` = its BA_SLOTS barriers (initialised by the caller); `uses` = chunks this
+// warp has taken through its slots so far (the barrier phases go on from there: 0 in a kernel of its own, carried
+// from layer to layer in the looped kernel).
 template <int HD, bool PACK>
-__device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* smem_raw) {
-    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+__device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint32_t warp, uint32_t lane, uint32_t ring, uint64_t* full,
+                                              volatile int* abort_flag, uint32_t& uses) {
     const uint32_t G = p.G;
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t ring = ((raw + 1023u) & ~1023u) + warp * BA_SLOTS * BA_SLOT_BYTES;   // this warp's slots
-    uint8_t* after = smem_raw + (((raw + 1023u) & ~1023u) - raw) + (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(after) + warp * BA_SLOTS;        // [BA_WARPS][BA_SLOTS]
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(after + BA_WARPS * BA_SLOTS * 8);
-
-    if (tid == 0) *abort_flag = 0;
-    if (lane == 0) {
-        for (int i = 0; i < BA_SLOTS; ++i) mbar_init(smem_u32(&full[i]), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-
     constexpr uint32_t pb = BA_SLOT_BYTES / (4u * HD);
     constexpr uint32_t box_bytes = pb * 128u;
     // lane b keeps the chunk count of sequence b; W = chunks of the whole step
@@ -677,6 +753,7 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
     };
     const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
     const uint64_t pol = l2_policy_evict_first();
+    const uint32_t use0 = uses;   // chunk k of the range is this warp's chunk number use0 + k - lo
     auto issue = [&](const BaCursor& x, uint32_t slot) {   // lane 0: the chunk under cursor x into this warp's slot
         const uint32_t n = (uint32_t)p.positions[x.b] + 1u;
         const AttnWindow w = attn_window(0u, n, pb, x.c);
@@ -695,7 +772,7 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
     BaCursor nxt = cur;   // cursor of the next chunk to request
     uint32_t issued = 0;
     for (; issued < (uint32_t)BA_SLOTS && lo + issued < hi; ++issued) {
-        if (lane == 0) issue(nxt, issued);
+        if (lane == 0) issue(nxt, (use0 + issued) % BA_SLOTS);
         advance(nxt);
     }
 
@@ -711,7 +788,7 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
                 const uint32_t k = kb * 16 + hf * 8 + 2 * t;
                 const uint32_t head = PACK ? (gq & 3u) : gq;   // PACK: column gq = hi (gq < 4) or lo half of head gq % 4
                 float2 xx = make_float2(0.f, 0.f);
-                if (head < G) xx = *reinterpret_cast<const float2*>(q + head * HD + k);
+                if (head < G) xx = __ldcg(reinterpret_cast<const float2*>(q + head * HD + k));   // written by the rotation step
                 const uint32_t qhi = pack_bf16(xx.x, xx.y);
                 const uint32_t qlo = pack_bf16(xx.x - bf_lo(qhi), xx.y - bf_hi(qhi));
                 st.qh[kb][hf] = (PACK && gq >= 4u) ? qlo : qhi;
@@ -755,7 +832,7 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
     begin_pair(cur);
     uint32_t k = lo;
     for (; k < hi; ++k) {
-        const uint32_t slot = (k - lo) % BA_SLOTS, phase = ((k - lo) / BA_SLOTS) & 1u;
+        const uint32_t slot = (use0 + k - lo) % BA_SLOTS, phase = ((use0 + k - lo) / BA_SLOTS) & 1u;
         if (!bg_wait(smem_u32(&full[slot]), phase, p.status, p.wait_ns, abort_flag)) break;
         const uint32_t kbase = ring + slot * BA_SLOT_BYTES;
         const AttnWindow w = attn_window(0u, (uint32_t)p.positions[cur.b] + 1u, pb, cur.c);
@@ -781,9 +858,22 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint8_t* sme
     // after a time-out copies may still be in flight: wait (bounded) for every chunk requested but not consumed
     if (k < hi && lane == 0) {
         const uint64_t t0 = globaltimer_ns();
-        for (uint32_t c = k - lo; c < issued; ++c)
+        for (uint32_t c = use0 + k - lo; c < use0 + issued; ++c)
             while (!mbar_try_wait(smem_u32(&full[c % BA_SLOTS]), (c / BA_SLOTS) & 1u))
                 if (globaltimer_ns() - t0 > p.wait_ns) break;
+    }
+    uses = use0 + issued;
+}
+
+// Picks the instantiation for the head size and the group size.
+__device__ __forceinline__ void b_attn_dispatch(const BAttnParams& p, uint32_t warp, uint32_t lane, uint32_t ring, uint64_t* full,
+                                                volatile int* abort_flag, uint32_t& uses) {
+    if (p.hd == 128) {
+        if (p.G <= 4) b_attn_stream<128, true>(p, warp, lane, ring, full, abort_flag, uses);
+        else b_attn_stream<128, false>(p, warp, lane, ring, full, abort_flag, uses);
+    } else {
+        if (p.G <= 4) b_attn_stream<64, true>(p, warp, lane, ring, full, abort_flag, uses);
+        else b_attn_stream<64, false>(p, warp, lane, ring, full, abort_flag, uses);
     }
 }
 
@@ -792,13 +882,21 @@ __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_c
     griddep_launch();
     griddep_wait();
     if (*p.status != 0) return;
-    if (p.hd == 128) {
-        if (p.G <= 4) b_attn_stream<128, true>(p, ba_smem_raw);
-        else b_attn_stream<128, false>(p, ba_smem_raw);
-    } else {
-        if (p.G <= 4) b_attn_stream<64, true>(p, ba_smem_raw);
-        else b_attn_stream<64, false>(p, ba_smem_raw);
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t raw = smem_u32(ba_smem_raw);
+    const uint32_t ring = ((raw + 1023u) & ~1023u) + warp * BA_SLOTS * BA_SLOT_BYTES;   // this warp's slots
+    uint8_t* after = ba_smem_raw + (((raw + 1023u) & ~1023u) - raw) + (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(after) + warp * BA_SLOTS;        // [BA_WARPS][BA_SLOTS]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(after + BA_WARPS * BA_SLOTS * 8);
+    if (tid == 0) *abort_flag = 0;
+    if (lane == 0) {
+        for (int i = 0; i < BA_SLOTS; ++i) mbar_init(smem_u32(&full[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    __syncthreads();
+    uint32_t uses = 0;
+    b_attn_dispatch(p, warp, lane, ring, full, abort_flag, uses);
 }
 
 // Combines the segments of every (sequence, kv head) pair and writes the attention output straight into the operand
@@ -808,15 +906,16 @@ __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_c
 // segments beyond BA_MERGE_SEGS in further rounds), then every thread adds up its two outputs over the segments --
 // independent loads, the additions in segment order.
 constexpr int BA_MERGE_SEGS = 64;
-__global__ void __launch_bounds__(64) kl_b_attn_merge_kernel(const BAttnParams p) {
-    const uint32_t hq = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+// Shared memory of one merge item (a group of hd / 2 <= 64 threads).
+struct BaMergeSmem {
+    uint32_t seg[2];
+    float wgt[BA_MERGE_SEGS];
+    float red[4];
+};
+// One item = (query head hq, sequence b), NT = hd / 2 threads (32 or 64), BAR = the group's barrier.
+template <int BAR, int NT>
+__device__ __forceinline__ void b_merge_item(const BAttnParams& p, uint32_t hq, uint32_t b, uint32_t tid, BaMergeSmem& sm) {
     const uint32_t G = p.G, hd = p.hd, g = hq / G, h = hq % G;
-    __shared__ uint32_t seg[2];
-    __shared__ float wgt[BA_MERGE_SEGS];
-    __shared__ float red[4];
-    griddep_launch();
-    griddep_wait();
-    if (*p.status != 0) return;
     if (tid < 32) {   // lane bb: chunks of sequence bb; W = all chunks, first = chunks before this pair
         const uint32_t pb = BA_SLOT_BYTES / (4u * hd);
         const uint32_t n = tid < p.B ? ba_chunks(p.positions[tid], pb) * p.nkv : 0u;
@@ -830,40 +929,50 @@ __global__ void __launch_bounds__(64) kl_b_attn_merge_kernel(const BAttnParams p
             const uint32_t nch = ba_chunks(p.positions[b], pb), NW = ba_workers(W, p.NW);
             first += g * nch;
             // the warp whose range holds chunk x: floor(((x + 1) * NW - 1) / W)  (every range holds at least one chunk)
-            seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
-            seg[1] = (uint32_t)((((uint64_t)first + nch) * NW - 1u) / W);
+            sm.seg[0] = (uint32_t)((((uint64_t)first + 1u) * NW - 1u) / W);
+            sm.seg[1] = (uint32_t)((((uint64_t)first + nch) * NW - 1u) / W);
         }
     }
-    __syncthreads();
-    const uint32_t w_first = seg[0], nseg = seg[1] - seg[0] + 1u;
+    group_bar<BAR, NT>();
+    const uint32_t w_first = sm.seg[0], nseg = sm.seg[1] - sm.seg[0] + 1u;
     const size_t pair = (size_t)b * p.nkv + g;
     const float* ml = p.part_ml + ((pair + w_first) * G + h) * 2;   // segment s: ml[s * G * 2], o[s * G * hd]
     const float* po = p.part_o + ((pair + w_first) * G + h) * hd;
     // running maximum over all segments
     float M = -INFINITY;
-    for (uint32_t s = tid; s < nseg; s += blockDim.x) M = fmaxf(M, ml[(size_t)s * G * 2]);
+    for (uint32_t s = tid; s < nseg; s += NT) M = fmaxf(M, __ldcg(ml + (size_t)s * G * 2));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-    if ((tid & 31) == 0) red[tid >> 5] = M;
-    __syncthreads();
-    M = fmaxf(red[0], blockDim.x > 32 ? red[1] : -INFINITY);
+    if ((tid & 31) == 0) sm.red[tid >> 5] = M;
+    group_bar<BAR, NT>();
+    M = fmaxf(sm.red[0], NT > 32 ? sm.red[1] : -INFINITY);
     float L = 0.f, A0 = 0.f, A1 = 0.f;
-    const uint32_t d = 2 * tid;   // hd is even; blockDim.x = hd / 2
+    const uint32_t d = 2 * tid;   // hd is even; NT = hd / 2
     for (uint32_t s0 = 0; s0 < nseg; s0 += BA_MERGE_SEGS) {
         const uint32_t ns = min((uint32_t)BA_MERGE_SEGS, nseg - s0);
-        __syncthreads();   // the previous round's weights have been used
-        for (uint32_t s = tid; s < ns; s += blockDim.x) wgt[s] = rescale(ml[(size_t)(s0 + s) * G * 2], M);
-        __syncthreads();
+        group_bar<BAR, NT>();   // the previous round's weights have been used
+        for (uint32_t s = tid; s < ns; s += NT) sm.wgt[s] = rescale(__ldcg(ml + (size_t)(s0 + s) * G * 2), M);
+        group_bar<BAR, NT>();
 #pragma unroll 4
         for (uint32_t s = 0; s < ns; ++s) {   // every thread also sums the segments' row sums itself, in segment order
-            const float c = wgt[s];
-            const float2 o = *reinterpret_cast<const float2*>(po + (size_t)(s0 + s) * G * hd + d);
-            L += __ldg(ml + (size_t)(s0 + s) * G * 2 + 1) * c;
+            const float c = sm.wgt[s];
+            const float2 o = __ldcg(reinterpret_cast<const float2*>(po + (size_t)(s0 + s) * G * hd + d));
+            L += __ldcg(ml + (size_t)(s0 + s) * G * 2 + 1) * c;
             A0 += o.x * c;
             A1 += o.y * c;
         }
     }
     if (d < hd) put_operand2(p.xop, p.QD, b, hq * hd + d, A0 / L, A1 / L);
+}
+
+// grid (query heads, batch), hd / 2 threads
+__global__ void __launch_bounds__(64) kl_b_attn_merge_kernel(const BAttnParams p) {
+    __shared__ BaMergeSmem sm;
+    griddep_launch();
+    griddep_wait();
+    if (*p.status != 0) return;
+    if (p.hd == 128) b_merge_item<0, 64>(p, blockIdx.x, blockIdx.y, threadIdx.x, sm);
+    else b_merge_item<0, 32>(p, blockIdx.x, blockIdx.y, threadIdx.x, sm);
 }
 
 }  // namespace kl
