@@ -11,6 +11,7 @@
 // streaming the next stage's (next layer's) chunks until the ring is full.
 #include "kl_device.cuh"
 #include "kl_batched.cuh"
+#include "kl_bloop.cuh"
 
 #include <math.h>
 #include <stdio.h>
@@ -515,6 +516,8 @@ struct kl_handle {
     float* hidden_all;     // [max_batch][H] hidden states of the sequences of the latest batched step
     // batched (tensor-core) path
     int bt_ok;             // 1: available for this shape
+    int bl_ok;             // 1: the looped kernel of the batched path can be resident (cooperative launch)
+    uint32_t* bbar;        // grid-barrier counters of the looped kernel: 16 per layer launch + 16
     int use_bt;            // 1 (default): batches take it; 0: sequence after sequence on the batch-1 kernels
     int use_pdl;           // 1 (default): the kernels of a batched step are launched with programmatic stream serialisation
     int use_stream;        // 1 (default): stream schedule for the projections of the layers; 0: (row tile, K split) items
@@ -575,7 +578,7 @@ struct Layout {
     size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
-    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, stplan, sbxop, sbssq, sbpart, sbq, sbao, sbaml, scratch_bytes;
+    size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, stplan, sbxop, sbssq, sbpart, sbq, sbao, sbaml, sbbar, scratch_bytes;
     uint32_t bsplit[5];
     uint32_t cps;
 };
@@ -683,6 +686,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
         const size_t aslots = B * d.n_kv_heads + (size_t)num_sms * BA_WARPS;   // attention partial results: pair + warp
         y.sbao = s;   s += on ? align_up(aslots * G * d.head_dim * 4) : 0;
         y.sbaml = s;  s += on ? align_up(aslots * G * 2 * 4) : 0;
+        y.sbbar = s;  s += on ? align_up(((size_t)d.n_layers + 1) * 16 * 4) : 0;
     }
     y.scratch_bytes = s;
     return y;
@@ -1038,6 +1042,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->bq = (float*)(sc + y.sbq);
     h->bao = (float*)(sc + y.sbao);
     h->baml = (float*)(sc + y.sbaml);
+    h->bbar = (uint32_t*)(sc + y.sbbar);
     for (int i = 0; i < 5; ++i) h->bsplit[i] = y.bsplit[i];
     h->use_bt = 1;
     h->use_stream = 1;
@@ -1050,6 +1055,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->bgraph_batch = 0;
     h->bgraph_launches = 0;
     h->bt_ok = 0;
+    h->bl_ok = 0;
     if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
         p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
         const uint32_t QR = p.QD + 2 * p.KVD;
@@ -1067,6 +1073,10 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
              cudaFuncSetAttribute(kl_b_attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ba_smem) == cudaSuccess;
         (void)cudaGetLastError();
         h->bt_ok = ok ? 1 : 0;
+        int bocc = 0;
+        h->bl_ok = ok && cudaFuncSetAttribute(kl_bloop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)BL_SMEM_BYTES) == cudaSuccess &&
+                   cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bocc, kl_bloop_kernel, BL_THREADS, BL_SMEM_BYTES) == cudaSuccess && bocc >= 1;
+        (void)cudaGetLastError();
     }
     h->argmax_idx = (uint32_t*)(h->argmax_val + (size_t)d.max_batch * ARGMAX_BLOCKS);
     h->argmax_tickets = h->argmax_idx + (size_t)d.max_batch * ARGMAX_BLOCKS;
@@ -1157,8 +1167,11 @@ size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch) {
     return (size_t)d.n_layers * 2 * batch * d.n_kv_heads * d.max_ctx * d.head_dim * 2;
 }
 
+static void drop_batched_graph(kl_handle* h);
+
 kl_status kl_set_mode(kl_handle* h, int mode) {
     if (!h || (mode != KL_MODE_LOOPED && mode != KL_MODE_PER_LAYER && mode != KL_MODE_PER_STAGE)) return KL_ERR_INVALID_ARG;
+    if (mode != h->mode) drop_batched_graph(h);   // a cached graph holds the launches of the old schedule
     h->mode = mode;
     return KL_OK;
 }
@@ -1295,6 +1308,87 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
     return KL_OK;
 }
 
+// Decode step of a batch as the looped kernel: one cooperative launch for the whole step (KL_MODE_LOOPED), or one
+// launch per layer from the same kernel (KL_MODE_PER_LAYER).
+static kl_status decode_step_batched_looped(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
+                                            float* logits_d, uint32_t batch, cudaStream_t st, bool per_layer) {
+    const Params& p = h->prm;
+    BLoopParams* b = new (std::nothrow) BLoopParams();   // 2.3 KB of kernel parameters (fourteen tensor maps)
+    if (!b) return KL_ERR_INVALID_ARG;
+    struct Free { BLoopParams* p; ~Free() { delete p; } } guard{b};
+    const kl_status trc = encode_kv_map(h, &b->kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
+    if (trc != KL_OK) return trc;
+    static const int plan_of[5] = {PL_QKV, PL_O, PL_GU, PL_D, PL_LM};
+    static const uint32_t xmap_of[5] = {0, 1, 0, 2, 0};
+    const uint32_t rows[5] = {p.QD + 2 * p.KVD, p.H, 2 * p.F, p.H, p.V};
+    for (int i = 0; i < 5; ++i) {
+        b->map_w[i] = h->bmap_w[i];
+        b->map_wl[i] = h->bmap_wl[i];
+        const GemvPlan& pl = p.plan[plan_of[i]];
+        BlGemm& g = b->g[i];
+        g.R = rows[i];
+        g.K = pl.K;
+        g.S = h->bsplit[i];
+        g.kp = pl.kp;
+        g.rpc = pl.rpc;
+        g.kb_piece = ceil_div(pl.kp, (uint32_t)BG_TILE_K);
+        if (pl.npieces == 1) {
+            g.pieces = 0;
+            g.nkb = ceil_div(pl.K, (uint32_t)BG_TILE_K);
+        } else {
+            g.pieces = pl.npieces;
+            g.nkb = (pl.npieces - 1) * g.kb_piece + ceil_div(pl.K - (pl.npieces - 1) * pl.kp, (uint32_t)BG_TILE_K);
+        }
+        const uint32_t T = ceil_div(g.R, (uint32_t)BG_TILE_M) * g.nkb;
+        g.stream = (i != 4 && h->use_stream && T >= (uint32_t)h->num_sms) ? 1u : 0u;
+        g.xmap = xmap_of[i];
+        g.normed = (i == 0 || i == 2 || i == 4) ? 1u : 0u;
+    }
+    for (int i = 0; i < 3; ++i) {
+        b->map_x[i] = h->bmap_x[i];
+        b->xop[i] = h->bxop[i];
+    }
+    b->tokens = tokens_d; b->positions = positions_d;
+    b->embed = p.embed; b->g1 = p.g1; b->g2 = p.g2; b->gf = p.gf; b->bqkv = p.bqkv;
+    b->layer_stride = p.layer_stride;
+    b->x = h->bx; b->ssq = h->bssq; b->part = h->bpart; b->q = h->bq; b->part_o = h->bao; b->part_ml = h->baml;
+    b->logits = logits_d; b->rope_cs = p.rope_cs; b->inv_freq = p.inv_freq;
+    b->kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
+    b->H = p.H; b->QD = p.QD; b->KVD = p.KVD; b->F = p.F; b->V = p.V; b->nq = p.nq; b->nkv = p.nkv; b->G = p.G; b->hd = p.hd;
+    b->B = batch; b->max_ctx = h->desc.max_ctx;
+    b->NW = (uint32_t)h->num_sms * BA_WARPS;
+    b->eps = p.eps;
+    b->status = p.status;
+    b->wait_ns = p.wait_ns;
+    if (cudaMemsetAsync(h->bbar, 0, ((size_t)p.L + 1) * 16 * 4, st) != cudaSuccess) return KL_ERR_CUDA;
+    cudaEvent_t* ev = h->prof_capacity ? h->prof_events + 3 * (h->prof_steps++ % h->prof_capacity) : nullptr;
+    if (ev && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
+    const uint32_t nlaunch = per_layer ? p.L : 1u;
+    for (uint32_t i = 0; i < nlaunch; ++i) {
+        b->l0 = per_layer ? i : 0u;
+        b->l1 = per_layer ? i + 1u : p.L;
+        b->first = i == 0 ? 1u : 0u;
+        b->last = i + 1u == nlaunch ? 1u : 0u;
+        b->bar = h->bbar + (size_t)i * 16;
+        void* args[] = {b};
+        if (cudaLaunchCooperativeKernel((const void*)kl_bloop_kernel, dim3(h->num_sms), dim3(BL_THREADS), args, BL_SMEM_BYTES, st) != cudaSuccess)
+            return KL_ERR_CUDA;
+        ++h->launches;
+    }
+    // the classifier is part of the (last) launch: both marks behind it
+    if (ev && (cudaEventRecord(ev[1], st) != cudaSuccess || cudaEventRecord(ev[2], st) != cudaSuccess)) return KL_ERR_CUDA;
+    return KL_OK;
+}
+
+// A batched step on the schedule kl_set_mode selected: the looped kernel (one launch), the same kernel launched per
+// layer, or one launch per operator group.
+static kl_status batched_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d, float* logits_d,
+                              uint32_t batch, cudaStream_t st) {
+    if (h->bl_ok && h->mode != KL_MODE_PER_STAGE)
+        return decode_step_batched_looped(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st, h->mode == KL_MODE_PER_LAYER);
+    return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
+}
+
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                          float* logits_d, uint32_t batch, void* stream) {
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
@@ -1304,7 +1398,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     h->chain_tok = nullptr;   // whatever kl_decode_greedy prepared for its next launch is overwritten by this step
     if (batch > 1 && h->bt_ok && h->use_bt) {
         h->last_batch = batch;
-        return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
+        return batched_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
     }
     Params p = h->prm;
     p.B = batch;
@@ -1389,7 +1483,7 @@ static bool replay_batched(kl_handle* h, const int32_t* tokens_d, const int32_t*
         if (!h->cap_stream && cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking) != cudaSuccess) h->cap_stream = nullptr;
         if (h->cap_stream && cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
             const uint64_t l0 = h->launches;
-            const kl_status crc = decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, h->cap_stream);
+            const kl_status crc = batched_step(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, h->cap_stream);
             cudaGraph_t graph = nullptr;
             const cudaError_t e = cudaStreamEndCapture(h->cap_stream, &graph);
             h->bgraph_launches = h->launches - l0;

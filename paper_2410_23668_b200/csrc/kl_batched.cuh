@@ -51,10 +51,8 @@ constexpr int BG_TMEM_COLS = 128;   // two accumulator buffers of 64 fp32 column
 constexpr size_t BG_SMEM_BYTES = (size_t)BG_STAGES * BG_STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 constexpr int BG_MAX_BATCH = 32;
 
-struct BgemmParams {
-    CUtensorMap map_w;     // weights: rank 3 (column, row, layer) or, for chunk-ordered matrices, rank 5
-    CUtensorMap map_wl;    // chunk-ordered matrices: the last (shorter) column piece, rank 4 (column, row in unit, unit, layer)
-    CUtensorMap map_x;     // inputs [64 rows, K] bf16: rows 0..31 hi halves, 32..63 lo halves
+// One projection as the three roles see it (everything but the tensor maps).
+struct BgView {
     float* out;            // tile schedule: [S][32][R] partial sums (S = 1: the result itself);
                            // stream schedule: [row tiles + CTAs][32][128] partial tiles, slot = tile + CTA
     uint32_t R, K, B, S, layer;
@@ -71,6 +69,11 @@ struct BgemmParams {
     float eps;
     int32_t* status;
     uint64_t wait_ns;
+};
+struct BgemmParams : BgView {
+    CUtensorMap map_w;     // weights: rank 3 (column, row, layer) or, for chunk-ordered matrices, rank 5
+    CUtensorMap map_wl;    // chunk-ordered matrices: the last (shorter) column piece, rank 4 (column, row in unit, unit, layer)
+    CUtensorMap map_x;     // inputs [64 rows, K] bf16: rows 0..31 hi halves, 32..63 lo halves
 };
 
 constexpr int BV_CHUNK = 512;        // elements per block of the vector kernels (256 threads x 2)
@@ -181,7 +184,7 @@ struct BgSeg {
 struct BgIter {
     uint32_t stream, nkb, S, nitems, item;   // tile schedule
     uint32_t g0, g1;                         // stream schedule: blocks of the list still to do
-    __device__ __forceinline__ BgIter(const BgemmParams& p, uint32_t ntiles)
+    __device__ __forceinline__ BgIter(const BgView& p, uint32_t ntiles)
         : stream(p.stream), nkb(p.nkb), S(p.S), nitems(ntiles * p.S), item(blockIdx.x) {
         const uint32_t T = ntiles * p.nkb;
         g0 = (uint32_t)(((uint64_t)blockIdx.x * T) / gridDim.x);
@@ -325,7 +328,7 @@ struct BgPipe {
 // has completed and its writes are visible.  Until then up to BG_STAGES weight tiles are requested ahead and their
 // input tiles follow afterwards.  Returns false when a wait gave up or `ready` refused (the step is a no-op).
 template <class Ready>
-__device__ __forceinline__ bool bg_produce(const BgemmParams& p, const CUtensorMap* map_w, const CUtensorMap* map_wl,
+__device__ __forceinline__ bool bg_produce(const BgView& p, const CUtensorMap* map_w, const CUtensorMap* map_wl,
                                            const CUtensorMap* map_x, const BgSmem& m, BgPipe& pipe, Ready&& ready) {
     const uint64_t pol = l2_policy_evict_first();
     // the input tiles are read again by every row tile: they should outlive the weights in L2
@@ -405,7 +408,7 @@ __device__ __forceinline__ void bg_drain(const BgSmem& m, const BgPipe& pipe, ui
 }
 
 // MMA issuer (one thread of the warp that owns TMEM).
-__device__ __forceinline__ void bg_mma(const BgemmParams& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base) {
+__device__ __forceinline__ void bg_mma(const BgView& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base) {
     const uint32_t idesc = umma_idesc_bf16(BG_TILE_M, BG_TILE_N);
     const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
     BgIter iter(p, ntiles);
@@ -436,7 +439,7 @@ __device__ __forceinline__ void bg_mma(const BgemmParams& p, const BgSmem& m, Bg
 
 // Epilogue warp (one of four): reads TMEM lanes 32 * quarter .. + 31 = rows of the tile, adds the hi and lo halves,
 // applies the RMSNorm factor and stores the partial tile.
-__device__ __forceinline__ void bg_epilogue(const BgemmParams& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base,
+__device__ __forceinline__ void bg_epilogue(const BgView& p, const BgSmem& m, BgPipe& pipe, uint32_t tmem_base,
                                             uint32_t quarter, uint32_t lane) {
     float inv = 1.0f;   // lane b: the RMSNorm factor of sequence b
     if (p.ssq != nullptr && lane < p.B) {
@@ -619,8 +622,7 @@ __global__ void __launch_bounds__(256) kl_b_embed_kernel(const int32_t* tokens, 
     b_embed_item<256>(tokens, positions, embed, x, H, V, max_ctx, inv_freq, cs, half, status, blockIdx.x, threadIdx.x);
 }
 
-struct BAttnParams {
-    CUtensorMap kv_map;       // the whole KV cache as [rows, head_dim] (same map as the batch-1 kernel)
+struct BAttnView {
     __nv_bfloat16* kv;
     const int32_t* positions;
     const float* cs;          // [32][hd / 2][2] (cos, sin) of the step's positions
@@ -634,12 +636,15 @@ struct BAttnParams {
     int32_t* status;
     uint64_t wait_ns;
 };
+struct BAttnParams : BAttnView {
+    CUtensorMap kv_map;       // the whole KV cache as [rows, head_dim] (same map as the batch-1 kernel)
+};
 
 // RoPE and cache append; grid (batch, n_q_heads + 2 * n_kv_heads), one head of one sequence per block of 128
 // threads: sums the splits of the QKV projection, rotates a q head (and scales it by log2(e) / sqrt(hd) for the base-2
 // softmax) or a k head at the sequence's position, rounds k and v to bf16 and writes them into row `position` of the
 // sequence's cache slabs.  The attention kernel that follows reads that row from the cache like any other.
-__device__ __forceinline__ void b_rope_item(const BAttnParams& p, uint32_t b, uint32_t head, uint32_t tid) {   // 128 threads
+__device__ __forceinline__ void b_rope_item(const BAttnView& p, uint32_t b, uint32_t head, uint32_t tid) {   // 128 threads
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
     const float* cs = p.cs + (size_t)b * hd;
@@ -713,8 +718,8 @@ struct BaCursor {
 // warp has taken through its slots so far (the barrier phases go on from there: 0 in a kernel of its own, carried
 // from layer to layer in the looped kernel).
 template <int HD, bool PACK>
-__device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint32_t warp, uint32_t lane, uint32_t ring, uint64_t* full,
-                                              volatile int* abort_flag, uint32_t& uses) {
+__device__ __forceinline__ void b_attn_stream(const BAttnView& p, const CUtensorMap* kv_map, uint32_t warp, uint32_t lane, uint32_t ring,
+                                              uint64_t* full, volatile int* abort_flag, uint32_t& uses) {
     const uint32_t G = p.G;
     constexpr uint32_t pb = BA_SLOT_BYTES / (4u * HD);
     constexpr uint32_t box_bytes = pb * 128u;
@@ -763,8 +768,8 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint32_t war
         mbar_arrive_expect_tx(bar, (uint32_t)BA_SLOT_BYTES);
 #pragma unroll
         for (uint32_t bx = 0; bx < HD / 64u; ++bx) {
-            tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)row0, bar, pol);
-            tma_tensor_2d_g2s(dst + BA_SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + vdelta), bar, pol);
+            tma_tensor_2d_g2s(dst + bx * box_bytes, kv_map, (int32_t)(bx * 64u), (int32_t)row0, bar, pol);
+            tma_tensor_2d_g2s(dst + BA_SLOT_BYTES / 2 + bx * box_bytes, kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + vdelta), bar, pol);
         }
     };
 
@@ -866,14 +871,15 @@ __device__ __forceinline__ void b_attn_stream(const BAttnParams& p, uint32_t war
 }
 
 // Picks the instantiation for the head size and the group size.
-__device__ __forceinline__ void b_attn_dispatch(const BAttnParams& p, uint32_t warp, uint32_t lane, uint32_t ring, uint64_t* full,
-                                                volatile int* abort_flag, uint32_t& uses) {
+// kv_map: the cache's tensor map, in the kernel's parameter space.
+__device__ __forceinline__ void b_attn_dispatch(const BAttnView& p, const CUtensorMap* kv_map, uint32_t warp, uint32_t lane,
+                                                uint32_t ring, uint64_t* full, volatile int* abort_flag, uint32_t& uses) {
     if (p.hd == 128) {
-        if (p.G <= 4) b_attn_stream<128, true>(p, warp, lane, ring, full, abort_flag, uses);
-        else b_attn_stream<128, false>(p, warp, lane, ring, full, abort_flag, uses);
+        if (p.G <= 4) b_attn_stream<128, true>(p, kv_map, warp, lane, ring, full, abort_flag, uses);
+        else b_attn_stream<128, false>(p, kv_map, warp, lane, ring, full, abort_flag, uses);
     } else {
-        if (p.G <= 4) b_attn_stream<64, true>(p, warp, lane, ring, full, abort_flag, uses);
-        else b_attn_stream<64, false>(p, warp, lane, ring, full, abort_flag, uses);
+        if (p.G <= 4) b_attn_stream<64, true>(p, kv_map, warp, lane, ring, full, abort_flag, uses);
+        else b_attn_stream<64, false>(p, kv_map, warp, lane, ring, full, abort_flag, uses);
     }
 }
 
@@ -896,7 +902,7 @@ __global__ void __launch_bounds__(BA_THREADS, 1) kl_b_attn_kernel(const __grid_c
     }
     __syncthreads();
     uint32_t uses = 0;
-    b_attn_dispatch(p, warp, lane, ring, full, abort_flag, uses);
+    b_attn_dispatch(p, &p.kv_map, warp, lane, ring, full, abort_flag, uses);
 }
 
 // Combines the segments of every (sequence, kv head) pair and writes the attention output straight into the operand
@@ -914,7 +920,7 @@ struct BaMergeSmem {
 };
 // One item = (query head hq, sequence b), NT = hd / 2 threads (32 or 64), BAR = the group's barrier.
 template <int BAR, int NT>
-__device__ __forceinline__ void b_merge_item(const BAttnParams& p, uint32_t hq, uint32_t b, uint32_t tid, BaMergeSmem& sm) {
+__device__ __forceinline__ void b_merge_item(const BAttnView& p, uint32_t hq, uint32_t b, uint32_t tid, BaMergeSmem& sm) {
     const uint32_t G = p.G, hd = p.hd, g = hq / G, h = hq % G;
     if (tid < 32) {   // lane bb: chunks of sequence bb; W = all chunks, first = chunks before this pair
         const uint32_t pb = BA_SLOT_BYTES / (4u * hd);
