@@ -648,13 +648,24 @@ def run_ours_batched(args, shape, batch, context):
         _DIST["on"] = True
     K, W = args.steps, max(args.warmup, 3)
     Ks = max(1, min(K, 4))   # the sequential schedule takes batch times longer per step: fewer steps
-    dec, cache, max_ctx = build_model(shape, batch, context, 7 * (K + W) + Ks + 3, seed=rank)
+    dec, cache, max_ctx = build_model(shape, batch, context, 9 * (K + W) + Ks + 3, seed=rank)
     tok0 = gen.make_tokens(shape, batch, rank, device="cuda")
     stream = torch.cuda.current_stream()
     sampler = ClockSampler(local)
     sampler.start()
     # the cache is not restored between the passes: the rows the passes append lie beyond the positions they read
     dec.kl_set_batched_path(True)
+    # the three call schedules of the batched step, from the same phase code (Section 2 of the paper, schedules
+    # (iii), (ii), (i)): one cooperative launch per step, that kernel launched per layer, one launch per operator group
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    l0 = dec.kl_launch_count()
+    ms_looped = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
+    looped_launches = (dec.kl_launch_count() - l0) // (K + W)
+    dec.kl_set_mode(binding.KL_MODE_PER_LAYER)
+    l0 = dec.kl_launch_count()
+    ms_layer = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
+    layer_launches = (dec.kl_launch_count() - l0) // (K + W)
+    dec.kl_set_mode(binding.KL_MODE_PER_STAGE)   # the fastest of the three on this GPU, and the default for batches
     l0 = dec.kl_launch_count()
     ms_batched = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
     launches = (dec.kl_launch_count() - l0) * K // (K + W)
@@ -675,7 +686,7 @@ def run_ours_batched(args, shape, batch, context):
     ms_plain = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, W, K, stream))
     dec.kl_set_dependent_launch(True)
     dec.kl_set_batched_path(False)
-    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)   # the batch-1 looped kernel, sequence after sequence
     ms_seq = max_over_ranks(run_device_loop(dec, cache, tok0, context, batch, 3, Ks, stream))
 
     tokens = K * batch * world
@@ -718,6 +729,12 @@ def run_ours_batched(args, shape, batch, context):
                        else {"value": None, "why": graph_err}),
         "launch_by_launch": {"value": tokens / (ms_batched * 1e-3), "ms_per_step": ms_batched / K,
                              "call": "kl_decode_step + kl_argmax_advance, every kernel launched from the host (dependent launch on)"},
+        "looped": {"value": tokens / (ms_looped * 1e-3), "ms_per_step": ms_looped / K, "launches_per_step": looped_launches,
+                   "what": "KL_MODE_LOOPED: one persistent kernel per step (grid barriers between the phases, weight stream running ahead)"},
+        "per_layer": {"value": tokens / (ms_layer * 1e-3), "ms_per_step": ms_layer / K, "launches_per_step": layer_launches,
+                      "looped_speedup": ms_layer / ms_looped},
+        "per_stage": {"value": tokens / (ms_batched * 1e-3), "ms_per_step": ms_batched / K, "launches_per_step": int(launches) // K,
+                      "looped_speedup": ms_batched / ms_looped},
         "plain_stream_order": {"value": tokens / (ms_plain * 1e-3), "ms_per_step": ms_plain / K,
                                "launches_per_step": int(launches) // K},
         "sequential_looped": {"value": Ks * batch * world / (ms_seq * 1e-3), "ms_per_step": ms_seq / Ks, "steps": Ks,

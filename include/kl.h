@@ -110,7 +110,13 @@ size_t kl_kv_cache_bytes(const kl_handle* h, uint32_t batch);
 /* KL_MODE_LOOPED (default): one persistent kernel runs all layers (4 launches per token with embedding, classifier
  * and sampling).  KL_MODE_PER_LAYER: one launch per layer (L + 3).  KL_MODE_PER_STAGE: one launch per operator group
  * of every layer -- QKV, attention, O, gate/up, down (5 L + 3): the three call schedules of Section 2, from the
- * same stage code. */
+ * same stage code.
+ * Batches on the tensor-core path (kl_set_batched_path) have the same three schedules from one set of phase functions,
+ * with identical results: KL_MODE_LOOPED = ONE cooperative launch per step (embedding, all layers, classifier; grid
+ * barriers between the phases, the projections' weight stream running ahead of them), KL_MODE_PER_LAYER = that kernel
+ * launched once per layer, KL_MODE_PER_STAGE = ten launches per layer joined by programmatic dependent launch
+ * (kl_set_dependent_launch).  A handle on which kl_set_mode has never been called decodes batches on the per-operator
+ * schedule, the fastest of the three on this GPU; after a call batches follow the mode like single sequences. */
 kl_status kl_set_mode(kl_handle* h, int mode);
 
 /* One decode step for `batch` sequences, asynchronous on `stream`.
@@ -273,9 +279,8 @@ kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
  * of the step (QKV, O, gate/up, down, classifier) is one dense contraction for the whole batch on the tcgen05 tensor
  * cores (M = 128 weight rows x N = 64 = 32 sequences x (hi, lo bf16 halves of the fp32 input), fp32 accumulators in
  * TMEM), so the weights are streamed once per step instead of once per sequence -- at batch 32 the projections are
- * dense contractions (Table 1 of the paper); attention runs as split-K units over (sequence, kv head, split).  The
- * step is a sequence of launches, one per operator group (Section 2's per-operator calls); kl_set_mode does not
- * apply to it.  on = 0: the batch-1 kernels in the mode of kl_set_mode, sequence after sequence.  Available when
+ * dense contractions (Table 1 of the paper); attention runs as one balanced stream of K|V chunks over all (sequence,
+ * kv head) pairs.  kl_set_mode selects the call schedule of the step (see there).  on = 0: the batch-1 kernels in the mode of kl_set_mode, sequence after sequence.  Available when
  * max_batch is 2..32, head_dim is 64 or 128, hidden / q width / ffn are multiples of 8, every projection has at
  * least 128 rows and the driver exports cuTensorMapEncodeTiled; otherwise KL_ERR_UNSUPPORTED_SHAPE for on = 1. */
 kl_status kl_set_batched_path(kl_handle* h, int on);

@@ -502,6 +502,7 @@ struct kl_handle {
     kl_model_desc desc;
     Params prm;
     int mode;
+    int mode_explicit;     // kl_set_mode has been called: batches follow `mode` too (until then they take the per-operator schedule)
     int device;
     int num_sms;
     size_t smem_bytes;
@@ -1171,8 +1172,9 @@ static void drop_batched_graph(kl_handle* h);
 
 kl_status kl_set_mode(kl_handle* h, int mode) {
     if (!h || (mode != KL_MODE_LOOPED && mode != KL_MODE_PER_LAYER && mode != KL_MODE_PER_STAGE)) return KL_ERR_INVALID_ARG;
-    if (mode != h->mode) drop_batched_graph(h);   // a cached graph holds the launches of the old schedule
+    if (mode != h->mode || !h->mode_explicit) drop_batched_graph(h);   // a cached graph holds the launches of the old schedule
     h->mode = mode;
+    h->mode_explicit = 1;
     return KL_OK;
 }
 
@@ -1384,8 +1386,11 @@ static kl_status decode_step_batched_looped(kl_handle* h, const int32_t* tokens_
 // layer, or one launch per operator group.
 static kl_status batched_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d, float* logits_d,
                               uint32_t batch, cudaStream_t st) {
-    if (h->bl_ok && h->mode != KL_MODE_PER_STAGE)
-        return decode_step_batched_looped(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st, h->mode == KL_MODE_PER_LAYER);
+    // Until kl_set_mode says otherwise a batch takes the per-operator schedule: with programmatic dependent launch its
+    // kernel boundaries cost less on this GPU than the grid barriers that replace them in the looped kernel (measured).
+    const int mode = h->mode_explicit ? h->mode : KL_MODE_PER_STAGE;
+    if (h->bl_ok && mode != KL_MODE_PER_STAGE)
+        return decode_step_batched_looped(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st, mode == KL_MODE_PER_LAYER);
     return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
 }
 

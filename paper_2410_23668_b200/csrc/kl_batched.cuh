@@ -247,16 +247,31 @@ __device__ __forceinline__ void bg_sum_partials(const BgPartials& q, uint32_t b,
         stride = (size_t)BG_MAX_BATCH * q.R;
         n = q.S;
     }
-    for (uint32_t s = 0; s < n; ++s, src += stride) {
-        if (N == 4) {
-            const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
-            v[0] += a.x; v[1] += a.y; v[2 % N] += a.z; v[3 % N] += a.w;
-        } else if (N == 2) {
-            const float2 a = __ldcg(reinterpret_cast<const float2*>(src));
-            v[0] += a.x; v[1 % N] += a.y;
-        } else {
-            v[0] += __ldcg(src);
+    // the loads of up to four partial results are issued together (one L2 round trip, not one per addend); the
+    // additions keep their order
+    for (uint32_t s0 = 0; s0 < n; s0 += 4, src += 4 * stride) {
+        float a[4][N];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (s0 + j < n) {
+                const float* sp = src + (size_t)j * stride;
+                if (N == 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(sp);
+                    a[j][0] = t.x; a[j][1] = t.y; a[j][2 % N] = t.z; a[j][3 % N] = t.w;
+                } else if (N == 2) {
+                    const float2 t = *reinterpret_cast<const float2*>(sp);
+                    a[j][0] = t.x; a[j][1 % N] = t.y;
+                } else {
+                    a[j][0] = *sp;
+                }
+            }
         }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (s0 + j < n) {
+#pragma unroll
+                for (int i = 0; i < N; ++i) v[i] += a[j][i];
+            }
     }
 }
 
@@ -444,7 +459,7 @@ __device__ __forceinline__ void bg_epilogue(const BgView& p, const BgSmem& m, Bg
     float inv = 1.0f;   // lane b: the RMSNorm factor of sequence b
     if (p.ssq != nullptr && lane < p.B) {
         float ss = 0.f;
-        for (uint32_t c = 0; c < p.ssq_n; ++c) ss += __ldcg(p.ssq + lane * BV_MAX_CHUNKS + c);
+        for (uint32_t c = 0; c < p.ssq_n; ++c) ss += p.ssq[lane * BV_MAX_CHUNKS + c];
         inv = rsqrtf(ss / (float)p.K + p.eps);
     }
     const uint32_t ntiles = (p.R + BG_TILE_M - 1) / BG_TILE_M;
@@ -531,6 +546,13 @@ __device__ __forceinline__ void put_operand2(__nv_bfloat16* xop, uint32_t K, uin
     *reinterpret_cast<uint32_t*>(xop + (size_t)(32 + b) * K + k) = lo;
 }
 
+// SwiGLU of two neighbouring features from their (gate, up) sums, written as the next projection's operand.
+__device__ __forceinline__ void b_swiglu_store(const float (&gu)[4], __nv_bfloat16* xop, uint32_t K, uint32_t b, uint32_t k) {
+    const float v0 = gu[0] / (1.0f + __expf(-gu[0])) * gu[1];
+    const float v1 = gu[2] / (1.0f + __expf(-gu[2])) * gu[3];
+    put_operand2(xop, K, b, k, v0, v1);
+}
+
 // Barrier among the NT threads that work on one item together: the whole block of a vector kernel (barrier 0), or a
 // group of warps of the looped kernel (a named barrier of its own).
 template <int BAR, int NT>
@@ -554,11 +576,9 @@ __device__ __forceinline__ void b_finish_item(const BgPartials& part, const floa
         if (swiglu) {
             float gu[4];   // gate f, up f, gate f + 1, up f + 1
             bg_sum_partials<4>(part, b, 2 * k, gu);
-            v0 = gu[0] / (1.0f + __expf(-gu[0])) * gu[1];
-            v1 = gu[2] / (1.0f + __expf(-gu[2])) * gu[3];
-            put_operand2(xop, K, b, k, v0, v1);
+            b_swiglu_store(gu, xop, K, b, k);
         } else {
-            const float2 r = __ldcg(reinterpret_cast<const float2*>(res + (size_t)b * K + k));
+            const float2 r = *reinterpret_cast<const float2*>(res + (size_t)b * K + k);
             float a[2];
             if (part.part != nullptr) bg_sum_partials<2>(part, b, k, a);
             else a[0] = a[1] = 0.f;
@@ -644,7 +664,8 @@ struct BAttnParams : BAttnView {
 // threads: sums the splits of the QKV projection, rotates a q head (and scales it by log2(e) / sqrt(hd) for the base-2
 // softmax) or a k head at the sequence's position, rounds k and v to bf16 and writes them into row `position` of the
 // sequence's cache slabs.  The attention kernel that follows reads that row from the cache like any other.
-__device__ __forceinline__ void b_rope_item(const BAttnView& p, uint32_t b, uint32_t head, uint32_t tid) {   // 128 threads
+template <int NT>   // threads that share the item
+__device__ __forceinline__ void b_rope_item(const BAttnView& p, uint32_t b, uint32_t head, uint32_t tid) {
     const uint32_t hd = p.hd, half = hd >> 1;
     const int32_t pos = p.positions[b];
     const float* cs = p.cs + (size_t)b * hd;
@@ -656,23 +677,23 @@ __device__ __forceinline__ void b_rope_item(const BAttnView& p, uint32_t b, uint
     const size_t slab = (size_t)p.max_ctx * hd;
     if (head < p.nq) {
         const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
-        for (uint32_t i = tid; i < half; i += 128u) {
-            const float a = val(head * hd + i), bb = val(head * hd + i + half), c = __ldcg(cs + 2 * i), sn = __ldcg(cs + 2 * i + 1);
+        for (uint32_t i = tid; i < half; i += NT) {
+            const float a = val(head * hd + i), bb = val(head * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
             p.q[(size_t)b * p.QD + head * hd + i] = (a * c - bb * sn) * qscale;
             p.q[(size_t)b * p.QD + head * hd + i + half] = (bb * c + a * sn) * qscale;
         }
     } else if (head < p.nq + p.nkv) {
         const uint32_t g = head - p.nq;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 0) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        for (uint32_t i = tid; i < half; i += 128u) {
-            const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = __ldcg(cs + 2 * i), sn = __ldcg(cs + 2 * i + 1);
+        for (uint32_t i = tid; i < half; i += NT) {
+            const float a = val(p.QD + g * hd + i), bb = val(p.QD + g * hd + i + half), c = cs[2 * i], sn = cs[2 * i + 1];
             row[i] = __float2bfloat16_rn(a * c - bb * sn);
             row[i + half] = __float2bfloat16_rn(bb * c + a * sn);
         }
     } else {
         const uint32_t g = head - p.nq - p.nkv;
         __nv_bfloat16* row = p.kv + ((((size_t)p.layer * 2 + 1) * p.B + b) * p.nkv + g) * slab + (size_t)pos * hd;
-        for (uint32_t d = tid; d < hd; d += 128u) row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
+        for (uint32_t d = tid; d < hd; d += NT) row[d] = __float2bfloat16_rn(val(p.QD + p.KVD + g * hd + d));
     }
 }
 
@@ -680,7 +701,7 @@ __global__ void __launch_bounds__(128) kl_b_rope_kernel(const BAttnParams p) {
     griddep_launch();
     griddep_wait();
     if (*p.status != 0) return;
-    b_rope_item(p, blockIdx.x, blockIdx.y, threadIdx.x);
+    b_rope_item<128>(p, blockIdx.x, blockIdx.y, threadIdx.x);
 }
 
 constexpr int BA_WARPS = 11;     // independent warps per CTA; one persistent CTA per SM (the looped kernel's twelfth warp streams weights)
@@ -793,7 +814,7 @@ __device__ __forceinline__ void b_attn_stream(const BAttnView& p, const CUtensor
                 const uint32_t k = kb * 16 + hf * 8 + 2 * t;
                 const uint32_t head = PACK ? (gq & 3u) : gq;   // PACK: column gq = hi (gq < 4) or lo half of head gq % 4
                 float2 xx = make_float2(0.f, 0.f);
-                if (head < G) xx = __ldcg(reinterpret_cast<const float2*>(q + head * HD + k));   // written by the rotation step
+                if (head < G) xx = *reinterpret_cast<const float2*>(q + head * HD + k);
                 const uint32_t qhi = pack_bf16(xx.x, xx.y);
                 const uint32_t qlo = pack_bf16(xx.x - bf_lo(qhi), xx.y - bf_hi(qhi));
                 st.qh[kb][hf] = (PACK && gq >= 4u) ? qlo : qhi;
@@ -946,7 +967,7 @@ __device__ __forceinline__ void b_merge_item(const BAttnView& p, uint32_t hq, ui
     const float* po = p.part_o + ((pair + w_first) * G + h) * hd;
     // running maximum over all segments
     float M = -INFINITY;
-    for (uint32_t s = tid; s < nseg; s += NT) M = fmaxf(M, __ldcg(ml + (size_t)s * G * 2));
+    for (uint32_t s = tid; s < nseg; s += NT) M = fmaxf(M, ml[(size_t)s * G * 2]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
     if ((tid & 31) == 0) sm.red[tid >> 5] = M;
@@ -957,13 +978,13 @@ __device__ __forceinline__ void b_merge_item(const BAttnView& p, uint32_t hq, ui
     for (uint32_t s0 = 0; s0 < nseg; s0 += BA_MERGE_SEGS) {
         const uint32_t ns = min((uint32_t)BA_MERGE_SEGS, nseg - s0);
         group_bar<BAR, NT>();   // the previous round's weights have been used
-        for (uint32_t s = tid; s < ns; s += NT) sm.wgt[s] = rescale(__ldcg(ml + (size_t)(s0 + s) * G * 2), M);
+        for (uint32_t s = tid; s < ns; s += NT) sm.wgt[s] = rescale(ml[(size_t)(s0 + s) * G * 2], M);
         group_bar<BAR, NT>();
 #pragma unroll 4
         for (uint32_t s = 0; s < ns; ++s) {   // every thread also sums the segments' row sums itself, in segment order
             const float c = sm.wgt[s];
-            const float2 o = __ldcg(reinterpret_cast<const float2*>(po + (size_t)(s0 + s) * G * hd + d));
-            L += __ldcg(ml + (size_t)(s0 + s) * G * 2 + 1) * c;
+            const float2 o = *reinterpret_cast<const float2*>(po + (size_t)(s0 + s) * G * hd + d);
+            L += ml[(size_t)(s0 + s) * G * 2 + 1] * c;
             A0 += o.x * c;
             A1 += o.y * c;
         }

@@ -27,7 +27,8 @@
 namespace kl {
 
 constexpr int BL_THREADS = 384;
-constexpr int BL_PHASE_THREADS = 352;   // warps 1..11
+constexpr int BL_PHASE_WARPS = 11;      // warps 1..11
+constexpr int BL_PHASE_THREADS = BL_PHASE_WARPS * 32;
 constexpr int BL_WORK_THREADS = 256;    // warps 4..11
 constexpr size_t BL_REGION_BYTES = (size_t)BG_STAGES * BG_STAGE_BYTES > (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES
                                        ? (size_t)BG_STAGES * BG_STAGE_BYTES : (size_t)BA_WARPS * BA_SLOTS * BA_SLOT_BYTES;
@@ -99,15 +100,20 @@ __device__ __forceinline__ BlSmem bl_carve(uint8_t* raw_ptr) {
 }
 
 // ---- grid barrier.  Counter `idx` counts the CTAs whose phase warps have finished the phase in front of it.
+__device__ __forceinline__ uint32_t bl_ld_relaxed(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Polls with relaxed loads; the caller's fence behind a successful wait is the acquire.
 __device__ __forceinline__ bool bl_counter_wait(const BLoopParams& p, uint32_t idx, volatile int* abort_flag) {
     const uint32_t* ctr = p.bar + idx;
-    if (ld_acquire(ctr) >= gridDim.x) return true;
+    if (bl_ld_relaxed(ctr) >= gridDim.x) return true;
     if (*abort_flag) return false;
     const uint64_t t0 = globaltimer_ns();
     uint32_t it = 0;
-    while (ld_acquire(ctr) < gridDim.x) {
-        __nanosleep(32);
-        if ((++it & 15u) == 0) {
+    while (bl_ld_relaxed(ctr) < gridDim.x) {
+        if ((++it & 31u) == 0) {
             if (*abort_flag) return false;
             if (__ldcg(p.status) != 0) {   // another CTA gave up: so does this one
                 *abort_flag = 1;
@@ -174,6 +180,21 @@ __device__ __forceinline__ void bl_finish_phase(const BLoopParams& p, const BgPa
         if (!swiglu) group_bar<2, BL_WORK_THREADS>();   // the next item of this CTA reuses `red`
     }
 }
+// SwiGLU between the gate/up and the down projection: no reduction, so the feature pairs of all sequences form one flat
+// list over the phase threads of the grid; every thread takes two pairs at a time and issues the loads of both before
+// it computes (the partial sums sit in L2: one round trip per two pairs).
+__device__ __forceinline__ void bl_swiglu_phase(const BLoopParams& p, const BgPartials& parts, uint32_t ptid) {
+    const uint32_t half = p.F / 2u, n = p.B * half, nthreads = gridDim.x * (uint32_t)BL_PHASE_THREADS;
+    for (uint32_t e = blockIdx.x * (uint32_t)BL_PHASE_THREADS + ptid; e < n; e += 2u * nthreads) {
+        const uint32_t e1 = e + nthreads;
+        float g0[4], g1[4] = {0.f, 0.f, 0.f, 0.f};
+        bg_sum_partials<4>(parts, e / half, 4u * (e % half), g0);
+        if (e1 < n) bg_sum_partials<4>(parts, e1 / half, 4u * (e1 % half), g1);
+        b_swiglu_store(g0, p.xop[2], p.F, e / half, 2u * (e % half));
+        if (e1 < n) b_swiglu_store(g1, p.xop[2], p.F, e1 / half, 2u * (e1 % half));
+    }
+}
+
 __device__ __forceinline__ BAttnView bl_attn_params(const BLoopParams& p, uint32_t layer) {
     BAttnView a;
     a.kv = p.kv;
@@ -316,9 +337,10 @@ __global__ void __launch_bounds__(BL_THREADS, 1) kl_bloop_kernel(const __grid_co
             if (!bl_gsync(p, bi++, ptid, abort_flag, m.step_ok)) { live = false; break; }
             // V2: rotation, cache append
             const BAttnView a = bl_attn_params(p, l);
-            if (worker) {
-                const uint32_t sub = wtid >> 7, t = wtid & 127u, n = p.B * (p.nq + 2u * p.nkv);
-                for (uint32_t i = blockIdx.x * 2u + sub; i < n; i += gridDim.x * 2u) b_rope_item(a, i / (p.nq + 2u * p.nkv), i % (p.nq + 2u * p.nkv), t);
+            {   // one (sequence, head) per warp, all eleven phase warps
+                const uint32_t nh = p.nq + 2u * p.nkv, n = p.B * nh;
+                for (uint32_t i = blockIdx.x * (uint32_t)BL_PHASE_WARPS + (warp - 1u); i < n; i += gridDim.x * (uint32_t)BL_PHASE_WARPS)
+                    b_rope_item<32>(a, i / nh, i % nh, lane);
             }
             if (!bl_gsync(p, bi++, ptid, abort_flag, m.step_ok)) { live = false; break; }
             // A: the attention stream (the rows appended above are read by bulk copies)
@@ -343,7 +365,7 @@ __global__ void __launch_bounds__(BL_THREADS, 1) kl_bloop_kernel(const __grid_co
             gemm_phase(2, l);
             if (!bl_gsync(p, bi++, ptid, abort_flag, m.step_ok)) { live = false; break; }
             // V5: operand = silu(gate) * up
-            if (worker) bl_finish_phase(p, bl_partials(p, 2), nullptr, 1, p.F, p.xop[2], wtid, m.red);
+            bl_swiglu_phase(p, bl_partials(p, 2), ptid);
             if (!bl_gsync(p, bi++, ptid, abort_flag, m.step_ok)) { live = false; break; }
             gemm_phase(3, l);
             if (!bl_gsync(p, bi++, ptid, abort_flag, m.step_ok)) live = false;
