@@ -301,6 +301,14 @@ kl_status kl_set_wait_limit_ns(kl_handle* h, uint64_t ns);
  * or endless loop is involved. */
 kl_status kl_debug_skip_signal_once(kl_handle* h, int stage);
 
+/* Test hook for the synchronisation protocol of the batch-1 persistent kernels (the tagged words and the counter that
+ * replace kernel boundaries, Section 3.2): with seed != 0 and max_ns > 0 every CTA sleeps a pseudo-random time below
+ * max_ns (at most 1 ms) whenever it enters a stage, a different one per (CTA, step, layer, stage), so that the CTAs
+ * meet every exchange in a different order from step to step; the kernels then run in their instantiation with the
+ * debug hooks compiled in.  Results must not change by a bit.  max_ns = 0 switches the hook off.  No counterpart in
+ * the paper. */
+kl_status kl_debug_set_jitter(kl_handle* h, uint32_t seed, uint32_t max_ns);
+
 /* Test hook for the step numbers behind the tags.  Every decoded token takes one step number; the tags hold 28 bits of
  * (step x n_layers + layer), so after *wrap_at steps (about 2^28 / n_layers: 8.4 million tokens at 32 layers) the
  * library clears its tagged scratch areas at the next launch boundary and starts numbering again at 1 -- a tagged word

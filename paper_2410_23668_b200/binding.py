@@ -34,7 +34,7 @@ EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_by
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
            "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
            "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy", "kl_decode_greedy_tokens",
-           "kl_decode_greedy_tokens_host", "kl_debug_set_step")
+           "kl_decode_greedy_tokens_host", "kl_debug_set_step", "kl_debug_set_jitter")
 
 
 class ModelDesc(C.Structure):
@@ -93,6 +93,8 @@ def lib():
     l.kl_set_wait_limit_ns.restype = i32
     l.kl_debug_skip_signal_once.argtypes = [vp, C.c_int]
     l.kl_debug_skip_signal_once.restype = i32
+    l.kl_debug_set_jitter.argtypes = [vp, u32, u32]
+    l.kl_debug_set_jitter.restype = i32
     l.kl_debug_set_step.argtypes = [vp, u32, C.POINTER(u32)]
     l.kl_debug_set_step.restype = i32
     l.kl_profile_enable.argtypes = [vp, u32]
@@ -266,6 +268,9 @@ class Decoder:
 
     def kl_debug_skip_signal_once(self, stage: int) -> None:
         _check(lib().kl_debug_skip_signal_once(self.handle, stage), "kl_debug_skip_signal_once")
+
+    def kl_debug_set_jitter(self, seed: int, max_ns: int) -> None:
+        _check(lib().kl_debug_set_jitter(self.handle, seed, max_ns), "kl_debug_set_jitter")
 
     def kl_debug_set_step(self, step: int | None = None) -> int:
         """Sets the step counter behind the tags (None: only queries); returns the step number at which it wraps."""

@@ -136,6 +136,7 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
                                           uint32_t xa_slot, uint32_t ctr_target, uint32_t cta, uint32_t ctid, uint32_t warp,
                                           uint32_t lane, RingCursor& rc, WarpRing& wr) {
     const StepCtx& cx = *s.ctx();
+    stage_jitter(p, s, cta, cx.step, l, st);
     const size_t lo = (size_t)l * p.layer_stride;
     const bool cls = l == p.L;
     // test hook: the results of one stage of layer 0 get a tag nobody waits for
@@ -466,8 +467,9 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
 // K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
+template <bool TR>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
-    const SmemT<false> s;
+    const SmemT<TR> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, t.rope)) return;
     if (warp == NCW) {
@@ -991,8 +993,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     {
         int tocc = 0;
-        h->token_ok = cudaFuncSetAttribute(kl_token_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+        h->token_ok = cudaFuncSetAttribute(kl_token_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
+                      cudaFuncSetAttribute(kl_token_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
+                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
@@ -1435,7 +1438,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
         uint32_t sbeg = 0, send = 5;
         // the instantiation with the trace stamps compiled in only while a trace buffer is set
-        const void* decoder_fn = p.trace != nullptr ? (const void*)kl_decoder_kernel<true> : (const void*)kl_decoder_kernel<false>;
+        const void* decoder_fn = (p.trace != nullptr || p.jitter_seed != 0u) ? (const void*)kl_decoder_kernel<true> : (const void*)kl_decoder_kernel<false>;
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1, &sbeg, &send};
@@ -1565,7 +1568,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     if (prc != KL_OK) return prc;
     TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, nullptr, 1u, p.rope_cs};
     void* args[] = {&p, &t};
-    const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
+    const kl_status rc = launch_persistent(h, p.jitter_seed ? (const void*)kl_token_kernel<true> : (const void*)kl_token_kernel<false>, args, st);
     if (rc != KL_OK) return rc;
     h->last_batch = 1;
     h->hidden_is_copy = 1;
@@ -1599,7 +1602,7 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
         ++h->launches;
         TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, out_tokens_d + done, K, h->plan_rope};
         void* args[] = {&p, &t};
-        const kl_status rc = launch_persistent(h, (const void*)kl_token_kernel, args, st);
+        const kl_status rc = launch_persistent(h, p.jitter_seed ? (const void*)kl_token_kernel<true> : (const void*)kl_token_kernel<false>, args, st);
         if (rc != KL_OK) return rc;
         h->last_batch = 1;
         h->hidden_is_copy = 1;
@@ -1833,6 +1836,13 @@ kl_status kl_set_dependent_launch(kl_handle* h, int on) {
 kl_status kl_debug_skip_signal_once(kl_handle* h, int stage) {
     if (!h || stage < -1 || stage > 4) return KL_ERR_INVALID_ARG;
     h->pending_skip_stage = stage;
+    return KL_OK;
+}
+
+kl_status kl_debug_set_jitter(kl_handle* h, uint32_t seed, uint32_t max_ns) {
+    if (!h || max_ns > 1000000u) return KL_ERR_INVALID_ARG;
+    h->prm.jitter_seed = max_ns ? seed : 0u;
+    h->prm.jitter_ns = max_ns;
     return KL_OK;
 }
 

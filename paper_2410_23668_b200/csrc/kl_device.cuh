@@ -74,6 +74,8 @@ struct Params {
     uint32_t cps;          // attention: CTA slots per (sequence, kv head)
     float eps;
     int32_t skip_stage;    // test hook: stage of layer 0 whose end is not signalled (-1 = none)
+    uint32_t jitter_seed;  // test hook: != 0 makes every CTA sleep a pseudo-random time (below jitter_ns) when it enters a stage
+    uint32_t jitter_ns;
     uint64_t wait_ns;
     uint64_t layer_stride; // elements between consecutive layers of any per-layer tensor
     const __nv_bfloat16* bqkv;   // biases of the q, k, v projections [L][QD + 2 KVD] (layer_stride apart), or null
@@ -122,6 +124,24 @@ template <class SM>
 __device__ __forceinline__ void chunk_stamp(const Params& p, const SM&, uint32_t cta, uint64_t n, int k) {
     if constexpr (SM::kTrace)
         if (p.chunk_trace != nullptr && cta == 0 && n < CHUNK_TRACE_ROWS) p.chunk_trace[n * 4 + k] = globaltimer_ns();
+}
+// Test hook of the synchronisation protocol (instantiations with the debug hooks only): every consumer thread of the
+// CTA sleeps the same pseudo-random time, a function of (seed, CTA, step, layer, stage), before it enters a stage, so
+// that the CTAs reach every exchange in a different order on every step.  Bounded: at most jitter_ns, in naps.
+template <class SM>
+__device__ __forceinline__ void stage_jitter(const Params& p, const SM&, uint32_t cta, uint32_t step, uint32_t layer, uint32_t st) {
+    if constexpr (SM::kTrace) {
+        if (p.jitter_seed != 0u) {
+            uint32_t h = p.jitter_seed ^ (cta * 0x9E3779B1u) ^ (step * 0x85EBCA77u) ^ ((layer * 8u + st) * 0xC2B2AE3Du);
+            h ^= h >> 15; h *= 0x2C1B3C6Du; h ^= h >> 12; h *= 0x297A2D39u; h ^= h >> 15;
+            uint32_t ns = (uint32_t)(((uint64_t)h * p.jitter_ns) >> 32);
+            while (ns > 0u) {
+                const uint32_t nap = ns < 1000u ? ns : 1000u;
+                __nanosleep(nap);
+                ns -= nap;
+            }
+        }
+    }
 }
 template <class SM>
 __device__ __forceinline__ void trace_stamp(const Params& p, const SM&, uint32_t cta, uint32_t layer, int k, uint32_t ctid) {

@@ -918,3 +918,48 @@ def test_step_numbers_wrap_without_a_stale_tag():
             got = chain(kind)
             assert all(torch.equal(g, w) for g, w in zip(got, want)), (kind, start)
     dec.close()
+
+
+@pytest.mark.parametrize("name,steps", [("tiny", 1500), ("llama31_8b_4layers", 150)])
+def test_sync_protocol_under_seeded_jitter(name, steps):
+    """Stress of the exchanges that replace kernel boundaries (tagged words, the gate/up counter, the token boundary
+    inside a launch): with kl_debug_set_jitter every CTA sleeps a seeded pseudo-random time of up to 20 us whenever it
+    enters a stage, so the CTAs reach every exchange in a different order on every step.  A long greedy run on the
+    looped kernel, on the one-launch-per-token chain and as multi-token launches must pick, token for token, what the
+    undisturbed per-layer schedule picks, and leave the same cache; no bounded wait may run out."""
+    import dataclasses
+    shape, ctx = {"tiny": (gen.TINY, 40), "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 512)}[name]
+    dec = helpers.make_decoder(shape, 1, ctx + steps + 8, 0)
+    cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + steps + 8, 0, "cuda")
+    tok0 = gen.make_tokens(shape, 1, 0).cuda()
+
+    def run(kind):
+        cache, tok = cache0.clone(), tok0.clone()
+        pos = torch.tensor([ctx], dtype=torch.int32, device="cuda")
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        out = torch.empty(steps, dtype=torch.int32, device="cuda")
+        if kind == "tokens":
+            dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, steps, 1, True)
+        else:
+            for i in range(steps):
+                if kind == "greedy":
+                    dec.kl_decode_greedy(tok, pos, cache, logits, 1, i == 0)
+                else:
+                    dec.kl_decode_step(tok, pos, cache, logits, 1)
+                    dec.kl_argmax_advance(logits, tok, pos, 1)
+                out[i] = tok[0]
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK, kind
+        return out.cpu(), logits.cpu(), cache.cpu().view(torch.uint16)
+
+    dec.kl_set_mode(binding.KL_MODE_PER_LAYER)
+    want = run("steps")
+    dec.kl_set_mode(binding.KL_MODE_LOOPED)
+    for seed, kind in ((1, "steps"), (2, "greedy"), (3, "tokens"), (4, "tokens")):
+        dec.kl_debug_set_jitter(seed, 20_000)
+        got = run(kind)
+        first_diff = int((got[0] != want[0]).nonzero()[0]) if not torch.equal(got[0], want[0]) else -1
+        assert first_diff < 0, (kind, seed, first_diff)
+        assert torch.equal(got[1], want[1]) and torch.equal(got[2], want[2]), (kind, seed)
+    dec.kl_debug_set_jitter(0, 0)
+    dec.close()
