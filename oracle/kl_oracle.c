@@ -18,6 +18,9 @@
  *     o[hq] = softmax(q[hq] . K[g]^T / sqrt(hd)) V[g],  g = hq div (nq/nkv), over 0..p
  *     x = x + Wo o
  *     m = rmsnorm(x; g2[l]);  x = x + Wd (silu(Wg m) * (Wu m))
+ *       (mixture-of-experts layers: r = Wr m; the top_k largest r_e, lowest index first among equals, chosen in
+ *        descending order; their weights = softmax over the chosen logits;
+ *        x = x + sum over the chosen e, in that order, of weight_e * Wd_e (silu(Wg_e m) * (Wu_e m)))
  *   hidden = x;  logits = Wlm rmsnorm(x; gf);  next = argmax(logits) (lowest index on ties)
  *
  * Precision: weights, gains, embedding and cached K/V are bf16 VALUES; every
@@ -55,6 +58,12 @@ typedef struct {
 typedef struct {
     const uint16_t *wq, *wk, *wv, *wo, *wgate, *wup, *wdown, *norm1, *norm2;
     const uint16_t *bq, *bk, *bv; /* optional biases of the q, k, v projections (NULL: none), bf16 */
+    /* Mixture-of-experts MLP (n_experts > 0; the paper's Table 2 lists such a decoder, Mixtral 8x7B): a router matrix
+     * [n_experts, hidden] and, per expert, gate / up [ffn, hidden] and down [hidden, ffn]; wgate / wup / wdown are then
+     * unused.  n_experts == 0: the dense MLP above. */
+    int32_t n_experts, top_k;
+    const uint16_t *router;
+    const uint16_t *const *ex_gate, *const *ex_up, *const *ex_down;
 } ko_layer_weights;
 
 /* ---------------------------------------------------------------- bf16 */
@@ -165,6 +174,26 @@ void ko_attention_head(const double *q, const uint16_t *K, const uint16_t *V, in
     }
 }
 
+/* Router of a mixture-of-experts layer: the k largest of E logits in descending order (among equal logits the lower
+ * index first), and the softmax over those k as their weights.  Equal to a softmax over all E followed by top-k and
+ * renormalisation. */
+void ko_moe_route(const double *logits, int E, int k, int32_t *idx, double *w) {
+    double chosen[64];
+    for (int s = 0; s < k; ++s) {
+        int best = -1;
+        for (int e = 0; e < E; ++e) {
+            int taken = 0;
+            for (int t = 0; t < s; ++t)
+                if (idx[t] == e) taken = 1;
+            if (taken) continue;
+            if (best < 0 || logits[e] > logits[best]) best = e;
+        }
+        idx[s] = best;
+        chosen[s] = logits[best];
+    }
+    ko_softmax(chosen, k, w);
+}
+
 /* ---------------------------------------------------------------- blocks */
 
 /* Embedding block: x = E[token]. */
@@ -241,13 +270,32 @@ int ko_decoder_layer(const ko_desc *d, const ko_layer_weights *w, uint16_t *kcac
 
     /* MLP half */
     ko_rmsnorm(x, w->norm2, H, d->rms_eps, a, c, count_only);
-    ko_matvec(w->wgate, F, H, a, gate, c, count_only);
-    ko_matvec(w->wup, F, H, a, up, c, count_only);
-    if (!count_only)
-        for (int f = 0; f < F; ++f) gate[f] = ko_silu(gate[f]) * up[f];
-    ko_matvec(w->wdown, H, F, gate, t, c, count_only);
-    if (!count_only)
-        for (int i = 0; i < H; ++i) x[i] += t[i];
+    if (w->n_experts > 0) {
+        const int E = w->n_experts, K = w->top_k;
+        if (K < 1 || K > E || E > 64) return -1;
+        double r[64], wt[64];
+        int32_t idx[64];
+        ko_matvec(w->router, E, H, a, r, c, count_only);
+        if (!count_only) ko_moe_route(r, E, K, idx, wt);
+        for (int s = 0; s < K; ++s) {
+            const int e = count_only ? 0 : idx[s];
+            ko_matvec(count_only ? NULL : w->ex_gate[e], F, H, a, gate, c, count_only);
+            ko_matvec(count_only ? NULL : w->ex_up[e], F, H, a, up, c, count_only);
+            if (!count_only)
+                for (int f = 0; f < F; ++f) gate[f] = ko_silu(gate[f]) * up[f];
+            ko_matvec(count_only ? NULL : w->ex_down[e], H, F, gate, t, c, count_only);
+            if (!count_only)
+                for (int i = 0; i < H; ++i) x[i] += wt[s] * t[i];
+        }
+    } else {
+        ko_matvec(w->wgate, F, H, a, gate, c, count_only);
+        ko_matvec(w->wup, F, H, a, up, c, count_only);
+        if (!count_only)
+            for (int f = 0; f < F; ++f) gate[f] = ko_silu(gate[f]) * up[f];
+        ko_matvec(w->wdown, H, F, gate, t, c, count_only);
+        if (!count_only)
+            for (int i = 0; i < H; ++i) x[i] += t[i];
+    }
 
     free(a); free(q); free(k); free(v); free(o); free(t); free(gate); free(up); free(sc);
     return 0;

@@ -43,7 +43,10 @@ class Counters(C.Structure):
 
 class LayerWeights(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "norm1", "norm2",
-                                           "bq", "bk", "bv")]   # the biases are optional (null: none)
+                                           "bq", "bk", "bv")] + \
+               [("n_experts", C.c_int32), ("top_k", C.c_int32), ("router", C.c_void_p),   # mixture-of-experts layers
+                ("ex_gate", C.POINTER(C.c_void_p)), ("ex_up", C.POINTER(C.c_void_p)), ("ex_down", C.POINTER(C.c_void_p))]
+DENSE_FIELDS = ("wq", "wk", "wv", "wo", "wgate", "wup", "wdown", "norm1", "norm2", "bq", "bk", "bv")
 
 
 _lib = None
@@ -76,6 +79,8 @@ def lib():
         l.ko_decoder_layer.restype = C.c_int
         l.ko_classifier.argtypes = [C.POINTER(Desc), vp, vp, dp, dp, cp, C.c_int]
         l.ko_classifier.restype = C.c_int
+        l.ko_moe_route.argtypes = [dp, C.c_int, C.c_int, C.POINTER(C.c_int32), dp]
+        l.ko_moe_route.restype = None
         l.ko_argmax.argtypes = [dp, C.c_int]
         l.ko_argmax.restype = C.c_int
         l.ko_num_threads.restype = C.c_int
@@ -176,6 +181,15 @@ def attention_head(q: np.ndarray, K_u16: np.ndarray, V_u16: np.ndarray) -> np.nd
     return out
 
 
+def moe_route(logits: np.ndarray, k: int):
+    """Chosen experts (descending logit, lower index first among equals) and their softmax weights."""
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    idx = (C.c_int32 * k)()
+    w = np.empty(k, dtype=np.float64)
+    lib().ko_moe_route(_dp(logits), logits.size, k, idx, _dp(w))
+    return list(idx), w
+
+
 def argmax(logits: np.ndarray) -> int:
     logits = np.ascontiguousarray(logits, dtype=np.float64)
     return int(lib().ko_argmax(_dp(logits), logits.size))
@@ -203,7 +217,18 @@ class Oracle:
     def _layer_struct(self, l: int):
         w = self._layer_weights(l)
         keep = {k: as_u16(v) for k, v in w.items()}
-        s = LayerWeights(*[C.c_void_p(keep[n].ctypes.data) if n in keep else None for n, _ in LayerWeights._fields_])
+        s = LayerWeights()
+        for n in DENSE_FIELDS:
+            if n in keep:
+                setattr(s, n, keep[n].ctypes.data)
+        E = int(getattr(self.shape, "n_experts", 0) or 0)
+        if E > 0:   # tensors router, wgate_e<i>, wup_e<i>, wdown_e<i>
+            s.n_experts, s.top_k = E, int(self.shape.top_k)
+            s.router = keep["router"].ctypes.data
+            for field, stem in (("ex_gate", "wgate_e"), ("ex_up", "wup_e"), ("ex_down", "wdown_e")):
+                arr = (C.c_void_p * E)(*[keep[f"{stem}{e}"].ctypes.data for e in range(E)])
+                keep["_" + field] = arr
+                setattr(s, field, C.cast(arr, C.POINTER(C.c_void_p)))
         return s, keep
 
     def embed(self, token: int) -> np.ndarray:
@@ -260,6 +285,7 @@ def count_step(shape, batch: int, position: int, max_ctx: int | None = None) -> 
         c = Counters()
         lib().ko_embed(C.byref(d), None, 0, None, C.byref(c), 1)
         lw = LayerWeights()
+        lw.n_experts, lw.top_k = int(getattr(shape, "n_experts", 0) or 0), int(getattr(shape, "top_k", 0) or 0)
         for _ in range(shape.n_layers):
             rc = lib().ko_decoder_layer(C.byref(d), C.byref(lw), None, None, position, None, C.byref(c), 1)
             assert rc == 0

@@ -52,6 +52,8 @@ class ModelShape:
     rms_eps: float = 1e-5
     rope_theta: float = 10000.0
     qkv_bias: bool = False   # q, k, v = W a + b (the 72B decoder of the paper's Table 2 has such biases)
+    n_experts: int = 0       # > 0: mixture-of-experts MLP (the 8x7B decoder of Table 2): a router and n_experts MLPs
+    top_k: int = 0           # experts that process a token
 
     @property
     def q_dim(self) -> int:
@@ -78,6 +80,11 @@ GLOBAL_TENSORS = ("embed", "norm_f", "lm_head")
 
 def tensor_shape(shape: ModelShape, name: str) -> tuple[int, ...]:
     s = shape
+    if name == "router":
+        return (s.n_experts, s.hidden)
+    for stem in ("wgate_e", "wup_e", "wdown_e"):   # expert matrices: the dense matrix's shape
+        if name.startswith(stem):
+            name = stem[:-2]
     return {
         "wq": (s.q_dim, s.hidden),
         "wk": (s.kv_dim, s.hidden),
@@ -188,9 +195,19 @@ def make_tensor(shape: ModelShape, name: str, layer: int = -1, seed: int = 0, de
     return t.view(*dims)
 
 
-def make_layer(shape: ModelShape, layer: int, seed: int = 0, device="cpu") -> dict[str, torch.Tensor]:
+def layer_tensor_names(shape: ModelShape) -> tuple[str, ...]:
+    """Names of one layer's tensors.  Mixture-of-experts layers have `router` and, per expert e, wgate_e<e>, wup_e<e>,
+    wdown_e<e> in place of the dense wgate, wup, wdown."""
     names = LAYER_TENSORS + (BIAS_TENSORS if shape.qkv_bias else ())
-    return {n: make_tensor(shape, n, layer, seed, device) for n in names}
+    if shape.n_experts > 0:
+        names = tuple(n for n in names if n not in ("wgate", "wup", "wdown")) + ("router",)
+        for e in range(shape.n_experts):
+            names += (f"wgate_e{e}", f"wup_e{e}", f"wdown_e{e}")
+    return names
+
+
+def make_layer(shape: ModelShape, layer: int, seed: int = 0, device="cpu") -> dict[str, torch.Tensor]:
+    return {n: make_tensor(shape, n, layer, seed, device) for n in layer_tensor_names(shape)}
 
 
 def make_globals(shape: ModelShape, seed: int = 0, device="cpu", with_embed_table: bool = True) -> dict[str, torch.Tensor]:

@@ -342,7 +342,16 @@ def _torch_reference_step(shape, layers, glob, cache_bf16, token, p):
         o = F.scaled_dot_product_attention(q.view(1, nq, 1, hd), K.unsqueeze(0), V.unsqueeze(0)).reshape(nq * hd)
         x = x + w["wo"].to(f64) @ o
         m = norm(x, w["norm2"])
-        x = x + w["wdown"].to(f64) @ (F.silu(w["wgate"].to(f64) @ m) * (w["wup"].to(f64) @ m))
+        if "router" in w:   # mixture of experts: top-k of the router logits, softmax over the chosen, weighted expert MLPs
+            r = w["router"].to(f64) @ m
+            val, idx = torch.topk(r, shape.top_k)
+            gates = torch.softmax(val, dim=0)
+            y = torch.zeros_like(x)
+            for g, e in zip(gates, idx.tolist()):
+                y = y + g * (w[f"wdown_e{e}"].to(f64) @ (F.silu(w[f"wgate_e{e}"].to(f64) @ m) * (w[f"wup_e{e}"].to(f64) @ m)))
+            x = x + y
+        else:
+            x = x + w["wdown"].to(f64) @ (F.silu(w["wgate"].to(f64) @ m) * (w["wup"].to(f64) @ m))
     logits = glob["lm_head"].to(f64) @ norm(x, glob["norm_f"])
     return x.numpy(), logits.numpy()
 
@@ -477,3 +486,87 @@ def test_generator_statistics_and_determinism():
     # embed_rows regenerates table rows without the table
     E = gen.make_tensor(gen.TINY, "embed", -1, 0)
     assert torch.equal(gen.embed_rows(gen.TINY, [5, 1000], 0), E[[5, 1000]])
+
+
+# ------------------------------------------------------------------ mixture-of-experts layers
+
+def test_moe_router_top_k_order_ties_and_weights():
+    """Router of a mixture-of-experts layer: the k largest logits in descending order, the lower index first among
+    equals; the weights are the softmax over the chosen logits, which is the softmax over ALL experts restricted to
+    the chosen ones and renormalised; k = E is the plain softmax; equal logits give equal weights 1/k."""
+    idx, w = ko.moe_route(np.array([0.1, 2.0, 2.0, -1.0, 0.5]), 3)
+    assert idx == [1, 2, 4]                                   # tie between experts 1 and 2: the lower index first
+    assert abs(w.sum() - 1.0) < 1e-15 and w[0] == w[1] > w[2]
+    idx, w = ko.moe_route(np.array([3.0, 3.0, 3.0, 3.0]), 2)
+    assert idx == [0, 1] and np.allclose(w, [0.5, 0.5], rtol=0, atol=1e-16)
+    idx, w = ko.moe_route(np.array([-5.0, 7.0, 1.0]), 1)
+    assert idx == [1] and w[0] == 1.0
+    rng = np.random.default_rng(1)
+    for _ in range(50):
+        E, k = int(rng.integers(2, 17)), 0
+        k = int(rng.integers(1, E + 1))
+        r = rng.normal(size=E) * 3.0
+        idx, w = ko.moe_route(r, k)
+        order = sorted(range(E), key=lambda e: (-r[e], e))[:k]          # brute force: sort by (-logit, index)
+        assert idx == order
+        full = np.exp(r - r.max())
+        full /= full.sum()                                              # softmax over all experts ...
+        assert np.allclose(w, full[order] / full[order].sum(), rtol=1e-13, atol=0)   # ... restricted and renormalised
+        if k == E:
+            assert np.allclose(w, full[order], rtol=1e-13, atol=0)
+
+
+def _moe_shape(**kw):
+    return dataclasses.replace(gen.TINY, n_experts=4, top_k=2, **kw)
+
+
+def test_moe_identical_experts_equal_the_dense_layer():
+    """Every expert holds the dense model's MLP matrices: whatever the router picks, the gates sum to one, so the
+    mixture-of-experts model computes exactly what the dense model does -- also with k = E and a zero router (all gates
+    equal: the plain mean of the experts), and with k = 1 (one expert, gate 1)."""
+    dense_shape, dense_layers, glob, cache = _tiny_setup()
+    for E, k, zero_router in ((4, 2, False), (4, 4, True), (3, 1, False)):
+        shape = dataclasses.replace(dense_shape, n_experts=E, top_k=k)
+        layers = []
+        for l, lw in enumerate(dense_layers):
+            d = {n: t for n, t in lw.items() if n not in ("wgate", "wup", "wdown")}
+            d["router"] = gen.make_tensor(shape, "router", l, 0, "cpu")
+            if zero_router:
+                d["router"] = torch.zeros_like(d["router"])
+            for e in range(E):
+                d[f"wgate_e{e}"], d[f"wup_e{e}"], d[f"wdown_e{e}"] = lw["wgate"], lw["wup"], lw["wdown"]
+            layers.append(d)
+        c_moe, c_dense = u16(cache).copy(), u16(cache).copy()
+        moe = ko.Oracle(shape, cache.shape[4], lambda l: layers[l], glob)
+        dense = ko.Oracle(dense_shape, cache.shape[4], lambda l: dense_layers[l], glob)
+        h1, l1, n1 = moe.step(c_moe, [5], [128])
+        h2, l2, n2 = dense.step(c_dense, [5], [128])
+        assert np.allclose(h1, h2, rtol=1e-12, atol=1e-13) and np.allclose(l1, l2, rtol=1e-11, atol=1e-12)
+        assert n1[0] == n2[0] and np.array_equal(c_moe, c_dense)
+
+
+def test_moe_whole_step_against_torch_library_restatement():
+    """Mixture-of-experts decoder (4 experts, 2 per token, all different) against the torch re-statement (topk,
+    softmax, matmul) for 8 greedy steps."""
+    shape = _moe_shape()
+    layers = [gen.make_layer(shape, l, 3, "cpu") for l in range(shape.n_layers)]
+    glob = gen.make_globals(shape, 3, "cpu")
+    cache = gen.make_kv_cache(shape, 1, 64, 80, 3, "cpu")
+    orc = ko.Oracle(shape, 80, lambda l: layers[l], glob)
+    c_or, c_ref = u16(cache).copy(), cache.clone()
+    tok = 11
+    for step in range(8):
+        p = 64 + step
+        hidden, logits, nxt = orc.step(c_or, [tok], [p])
+        h_ref, l_ref = _torch_reference_step(shape, layers, glob, c_ref, tok, p)
+        assert np.allclose(hidden[0], h_ref, rtol=1e-10, atol=1e-11)
+        assert np.allclose(logits[0], l_ref, rtol=1e-9, atol=1e-10)
+        assert np.array_equal(c_or, u16(c_ref))
+        assert int(nxt[0]) == int(np.argmax(l_ref))
+        tok = int(nxt[0])
+    # the counters: a mixture-of-experts layer touches the router and top_k experts, not all of them
+    cnt = ko.count_step(shape, 1, 64)
+    per_expert = 3 * shape.hidden * shape.ffn
+    attn = shape.hidden * shape.head_dim * (2 * shape.n_q_heads + 2 * shape.n_kv_heads)
+    mlp = shape.top_k * per_expert + shape.n_experts * shape.hidden
+    assert cnt["weight_bytes"] == 2 * (shape.n_layers * (attn + mlp + 2 * shape.hidden) + shape.hidden + shape.vocab * shape.hidden)
