@@ -54,6 +54,9 @@ WORKLOADS = {
     # the 3B decoder of Table 2 by its public dimensions
     "llama32_3b_b1_ctx4096": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 1, 4096, 64),
     "llama32_3b_b16_ctx8192": (gen.ModelShape(28, 3072, 24, 8, 128, 8192, 128256, 1e-5, 500000.0), 16, 8192, 16),
+    # the mixture-of-experts decoder of Table 2 by its public dimensions: 8 experts of FFN 14336, 2 per token (93 GB of
+    # weights, of which a step reads 25 GB)
+    "mixtral_8x7b_shape_b1_ctx4096": (gen.ModelShape(32, 4096, 32, 8, 128, 14336, 32000, 1e-5, 1000000.0, False, 8, 2), 1, 4096, 32),
     "llama31_70b_2layers_b8_ctx4096": (gen.ModelShape(2, 8192, 64, 8, 128, 28672, 128256, 1e-5, 500000.0), 8, 4096, 4),
     # two layers, 32 sequences at the full context: a few GB on the device, for profiler captures of the batched path
     "llama31_8b_2layers_b32_ctx4096": (gen.ModelShape(2, 4096, 32, 8, 128, 14336, 128256, 1e-5, 500000.0), 32, 4096, 4),
@@ -63,7 +66,12 @@ NOMINAL_HBM_GBS = 8000.0
 
 
 def layer_weight_bytes(s) -> int:
-    return 2 * (s.hidden * s.head_dim * (2 * s.n_q_heads + 2 * s.n_kv_heads) + 3 * s.hidden * s.ffn + 2 * s.hidden)
+    """Weight bytes one decode step reads per layer.  A mixture-of-experts layer reads its router and the top_k chosen
+    experts, not all of them."""
+    mlp = 3 * s.hidden * s.ffn
+    if getattr(s, "n_experts", 0):
+        mlp = s.top_k * mlp + s.n_experts * s.hidden
+    return 2 * (s.hidden * s.head_dim * (2 * s.n_q_heads + 2 * s.n_kv_heads) + mlp + 2 * s.hidden)
 
 
 def kv_bytes(s, batch: int, position: int) -> int:
@@ -365,7 +373,10 @@ def replica_throughput(steps: int, batch: int, world: int, ms_local: float) -> t
 def oracle_layers_that_fit(shape, budget_bytes=24e9) -> int:
     """Decoder layers whose weights the oracle's host can hold at once: all of them for models up to the 8B shape (whole
     decode steps are executed), a bounded sample for the larger ones."""
-    return shape.n_layers if shape.n_layers * layer_weight_bytes(shape) <= budget_bytes else 0
+    stored = layer_weight_bytes(shape)
+    if getattr(shape, "n_experts", 0):   # the host holds every expert
+        stored += 2 * 3 * shape.hidden * shape.ffn * (shape.n_experts - shape.top_k)
+    return shape.n_layers if shape.n_layers * stored <= budget_bytes else 0
 
 
 class OracleSampler:

@@ -60,7 +60,10 @@ enum {
     /* only for models created with KL_FLAG_QKV_BIAS: q, k, v = W a + b, the bias added before the rotation */
     KL_BQ = 12,     /* [n_q_heads*head_dim] */
     KL_BK = 13,     /* [n_kv_heads*head_dim] */
-    KL_BV = 14      /* [n_kv_heads*head_dim] */
+    KL_BV = 14,     /* [n_kv_heads*head_dim] */
+    /* only for mixture-of-experts models (n_experts > 0) */
+    KL_WROUTER = 15 /* [n_experts, hidden]  router of the layer's MLP; the experts' KL_WGATE / KL_WUP / KL_WDOWN are loaded
+                       with kl_load_expert_weights */
 };
 
 /* kl_model_desc.flags: the q, k, v projections carry biases (KL_BQ, KL_BK, KL_BV must be loaded for every layer).
@@ -78,6 +81,13 @@ typedef struct {
     uint32_t max_batch;
     uint32_t max_ctx; /* capacity of the KV cache in positions */
     uint32_t flags;   /* 0 or KL_FLAG_QKV_BIAS */
+    /* Mixture-of-experts MLP (the 8x7B decoder of the paper's Table 2 is of this kind; the paper's operator list has no
+     * such term): n_experts > 0 gives every layer a router [n_experts, hidden] and n_experts MLPs of width ffn, of
+     * which the top_k with the largest router logits (the lower index first among equals) process a token, weighted
+     * by the softmax over those top_k logits.  0, 0 = dense MLP.  Limits: n_experts <= 16, top_k <= 4 and
+     * top_k x (column pieces of the down projection) <= 20, i.e. top_k <= 2 at ffn 14336.  Such models decode batches
+     * sequence after sequence (no tensor-core path), and KL_MODE_PER_STAGE keeps gate/up and down in one launch. */
+    uint32_t n_experts, top_k;
 } kl_model_desc;
 
 /* Sizes of the two device arenas the caller must provide to kl_create (both 256-byte aligned).
@@ -100,6 +110,12 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
  * by the loop variable; the closing paragraph of that section: grouped tensors stored contiguously, in loop order).  `bytes` must equal the tensor's size.  layer = -1 for KL_EMBED, KL_NORM_F,
  * KL_LM_HEAD.  The copy is ordered on `stream`; the source may be released once the stream has passed it. */
 kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, size_t bytes, void* stream);
+
+/* The same for one expert's matrix of a mixture-of-experts model: tensor = KL_WGATE, KL_WUP or KL_WDOWN, expert in
+ * [0, n_experts).  In the looped kernel the experts' matrices are the one grouped parameter whose ADDRESS depends on an
+ * activation (Section 3.2's grouping assumes addresses known up front): the weight stream of a layer's MLP starts when
+ * the layer's router has run; everything else is requested ahead as for a dense model. */
+kl_status kl_load_expert_weights(kl_handle* h, int tensor, int layer, int expert, const void* src, size_t bytes, void* stream);
 
 /* Bytes of a KV cache for `batch` sequences: layout [n_layers][2 (K,V)][batch][n_kv_heads][max_ctx][head_dim]
  * bf16.  The cache is read, written and live after the call, i.e. element (6) {In, Live, Out} of the lattice of

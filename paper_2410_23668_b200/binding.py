@@ -25,7 +25,7 @@ KL_MODE_PER_LAYER = 1
 KL_MODE_PER_STAGE = 2
 
 TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup": 6, "wdown": 7,
-              "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11, "bq": 12, "bk": 13, "bv": 14}
+              "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11, "bq": 12, "bk": 13, "bv": 14, "router": 15}
 KL_FLAG_QKV_BIAS = 1
 
 # every symbol include/kl.h declares
@@ -34,14 +34,14 @@ EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_by
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
            "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
            "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy", "kl_decode_greedy_tokens",
-           "kl_decode_greedy_tokens_host", "kl_debug_set_step", "kl_debug_set_jitter")
+           "kl_decode_greedy_tokens_host", "kl_debug_set_step", "kl_debug_set_jitter", "kl_load_expert_weights")
 
 
 class ModelDesc(C.Structure):
     _fields_ = [("n_layers", C.c_uint32), ("hidden", C.c_uint32), ("n_q_heads", C.c_uint32),
                 ("n_kv_heads", C.c_uint32), ("head_dim", C.c_uint32), ("ffn", C.c_uint32), ("vocab", C.c_uint32),
                 ("rms_eps", C.c_float), ("rope_theta", C.c_float), ("max_batch", C.c_uint32),
-                ("max_ctx", C.c_uint32), ("flags", C.c_uint32)]
+                ("max_ctx", C.c_uint32), ("flags", C.c_uint32), ("n_experts", C.c_uint32), ("top_k", C.c_uint32)]
 
 
 _lib = None
@@ -63,6 +63,8 @@ def lib():
     l.kl_create.restype = i32
     l.kl_load_weights.argtypes = [vp, C.c_int, C.c_int, vp, C.c_size_t, vp]
     l.kl_load_weights.restype = i32
+    l.kl_load_expert_weights.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp, C.c_size_t, vp]
+    l.kl_load_expert_weights.restype = i32
     l.kl_kv_cache_bytes.argtypes = [vp, u32]
     l.kl_kv_cache_bytes.restype = C.c_size_t
     l.kl_set_mode.argtypes = [vp, C.c_int]
@@ -135,7 +137,8 @@ def _check(code: int, where: str) -> None:
 def make_desc(shape, max_batch: int, max_ctx: int) -> ModelDesc:
     return ModelDesc(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                      shape.vocab, float(shape.rms_eps), float(shape.rope_theta), max_batch, max_ctx,
-                     KL_FLAG_QKV_BIAS if getattr(shape, "qkv_bias", False) else 0)
+                     KL_FLAG_QKV_BIAS if getattr(shape, "qkv_bias", False) else 0,
+                     int(getattr(shape, "n_experts", 0) or 0), int(getattr(shape, "top_k", 0) or 0))
 
 
 def kl_workspace_bytes(desc: ModelDesc) -> tuple[int, int]:
@@ -190,8 +193,13 @@ class Decoder:
     def kl_load_weights(self, name: str, layer: int, tensor, stream=None) -> None:
         t = tensor.contiguous()
         assert t.dtype == self.torch.bfloat16
-        _check(lib().kl_load_weights(self.handle, TENSOR_IDS[name], layer, _ptr(t), t.numel() * 2, _stream_ptr(stream)),
-               f"kl_load_weights({name}, {layer})")
+        if "_e" in name:   # an expert's matrix of a mixture-of-experts layer: wgate_e<i>, wup_e<i>, wdown_e<i>
+            stem, expert = name.rsplit("_e", 1)
+            _check(lib().kl_load_expert_weights(self.handle, TENSOR_IDS[stem], layer, int(expert), _ptr(t), t.numel() * 2,
+                                                _stream_ptr(stream)), f"kl_load_expert_weights({name}, {layer})")
+        else:
+            _check(lib().kl_load_weights(self.handle, TENSOR_IDS[name], layer, _ptr(t), t.numel() * 2, _stream_ptr(stream)),
+                   f"kl_load_weights({name}, {layer})")
         if t.device.type == "cpu":
             self.torch.cuda.synchronize()  # pageable source must outlive the copy
 

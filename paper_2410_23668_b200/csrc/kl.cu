@@ -111,6 +111,7 @@ __device__ __forceinline__ bool cta_begin(const Params& p, const SM& s, uint32_t
         s.ctx()->step = ld_step(p.step_dev);
         s.ctx()->pos = (uint32_t)p.positions[p.b0];
         s.ctx()->rope_cs = rope;
+        if constexpr (SM::kMoe) s.moe()->seq = 0u;
         for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
             mbar_init(smem_u32(&s.full()[i]), 1);
             mbar_init(smem_u32(&s.empty()[i]), 1);
@@ -175,6 +176,7 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
         trace_stamp(p, s, cta, l, 7, ctid);
         // RMSNorm + gate/up projections + SwiGLU
         xscale = load_vec(p, s, p.xb, p.H, tag_of(p, cx, l, TG_XB), true, p.g2 + lo, ctid);
+        if constexpr (SM::kMoe) moe_router(p, s, l, xscale, ctid);   // which experts, with which gate weights
         trace_stamp(p, s, cta, l, 9, ctid);
         out = {nullptr, p.h, nullptr, 0u};
         plan = PL_GU;
@@ -190,7 +192,24 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
         ep = EP_RESIDUAL;
         xsrc = p.h;
     }
-    gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+    if constexpr (SM::kMoe) {
+        if (st == ST_GU || st == ST_D) {
+            // the stage runs over the chosen experts: their (gate, up) rows one expert after the other; in the down
+            // projection their matrices side by side, the input vector being the experts' (gated) SwiGLU outputs
+            GemvPlan pm = p.plan[plan];
+            if (st == ST_GU) {
+                pm.R *= p.top_k;
+                pm.nunits *= p.top_k;
+            } else {
+                pm.nseg = p.top_k;
+            }
+            gemv_stage(p, s, pm, ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+        } else {
+            gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+        }
+    } else {
+        gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
+    }
     if (st == ST_GU) {
         stage_signal(p.counters + l, ctid, skip == ST_GU);
         trace_stamp(p, s, cta, l, 10, ctid);
@@ -202,10 +221,10 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
 // stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
 // boundary after every operator group).
-template <bool TR>
+template <bool TR, bool MOE>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
                                                                  uint32_t sbeg, uint32_t send) {
-    const SmemT<TR> s;
+    const SmemT<TR, MOE> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;   // an earlier kernel of this step flagged bad input: the step is a no-op
     if (warp == NCW) {
@@ -337,6 +356,7 @@ template <class SM>
 __device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uint32_t cta, const TokenParams& t) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     const uint32_t step0 = ld_step(p.step_dev), pos0 = (uint32_t)p.positions[0];
+    uint32_t routed = 0, ex[MAX_TOP_K] = {0u, 0u, 0u, 0u};   // mixture of experts: layers routed so far, the chosen experts
     for (uint32_t k = 0; k < t.K && !r.aborted; ++k) {
         const AttnUnit u = attn_unit(p, cta, pos0 + k);
         for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
@@ -361,8 +381,14 @@ __device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uin
             }
             produce_attention(p, s, r, u, l);
             produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
-            produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
-            produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+            if constexpr (SM::kMoe) {
+                if (!moe_wait_route(p, s, ++routed, ex)) r.aborted = true;   // the experts of this layer are known now
+                if (!r.aborted) produce_matrix_moe(p, s, r, p.plan[PL_GU], p.wgu + lo, cta, ex, false);
+                if (!r.aborted) produce_matrix_moe(p, s, r, p.plan[PL_D], p.wd + lo, cta, ex, true);
+            } else {
+                produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
+                produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
+            }
         }
         if (!r.aborted) produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
     }
@@ -467,9 +493,9 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
 // K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
-template <bool TR>
+template <bool TR, bool MOE>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
-    const SmemT<TR> s;
+    const SmemT<TR, MOE> s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, t.rope)) return;
     if (warp == NCW) {
@@ -578,7 +604,7 @@ inline uint32_t ceil_div(uint32_t a, uint32_t b) { return (a + b - 1) / b; }
 
 struct Layout {
     // weight arena, element offsets (bf16)
-    size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, layer_stride;
+    size_t off_qkv, off_o, off_gu, off_d, off_g1, off_g2, off_bqkv, off_router, expert_stride, layer_stride;
     size_t off_gf, off_lm, off_embed, weight_elems;
     // scratch arena, byte offsets
     size_t sxa, sxb, sqkv, so, sh, spart, spart_ml, srope, sinvf, scounters, sstatus, sstep, stok, spos, slogits, samax, shid, stokp, stplan, sbxop, sbssq, sbpart, sbq, sbao, sbaml, sbbar, scratch_bytes;
@@ -599,6 +625,9 @@ bool shape_supported(const kl_model_desc& d, int num_sms) {
     if (!pow2 && !(G <= 8 && (d.head_dim == 64 || d.head_dim == 128))) return false;
     if ((uint64_t)d.n_kv_heads > (uint64_t)num_sms) return false;
     if (!(d.rms_eps >= 0.f) || !(d.rope_theta > 0.f)) return false;
+    if (d.n_experts || d.top_k) {
+        if (d.n_experts > (uint32_t)MAX_EXPERTS || d.top_k < 1 || d.top_k > (uint32_t)MAX_TOP_K || d.top_k > d.n_experts) return false;
+    }
     return true;
 }
 
@@ -632,11 +661,16 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     size_t o = 0;
     y.off_qkv = o; o += (QD + 2 * KVD) * H;
     y.off_o = o;   o += H * QD;
-    y.off_gu = o;  o += 2 * F * H;
-    y.off_d = o;   o += H * F;
+    // dense: gate/up | down; mixture of experts: that pair once per expert, expert_stride elements apart
+    const size_t NE = d.n_experts ? d.n_experts : 1;
+    y.expert_stride = 3 * F * H;
+    y.off_gu = o;
+    y.off_d = o + 2 * F * H;
+    o += NE * y.expert_stride;
     y.off_g1 = o;  o += H;
     y.off_g2 = o;  o += H;
     y.off_bqkv = o; o += (d.flags & KL_FLAG_QKV_BIAS) ? align_up((QD + 2 * KVD) * 2, 16) / 2 : 0;
+    y.off_router = o; o += d.n_experts ? align_up((size_t)d.n_experts * H * 2, 16) / 2 : 0;
     y.layer_stride = align_up(o * 2, ALIGN) / 2;
     o = y.layer_stride * d.n_layers;
     y.off_gf = o;    o += align_up(H * 2, ALIGN) / 2;
@@ -653,7 +687,7 @@ Layout make_layout(const kl_model_desc& d, int num_sms) {
     y.sxb = s;       s += align_up(B * H * 8);
     y.sqkv = s;      s += align_up(B * (QD + 2 * KVD) * 8);
     y.so = s;        s += align_up(B * QD * 8);
-    y.sh = s;        s += align_up(B * F * 4);
+    y.sh = s;        s += align_up(B * F * 4 * (d.top_k ? d.top_k : 1));
     y.spart = s;     s += align_up(units * G * d.head_dim * 8);
     y.spart_ml = s;  s += align_up(units * G * 2 * 8);
     y.srope = s;     s += align_up((B > 1 ? 32 : B) * d.head_dim * 4);
@@ -943,7 +977,8 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
         else
             h->use_tc_attention = 0;
     }
-    h->loaded = (uint8_t*)calloc((size_t)(KL_BV + 1) * (size_t)d.n_layers, 1);
+    // one flag per (tensor, layer), then one per (expert matrix kind, expert, layer)
+    h->loaded = (uint8_t*)calloc((size_t)(KL_WROUTER + 1 + 3 * (size_t)d.n_experts) * (size_t)d.n_layers, 1);
     if (!h->loaded) { delete h; return KL_ERR_INVALID_ARG; }
 
     Params& p = h->prm;
@@ -965,6 +1000,16 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0, false);
     p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0, true);
     if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    p.n_experts = d.n_experts;
+    p.top_k = d.top_k;
+    p.expert_stride = y.expert_stride;
+    for (int i = 0; i < PL_COUNT; ++i) p.plan[i].nseg = 1;
+    if (d.n_experts) {
+        // the chosen experts' pieces of a down-projection unit meet in one table; (gate, up) units must not straddle experts
+        if (p.plan[PL_D].npieces * d.top_k > (uint32_t)MAX_PIECES || (2 * p.F) % p.plan[PL_GU].rpc || p.plan[PL_GU].R % p.plan[PL_GU].rpc) {
+            free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE;
+        }
+    }
 
     // shared memory: input vector area (also the attention workspace), then as many ring slots as fit
     uint32_t vecf = p.H > p.QD ? p.H : p.QD;  // the down projection reads its input from L2, not from this area
@@ -988,18 +1033,20 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
     // The shared-memory limit is an attribute of the kernel, not of a handle: it is raised to the device's opt-in
     // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
-    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
-    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     {
         int tocc = 0;
-        h->token_ok = cudaFuncSetAttribute(kl_token_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaFuncSetAttribute(kl_token_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+        h->token_ok = cudaFuncSetAttribute(kl_token_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
+                      cudaFuncSetAttribute(kl_token_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
+                      cudaFuncSetAttribute(kl_token_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
+                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
-    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true>, NTHREADS, h->smem_bytes);
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false>, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
         fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
                         "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
@@ -1010,6 +1057,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.wqkv = w + y.off_qkv; p.wo = w + y.off_o; p.wgu = w + y.off_gu; p.wd = w + y.off_d;
     p.bqkv = (d.flags & KL_FLAG_QKV_BIAS) ? w + y.off_bqkv : nullptr;
     p.g1 = w + y.off_g1; p.g2 = w + y.off_g2; p.gf = w + y.off_gf; p.wlm = w + y.off_lm; p.embed = w + y.off_embed;
+    p.wrouter = d.n_experts ? w + y.off_router : nullptr;
     uint8_t* sc = h->scratch;
     p.xa = (TW*)(sc + y.sxa); p.xb = (TW*)(sc + y.sxb); p.qkv = (TW*)(sc + y.sqkv); p.o = (TW*)(sc + y.so);
     p.h = (float*)(sc + y.sh);
@@ -1060,7 +1108,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->bgraph_launches = 0;
     h->bt_ok = 0;
     h->bl_ok = 0;
-    if (d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
+    if (d.n_experts == 0 && d.max_batch > 1 && d.max_batch <= (uint32_t)BG_MAX_BATCH && (p.hd == 64 || p.hd == 128) && p.G <= (uint32_t)MAX_G &&
         p.H % 8 == 0 && p.QD % 8 == 0 && p.F % 8 == 0) {
         const uint32_t QR = p.QD + 2 * p.KVD;
         const size_t ba_smem = batched_attn_smem();
@@ -1100,8 +1148,9 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
     const Params& p = h->prm;
     const Layout y = make_layout(h->desc, h->num_sms);
     const bool global_t = (tensor == KL_EMBED || tensor == KL_NORM_F || tensor == KL_LM_HEAD);
-    if (tensor < 0 || tensor > KL_BV) return KL_ERR_INVALID_ARG;
-    if (tensor > KL_LM_HEAD && !(h->desc.flags & KL_FLAG_QKV_BIAS)) return KL_ERR_INVALID_ARG;   // this model has no biases
+    if (tensor < 0 || tensor > KL_WROUTER) return KL_ERR_INVALID_ARG;
+    if (tensor > KL_LM_HEAD && tensor <= KL_BV && !(h->desc.flags & KL_FLAG_QKV_BIAS)) return KL_ERR_INVALID_ARG;   // this model has no biases
+    if (tensor == KL_WROUTER && !p.n_experts) return KL_ERR_INVALID_ARG;   // this model has no router
     if (global_t ? (layer != -1) : (layer < 0 || layer >= (int)p.L)) return KL_ERR_INVALID_ARG;
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(h->weights);
     const size_t lo = global_t ? 0 : (size_t)layer * y.layer_stride;
@@ -1125,14 +1174,36 @@ kl_status kl_load_weights(kl_handle* h, int tensor, int layer, const void* src, 
         case KL_BQ: rows = 1; cols = p.QD; dst = lo + y.off_bqkv; break;
         case KL_BK: rows = 1; cols = p.KVD; dst = lo + y.off_bqkv + p.QD; break;
         case KL_BV: rows = 1; cols = p.KVD; dst = lo + y.off_bqkv + p.QD + p.KVD; break;
+        case KL_WROUTER: rows = p.n_experts; cols = p.H; dst = lo + y.off_router; break;
         default: return KL_ERR_INVALID_ARG;
     }
+    if (p.n_experts && (tensor == KL_WGATE || tensor == KL_WUP || tensor == KL_WDOWN)) return KL_ERR_INVALID_ARG;   // per expert
     if (bytes != rows * cols * 2) return KL_ERR_INVALID_ARG;
     cudaError_t e;
     if (pl) e = store_rows(*pl, w + dst, reinterpret_cast<const __nv_bfloat16*>(src), rows, v0, vstep, as_stream(stream));
     else e = cudaMemcpyAsync(w + dst, src, bytes, cudaMemcpyDefault, as_stream(stream));
     if (e != cudaSuccess) return KL_ERR_CUDA;
     h->loaded[(size_t)tensor * p.L + (global_t ? 0 : layer)] = 1;
+    return KL_OK;
+}
+
+kl_status kl_load_expert_weights(kl_handle* h, int tensor, int layer, int expert, const void* src, size_t bytes, void* stream) {
+    if (!h || !src) return KL_ERR_INVALID_ARG;
+    const Params& p = h->prm;
+    if (!p.n_experts || expert < 0 || expert >= (int)p.n_experts || layer < 0 || layer >= (int)p.L) return KL_ERR_INVALID_ARG;
+    if (tensor != KL_WGATE && tensor != KL_WUP && tensor != KL_WDOWN) return KL_ERR_INVALID_ARG;
+    const Layout y = make_layout(h->desc, h->num_sms);
+    __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(h->weights);
+    const size_t lo = (size_t)layer * y.layer_stride + (size_t)expert * y.expert_stride;
+    const bool down = tensor == KL_WDOWN;
+    const size_t rows = down ? p.H : p.F, cols = down ? p.F : p.H;
+    if (bytes != rows * cols * 2) return KL_ERR_INVALID_ARG;
+    const cudaError_t e = down ? store_rows(p.plan[PL_D], w + lo + y.off_d, reinterpret_cast<const __nv_bfloat16*>(src), rows, 0, 1, as_stream(stream))
+                               : store_rows(p.plan[PL_GU], w + lo + y.off_gu, reinterpret_cast<const __nv_bfloat16*>(src), rows,
+                                            tensor == KL_WUP ? 1u : 0u, 2, as_stream(stream));
+    if (e != cudaSuccess) return KL_ERR_CUDA;
+    const int kind = tensor == KL_WGATE ? 0 : tensor == KL_WUP ? 1 : 2;
+    h->loaded[((size_t)(KL_WROUTER + 1) + (size_t)kind * p.n_experts + (size_t)expert) * p.L + (size_t)layer] = 1;
     return KL_OK;
 }
 
@@ -1156,12 +1227,17 @@ static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d,
 
 static bool all_loaded(const kl_handle* h) {
     const uint32_t L = h->prm.L;
-    const int last = (h->desc.flags & KL_FLAG_QKV_BIAS) ? KL_BV : KL_LM_HEAD;
-    for (int t = 0; t <= last; ++t) {
+    const uint32_t E = h->prm.n_experts;
+    for (int t = 0; t <= KL_WROUTER; ++t) {
+        if (t > KL_LM_HEAD && t <= KL_BV && !(h->desc.flags & KL_FLAG_QKV_BIAS)) continue;
+        if (t == KL_WROUTER && !E) continue;
+        if (E && (t == KL_WGATE || t == KL_WUP || t == KL_WDOWN)) continue;   // loaded per expert, checked below
         const bool global_t = (t == KL_EMBED || t == KL_NORM_F || t == KL_LM_HEAD);
         for (uint32_t l = 0; l < (global_t ? 1u : L); ++l)
             if (!h->loaded[(size_t)t * L + l]) return false;
     }
+    for (size_t i = 0; i < (size_t)3 * E * L; ++i)
+        if (!h->loaded[(size_t)(KL_WROUTER + 1) * L + i]) return false;
     return true;
 }
 
@@ -1438,7 +1514,9 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
         uint32_t sbeg = 0, send = 5;
         // the instantiation with the trace stamps compiled in only while a trace buffer is set
-        const void* decoder_fn = (p.trace != nullptr || p.jitter_seed != 0u) ? (const void*)kl_decoder_kernel<true> : (const void*)kl_decoder_kernel<false>;
+        const void* decoder_fn = p.n_experts ? (const void*)kl_decoder_kernel<false, true>
+                                 : (p.trace != nullptr || p.jitter_seed != 0u) ? (const void*)kl_decoder_kernel<true, false>
+                                                                                : (const void*)kl_decoder_kernel<false, false>;
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1, &sbeg, &send};
@@ -1451,8 +1529,10 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
             }
         } else {
             for (uint32_t l = 0; l < p.L; ++l)
-                for (uint32_t sg = 0; sg < 5; ++sg) {
-                    uint32_t l0 = l, l1 = l + 1, s0 = sg, s1 = sg + 1;
+                for (uint32_t sg = 0; sg < (p.n_experts ? 4u : 5u); ++sg) {
+                    // mixture of experts: the down projection needs the router's choice, which lives in the launch
+                    // that made it -- gate/up and down stay together
+                    uint32_t l0 = l, l1 = l + 1, s0 = sg, s1 = (p.n_experts && sg == 3) ? 5u : sg + 1;
                     void* args[] = {&p, &l0, &l1, &s0, &s1};
                     if ((rc = launch_persistent(h, decoder_fn, args, st)) != KL_OK) return rc;
                 }
@@ -1568,7 +1648,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     if (prc != KL_OK) return prc;
     TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, nullptr, 1u, p.rope_cs};
     void* args[] = {&p, &t};
-    const kl_status rc = launch_persistent(h, p.jitter_seed ? (const void*)kl_token_kernel<true> : (const void*)kl_token_kernel<false>, args, st);
+    const kl_status rc = launch_persistent(h, p.n_experts ? (const void*)kl_token_kernel<false, true> : p.jitter_seed ? (const void*)kl_token_kernel<true, false> : (const void*)kl_token_kernel<false, false>, args, st);
     if (rc != KL_OK) return rc;
     h->last_batch = 1;
     h->hidden_is_copy = 1;
@@ -1602,7 +1682,7 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
         ++h->launches;
         TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, out_tokens_d + done, K, h->plan_rope};
         void* args[] = {&p, &t};
-        const kl_status rc = launch_persistent(h, p.jitter_seed ? (const void*)kl_token_kernel<true> : (const void*)kl_token_kernel<false>, args, st);
+        const kl_status rc = launch_persistent(h, p.n_experts ? (const void*)kl_token_kernel<false, true> : p.jitter_seed ? (const void*)kl_token_kernel<true, false> : (const void*)kl_token_kernel<false, false>, args, st);
         if (rc != KL_OK) return rc;
         h->last_batch = 1;
         h->hidden_is_copy = 1;

@@ -33,6 +33,8 @@ constexpr int UNIT_SLOTS = 8;             // in-flight multi-chunk units tracked
 constexpr int MAX_RPC_SPLIT = 4;           // rows per unit when units are split into column pieces
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
 constexpr int MAX_G = 8;                   // query heads per KV head
+constexpr int MAX_EXPERTS = 16;            // experts of a mixture-of-experts layer
+constexpr int MAX_TOP_K = 4;               // experts per token
 constexpr int SMEM_MISC_BYTES = 7168;  // barriers, reduction scratch, unit table, step context (see SmemT); a multiple of 1024
 
 enum StageId { ST_QKV = 0, ST_ATTN = 1, ST_O = 2, ST_GU = 3, ST_D = 4, ST_LM = 5 };
@@ -55,6 +57,8 @@ struct GemvPlan {
     uint32_t kp;
     uint32_t npieces;
     uint32_t nunits;
+    uint32_t nseg;      // mixture-of-experts down projection: the chosen experts' matrices side by side, K columns and
+                        // npieces pieces EACH (1 everywhere else)
 };
 #ifndef KL_MAX_KP
 #define KL_MAX_KP 1536
@@ -79,6 +83,11 @@ struct Params {
     uint64_t wait_ns;
     uint64_t layer_stride; // elements between consecutive layers of any per-layer tensor
     const __nv_bfloat16* bqkv;   // biases of the q, k, v projections [L][QD + 2 KVD] (layer_stride apart), or null
+    // mixture-of-experts layers (n_experts > 0): wgu / wd point at expert 0 of layer 0, the experts of a layer lie
+    // expert_stride elements apart; wrouter [L][n_experts][H] (layer_stride apart)
+    uint32_t n_experts, top_k;
+    uint64_t expert_stride;
+    const __nv_bfloat16* wrouter;
     GemvPlan plan[PL_COUNT];
     const __nv_bfloat16 *wqkv, *wo, *wgu, *wd, *g1, *g2, *gf, *wlm, *embed;
     __nv_bfloat16* kv;
@@ -272,9 +281,17 @@ __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 
 //                                                            or the attention workspace
 // TR selects the instantiation with the trace stamps compiled in (kl_set_trace); the production kernels carry none.
 extern __shared__ __align__(1024) uint8_t kl_smem[];
-template <bool TR>
+// What the router of a mixture-of-experts layer chose, for the producer thread and the consumer warps of this CTA.
+struct MoeSel {
+    volatile uint32_t seq;          // layers routed so far in this launch (written last)
+    uint32_t e[MAX_TOP_K];          // the chosen experts, in descending order of their logits
+    float w[MAX_TOP_K];             // and their gate weights
+};
+template <bool TR, bool MOE = false>
 struct SmemT {
     static constexpr bool kTrace = TR;
+    static constexpr bool kMoe = MOE;
+    __device__ __forceinline__ static MoeSel* moe() { return reinterpret_cast<MoeSel*>(kl_smem + 6240); }
     __device__ __forceinline__ static uint64_t* full() { return reinterpret_cast<uint64_t*>(kl_smem); }
     __device__ __forceinline__ static uint64_t* empty() { return reinterpret_cast<uint64_t*>(kl_smem + 256); }
     __device__ __forceinline__ static float* red() { return reinterpret_cast<float*>(kl_smem + 1536); }
@@ -368,19 +385,27 @@ struct ChunkGeom {
     uint32_t kofs;      // first column
     uint32_t klen;      // columns (row pitch inside the slot = klen * 2 bytes)
 };
+template <bool MOE = false>
 __device__ __forceinline__ ChunkGeom chunk_geom(const GemvPlan& pl, uint32_t u0, uint32_t i) {
     ChunkGeom g;
-    if (pl.npieces == 1) {
+    const uint32_t tp = MOE ? pl.npieces * pl.nseg : pl.npieces;
+    if (tp == 1) {
         g.unit = u0 + i;
         g.piece = 0;
     } else {
-        g.unit = u0 + i / pl.npieces;
-        g.piece = i % pl.npieces;
+        g.unit = u0 + i / tp;
+        g.piece = i % tp;
     }
     g.row = g.unit * pl.rpc;
     g.nrows = min(pl.rpc, pl.R - g.row);
-    g.kofs = g.piece * pl.kp;
-    g.klen = min(pl.kp, pl.K - g.kofs);
+    if (MOE && pl.nseg > 1) {   // piece j of segment sg: columns sg * K + j * kp ... of the concatenated input vector
+        const uint32_t sg = g.piece / pl.npieces, j = g.piece % pl.npieces;
+        g.kofs = sg * pl.K + j * pl.kp;
+        g.klen = min(pl.kp, pl.K - j * pl.kp);
+    } else {
+        g.kofs = g.piece * pl.kp;
+        g.klen = min(pl.kp, pl.K - g.kofs);
+    }
     return g;
 }
 
@@ -622,12 +647,17 @@ __device__ __forceinline__ void produce_decoder(const Params& p, const SM& s, ui
                                                 uint32_t sbeg, uint32_t send) {
     RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
     const AttnUnit u = attn_unit(p, cta, (uint32_t)p.positions[p.b0]);
+    uint32_t routed = 0, ex[MAX_TOP_K] = {0u, 0u, 0u, 0u};   // mixture of experts: layers routed so far, the chosen experts
     for (uint32_t l = l0; l < l1 && !r.aborted; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         for (uint32_t st = sbeg; st < send; ++st) {
             if (st == ST_QKV) produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
             else if (st == ST_ATTN) produce_attention(p, s, r, u, l);
             else if (st == ST_O) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+            else if (SM::kMoe) {
+                if (st == ST_GU && !moe_wait_route(p, s, ++routed, ex)) r.aborted = true;   // the experts of this layer are known now
+                if (!r.aborted) produce_matrix_moe(p, s, r, p.plan[st == ST_GU ? PL_GU : PL_D], (st == ST_GU ? p.wgu : p.wd) + lo, cta, ex, st != ST_GU);
+            }
             else if (st == ST_GU) produce_matrix(p, s, r, p.plan[PL_GU], p.wgu + lo, cta);
             else produce_matrix(p, s, r, p.plan[PL_D], p.wd + lo, cta);
         }
@@ -975,16 +1005,129 @@ __device__ __forceinline__ bool unit_combine(const SM& s, const GemvPlan& pl, co
     for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) part[g.piece * MAX_RPC_SPLIT + rr] = y[rr];
     __threadfence_block();
     const int old = atomicAdd(&s.unit_cnt()[us], 1);
-    if (old != (int)pl.npieces - 1) return false;
+    const uint32_t tp = SM::kMoe ? pl.npieces * pl.nseg : pl.npieces;
+    if (old != (int)tp - 1) return false;
     __threadfence_block();
     s.unit_cnt()[us] = 0;
 #pragma unroll
     for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] = 0.f;
-    for (uint32_t j = 0; j < pl.npieces; ++j) {
+    for (uint32_t j = 0; j < tp; ++j) {
 #pragma unroll
         for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) y[rr] += part[j * MAX_RPC_SPLIT + rr];
     }
     return true;
+}
+
+// Router of a mixture-of-experts layer, computed by EVERY CTA for itself from the normalised hidden state in the vector
+// area (g2 * x; xscale is RMSNorm's normaliser): logits r_e = xscale * W_r[e] . vec, the top_k largest in descending
+// order (the lower index first among equals), their softmax as gate weights.  The result goes to shared memory for the
+// consumer warps (gate weights) and the producer thread, which cannot request an expert's tiles before it knows which
+// expert it is -- the one place where the weight stream of the looped kernel depends on an activation.
+template <class SM>
+__device__ __noinline__ void moe_router(const Params& p, const SM& s, uint32_t layer, float xscale, uint32_t ctid) {
+    const uint32_t warp = ctid >> 5, lane = ctid & 31u, E = p.n_experts;
+    float* logits = s.unit_part();   // the unit table is idle between the stages
+    const __nv_bfloat16* wr = p.wrouter + (size_t)layer * p.layer_stride;
+    const float4* v4 = reinterpret_cast<const float4*>(s.vec(p)) + lane;
+    for (uint32_t e = warp; e < E; e += NCW) {
+        const uint8_t* row = reinterpret_cast<const uint8_t*>(wr + (size_t)e * p.H) + (size_t)lane * 16;
+        float acc = 0.f;
+        for (uint32_t b = 0; b * 256u < p.H; ++b) {
+            if (b * 256u + lane * 8u < p.H) {   // H is a multiple of 8
+                const uint4 q = __ldg(reinterpret_cast<const uint4*>(row + (size_t)b * 512));
+                const float4 lo = v4[b * 64], hi = v4[b * 64 + 32];
+                acc = fmaf(bf_lo(q.x), lo.x, acc); acc = fmaf(bf_hi(q.x), lo.y, acc);
+                acc = fmaf(bf_lo(q.y), lo.z, acc); acc = fmaf(bf_hi(q.y), lo.w, acc);
+                acc = fmaf(bf_lo(q.z), hi.x, acc); acc = fmaf(bf_hi(q.z), hi.y, acc);
+                acc = fmaf(bf_lo(q.w), hi.z, acc); acc = fmaf(bf_hi(q.w), hi.w, acc);
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) logits[e] = acc * xscale;
+    }
+    consumer_bar();
+    if (ctid == 0) {
+        MoeSel* m = s.moe();
+        uint32_t taken = 0u;
+        float top[MAX_TOP_K];
+        for (uint32_t k = 0; k < p.top_k; ++k) {
+            uint32_t best = 0xffffffffu;
+            for (uint32_t e = 0; e < E; ++e)
+                if (!((taken >> e) & 1u) && (best == 0xffffffffu || logits[e] > logits[best])) best = e;
+            taken |= 1u << best;
+            m->e[k] = best;
+            top[k] = logits[best];
+        }
+        float sum = 0.f;
+        const float mx = top[0];   // chosen in descending order: the first is the maximum
+        for (uint32_t k = 0; k < p.top_k; ++k) {
+            top[k] = expf(top[k] - mx);
+            sum += top[k];
+        }
+        for (uint32_t k = 0; k < p.top_k; ++k) m->w[k] = top[k] / sum;
+        __threadfence_block();
+        m->seq = m->seq + 1u;   // the producer thread waits for this
+    }
+    consumer_bar();
+}
+
+// Producer side of a mixture-of-experts layer: waits (bounded) until the consumers have routed the n-th layer of the
+// launch, then streams this CTA's share of the chosen experts' gate/up matrices and down matrices.
+template <class SM>
+__device__ __forceinline__ bool moe_wait_route(const Params& p, const SM& s, uint32_t n, uint32_t (&ex)[MAX_TOP_K]) {
+    const MoeSel* m = s.moe();
+    if (m->seq < n) {
+        const uint64_t t0 = globaltimer_ns();
+        uint32_t it = 0;
+        while (m->seq < n) {
+            if ((++it & 63u) == 0) {
+                if (*s.abort_flag()) return false;
+                if (globaltimer_ns() - t0 > p.wait_ns) {
+                    raise_abort(p, s, ERR_SYNC_TIMEOUT, 800);
+                    return false;
+                }
+            }
+        }
+    }
+    __threadfence_block();
+    for (uint32_t k = 0; k < (uint32_t)MAX_TOP_K; ++k) ex[k] = k < p.top_k ? m->e[k] : 0u;
+    return true;
+}
+// gate/up: the chosen experts' row units one expert after the other (unit u of the stage = unit u % nunits of chosen
+// expert u / nunits); down: every row unit has the pieces of all chosen experts, expert after expert.
+template <class SM>
+__device__ __forceinline__ void produce_matrix_moe(const Params& p, const SM& s, RingProd& r, const GemvPlan& pl,
+                                                   const __nv_bfloat16* base, uint32_t cta, const uint32_t (&ex)[MAX_TOP_K], bool down) {
+    const uint32_t k = p.top_k;
+    const uint32_t last_len = pl.K - (pl.npieces - 1) * pl.kp;
+    if (!down) {
+        GemvPlan all = pl;
+        all.nunits = pl.nunits * k;
+        const CtaRange cr = cta_units(all, cta, p.P);
+        for (uint32_t u = cr.u0; u < cr.u1; ++u) {
+            const uint32_t sl = u / pl.nunits, ue = u - sl * pl.nunits;
+            const uint8_t* ptr = reinterpret_cast<const uint8_t*>(base + (size_t)ex[sl] * p.expert_stride) + (size_t)ue * pl.rpc * pl.K * 2u;
+            const uint32_t rows = min(pl.rpc, pl.R - ue * pl.rpc);
+            for (uint32_t j = 0; j < pl.npieces; ++j) {
+                const uint32_t bytes = rows * ((j == pl.npieces - 1) ? last_len : pl.kp) * 2u;
+                prod_issue(p, s, r, ptr, bytes, nullptr, 0u, 0u);
+                ptr += bytes;
+            }
+        }
+    } else {
+        const CtaRange cr = cta_units(pl, cta, p.P);
+        for (uint32_t u = cr.u0; u < cr.u1; ++u) {
+            const uint32_t rows = min(pl.rpc, pl.R - u * pl.rpc);
+            for (uint32_t sl = 0; sl < k; ++sl) {
+                const uint8_t* ptr = reinterpret_cast<const uint8_t*>(base + (size_t)ex[sl] * p.expert_stride) + (size_t)u * pl.rpc * pl.K * 2u;
+                for (uint32_t j = 0; j < pl.npieces; ++j) {
+                    const uint32_t bytes = rows * ((j == pl.npieces - 1) ? last_len : pl.kp) * 2u;
+                    prod_issue(p, s, r, ptr, bytes, nullptr, 0u, 0u);
+                    ptr += bytes;
+                }
+            }
+        }
+    }
 }
 
 template <class SM>
@@ -993,14 +1136,17 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
                                         const float* xsrc, float xscale) {
     // xsrc == nullptr: the input vector is staged in s.vec(p); otherwise it is read from global memory per piece
     const CtaRange r = cta_units(pl, cta, p.P);
-    const uint32_t nch = (r.u1 - r.u0) * pl.npieces;
+    const uint32_t tp = SM::kMoe ? pl.npieces * pl.nseg : pl.npieces;   // chunks per unit
+    const uint32_t nch = (r.u1 - r.u0) * tp;
     const uint32_t first = rc.first_chunk(warp, p.nslots);
     XRegs x;
     uint32_t x_piece = 0xffffffffu;
     // rows that come whole and find their vector in shared memory are multiplied against it block by block
     const bool smemx = xsrc == nullptr && pl.rpc <= (uint32_t)MAX_RPC_SPLIT;
     for (uint32_t i = first; i < nch; i += p.nslots) {
-        const ChunkGeom g = chunk_geom(pl, r.u0, i);
+        const ChunkGeom g = chunk_geom<SM::kMoe>(pl, r.u0, i);
+        // mixture of experts: the gate weight of the expert whose (gate, up) rows these are goes into the SwiGLU output
+        const float gw = (SM::kMoe && ep == EP_SWIGLU) ? s.moe()->w[g.row / (2u * p.F)] : 1.f;
         if (!smemx && g.piece != x_piece) {  // same piece on every turn when the piece count divides the consumer count
             if (xsrc) load_xregs_global(x, xsrc, g.kofs, g.klen, lane);
             else load_xregs(x, s.vec(p), g.kofs, g.klen, lane);
@@ -1045,11 +1191,11 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
                 y[2] = warp_sum(y[2]);
                 y[3] = warp_sum(y[3]);
             }
-            if (pl.npieces > 1) {
+            if (tp > 1) {
                 if (lane == 0 && unit_combine(s, pl, g, r.u0, y)) {
                     if (ep == EP_SWIGLU) {
-                        emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
-                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
+                        emit_value(out, g.row >> 1, gw * silu(y[0] * xscale) * (y[1] * xscale));
+                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, gw * silu(y[2] * xscale) * (y[3] * xscale));
                     } else {
 #pragma unroll
                         for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
@@ -1058,8 +1204,8 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
                     }
                 }
             } else if (ep == EP_SWIGLU) {
-                if (lane == 0) emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
-                if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
+                if (lane == 0) emit_value(out, g.row >> 1, gw * silu(y[0] * xscale) * (y[1] * xscale));
+                if (lane == 1 && g.nrows == 4) emit_value(out, (g.row >> 1) + 1, gw * silu(y[2] * xscale) * (y[3] * xscale));
             } else if (lane < g.nrows) {
                 // lane rr emits row rr (every lane holds all sums after the butterfly)
                 const float v = lane == 0 ? y[0] : lane == 1 ? y[1] : lane == 2 ? y[2] : y[3];
@@ -1101,11 +1247,11 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
             for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr) rs[rr] = __shfl_sync(0xffffffffu, res, rr);
             if (lane == 0) {
                 bool emit = true;
-                if (pl.npieces > 1) emit = unit_combine(s, pl, g, r.u0, y);
+                if (tp > 1) emit = unit_combine(s, pl, g, r.u0, y);
                 if (emit) {
                     if (ep == EP_SWIGLU) {
-                        emit_value(out, g.row >> 1, silu(y[0] * xscale) * (y[1] * xscale));
-                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, silu(y[2] * xscale) * (y[3] * xscale));
+                        emit_value(out, g.row >> 1, gw * silu(y[0] * xscale) * (y[1] * xscale));
+                        if (g.nrows == 4) emit_value(out, (g.row >> 1) + 1, gw * silu(y[2] * xscale) * (y[3] * xscale));
                     } else {
 #pragma unroll
                         for (int rr = 0; rr < MAX_RPC_SPLIT; ++rr)
@@ -1145,7 +1291,7 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
                         emit_value(out, row, rs0 + y0 * xscale);
                         if (two) emit_value(out, row + 1, rs1 + y1 * xscale);
                     } else {
-                        emit_value(out, row >> 1, silu(y0 * xscale) * (y1 * xscale));
+                        emit_value(out, row >> 1, gw * silu(y0 * xscale) * (y1 * xscale));
                     }
                 }
             }

@@ -37,3 +37,11 @@ def test_llama31_70b_all_layers():
     device and, for the oracle, layer by layer on the host), batch 1, context 4096."""
     worst = helpers.run_full_depth(gen.LLAMA31_70B, context=4096, steps=2)
     print("config 5, 80 layers:", worst)
+
+
+def test_mixtral_8x7b_shape_all_layers():
+    """The mixture-of-experts decoder at full depth: 32 layers of 8 experts (93 GB of weights on the device, one layer at
+    a time on the host), batch 1, context 4096; 64 routing decisions per step have to agree with the oracle's."""
+    shape = gen.ModelShape(32, 4096, 32, 8, 128, 14336, 32000, 1e-5, 1000000.0, False, 8, 2)
+    worst = helpers.run_full_depth(shape, context=4096, steps=2)
+    print("mixture of experts, 32 layers:", worst)

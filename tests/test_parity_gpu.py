@@ -963,3 +963,54 @@ def test_sync_protocol_under_seeded_jitter(name, steps):
         assert torch.equal(got[1], want[1]) and torch.equal(got[2], want[2]), (kind, seed)
     dec.kl_debug_set_jitter(0, 0)
     dec.close()
+
+
+MOE_SHAPES = {
+    # the tiny decoder with four experts, two per token
+    "tiny_4x2": gen.ModelShape(4, 256, 4, 2, 64, 512, 1024, 1e-5, 10000.0, False, 4, 2),
+    # eight experts, two per token, FFN wider than a ring slot (the down projection in column pieces per expert), G = 4, head size 128
+    "hd128_8x2_split_down": gen.ModelShape(2, 512, 8, 2, 128, 3072, 1000, 1e-5, 500000.0, False, 8, 2),
+    # one expert per token, three experts, row counts that are no multiples of the CTA count
+    "odd_3x1": gen.ModelShape(3, 328, 8, 2, 128, 1008, 1544, 1e-5, 500000.0, False, 3, 1),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MOE_SHAPES))
+def test_mixture_of_experts_decoder(name):
+    """Decoders whose MLP is a mixture of experts (the paper's Table 2 lists one): router, top-k, gate weights and the
+    gathered expert MLPs run inside the looped kernel -- the expert tiles are the one part of the weight stream whose
+    addresses depend on an activation.  All three schedules against the oracle for several steps (the router must pick
+    the oracle's experts or the logits would be far off), bit-identical to each other; then the one-launch-per-token
+    chain and a multi-token launch pick the same tokens; a batch decodes sequence after sequence."""
+    shape = MOE_SHAPES[name]
+    rep = helpers.run_parity(shape, context=150, steps=6, seed=2)
+    helpers.assert_parity(rep, 6)
+    want = [r["next"][0] for r in rep["ref"]]
+    dec = helpers.make_decoder(shape, 1, 170, 2)
+    for kind in ("greedy", "tokens"):
+        cache = gen.make_kv_cache(shape, 1, 150, 170, 2, "cuda")
+        tok = gen.make_tokens(shape, 1, 2).cuda()
+        pos = torch.tensor([150], dtype=torch.int32, device="cuda")
+        logits = torch.empty(1, shape.vocab, device="cuda")
+        out = torch.empty(6, dtype=torch.int32, device="cuda")
+        if kind == "tokens":
+            dec.kl_decode_greedy_tokens(tok, pos, cache, logits, out, 6, 1, True)
+        else:
+            for i in range(6):
+                dec.kl_decode_greedy(tok, pos, cache, logits, 1, i == 0)
+                out[i] = tok[0]
+        torch.cuda.synchronize()
+        assert dec.kl_last_status() == binding.KL_OK
+        assert out.tolist() == want, kind
+    dec.close()
+    rep = helpers.run_parity(shape, context=150, steps=2, seed=2, batch=3, positions0=[5, 64, 150], modes=(binding.KL_MODE_LOOPED,))
+    helpers.assert_parity(rep, 2, batch=3)
+
+
+def test_mixtral_8x7b_shape_two_layers():
+    """The mixture-of-experts decoder of the paper's Table 2 by its public dimensions (hidden 4096, 32 / 8 heads of 128,
+    8 experts of FFN 14336 with 2 per token: per expert the down projection in ten column pieces, twenty per row unit),
+    two layers, context 1024, three steps, all schedules."""
+    shape = gen.ModelShape(2, 4096, 32, 8, 128, 14336, 32000, 1e-5, 1000000.0, False, 8, 2)
+    rep = helpers.run_parity(shape, context=1024, steps=3, seed=0, max_ctx=1024 + 8, check_cache=False)
+    helpers.assert_parity(rep, 3, check_cache=False)
