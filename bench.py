@@ -590,11 +590,13 @@ def run_ours(args, shape, batch, context):
         "roofline": {"bound": "hbm", "kernel": "kl_token_kernel (all layers + classifier + sampling, one launch per step)",
                      "achieved": bytes_step / (ms_token / K * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": bytes_step / (ms_token / K * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": (ncu_traffic(shape, batch, context) + NCU_DRAM_BYTES_CLASSIFIER_V128256_H4096
+                     "traffic": (ncu_traffic(shape, batch, context) + NCU_DRAM_BYTES_CLASSIFIER_STAGE_V128256_H4096
                                  if ncu_traffic(shape, batch, context) and (shape.vocab, shape.hidden) == (128256, 4096) else None),
-                     "traffic_source": "ncu dram bytes of the decoder layers (4-layer capture scaled by layers/4) + of the classifier "
-                                       "stage (profiles/kl_decoder_kernel_llama31_8b_4layers_b1_ctx4096.txt, "
-                                       "profiles/kl_classifier_kernel_llama31_8b_vocab128256.txt)",
+                     "traffic_source": "ncu dram bytes read+written of a 4-layer kl_token_kernel launch: its decoder layers (the "
+                                       "4-layer kl_decoder_kernel capture) scaled by layers/4, its classifier and sampling stages "
+                                       "(the difference of the two captures) once "
+                                       "(profiles/kl_token_kernel_llama31_8b_4layers_b1_ctx4096.txt, "
+                                       "profiles/kl_decoder_kernel_llama31_8b_4layers_b1_ctx4096.txt)",
                      "bytes_per_launch": bytes_step, "ms_per_launch": ms_token / K},
         "looped_four_launches": {"value": tokens / (ms_looped * 1e-3), "ms_per_step": ms_looped / K,
                                  "launches_per_step": int(launches) // K},
@@ -772,15 +774,16 @@ def run_ours_batched(args, shape, batch, context):
 # dram__bytes_read.sum + dram__bytes_write.sum of one looped launch over 4 layers of the 8B shape at batch 1,
 # context 4096 (ncu capture summarised under profiles/), per layer.  Every layer streams its own weights and KV once,
 # so a full launch is this times the layer count.
-NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813534e9 + 15.228672e6) / 4
+NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813368e9 + 18.063104e6) / 4
 
 
 # the same for the ten launches of one layer of the batched path at batch 32, context 4096
-NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1002.2e6
+NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1001.8e6
 
 
-# dram bytes of the classifier kernel at vocabulary 128256, hidden 4096 (ncu capture summarised under profiles/)
-NCU_DRAM_BYTES_CLASSIFIER_V128256_H4096 = 1.050799e9 + 5.4e6
+# dram bytes of the classifier and sampling stages of kl_token_kernel at vocabulary 128256, hidden 4096: a 4-layer
+# kl_token_kernel launch minus a 4-layer kl_decoder_kernel launch (both captures summarised under profiles/)
+NCU_DRAM_BYTES_CLASSIFIER_STAGE_V128256_H4096 = (2.864128e9 + 21.771008e6) - (1.813368e9 + 18.063104e6)
 
 
 def ncu_traffic(shape, batch, context):
