@@ -181,7 +181,8 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
  * step k.  logits_d holds the last step's logits.
  * For batch 1 the loop over the decoder layers (Section 3.3) is extended to a loop over TOKENS: one launch of the
  * persistent kernel decodes up to 256 consecutive tokens (longer runs are cut into launches of 256), with a small
- * launch before it that lays out what changes from token to token (position, step number of the tags, rotary table).
+ * launch before it that writes the rotary tables of the tokens' positions (position and step number advance inside the
+ * kernel).
  * Inside the launch the CTA that finishes a token's sampling writes the next embedding while every other CTA already
  * holds the next token's first weight tiles: neither a launch boundary nor a pipeline restart between tokens.
  * The launch needs position + n_tokens <= max_ctx (checked on the device before anything is decoded: otherwise the
