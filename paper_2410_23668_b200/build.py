@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libkl.so"
 SOURCES = [CSRC / "kl.cu"]
-HEADERS = [CSRC / "kl_device.cuh", CSRC / "kl_attention_tc.cuh", CSRC / "kl_batched.cuh", PKG.parent / "include" / "kl.h"]
+HEADERS = [CSRC / "kl_device.cuh", CSRC / "kl_attention_tc.cuh", CSRC / "kl_batched.cuh", CSRC / "kl_bloop.cuh", PKG.parent / "include" / "kl.h"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

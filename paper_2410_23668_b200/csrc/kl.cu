@@ -111,18 +111,49 @@ __device__ __forceinline__ bool cta_begin(const Params& p, const SM& s, uint32_t
         s.ctx()->step = ld_step(p.step_dev);
         s.ctx()->pos = (uint32_t)p.positions[p.b0];
         s.ctx()->rope_cs = rope;
+        s.ctx()->wait_ns = p.wait_ns;
+        s.ctx()->status = p.status;
         if constexpr (SM::kMoe) s.moe()->seq = 0u;
         for (uint32_t i = 0; i < p.nslots * p.nsw; ++i) {
             mbar_init(smem_u32(&s.full()[i]), 1);
-            mbar_init(smem_u32(&s.empty()[i]), 1);
+            mbar_init(smem_u32(&s.empty()[i]), SM::kTmem ? 2 : 1);   // stash mode: the stash thread and the slot's reader
+        }
+        if constexpr (SM::kTmem) {
+            for (uint32_t i = 0; i < 2u * T_NREG; ++i) {
+                mbar_init(smem_u32(&s.tfull()[i]), 1);
+                mbar_init(smem_u32(&s.tfree()[i]), 4);   // the four warps of the team
+            }
+            for (uint32_t i = 0; i < 2u * T_NSP; ++i) mbar_init(smem_u32(&s.kvready()[i]), 1);
+            mbar_init(smem_u32(&s.tdone()[0]), 1);
+            mbar_init(smem_u32(&s.tdone()[1]), 1);
         }
         *s.abort_flag() = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (tid < UNIT_SLOTS) s.unit_cnt()[tid] = 0;
-    __syncthreads();
-    return *p.status == 0;
+    if constexpr (SM::kTmem) {
+        if (tid < 2u * T_USLOTS) s.t_ucnt()[tid] = 0;
+    }
+    if (__syncthreads_or(*p.status != 0)) return false;   // the same answer in every thread
+    if constexpr (SM::kTmem) {
+        // all of tensor memory (one CTA per SM; the tensor-core kernels of the batched path never overlap this one)
+        if ((tid >> 5) == (uint32_t)SM::NCW + 1u) tm_alloc(smem_u32(s.tbase()), 512u);
+        tm_fence_before();
+        __syncthreads();
+        tm_fence_after();
+    }
+    return true;
+}
+// ... and ends with in stash mode: every warp has left its loop; the warp that allocated tensor memory releases it.
+template <class SM>
+__device__ __forceinline__ void cta_end(const SM& s, uint32_t tid) {
+    if constexpr (SM::kTmem) {
+        tm_fence_before();
+        __syncthreads();
+        tm_fence_after();
+        if ((tid >> 5) == (uint32_t)SM::NCW + 1u) tm_dealloc(*s.tbase(), 512u);
+    }
 }
 
 // ONE stage of one layer on the consumer warps -- the only copy of the stage sequence; every persistent kernel calls
@@ -135,7 +166,7 @@ __device__ __forceinline__ bool cta_begin(const Params& p, const SM& s, uint32_t
 template <class SM>
 __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t l, uint32_t st,
                                           uint32_t xa_slot, uint32_t ctr_target, uint32_t cta, uint32_t ctid, uint32_t warp,
-                                          uint32_t lane, RingCursor& rc, WarpRing& wr) {
+                                          uint32_t lane, RingCursor& rc, WarpRing& wr, TCur& tc) {
     const StepCtx& cx = *s.ctx();
     stage_jitter(p, s, cta, cx.step, l, st);
     const size_t lo = (size_t)l * p.layer_stride;
@@ -162,7 +193,22 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
     } else if (st == ST_ATTN) {
         trace_stamp(p, s, cta, l, 2, ctid);
         // RoPE, split-K attention, merge.  Each unit polls the q (k, v) rows it needs.
-        attention_block(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
+        if constexpr (SM::kTmem) {
+            // chunks so far in this warp's pipeline: behind the head of W_o where that has been streamed ahead
+            uint32_t c0 = tc.c;
+            if (tc.ohead) {
+                const CtaRange co = cta_units(p.plan[PL_O], cta, p.P);
+                c0 += t_count(tc.uc, t_o_head(p.plan[PL_O], co.u1 - co.u0), warp >> 2) * p.plan[PL_O].npieces;
+            }
+            RingCursor ac = {c0, tc.kv};
+            attention_block(p, s, cx, l, cta, ctid, warp, lane, ac, wr);
+            const uint32_t nring = attn_unit(p, cta, cx.pos).nring;
+            const uint32_t first = 2u * (((warp & 3u) - c0) & 3u) + (warp >> 2);   // as in attention_stage
+            if (first < nring) tc.kv += (nring - first + 7u) >> 3;
+            tc.c += (nring + ((warp >> 2) == 0u ? 1u : 0u)) >> 1;
+        } else {
+            attention_block(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
+        }
         trace_stamp(p, s, cta, l, 4, ctid);
         return;
     } else if (st == ST_O) {
@@ -191,6 +237,7 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
         plan = PL_D;
         ep = EP_RESIDUAL;
         xsrc = p.h;
+        if constexpr (SM::kTmem) load_plain_vec(p, s, p.h, p.F, ctid);   // stash mode multiplies against shared memory
     }
     if constexpr (SM::kMoe) {
         if (st == ST_GU || st == ST_D) {
@@ -207,11 +254,13 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
         } else {
             gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
         }
+    } else if constexpr (SM::kTmem) {
+        gemv_stage_t(p, s, p.plan[plan], ep, out, cta, warp, lane, tc, xscale);
     } else {
         gemv_stage(p, s, p.plan[plan], ep, out, cta, warp, lane, rc, wr, xsrc, xscale);
     }
     if (st == ST_GU) {
-        stage_signal(p.counters + l, ctid, skip == ST_GU);
+        stage_signal<SM>(p.counters + l, ctid, skip == ST_GU);
         trace_stamp(p, s, cta, l, 10, ctid);
     } else if (st == ST_D) {
         trace_stamp(p, s, cta, l, 13, ctid);
@@ -221,35 +270,43 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
 // stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
 // boundary after every operator group).
-template <bool TR, bool MOE>
+template <bool TR, bool MOE, bool TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
                                                                  uint32_t sbeg, uint32_t send) {
-    const SmemT<TR, MOE> s;
+    using SM = SmemT<TR, MOE, TM>;
+    const SM s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;   // an earlier kernel of this step flagged bad input: the step is a no-op
-    if (warp == NCW) {
-        // producer warp: one thread streams the CTA's chunk sequence into the ring
-        if (lane == 0) produce_decoder(p, s, cta, l0, l1, sbeg, send);
-        return;
+    if (warp >= (uint32_t)SM::NCW) {
+        // producer warp: one thread streams the CTA's chunk sequence into the ring (stash mode: two more warps, one
+        // thread each, move the chunks on into tensor memory)
+        if (lane == 0) produce_decoder(p, s, cta, l0, l1, sbeg, send, warp - SM::NCW);
+    } else {
+        WarpRing wr = ring_begin();
+        RingCursor rc = {0u, 0u};
+        TCur tc = {0u, 0u, 0u, 0u, (sbeg <= ST_ATTN && send > ST_O) ? 1u : 0u, 0u};
+        for (uint32_t l = l0; l < l1; ++l)
+            for (uint32_t st = sbeg; st < send; ++st) run_stage(p, s, l, st, TG_XA, p.P, cta, tid, warp, lane, rc, wr, tc);
     }
-    WarpRing wr = ring_begin();
-    RingCursor rc = {0u, 0u};
-    for (uint32_t l = l0; l < l1; ++l)
-        for (uint32_t st = sbeg; st < send; ++st) run_stage(p, s, l, st, TG_XA, p.P, cta, tid, warp, lane, rc, wr);
+    cta_end(s, tid);
 }
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
+template <bool TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid_constant__ Params p) {
-    const SmemT<false> s;
+    using SM = SmemT<false, false, TM>;
+    const SM s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;
-    if (warp == NCW) {
-        if (lane == 0) produce_classifier(p, s, cta);
-        return;
+    if (warp >= (uint32_t)SM::NCW) {
+        if (lane == 0) produce_classifier(p, s, cta, warp - SM::NCW);
+    } else {
+        WarpRing wr = ring_begin();
+        RingCursor rc = {0u, 0u};
+        TCur tc = {0u, 0u, 0u, 0u, 0u, 0u};
+        run_stage(p, s, p.L, ST_QKV, TG_XA, p.P, cta, tid, warp, lane, rc, wr, tc);
     }
-    WarpRing wr = ring_begin();
-    RingCursor rc = {0u, 0u};
-    run_stage(p, s, p.L, ST_QKV, TG_XA, p.P, cta, tid, warp, lane, rc, wr);
+    cta_end(s, tid);
 }
 
 // Sampling block (greedy): lowest index among the maxima; then advance the position.  ARGMAX_BLOCKS CTAs per
@@ -353,16 +410,21 @@ __global__ void kl_token_plan_kernel(const __grid_constant__ Params p, float* ro
 }
 
 template <class SM>
-__device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uint32_t cta, const TokenParams& t) {
-    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+__device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uint32_t cta, const TokenParams& t, uint32_t role = 0u) {
+    RingProd r = ring_prod_begin(role);
     const uint32_t step0 = ld_step(p.step_dev), pos0 = (uint32_t)p.positions[0];
     uint32_t routed = 0, ex[MAX_TOP_K] = {0u, 0u, 0u, 0u};   // mixture of experts: layers routed so far, the chosen experts
+    uint32_t ohead = 0u;   // stash mode: the head of W_o goes ahead of the K/V chunks
+    if constexpr (SM::kTmem) {
+        const CtaRange co = cta_units(p.plan[PL_O], cta, p.P);
+        ohead = t_o_head(p.plan[PL_O], co.u1 - co.u0);
+    }
     for (uint32_t k = 0; k < t.K && !r.aborted; ++k) {
         const AttnUnit u = attn_unit(p, cta, pos0 + k);
         for (uint32_t l = 0; l < p.L && !r.aborted; ++l) {
             const size_t lo = (size_t)l * p.layer_stride;
             produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
-            if (k > 0 && l == 0) {
+            if (k > 0 && l == 0 && role == 0u) {
                 // The cache rows of the previous token are read by this token's copies: none is requested before the
                 // previous token is complete in every CTA, which the first word of this token's embedding says (it
                 // keeps its tag until the first down projection of this token, which cannot start before this point
@@ -379,8 +441,9 @@ __device__ __forceinline__ void produce_tokens(const Params& p, const SM& s, uin
                 asm volatile("fence.proxy.async;" ::: "memory");
                 if (r.aborted) break;
             }
+            if (ohead) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta, 0u, ohead);
             produce_attention(p, s, r, u, l);
-            produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+            produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta, ohead);
             if constexpr (SM::kMoe) {
                 if (!moe_wait_route(p, s, ++routed, ex)) r.aborted = true;   // the experts of this layer are known now
                 if (!r.aborted) produce_matrix_moe(p, s, r, p.plan[PL_GU], p.wgu + lo, cta, ex, false);
@@ -408,31 +471,31 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
     // ---- greedy sampling: this CTA's rows first
     const GemvPlan& plm = p.plan[PL_LM];
     asm volatile("fence.proxy.async;" ::: "memory");   // the cache rows this thread appended: readable by later bulk copies
-    consumer_bar();   // the rows this CTA stored are visible to all of its threads
+    consumer_bar<SM>();   // the rows this CTA stored are visible to all of its threads
     float* sv = s.unit_part();                                           // [NCW] maxima, then [NCW] indices, then flags
-    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part()) + NCW;
+    uint32_t* si = reinterpret_cast<uint32_t*>(s.unit_part()) + SM::NCW;
     // [0] this CTA drew the last ticket, [1] token, [2] position, [3] next step number, [4] stop: a wait of this launch gave up
-    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part()) + 2 * NCW;
+    volatile uint32_t* sh = reinterpret_cast<volatile uint32_t*>(s.unit_part()) + 2 * SM::NCW;
     const CtaRange cr = cta_units(plm, cta, p.P);
     const uint32_t r0 = cr.u0 * plm.rpc, r1 = min(cr.u1 * plm.rpc, p.V);
     float bv = -INFINITY;
     uint32_t bi = 0xffffffffu;
-    for (uint32_t i = r0 + ctid; i < r1; i += NCT) argmax_merge(bv, bi, p.logits[i], i);
+    for (uint32_t i = r0 + ctid; i < r1; i += SM::NCT) argmax_merge(bv, bi, p.logits[i], i);
     for (int o = 16; o > 0; o >>= 1)
         argmax_merge(bv, bi, __shfl_xor_sync(0xffffffffu, bv, o), __shfl_xor_sync(0xffffffffu, bi, o));
     if (lane == 0) {
         sv[warp] = bv;
         si[warp] = bi;
     }
-    consumer_bar();
+    consumer_bar<SM>();
     if (ctid == 0) {
-        for (uint32_t w = 1; w < (uint32_t)NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
+        for (uint32_t w = 1; w < (uint32_t)SM::NCW; ++w) argmax_merge(bv, bi, sv[w], si[w]);
         t.part_val[cta] = bv;
         t.part_idx[cta] = bi;
         sh[0] = (atom_add_acq_rel(t.ticket, 1u) == p.P * (k + 1u) - 1u) ? 1u : 0u;
         sh[4] = (*s.abort_flag() != 0 || __ldcg(p.status) != 0) ? 1u : 0u;
     }
-    consumer_bar();
+    consumer_bar<SM>();
     const bool last_cta = sh[0] != 0u, stop = sh[4] != 0u;
     if (last_cta && stop) {
         if (ctid == 0) *t.ticket = 0u;
@@ -456,22 +519,22 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
                 sh[2] = (uint32_t)pos;
             }
         }
-        consumer_bar();
+        consumer_bar<SM>();
         uint32_t next_step = cx.step + 1u;
         if (final) {   // what the next launch needs: hidden state kept, rotary table, counters at zero, step number
-            for (uint32_t i = ctid; i < p.H; i += NCT) t.hidden[i] = ld_tw(p.xa + i).v;   // before xa is overwritten below
-            for (uint32_t i = ctid; i < p.hd / 2; i += NCT) {
+            for (uint32_t i = ctid; i < p.H; i += SM::NCT) t.hidden[i] = ld_tw(p.xa + i).v;   // before xa is overwritten below
+            for (uint32_t i = ctid; i < p.hd / 2; i += SM::NCT) {
                 double sn, cs;
                 sincos((double)sh[2] * p.inv_freq[i], &sn, &cs);
                 p.rope_cs[2 * i] = (float)cs;
                 p.rope_cs[2 * i + 1] = (float)sn;
             }
-            for (uint32_t i = ctid; i < p.L; i += NCT) p.counters[i] = 0u;
-            consumer_bar();
+            for (uint32_t i = ctid; i < p.L; i += SM::NCT) p.counters[i] = 0u;
+            consumer_bar<SM>();
             if (next_step >= step_wrap(p.L)) {   // every other CTA has left its last stage: the step numbers start over
-                clear_tagged(p, ctid, NCT);
+                clear_tagged(p, ctid, SM::NCT);
                 next_step = 1u;
-                consumer_bar();
+                consumer_bar<SM>();
             }
             if (ctid == 0) *p.step_dev = next_step;
         }
@@ -479,45 +542,48 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
         // the next launch expects the usual tag, the next token of this launch the one of its own
         const uint32_t xtag = tag_from(next_step, p.L, 0, final ? (uint32_t)TG_XA : TG_NEXT);
         __threadfence();   // release side of the token boundary (the producers' poll above is the acquire side)
-        for (uint32_t i = ctid; i < p.H; i += NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
+        for (uint32_t i = ctid; i < p.H; i += SM::NCT) st_tw(p.xa + i, __bfloat162float(row[i]), xtag);
     }
     if (ctid == 0) {   // the next token of the launch: one step and one position further, the next rotary table
         s.ctx()->step = cx.step + 1u;
         s.ctx()->pos = cx.pos + 1u;
         s.ctx()->rope_cs = cx.rope_cs + p.hd;
     }
-    consumer_bar();   // the flags above are read before the next stage reuses the area
+    consumer_bar<SM>();   // the flags above are read before the next stage reuses the area
     return !stop && !final;
 }
 
 // K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
-template <bool TR, bool MOE>
+template <bool TR, bool MOE, bool TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
-    const SmemT<TR, MOE> s;
+    using SM = SmemT<TR, MOE, TM>;
+    const SM s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, t.rope)) return;
-    if (warp == NCW) {
-        if (lane == 0) produce_tokens(p, s, cta, t);
-        return;
-    }
-    WarpRing wr = ring_begin();
-    RingCursor rc = {0u, 0u};
-    uint32_t k = 0, l = 0;
+    if (warp >= (uint32_t)SM::NCW) {
+        if (lane == 0) produce_tokens(p, s, cta, t, warp - SM::NCW);
+    } else {
+        WarpRing wr = ring_begin();
+        RingCursor rc = {0u, 0u};
+        TCur tc = {0u, 0u, 0u, 0u, 1u, 0u};
+        uint32_t k = 0, l = 0;
 #pragma unroll 1
-    for (;;) {
-        const bool cls = l == p.L;
-        for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st)
-            run_stage(p, s, l, st, (k > 0 && l == 0) ? TG_NEXT : (uint32_t)TG_XA, p.P * (k + 1u), cta, tid, warp, lane, rc, wr);
-        if (cls) {
-            if (!sample_token(p, s, t, k, cta, tid, warp, lane)) break;
-            ++k;
-            l = 0;
-        } else {
-            ++l;
+        for (;;) {
+            const bool cls = l == p.L;
+            for (uint32_t st = 0; st < (cls ? 1u : 5u); ++st)
+                run_stage(p, s, l, st, (k > 0 && l == 0) ? TG_NEXT : (uint32_t)TG_XA, p.P * (k + 1u), cta, tid, warp, lane, rc, wr, tc);
+            if (cls) {
+                if (!sample_token(p, s, t, k, cta, tid, warp, lane)) break;
+                ++k;
+                l = 0;
+            } else {
+                ++l;
+            }
         }
     }
+    cta_end(s, tid);
 }
 
 }  // namespace kl
@@ -588,6 +654,7 @@ struct kl_handle {
     uint8_t* loaded;                   // [12][L] flags (host)
     int pending_skip_stage;
     int use_tc_attention;
+    int stash;             // 1: the batch-1 kernels run in stash mode (ring -> TMEM -> registers; plans cut for it)
     void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no link against libcuda)
     // optional event recording around the decoder and classifier launches
     uint32_t prof_capacity;
@@ -784,6 +851,43 @@ bool plans_ok(const Params& p) {
         if (pl.kp > MAX_KP && (i == PL_D || pl.rpc > (uint32_t)MAX_RPC_SPLIT)) return false;
         if (pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES) return false;
         if (pl.npieces > 1 && (pl.rpc > (uint32_t)MAX_RPC_SPLIT || pl.kp % (i == PL_D ? 8 : 256))) return false;
+        if (i == PL_GU && (pl.rpc & 1u)) return false;
+    }
+    return true;
+}
+
+// Plans of the stash mode: pieces of kp columns with kp a multiple of 1024 that divides K (whole rows where two of them,
+// or a (gate, up) pair, fit a slot), chunks of 16 KB at most.  rpc == 0: the matrix cannot be cut this way.
+GemvPlan make_plan_t(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t align) {
+    GemvPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    pl.R = R;
+    pl.K = K;
+    pl.nseg = 1;
+    const uint32_t minrows = pairs ? 2u : 1u;
+    uint32_t kp = 0;
+    const uint32_t cand[2] = {4096u, 2048u};   // the widths the consumer loop is instantiated for
+    for (int i = 0; i < 2 && !kp; ++i)
+        if (K % cand[i] == 0 && cand[i] * 2u * minrows <= (uint32_t)SLOT_BYTES) kp = cand[i];
+    if (!kp) return pl;
+    pl.kp = kp;
+    pl.npieces = K / kp;
+    uint32_t rpc = SLOT_BYTES / (kp * 2u);
+    if (pl.npieces == 1) {   // whole rows: keep at least ~2 chunks per CTA on small matrices
+        uint32_t cap = R / (2 * P);
+        if (cap < minrows) cap = minrows;
+        if (rpc > cap) rpc = cap;
+    }
+    if (pairs) rpc &= ~1u;
+    while (align && rpc > 1 && align % rpc) --rpc;
+    pl.rpc = rpc;
+    pl.nunits = rpc ? ceil_div(R, rpc) : 0;
+    return pl;
+}
+bool plans_ok_t(const Params& p) {
+    for (int i = 0; i < PL_COUNT; ++i) {
+        const GemvPlan& pl = p.plan[i];
+        if (pl.rpc < 1 || pl.rpc * pl.kp * 2 > (uint32_t)SLOT_BYTES || pl.npieces > 32) return false;
         if (i == PL_GU && (pl.rpc & 1u)) return false;
     }
     return true;
@@ -994,12 +1098,31 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.skip_stage = -1;
     p.wait_ns = 2000000000ull;
     p.layer_stride = y.layer_stride;
-    p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD, true);  // KVD divides QD: Wq | Wk | Wv stay aligned
-    p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P, 0, true);
-    p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P, 0, true);
-    p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0, false);
-    p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0, true);
-    if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    // stash mode where the shape allows it (dense layers, the tensor-core attention loop, widths the mode is built for)
+    h->stash = 0;
+    {
+        const char* e = getenv("KL_STASH");
+        if (d.n_experts == 0 && h->use_tc_attention && !(e && e[0] == '0')) {
+            p.plan[PL_QKV] = make_plan_t(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD);
+            p.plan[PL_O] = make_plan_t(p.H, p.QD, false, p.P, 0);
+            p.plan[PL_GU] = make_plan_t(2 * p.F, p.H, true, p.P, 0);
+            p.plan[PL_D] = make_plan_t(p.H, p.F, false, p.P, 0);
+            p.plan[PL_LM] = make_plan_t(p.V, p.H, false, p.P, 0);
+            // the vector area holds the widest input (the down projection's too), the ring is 2 x T_NSP slots
+            const size_t vmax = (size_t)ceil_div(p.F > p.H ? (p.F > p.QD ? p.F : p.QD) : (p.H > p.QD ? p.H : p.QD), 256) * 256;
+            int optin = 0;
+            h->stash = plans_ok_t(p) && cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) == cudaSuccess &&
+                       (size_t)2 * T_NSP * SLOT_BYTES + vmax * 4 + SMEM_MISC_BYTES + 16384 <= (size_t)optin;
+        }
+    }
+    if (!h->stash) {
+        p.plan[PL_QKV] = make_plan(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD, true);  // KVD divides QD: Wq | Wk | Wv stay aligned
+        p.plan[PL_O] = make_plan(p.H, p.QD, false, p.P, 0, true);
+        p.plan[PL_GU] = make_plan(2 * p.F, p.H, true, p.P, 0, true);
+        p.plan[PL_D] = make_plan(p.H, p.F, false, p.P, 0, false);
+        p.plan[PL_LM] = make_plan(p.V, p.H, false, p.P, 0, true);
+        if (!plans_ok(p)) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    }
     p.n_experts = d.n_experts;
     p.top_k = d.top_k;
     p.expert_stride = y.expert_stride;
@@ -1024,6 +1147,15 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     if (cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
         free(h->loaded); delete h; return KL_ERR_CUDA;
     }
+    if (h->stash) {
+        // the down projection multiplies against shared memory too; the ring is two pipelines of T_NSP slots
+        if (p.F > vecf) vecf = ceil_div(p.F, 256) * 256;
+        p.vec_floats = vecf;
+        p.nslots = 2 * T_NSP;
+        p.nsw = 1;
+        h->smem_bytes = (size_t)2 * T_NSP * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
+        if (h->smem_bytes > (size_t)max_optin) { free(h->loaded); delete h; return KL_ERR_UNSUPPORTED_SHAPE; }
+    } else {
     const long avail = (long)max_optin - (long)vecf * 4 - SMEM_MISC_BYTES;
     long nsw = avail / ((long)NCW * SLOT_BYTES);
     if (nsw > MAX_NSW) nsw = MAX_NSW;
@@ -1031,22 +1163,32 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     p.nslots = NCW;
     p.nsw = (uint32_t)nsw;
     h->smem_bytes = (size_t)NCW * nsw * SLOT_BYTES + (size_t)vecf * 4 + SMEM_MISC_BYTES;
+    }
     // The shared-memory limit is an attribute of the kernel, not of a handle: it is raised to the device's opt-in
     // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
-    cudaError_t ce = cudaFuncSetAttribute(kl_decoder_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
-    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
-    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_decoder_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
-    if (ce == cudaSuccess) ce = cudaFuncSetAttribute(kl_classifier_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    cudaError_t ce = cudaSuccess;
+    {
+        const void* fns[] = {(const void*)kl_decoder_kernel<false, false, false>, (const void*)kl_decoder_kernel<true, false, false>,
+                             (const void*)kl_decoder_kernel<false, true, false>, (const void*)kl_decoder_kernel<false, false, true>,
+                             (const void*)kl_decoder_kernel<true, false, true>, (const void*)kl_classifier_kernel<false>,
+                             (const void*)kl_classifier_kernel<true>};
+        for (const void* f : fns)
+            if (ce == cudaSuccess) ce = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
+    }
     {
         int tocc = 0;
-        h->token_ok = cudaFuncSetAttribute(kl_token_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaFuncSetAttribute(kl_token_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaFuncSetAttribute(kl_token_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) == cudaSuccess &&
-                      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+        const void* fns[] = {(const void*)kl_token_kernel<false, false, false>, (const void*)kl_token_kernel<true, false, false>,
+                             (const void*)kl_token_kernel<false, true, false>, (const void*)kl_token_kernel<false, false, true>,
+                             (const void*)kl_token_kernel<true, false, true>};
+        h->token_ok = 1;
+        for (const void* f : fns)
+            if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) != cudaSuccess) h->token_ok = 0;
+        if (h->token_ok)
+            h->token_ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false, false>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
-    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false>, NTHREADS, h->smem_bytes);
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false, false>, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
         fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
                         "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
@@ -1473,6 +1615,14 @@ static kl_status batched_step(kl_handle* h, const int32_t* tokens_d, const int32
     return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
 }
 
+static const void* token_fn(const kl_handle* h) {
+    const Params& p = h->prm;
+    if (p.n_experts) return (const void*)kl_token_kernel<false, true, false>;
+    const bool dbg = p.jitter_seed != 0u || p.trace != nullptr;
+    if (h->stash) return dbg ? (const void*)kl_token_kernel<true, false, true> : (const void*)kl_token_kernel<false, false, true>;
+    return dbg ? (const void*)kl_token_kernel<true, false, false> : (const void*)kl_token_kernel<false, false, false>;
+}
+
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
                          float* logits_d, uint32_t batch, void* stream) {
     if (!h || !tokens_d || !positions_d || !kv_cache_d || !logits_d) return KL_ERR_INVALID_ARG;
@@ -1514,9 +1664,11 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
         uint32_t sbeg = 0, send = 5;
         // the instantiation with the trace stamps compiled in only while a trace buffer is set
-        const void* decoder_fn = p.n_experts ? (const void*)kl_decoder_kernel<false, true>
-                                 : (p.trace != nullptr || p.jitter_seed != 0u) ? (const void*)kl_decoder_kernel<true, false>
-                                                                                : (const void*)kl_decoder_kernel<false, false>;
+        const bool dbg = p.trace != nullptr || p.jitter_seed != 0u;
+        const void* decoder_fn = p.n_experts ? (const void*)kl_decoder_kernel<false, true, false>
+                                 : h->stash ? (dbg ? (const void*)kl_decoder_kernel<true, false, true> : (const void*)kl_decoder_kernel<false, false, true>)
+                                 : dbg      ? (const void*)kl_decoder_kernel<true, false, false>
+                                            : (const void*)kl_decoder_kernel<false, false, false>;
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1, &sbeg, &send};
@@ -1542,7 +1694,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
             Params pc = p;
             pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
             void* cargs[] = {&pc};
-            if ((rc = launch_persistent(h, (const void*)kl_classifier_kernel, cargs, st)) != KL_OK) return rc;
+            if ((rc = launch_persistent(h, h->stash ? (const void*)kl_classifier_kernel<true> : (const void*)kl_classifier_kernel<false>, cargs, st)) != KL_OK) return rc;
         }
         if (ev && b == 0 && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
         if (batch > 1) {
@@ -1612,7 +1764,7 @@ static kl_status token_chain_params(kl_handle* h, Params* out, int32_t* tokens_d
     p.logits = logits_d;
     p.skip_stage = h->pending_skip_stage;   // test hook of the bounded waits: applies to the next launch only
     h->pending_skip_stage = -1;
-    p.trace = nullptr;
+    // the stage stamps of kl_set_trace are taken here too (decoder layers only); the chunk log is not
     p.chunk_trace = nullptr;
     p.attn_tc = 0;
     if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
@@ -1648,7 +1800,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     if (prc != KL_OK) return prc;
     TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, nullptr, 1u, p.rope_cs};
     void* args[] = {&p, &t};
-    const kl_status rc = launch_persistent(h, p.n_experts ? (const void*)kl_token_kernel<false, true> : p.jitter_seed ? (const void*)kl_token_kernel<true, false> : (const void*)kl_token_kernel<false, false>, args, st);
+    const kl_status rc = launch_persistent(h, token_fn(h), args, st);
     if (rc != KL_OK) return rc;
     h->last_batch = 1;
     h->hidden_is_copy = 1;
@@ -1682,7 +1834,7 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
         ++h->launches;
         TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, out_tokens_d + done, K, h->plan_rope};
         void* args[] = {&p, &t};
-        const kl_status rc = launch_persistent(h, p.n_experts ? (const void*)kl_token_kernel<false, true> : p.jitter_seed ? (const void*)kl_token_kernel<true, false> : (const void*)kl_token_kernel<false, false>, args, st);
+        const kl_status rc = launch_persistent(h, token_fn(h), args, st);
         if (rc != KL_OK) return rc;
         h->last_batch = 1;
         h->hidden_is_copy = 1;

@@ -11,6 +11,9 @@
 #ifndef KL_POLL_NS
 #define KL_POLL_NS 64
 #endif
+#ifndef KL_T_OHEAD
+#define KL_T_OHEAD 1   // stash mode: stream the head of W_o ahead of the K/V chunks (see t_o_head)
+#endif
 #ifndef KL_ST_TW
 #define KL_ST_TW "st.relaxed.gpu.global.b64"
 #endif
@@ -33,6 +36,10 @@ constexpr int UNIT_SLOTS = 8;             // in-flight multi-chunk units tracked
 constexpr int MAX_RPC_SPLIT = 4;           // rows per unit when units are split into column pieces
 constexpr int MIN_POS_PER_CHUNK = 64;      // attention: fewest cached positions worth a CTA
 constexpr int MAX_G = 8;                   // query heads per KV head
+constexpr int T_NCW = 8;                   // stash mode: consumer warps (two teams of four, one per TMEM lane quarter)
+constexpr int T_NSP = 4;                   // stash mode: ring slots per pipeline (two pipelines, one per team)
+constexpr int T_NREG = 8;                  // stash mode: TMEM regions (16 KB, 32 columns) per pipeline
+constexpr int T_USLOTS = 16;               // stash mode: units of a team whose quarter sums may be in flight
 constexpr int MAX_EXPERTS = 16;            // experts of a mixture-of-experts layer
 constexpr int MAX_TOP_K = 4;               // experts per token
 constexpr int SMEM_MISC_BYTES = 7168;  // barriers, reduction scratch, unit table, step context (see SmemT); a multiple of 1024
@@ -115,6 +122,8 @@ struct StepCtx {
     uint32_t step;
     uint32_t pos;
     const float* rope_cs;
+    uint64_t wait_ns;    // copies of the launch's wait limit and status word, for code that runs as a call
+    int32_t* status;
 };
 
 
@@ -155,7 +164,7 @@ __device__ __forceinline__ void stage_jitter(const Params& p, const SM&, uint32_
 template <class SM>
 __device__ __forceinline__ void trace_stamp(const Params& p, const SM&, uint32_t cta, uint32_t layer, int k, uint32_t ctid) {
     if constexpr (SM::kTrace)
-        if (p.trace != nullptr && ctid == 0) p.trace[((size_t)cta * p.L + layer) * TRACE_STAMPS + k] = globaltimer_ns();
+        if (p.trace != nullptr && ctid == 0 && layer < p.L) p.trace[((size_t)cta * p.L + layer) * TRACE_STAMPS + k] = globaltimer_ns();
 }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -216,6 +225,54 @@ __device__ __forceinline__ uint4 ldg_stream16(const void* p) {
 // tag it expects has the value -- no fence on the writer's side, no counter to poll, one L2 round trip on the
 // reader's side.  Tags are odd numbers built from (decode step, layer, stage), so a word left over from an earlier
 // layer or step never matches, and neither does zero-initialised memory.
+// ---- stash mode: tensor memory as a second stage of the weight ring (tcgen05.cp from shared memory, tcgen05.ld into
+// registers).  One allocation of all 512 columns per CTA, made and released by one warp.
+__device__ __forceinline__ void tm_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tm_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tm_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tm_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tm_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 128 lanes x 32 bytes: lane r takes the two 16-byte granules at start + 16 r and start + 16 r + 2048 (descriptor
+// without swizzle: 16 bytes between consecutive rows of a group of eight, 128 bytes between groups, 2048 bytes
+// between the two granules of a row), i.e. a linear run of 4 KB lands as granule (r + 128 k) in lane r, columns 4 k .. 4 k + 3
+__device__ __forceinline__ void tm_cp_4k(uint32_t taddr, uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(2048u >> 4) << 16;
+    d |= (uint64_t)(128u >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(d) : "memory");
+}
+__device__ __forceinline__ void tm_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, "
+        "%25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tm_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tm_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 struct __align__(8) TW {
     float v;
     uint32_t tag;
@@ -264,10 +321,21 @@ __device__ __forceinline__ StepCtx step_ctx(const Params& p) {
     return cx;
 }
 
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(NCT) : "memory"); }
+template <class SM>
+__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(SM::NCT) : "memory"); }
 
 __device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
 __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+// d0 += a0 * b0, d1 += a1 * b1 as ONE instruction (packed fp32 multiply-add of sm_100): the even and the odd columns
+// of a weight register are the two halves of the pair, so the multiply-adds of a chunk take half the issue slots.
+__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%0, %1};\n\t"
+        "fma.rn.f32x2 rc, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rc;\n\t}"
+        : "+f"(d0), "+f"(d1)
+        : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
 
 // ------------------------------------------------------------------------------------------------ shared state
 
@@ -287,19 +355,39 @@ struct MoeSel {
     uint32_t e[MAX_TOP_K];          // the chosen experts, in descending order of their logits
     float w[MAX_TOP_K];             // and their gate weights
 };
-template <bool TR, bool MOE = false>
+template <bool TR, bool MOE = false, bool TM = false>
 struct SmemT {
     static constexpr bool kTrace = TR;
     static constexpr bool kMoe = MOE;
+    static constexpr bool kTmem = TM;            // stash mode: weights go ring -> TMEM -> registers (see the stash section)
+    static constexpr int NCW = TM ? T_NCW : kl::NCW;   // consumer warps
+    static constexpr int NCT = NCW * 32;               // consumer threads (they take part in the CTA-wide steps)
     __device__ __forceinline__ static MoeSel* moe() { return reinterpret_cast<MoeSel*>(kl_smem + 6240); }
     __device__ __forceinline__ static uint64_t* full() { return reinterpret_cast<uint64_t*>(kl_smem); }
     __device__ __forceinline__ static uint64_t* empty() { return reinterpret_cast<uint64_t*>(kl_smem + 256); }
+    // stash mode: per TMEM region "copy complete" / "all four warps have read it", the drain barriers of the two stash
+    // threads, the TMEM base address, the arrival counters of the units whose quarter sums meet in unit_part()
+    __device__ __forceinline__ static uint64_t* tfull() { return reinterpret_cast<uint64_t*>(kl_smem + 512); }
+    __device__ __forceinline__ static uint64_t* tfree() { return reinterpret_cast<uint64_t*>(kl_smem + 640); }
+    __device__ __forceinline__ static uint64_t* tdone() { return reinterpret_cast<uint64_t*>(kl_smem + 768); }
+    __device__ __forceinline__ static uint32_t* tbase() { return reinterpret_cast<uint32_t*>(kl_smem + 784); }
+    // stash mode: "the K/V chunk in this slot has landed", signalled by the stash thread, which sees every use of a slot
+    // land in order (a reader that tested the slot's own barrier could be two phases behind: the uses before its chunk
+    // are weight chunks it never waits for)
+    __device__ __forceinline__ static uint64_t* kvready() { return reinterpret_cast<uint64_t*>(kl_smem + 800); }
+    // the barrier a reader of K/V chunks in ring slot `slot` waits on
+    __device__ __forceinline__ static uint64_t* kv_bar(uint32_t slot) { return ((TM && KL_T_OHEAD) ? kvready() : full()) + slot; }
+    __device__ __forceinline__ static int* t_ucnt() { return reinterpret_cast<int*>(kl_smem + 1024); }
     __device__ __forceinline__ static float* red() { return reinterpret_cast<float*>(kl_smem + 1536); }
     __device__ __forceinline__ static float* unit_part() { return reinterpret_cast<float*>(kl_smem + 2048); }
     __device__ __forceinline__ static int* unit_cnt() { return reinterpret_cast<int*>(kl_smem + 6144); }
     __device__ __forceinline__ static volatile int* abort_flag() { return reinterpret_cast<volatile int*>(kl_smem + 6144 + 4 * UNIT_SLOTS); }
     __device__ __forceinline__ static StepCtx* ctx() { return reinterpret_cast<StepCtx*>(kl_smem + 6208); }
     __device__ __forceinline__ static uint8_t* ring() { return kl_smem + SMEM_MISC_BYTES; }
+    // stash mode: the ring is always 2 * T_NSP slots
+    __device__ __forceinline__ static float* vec_t() {
+        return reinterpret_cast<float*>(kl_smem + SMEM_MISC_BYTES + (size_t)2 * T_NSP * SLOT_BYTES);
+    }
     __device__ __forceinline__ static float* vec(const Params& p) {
         return reinterpret_cast<float*>(kl_smem + SMEM_MISC_BYTES + (size_t)p.nslots * p.nsw * SLOT_BYTES);
     }
@@ -377,6 +465,15 @@ __device__ __forceinline__ CtaRange cta_units(const GemvPlan& pl, uint32_t cta, 
     return r;
 }
 
+// Stash mode streams the first units of the output projection BEFORE the K/V chunks of the attention unit: K/V chunks
+// stay in their ring slots until the attention stage reads them, and whatever is queued behind them waits; the head of
+// W_o moves on into tensor memory while the QKV stage still runs, so the copies do not stop there.  At most eight
+// chunks per pipeline -- what its TMEM regions hold -- or the K/V chunks behind them could never be requested.
+__device__ __forceinline__ uint32_t t_o_head(const GemvPlan& pl, uint32_t nu) {
+    if (!KL_T_OHEAD) return 0u;
+    const uint32_t h = 2u * ((uint32_t)T_NREG / pl.npieces);
+    return nu < h ? nu : h;
+}
 struct ChunkGeom {
     uint32_t unit;      // unit index (matrix-wide)
     uint32_t piece;     // column piece
@@ -520,15 +617,101 @@ struct RingProd {
     uint32_t c, k, use, n;   // consumer, slot of that consumer, use count of that slot, chunk index (for the log)
     uint64_t pol;
     bool aborted;
+    // stash mode: the chunk sequence is dealt to two pipelines (team 0 / team 1 of the consumer warps), each with
+    // T_NSP ring slots and T_NREG TMEM regions of its own.  The producer thread and the two stash threads walk the same
+    // sequence: role 0 issues the copies, role 1 + t moves the chunks of pipeline t from the ring into TMEM.
+    uint32_t role, pi;       // role of this thread; pipeline of the next chunk
+    uint32_t uc;             // units of all stages so far (unit k of a stage goes to pipeline (uc + k) & 1)
+    uint32_t tc[2];          // chunks so far per pipeline
+    uint32_t tg;             // stash thread: weight chunks of its pipeline so far
 };
+__device__ __forceinline__ RingProd ring_prod_begin(uint32_t role) {
+    RingProd r;
+    r.c = r.k = r.use = r.n = 0u;
+    r.pol = l2_policy_evict_first();
+    r.aborted = false;
+    r.role = role;
+    r.pi = r.uc = r.tg = 0u;
+    r.tc[0] = r.tc[1] = 0u;
+    return r;
+}
+// Stash mode, the stash thread's part in a chunk of its pipeline.  A weight chunk: wait for the copy, wait for the
+// TMEM region, move the slot's 16 KB into it (four copies of 4 KB), let the completion of the copies signal the region
+// full and the slot empty.  A chunk of K/V rows is read from the ring by a consumer warp: the stash thread only sees it
+// land.  Every slot's barrier completes a phase on two arrivals -- the stash thread's and the reader's (for a weight
+// chunk both are the stash thread's) -- so neither side can fall two phases behind on a parity wait.
+template <class SM>
+__device__ __forceinline__ void stash_chunk(const Params& p, const SM& s, RingProd& r, bool weights) {
+    const uint32_t pi = r.role - 1u, seq = r.tc[0]++;   // a stash thread only counts the chunks of its own pipeline
+    if (r.aborted) return;
+    const uint32_t slot = pi * T_NSP + seq % T_NSP;
+    if (!mbar_wait(p, s, smem_u32(&s.full()[slot]), (seq / T_NSP) & 1u)) {
+        r.aborted = true;
+        return;
+    }
+    const uint32_t ebar = smem_u32(&s.empty()[slot]);
+    if (weights) {
+        const uint32_t g = r.tg++, reg = pi * T_NREG + g % T_NREG;
+        if (g >= (uint32_t)T_NREG && !mbar_wait(p, s, smem_u32(&s.tfree()[reg]), ((g / T_NREG) - 1u) & 1u)) {
+            r.aborted = true;
+            return;
+        }
+        tm_fence_after();
+        const uint32_t src = smem_u32(s.ring()) + slot * SLOT_BYTES, dst = *s.tbase() + reg * 32u;
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) tm_cp_4k(dst + i * 8u, src + i * 4096u);
+        tm_commit(smem_u32(&s.tfull()[reg]));
+        tm_commit(ebar);
+    } else {
+        mbar_arrive(smem_u32(&s.kvready()[slot]));
+    }
+    mbar_arrive(ebar);
+}
+// The stash thread is done: no copy into TMEM may be in flight when the allocation is released.
+template <class SM>
+__device__ __forceinline__ void stash_drain(const Params& p, const SM& s, const RingProd& r) {
+    const uint32_t bar = smem_u32(&s.tdone()[r.role - 1u]);
+    tm_commit(bar);
+    const uint64_t t0 = globaltimer_ns();
+    while (!mbar_try_wait(bar, 0u)) {
+        if (globaltimer_ns() - t0 > p.wait_ns) return;
+    }
+}
+// Slot and use count of the next chunk, and the step to the one after it.
+template <class SM>
+__device__ __forceinline__ void prod_slot(const Params& p, const RingProd& r, uint32_t& slot, uint32_t& use) {
+    if constexpr (SM::kTmem) {
+        slot = r.pi * T_NSP + r.tc[r.pi] % T_NSP;
+        use = r.tc[r.pi] / T_NSP;
+    } else {
+        slot = r.c * p.nsw + r.k;
+        use = r.use;
+    }
+}
+template <class SM>
+__device__ __forceinline__ void prod_advance(const Params& p, RingProd& r) {
+    ++r.n;
+    if constexpr (SM::kTmem) {
+        ++r.tc[r.pi];
+    } else {
+        if (++r.c == p.nslots) {
+            r.c = 0;
+            if (++r.k == p.nsw) {
+                r.k = 0;
+                ++r.use;
+            }
+        }
+    }
+}
 
 // Waits for the slot of the next chunk, arms its barrier and starts one or two linear copies into it.
 template <class SM>
 __device__ __forceinline__ void prod_issue(const Params& p, const SM& s, RingProd& r, const uint8_t* src0, uint32_t bytes0,
                                            const uint8_t* src1, uint32_t bytes1, uint32_t dst1) {
     if (r.aborted) return;
-    const uint32_t slot = r.c * p.nsw + r.k;
-    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (r.use - 1u) & 1u)) {
+    uint32_t slot, use;
+    prod_slot<SM>(p, r, slot, use);
+    if (use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (use - 1u) & 1u)) {
         r.aborted = true;
         return;
     }
@@ -538,14 +721,7 @@ __device__ __forceinline__ void prod_issue(const Params& p, const SM& s, RingPro
     mbar_arrive_expect_tx(bar, bytes0 + bytes1);
     tma_bulk_g2s(dst, src0, bytes0, bar, r.pol);
     if (bytes1) tma_bulk_g2s(dst + dst1, src1, bytes1, bar, r.pol);
-    ++r.n;
-    if (++r.c == p.nslots) {
-        r.c = 0;
-        if (++r.k == p.nsw) {
-            r.k = 0;
-            ++r.use;
-        }
-    }
+    prod_advance<SM>(p, r);
 }
 // Same for a chunk of K/V rows as swizzled boxes of the cache tensor: [pb rows] x [64 columns] per box, K boxes in
 // the first half of the slot, V boxes in the second; a box is always written whole (rows outside the chunk's own
@@ -553,8 +729,9 @@ __device__ __forceinline__ void prod_issue(const Params& p, const SM& s, RingPro
 template <class SM>
 __device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, RingProd& r, int32_t yk, int32_t yv) {
     if (r.aborted) return;
-    const uint32_t slot = r.c * p.nsw + r.k;
-    if (r.use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (r.use - 1u) & 1u)) {
+    uint32_t slot, use;
+    prod_slot<SM>(p, r, slot, use);
+    if (use > 0 && !mbar_wait(p, s, smem_u32(&s.empty()[slot]), (use - 1u) & 1u)) {
         r.aborted = true;
         return;
     }
@@ -567,31 +744,44 @@ __device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, R
         tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yk, bar, r.pol);
         tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yv, bar, r.pol);
     }
-    ++r.n;
-    if (++r.c == p.nslots) {
-        r.c = 0;
-        if (++r.k == p.nsw) {
-            r.k = 0;
-            ++r.use;
-        }
-    }
+    prod_advance<SM>(p, r);
 }
 
 // Streams this CTA's share of one matrix (units [u0, u1) of the plan): one linear run of bytes cut into chunks,
 // per chunk only pointer increments.
 template <class SM>
 __device__ __forceinline__ void produce_matrix(const Params& p, const SM& s, RingProd& r, const GemvPlan& pl,
-                                               const __nv_bfloat16* base, uint32_t cta) {
-    const CtaRange cr = cta_units(pl, cta, p.P);
+                                               const __nv_bfloat16* base, uint32_t cta, uint32_t kb = 0u, uint32_t ke = 0xffffffffu) {
+    // units [kb, ke) of the CTA's share (stash mode streams a matrix in two parts where it pays)
+    CtaRange cr = cta_units(pl, cta, p.P);
+    const uint32_t nu = cr.u1 - cr.u0;
+    const bool last = ke == 0xffffffffu;   // the call that ends the matrix moves the unit count on
+    if (ke > nu) ke = nu;
+    if (kb > ke) kb = ke;
+    if constexpr (SM::kTmem) {
+        if (r.role) {   // stash thread: the chunks of the units of its pipeline, nothing else
+            for (uint32_t k = kb + ((((r.uc + kb) & 1u) == r.role - 1u) ? 0u : 1u); k < ke; k += 2)
+                for (uint32_t j = 0; j < pl.npieces; ++j) stash_chunk(p, s, r, true);
+            if (last) r.uc += nu;
+            return;
+        }
+    }
+    const uint32_t ubase = cr.u0;
+    cr.u1 = cr.u0 + ke;
+    cr.u0 += kb;
     const uint8_t* ptr = reinterpret_cast<const uint8_t*>(base) + (size_t)cr.u0 * pl.rpc * pl.K * 2u;
     const uint32_t last_len = pl.K - (pl.npieces - 1) * pl.kp;
     for (uint32_t u = cr.u0; u < cr.u1; ++u) {
         const uint32_t rows = min(pl.rpc, pl.R - u * pl.rpc);   // only the matrix's last unit can be short
+        if constexpr (SM::kTmem) r.pi = (r.uc + (u - ubase)) & 1u;
         for (uint32_t j = 0; j < pl.npieces; ++j) {
             const uint32_t bytes = rows * ((j == pl.npieces - 1) ? last_len : pl.kp) * 2u;
             prod_issue(p, s, r, ptr, bytes, nullptr, 0u, 0u);
             ptr += bytes;
         }
+    }
+    if constexpr (SM::kTmem) {
+        if (last) r.uc += nu;
     }
 }
 
@@ -600,12 +790,19 @@ template <class SM>
 __device__ __forceinline__ void produce_attention(const Params& p, const SM& s, RingProd& r, const AttnUnit& u,
                                                   uint32_t layer) {
     if (!u.active) return;
+    if constexpr (SM::kTmem) {
+        if (r.role) {   // stash thread: chunk i of the unit belongs to pipeline i & 1
+            for (uint32_t i = r.role - 1u; i < u.nring; i += 2) stash_chunk(p, s, r, false);
+            return;
+        }
+    }
     const uint32_t pb = attn_positions_per_chunk(p);
     if (p.attn_tc) {
         const uint32_t vdelta = p.B * p.nkv * p.max_ctx;
         const uint32_t row0 = layer * 2u * vdelta + (u.b * p.nkv + u.g) * p.max_ctx;
         for (uint32_t i = 0; i < u.nring; ++i) {
             const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
+            if constexpr (SM::kTmem) r.pi = i & 1u;
             prod_issue_boxes(p, s, r, (int32_t)(row0 + w.w0), (int32_t)(row0 + w.w0 + vdelta));
         }
     } else {
@@ -615,6 +812,7 @@ __device__ __forceinline__ void produce_attention(const Params& p, const SM& s, 
         uint32_t left = u.cend - u.c0;
         for (uint32_t i = 0; i < u.nring; ++i) {
             const uint32_t np = left < pb ? left : pb;
+            if constexpr (SM::kTmem) r.pi = i & 1u;
             prod_issue(p, s, r, ks, np * row_bytes, vs, np * row_bytes, SLOT_BYTES / 2);
             ks += np * row_bytes;
             vs += np * row_bytes;
@@ -627,8 +825,26 @@ __device__ __forceinline__ void produce_attention(const Params& p, const SM& s, 
 // for the last copy armed on every slot.
 template <class SM>
 __device__ __forceinline__ void produce_drain(const Params& p, const SM& s, const RingProd& r) {
+    if constexpr (SM::kTmem) {
+        if (r.role) {
+            stash_drain(p, s, r);
+            return;
+        }
+    }
     if (!r.aborted) return;
     const uint64_t t0 = globaltimer_ns();
+    if constexpr (SM::kTmem) {
+        for (uint32_t pi = 0; pi < 2; ++pi)
+            for (uint32_t kk = 0; kk < (uint32_t)T_NSP; ++kk) {
+                const uint32_t cnt = (r.tc[pi] + T_NSP - 1u - kk) / T_NSP;   // uses of this slot so far
+                if (cnt == 0) continue;
+                const uint32_t bar = smem_u32(&s.full()[pi * T_NSP + kk]);
+                while (!mbar_try_wait(bar, (cnt - 1u) & 1u)) {
+                    if (globaltimer_ns() - t0 > p.wait_ns) return;
+                }
+            }
+        return;
+    }
     for (uint32_t cc = 0; cc < p.nslots; ++cc) {
         for (uint32_t kk = 0; kk < p.nsw; ++kk) {
             const uint32_t cnt = r.use + ((kk < r.k || (kk == r.k && cc < r.c)) ? 1u : 0u);  // uses of this slot so far
@@ -644,16 +860,26 @@ __device__ __forceinline__ void produce_drain(const Params& p, const SM& s, cons
 // The producer thread of the decoder kernel: layers [l0, l1).
 template <class SM>
 __device__ __forceinline__ void produce_decoder(const Params& p, const SM& s, uint32_t cta, uint32_t l0, uint32_t l1,
-                                                uint32_t sbeg, uint32_t send) {
-    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+                                                uint32_t sbeg, uint32_t send, uint32_t role = 0u) {
+    RingProd r = ring_prod_begin(role);
     const AttnUnit u = attn_unit(p, cta, (uint32_t)p.positions[p.b0]);
     uint32_t routed = 0, ex[MAX_TOP_K] = {0u, 0u, 0u, 0u};   // mixture of experts: layers routed so far, the chosen experts
+    // stash mode, launches that hold both the attention and the O stage: the head of W_o goes ahead of the K/V chunks
+    uint32_t ohead = 0u;
+    if constexpr (SM::kTmem) {
+        if (sbeg <= ST_ATTN && send > ST_O) {
+            const CtaRange co = cta_units(p.plan[PL_O], cta, p.P);
+            ohead = t_o_head(p.plan[PL_O], co.u1 - co.u0);
+        }
+    }
     for (uint32_t l = l0; l < l1 && !r.aborted; ++l) {
         const size_t lo = (size_t)l * p.layer_stride;
         for (uint32_t st = sbeg; st < send; ++st) {
             if (st == ST_QKV) produce_matrix(p, s, r, p.plan[PL_QKV], p.wqkv + lo, cta);
-            else if (st == ST_ATTN) produce_attention(p, s, r, u, l);
-            else if (st == ST_O) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta);
+            else if (st == ST_ATTN) {
+                if (ohead) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta, 0u, ohead);
+                produce_attention(p, s, r, u, l);
+            } else if (st == ST_O) produce_matrix(p, s, r, p.plan[PL_O], p.wo + lo, cta, ohead);
             else if (SM::kMoe) {
                 if (st == ST_GU && !moe_wait_route(p, s, ++routed, ex)) r.aborted = true;   // the experts of this layer are known now
                 if (!r.aborted) produce_matrix_moe(p, s, r, p.plan[st == ST_GU ? PL_GU : PL_D], (st == ST_GU ? p.wgu : p.wd) + lo, cta, ex, st != ST_GU);
@@ -666,8 +892,8 @@ __device__ __forceinline__ void produce_decoder(const Params& p, const SM& s, ui
 }
 // ... and of the classifier kernel.
 template <class SM>
-__device__ __forceinline__ void produce_classifier(const Params& p, const SM& s, uint32_t cta) {
-    RingProd r = {0u, 0u, 0u, 0u, l2_policy_evict_first(), false};
+__device__ __forceinline__ void produce_classifier(const Params& p, const SM& s, uint32_t cta, uint32_t role = 0u) {
+    RingProd r = ring_prod_begin(role);
     produce_matrix(p, s, r, p.plan[PL_LM], p.wlm, cta);
     produce_drain(p, s, r);
 }
@@ -693,9 +919,9 @@ __device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* s
     constexpr int NB = 4;  // groups of four values kept in flight per thread (two 16-byte loads each)
     // The vector area is about to be overwritten: every warp of the CTA must be done with what the previous stage
     // kept there (the stage's input vector, read block by block until a warp's last chunk; the attention workspace).
-    consumer_bar();
+    consumer_bar<SM>();
     float ss = 0.f;
-    for (uint32_t base = 0; base < n; base += NB * NCT * 4) {
+    for (uint32_t base = 0; base < n; base += NB * SM::NCT * 4) {
         float4 v[NB];
         uint2 gk[NB];
         // Only the groups whose tags are not all in place yet are read again: the words that are late come from the
@@ -704,7 +930,7 @@ __device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* s
         uint32_t pend = 0u;
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
-            const uint32_t e = base + (ctid + i * NCT) * 4;
+            const uint32_t e = base + (ctid + i * SM::NCT) * 4;
             v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
             gk[i] = make_uint2(0x3f803f80u, 0x3f803f80u);   // bf16 ones
             if (e < n) {
@@ -717,7 +943,7 @@ __device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* s
 #pragma unroll
             for (int i = 0; i < NB; ++i) {
                 if ((pend >> i) & 1u) {
-                    const uint32_t e = base + (ctid + i * NCT) * 4;
+                    const uint32_t e = base + (ctid + i * SM::NCT) * 4;
                     const uint4 a = ld_tw2(src + e), b = ld_tw2(src + e + 2);
                     if (a.y == tag && a.w == tag && b.y == tag && b.w == tag) {
                         v[i] = make_float4(__uint_as_float(a.x), __uint_as_float(a.z), __uint_as_float(b.x), __uint_as_float(b.z));
@@ -729,7 +955,7 @@ __device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* s
         }
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
-            const uint32_t e = base + (ctid + i * NCT) * 4;
+            const uint32_t e = base + (ctid + i * SM::NCT) * 4;
             ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
             if (e < n) {
                 // the gains go in now, the normaliser (one number for the whole vector) is applied to the stage's outputs
@@ -749,11 +975,11 @@ __device__ __noinline__ float load_vec(const Params& p, const SM& s, const TW* s
         for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
         if ((ctid & 31) == 0) s.red()[ctid >> 5] = ss;
     }
-    consumer_bar();
+    consumer_bar<SM>();
     if (norm) {
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) tot += s.red()[w];
+        for (int w = 0; w < SM::NCW; ++w) tot += s.red()[w];
         inv = rsqrtf(tot / (float)n + p.eps);
     }
     return inv;
@@ -831,14 +1057,10 @@ __device__ __forceinline__ void dot_rows(const uint8_t* w, uint32_t pitch, uint3
                 const int b = b0 + u < MAX_XB ? b0 + u : MAX_XB - 1;   // blocks past the end hold zero weights
 #pragma unroll
                 for (int r = 0; r < NR; ++r) {
-                    e[r] = fmaf(bf_lo(q[u][r].x), x.v[b][0], e[r]);
-                    o[r] = fmaf(bf_hi(q[u][r].x), x.v[b][1], o[r]);
-                    e[r] = fmaf(bf_lo(q[u][r].y), x.v[b][2], e[r]);
-                    o[r] = fmaf(bf_hi(q[u][r].y), x.v[b][3], o[r]);
-                    e[r] = fmaf(bf_lo(q[u][r].z), x.v[b][4], e[r]);
-                    o[r] = fmaf(bf_hi(q[u][r].z), x.v[b][5], o[r]);
-                    e[r] = fmaf(bf_lo(q[u][r].w), x.v[b][6], e[r]);
-                    o[r] = fmaf(bf_hi(q[u][r].w), x.v[b][7], o[r]);
+                    ffma2(e[r], o[r], bf_lo(q[u][r].x), bf_hi(q[u][r].x), x.v[b][0], x.v[b][1]);
+                    ffma2(e[r], o[r], bf_lo(q[u][r].y), bf_hi(q[u][r].y), x.v[b][2], x.v[b][3]);
+                    ffma2(e[r], o[r], bf_lo(q[u][r].z), bf_hi(q[u][r].z), x.v[b][4], x.v[b][5]);
+                    ffma2(e[r], o[r], bf_lo(q[u][r].w), bf_hi(q[u][r].w), x.v[b][6], x.v[b][7]);
                 }
             }
         }
@@ -862,14 +1084,10 @@ __device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, 
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)b * 512);
-            e[r] = fmaf(bf_lo(q.x), x.v[b][0], e[r]);
-            o[r] = fmaf(bf_hi(q.x), x.v[b][1], o[r]);
-            e[r] = fmaf(bf_lo(q.y), x.v[b][2], e[r]);
-            o[r] = fmaf(bf_hi(q.y), x.v[b][3], o[r]);
-            e[r] = fmaf(bf_lo(q.z), x.v[b][4], e[r]);
-            o[r] = fmaf(bf_hi(q.z), x.v[b][5], o[r]);
-            e[r] = fmaf(bf_lo(q.w), x.v[b][6], e[r]);
-            o[r] = fmaf(bf_hi(q.w), x.v[b][7], o[r]);
+            ffma2(e[r], o[r], bf_lo(q.x), bf_hi(q.x), x.v[b][0], x.v[b][1]);
+            ffma2(e[r], o[r], bf_lo(q.y), bf_hi(q.y), x.v[b][2], x.v[b][3]);
+            ffma2(e[r], o[r], bf_lo(q.z), bf_hi(q.z), x.v[b][4], x.v[b][5]);
+            ffma2(e[r], o[r], bf_lo(q.w), bf_hi(q.w), x.v[b][6], x.v[b][7]);
         }
     }
     if constexpr (NB < MAX_XB) {
@@ -877,14 +1095,10 @@ __device__ __forceinline__ void dot_rows_full(const uint8_t* w, uint32_t pitch, 
 #pragma unroll
             for (int r = 0; r < NR; ++r) {
                 const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)NB * 512);
-                e[r] = fmaf(bf_lo(q.x), x.v[NB][0], e[r]);
-                o[r] = fmaf(bf_hi(q.x), x.v[NB][1], o[r]);
-                e[r] = fmaf(bf_lo(q.y), x.v[NB][2], e[r]);
-                o[r] = fmaf(bf_hi(q.y), x.v[NB][3], o[r]);
-                e[r] = fmaf(bf_lo(q.z), x.v[NB][4], e[r]);
-                o[r] = fmaf(bf_hi(q.z), x.v[NB][5], o[r]);
-                e[r] = fmaf(bf_lo(q.w), x.v[NB][6], e[r]);
-                o[r] = fmaf(bf_hi(q.w), x.v[NB][7], o[r]);
+                ffma2(e[r], o[r], bf_lo(q.x), bf_hi(q.x), x.v[NB][0], x.v[NB][1]);
+                ffma2(e[r], o[r], bf_lo(q.y), bf_hi(q.y), x.v[NB][2], x.v[NB][3]);
+                ffma2(e[r], o[r], bf_lo(q.z), bf_hi(q.z), x.v[NB][4], x.v[NB][5]);
+                ffma2(e[r], o[r], bf_lo(q.w), bf_hi(q.w), x.v[NB][6], x.v[NB][7]);
             }
         }
     }
@@ -920,14 +1134,10 @@ __device__ __forceinline__ void dot_rows_smemx(const uint8_t* w, uint32_t pitch,
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)b * 512);
-            e[r] = fmaf(bf_lo(q.x), lo.x, e[r]);
-            o[r] = fmaf(bf_hi(q.x), lo.y, o[r]);
-            e[r] = fmaf(bf_lo(q.y), lo.z, e[r]);
-            o[r] = fmaf(bf_hi(q.y), lo.w, o[r]);
-            e[r] = fmaf(bf_lo(q.z), hi.x, e[r]);
-            o[r] = fmaf(bf_hi(q.z), hi.y, o[r]);
-            e[r] = fmaf(bf_lo(q.w), hi.z, e[r]);
-            o[r] = fmaf(bf_hi(q.w), hi.w, o[r]);
+            ffma2(e[r], o[r], bf_lo(q.x), bf_hi(q.x), lo.x, lo.y);
+            ffma2(e[r], o[r], bf_lo(q.y), bf_hi(q.y), lo.z, lo.w);
+            ffma2(e[r], o[r], bf_lo(q.z), bf_hi(q.z), hi.x, hi.y);
+            ffma2(e[r], o[r], bf_lo(q.w), bf_hi(q.w), hi.z, hi.w);
         }
     }
     if ((klen & 255u) && nb * 256u + lane * 8u < klen) {   // last, partial block
@@ -935,14 +1145,10 @@ __device__ __forceinline__ void dot_rows_smemx(const uint8_t* w, uint32_t pitch,
 #pragma unroll
         for (int r = 0; r < NR; ++r) {
             const uint4 q = *reinterpret_cast<const uint4*>(wl + (size_t)r * pitch + (size_t)nb * 512);
-            e[r] = fmaf(bf_lo(q.x), lo.x, e[r]);
-            o[r] = fmaf(bf_hi(q.x), lo.y, o[r]);
-            e[r] = fmaf(bf_lo(q.y), lo.z, e[r]);
-            o[r] = fmaf(bf_hi(q.y), lo.w, o[r]);
-            e[r] = fmaf(bf_lo(q.z), hi.x, e[r]);
-            o[r] = fmaf(bf_hi(q.z), hi.y, o[r]);
-            e[r] = fmaf(bf_lo(q.w), hi.z, e[r]);
-            o[r] = fmaf(bf_hi(q.w), hi.w, o[r]);
+            ffma2(e[r], o[r], bf_lo(q.x), bf_hi(q.x), lo.x, lo.y);
+            ffma2(e[r], o[r], bf_lo(q.y), bf_hi(q.y), lo.z, lo.w);
+            ffma2(e[r], o[r], bf_lo(q.z), bf_hi(q.z), hi.x, hi.y);
+            ffma2(e[r], o[r], bf_lo(q.w), bf_hi(q.w), hi.z, hi.w);
         }
     }
 #pragma unroll
@@ -1029,7 +1235,7 @@ __device__ __noinline__ void moe_router(const Params& p, const SM& s, uint32_t l
     float* logits = s.unit_part();   // the unit table is idle between the stages
     const __nv_bfloat16* wr = p.wrouter + (size_t)layer * p.layer_stride;
     const float4* v4 = reinterpret_cast<const float4*>(s.vec(p)) + lane;
-    for (uint32_t e = warp; e < E; e += NCW) {
+    for (uint32_t e = warp; e < E; e += SM::NCW) {
         const uint8_t* row = reinterpret_cast<const uint8_t*>(wr + (size_t)e * p.H) + (size_t)lane * 16;
         float acc = 0.f;
         for (uint32_t b = 0; b * 256u < p.H; ++b) {
@@ -1045,7 +1251,7 @@ __device__ __noinline__ void moe_router(const Params& p, const SM& s, uint32_t l
         acc = warp_sum(acc);
         if (lane == 0) logits[e] = acc * xscale;
     }
-    consumer_bar();
+    consumer_bar<SM>();
     if (ctid == 0) {
         MoeSel* m = s.moe();
         uint32_t taken = 0u;
@@ -1068,7 +1274,7 @@ __device__ __noinline__ void moe_router(const Params& p, const SM& s, uint32_t l
         __threadfence_block();
         m->seq = m->seq + 1u;   // the producer thread waits for this
     }
-    consumer_bar();
+    consumer_bar<SM>();
 }
 
 // Producer side of a mixture-of-experts layer: waits (bounded) until the consumers have routed the n-th layer of the
@@ -1303,9 +1509,322 @@ __device__ __forceinline__ void gemv_stage(const Params& p, const SM& s, const G
     rc.advance(nch, p.nslots);
 }
 
+// ------------------------------------------------------------------------------------------------ stash mode
+// The ring alone holds nslots * 16 KB per SM -- about 3.6 us of HBM time over the whole GPU -- and every exchange between
+// dependent stages that lasts longer stops the weight stream.  Tensor memory is otherwise idle in this kernel: in stash
+// mode each weight chunk is moved on from its ring slot into one of 16 TMEM regions of 16 KB by an asynchronous copy
+// (tcgen05.cp, issued by two stash threads, one per pipeline), which frees the slot for the next bulk copy at once; the
+// consumer warps read the regions into registers (tcgen05.ld).  Ring + TMEM hold 24 chunks = 384 KB per SM.
+//   * A TMEM lane quarter is readable by the warps w with w % 4 == quarter only, and the copy spreads a chunk over all
+//     128 lanes: lane r receives the 16-byte granules r, r + 128, ... of the chunk.  A chunk is therefore multiplied by
+//     a TEAM of four warps (warps 0..3: team 0, warps 4..7: team 1); quarter q holds, of every row, the columns
+//     1024 j + 256 q + 8 lane .. + 7 (j = 0 .. kp / 1024 - 1), which is block 4 j + q, lane `lane` of the staged vector.
+//   * Plans of this mode have kp a multiple of 1024 that divides K, so every row of a chunk meets the same columns.
+//   * All chunks of a unit go to the same team; its four warps add up their quarters over the unit's pieces in registers
+//     and meet in shared memory, where the last warp to arrive adds the quarters in order and emits the rows.
+//   * K/V chunks of the attention units stay in the ring and are read there, as in the plain mode.
+struct TCur {
+    uint32_t uc;   // units of all stages so far
+    uint32_t c;    // chunks so far in this warp's pipeline
+    uint32_t g;    // weight chunks so far in this warp's pipeline
+    uint32_t tu;   // units so far of this warp's team
+    uint32_t ohead;   // 1: the first units of the O projection are streamed ahead of the K/V chunks (see t_o_head)
+    uint32_t kv;      // K/V chunks this warp has read from its ring slot so far
+};
+// how many k in [0, n) have ((uc + k) & 1) == t
+__device__ __forceinline__ uint32_t t_count(uint32_t uc, uint32_t n, uint32_t t) { return (n + (((uc & 1u) == t) ? 1u : 0u)) >> 1; }
+
+// Half a chunk (16 registers = four granules per lane): acc[row][.] += the lane's granules of `row` times its slice of
+// the vector.  NJ granules per row: with NJ = 4 a half is one row, with NJ = 2 two rows (HALF selects rows NR/2 ...).
+template <int NJ, int HALF>
+__device__ __forceinline__ void t_dot(const uint32_t (&w)[16], const float4* v4, uint32_t blk0, uint32_t q, uint32_t lane,
+                                      float (&acc)[8 / NJ][2]) {
+
+    static_assert(NJ == 2 || NJ == 4, "widths the stash mode is built for");
+#pragma unroll
+    for (int jj = 0; jj < NJ; ++jj) {
+        const float4 lo = v4[(blk0 + 4u * jj + q) * 64u + lane], hi = v4[(blk0 + 4u * jj + q) * 64u + 32u + lane];
+#pragma unroll
+        for (int rh = 0; rh < 4 / NJ; ++rh) {
+            const int row = HALF * (4 / NJ) + rh;
+            const int m = (rh * NJ + jj) * 4;
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[m]), bf_hi(w[m]), lo.x, lo.y);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 1]), bf_hi(w[m + 1]), lo.z, lo.w);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 2]), bf_hi(w[m + 2]), hi.x, hi.y);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 3]), bf_hi(w[m + 3]), hi.z, hi.w);
+        }
+    }
+}
+
+// The same with the lane's slice of the vector in registers (whole rows of 4096 columns: blocks q, 4 + q, 8 + q, 12 + q).
+template <int HALF>
+__device__ __forceinline__ void t_dot_xr(const uint32_t (&w)[16], const float (&x)[4][8], float (&acc)[2][2]) {
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+        const int m = jj * 4;
+#ifdef KL_NO_FFMA2
+        acc[HALF][0] = fmaf(bf_lo(w[m]), x[jj][0], acc[HALF][0]);
+        acc[HALF][1] = fmaf(bf_hi(w[m]), x[jj][1], acc[HALF][1]);
+        acc[HALF][0] = fmaf(bf_lo(w[m + 1]), x[jj][2], acc[HALF][0]);
+        acc[HALF][1] = fmaf(bf_hi(w[m + 1]), x[jj][3], acc[HALF][1]);
+        acc[HALF][0] = fmaf(bf_lo(w[m + 2]), x[jj][4], acc[HALF][0]);
+        acc[HALF][1] = fmaf(bf_hi(w[m + 2]), x[jj][5], acc[HALF][1]);
+        acc[HALF][0] = fmaf(bf_lo(w[m + 3]), x[jj][6], acc[HALF][0]);
+        acc[HALF][1] = fmaf(bf_hi(w[m + 3]), x[jj][7], acc[HALF][1]);
+#else
+        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m]), bf_hi(w[m]), x[jj][0], x[jj][1]);
+        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 1]), bf_hi(w[m + 1]), x[jj][2], x[jj][3]);
+        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 2]), bf_hi(w[m + 2]), x[jj][4], x[jj][5]);
+        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 3]), bf_hi(w[m + 3]), x[jj][6], x[jj][7]);
+#endif
+    }
+}
+
+// Sums N values per lane over the 32 lanes with N - 1 + log2(32 / N) shuffles: every step halves the values a lane still
+// carries (the lane keeps the half named by one of its bits and adds the partner's copy of it), then the single value
+// left is summed over the remaining lanes.  Afterwards v[0] of lane l is the total of value (l >> log2(32 / N)) % N --
+// a fixed order of additions, the same in every launch.
+template <int N>
+__device__ __forceinline__ void lanes_reduce(float (&v)[N], uint32_t lane) {
+    int o = 16;
+#pragma unroll
+    for (int n = N; n > 1; n >>= 1, o >>= 1) {
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < n / 2; ++i) {
+            const float send = up ? v[i] : v[i + n / 2], keep = up ? v[i + n / 2] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    for (; o > 0; o >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], o);
+}
+
+// What the stash-mode stage needs, by value: the stage is a real call (its registers are allocated on their own, whatever
+// the calling kernel keeps live), and a callee that reached into the kernel's parameter block would pay a generic load
+// for every field.
+struct TStageArgs {
+    uint32_t R, rpc, kp, tp;      // the plan: rows, rows per unit, columns per chunk, chunks per unit
+    uint32_t u0, nu;              // this CTA's units
+    int ep;
+    GemvOut out;
+    float xscale;
+    uint32_t warp, lane;
+    uint32_t uc, g, tu;           // cursor on entry (see TCur)
+};
+struct TStageRet {
+    uint32_t g, tu;
+};
+// Bounded mbarrier wait of the stash-mode stage: limit and status word come from the CTA's shared-memory record.
+template <class SM>
+__device__ __forceinline__ bool mbar_wait_c(const SM& s, uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*s.abort_flag()) return false;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 63u) == 0) {
+            if (*s.abort_flag()) return false;
+            if (globaltimer_ns() - t0 > s.ctx()->wait_ns) {
+                int32_t* st = s.ctx()->status;
+                if (atomicCAS(st, 0, ERR_SYNC_TIMEOUT) == 0) {
+                    st[1] = 510;
+                    st[2] = (int)blockIdx.x;
+                    st[3] = (int)threadIdx.x;
+                }
+                *s.abort_flag() = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// One GROUP of units of this warp's team: GU = 8 / NR units of one chunk each (WHOLE rows), or one unit of tp chunks.
+// The warp adds up its quarter of every row in registers -- the tensor-memory load of the next half chunk in flight
+// under the multiplications of the current one -- and the group's (up to) eight row sums are reduced over the lanes
+// together; the four quarters meet in shared memory, where the last warp to arrive adds them in quarter order and emits
+// the rows.  Value v of a group is row v % NR of its unit v / NR.
+//   wa: the first half of the group's first chunk, its load already in flight; on return, if `more`, that of the next
+//       group's first chunk (so that the reduction runs under a load, too)
+//   xr: whole rows of 4096 columns keep the lane's slice of the vector in registers
+template <int NJ, bool WHOLE, class SM>
+__device__ __forceinline__ void gemv_group_t(const SM& s, const TStageArgs& a, uint32_t unit0, uint32_t nun, uint32_t T, uint32_t q,
+                                             uint32_t& g, uint32_t tu, uint32_t (&wa)[16], bool more, const float (&xr)[4][8]) {
+    constexpr int NR = 8 / NJ, GU = WHOLE ? 8 / NR : 1;
+    const uint32_t lane = a.lane;
+    const float4* v4 = reinterpret_cast<const float4*>(s.vec_t());
+    const uint32_t tbase = *s.tbase() + ((32u * q) << 16) + T * T_NREG * 32u;
+    const uint32_t bars = smem_u32(&s.tfull()[T * T_NREG]), barf = smem_u32(&s.tfree()[T * T_NREG]);
+    const uint32_t vrow = (unit0 + 2u * (lane / NR)) * a.rpc + lane % NR;   // units of a team are two apart
+    const bool vok = lane < (uint32_t)(GU * NR) && lane / NR < nun && lane % NR < a.rpc && vrow < a.R;
+    float res = 0.f;   // fetched before the waits: the L2 latency hides behind them
+    if (a.ep == EP_RESIDUAL && vok) res = ld_tw(a.out.res + vrow).v;
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = 0.f;
+    float acc[NR][2];
+#pragma unroll
+    for (int rr = 0; rr < NR; ++rr) acc[rr][0] = acc[rr][1] = 0.f;
+    // Half chunks of 16 registers: while one half is multiplied the load of the next one is in flight.
+    uint32_t wb[16];
+    auto fetch0 = [&]() {   // first half of chunk g
+        mbar_wait_c(s, bars + (g % T_NREG) * 8u, (g / T_NREG) & 1u);
+        tm_fence_after();
+        tm_ld16(tbase + (g % T_NREG) * 32u, wa);
+    };
+    auto second = [&]() { tm_ld16(tbase + (g % T_NREG) * 32u + 16u, wb); };
+    auto landed = [&]() {   // both halves of chunk g are in registers: its region may be overwritten
+        tm_fence_before();
+        if (lane == 0) mbar_arrive(barf + (g % T_NREG) * 8u);
+        ++g;
+    };
+    if constexpr (WHOLE) {
+        // whole rows: chunk c is unit c of the group
+#pragma unroll
+        for (int c = 0; c < GU; ++c) {
+            if ((uint32_t)c < nun) {
+                tm_ld_wait();
+                second();
+                if constexpr (NJ == 4) t_dot_xr<0>(wa, xr, acc);
+                else t_dot<NJ, 0>(wa, v4, 0u, q, lane, acc);
+                tm_ld_wait();
+                landed();
+                if ((uint32_t)c + 1u < nun || more) fetch0();
+                if constexpr (NJ == 4) t_dot_xr<1>(wb, xr, acc);
+                else t_dot<NJ, 1>(wb, v4, 0u, q, lane, acc);
+#pragma unroll
+                for (int rr = 0; rr < NR; ++rr) {
+                    y[c * NR + rr] = acc[rr][0] + acc[rr][1];
+                    acc[rr][0] = acc[rr][1] = 0.f;
+                }
+            }
+        }
+    } else {
+        // one unit of tp column pieces
+        for (uint32_t j = 0; j < a.tp; ++j) {
+            const uint32_t blk0 = (j * a.kp) >> 8;
+            tm_ld_wait();
+            second();
+            t_dot<NJ, 0>(wa, v4, blk0, q, lane, acc);
+            tm_ld_wait();
+            landed();
+            if (j + 1u < a.tp || more) fetch0();
+            t_dot<NJ, 1>(wb, v4, blk0, q, lane, acc);
+        }
+#pragma unroll
+        for (int rr = 0; rr < NR; ++rr) y[rr] = acc[rr][0] + acc[rr][1];
+    }
+    lanes_reduce<8>(y, lane);
+    const uint32_t us = T * T_USLOTS + tu % T_USLOTS;
+    volatile float* part = s.unit_part() + us * 32u;
+    if ((lane & 3u) == 0u) part[q * 8u + (lane >> 2)] = y[0];
+    __syncwarp();
+    int old = 0;
+    if (lane == 0) {
+        // release the quarter sums written above (ordered before this by __syncwarp), acquire the other warps'
+        asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;" : "=r"(old) : "r"(smem_u32(&s.t_ucnt()[us])) : "memory");
+    }
+    old = __shfl_sync(0xffffffffu, old, 0);
+    if (old == 3) {
+        if (lane == 0) s.t_ucnt()[us] = 0;
+        if (a.ep == EP_SWIGLU) {
+            // rows come in (gate, up) pairs: values 2 i and 2 i + 1
+            const uint32_t v = 2u * lane;
+            const uint32_t prow = (unit0 + 2u * (v / NR)) * a.rpc + v % NR;
+            if (v < (uint32_t)(GU * NR) && v / NR < nun && v % NR < a.rpc && prow < a.R) {
+                const float ga = part[v] + part[8u + v] + part[16u + v] + part[24u + v];
+                const float up = part[v + 1u] + part[8u + v + 1u] + part[16u + v + 1u] + part[24u + v + 1u];
+                emit_value(a.out, prow >> 1, silu(ga * a.xscale) * (up * a.xscale));
+            }
+        } else if (vok) {
+            const float sum = part[lane] + part[8u + lane] + part[16u + lane] + part[24u + lane];
+            emit_value(a.out, vrow, (a.ep == EP_RESIDUAL ? res : 0.f) + sum * a.xscale);
+        }
+    }
+}
+
+// The units of this warp's team in one stage (see the stash section above).
+template <int NJ, class SM>
+__device__ __noinline__ TStageRet gemv_units_t(const TStageArgs a) {
+    const SM s;
+    constexpr int NR = 8 / NJ, GU = 8 / NR;
+    const uint32_t T = a.warp >> 2, q = a.warp & 3u, lane = a.lane;
+    const uint32_t mine = t_count(a.uc, a.nu, T);
+    const uint32_t k0 = ((a.uc & 1u) == T) ? 0u : 1u;
+    uint32_t g = a.g, tu = a.tu;
+    uint32_t wa[16];
+    if (mine) {   // first half of the warp's first chunk of the stage
+        mbar_wait_c(s, smem_u32(&s.tfull()[T * T_NREG + g % T_NREG]), (g / T_NREG) & 1u);
+        tm_fence_after();
+        tm_ld16(*s.tbase() + ((32u * q) << 16) + (T * T_NREG + g % T_NREG) * 32u, wa);
+    }
+    float xr[4][8];
+    if (NJ == 4 && a.tp == 1) {
+        const float4* v4 = reinterpret_cast<const float4*>(s.vec_t());
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const float4 lo = v4[(4u * jj + q) * 64u + lane], hi = v4[(4u * jj + q) * 64u + 32u + lane];
+            xr[jj][0] = lo.x; xr[jj][1] = lo.y; xr[jj][2] = lo.z; xr[jj][3] = lo.w;
+            xr[jj][4] = hi.x; xr[jj][5] = hi.y; xr[jj][6] = hi.z; xr[jj][7] = hi.w;
+        }
+    }
+    if (a.tp == 1) {
+        for (uint32_t m = 0; m < mine; m += GU, ++tu)
+            gemv_group_t<NJ, true>(s, a, a.u0 + k0 + 2u * m, min((uint32_t)GU, mine - m), T, q, g, tu, wa, m + GU < mine, xr);
+    } else {
+        for (uint32_t m = 0; m < mine; ++m, ++tu)
+            gemv_group_t<NJ, false>(s, a, a.u0 + k0 + 2u * m, 1u, T, q, g, tu, wa, m + 1u < mine, xr);
+    }
+    TStageRet r;
+    r.g = g;
+    r.tu = tu;
+    return r;
+}
+
+// Consumes this CTA's share of one matrix in stash mode: y = W vec and the stage's epilogue (see gemv_stage).  The input
+// vector is staged in the vector area in the lane-permuted layout.
+template <class SM>
+__device__ __forceinline__ void gemv_stage_t(const Params& p, const SM& s, const GemvPlan& pl, int ep, const GemvOut& out,
+                                             uint32_t cta, uint32_t warp, uint32_t lane, TCur& tc, float xscale) {
+    const CtaRange r = cta_units(pl, cta, p.P);
+    TStageArgs a;
+    a.R = pl.R; a.rpc = pl.rpc; a.kp = pl.kp; a.tp = pl.npieces;
+    a.u0 = r.u0; a.nu = r.u1 - r.u0;
+    a.ep = ep; a.out = out; a.xscale = xscale;
+    a.warp = warp; a.lane = lane;
+    a.uc = tc.uc; a.g = tc.g; a.tu = tc.tu;
+    const TStageRet ret = pl.kp == 4096u ? gemv_units_t<4, SM>(a) : gemv_units_t<2, SM>(a);
+    const uint32_t mine = t_count(tc.uc, a.nu, warp >> 2);
+    tc.uc += a.nu;
+    tc.c += mine * a.tp;
+    tc.g = ret.g;
+    tc.tu = ret.tu;
+}
+
+// Stages a plain fp32 vector written by other CTAs (guarded by a counter the caller has waited on) in the vector area.
+template <class SM>
+__device__ __forceinline__ void load_plain_vec(const Params& p, const SM& s, const float* src, uint32_t n, uint32_t ctid) {
+    constexpr int NB = 7;
+    for (uint32_t base = 0; base < n; base += NB * SM::NCT * 4) {
+        float4 v[NB];
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            const uint32_t e = base + (ctid + i * SM::NCT) * 4;
+            if (e < n) v[i] = __ldcg(reinterpret_cast<const float4*>(src + e));
+        }
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+            const uint32_t e = base + (ctid + i * SM::NCT) * 4;
+            if (e < n) *reinterpret_cast<float4*>(s.vec(p) + vec_perm(e)) = v[i];
+        }
+    }
+    consumer_bar<SM>();
+}
+
 // End of a stage: all consumer warps have written their outputs; one thread publishes the CTA's arrival.
+template <class SM>
 __device__ __forceinline__ void stage_signal(uint32_t* ctr, uint32_t ctid, bool skip) {
-    consumer_bar();
+    consumer_bar<SM>();
     if (ctid == 0 && !skip) red_release_add(ctr, 1u);  // release: cumulative over the CTA barrier above
 }
 
@@ -1332,7 +1851,7 @@ __device__ __forceinline__ void stage_wait(const Params& p, const SM& s, const u
             }
         }
     }
-    consumer_bar();
+    consumer_bar<SM>();
 }
 
 // ------------------------------------------------------------------------------------------------ attention
@@ -1436,7 +1955,7 @@ __device__ __forceinline__ void attn_chunks_tc(const Params& p, const SM& s, con
     const uint32_t box_bytes = pb * 128u;
     for (uint32_t i = first; i < u.nring; i += p.nslots) {
         const uint32_t slot = warp * p.nsw + wr.cslot;
-        mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+        mbar_wait(p, s, smem_u32(s.kv_bar(slot)), wr.cphase);
         if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
         ring_advance_consume(p, wr);
         const uint32_t kbase = smem_u32(s.ring()) + slot * SLOT_BYTES;
@@ -1514,12 +2033,12 @@ __device__ __noinline__ void attn_merge(const Params& p, const SM& s, const Step
     const uint32_t t_lo = min(total, u.ch * S), t_hi = min(total, t_lo + S);
     const uint32_t ns = t_hi - t_lo;
     // the tables sit behind the per-warp partials, which other threads of the CTA may still be reading
-    float* wtab = comb + (size_t)NCW * G * (hd + 2);   // [2][G][nchunk]: maxima, sums; then weights in the first half
+    float* wtab = comb + (size_t)SM::NCW * G * (hd + 2);   // [2][G][nchunk]: maxima, sums; then weights in the first half
     float* pv = wtab + 2 * G * nchunk;                 // [ns][nchunk] partial outputs of this unit's slice
     // all loads of a thread are issued before it waits on any of them; only those that are late are repeated
     constexpr int NL = 2;
     const uint32_t nml = G * nchunk, npv = ns * nchunk;
-    for (uint32_t i0 = 0; i0 < max(nml, (npv + NL - 1) / NL); i0 += NCT) {
+    for (uint32_t i0 = 0; i0 < max(nml, (npv + NL - 1) / NL); i0 += SM::NCT) {
         const uint32_t i = i0 + ctid;
         bool ml_pend = i < nml;
         uint32_t pend = 0u;
@@ -1553,9 +2072,9 @@ __device__ __noinline__ void attn_merge(const Params& p, const SM& s, const Step
         }
     }
     trace_stamp(p, s, blockIdx.x, layer, 5, ctid);
-    consumer_bar();
+    consumer_bar<SM>();
     // one warp per head: maximum and normaliser by butterfly reductions (every lane ends with the same value)
-    for (uint32_t h = ctid >> 5; h < G; h += NCW) {
+    for (uint32_t h = ctid >> 5; h < G; h += SM::NCW) {
         const uint32_t lane = ctid & 31u;
         float Mx = -INFINITY;
         for (uint32_t c = lane; c < nchunk; c += 32) Mx = fmaxf(Mx, wtab[h * nchunk + c]);
@@ -1572,8 +2091,8 @@ __device__ __noinline__ void attn_merge(const Params& p, const SM& s, const Step
         const float inv = 1.0f / Lx;
         for (uint32_t c = lane; c < nchunk; c += 32) wtab[h * nchunk + c] *= inv;
     }
-    consumer_bar();
-    for (uint32_t j = ctid; j < ns; j += NCT) {
+    consumer_bar<SM>();
+    for (uint32_t j = ctid; j < ns; j += SM::NCT) {
         const uint32_t t = t_lo + j, h = t / hd, d = t % hd;
         float acc = 0.f;
         for (uint32_t c = 0; c < nchunk; ++c) acc += pv[j * nchunk + c] * wtab[h * nchunk + c];
@@ -1604,18 +2123,18 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
     // boxes are packed 128 bytes apart; the 15 ignored rows the tile loop also reads overlap whatever follows.
     uint8_t* stage_k = reinterpret_cast<uint8_t*>(new_v + hd);   // [hd/64][128 B]
     uint8_t* stage_v = stage_k + 256;
-    float* comb = reinterpret_cast<float*>(stage_v + 256);       // [NCW][G][hd + 2]
+    float* comb = reinterpret_cast<float*>(stage_v + 256);       // [SM::NCW][G][hd + 2]
 
     // q (and, for the unit that owns the new position, k and v) of this step: tagged words written by whichever CTAs
     // own those rows of the QKV projection.  The unit waits for exactly the rows it needs, not for the whole stage.
-    consumer_bar();   // the workspace below overlays the QKV stage's input vector: wait for this CTA's last QKV chunk
+    consumer_bar<SM>();   // the workspace below overlays the QKV stage's input vector: wait for this CTA's last QKV chunk
     const TW* qkv = p.qkv + (size_t)b * (p.QD + 2 * p.KVD);
     const uint32_t qtag = tag_of(p, cx, layer, TG_QKV);
     const float* cs = cx.rope_cs + (size_t)b * hd;  // [half][2]
     const float qscale = 1.4426950408889634f * rsqrtf((float)hd);
     // biases of the projections (decoders that have them): added to the polled values, before the rotation
     const __nv_bfloat16* bias = p.bqkv ? p.bqkv + (size_t)layer * p.layer_stride : nullptr;
-    for (uint32_t idx = ctid; idx < G * half; idx += NCT) {
+    for (uint32_t idx = ctid; idx < G * half; idx += SM::NCT) {
         const uint32_t h = idx / half, i = idx % half;
         const TW* qr = qkv + (size_t)(g * G + h) * hd;
         float a, bb;
@@ -1632,7 +2151,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
         const TW* kr = qkv + p.QD + (size_t)g * hd;
         const TW* vr = qkv + p.QD + p.KVD + (size_t)g * hd;
         // row 0 of a swizzled box is stored unswizzled: column k of box k/64 sits at byte (k % 64) * 2 of the box
-        for (uint32_t i = ctid; i < half; i += NCT) {
+        for (uint32_t i = ctid; i < half; i += SM::NCT) {
             float a, bb;
             poll_pair(p, s, kr + i, kr + i + half, qtag, a, bb);
             if (bias) {
@@ -1650,7 +2169,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
                 *reinterpret_cast<__nv_bfloat16*>(stage_k + (j >> 6) * 128u + (j & 63u) * 2u) = k1;
             }
         }
-        for (uint32_t d = ctid; d < hd; d += NCT) {
+        for (uint32_t d = ctid; d < hd; d += SM::NCT) {
             float va, vb;
             poll_pair(p, s, vr + d, vr + d, qtag, va, vb);
             if (bias) va += __bfloat162float(bias[p.QD + p.KVD + g * hd + d]);
@@ -1659,10 +2178,20 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
             if (GT == 0) *reinterpret_cast<__nv_bfloat16*>(stage_v + (d >> 6) * 128u + (d & 63u) * 2u) = v0;
         }
     }
-    consumer_bar();
+    consumer_bar<SM>();
     trace_stamp(p, s, cta, layer, 14, ctid);
 
-    const uint32_t first = rc.first_chunk(warp, p.nslots);
+    uint32_t first;
+    if constexpr (SM::kTmem) {
+        // stash mode: chunk i of the unit is chunk rc.start + i / 2 of pipeline i & 1 and sits in slot (that % 4) of the
+        // pipeline; slot 4 T + q is read by warp 4 T + q, whose chunks are therefore eight apart, each in the next phase
+        first = 2u * (((warp & 3u) - rc.start) & 3u) + (warp >> 2);
+        wr.cslot = 0u;
+        wr.cphase = KL_T_OHEAD ? (rc.n0 & 1u)   // K/V chunks this warp has read from its slot so far
+                               : (((rc.start + (first >> 1)) >> 2) & 1u);
+    } else {
+        first = rc.first_chunk(warp, p.nslots);
+    }
     if constexpr (GT == 0) {
         if (hd == 128) {
             if (G <= 4) attn_chunks_tc<128, true>(p, s, u, cta, warp, lane, first, rc, wr, q_s, comb, stage_k, stage_v);
@@ -1700,7 +2229,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
         for (uint32_t i = (warp < p.nslots ? first : u.nring); i < u.nring; i += p.nslots) {
             if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 1);
             const uint32_t slot = warp * p.nsw + wr.cslot;
-            mbar_wait(p, s, smem_u32(&s.full()[slot]), wr.cphase);
+            mbar_wait(p, s, smem_u32(s.kv_bar(slot)), wr.cphase);
             if (lane == 0) chunk_stamp(p, s, cta, rc.n0 + i, 2);
             ring_advance_consume(p, wr);
             const uint8_t* kp = s.ring() + (size_t)slot * SLOT_BYTES;
@@ -1774,26 +2303,26 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
         }
     }
     trace_stamp(p, s, cta, layer, 15, ctid);
-    consumer_bar();
+    consumer_bar<SM>();
 
     // merge the warps.  First one thread per (warp, head) turns that warp's maximum into its weight exp2(m - M_h);
-    // then thread t owns (head, column) and adds the NCW weighted terms in warp order.
+    // then thread t owns (head, column) and adds the SM::NCW weighted terms in warp order.
     const uint32_t unit = u.bg * p.cps + u.ch;
-    float* ftab = s.unit_part();   // [NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
-    if (ctid < NCW * G) {
+    float* ftab = s.unit_part();   // [SM::NCW][G] weights, then [G] maxima (the unit table is idle outside the GEMV stages)
+    if (ctid < SM::NCW * G) {
         const uint32_t w = ctid / G, h = ctid % G;
         float Mh = -INFINITY;
 #pragma unroll
-        for (int ww = 0; ww < NCW; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (hd + 2) + hd]);
+        for (int ww = 0; ww < SM::NCW; ++ww) Mh = fmaxf(Mh, comb[((size_t)ww * G + h) * (hd + 2) + hd]);
         ftab[w * G + h] = rescale(comb[((size_t)w * G + h) * (hd + 2) + hd], Mh);
-        if (w == 0) ftab[NCW * G + h] = Mh;
+        if (w == 0) ftab[SM::NCW * G + h] = Mh;
     }
-    consumer_bar();
-    for (uint32_t t = ctid; t < G * hd; t += NCT) {
+    consumer_bar<SM>();
+    for (uint32_t t = ctid; t < G * hd; t += SM::NCT) {
         const uint32_t h = t / hd, d = t % hd;
         float A = 0.f, Lsum = 0.f;
 #pragma unroll
-        for (int w = 0; w < NCW; ++w) {
+        for (int w = 0; w < SM::NCW; ++w) {
             const float* src = comb + ((size_t)w * G + h) * (hd + 2);
             const float c = ftab[w * G + h];
             A += src[d] * c;
@@ -1805,7 +2334,7 @@ __device__ __noinline__ void attention_stage(const Params& p, const SM& s, const
             const uint32_t ptag = tag_of(p, cx, layer, TG_PART);
             st_tw(p.part + ((size_t)unit * G + h) * hd + d, A, ptag);
             if (d == 0) {
-                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, ftab[NCW * G + h], ptag);
+                st_tw(p.part_ml + ((size_t)unit * G + h) * 2, ftab[SM::NCW * G + h], ptag);
                 st_tw(p.part_ml + ((size_t)unit * G + h) * 2 + 1, Lsum, ptag);
             }
         }

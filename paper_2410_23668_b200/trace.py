@@ -35,6 +35,7 @@ def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="llama31_8b_b1_ctx4096", choices=sorted(bench.WORKLOADS))
     ap.add_argument("--warm", type=int, default=5)
+    ap.add_argument("--greedy", action="store_true", help="trace the one-launch-per-token kernel (kl_decode_greedy)")
     args = ap.parse_args()
     shape, batch, context, _ = bench.WORKLOADS[args.workload]
     assert batch == 1, "the timeline is read for one sequence"
@@ -48,8 +49,13 @@ def main() -> None:
     for _ in range(args.warm):
         dec.kl_decode_step(tok, pos, cache, logits, batch)
         dec.kl_argmax_advance(logits, tok, pos, batch)
+    if args.greedy:
+        dec.kl_decode_greedy(tok, pos, cache, logits, batch, True)
     dec.kl_set_trace(buf)
-    dec.kl_decode_step(tok, pos, cache, logits, batch)
+    if args.greedy:
+        dec.kl_decode_greedy(tok, pos, cache, logits, batch, False)
+    else:
+        dec.kl_decode_step(tok, pos, cache, logits, batch)
     torch.cuda.synchronize()
     status = dec.kl_last_status()
     raw = buf.cpu().numpy()
