@@ -69,6 +69,13 @@ enum {
 /* kl_model_desc.flags: the q, k, v projections carry biases (KL_BQ, KL_BK, KL_BV must be loaded for every layer).
  * The paper's operator list has no such term; its Table 2 includes a 72B decoder that does. */
 #define KL_FLAG_QKV_BIAS 1u
+/* kl_model_desc.flags: keep the batch-1 kernels in their plain mode (weights consumed from the shared-memory ring).  By
+ * default, shapes that allow it -- dense layers, head_dim 64 or 128, hidden, n_q_heads * head_dim and ffn multiples of
+ * 2048, an input vector of ffn floats next to an eight-slot ring in shared memory -- run in stash mode: every weight
+ * chunk moves on from its ring slot into tensor memory and is multiplied from there, which more than doubles what an SM
+ * holds ahead of its consumers (the cross-layer weight prefetch of Section 2, deeper).  Both modes compute the same
+ * function; their sums are taken in different orders.  No counterpart in the paper. */
+#define KL_FLAG_NO_STASH 2u
 
 /* Shapes the kernels cover (anything else: KL_ERR_UNSUPPORTED_SHAPE): head_dim 32, 64, 128 or 256; hidden and ffn
  * multiples of 8; n_q_heads a multiple of n_kv_heads with 1, 2, 4 or 8 query heads per kv head -- any group size up
@@ -80,7 +87,7 @@ typedef struct {
     float rope_theta; /* RoPE base; pair (i, i + head_dim/2) rotates by position * theta^(-2i/head_dim) */
     uint32_t max_batch;
     uint32_t max_ctx; /* capacity of the KV cache in positions */
-    uint32_t flags;   /* 0 or KL_FLAG_QKV_BIAS */
+    uint32_t flags;   /* 0 or a combination of KL_FLAG_QKV_BIAS, KL_FLAG_NO_STASH */
     /* Mixture-of-experts MLP (the 8x7B decoder of the paper's Table 2 is of this kind; the paper's operator list has no
      * such term): n_experts > 0 gives every layer a router [n_experts, hidden] and n_experts MLPs of width ffn, of
      * which the top_k with the largest router logits (the lower index first among equals) process a token, weighted
@@ -291,6 +298,10 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes;
  * built for 1, 2, 4 and 8 query heads per kv head: KL_ERR_UNSUPPORTED_SHAPE for other group sizes). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
+
+/* 1: the handle's batch-1 kernels run in stash mode (see KL_FLAG_NO_STASH), 0: plain mode, negative: h is null.  No
+ * counterpart in the paper. */
+int kl_stash_mode(const kl_handle* h);
 
 /* Decode steps of a batch (batch > 1).  on = 1 (default when available): the tensor-core path -- every projection
  * of the step (QKV, O, gate/up, down, classifier) is one dense contraction for the whole batch on the tcgen05 tensor

@@ -27,12 +27,13 @@ KL_MODE_PER_STAGE = 2
 TENSOR_IDS = {"embed": 0, "wq": 1, "wk": 2, "wv": 3, "wo": 4, "wgate": 5, "wup": 6, "wdown": 7,
               "norm1": 8, "norm2": 9, "norm_f": 10, "lm_head": 11, "bq": 12, "bk": 13, "bv": 14, "router": 15}
 KL_FLAG_QKV_BIAS = 1
+KL_FLAG_NO_STASH = 2
 
 # every symbol include/kl.h declares
 EXPORTS = ("kl_workspace_bytes", "kl_create", "kl_load_weights", "kl_kv_cache_bytes", "kl_set_mode", "kl_decode_step",
            "kl_decode_step_host", "kl_argmax_advance", "kl_read_hidden", "kl_last_status", "kl_launch_count",
            "kl_set_wait_limit_ns", "kl_debug_skip_signal_once", "kl_status_string", "kl_destroy", "kl_profile_enable",
-           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_argmax_advance_static", "kl_set_batched_path",
+           "kl_profile_read", "kl_set_trace", "kl_set_tensor_core_attention", "kl_stash_mode", "kl_argmax_advance_static", "kl_set_batched_path",
            "kl_set_dependent_launch", "kl_decode_greedy_host", "kl_decode_greedy", "kl_decode_greedy_tokens",
            "kl_decode_greedy_tokens_host", "kl_debug_set_step", "kl_debug_set_jitter", "kl_load_expert_weights")
 
@@ -107,6 +108,8 @@ def lib():
     l.kl_set_trace.restype = i32
     l.kl_set_tensor_core_attention.argtypes = [vp, C.c_int]
     l.kl_set_tensor_core_attention.restype = i32
+    l.kl_stash_mode.argtypes = [vp]
+    l.kl_stash_mode.restype = C.c_int
     l.kl_set_batched_path.argtypes = [vp, C.c_int]
     l.kl_set_batched_path.restype = i32
     l.kl_set_dependent_launch.argtypes = [vp, C.c_int]
@@ -134,10 +137,10 @@ def _check(code: int, where: str) -> None:
         raise KlError(code, where)
 
 
-def make_desc(shape, max_batch: int, max_ctx: int) -> ModelDesc:
+def make_desc(shape, max_batch: int, max_ctx: int, stash: bool = True) -> ModelDesc:
     return ModelDesc(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, shape.ffn,
                      shape.vocab, float(shape.rms_eps), float(shape.rope_theta), max_batch, max_ctx,
-                     KL_FLAG_QKV_BIAS if getattr(shape, "qkv_bias", False) else 0,
+                     (KL_FLAG_QKV_BIAS if getattr(shape, "qkv_bias", False) else 0) | (0 if stash else KL_FLAG_NO_STASH),
                      int(getattr(shape, "n_experts", 0) or 0), int(getattr(shape, "top_k", 0) or 0))
 
 
@@ -164,12 +167,12 @@ def kl_argmax_advance_static(logits_d, tokens_d, positions_d, batch: int, stream
 class Decoder:
     """One model instance on the current CUDA device.  Owns the two arenas as torch uint8 tensors."""
 
-    def __init__(self, shape, max_batch: int, max_ctx: int, device="cuda"):
+    def __init__(self, shape, max_batch: int, max_ctx: int, device="cuda", stash: bool = True):
         import torch
         self.torch = torch
         self.shape = shape
         self.max_batch, self.max_ctx = max_batch, max_ctx
-        self.desc = make_desc(shape, max_batch, max_ctx)
+        self.desc = make_desc(shape, max_batch, max_ctx, stash)
         wb, sb = kl_workspace_bytes(self.desc)
         self.weight_bytes, self.scratch_bytes = wb, sb
         self.weight_arena = torch.empty(wb, dtype=torch.uint8, device=device)
@@ -261,6 +264,9 @@ class Decoder:
         a, b, c = C.c_uint32(), C.c_uint32(), C.c_uint32()
         _check(lib().kl_set_trace(self.handle, _ptr(trace_d), C.byref(a), C.byref(b), C.byref(c)), "kl_set_trace")
         return a.value, b.value, c.value
+
+    def kl_stash_mode(self) -> int:
+        return int(lib().kl_stash_mode(self.handle))
 
     def kl_set_tensor_core_attention(self, on: bool) -> None:
         _check(lib().kl_set_tensor_core_attention(self.handle, 1 if on else 0), "kl_set_tensor_core_attention")

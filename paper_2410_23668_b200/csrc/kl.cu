@@ -681,7 +681,7 @@ struct Layout {
 
 bool shape_supported(const kl_model_desc& d, int num_sms) {
     if (!d.n_layers || !d.hidden || !d.n_q_heads || !d.n_kv_heads || !d.head_dim || !d.ffn || !d.vocab) return false;
-    if (!d.max_batch || !d.max_ctx || (d.flags & ~(uint32_t)KL_FLAG_QKV_BIAS) != 0) return false;
+    if (!d.max_batch || !d.max_ctx || (d.flags & ~(uint32_t)(KL_FLAG_QKV_BIAS | KL_FLAG_NO_STASH)) != 0) return false;
     if (d.head_dim != 32 && d.head_dim != 64 && d.head_dim != 128 && d.head_dim != 256) return false;
     if (d.hidden % 8 || d.ffn % 8) return false;
     if (d.n_q_heads % d.n_kv_heads) return false;
@@ -1102,7 +1102,7 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     h->stash = 0;
     {
         const char* e = getenv("KL_STASH");
-        if (d.n_experts == 0 && h->use_tc_attention && !(e && e[0] == '0')) {
+        if (d.n_experts == 0 && h->use_tc_attention && !(d.flags & KL_FLAG_NO_STASH) && !(e && e[0] == '0')) {
             p.plan[PL_QKV] = make_plan_t(p.QD + 2 * p.KVD, p.H, false, p.P, p.KVD);
             p.plan[PL_O] = make_plan_t(p.H, p.QD, false, p.P, 0);
             p.plan[PL_GU] = make_plan_t(2 * p.F, p.H, true, p.P, 0);
@@ -2040,6 +2040,8 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
     if (n_stamps) *n_stamps = TRACE_STAMPS;
     return KL_OK;
 }
+
+int kl_stash_mode(const kl_handle* h) { return h ? h->stash : -1; }
 
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;

@@ -471,7 +471,10 @@ __device__ __forceinline__ CtaRange cta_units(const GemvPlan& pl, uint32_t cta, 
 // chunks per pipeline -- what its TMEM regions hold -- or the K/V chunks behind them could never be requested.
 __device__ __forceinline__ uint32_t t_o_head(const GemvPlan& pl, uint32_t nu) {
     if (!KL_T_OHEAD) return 0u;
-    const uint32_t h = 2u * ((uint32_t)T_NREG / pl.npieces);
+#ifndef KL_T_OHEAD_REGIONS
+#define KL_T_OHEAD_REGIONS T_NREG
+#endif
+    const uint32_t h = 2u * ((uint32_t)(KL_T_OHEAD_REGIONS) / pl.npieces);
     return nu < h ? nu : h;
 }
 struct ChunkGeom {

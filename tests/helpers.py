@@ -50,10 +50,11 @@ class HostWeights:
         return self._cache["g"]
 
 
-def make_decoder(shape, max_batch, max_ctx, seed, overrides=None):
-    """CUDA-path model with weights generated on the device, one layer at a time."""
+def make_decoder(shape, max_batch, max_ctx, seed, overrides=None, stash=True):
+    """CUDA-path model with weights generated on the device, one layer at a time.  stash=False keeps the batch-1
+    kernels in their plain mode on shapes that would take the stash mode."""
     build.build_library()
-    dec = binding.Decoder(shape, max_batch, max_ctx)
+    dec = binding.Decoder(shape, max_batch, max_ctx, stash=stash)
     overrides = overrides or {}
     for l in range(shape.n_layers):
         for name, t in gen.make_layer(shape, l, seed, "cuda").items():
@@ -77,7 +78,7 @@ def bf16_decode(u16: np.ndarray) -> np.ndarray:
 
 def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
                modes=(binding.KL_MODE_LOOPED, binding.KL_MODE_PER_LAYER, binding.KL_MODE_PER_STAGE),
-               overrides=None, positions0=None, stream_layers=False, check_cache=True, batched_path=None):
+               overrides=None, positions0=None, stream_layers=False, check_cache=True, batched_path=None, stash=True):
     """Teacher-forced greedy decode: the oracle runs `steps` steps on its own tokens; each CUDA mode consumes the
     oracle's token of the previous step.  Returns a report dict; asserts nothing.  batched_path: None leaves the
     library's default (batches take the tensor-core path when the shape allows), True / False forces the choice
@@ -100,7 +101,8 @@ def run_parity(shape, context, steps, seed=0, batch=1, max_ctx=None,
         t, p = nxt.tolist(), [q + 1 for q in p]
 
     report = dict(ref=ref, modes={}, cache_ref=cache_or, cache0=cache0.cpu().view(torch.uint16).numpy())
-    dec = make_decoder(shape, batch, max_ctx, seed, overrides)
+    dec = make_decoder(shape, batch, max_ctx, seed, overrides, stash)
+    report["stash_mode"] = dec.kl_stash_mode()
     if batched_path is not None:
         dec.kl_set_batched_path(batched_path)
     for mode in modes:

@@ -53,6 +53,34 @@ def test_odd_shapes(name):
     helpers.assert_parity(rep, 3)
 
 
+# Shapes that take the stash mode (weights through tensor memory) on paths the 8B shape does not use: rows of 2048
+# columns (four rows per chunk, two units per group) and a down projection of two pieces of 4096 columns.
+STASH_SHAPES = {
+    "rows_of_2048": gen.ModelShape(2, 2048, 16, 4, 128, 4096, 1544, 1e-5, 500000.0),
+    "down_in_two_pieces": gen.ModelShape(2, 4096, 32, 8, 128, 8192, 1544, 1e-5, 500000.0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(STASH_SHAPES))
+def test_stash_mode_shapes(name):
+    rep = helpers.run_parity(STASH_SHAPES[name], context=300, steps=3, seed=5)
+    assert rep["stash_mode"] == 1
+    helpers.assert_parity(rep, 3)
+
+
+def test_llama31_8b_layer_shape_both_modes():
+    """The 8B layer shape (two layers) in stash mode and with KL_FLAG_NO_STASH: both match the oracle, and the odd shapes
+    above never take the stash mode."""
+    import dataclasses
+    shape = dataclasses.replace(gen.LLAMA31_8B, n_layers=2)
+    for stash in (True, False):
+        rep = helpers.run_parity(shape, context=700, steps=3, seed=2, stash=stash)
+        assert rep["stash_mode"] == (1 if stash else 0)
+        helpers.assert_parity(rep, 3)
+    rep = helpers.run_parity(SHAPES["odd_rows_hd128"], context=20, steps=1, seed=1)
+    assert rep["stash_mode"] == 0
+
+
 def test_llama31_8b_shape_16_greedy_steps():
     """Config 2: Llama-3.1-8B shape, batch 1, context 4096, first 16 decode steps, looped and per-layer."""
     rep = helpers.run_parity(gen.LLAMA31_8B, context=4096, steps=16, seed=0, max_ctx=4096 + 136, check_cache=False)
