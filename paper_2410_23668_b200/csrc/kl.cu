@@ -270,7 +270,7 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
 // stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
 // boundary after every operator group).
-template <bool TR, bool MOE, bool TM>
+template <bool TR, bool MOE, int TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
                                                                  uint32_t sbeg, uint32_t send) {
     using SM = SmemT<TR, MOE, TM>;
@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_co
 }
 
 // Classifier block: logits = W_lm rmsnorm(x; g_f).  Same ring, one stage, no inter-CTA dependency.
-template <bool TM>
+template <int TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_classifier_kernel(const __grid_constant__ Params p) {
     using SM = SmemT<false, false, TM>;
     const SM s;
@@ -556,7 +556,7 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
 // K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
-template <bool TR, bool MOE, bool TM>
+template <bool TR, bool MOE, int TM>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
     using SM = SmemT<TR, MOE, TM>;
     const SM s;
@@ -866,8 +866,8 @@ GemvPlan make_plan_t(uint32_t R, uint32_t K, bool pairs, uint32_t P, uint32_t al
     pl.nseg = 1;
     const uint32_t minrows = pairs ? 2u : 1u;
     uint32_t kp = 0;
-    const uint32_t cand[2] = {4096u, 2048u};   // the widths the consumer loop is instantiated for
-    for (int i = 0; i < 2 && !kp; ++i)
+    const uint32_t cand[4] = {4096u, 3072u, 2048u, 1024u};   // the widths the consumer loop is instantiated for
+    for (int i = 0; i < 4 && !kp; ++i)
         if (K % cand[i] == 0 && cand[i] * 2u * minrows <= (uint32_t)SLOT_BYTES) kp = cand[i];
     if (!kp) return pl;
     pl.kp = kp;
@@ -1113,6 +1113,9 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
             int optin = 0;
             h->stash = plans_ok_t(p) && cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) == cudaSuccess &&
                        (size_t)2 * T_NSP * SLOT_BYTES + vmax * 4 + SMEM_MISC_BYTES + 16384 <= (size_t)optin;
+            if (h->stash)   // 1: chunks of 2048 / 4096 columns only (the kernel without the other widths), 2: any
+                for (int i = 0; i < PL_COUNT; ++i)
+                    if (p.plan[i].kp != 2048u && p.plan[i].kp != 4096u) h->stash = 2;
         }
     }
     if (!h->stash) {
@@ -1168,27 +1171,29 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
     cudaError_t ce = cudaSuccess;
     {
-        const void* fns[] = {(const void*)kl_decoder_kernel<false, false, false>, (const void*)kl_decoder_kernel<true, false, false>,
-                             (const void*)kl_decoder_kernel<false, true, false>, (const void*)kl_decoder_kernel<false, false, true>,
-                             (const void*)kl_decoder_kernel<true, false, true>, (const void*)kl_classifier_kernel<false>,
-                             (const void*)kl_classifier_kernel<true>};
+        const void* fns[] = {(const void*)kl_decoder_kernel<false, false, 0>, (const void*)kl_decoder_kernel<true, false, 0>,
+                             (const void*)kl_decoder_kernel<false, true, 0>, (const void*)kl_decoder_kernel<false, false, 1>,
+                             (const void*)kl_decoder_kernel<true, false, 1>, (const void*)kl_decoder_kernel<false, false, 2>,
+                             (const void*)kl_decoder_kernel<true, false, 2>, (const void*)kl_classifier_kernel<0>,
+                             (const void*)kl_classifier_kernel<1>, (const void*)kl_classifier_kernel<2>};
         for (const void* f : fns)
             if (ce == cudaSuccess) ce = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     }
     {
         int tocc = 0;
-        const void* fns[] = {(const void*)kl_token_kernel<false, false, false>, (const void*)kl_token_kernel<true, false, false>,
-                             (const void*)kl_token_kernel<false, true, false>, (const void*)kl_token_kernel<false, false, true>,
-                             (const void*)kl_token_kernel<true, false, true>};
+        const void* fns[] = {(const void*)kl_token_kernel<false, false, 0>, (const void*)kl_token_kernel<true, false, 0>,
+                             (const void*)kl_token_kernel<false, true, 0>, (const void*)kl_token_kernel<false, false, 1>,
+                             (const void*)kl_token_kernel<true, false, 1>, (const void*)kl_token_kernel<false, false, 2>,
+                             (const void*)kl_token_kernel<true, false, 2>};
         h->token_ok = 1;
         for (const void* f : fns)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) != cudaSuccess) h->token_ok = 0;
         if (h->token_ok)
-            h->token_ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false, false>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+            h->token_ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false, 0>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
-    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false, false>, NTHREADS, h->smem_bytes);
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false, 0>, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
         fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
                         "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
@@ -1615,12 +1620,26 @@ static kl_status batched_step(kl_handle* h, const int32_t* tokens_d, const int32
     return decode_step_batched(h, tokens_d, positions_d, kv_cache_d, logits_d, batch, st);
 }
 
+// The instantiation a launch takes: mixture of experts, stash mode (1: chunks of 2048 / 4096 columns only, 2: all
+// widths), and the debug hooks (trace stamps, jitter) only while one of them is set.
 static const void* token_fn(const kl_handle* h) {
     const Params& p = h->prm;
-    if (p.n_experts) return (const void*)kl_token_kernel<false, true, false>;
     const bool dbg = p.jitter_seed != 0u || p.trace != nullptr;
-    if (h->stash) return dbg ? (const void*)kl_token_kernel<true, false, true> : (const void*)kl_token_kernel<false, false, true>;
-    return dbg ? (const void*)kl_token_kernel<true, false, false> : (const void*)kl_token_kernel<false, false, false>;
+    if (p.n_experts) return (const void*)kl_token_kernel<false, true, 0>;
+    if (h->stash == 1) return dbg ? (const void*)kl_token_kernel<true, false, 1> : (const void*)kl_token_kernel<false, false, 1>;
+    if (h->stash == 2) return dbg ? (const void*)kl_token_kernel<true, false, 2> : (const void*)kl_token_kernel<false, false, 2>;
+    return dbg ? (const void*)kl_token_kernel<true, false, 0> : (const void*)kl_token_kernel<false, false, 0>;
+}
+static const void* decoder_fn(const kl_handle* h, const Params& p) {
+    const bool dbg = p.trace != nullptr || p.jitter_seed != 0u;
+    if (p.n_experts) return (const void*)kl_decoder_kernel<false, true, 0>;
+    if (h->stash == 1) return dbg ? (const void*)kl_decoder_kernel<true, false, 1> : (const void*)kl_decoder_kernel<false, false, 1>;
+    if (h->stash == 2) return dbg ? (const void*)kl_decoder_kernel<true, false, 2> : (const void*)kl_decoder_kernel<false, false, 2>;
+    return dbg ? (const void*)kl_decoder_kernel<true, false, 0> : (const void*)kl_decoder_kernel<false, false, 0>;
+}
+static const void* classifier_fn(const kl_handle* h) {
+    return h->stash == 1 ? (const void*)kl_classifier_kernel<1> : h->stash == 2 ? (const void*)kl_classifier_kernel<2>
+                                                                                  : (const void*)kl_classifier_kernel<0>;
 }
 
 kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* positions_d, void* kv_cache_d,
@@ -1664,11 +1683,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
         if (ev && b == 0 && cudaEventRecord(ev[0], st) != cudaSuccess) return KL_ERR_CUDA;
         uint32_t sbeg = 0, send = 5;
         // the instantiation with the trace stamps compiled in only while a trace buffer is set
-        const bool dbg = p.trace != nullptr || p.jitter_seed != 0u;
-        const void* decoder_fn = p.n_experts ? (const void*)kl_decoder_kernel<false, true, false>
-                                 : h->stash ? (dbg ? (const void*)kl_decoder_kernel<true, false, true> : (const void*)kl_decoder_kernel<false, false, true>)
-                                 : dbg      ? (const void*)kl_decoder_kernel<true, false, false>
-                                            : (const void*)kl_decoder_kernel<false, false, false>;
+        const void* decoder_fn = ::decoder_fn(h, p);
         if (h->mode == KL_MODE_LOOPED) {
             uint32_t l0 = 0, l1 = p.L;
             void* args[] = {&p, &l0, &l1, &sbeg, &send};
@@ -1694,7 +1709,7 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
             Params pc = p;
             pc.chunk_trace = nullptr;  // the chunk log covers the decoder kernel only
             void* cargs[] = {&pc};
-            if ((rc = launch_persistent(h, h->stash ? (const void*)kl_classifier_kernel<true> : (const void*)kl_classifier_kernel<false>, cargs, st)) != KL_OK) return rc;
+            if ((rc = launch_persistent(h, classifier_fn(h), cargs, st)) != KL_OK) return rc;
         }
         if (ev && b == 0 && cudaEventRecord(ev[2], st) != cudaSuccess) return KL_ERR_CUDA;
         if (batch > 1) {
@@ -2041,7 +2056,7 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
     return KL_OK;
 }
 
-int kl_stash_mode(const kl_handle* h) { return h ? h->stash : -1; }
+int kl_stash_mode(const kl_handle* h) { return h ? (h->stash ? 1 : 0) : -1; }
 
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;

@@ -355,11 +355,15 @@ struct MoeSel {
     uint32_t e[MAX_TOP_K];          // the chosen experts, in descending order of their logits
     float w[MAX_TOP_K];             // and their gate weights
 };
-template <bool TR, bool MOE = false, bool TM = false>
+template <bool TR, bool MOE = false, int TM = 0>
 struct SmemT {
     static constexpr bool kTrace = TR;
     static constexpr bool kMoe = MOE;
-    static constexpr bool kTmem = TM;            // stash mode: weights go ring -> TMEM -> registers (see the stash section)
+    static constexpr bool kTmem = TM != 0;       // stash mode: weights go ring -> TMEM -> registers (see the stash section)
+    // TM == 1: the stage exists for chunks of 2048 and 4096 columns only; TM == 2: for 1024 and 3072 as well.  Two kernels,
+    // because the code the common shapes never run costs them time by lying between the code they do run
+    // (measured: 3.04 against 2.97 ms per token on the 8B shape).
+    static constexpr bool kAllWidths = TM == 2;
     static constexpr int NCW = TM ? T_NCW : kl::NCW;   // consumer warps
     static constexpr int NCT = NCW * 32;               // consumer threads (they take part in the CTA-wide steps)
     __device__ __forceinline__ static MoeSel* moe() { return reinterpret_cast<MoeSel*>(kl_smem + 6240); }
@@ -376,7 +380,7 @@ struct SmemT {
     // are weight chunks it never waits for)
     __device__ __forceinline__ static uint64_t* kvready() { return reinterpret_cast<uint64_t*>(kl_smem + 800); }
     // the barrier a reader of K/V chunks in ring slot `slot` waits on
-    __device__ __forceinline__ static uint64_t* kv_bar(uint32_t slot) { return ((TM && KL_T_OHEAD) ? kvready() : full()) + slot; }
+    __device__ __forceinline__ static uint64_t* kv_bar(uint32_t slot) { return ((TM != 0 && KL_T_OHEAD) ? kvready() : full()) + slot; }
     __device__ __forceinline__ static int* t_ucnt() { return reinterpret_cast<int*>(kl_smem + 1024); }
     __device__ __forceinline__ static float* red() { return reinterpret_cast<float*>(kl_smem + 1536); }
     __device__ __forceinline__ static float* unit_part() { return reinterpret_cast<float*>(kl_smem + 2048); }
@@ -1537,49 +1541,48 @@ struct TCur {
 // how many k in [0, n) have ((uc + k) & 1) == t
 __device__ __forceinline__ uint32_t t_count(uint32_t uc, uint32_t n, uint32_t t) { return (n + (((uc & 1u) == t) ? 1u : 0u)) >> 1; }
 
-// Half a chunk (16 registers = four granules per lane): acc[row][.] += the lane's granules of `row` times its slice of
-// the vector.  NJ granules per row: with NJ = 4 a half is one row, with NJ = 2 two rows (HALF selects rows NR/2 ...).
+// Half a chunk (16 registers = four 16-byte granules per lane) times the lane's slice of the vector.  Granule m of a
+// chunk (m = 0 .. 7) belongs to row m / NJ and to column block 4 (m % NJ) + q of the piece; rows beyond 8 / NJ do not
+// exist (NJ = 3 leaves two granules unused).  acc[row][0] takes the even columns, acc[row][1] the odd ones.
 template <int NJ, int HALF>
 __device__ __forceinline__ void t_dot(const uint32_t (&w)[16], const float4* v4, uint32_t blk0, uint32_t q, uint32_t lane,
                                       float (&acc)[8 / NJ][2]) {
-
-    static_assert(NJ == 2 || NJ == 4, "widths the stash mode is built for");
+    constexpr int NR = 8 / NJ;
 #pragma unroll
     for (int jj = 0; jj < NJ; ++jj) {
-        const float4 lo = v4[(blk0 + 4u * jj + q) * 64u + lane], hi = v4[(blk0 + 4u * jj + q) * 64u + 32u + lane];
+        // the vector block of column group jj is loaded once for all rows of this half that meet it
+        bool used = false;
 #pragma unroll
-        for (int rh = 0; rh < 4 / NJ; ++rh) {
-            const int row = HALF * (4 / NJ) + rh;
-            const int m = (rh * NJ + jj) * 4;
-            ffma2(acc[row][0], acc[row][1], bf_lo(w[m]), bf_hi(w[m]), lo.x, lo.y);
-            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 1]), bf_hi(w[m + 1]), lo.z, lo.w);
-            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 2]), bf_hi(w[m + 2]), hi.x, hi.y);
-            ffma2(acc[row][0], acc[row][1], bf_lo(w[m + 3]), bf_hi(w[m + 3]), hi.z, hi.w);
+        for (int row = 0; row < NR; ++row) used = used || (row * NJ + jj) / 4 == HALF;
+        if (used) {
+            const float4 lo = v4[(blk0 + 4u * jj + q) * 64u + lane], hi = v4[(blk0 + 4u * jj + q) * 64u + 32u + lane];
+#pragma unroll
+            for (int row = 0; row < NR; ++row) {
+                const int m = row * NJ + jj;
+                if (m / 4 == HALF) {
+                    const int gi = (m % 4) * 4;
+                    ffma2(acc[row][0], acc[row][1], bf_lo(w[gi]), bf_hi(w[gi]), lo.x, lo.y);
+                    ffma2(acc[row][0], acc[row][1], bf_lo(w[gi + 1]), bf_hi(w[gi + 1]), lo.z, lo.w);
+                    ffma2(acc[row][0], acc[row][1], bf_lo(w[gi + 2]), bf_hi(w[gi + 2]), hi.x, hi.y);
+                    ffma2(acc[row][0], acc[row][1], bf_lo(w[gi + 3]), bf_hi(w[gi + 3]), hi.z, hi.w);
+                }
+            }
         }
     }
 }
-
-// The same with the lane's slice of the vector in registers (whole rows of 4096 columns: blocks q, 4 + q, 8 + q, 12 + q).
-template <int HALF>
-__device__ __forceinline__ void t_dot_xr(const uint32_t (&w)[16], const float (&x)[4][8], float (&acc)[2][2]) {
+// The same with the lane's slice of the vector in registers (whole rows: x[jj] is column block 4 jj + q).
+template <int NJ, int HALF>
+__device__ __forceinline__ void t_dot_xr(const uint32_t (&w)[16], const float (&x)[NJ][8], float (&acc)[8 / NJ][2]) {
 #pragma unroll
-    for (int jj = 0; jj < 4; ++jj) {
-        const int m = jj * 4;
-#ifdef KL_NO_FFMA2
-        acc[HALF][0] = fmaf(bf_lo(w[m]), x[jj][0], acc[HALF][0]);
-        acc[HALF][1] = fmaf(bf_hi(w[m]), x[jj][1], acc[HALF][1]);
-        acc[HALF][0] = fmaf(bf_lo(w[m + 1]), x[jj][2], acc[HALF][0]);
-        acc[HALF][1] = fmaf(bf_hi(w[m + 1]), x[jj][3], acc[HALF][1]);
-        acc[HALF][0] = fmaf(bf_lo(w[m + 2]), x[jj][4], acc[HALF][0]);
-        acc[HALF][1] = fmaf(bf_hi(w[m + 2]), x[jj][5], acc[HALF][1]);
-        acc[HALF][0] = fmaf(bf_lo(w[m + 3]), x[jj][6], acc[HALF][0]);
-        acc[HALF][1] = fmaf(bf_hi(w[m + 3]), x[jj][7], acc[HALF][1]);
-#else
-        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m]), bf_hi(w[m]), x[jj][0], x[jj][1]);
-        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 1]), bf_hi(w[m + 1]), x[jj][2], x[jj][3]);
-        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 2]), bf_hi(w[m + 2]), x[jj][4], x[jj][5]);
-        ffma2(acc[HALF][0], acc[HALF][1], bf_lo(w[m + 3]), bf_hi(w[m + 3]), x[jj][6], x[jj][7]);
-#endif
+    for (int gi = 0; gi < 4; ++gi) {
+        constexpr int NR = 8 / NJ;
+        const int m = HALF * 4 + gi, row = m / NJ, jj = m % NJ;
+        if (row < NR) {
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[gi * 4]), bf_hi(w[gi * 4]), x[jj][0], x[jj][1]);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[gi * 4 + 1]), bf_hi(w[gi * 4 + 1]), x[jj][2], x[jj][3]);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[gi * 4 + 2]), bf_hi(w[gi * 4 + 2]), x[jj][4], x[jj][5]);
+            ffma2(acc[row][0], acc[row][1], bf_lo(w[gi * 4 + 3]), bf_hi(w[gi * 4 + 3]), x[jj][6], x[jj][7]);
+        }
     }
 }
 
@@ -1649,10 +1652,10 @@ __device__ __forceinline__ bool mbar_wait_c(const SM& s, uint32_t bar, uint32_t 
 // the rows.  Value v of a group is row v % NR of its unit v / NR.
 //   wa: the first half of the group's first chunk, its load already in flight; on return, if `more`, that of the next
 //       group's first chunk (so that the reduction runs under a load, too)
-//   xr: whole rows of 4096 columns keep the lane's slice of the vector in registers
+//   xr: whole rows keep the lane's slice of the vector in registers
 template <int NJ, bool WHOLE, class SM>
 __device__ __forceinline__ void gemv_group_t(const SM& s, const TStageArgs& a, uint32_t unit0, uint32_t nun, uint32_t T, uint32_t q,
-                                             uint32_t& g, uint32_t tu, uint32_t (&wa)[16], bool more, const float (&xr)[4][8]) {
+                                             uint32_t& g, uint32_t tu, uint32_t (&wa)[16], bool more, const float (&xr)[NJ][8]) {
     constexpr int NR = 8 / NJ, GU = WHOLE ? 8 / NR : 1;
     const uint32_t lane = a.lane;
     const float4* v4 = reinterpret_cast<const float4*>(s.vec_t());
@@ -1688,13 +1691,11 @@ __device__ __forceinline__ void gemv_group_t(const SM& s, const TStageArgs& a, u
             if ((uint32_t)c < nun) {
                 tm_ld_wait();
                 second();
-                if constexpr (NJ == 4) t_dot_xr<0>(wa, xr, acc);
-                else t_dot<NJ, 0>(wa, v4, 0u, q, lane, acc);
+                t_dot_xr<NJ, 0>(wa, xr, acc);
                 tm_ld_wait();
                 landed();
                 if ((uint32_t)c + 1u < nun || more) fetch0();
-                if constexpr (NJ == 4) t_dot_xr<1>(wb, xr, acc);
-                else t_dot<NJ, 1>(wb, v4, 0u, q, lane, acc);
+                t_dot_xr<NJ, 1>(wb, xr, acc);
 #pragma unroll
                 for (int rr = 0; rr < NR; ++rr) {
                     y[c * NR + rr] = acc[rr][0] + acc[rr][1];
@@ -1761,11 +1762,11 @@ __device__ __noinline__ TStageRet gemv_units_t(const TStageArgs a) {
         tm_fence_after();
         tm_ld16(*s.tbase() + ((32u * q) << 16) + (T * T_NREG + g % T_NREG) * 32u, wa);
     }
-    float xr[4][8];
-    if (NJ == 4 && a.tp == 1) {
+    float xr[NJ][8];   // whole rows: the lane's slice of the vector stays in registers for the stage
+    if (a.tp == 1) {
         const float4* v4 = reinterpret_cast<const float4*>(s.vec_t());
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
+        for (int jj = 0; jj < NJ; ++jj) {
             const float4 lo = v4[(4u * jj + q) * 64u + lane], hi = v4[(4u * jj + q) * 64u + 32u + lane];
             xr[jj][0] = lo.x; xr[jj][1] = lo.y; xr[jj][2] = lo.z; xr[jj][3] = lo.w;
             xr[jj][4] = hi.x; xr[jj][5] = hi.y; xr[jj][6] = hi.z; xr[jj][7] = hi.w;
@@ -1796,7 +1797,14 @@ __device__ __forceinline__ void gemv_stage_t(const Params& p, const SM& s, const
     a.ep = ep; a.out = out; a.xscale = xscale;
     a.warp = warp; a.lane = lane;
     a.uc = tc.uc; a.g = tc.g; a.tu = tc.tu;
-    const TStageRet ret = pl.kp == 4096u ? gemv_units_t<4, SM>(a) : gemv_units_t<2, SM>(a);
+    const uint32_t nj = pl.kp >> 10;
+    TStageRet ret;
+    if constexpr (SM::kAllWidths) {
+        ret = nj == 4u ? gemv_units_t<4, SM>(a) : nj == 2u ? gemv_units_t<2, SM>(a)
+            : nj == 3u ? gemv_units_t<3, SM>(a) : gemv_units_t<1, SM>(a);
+    } else {
+        ret = nj == 4u ? gemv_units_t<4, SM>(a) : gemv_units_t<2, SM>(a);
+    }
     const uint32_t mine = t_count(tc.uc, a.nu, warp >> 2);
     tc.uc += a.nu;
     tc.c += mine * a.tp;
