@@ -296,7 +296,9 @@ kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32
 
 /* Attention inner loop.  on = 1 (default when head_dim is 64 or 128): tensor-core loop (mma.sync on 128-byte
  * swizzled TMA boxes of the cache); on = 0: CUDA-core loop on linear copies (always used for other head sizes;
- * built for 1, 2, 4 and 8 query heads per kv head: KL_ERR_UNSUPPORTED_SHAPE for other group sizes). */
+ * built for 1, 2, 4 and 8 query heads per kv head: KL_ERR_UNSUPPORTED_SHAPE for other group sizes, and for handles
+ * in stash mode, whose kernels carry the tensor-core loop only -- create the model with KL_FLAG_NO_STASH to use
+ * on = 0).  In stash mode the chunk log of kl_set_trace stays empty (stage stamps are taken). */
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on);
 
 /* 1: the handle's batch-1 kernels run in stash mode (see KL_FLAG_NO_STASH), 0: plain mode, negative: h is null.  No

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
 template <class SM>
 __device__ __noinline__ void attention_block(const Params& p, const SM& s, const StepCtx& cx, uint32_t l, uint32_t cta,
                                              uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
-    if (p.attn_tc) {
+    if (SM::kTmem || p.attn_tc) {   // the stash-mode kernels carry the tensor-core loop only
         attention_stage_and_advance<0>(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
     } else switch (p.G) {
         case 1: attention_stage_and_advance<1>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
@@ -2060,6 +2060,7 @@ int kl_stash_mode(const kl_handle* h) { return h ? (h->stash ? 1 : 0) : -1; }
 
 kl_status kl_set_tensor_core_attention(kl_handle* h, int on) {
     if (!h) return KL_ERR_INVALID_ARG;
+    if (!on && h->stash) return KL_ERR_UNSUPPORTED_SHAPE;   // the stash-mode kernels have no CUDA-core attention loop
     if (on && !h->encode_tiled) return KL_ERR_CUDA;
     const uint32_t G = h->prm.G;
     if (!on && G != 1 && G != 2 && G != 4 && G != 8) return KL_ERR_UNSUPPORTED_SHAPE;   // no CUDA-core loop for this group size
