@@ -149,10 +149,10 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def build_model(shape, batch, context, steps_total, seed=0):
+def build_model(shape, batch, context, steps_total, seed=0, stash=True):
     from paper_2410_23668_b200 import binding
     max_ctx = context + steps_total + 8
-    dec = binding.Decoder(shape, batch, max_ctx)
+    dec = binding.Decoder(shape, batch, max_ctx, stash=stash)
     for l in range(shape.n_layers):
         for name, t in gen.make_layer(shape, l, seed, "cuda").items():
             dec.kl_load_weights(name, l, t)
@@ -556,6 +556,22 @@ def run_ours(args, shape, batch, context):
     ms_e2e_logits = max_over_ranks(run_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
     ms_e2e = max_over_ranks(run_greedy_host_loop(dec, fresh_cache(), tok0, context, batch, W, K, stream))
     ms_e2e_tokens = max_over_ranks(run_tokens_per_launch(dec, fresh_cache(), tok0, context, W, K, stream, host=True))
+    # 5. where the model runs in stash mode: the same tokens in the plain mode (a second handle with KL_FLAG_NO_STASH),
+    #    if both copies of the weights fit the device
+    stash_mode = dec.kl_stash_mode()
+    plain = None
+    free_b, _ = torch.cuda.mem_get_info()
+    if stash_mode == 1 and batch == 1 and free_b > dec.weight_bytes + dec.scratch_bytes + cache.numel() * 2 + (4 << 30):
+        dec2, cache2, _ = build_model(shape, batch, context, 2 * (K + W), seed=rank, stash=False)
+        ms_p_token = max_over_ranks(run_token_loop(dec2, cache2, tok0, context, batch, W, K, stream))
+        dec2.kl_set_mode(binding.KL_MODE_LOOPED)
+        cache2, = (gen.make_kv_cache(shape, batch, context, context + 2 * (K + W) + 8, rank, "cuda"),)
+        ms_p_looped = max_over_ranks(run_device_loop(dec2, cache2, tok0, context, batch, W, K, stream))
+        plain = {"one_launch_per_token": {"value": K * batch * world / (ms_p_token * 1e-3), "ms_per_step": ms_p_token / K},
+                 "looped_four_launches": {"value": K * batch * world / (ms_p_looped * 1e-3), "ms_per_step": ms_p_looped / K},
+                 "what": "the same model created with KL_FLAG_NO_STASH: weights consumed from the shared-memory ring"}
+        dec2.close()
+        del dec2, cache2
 
     tokens = K * batch * world
     # headline: the fastest schedule of the same work -- one launch per token (decoder layers, classifier and sampling in
@@ -577,6 +593,7 @@ def run_ours(args, shape, batch, context):
         "config": {"workload": args.workload, "batch": batch, "context": context, "l2": "inputs larger than L2 (weights and KV streamed once per step)"},
         "details": {"mode": "looped, one launch per token (kl_decode_greedy: decoder layers + classifier + sampling)",
                     "storage": "bf16 weights and KV, fp32 activations and accumulation",
+                    "stash_mode": stash_mode,
                     "parallelism": "replicas only" if world > 1 else "single GPU",
                     "batch_schedule": "one sequence after another (weights streamed once per sequence)" if batch > 1 else "n/a",
                     "max_ctx": max_ctx},
@@ -625,6 +642,8 @@ def run_ours(args, shape, batch, context):
                       "launches_per_step": shape.n_layers + 3,
                       "looped_speedup": ms_layer / ms_looped},
     }
+    if plain is not None:
+        line["plain_mode"] = plain
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import kl_oracle as ko
         ko.build()

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) kl_embed_kernel(const Params p) {
 template <class SM>
 __device__ __noinline__ void attention_block(const Params& p, const SM& s, const StepCtx& cx, uint32_t l, uint32_t cta,
                                              uint32_t ctid, uint32_t warp, uint32_t lane, RingCursor& rc, WarpRing& wr) {
-    if (SM::kTmem || p.attn_tc) {   // the stash-mode kernels carry the tensor-core loop only
+    if (!SM::kCudaCoreAttn || p.attn_tc) {   // kernels without the CUDA-core loops are launched only when this one runs
         attention_stage_and_advance<0>(p, s, cx, l, cta, ctid, warp, lane, rc, wr);
     } else switch (p.G) {
         case 1: attention_stage_and_advance<1>(p, s, cx, l, cta, ctid, warp, lane, rc, wr); break;
@@ -270,10 +270,10 @@ __device__ __forceinline__ void run_stage(const Params& p, const SM& s, uint32_t
 // Stages [sbeg, send) of layers [l0, l1) of the decoder.  All five stages of all L layers is the looped kernel; all
 // stages of one layer the per-layer launch; one stage of one layer the per-stage launch (the schedule with a kernel
 // boundary after every operator group).
-template <bool TR, bool MOE, int TM>
+template <bool TR, bool MOE, int TM, bool CC>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_decoder_kernel(const __grid_constant__ Params p, uint32_t l0, uint32_t l1,
                                                                  uint32_t sbeg, uint32_t send) {
-    using SM = SmemT<TR, MOE, TM>;
+    using SM = SmemT<TR, MOE, TM, CC>;
     const SM s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, p.rope_cs)) return;   // an earlier kernel of this step flagged bad input: the step is a no-op
@@ -556,9 +556,9 @@ __device__ __noinline__ bool sample_token(const Params& p, const SM& s, const To
 // K tokens of one sequence per launch (K = 1: one launch per token).  ONE loop over (token, layer) pairs, the
 // classifier being the only stage of a layer L behind the decoder layers and the sampling a call behind that: with a
 // loop over tokens around the loop over layers the compiler holds more in registers through the stage code.
-template <bool TR, bool MOE, int TM>
+template <bool TR, bool MOE, int TM, bool CC>
 __global__ void __launch_bounds__(NTHREADS, 1) kl_token_kernel(const __grid_constant__ Params p, const __grid_constant__ TokenParams t) {
-    using SM = SmemT<TR, MOE, TM>;
+    using SM = SmemT<TR, MOE, TM, CC>;
     const SM s;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, cta = blockIdx.x;
     if (!cta_begin(p, s, tid, t.rope)) return;
@@ -1171,29 +1171,31 @@ kl_status kl_create(const kl_model_desc* desc, void* weight_arena_d, void* scrat
     // maximum, so that handles of different shapes (each launching with its own smem_bytes) can be alive together.
     cudaError_t ce = cudaSuccess;
     {
-        const void* fns[] = {(const void*)kl_decoder_kernel<false, false, 0>, (const void*)kl_decoder_kernel<true, false, 0>,
-                             (const void*)kl_decoder_kernel<false, true, 0>, (const void*)kl_decoder_kernel<false, false, 1>,
-                             (const void*)kl_decoder_kernel<true, false, 1>, (const void*)kl_decoder_kernel<false, false, 2>,
-                             (const void*)kl_decoder_kernel<true, false, 2>, (const void*)kl_classifier_kernel<0>,
-                             (const void*)kl_classifier_kernel<1>, (const void*)kl_classifier_kernel<2>};
+        const void* fns[] = {(const void*)kl_decoder_kernel<false, false, 0, false>, (const void*)kl_decoder_kernel<false, false, 0, true>,
+                             (const void*)kl_decoder_kernel<true, false, 0, false>, (const void*)kl_decoder_kernel<true, false, 0, true>,
+                             (const void*)kl_decoder_kernel<false, true, 0, false>, (const void*)kl_decoder_kernel<false, true, 0, true>,
+                             (const void*)kl_decoder_kernel<false, false, 1, false>, (const void*)kl_decoder_kernel<true, false, 1, false>,
+                             (const void*)kl_decoder_kernel<false, false, 2, false>, (const void*)kl_decoder_kernel<true, false, 2, false>,
+                             (const void*)kl_classifier_kernel<0>, (const void*)kl_classifier_kernel<1>, (const void*)kl_classifier_kernel<2>};
         for (const void* f : fns)
             if (ce == cudaSuccess) ce = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin);
     }
     {
         int tocc = 0;
-        const void* fns[] = {(const void*)kl_token_kernel<false, false, 0>, (const void*)kl_token_kernel<true, false, 0>,
-                             (const void*)kl_token_kernel<false, true, 0>, (const void*)kl_token_kernel<false, false, 1>,
-                             (const void*)kl_token_kernel<true, false, 1>, (const void*)kl_token_kernel<false, false, 2>,
-                             (const void*)kl_token_kernel<true, false, 2>};
+        const void* fns[] = {(const void*)kl_token_kernel<false, false, 0, false>, (const void*)kl_token_kernel<false, false, 0, true>,
+                             (const void*)kl_token_kernel<true, false, 0, false>, (const void*)kl_token_kernel<true, false, 0, true>,
+                             (const void*)kl_token_kernel<false, true, 0, false>, (const void*)kl_token_kernel<false, true, 0, true>,
+                             (const void*)kl_token_kernel<false, false, 1, false>, (const void*)kl_token_kernel<true, false, 1, false>,
+                             (const void*)kl_token_kernel<false, false, 2, false>, (const void*)kl_token_kernel<true, false, 2, false>};
         h->token_ok = 1;
         for (const void* f : fns)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin) != cudaSuccess) h->token_ok = 0;
         if (h->token_ok)
-            h->token_ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false, 0>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
+            h->token_ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&tocc, kl_token_kernel<true, false, 0, true>, NTHREADS, h->smem_bytes) == cudaSuccess && tocc >= 1;
         (void)cudaGetLastError();
     }
     int occ = 0;
-    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false, 0>, NTHREADS, h->smem_bytes);
+    if (ce == cudaSuccess) ce = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kl_decoder_kernel<true, false, 0, true>, NTHREADS, h->smem_bytes);
     if (ce != cudaSuccess || occ < 1) {
         fprintf(stderr, "kl_create: the persistent kernel cannot be resident (%s; %zu bytes of shared memory, %d threads, "
                         "occupancy %d)\n", cudaGetErrorString(ce), h->smem_bytes, NTHREADS, occ);
@@ -1621,21 +1623,23 @@ static kl_status batched_step(kl_handle* h, const int32_t* tokens_d, const int32
 }
 
 // The instantiation a launch takes: mixture of experts, stash mode (1: chunks of 2048 / 4096 columns only, 2: all
-// widths), and the debug hooks (trace stamps, jitter) only while one of them is set.
-static const void* token_fn(const kl_handle* h) {
-    const Params& p = h->prm;
-    const bool dbg = p.jitter_seed != 0u || p.trace != nullptr;
-    if (p.n_experts) return (const void*)kl_token_kernel<false, true, 0>;
-    if (h->stash == 1) return dbg ? (const void*)kl_token_kernel<true, false, 1> : (const void*)kl_token_kernel<false, false, 1>;
-    if (h->stash == 2) return dbg ? (const void*)kl_token_kernel<true, false, 2> : (const void*)kl_token_kernel<false, false, 2>;
-    return dbg ? (const void*)kl_token_kernel<true, false, 0> : (const void*)kl_token_kernel<false, false, 0>;
+// widths), the debug hooks (trace stamps, jitter) only while one of them is set, the CUDA-core attention loops only
+// when the launch runs them.
+static const void* token_fn(const kl_handle* h, const Params& p) {
+    const bool dbg = p.jitter_seed != 0u || p.trace != nullptr, cc = !p.attn_tc;
+    if (p.n_experts) return cc ? (const void*)kl_token_kernel<false, true, 0, true> : (const void*)kl_token_kernel<false, true, 0, false>;
+    if (h->stash == 1) return dbg ? (const void*)kl_token_kernel<true, false, 1, false> : (const void*)kl_token_kernel<false, false, 1, false>;
+    if (h->stash == 2) return dbg ? (const void*)kl_token_kernel<true, false, 2, false> : (const void*)kl_token_kernel<false, false, 2, false>;
+    if (cc) return dbg ? (const void*)kl_token_kernel<true, false, 0, true> : (const void*)kl_token_kernel<false, false, 0, true>;
+    return dbg ? (const void*)kl_token_kernel<true, false, 0, false> : (const void*)kl_token_kernel<false, false, 0, false>;
 }
 static const void* decoder_fn(const kl_handle* h, const Params& p) {
-    const bool dbg = p.trace != nullptr || p.jitter_seed != 0u;
-    if (p.n_experts) return (const void*)kl_decoder_kernel<false, true, 0>;
-    if (h->stash == 1) return dbg ? (const void*)kl_decoder_kernel<true, false, 1> : (const void*)kl_decoder_kernel<false, false, 1>;
-    if (h->stash == 2) return dbg ? (const void*)kl_decoder_kernel<true, false, 2> : (const void*)kl_decoder_kernel<false, false, 2>;
-    return dbg ? (const void*)kl_decoder_kernel<true, false, 0> : (const void*)kl_decoder_kernel<false, false, 0>;
+    const bool dbg = p.trace != nullptr || p.jitter_seed != 0u, cc = !p.attn_tc;
+    if (p.n_experts) return cc ? (const void*)kl_decoder_kernel<false, true, 0, true> : (const void*)kl_decoder_kernel<false, true, 0, false>;
+    if (h->stash == 1) return dbg ? (const void*)kl_decoder_kernel<true, false, 1, false> : (const void*)kl_decoder_kernel<false, false, 1, false>;
+    if (h->stash == 2) return dbg ? (const void*)kl_decoder_kernel<true, false, 2, false> : (const void*)kl_decoder_kernel<false, false, 2, false>;
+    if (cc) return dbg ? (const void*)kl_decoder_kernel<true, false, 0, true> : (const void*)kl_decoder_kernel<false, false, 0, true>;
+    return dbg ? (const void*)kl_decoder_kernel<true, false, 0, false> : (const void*)kl_decoder_kernel<false, false, 0, false>;
 }
 static const void* classifier_fn(const kl_handle* h) {
     return h->stash == 1 ? (const void*)kl_classifier_kernel<1> : h->stash == 2 ? (const void*)kl_classifier_kernel<2>
@@ -1815,7 +1819,7 @@ kl_status kl_decode_greedy(kl_handle* h, int32_t* tokens_d, int32_t* positions_d
     if (prc != KL_OK) return prc;
     TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, nullptr, 1u, p.rope_cs};
     void* args[] = {&p, &t};
-    const kl_status rc = launch_persistent(h, token_fn(h), args, st);
+    const kl_status rc = launch_persistent(h, token_fn(h, p), args, st);
     if (rc != KL_OK) return rc;
     h->last_batch = 1;
     h->hidden_is_copy = 1;
@@ -1849,7 +1853,7 @@ kl_status kl_decode_greedy_tokens(kl_handle* h, int32_t* tokens_d, int32_t* posi
         ++h->launches;
         TokenParams t = {tokens_d, positions_d, h->tok_val, h->tok_idx, h->tok_ticket, h->hidden_all, out_tokens_d + done, K, h->plan_rope};
         void* args[] = {&p, &t};
-        const kl_status rc = launch_persistent(h, token_fn(h), args, st);
+        const kl_status rc = launch_persistent(h, token_fn(h, p), args, st);
         if (rc != KL_OK) return rc;
         h->last_batch = 1;
         h->hidden_is_copy = 1;

@@ -355,10 +355,14 @@ struct MoeSel {
     uint32_t e[MAX_TOP_K];          // the chosen experts, in descending order of their logits
     float w[MAX_TOP_K];             // and their gate weights
 };
-template <bool TR, bool MOE = false, int TM = 0>
+template <bool TR, bool MOE = false, int TM = 0, bool CC = true>
 struct SmemT {
     static constexpr bool kTrace = TR;
     static constexpr bool kMoe = MOE;
+    // CC: the CUDA-core attention loops are compiled in.  Launches that run the tensor-core loop take kernels without
+    // them: code a launch never runs costs time by being there (3.5 % of a token on the 8B shape).  The stash-mode
+    // kernels never carry them.
+    static constexpr bool kCudaCoreAttn = CC && TM == 0;
     static constexpr bool kTmem = TM != 0;       // stash mode: weights go ring -> TMEM -> registers (see the stash section)
     // TM == 1: the stage exists for chunks of 2048 and 4096 columns only; TM == 2: for 1024 and 3072 as well.  Two kernels,
     // because the code the common shapes never run costs them time by lying between the code they do run
