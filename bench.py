@@ -793,7 +793,7 @@ def run_ours_batched(args, shape, batch, context):
 # dram__bytes_read.sum + dram__bytes_write.sum of one looped launch over 4 layers of the 8B shape at batch 1,
 # context 4096 (ncu capture summarised under profiles/), per layer.  Every layer streams its own weights and KV once,
 # so a full launch is this times the layer count.
-NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.813368e9 + 18.063104e6) / 4
+NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.814647e9 + 20.904704e6) / 4
 
 
 # the same for the ten launches of one layer of the batched path at batch 32, context 4096
@@ -802,7 +802,7 @@ NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1001.8e6
 
 # dram bytes of the classifier and sampling stages of kl_token_kernel at vocabulary 128256, hidden 4096: a 4-layer
 # kl_token_kernel launch minus a 4-layer kl_decoder_kernel launch (both captures summarised under profiles/)
-NCU_DRAM_BYTES_CLASSIFIER_STAGE_V128256_H4096 = (2.864128e9 + 21.771008e6) - (1.813368e9 + 18.063104e6)
+NCU_DRAM_BYTES_CLASSIFIER_STAGE_V128256_H4096 = (2.864009e9 + 22.105344e6) - (1.814647e9 + 20.904704e6)
 
 
 def ncu_traffic(shape, batch, context):
