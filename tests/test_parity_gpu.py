@@ -374,11 +374,17 @@ def test_repeated_steps_are_bit_identical():
     dec.close()
 
 
-def test_bounded_wait_reports_timeout_and_recovers():
+# the bounded waits in both modes of the batch-1 kernels: the tiny shape runs in the plain mode, the other in stash mode
+WAIT_SHAPES = {"plain": gen.TINY, "stash": gen.ModelShape(2, 2048, 16, 4, 128, 4096, 1544, 1e-5, 500000.0)}
+
+
+@pytest.mark.parametrize("mode_name", sorted(WAIT_SHAPES))
+def test_bounded_wait_reports_timeout_and_recovers(mode_name):
     """A stage end that is never signalled makes the waits on it run out: the step reports KL_ERR_SYNC_TIMEOUT
     (no hang, no trap) and the next step on the same handle is correct again."""
-    shape = gen.TINY
+    shape = WAIT_SHAPES[mode_name]
     dec = helpers.make_decoder(shape, 1, 200, 0)
+    assert dec.kl_stash_mode() == (1 if mode_name == "stash" else 0)
     cache = gen.make_kv_cache(shape, 1, 128, 200, 0, "cuda")
     tok = gen.make_tokens(shape, 1, 0).cuda()
     pos = torch.tensor([128], dtype=torch.int32, device="cuda")
@@ -877,12 +883,14 @@ def test_two_handles_of_different_shapes_step_alternately():
     b.close()
 
 
-def test_bounded_wait_on_the_greedy_chain_leaves_token_and_position_alone():
+@pytest.mark.parametrize("mode_name", sorted(WAIT_SHAPES))
+def test_bounded_wait_on_the_greedy_chain_leaves_token_and_position_alone(mode_name):
     """A wait that runs out inside the one-launch-per-token kernel: the call reports KL_ERR_SYNC_TIMEOUT, does not touch
     the token or the position (the step's logits and cache row are undefined), and the next call starts a new chain that
     gives the bits of an undisturbed run."""
-    shape = gen.TINY
+    shape = WAIT_SHAPES[mode_name]
     dec = helpers.make_decoder(shape, 1, 200, 0)
+    assert dec.kl_stash_mode() == (1 if mode_name == "stash" else 0)
     cache0 = gen.make_kv_cache(shape, 1, 128, 200, 0, "cuda")
     tok0 = gen.make_tokens(shape, 1, 0).cuda()
     logits_ok, logits = torch.empty(1, shape.vocab, device="cuda"), torch.empty(1, shape.vocab, device="cuda")
