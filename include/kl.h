@@ -74,7 +74,8 @@ enum {
  * 2048, an input vector of ffn floats next to an eight-slot ring in shared memory -- run in stash mode: every weight
  * chunk moves on from its ring slot into tensor memory and is multiplied from there, which more than doubles what an SM
  * holds ahead of its consumers (the cross-layer weight prefetch of Section 2, deeper).  Both modes compute the same
- * function; their sums are taken in different orders.  No counterpart in the paper. */
+ * function; their sums are taken in different orders.  The environment variable KL_STASH=0 acts as this flag for every
+ * handle the process creates (for measurements that must not touch the caller's code).  No counterpart in the paper. */
 #define KL_FLAG_NO_STASH 2u
 
 /* Shapes the kernels cover (anything else: KL_ERR_UNSUPPORTED_SHAPE): head_dim 32, 64, 128 or 256; hidden and ffn
