@@ -59,7 +59,7 @@ def test_workspace_sizes_and_shape_validation(lib):
     qr = s.q_dim + 2 * s.kv_dim
     assert s.n_layers * qr * 2 <= wb2 - wb <= s.n_layers * (qr * 2 + 256)
     bad = binding.make_desc(s, 1, 64)
-    bad.flags = 2
+    bad.flags = 4   # not a flag of the interface (1: biases, 2: no stash mode)
     assert lib.kl_workspace_bytes(C.byref(bad), C.byref(w), C.byref(sc)) == binding.KL_ERR_UNSUPPORTED_SHAPE
     # a batched handle (max_batch > 1) carries the operand, partial-result and attention buffers of the batched path
     _, sb32 = binding.kl_workspace_bytes(binding.make_desc(s, 32, 4096 + 256))
