@@ -292,7 +292,8 @@ kl_status kl_profile_read(kl_handle* h, uint32_t* n, float* decoder_ms, float* c
  *   12 counter of the gate/up stage passed                 13 down-projection rows done
  * The trailing 8192 x 4 block logs the first 8192 ring chunks of CTA 0: [0] issue by the producer, [2] chunk seen
  * landed by its consumer warp, [1] dot product done, [3] results emitted.  Stamps of the latest step overwrite
- * earlier ones. */
+ * earlier ones.  kl_decode_step and kl_decode_greedy (batch 1) both take the stage stamps; the chunk log is written by
+ * kl_decode_step in the plain mode only. */
 kl_status kl_set_trace(kl_handle* h, uint64_t* trace_d, uint32_t* n_ctas, uint32_t* n_layers, uint32_t* n_stamps);
 
 /* Attention inner loop.  on = 1 (default when head_dim is 64 or 128): tensor-core loop (mma.sync on 128-byte

@@ -1,8 +1,9 @@
 """Stage timeline of the looped decoder kernel, read through kl_set_trace.
 
-    python -m paper_2410_23668_b200.trace [--workload llama31_8b_b1_ctx4096] [--warm 5]
+    python -m paper_2410_23668_b200.trace [--workload llama31_8b_b1_ctx4096] [--warm 5] [--greedy]
 
-Runs a few warm-up steps, then one traced decode step, and prints per stage of a layer the median / maximum /
+Runs a few warm-up steps, then one traced decode step (kl_decode_step: the decoder kernel; with --greedy
+kl_decode_greedy: the one-launch-per-token kernel, whose decoder layers take the same stamps), and prints per stage of a layer the median / maximum /
 minimum over the CTAs of the time between consecutive stamps (microseconds, averaged over layers 1..L-1), the
 sub-steps of the attention block for the CTAs that own a split-K unit, and the per-chunk statistics of CTA 0.
 Stamp meanings are listed next to kl_set_trace in include/kl.h.  Tracing costs a few percent: use bench.py for
