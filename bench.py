@@ -561,7 +561,9 @@ def run_ours(args, shape, batch, context):
     stash_mode = dec.kl_stash_mode()
     plain = None
     free_b, _ = torch.cuda.mem_get_info()
-    if stash_mode == 1 and batch == 1 and free_b > dec.weight_bytes + dec.scratch_bytes + cache.numel() * 2 + (4 << 30):
+    fits = free_b > dec.weight_bytes + dec.scratch_bytes + cache.numel() * 2 + (4 << 30)
+    fits = max_over_ranks(0.0 if fits else 1.0) == 0.0   # the same decision on every replica: the passes below synchronise them
+    if stash_mode == 1 and batch == 1 and fits:
         dec2, cache2, _ = build_model(shape, batch, context, 2 * (K + W), seed=rank, stash=False)
         ms_p_token = max_over_ranks(run_token_loop(dec2, cache2, tok0, context, batch, W, K, stream))
         dec2.kl_set_mode(binding.KL_MODE_LOOPED)
