@@ -58,6 +58,11 @@ def test_odd_shapes(name):
 STASH_SHAPES = {
     "rows_of_2048": gen.ModelShape(2, 2048, 16, 4, 128, 4096, 1544, 1e-5, 500000.0),
     "down_in_two_pieces": gen.ModelShape(2, 4096, 32, 8, 128, 8192, 1544, 1e-5, 500000.0),
+    # one layer, a classifier of 50 units for 148 CTAs (most CTAs stream nothing in that stage), rows of 3072 columns
+    # (three granules per row: two granules of every chunk stay unused), G = 3
+    "few_units_rows_of_3072": gen.ModelShape(1, 3072, 24, 8, 128, 1024, 200, 1e-5, 500000.0),
+    # chunks of 1024 columns, eight rows each (FFN 5120 = 5 x 1024)
+    "pieces_of_1024": gen.ModelShape(2, 2048, 16, 4, 128, 5120, 1544, 1e-5, 500000.0),
 }
 
 
