@@ -1358,6 +1358,25 @@ kl_status kl_load_expert_weights(kl_handle* h, int tensor, int layer, int expert
 
 // The KV cache as a 2-D bf16 tensor [n_layers*2*batch*n_kv_heads*max_ctx rows, head_dim columns]; boxes of
 // [positions per chunk] x [64 columns] with the 128-byte swizzle.  Encoded per call because the cache is the caller's.
+// The cache as the 4-D tensor of the batch-1 kernels' ring copies (see Params::kv_map4): dimension 0 = 64 columns,
+// 1 = rows (all slabs one after the other), 2 = 64-column halves of a row, 3 = K | V, a slab of `batch` sequences apart.
+static kl_status encode_kv_map4(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch) {
+    if (!h->encode_tiled) return KL_ERR_CUDA;
+    if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
+    const kl_model_desc& d = h->desc;
+    const cuuint64_t rows = (cuuint64_t)d.n_layers * 2 * batch * d.n_kv_heads * d.max_ctx;
+    if (rows > 0x7fffffffull) return KL_ERR_UNSUPPORTED_SHAPE;  // box coordinates are 32-bit signed
+    const cuuint64_t vdelta = (cuuint64_t)batch * d.n_kv_heads * d.max_ctx;   // rows between a K slab and its V slab
+    const cuuint64_t gdim[4] = {64, rows, d.head_dim / 64, 2};
+    const cuuint64_t gstride[3] = {(cuuint64_t)d.head_dim * 2, 128, vdelta * d.head_dim * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)(SLOT_BYTES / (4 * d.head_dim)), d.head_dim / 64, 2};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUresult r = ((encode_tiled_fn)h->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, kv_cache_d, gdim, gstride, box,
+                                                         estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                         CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? KL_OK : KL_ERR_CUDA;
+}
+
 static kl_status encode_kv_map(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch, uint32_t slot_bytes = SLOT_BYTES) {
     if (!h->encode_tiled) return KL_ERR_CUDA;
     if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
@@ -1667,7 +1686,8 @@ kl_status kl_decode_step(kl_handle* h, const int32_t* tokens_d, const int32_t* p
     h->pending_skip_stage = -1;
     p.attn_tc = 0;
     if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
-        const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, batch);
+        kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, batch);
+        if (trc == KL_OK) trc = encode_kv_map4(h, &p.kv_map4, kv_cache_d, batch);
         if (trc != KL_OK) return trc;
         p.attn_tc = 1;
     }
@@ -1787,7 +1807,8 @@ static kl_status token_chain_params(kl_handle* h, Params* out, int32_t* tokens_d
     p.chunk_trace = nullptr;
     p.attn_tc = 0;
     if (h->use_tc_attention && (p.hd == 64 || p.hd == 128)) {
-        const kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, 1);
+        kl_status trc = encode_kv_map(h, &p.kv_map, kv_cache_d, 1);
+        if (trc == KL_OK) trc = encode_kv_map4(h, &p.kv_map4, kv_cache_d, 1);
         if (trc != KL_OK) return trc;
         p.attn_tc = 1;
     }

@@ -127,14 +127,6 @@ __device__ __forceinline__ void tma_tensor_3d_g2s(uint32_t dst, const void* tmap
         ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(pol)
         : "memory");
 }
-__device__ __forceinline__ void tma_tensor_4d_g2s(uint32_t dst, const void* tmap, int32_t c0, int32_t c1, int32_t c2, int32_t c3,
-                                                  uint32_t bar, uint64_t pol) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
-        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(pol)
-        : "memory");
-}
 __device__ __forceinline__ void tma_tensor_5d_g2s(uint32_t dst, const void* tmap, int32_t c0, int32_t c1, int32_t c2, int32_t c3,
                                                   int32_t c4, uint32_t bar, uint64_t pol) {
     asm volatile(

@@ -115,6 +115,12 @@ struct Params {
     int32_t* status;
     unsigned long long* trace;  // optional [P][L][TRACE_STAMPS] globaltimer stamps of consumer thread 0, or null
     unsigned long long* chunk_trace;  // optional [CHUNK_TRACE_ROWS][4] per-chunk stamps of CTA 0 (issue, wait, full, done)
+    // the KV cache once more, as a 4-D tensor [64 columns][rows][head_dim / 64 column halves][K | V of the same (layer, sequence, head)]:
+    // ONE copy brings the K and the V rows of a chunk, every 64-column half as a box of its own.  The producer thread
+    // pays per instruction, and a unit at a long context is hundreds of chunks: units of more chunks than the ring has
+    // slots take this form (context 65536: 236 against 221 tok/s), shorter ones -- whose chunks are all in flight at
+    // once and whose last arrival is what the attention block waits for -- the four separate boxes, which land sooner.
+    CUtensorMap kv_map4;
 };
 constexpr uint32_t CHUNK_TRACE_ROWS = 8192;
 
@@ -567,6 +573,14 @@ __device__ __forceinline__ void tma_tensor_2d_g2s(uint32_t dst, const void* tmap
         ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar), "l"(pol)
         : "memory");
 }
+__device__ __forceinline__ void tma_tensor_4d_g2s(uint32_t dst, const void* tmap, int32_t x, int32_t y, int32_t z, int32_t w,
+                                                  uint32_t bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar), "l"(pol)
+        : "memory");
+}
 
 // Window of cache rows a ring chunk of the tensor-core path holds.  Chunk i of a unit covers positions
 // [c0 + i*pb, min(.. + pb, cend)); the box always has pb rows, so a short last chunk is slid back to end at cend
@@ -737,10 +751,11 @@ __device__ __forceinline__ void prod_issue(const Params& p, const SM& s, RingPro
     prod_advance<SM>(p, r);
 }
 // Same for a chunk of K/V rows as swizzled boxes of the cache tensor: [pb rows] x [64 columns] per box, K boxes in
-// the first half of the slot, V boxes in the second; a box is always written whole (rows outside the chunk's own
-// positions are ignored by the consumer).
+// the first half of the slot, V boxes in the second, written by one copy each or all of them by one copy (the boxes
+// are the outer dimensions of the 4-D tensor map); a box is always written whole (rows outside the chunk's own
+// positions are ignored by the consumer).  yk, yv: cache rows of the first row of the K and of the V boxes.
 template <class SM>
-__device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, RingProd& r, int32_t yk, int32_t yv) {
+__device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, RingProd& r, int32_t yk, int32_t yv, bool one_copy) {
     if (r.aborted) return;
     uint32_t slot, use;
     prod_slot<SM>(p, r, slot, use);
@@ -752,10 +767,14 @@ __device__ __forceinline__ void prod_issue_boxes(const Params& p, const SM& s, R
     const uint32_t dst = smem_u32(s.ring()) + slot * SLOT_BYTES;
     chunk_stamp(p, s, blockIdx.x, r.n, 0);
     mbar_arrive_expect_tx(bar, (uint32_t)SLOT_BYTES);
-    const uint32_t box_bytes = SLOT_BYTES / 2 / (p.hd / 64u);
-    for (uint32_t bx = 0; bx < p.hd / 64u; ++bx) {
-        tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yk, bar, r.pol);
-        tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yv, bar, r.pol);
+    if (one_copy) {
+        tma_tensor_4d_g2s(dst, &p.kv_map4, 0, yk, 0, 0, bar, r.pol);
+    } else {
+        const uint32_t box_bytes = SLOT_BYTES / 2 / (p.hd / 64u);
+        for (uint32_t bx = 0; bx < p.hd / 64u; ++bx) {
+            tma_tensor_2d_g2s(dst + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yk, bar, r.pol);
+            tma_tensor_2d_g2s(dst + SLOT_BYTES / 2 + bx * box_bytes, &p.kv_map, (int32_t)(bx * 64u), yv, bar, r.pol);
+        }
     }
     prod_advance<SM>(p, r);
 }
@@ -816,7 +835,7 @@ __device__ __forceinline__ void produce_attention(const Params& p, const SM& s, 
         for (uint32_t i = 0; i < u.nring; ++i) {
             const AttnWindow w = attn_window(u.c0, u.cend, pb, i);
             if constexpr (SM::kTmem) r.pi = i & 1u;
-            prod_issue_boxes(p, s, r, (int32_t)(row0 + w.w0), (int32_t)(row0 + w.w0 + vdelta));
+            prod_issue_boxes(p, s, r, (int32_t)(row0 + w.w0), (int32_t)(row0 + w.w0 + vdelta), u.nring > p.nslots);
         }
     } else {
         const uint32_t row_bytes = p.hd * 2u;
