@@ -1360,7 +1360,7 @@ kl_status kl_load_expert_weights(kl_handle* h, int tensor, int layer, int expert
 // [positions per chunk] x [64 columns] with the 128-byte swizzle.  Encoded per call because the cache is the caller's.
 // The cache as the 4-D tensor of the batch-1 kernels' ring copies (see Params::kv_map4): dimension 0 = 64 columns,
 // 1 = rows (all slabs one after the other), 2 = 64-column halves of a row, 3 = K | V, a slab of `batch` sequences apart.
-static kl_status encode_kv_map4(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch) {
+static kl_status encode_kv_map4(kl_handle* h, CUtensorMap* map, void* kv_cache_d, uint32_t batch, uint32_t slot_bytes = SLOT_BYTES) {
     if (!h->encode_tiled) return KL_ERR_CUDA;
     if ((uintptr_t)kv_cache_d & 15u) return KL_ERR_INVALID_ARG;
     const kl_model_desc& d = h->desc;
@@ -1369,7 +1369,7 @@ static kl_status encode_kv_map4(kl_handle* h, CUtensorMap* map, void* kv_cache_d
     const cuuint64_t vdelta = (cuuint64_t)batch * d.n_kv_heads * d.max_ctx;   // rows between a K slab and its V slab
     const cuuint64_t gdim[4] = {64, rows, d.head_dim / 64, 2};
     const cuuint64_t gstride[3] = {(cuuint64_t)d.head_dim * 2, 128, vdelta * d.head_dim * 2};
-    const cuuint32_t box[4] = {64, (cuuint32_t)(SLOT_BYTES / (4 * d.head_dim)), d.head_dim / 64, 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)(slot_bytes / (4 * d.head_dim)), d.head_dim / 64, 2};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUresult r = ((encode_tiled_fn)h->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, kv_cache_d, gdim, gstride, box,
                                                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1501,7 +1501,7 @@ static kl_status decode_step_batched(kl_handle* h, const int32_t* tokens_d, cons
                                      float* logits_d, uint32_t batch, cudaStream_t st) {
     const Params& p = h->prm;
     BAttnParams a;
-    const kl_status trc = encode_kv_map(h, &a.kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
+    const kl_status trc = encode_kv_map4(h, &a.kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
     if (trc != KL_OK) return trc;
     a.kv = reinterpret_cast<__nv_bfloat16*>(kv_cache_d);
     a.positions = positions_d;
@@ -1565,7 +1565,7 @@ static kl_status decode_step_batched_looped(kl_handle* h, const int32_t* tokens_
     BLoopParams* b = new (std::nothrow) BLoopParams();   // 2.3 KB of kernel parameters (fourteen tensor maps)
     if (!b) return KL_ERR_INVALID_ARG;
     struct Free { BLoopParams* p; ~Free() { delete p; } } guard{b};
-    const kl_status trc = encode_kv_map(h, &b->kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
+    const kl_status trc = encode_kv_map4(h, &b->kv_map, kv_cache_d, batch, BA_SLOT_BYTES);
     if (trc != KL_OK) return trc;
     static const int plan_of[5] = {PL_QKV, PL_O, PL_GU, PL_D, PL_LM};
     static const uint32_t xmap_of[5] = {0, 1, 0, 2, 0};

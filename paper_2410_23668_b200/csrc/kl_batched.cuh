@@ -649,7 +649,7 @@ struct BAttnView {
     uint64_t wait_ns;
 };
 struct BAttnParams : BAttnView {
-    CUtensorMap kv_map;       // the whole KV cache as [rows, head_dim] (same map as the batch-1 kernel)
+    CUtensorMap kv_map;       // the whole KV cache as a 4-D tensor: 64 columns, rows, column halves, K | V (one copy per chunk)
 };
 
 // RoPE and cache append; grid (batch, n_q_heads + 2 * n_kv_heads), one head of one sequence per block of 128
@@ -779,11 +779,8 @@ __device__ __forceinline__ void b_attn_stream(const BAttnView& p, const CUtensor
         const uint32_t bar = smem_u32(&full[slot]);
         const uint32_t dst = ring + slot * BA_SLOT_BYTES;
         mbar_arrive_expect_tx(bar, (uint32_t)BA_SLOT_BYTES);
-#pragma unroll
-        for (uint32_t bx = 0; bx < HD / 64u; ++bx) {
-            tma_tensor_2d_g2s(dst + bx * box_bytes, kv_map, (int32_t)(bx * 64u), (int32_t)row0, bar, pol);
-            tma_tensor_2d_g2s(dst + BA_SLOT_BYTES / 2 + bx * box_bytes, kv_map, (int32_t)(bx * 64u), (int32_t)(row0 + vdelta), bar, pol);
-        }
+        // one copy: the K and the V rows of the chunk, every 64-column half a box of its own (the outer dimensions of the map)
+        tma_tensor_4d_g2s(dst, kv_map, 0, (int32_t)row0, 0, 0, bar, pol);
     };
 
     // the first chunks of the range go out before anything else

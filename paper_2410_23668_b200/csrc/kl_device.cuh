@@ -875,15 +875,15 @@ __device__ __forceinline__ void produce_drain(const Params& p, const SM& s, cons
                     if (globaltimer_ns() - t0 > p.wait_ns) return;
                 }
             }
-        return;
-    }
-    for (uint32_t cc = 0; cc < p.nslots; ++cc) {
-        for (uint32_t kk = 0; kk < p.nsw; ++kk) {
-            const uint32_t cnt = r.use + ((kk < r.k || (kk == r.k && cc < r.c)) ? 1u : 0u);  // uses of this slot so far
-            if (cnt == 0) continue;
-            const uint32_t bar = smem_u32(&s.full()[cc * p.nsw + kk]);
-            while (!mbar_try_wait(bar, (cnt - 1u) & 1u)) {
-                if (globaltimer_ns() - t0 > p.wait_ns) return;
+    } else {
+        for (uint32_t cc = 0; cc < p.nslots; ++cc) {
+            for (uint32_t kk = 0; kk < p.nsw; ++kk) {
+                const uint32_t cnt = r.use + ((kk < r.k || (kk == r.k && cc < r.c)) ? 1u : 0u);  // uses of this slot so far
+                if (cnt == 0) continue;
+                const uint32_t bar = smem_u32(&s.full()[cc * p.nsw + kk]);
+                while (!mbar_try_wait(bar, (cnt - 1u) & 1u)) {
+                    if (globaltimer_ns() - t0 > p.wait_ns) return;
+                }
             }
         }
     }
