@@ -805,7 +805,7 @@ NCU_DRAM_BYTES_PER_LAYER_8B_B1_CTX4096 = (1.814647e9 + 20.904704e6) / 4
 
 
 # the same for the ten launches of one layer of the batched path at batch 32, context 4096
-NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1001.8e6
+NCU_DRAM_BYTES_PER_LAYER_8B_B32_CTX4096 = 1000.9e6
 
 
 # dram bytes of the classifier and sampling stages of kl_token_kernel at vocabulary 128256, hidden 4096: a 4-layer
