@@ -607,7 +607,7 @@ def test_one_launch_per_token_edge_cases():
     dec.close()
 
 
-@pytest.mark.parametrize("name", ["tiny", "odd_rows_hd128", "llama31_8b_4layers", "llama32_3b_2layers_bias"])
+@pytest.mark.parametrize("name", ["tiny", "odd_rows_hd128", "llama31_8b_4layers", "llama32_3b_2layers_bias", "stash_one_small_layer"])
 def test_tokens_per_launch_match_the_chain_of_single_launches(name):
     """kl_decode_greedy_tokens at batch 1 (the loop over layers extended to a loop over tokens: K tokens in one launch)
     gives the bits of K chained one-token launches: picked tokens, final token / position, logits and hidden state of
@@ -616,7 +616,9 @@ def test_tokens_per_launch_match_the_chain_of_single_launches(name):
     import dataclasses
     shape, ctx, K = {"tiny": (gen.TINY, 128, 9), "odd_rows_hd128": (SHAPES["odd_rows_hd128"], 150, 5),
                      "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 1024, 6),
-                     "llama32_3b_2layers_bias": (dataclasses.replace(LLAMA32_3B_2L, qkv_bias=True), 0, 7)}[name]
+                     "llama32_3b_2layers_bias": (dataclasses.replace(LLAMA32_3B_2L, qkv_bias=True), 0, 7),
+                     # stash mode with a whole token's weights on chip at once: producer and stash threads run a token ahead
+                     "stash_one_small_layer": (STASH_SHAPES["few_units_rows_of_3072"], 40, 12)}[name]
     total = 2 * K + 1
     dec = helpers.make_decoder(shape, 1, ctx + total + 8, 0)
     cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + total + 8, 0, "cuda")
