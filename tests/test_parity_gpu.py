@@ -963,7 +963,7 @@ def test_step_numbers_wrap_without_a_stale_tag():
     dec.close()
 
 
-@pytest.mark.parametrize("name,steps", [("tiny", 1500), ("llama31_8b_4layers", 150)])
+@pytest.mark.parametrize("name,steps", [("tiny", 1500), ("llama31_8b_4layers", 150), ("stash_one_small_layer", 800)])
 def test_sync_protocol_under_seeded_jitter(name, steps):
     """Stress of the exchanges that replace kernel boundaries (tagged words, the gate/up counter, the token boundary
     inside a launch): with kl_debug_set_jitter every CTA sleeps a seeded pseudo-random time of up to 20 us whenever it
@@ -971,7 +971,9 @@ def test_sync_protocol_under_seeded_jitter(name, steps):
     looped kernel, on the one-launch-per-token chain and as multi-token launches must pick, token for token, what the
     undisturbed per-layer schedule picks, and leave the same cache; no bounded wait may run out."""
     import dataclasses
-    shape, ctx = {"tiny": (gen.TINY, 40), "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 512)}[name]
+    shape, ctx = {"tiny": (gen.TINY, 40), "llama31_8b_4layers": (dataclasses.replace(gen.LLAMA31_8B, n_layers=4), 512),
+                  # stash mode, a whole token's weights on chip at once: the stash threads run a token ahead of the consumers
+                  "stash_one_small_layer": (STASH_SHAPES["few_units_rows_of_3072"], 40)}[name]
     dec = helpers.make_decoder(shape, 1, ctx + steps + 8, 0)
     cache0 = gen.make_kv_cache(shape, 1, ctx, ctx + steps + 8, 0, "cuda")
     tok0 = gen.make_tokens(shape, 1, 0).cuda()
